@@ -1,0 +1,233 @@
+/*
+ * preserve.h — C ABI of the B200 (sm_100a) decode-step library.
+ *
+ * One handle = one tensor-parallel shard of one decoder layer.  A decode step
+ * consumes the previous block's partial sums, runs the layer's memory-bound
+ * kernels (skinny GEMMs over the shard's QKV / O / gate-up / down weights and
+ * grouped-query decode attention over the KV-cache) and emits this shard's
+ * partial sums.  While each "communication window" runs, a side stream
+ * prefetches the weights and KV-cache entries of the following operators into
+ * L2, up to a byte budget.
+ *
+ * Paper passages behind the entry points:
+ *   - prefetching read-only weights and KV-cache into L2 in a stream parallel
+ *     to the collective: Section 3, "Execution with the proposed method";
+ *   - which operators get a prefetch and the running budget: Algorithm 1
+ *     ("Prefetch Operator Insertion") and Section 3, "L2 capacity requirements";
+ *   - prefetch stream parallel to the main stream, ordered by events:
+ *     Section 3, "PRESERVE" (runtime paragraph);
+ *   - the layer's blocks and the tensor-parallel split (heads; MLP
+ *     intermediate dimension; one allreduce per block): Section 2.
+ * On one GPU the communication window is a local stand-in that computes what
+ * the allreduce plus its epilogue would deliver: the sum of P partial-sum
+ * buffers already in device memory, the residual add and RMSNorm.
+ *
+ * General rules
+ *   - All tensors are bf16 unless stated; "device" / "host" says where a
+ *     pointer must live.  Device pointers must be 16-byte aligned.
+ *   - The caller owns every pointer it passes.  Weights are borrowed only for
+ *     the duration of preserve_layer_init (the library keeps its own packed
+ *     copy).  Buffers named in a step must stay valid until the work queued on
+ *     the stream has finished.
+ *   - Every call returns PRESERVE_OK (0) or a negative PRESERVE_E* code; no
+ *     exception, abort or print crosses the boundary.  preserve_decode_* are
+ *     asynchronous on the given stream; a device-side failure (a bounded wait
+ *     that gave up) is reported by preserve_last_status.
+ *   - Results are a pure function of the inputs: they do not depend, bit for
+ *     bit, on the prefetch budget or mode.
+ *   - A handle is not thread-safe; distinct handles are independent.
+ *   - The library needs a device of compute capability 10.x and fails with
+ *     PRESERVE_EARCH elsewhere; it has no CPU fallback.
+ */
+#ifndef PRESERVE_H
+#define PRESERVE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* The library is built with hidden visibility; only these entry points are exported. */
+#if defined(__GNUC__)
+#define PRESERVE_API __attribute__((visibility("default")))
+#else
+#define PRESERVE_API
+#endif
+
+#define PRESERVE_OK        0
+#define PRESERVE_EINVAL   (-1)  /* null pointer, bad enum, bad count                */
+#define PRESERVE_EALIGN   (-2)  /* a device pointer is not 16-byte aligned          */
+#define PRESERVE_ESHAPE   (-3)  /* unsupported sizes (see preserve_layer_config_t)  */
+#define PRESERVE_ENOMEM   (-4)  /* device or host allocation failed                 */
+#define PRESERVE_ECUDA    (-5)  /* a CUDA call failed; see preserve_last_cuda_error */
+#define PRESERVE_EARCH    (-6)  /* no sm_100 device / driver entry point missing    */
+#define PRESERVE_ETIMEOUT (-7)  /* a bounded device-side wait gave up               */
+
+/* Prefetch planning modes. */
+#define PRESERVE_PLAN_WHOLE_NODE 0  /* Algorithm 1: a tensor is prefetched whole or not at all      */
+#define PRESERVE_PLAN_TRUNCATE   1  /* the first tensor that does not fit is prefetched for its
+                                       leading bytes (in the order its consumer reads them)          */
+
+/* flags for preserve_layer_config_t.flags */
+#define PRESERVE_FLAG_NO_GRAPH   1u /* launch kernels directly instead of replaying a CUDA graph     */
+#define PRESERVE_FLAG_PERSIST_L2 2u /* mark prefetched lines as persisting (access-policy window)    */
+
+typedef struct preserve_layer preserve_layer_t;   /* opaque, owned by the library */
+
+/* Per-shard sizes.  Supported: head_dim == 128; n_q_heads a multiple of
+ * n_kv_heads with at most 16 query heads per KV head; hidden a multiple of 128
+ * and at most 16384; ffn a multiple of 32 (128 when max_batch >= 16);
+ * 1 <= tp_degree <= 16; 1 <= max_batch <= 128. */
+typedef struct {
+    int32_t hidden;       /* H                                                       */
+    int32_t n_q_heads;    /* query heads held by this shard                          */
+    int32_t n_kv_heads;   /* KV heads held by this shard                             */
+    int32_t head_dim;     /* d                                                       */
+    int32_t ffn;          /* F: this shard's slice of the MLP intermediate dimension */
+    int32_t tp_degree;    /* P: partial-sum buffers summed in each window            */
+    int32_t max_batch;    /* largest batch of any step                               */
+    int32_t max_ctx;      /* most tokens ever cached per sequence; KV capacity is max_ctx + 1 */
+    float   rms_eps;      /* RMSNorm epsilon (inside the square root)                */
+    float   rope_theta;   /* rotary base; <= 0 disables the rotary embedding         */
+    uint32_t flags;       /* PRESERVE_FLAG_*                                         */
+} preserve_layer_config_t;
+
+/* Device pointers, row-major [in, out] (y = x W), no biases. */
+typedef struct {
+    const void *w_q;      /* [hidden, n_q_heads*head_dim]  */
+    const void *w_k;      /* [hidden, n_kv_heads*head_dim] */
+    const void *w_v;      /* [hidden, n_kv_heads*head_dim] */
+    const void *w_o;      /* [n_q_heads*head_dim, hidden]  */
+    const void *w_gate;   /* [hidden, ffn]                 */
+    const void *w_up;     /* [hidden, ffn]                 */
+    const void *w_down;   /* [ffn, hidden]                 */
+    const void *g_attn;   /* [hidden] RMSNorm gain before attention */
+    const void *g_mlp;    /* [hidden] RMSNorm gain before the MLP   */
+} preserve_layer_weights_t;
+
+/* One decode step.  ctx_len[b] = tokens already cached for sequence b; the
+ * step writes the new key/value at slot ctx_len[b] and attends over slots
+ * 0..ctx_len[b].  The library never advances ctx_len. */
+typedef struct {
+    int32_t batch;                          /* 1..max_batch                                         */
+    const int32_t *ctx_len;                 /* device [batch], each 0..max_ctx                      */
+    const int32_t *ctx_len_host;            /* host copy of the same values (used for planning)     */
+    const void *const *partials_in;         /* host array of P device pointers, each [batch,hidden]:
+                                               the partial sums reduced in the first window         */
+    const void *const *attn_peer_partials;  /* host array of P-1 device pointers, [batch,hidden]:
+                                               the other shards' attention partial sums (second
+                                               window; slot 0 there is this shard's own result)      */
+    const void *residual_in;                /* device [batch,hidden]                                */
+    void *k_cache;                          /* device [max_batch,n_kv_heads,max_ctx+1,head_dim]     */
+    void *v_cache;                          /* same shape; both are read, and written at one slot   */
+    void *residual_out;                     /* device [batch,hidden]: residual after the attention block */
+    void *mlp_partial_out;                  /* device [batch,hidden]: this shard's MLP partial sum  */
+    void *attn_partial_out;                 /* optional (NULL ok) [batch,hidden]: attention partial sum */
+} preserve_step_io_t;
+
+/* Same step with HOST activation buffers: the call copies partials, peers and
+ * residual to the device, runs the step and copies the two outputs back, all on
+ * the given stream.  The KV-cache stays on the device. */
+typedef struct {
+    int32_t batch;
+    const int32_t *ctx_len_host;            /* host [batch]                                          */
+    const void *const *partials_in;         /* host array of P HOST pointers, [batch,hidden]         */
+    const void *const *attn_peer_partials;  /* host array of P-1 HOST pointers                       */
+    const void *residual_in;                /* HOST [batch,hidden]                                   */
+    void *k_cache, *v_cache;                /* device                                                */
+    void *residual_out;                     /* HOST [batch,hidden]                                   */
+    void *mlp_partial_out;                  /* HOST [batch,hidden]                                   */
+} preserve_host_io_t;
+
+typedef struct {
+    int32_t sm_count;
+    int32_t l2_bytes;                 /* cudaDevAttrL2CacheSize                         */
+    int32_t max_persisting_l2_bytes;  /* cudaDevAttrMaxPersistingL2CacheSize            */
+    int32_t max_access_window_bytes;  /* cudaDevAttrMaxAccessPolicyWindowSize           */
+    int32_t uses_tensor_path;         /* 1: tcgen05 GEMM (max_batch >= 16); 0: split-K GEMV */
+    int32_t plan_mode;
+    uint64_t prefetch_budget;         /* bytes per window                               */
+    uint64_t weight_bytes[4];         /* Wqkv, Wo, Wgate|up, Wdown                      */
+    uint64_t kv_bytes;                /* K+V bytes read by the last planned step        */
+    uint64_t planned_bytes[2][3];     /* last plan: window A {Wqkv,KV,Wo}; window B {Wgate|up,Wdown,-} */
+    uint64_t algorithmic_bytes;       /* weights + KV + activations of the last planned step */
+} preserve_info_t;
+
+/* Create a layer: validates the sizes, packs the weights into a library-owned
+ * arena laid out in the order the kernels consume them, allocates workspaces,
+ * a side stream and events on the CURRENT device.  The weight pointers may be
+ * freed after the call returns.  *out is NULL on failure.
+ * The prefetch budget starts at the device's L2 size, mode PRESERVE_PLAN_TRUNCATE. */
+PRESERVE_API int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer_weights_t *w,
+                        preserve_layer_t **out);
+
+/* Upper limit, in bytes, on what one window's prefetch may bring into L2
+ * (Algorithm 1's C; Section 3 "L2 capacity requirements").  0 switches the
+ * prefetch off entirely: no side-stream work is queued. */
+PRESERVE_API int preserve_set_prefetch_bytes(preserve_layer_t *layer, size_t bytes_per_window);
+
+/* PRESERVE_PLAN_WHOLE_NODE (Algorithm 1 as printed) or PRESERVE_PLAN_TRUNCATE. */
+PRESERVE_API int preserve_set_plan_mode(preserve_layer_t *layer, int mode);
+
+/* Queue one decode step of this layer on `cuda_stream` (a cudaStream_t; NULL =
+ * the legacy default stream).  Steps: window A (sum of partials_in + residual_in,
+ * RMSNorm) || prefetch {Wqkv, K/V, Wo};  QKV projection + rotary embedding + KV
+ * append;  split-KV attention;  output projection;  window B (own + peers'
+ * attention partials + residual, RMSNorm) || prefetch {Wgate|up, Wdown};  gate/up
+ * projection + SwiGLU;  down projection. */
+PRESERVE_API int preserve_decode_step(preserve_layer_t *layer, const preserve_step_io_t *io, void *cuda_stream);
+
+/* Queue n layers back to back (a chain): ios[i] describes layer i's buffers as
+ * given; when link != 0, layer i+1's partials_in[0] and residual_in are taken
+ * from layer i's mlp_partial_out and residual_out instead of ios[i+1]'s.  All
+ * layers must share batch.  The whole chain is replayed as one CUDA graph. */
+PRESERVE_API int preserve_decode_chain(preserve_layer_t *const *layers, int32_t n, const preserve_step_io_t *ios,
+                          int32_t link, void *cuda_stream);
+
+/* The step with host activation buffers (see preserve_host_io_t).  Host
+ * buffers should be pinned for the copies to be asynchronous. */
+PRESERVE_API int preserve_decode_step_host(preserve_layer_t *layer, const preserve_host_io_t *io, void *cuda_stream);
+
+/* Sizes, device attributes and the last plan. */
+PRESERVE_API int preserve_layer_get_info(const preserve_layer_t *layer, preserve_info_t *info);
+
+/* Synchronises the device work queued by this handle and returns the device
+ * status word: PRESERVE_OK, or PRESERVE_ETIMEOUT if a bounded wait gave up. */
+PRESERVE_API int preserve_last_status(preserve_layer_t *layer);
+
+/* The cudaError_t of the most recent failing CUDA call made for this handle. */
+PRESERVE_API int preserve_last_cuda_error(const preserve_layer_t *layer);
+
+/* Copy an intermediate of the last step into a caller's device buffer (for
+ * kernel-level checks).  which: 0 h (fp32 [batch,hidden]), 1 x, 2 q (after the
+ * rotary embedding, [batch,n_q_heads,head_dim]), 3 o (attention output, same
+ * shape), 4 x2, 5 a ([batch,ffn]); 1..5 are bf16.  `bytes` must not exceed the
+ * intermediate's size.  Asynchronous on `cuda_stream`. */
+PRESERVE_API int preserve_debug_copy(preserve_layer_t *layer, int32_t which, void *dst_device, size_t bytes,
+                        void *cuda_stream);
+
+/* Frees everything the library allocated for the handle (NULL is allowed). */
+PRESERVE_API void preserve_layer_destroy(preserve_layer_t *layer);
+
+/* Static description of a PRESERVE_E* code. */
+PRESERVE_API const char *preserve_strerror(int code);
+
+/* Host-only: prefetch planning for one window (Algorithm 1 applied to an
+ * ordered list of MatMul / SelfAttention nodes between two communication ops).
+ * node_bytes[i] = bytes a prefetch of node i brings in; out_bytes[i] receives
+ * what is prefetched (0, the whole node, or in TRUNCATE mode a leading part
+ * rounded down to 128 bytes).  Needs no GPU. */
+PRESERVE_API int preserve_plan_window(const uint64_t *node_bytes, int32_t n_nodes, uint64_t budget, int32_t mode,
+                         uint64_t *out_bytes);
+
+/* Host-only: bytes one step must move once (weights + K/V of the cached tokens
+ * + activations), the numerator of the effective-bandwidth figure.
+ * sum_ctx = sum over the batch of tokens already cached. */
+PRESERVE_API uint64_t preserve_algorithmic_bytes(const preserve_layer_config_t *cfg, int32_t batch, uint64_t sum_ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PRESERVE_H */

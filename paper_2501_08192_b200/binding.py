@@ -1,0 +1,227 @@
+"""Thin ctypes binding over libpreserve.so (same names as include/preserve.h).
+
+Argument marshalling only: every step of the decode path runs inside the CUDA
+library.  torch is used for device memory and streams.  There is no CPU
+fallback: if the library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpreserve.so")
+
+PRESERVE_OK = 0
+PRESERVE_EINVAL, PRESERVE_EALIGN, PRESERVE_ESHAPE, PRESERVE_ENOMEM = -1, -2, -3, -4
+PRESERVE_ECUDA, PRESERVE_EARCH, PRESERVE_ETIMEOUT = -5, -6, -7
+PLAN_WHOLE_NODE, PLAN_TRUNCATE = 0, 1
+FLAG_NO_GRAPH, FLAG_PERSIST_L2 = 1, 2
+
+EXPORTS = (
+    "preserve_layer_init", "preserve_set_prefetch_bytes", "preserve_set_plan_mode", "preserve_decode_step",
+    "preserve_decode_chain", "preserve_decode_step_host", "preserve_layer_get_info", "preserve_last_status",
+    "preserve_last_cuda_error", "preserve_debug_copy", "preserve_layer_destroy", "preserve_strerror",
+    "preserve_plan_window", "preserve_algorithmic_bytes",
+)
+
+
+class LayerConfig(C.Structure):
+    _fields_ = [("hidden", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("ffn", C.c_int32), ("tp_degree", C.c_int32),
+                ("max_batch", C.c_int32), ("max_ctx", C.c_int32), ("rms_eps", C.c_float),
+                ("rope_theta", C.c_float), ("flags", C.c_uint32)]
+
+
+class LayerWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("w_q", "w_k", "w_v", "w_o", "w_gate", "w_up", "w_down",
+                                           "g_attn", "g_mlp")]
+
+
+class StepIO(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("ctx_len", C.c_void_p), ("ctx_len_host", C.c_void_p),
+                ("partials_in", C.POINTER(C.c_void_p)), ("attn_peer_partials", C.POINTER(C.c_void_p)),
+                ("residual_in", C.c_void_p), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+                ("residual_out", C.c_void_p), ("mlp_partial_out", C.c_void_p),
+                ("attn_partial_out", C.c_void_p)]
+
+
+class HostIO(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("ctx_len_host", C.c_void_p),
+                ("partials_in", C.POINTER(C.c_void_p)), ("attn_peer_partials", C.POINTER(C.c_void_p)),
+                ("residual_in", C.c_void_p), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+                ("residual_out", C.c_void_p), ("mlp_partial_out", C.c_void_p)]
+
+
+class Info(C.Structure):
+    _fields_ = [("sm_count", C.c_int32), ("l2_bytes", C.c_int32), ("max_persisting_l2_bytes", C.c_int32),
+                ("max_access_window_bytes", C.c_int32), ("uses_tensor_path", C.c_int32),
+                ("plan_mode", C.c_int32), ("prefetch_budget", C.c_uint64),
+                ("weight_bytes", C.c_uint64 * 4), ("kv_bytes", C.c_uint64),
+                ("planned_bytes", (C.c_uint64 * 3) * 2), ("algorithmic_bytes", C.c_uint64)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libpreserve.so (built by paper_2501_08192_b200.build); raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not found: run `python -m paper_2501_08192_b200.build` "
+                               "(there is no fallback path)")
+        L = C.CDLL(LIB_PATH)
+        L.preserve_layer_init.argtypes = [C.POINTER(LayerConfig), C.POINTER(LayerWeights), C.POINTER(C.c_void_p)]
+        L.preserve_set_prefetch_bytes.argtypes = [C.c_void_p, C.c_size_t]
+        L.preserve_set_plan_mode.argtypes = [C.c_void_p, C.c_int]
+        L.preserve_decode_step.argtypes = [C.c_void_p, C.POINTER(StepIO), C.c_void_p]
+        L.preserve_decode_chain.argtypes = [C.POINTER(C.c_void_p), C.c_int32, C.POINTER(StepIO), C.c_int32,
+                                            C.c_void_p]
+        L.preserve_decode_step_host.argtypes = [C.c_void_p, C.POINTER(HostIO), C.c_void_p]
+        L.preserve_layer_get_info.argtypes = [C.c_void_p, C.POINTER(Info)]
+        L.preserve_last_status.argtypes = [C.c_void_p]
+        L.preserve_last_cuda_error.argtypes = [C.c_void_p]
+        L.preserve_debug_copy.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.preserve_layer_destroy.argtypes = [C.c_void_p]
+        L.preserve_layer_destroy.restype = None
+        L.preserve_strerror.argtypes = [C.c_int]
+        L.preserve_strerror.restype = C.c_char_p
+        L.preserve_plan_window.argtypes = [C.POINTER(C.c_uint64), C.c_int32, C.c_uint64, C.c_int32,
+                                           C.POINTER(C.c_uint64)]
+        L.preserve_algorithmic_bytes.argtypes = [C.POINTER(LayerConfig), C.c_int32, C.c_uint64]
+        L.preserve_algorithmic_bytes.restype = C.c_uint64
+        _lib = L
+    return _lib
+
+
+class PreserveError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {preserve_strerror(code)} ({code})")
+
+
+def _check(code: int, what: str) -> None:
+    if code != PRESERVE_OK:
+        raise PreserveError(code, what)
+
+
+def preserve_strerror(code: int) -> str:
+    return lib().preserve_strerror(code).decode()
+
+
+def preserve_plan_window(node_bytes: Sequence[int], budget: int, mode: int = PLAN_WHOLE_NODE) -> List[int]:
+    n = len(node_bytes)
+    src = (C.c_uint64 * max(n, 1))(*node_bytes)
+    dst = (C.c_uint64 * max(n, 1))()
+    _check(lib().preserve_plan_window(src, n, budget, mode, dst), "preserve_plan_window")
+    return [int(dst[i]) for i in range(n)]
+
+
+def make_config(shape, max_batch: Optional[int] = None, max_ctx: Optional[int] = None, flags: int = 0) -> LayerConfig:
+    """LayerConfig from an inputs.ShardShape-like object."""
+    return LayerConfig(shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn,
+                       shape.tp_degree, shape.batch if max_batch is None else max_batch,
+                       shape.ctx if max_ctx is None else max_ctx, shape.rms_eps, shape.rope_theta, flags)
+
+
+def preserve_algorithmic_bytes(cfg: LayerConfig, batch: int, sum_ctx: int) -> int:
+    return int(lib().preserve_algorithmic_bytes(C.byref(cfg), batch, sum_ctx))
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else int(t.data_ptr())
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+class Layer:
+    """Owns one preserve_layer_t handle.  Methods mirror the C entry points."""
+
+    def __init__(self, cfg: LayerConfig, weights: dict):
+        """weights: name -> CUDA bf16 tensor ([in,out] row-major) for w_q..w_down, g_attn, g_mlp."""
+        self.cfg = cfg
+        w = LayerWeights(*[_ptr(weights[n].contiguous()) for n, _ in LayerWeights._fields_])
+        h = C.c_void_p()
+        _check(lib().preserve_layer_init(C.byref(cfg), C.byref(w), C.byref(h)), "preserve_layer_init")
+        self.handle = h
+        self._keep = []
+
+    def close(self) -> None:
+        if self.handle:
+            lib().preserve_layer_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_prefetch_bytes(self, n: int) -> None:
+        _check(lib().preserve_set_prefetch_bytes(self.handle, n), "preserve_set_prefetch_bytes")
+
+    def set_plan_mode(self, mode: int) -> None:
+        _check(lib().preserve_set_plan_mode(self.handle, mode), "preserve_set_plan_mode")
+
+    def make_io(self, batch, ctx_len_dev, ctx_len_host, partials_in, attn_peer_partials, residual_in,
+                k_cache, v_cache, residual_out, mlp_partial_out, attn_partial_out=None) -> StepIO:
+        """Marshal tensors into a StepIO.  ctx_len_host: int32 numpy array or CPU tensor (kept alive here)."""
+        P = self.cfg.tp_degree
+        parts = (C.c_void_p * P)(*[_ptr(t) for t in partials_in])
+        peers = (C.c_void_p * max(P - 1, 1))(*[_ptr(t) for t in attn_peer_partials])
+        host_ptr = ctx_len_host.ctypes.data if hasattr(ctx_len_host, "ctypes") else ctx_len_host.data_ptr()
+        io = StepIO(batch, _ptr(ctx_len_dev), host_ptr, parts, peers, _ptr(residual_in), _ptr(k_cache),
+                    _ptr(v_cache), _ptr(residual_out), _ptr(mlp_partial_out), _ptr(attn_partial_out))
+        io._keep = (parts, peers, ctx_len_host, ctx_len_dev, partials_in, attn_peer_partials, residual_in,
+                    k_cache, v_cache, residual_out, mlp_partial_out, attn_partial_out)
+        return io
+
+    def decode_step(self, io: StepIO, stream=None) -> None:
+        _check(lib().preserve_decode_step(self.handle, C.byref(io), _stream_ptr(stream)), "preserve_decode_step")
+
+    def decode_step_host(self, io: HostIO, stream=None) -> None:
+        _check(lib().preserve_decode_step_host(self.handle, C.byref(io), _stream_ptr(stream)),
+               "preserve_decode_step_host")
+
+    def get_info(self) -> Info:
+        info = Info()
+        _check(lib().preserve_layer_get_info(self.handle, C.byref(info)), "preserve_layer_get_info")
+        return info
+
+    def last_status(self) -> int:
+        return int(lib().preserve_last_status(self.handle))
+
+    def last_cuda_error(self) -> int:
+        return int(lib().preserve_last_cuda_error(self.handle))
+
+    def debug_copy(self, which: int, dst, stream=None) -> None:
+        _check(lib().preserve_debug_copy(self.handle, which, _ptr(dst), dst.numel() * dst.element_size(),
+                                         _stream_ptr(stream)), "preserve_debug_copy")
+
+
+def preserve_decode_chain(layers: Sequence[Layer], ios: Sequence[StepIO], link: bool, stream=None) -> None:
+    n = len(layers)
+    hs = (C.c_void_p * n)(*[l.handle for l in layers])
+    arr = (StepIO * n)(*ios)
+    _check(lib().preserve_decode_chain(hs, n, arr, 1 if link else 0, _stream_ptr(stream)), "preserve_decode_chain")
+
+
+def make_host_io(cfg: LayerConfig, batch, ctx_len_host, partials_in, attn_peer_partials, residual_in,
+                 k_cache, v_cache, residual_out, mlp_partial_out) -> HostIO:
+    """HostIO from pinned CPU tensors (activations) and CUDA tensors (caches)."""
+    P = cfg.tp_degree
+    parts = (C.c_void_p * P)(*[_ptr(t) for t in partials_in])
+    peers = (C.c_void_p * max(P - 1, 1))(*[_ptr(t) for t in attn_peer_partials])
+    host_ptr = ctx_len_host.ctypes.data if hasattr(ctx_len_host, "ctypes") else ctx_len_host.data_ptr()
+    io = HostIO(batch, host_ptr, parts, peers, _ptr(residual_in), _ptr(k_cache), _ptr(v_cache),
+                _ptr(residual_out), _ptr(mlp_partial_out))
+    io._keep = (parts, peers, ctx_len_host, partials_in, attn_peer_partials, residual_in, k_cache, v_cache,
+                residual_out, mlp_partial_out)
+    return io

@@ -1,0 +1,931 @@
+// Layer runtime and C ABI: weight arena, workspaces, the prefetch planner
+// (Algorithm 1 over the layer's fixed operator list), the two-stream schedule
+// (Section 3, "PRESERVE": prefetch operators run in a stream parallel to the main
+// stream and are ordered by events) and CUDA-graph replay of whole steps.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/preserve.h"
+#include "kernels.h"
+
+using namespace prsv;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor map: `rows` rows of `cols` contiguous elements, box (box_cols x box_rows), 128-byte swizzle.
+bool make_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_cols, uint32_t box_rows)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn)
+        return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct GraphEntry {
+    uint64_t key;
+    cudaGraphExec_t exec;
+    uint64_t stamp;
+};
+
+}  // namespace
+
+struct preserve_layer {
+    preserve_layer_config_t cfg;
+    int dev, sm_count, l2_bytes, max_persist, max_window;
+    bool tensor_path;
+    int group;
+
+    uint8_t *arena;              // packed weights: Wqkv | Wo | Wgate,up | Wdown, then gains
+    size_t arena_bytes;
+    size_t off[4];
+    uint64_t wbytes[4];
+    void *g_attn, *g_mlp;
+    double *inv_freq;
+
+    float *h_f32;
+    void *x, *q, *o, *attn_partial, *x2, *a;
+    float *part_o, *part_ml;
+    int max_items, attn_grid;
+    int *status;
+
+    // staging for the host-buffer entry point
+    uint8_t *stage_in, *stage_out;
+    int *ctx_dev;
+
+    // tensor path
+    CUtensorMap wmap[4];
+    CUtensorMap xmap[4];         // x, o, x2, a as B operands
+    int nb_pad;
+
+    // K/V maps (re-encoded when the cache pointers change)
+    const void *k_ptr, *v_ptr;
+    CUtensorMap k_map, v_map;
+
+    cudaStream_t side;
+    cudaEvent_t ev_a, ev_b, ev_join;
+
+    size_t budget;
+    int plan_mode;
+    uint64_t planned[2][3];
+    uint64_t kv_bytes, alg_bytes;
+    int last_cuda;
+    int prefetch_ctas;
+
+    std::vector<GraphEntry> graphs;
+    uint64_t stamp;
+};
+
+namespace {
+
+int cuda_fail(preserve_layer *L, cudaError_t e)
+{
+    if (L)
+        L->last_cuda = (int)e;
+    (void)cudaGetLastError();
+    return e == cudaErrorMemoryAllocation ? PRESERVE_ENOMEM : PRESERVE_ECUDA;
+}
+
+#define CK(L, expr)                                \
+    do {                                           \
+        cudaError_t e__ = (expr);                  \
+        if (e__ != cudaSuccess)                    \
+            return cuda_fail((L), e__);            \
+    } while (0)
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+uint64_t fnv1a(uint64_t h, const void *data, size_t n)
+{
+    const uint8_t *p = static_cast<const uint8_t *>(data);
+    for (size_t i = 0; i < n; ++i) {
+        h ^= p[i];
+        h *= 1099511628211ull;
+    }
+    return h;
+}
+
+int validate_config(const preserve_layer_config_t *c)
+{
+    if (c->head_dim != kHeadDim)
+        return PRESERVE_ESHAPE;
+    if (c->n_q_heads < 1 || c->n_kv_heads < 1 || c->n_q_heads % c->n_kv_heads || c->n_q_heads / c->n_kv_heads > 16)
+        return PRESERVE_ESHAPE;
+    if (c->hidden < 128 || c->hidden % 128 || c->hidden > 16384)
+        return PRESERVE_ESHAPE;
+    if (c->max_batch < 1 || c->max_batch > 128)
+        return PRESERVE_ESHAPE;
+    if (c->ffn < 32 || c->ffn % 32 || (c->max_batch >= 16 && c->ffn % 128))
+        return PRESERVE_ESHAPE;
+    if (c->tp_degree < 1 || c->tp_degree > kMaxParts)
+        return PRESERVE_ESHAPE;
+    if (c->max_ctx < 0 || (long long)c->max_batch * c->n_kv_heads > 2048)
+        return PRESERVE_ESHAPE;
+    if ((long long)c->max_batch * c->n_kv_heads * ((long long)c->max_ctx + 1) > 0x7fffffffll)
+        return PRESERVE_ESHAPE;
+    return PRESERVE_OK;
+}
+
+struct Dims {
+    int n[4], k[4];
+};
+Dims layer_dims(const preserve_layer_config_t &c)
+{
+    Dims d;
+    d.n[0] = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim; d.k[0] = c.hidden;
+    d.n[1] = c.hidden;                                      d.k[1] = c.n_q_heads * c.head_dim;
+    d.n[2] = 2 * c.ffn;                                     d.k[2] = c.hidden;
+    d.n[3] = c.hidden;                                      d.k[3] = c.ffn;
+    return d;
+}
+
+uint64_t activation_bytes(const preserve_layer_config_t &c, int B)
+{
+    const uint64_t BH = (uint64_t)B * c.hidden * 2, Bq = (uint64_t)B * c.n_q_heads * c.head_dim * 2;
+    const uint64_t Bkv = (uint64_t)B * c.n_kv_heads * c.head_dim * 2, BF = (uint64_t)B * c.ffn * 2;
+    const uint64_t gain = (uint64_t)c.hidden * 2, P = c.tp_degree;
+    uint64_t t = 0;
+    t += (P + 1) * BH + gain + 2 * BH;   // window A: reads, gain, writes h and x
+    t += BH + Bq + 2 * Bkv;              // QKV: reads x, writes q, appends k and v
+    t += Bq + Bq;                        // attention: reads q, writes o
+    t += Bq + BH;                        // O: reads o, writes the attention partial
+    t += (P + 1) * BH + gain + 2 * BH;   // window B
+    t += BH + BF;                        // gate/up: reads x2, writes a
+    t += BF + BH;                        // down: reads a, writes the MLP partial
+    return t;
+}
+
+void plan_window(const uint64_t *node_bytes, int n, uint64_t budget, int mode, uint64_t *out)
+{
+    // Algorithm 1 for one communication op whose successors, in breadth-first order, are the
+    // given MatMul / SelfAttention nodes followed by the next communication op.
+    uint64_t cache_sum = 0;
+    for (int i = 0; i < n; ++i)
+        out[i] = 0;
+    for (int i = 0; i < n; ++i) {
+        if (cache_sum + node_bytes[i] < budget) {       // strict, as in the listing
+            cache_sum += node_bytes[i];
+            out[i] = node_bytes[i];
+        } else {
+            if (mode == PRESERVE_PLAN_TRUNCATE) {
+                const uint64_t room = budget > cache_sum ? budget - cache_sum : 0;
+                uint64_t part = room & ~uint64_t(127);
+                if (part > node_bytes[i])
+                    part = node_bytes[i];
+                out[i] = part;
+            }
+            break;                                      // end of the walk for this op
+        }
+    }
+}
+
+// ------------------------------------------------------------------ one step
+struct StepPtrs {
+    int batch;
+    const int *ctx_len;
+    const int *ctx_len_host;
+    const void *parts[kMaxParts];
+    const void *peers[kMaxParts];
+    const void *residual_in;
+    void *k_cache, *v_cache;
+    void *residual_out, *mlp_partial_out, *attn_partial_out;
+};
+
+int check_step(preserve_layer *L, const preserve_step_io_t *io, StepPtrs *sp)
+{
+    if (!L || !io)
+        return PRESERVE_EINVAL;
+    const auto &c = L->cfg;
+    if (io->batch < 1 || io->batch > c.max_batch)
+        return PRESERVE_ESHAPE;
+    if (!io->ctx_len || !io->ctx_len_host || !io->partials_in || !io->residual_in || !io->k_cache || !io->v_cache ||
+        !io->residual_out || !io->mlp_partial_out)
+        return PRESERVE_EINVAL;
+    if (c.tp_degree > 1 && !io->attn_peer_partials)
+        return PRESERVE_EINVAL;
+    sp->batch = io->batch;
+    sp->ctx_len = io->ctx_len;
+    sp->ctx_len_host = io->ctx_len_host;
+    for (int i = 0; i < c.tp_degree; ++i) {
+        if (!io->partials_in[i])
+            return PRESERVE_EINVAL;
+        if (!aligned16(io->partials_in[i]))
+            return PRESERVE_EALIGN;
+        sp->parts[i] = io->partials_in[i];
+    }
+    for (int i = 0; i + 1 < c.tp_degree; ++i) {
+        if (!io->attn_peer_partials[i])
+            return PRESERVE_EINVAL;
+        if (!aligned16(io->attn_peer_partials[i]))
+            return PRESERVE_EALIGN;
+        sp->peers[i] = io->attn_peer_partials[i];
+    }
+    const void *ptrs[] = {io->residual_in, io->k_cache, io->v_cache, io->residual_out, io->mlp_partial_out,
+                          io->attn_partial_out};
+    for (const void *p : ptrs)
+        if (p && !aligned16(p))
+            return PRESERVE_EALIGN;
+    if (reinterpret_cast<uintptr_t>(io->ctx_len) & 3)
+        return PRESERVE_EALIGN;
+    for (int b = 0; b < io->batch; ++b)
+        if (io->ctx_len_host[b] < 0 || io->ctx_len_host[b] > c.max_ctx)
+            return PRESERVE_ESHAPE;
+    sp->residual_in = io->residual_in;
+    sp->k_cache = io->k_cache;
+    sp->v_cache = io->v_cache;
+    sp->residual_out = io->residual_out;
+    sp->mlp_partial_out = io->mlp_partial_out;
+    sp->attn_partial_out = io->attn_partial_out;
+    return PRESERVE_OK;
+}
+
+int launch_gemm(preserve_layer *L, int which, const void *x, int B, const EpilogueArgs &epi, cudaStream_t s)
+{
+    const Dims d = layer_dims(L->cfg);
+    if (L->tensor_path) {
+        GemmTcArgs a;
+        a.w_map = L->wmap[which];
+        a.x_map = L->xmap[which];
+        a.B = B; a.NB = L->nb_pad; a.N = d.n[which]; a.K = d.k[which];
+        a.epi = epi;
+        a.status = L->status;
+        CK(L, launch_gemm_tc(a, L->sm_count, s));
+        return PRESERVE_OK;
+    }
+    for (int b0 = 0; b0 < B; b0 += 16) {
+        GemvArgs a;
+        a.w = L->arena + L->off[which];
+        a.x = x;
+        a.B = B - b0 < 16 ? B - b0 : 16;
+        a.b0 = b0;
+        a.N = d.n[which]; a.K = d.k[which];
+        a.epi = epi;
+        CK(L, launch_gemv(a, L->sm_count, s));
+    }
+    return PRESERVE_OK;
+}
+
+// Queue one layer step on `s` (directly, or into an ongoing capture of `s`).
+int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
+{
+    const auto &c = L->cfg;
+    const int B = sp.batch, H = c.hidden, cap = c.max_ctx + 1;
+    const Dims d = layer_dims(c);
+
+    // ---- plan (host): Algorithm 1 per window over {Wqkv, KV, Wo} and {Wgate|up, Wdown}
+    uint64_t sum_ctx = 0, total_tiles = 0;
+    for (int b = 0; b < B; ++b) {
+        sum_ctx += (uint64_t)sp.ctx_len_host[b];
+        total_tiles += (uint64_t)c.n_kv_heads * ((sp.ctx_len_host[b] + 1 + 63) / 64);
+    }
+    L->kv_bytes = 2 * sum_ctx * c.n_kv_heads * c.head_dim * 2;
+    const uint64_t nodes_a[3] = {L->wbytes[0], L->kv_bytes, L->wbytes[1]};
+    const uint64_t nodes_b[2] = {L->wbytes[2], L->wbytes[3]};
+    plan_window(nodes_a, 3, L->budget, L->plan_mode, L->planned[0]);
+    plan_window(nodes_b, 2, L->budget, L->plan_mode, L->planned[1]);
+    L->planned[1][2] = 0;
+    L->alg_bytes = L->wbytes[0] + L->wbytes[1] + L->wbytes[2] + L->wbytes[3] + L->kv_bytes + activation_bytes(c, B);
+    const bool pf_a = L->planned[0][0] + L->planned[0][1] + L->planned[0][2] > 0;
+    const bool pf_b = L->planned[1][0] + L->planned[1][1] > 0;
+
+    // ---- K/V tensor maps
+    if (sp.k_cache != L->k_ptr || sp.v_cache != L->v_ptr) {
+        const uint64_t rows = (uint64_t)c.max_batch * c.n_kv_heads * cap;
+        if (!make_map_2d(&L->k_map, sp.k_cache, kHeadDim, rows, 64, 64) ||
+            !make_map_2d(&L->v_map, sp.v_cache, kHeadDim, rows, 64, 64))
+            return PRESERVE_EARCH;
+        L->k_ptr = sp.k_cache;
+        L->v_ptr = sp.v_cache;
+    }
+
+    // ---- window A  ||  prefetch {Wqkv, K/V, Wo}
+    if (pf_a) {
+        CK(L, cudaEventRecord(L->ev_a, s));
+        CK(L, cudaStreamWaitEvent(L->side, L->ev_a, 0));
+        PrefetchArgs pa = {};
+        pa.ctx_len = sp.ctx_len;
+        int n = 0;
+        if (L->planned[0][0]) {
+            pa.seg[n].base = L->arena + L->off[0];
+            pa.seg[n].bytes = L->planned[0][0];
+            ++n;
+        }
+        if (L->planned[0][1]) {
+            pa.seg[n].base = sp.k_cache;
+            pa.seg[n].base2 = sp.v_cache;
+            pa.seg[n].stride = (uint64_t)cap * kHeadDim * 2;
+            pa.seg[n].bytes = L->planned[0][1];
+            pa.seg[n].count = B * c.n_kv_heads;
+            pa.seg[n].per_seq_tokens = 1;
+            pa.seg[n].ranges_per_seq = c.n_kv_heads;
+            pa.seg[n].token_bytes = kHeadDim * 2;
+            ++n;
+        }
+        if (L->planned[0][2]) {
+            pa.seg[n].base = L->arena + L->off[1];
+            pa.seg[n].bytes = L->planned[0][2];
+            ++n;
+        }
+        pa.n_segs = n;
+        CK(L, launch_prefetch(pa, L->prefetch_ctas, L->side, nullptr, 0));
+    }
+    {
+        WindowArgs w = {};
+        for (int i = 0; i < c.tp_degree; ++i)
+            w.parts[i] = sp.parts[i];
+        w.n_parts = c.tp_degree;
+        w.resid = sp.residual_in;
+        w.resid_is_f32 = 0;
+        w.gain = L->g_attn;
+        w.eps = c.rms_eps;
+        w.h_f32 = L->h_f32;
+        w.h_bf16 = nullptr;
+        w.x_bf16 = L->x;
+        w.B = B; w.H = H;
+        CK(L, launch_window(w, s));
+    }
+    // ---- QKV projection + rotary embedding + KV append
+    {
+        EpilogueArgs e = {};
+        e.kind = EPI_QKV;
+        e.q_out = L->q;
+        e.k_cache = sp.k_cache;
+        e.v_cache = sp.v_cache;
+        e.ctx_len = sp.ctx_len;
+        e.nq = c.n_q_heads; e.nkv = c.n_kv_heads; e.cap = cap;
+        e.inv_freq = c.rope_theta > 0.f ? L->inv_freq : nullptr;
+        int rc = launch_gemm(L, 0, L->x, B, e, s);
+        if (rc)
+            return rc;
+    }
+    // ---- attention
+    {
+        AttnArgs a = {};
+        a.k_map = L->k_map;
+        a.v_map = L->v_map;
+        a.q = L->q;
+        a.ctx_len = sp.ctx_len;
+        a.B = B; a.nq = c.n_q_heads; a.nkv = c.n_kv_heads; a.cap = cap;
+        a.grid = L->attn_grid;
+        uint64_t tpi = (total_tiles + (uint64_t)L->attn_grid * 4 - 1) / ((uint64_t)L->attn_grid * 4);
+        a.tiles_per_item = tpi < 1 ? 1 : (int)tpi;
+        a.max_items = L->max_items;
+        a.part_o = L->part_o;
+        a.part_ml = L->part_ml;
+        a.o_out = L->o;
+        a.status = L->status;
+        CK(L, launch_attention(a, s));
+    }
+    // ---- output projection -> this shard's attention partial sum
+    {
+        EpilogueArgs e = {};
+        e.kind = EPI_PLAIN;
+        e.out = L->attn_partial;
+        e.out2 = sp.attn_partial_out;
+        int rc = launch_gemm(L, 1, L->o, B, e, s);
+        if (rc)
+            return rc;
+    }
+    // ---- window B  ||  prefetch {Wgate|up, Wdown}
+    if (pf_b) {
+        CK(L, cudaEventRecord(L->ev_b, s));
+        CK(L, cudaStreamWaitEvent(L->side, L->ev_b, 0));
+        PrefetchArgs pa = {};
+        pa.ctx_len = sp.ctx_len;
+        int n = 0;
+        for (int i = 0; i < 2; ++i)
+            if (L->planned[1][i]) {
+                pa.seg[n].base = L->arena + L->off[2 + i];
+                pa.seg[n].bytes = L->planned[1][i];
+                ++n;
+            }
+        pa.n_segs = n;
+        CK(L, launch_prefetch(pa, L->prefetch_ctas, L->side, nullptr, 0));
+    }
+    {
+        WindowArgs w = {};
+        w.parts[0] = L->attn_partial;
+        for (int i = 0; i + 1 < c.tp_degree; ++i)
+            w.parts[i + 1] = sp.peers[i];
+        w.n_parts = c.tp_degree;
+        w.resid = L->h_f32;
+        w.resid_is_f32 = 1;
+        w.gain = L->g_mlp;
+        w.eps = c.rms_eps;
+        w.h_f32 = nullptr;
+        w.h_bf16 = sp.residual_out;
+        w.x_bf16 = L->x2;
+        w.B = B; w.H = H;
+        CK(L, launch_window(w, s));
+    }
+    // ---- gate/up projection + SwiGLU, down projection
+    {
+        EpilogueArgs e = {};
+        e.kind = EPI_SWIGLU;
+        e.out = L->a;
+        int rc = launch_gemm(L, 2, L->x2, B, e, s);
+        if (rc)
+            return rc;
+    }
+    {
+        EpilogueArgs e = {};
+        e.kind = EPI_PLAIN;
+        e.out = sp.mlp_partial_out;
+        int rc = launch_gemm(L, 3, L->a, B, e, s);
+        if (rc)
+            return rc;
+    }
+    // ---- join the side stream
+    if (pf_a || pf_b) {
+        CK(L, cudaEventRecord(L->ev_join, L->side));
+        CK(L, cudaStreamWaitEvent(s, L->ev_join, 0));
+    }
+    (void)d;
+    return PRESERVE_OK;
+}
+
+uint64_t step_key(const preserve_layer *L, const StepPtrs &sp, uint64_t h)
+{
+    h = fnv1a(h, &L, sizeof(L));
+    h = fnv1a(h, &sp.batch, sizeof(int));
+    h = fnv1a(h, &sp.ctx_len, sizeof(void *));
+    h = fnv1a(h, sp.ctx_len_host, sizeof(int) * sp.batch);
+    h = fnv1a(h, sp.parts, sizeof(void *) * L->cfg.tp_degree);
+    h = fnv1a(h, sp.peers, sizeof(void *) * (L->cfg.tp_degree - 1));
+    const void *ptrs[] = {sp.residual_in, sp.k_cache, sp.v_cache, sp.residual_out, sp.mlp_partial_out,
+                          sp.attn_partial_out};
+    h = fnv1a(h, ptrs, sizeof(ptrs));
+    h = fnv1a(h, &L->budget, sizeof(L->budget));
+    h = fnv1a(h, &L->plan_mode, sizeof(int));
+    return h;
+}
+
+// Run `n` steps (already validated) as one replayed graph, or directly.
+int run_steps(preserve_layer *const *layers, const StepPtrs *sps, int n, cudaStream_t s)
+{
+    preserve_layer *L0 = layers[0];
+    const bool direct = (L0->cfg.flags & PRESERVE_FLAG_NO_GRAPH) || s == nullptr || s == cudaStreamLegacy;
+    if (direct) {
+        for (int i = 0; i < n; ++i) {
+            int rc = enqueue_step(layers[i], sps[i], s);
+            if (rc)
+                return rc;
+        }
+        return PRESERVE_OK;
+    }
+    uint64_t key = 1469598103934665603ull;
+    for (int i = 0; i < n; ++i)
+        key = step_key(layers[i], sps[i], key);
+    key = fnv1a(key, &s, sizeof(s));
+    for (auto &g : L0->graphs)
+        if (g.key == key) {
+            g.stamp = ++L0->stamp;
+            CK(L0, cudaGraphLaunch(g.exec, s));
+            return PRESERVE_OK;
+        }
+    // capture
+    cudaStreamCaptureStatus cs;
+    CK(L0, cudaStreamIsCapturing(s, &cs));
+    if (cs != cudaStreamCaptureStatusNone) {
+        // the caller is capturing already: just add our nodes to their graph
+        for (int i = 0; i < n; ++i) {
+            int rc = enqueue_step(layers[i], sps[i], s);
+            if (rc)
+                return rc;
+        }
+        return PRESERVE_OK;
+    }
+    CK(L0, cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal));
+    int rc = PRESERVE_OK;
+    for (int i = 0; i < n && rc == PRESERVE_OK; ++i)
+        rc = enqueue_step(layers[i], sps[i], s);
+    cudaGraph_t graph = nullptr;
+    cudaError_t e = cudaStreamEndCapture(s, &graph);
+    if (rc != PRESERVE_OK) {
+        if (graph)
+            cudaGraphDestroy(graph);
+        return rc;
+    }
+    if (e != cudaSuccess)
+        return cuda_fail(L0, e);
+    cudaGraphExec_t exec = nullptr;
+    e = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess)
+        return cuda_fail(L0, e);
+    if (L0->graphs.size() >= 16) {
+        size_t victim = 0;
+        for (size_t i = 1; i < L0->graphs.size(); ++i)
+            if (L0->graphs[i].stamp < L0->graphs[victim].stamp)
+                victim = i;
+        cudaGraphExecDestroy(L0->graphs[victim].exec);
+        L0->graphs.erase(L0->graphs.begin() + victim);
+    }
+    L0->graphs.push_back({key, exec, ++L0->stamp});
+    CK(L0, cudaGraphLaunch(exec, s));
+    return PRESERVE_OK;
+}
+
+void drop_graphs(preserve_layer *L)
+{
+    for (auto &g : L->graphs)
+        cudaGraphExecDestroy(g.exec);
+    L->graphs.clear();
+}
+
+}  // namespace
+
+// ============================================================== C ABI
+extern "C" {
+
+const char *preserve_strerror(int code)
+{
+    switch (code) {
+    case PRESERVE_OK: return "ok";
+    case PRESERVE_EINVAL: return "invalid argument";
+    case PRESERVE_EALIGN: return "device pointer not 16-byte aligned";
+    case PRESERVE_ESHAPE: return "unsupported shape";
+    case PRESERVE_ENOMEM: return "out of memory";
+    case PRESERVE_ECUDA: return "CUDA call failed";
+    case PRESERVE_EARCH: return "needs an sm_100 device";
+    case PRESERVE_ETIMEOUT: return "a bounded device-side wait gave up";
+    default: return "unknown error";
+    }
+}
+
+int preserve_plan_window(const uint64_t *node_bytes, int32_t n_nodes, uint64_t budget, int32_t mode,
+                         uint64_t *out_bytes)
+{
+    if (!node_bytes || !out_bytes || n_nodes < 0)
+        return PRESERVE_EINVAL;
+    if (mode != PRESERVE_PLAN_WHOLE_NODE && mode != PRESERVE_PLAN_TRUNCATE)
+        return PRESERVE_EINVAL;
+    plan_window(node_bytes, n_nodes, budget, mode, out_bytes);
+    return PRESERVE_OK;
+}
+
+uint64_t preserve_algorithmic_bytes(const preserve_layer_config_t *cfg, int32_t batch, uint64_t sum_ctx)
+{
+    if (!cfg || validate_config(cfg) != PRESERVE_OK || batch < 1)
+        return 0;
+    const Dims d = layer_dims(*cfg);
+    uint64_t w = 0;
+    for (int i = 0; i < 4; ++i)
+        w += (uint64_t)d.n[i] * d.k[i] * 2;
+    const uint64_t kv = 2 * sum_ctx * cfg->n_kv_heads * cfg->head_dim * 2;
+    return w + kv + activation_bytes(*cfg, batch);
+}
+
+void preserve_layer_destroy(preserve_layer_t *L)
+{
+    if (!L)
+        return;
+    cudaSetDevice(L->dev);
+    if (L->side)
+        cudaStreamSynchronize(L->side);
+    drop_graphs(L);
+    void *ptrs[] = {L->arena, L->inv_freq, L->h_f32, L->x, L->q, L->o, L->attn_partial, L->x2, L->a,
+                    L->part_o, L->part_ml, L->status, L->stage_in, L->stage_out, L->ctx_dev};
+    for (void *p : ptrs)
+        if (p)
+            cudaFree(p);
+    if (L->ev_a) cudaEventDestroy(L->ev_a);
+    if (L->ev_b) cudaEventDestroy(L->ev_b);
+    if (L->ev_join) cudaEventDestroy(L->ev_join);
+    if (L->side) cudaStreamDestroy(L->side);
+    delete L;
+}
+
+int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer_weights_t *w,
+                        preserve_layer_t **out)
+{
+    if (out)
+        *out = nullptr;
+    if (!cfg || !w || !out)
+        return PRESERVE_EINVAL;
+    int rc = validate_config(cfg);
+    if (rc)
+        return rc;
+    const void *wp[] = {w->w_q, w->w_k, w->w_v, w->w_o, w->w_gate, w->w_up, w->w_down, w->g_attn, w->g_mlp};
+    for (const void *p : wp) {
+        if (!p)
+            return PRESERVE_EINVAL;
+        if (!aligned16(p))
+            return PRESERVE_EALIGN;
+    }
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return PRESERVE_EARCH;
+    }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess || prop.major != 10) {
+        (void)cudaGetLastError();
+        return PRESERVE_EARCH;
+    }
+    if (!get_encode_fn())
+        return PRESERVE_EARCH;
+
+    preserve_layer *L = new (std::nothrow) preserve_layer();
+    if (!L)
+        return PRESERVE_ENOMEM;
+    L->cfg = *cfg;
+    L->dev = dev;
+    L->sm_count = prop.multiProcessorCount;
+    L->l2_bytes = prop.l2CacheSize;
+    L->max_persist = prop.persistingL2CacheMaxSize;
+    L->max_window = prop.accessPolicyMaxWindowSize;
+    L->group = cfg->n_q_heads / cfg->n_kv_heads;
+    const char *force = getenv("PRESERVE_FORCE_GEMV");
+    L->tensor_path = cfg->max_batch >= 16 && !(force && force[0] == '1');
+    const char *pdl = getenv("PRESERVE_PDL");
+    if (pdl)
+        g_pdl = pdl[0] == '1';
+    const char *pfm = getenv("PRESERVE_PREFETCH_MODE");
+    const char *pfc = getenv("PRESERVE_PREFETCH_CHUNK");
+    if (pfm || pfc)
+        set_prefetch_kernel_mode(pfm ? atoi(pfm) : 0, pfc ? (uint32_t)atoi(pfc) : 4096u);
+    const char *pfn = getenv("PRESERVE_PREFETCH_CTAS");
+    L->prefetch_ctas = pfn ? atoi(pfn) : 8;
+    if (L->prefetch_ctas < 1)
+        L->prefetch_ctas = 1;
+    L->budget = (size_t)L->l2_bytes;
+    L->plan_mode = PRESERVE_PLAN_TRUNCATE;
+
+#define CKI(expr)                                   \
+    do {                                            \
+        cudaError_t e__ = (expr);                   \
+        if (e__ != cudaSuccess) {                   \
+            int r__ = cuda_fail(L, e__);            \
+            preserve_layer_destroy(L);              \
+            return r__;                             \
+        }                                           \
+    } while (0)
+
+    const auto &c = L->cfg;
+    const Dims d = layer_dims(c);
+    const int H = c.hidden, B = c.max_batch;
+    size_t off = 0;
+    for (int i = 0; i < 4; ++i) {
+        L->off[i] = off;
+        L->wbytes[i] = (uint64_t)d.n[i] * d.k[i] * 2;
+        off += (size_t)L->wbytes[i];
+    }
+    const size_t gains_off = off;
+    off += (size_t)2 * H * 2;
+    L->arena_bytes = off;
+    CKI(cudaMalloc(&L->arena, L->arena_bytes));
+    L->g_attn = L->arena + gains_off;
+    L->g_mlp = L->arena + gains_off + (size_t)H * 2;
+    CKI(cudaMemcpy(L->g_attn, w->g_attn, (size_t)H * 2, cudaMemcpyDeviceToDevice));
+    CKI(cudaMemcpy(L->g_mlp, w->g_mlp, (size_t)H * 2, cudaMemcpyDeviceToDevice));
+
+    // pack the four weight blocks in consumption order
+    {
+        const void *s_qkv[3] = {w->w_q, w->w_k, w->w_v};
+        const int c_qkv[3] = {c.n_q_heads * c.head_dim, c.n_kv_heads * c.head_dim, c.n_kv_heads * c.head_dim};
+        const void *s_o[1] = {w->w_o};
+        const int c_o[1] = {H};
+        const void *s_gu[2] = {w->w_gate, w->w_up};
+        const int c_gu[2] = {c.ffn, c.ffn};
+        const void *s_dn[1] = {w->w_down};
+        const int c_dn[1] = {H};
+        auto pack = L->tensor_path ? launch_pack_rows : launch_pack_gemv;
+        CKI(pack(s_qkv, c_qkv, 3, d.k[0], EPI_QKV, L->arena + L->off[0], nullptr));
+        CKI(pack(s_o, c_o, 1, d.k[1], EPI_PLAIN, L->arena + L->off[1], nullptr));
+        CKI(pack(s_gu, c_gu, 2, d.k[2], EPI_SWIGLU, L->arena + L->off[2], nullptr));
+        CKI(pack(s_dn, c_dn, 1, d.k[3], EPI_PLAIN, L->arena + L->off[3], nullptr));
+    }
+    // rotary frequencies theta^(-2i/d)
+    {
+        double f[kHeadDim / 2];
+        for (int i = 0; i < kHeadDim / 2; ++i)
+            f[i] = c.rope_theta > 0.f ? std::pow((double)c.rope_theta, -2.0 * i / (double)kHeadDim) : 0.0;
+        CKI(cudaMalloc(&L->inv_freq, sizeof(f)));
+        CKI(cudaMemcpy(L->inv_freq, f, sizeof(f), cudaMemcpyHostToDevice));
+    }
+    // workspaces
+    const size_t BH = (size_t)B * H, Bq = (size_t)B * c.n_q_heads * c.head_dim;
+    CKI(cudaMalloc(&L->h_f32, BH * 4));
+    CKI(cudaMalloc(&L->x, BH * 2));
+    CKI(cudaMalloc(&L->q, Bq * 2));
+    CKI(cudaMalloc(&L->o, Bq * 2));
+    CKI(cudaMalloc(&L->attn_partial, BH * 2));
+    CKI(cudaMalloc(&L->x2, BH * 2));
+    CKI(cudaMalloc(&L->a, (size_t)B * c.ffn * 2));
+    CKI(cudaMemset(L->x, 0, BH * 2));
+    CKI(cudaMemset(L->o, 0, Bq * 2));
+    CKI(cudaMemset(L->x2, 0, BH * 2));
+    CKI(cudaMemset(L->a, 0, (size_t)B * c.ffn * 2));
+    L->attn_grid = L->sm_count;
+    L->max_items = L->attn_grid * 4 + B * c.n_kv_heads + 8;
+    CKI(cudaMalloc(&L->part_o, (size_t)L->max_items * L->group * kHeadDim * 4));
+    CKI(cudaMalloc(&L->part_ml, (size_t)L->max_items * L->group * 2 * 4));
+    CKI(cudaMalloc(&L->status, 256));
+    CKI(cudaMemset(L->status, 0, 256));
+    const size_t n_in = (size_t)(2 * c.tp_degree) * BH * 2;
+    CKI(cudaMalloc(&L->stage_in, n_in));
+    CKI(cudaMalloc(&L->stage_out, 2 * BH * 2));
+    CKI(cudaMalloc(&L->ctx_dev, (size_t)B * 4));
+
+    if (L->tensor_path) {
+        L->nb_pad = ((B + 15) / 16) * 16;
+        const void *xb[4] = {L->x, L->o, L->x2, L->a};
+        for (int i = 0; i < 4; ++i) {
+            if (!make_map_2d(&L->wmap[i], L->arena + L->off[i], d.k[i], d.n[i], 64, 128) ||
+                !make_map_2d(&L->xmap[i], xb[i], d.k[i], B, 64, L->nb_pad > 256 ? 256 : L->nb_pad)) {
+                preserve_layer_destroy(L);
+                return PRESERVE_EARCH;
+            }
+        }
+    }
+    CKI(cudaStreamCreateWithFlags(&L->side, cudaStreamNonBlocking));
+    CKI(cudaEventCreateWithFlags(&L->ev_a, cudaEventDisableTiming));
+    CKI(cudaEventCreateWithFlags(&L->ev_b, cudaEventDisableTiming));
+    CKI(cudaEventCreateWithFlags(&L->ev_join, cudaEventDisableTiming));
+    CKI(cudaDeviceSynchronize());
+#undef CKI
+    *out = L;
+    return PRESERVE_OK;
+}
+
+int preserve_set_prefetch_bytes(preserve_layer_t *L, size_t bytes_per_window)
+{
+    if (!L)
+        return PRESERVE_EINVAL;
+    L->budget = bytes_per_window;
+    return PRESERVE_OK;
+}
+
+int preserve_set_plan_mode(preserve_layer_t *L, int mode)
+{
+    if (!L || (mode != PRESERVE_PLAN_WHOLE_NODE && mode != PRESERVE_PLAN_TRUNCATE))
+        return PRESERVE_EINVAL;
+    L->plan_mode = mode;
+    return PRESERVE_OK;
+}
+
+int preserve_decode_step(preserve_layer_t *L, const preserve_step_io_t *io, void *cuda_stream)
+{
+    StepPtrs sp = {};
+    int rc = check_step(L, io, &sp);
+    if (rc)
+        return rc;
+    preserve_layer *layers[1] = {L};
+    return run_steps(layers, &sp, 1, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int preserve_decode_chain(preserve_layer_t *const *layers, int32_t n, const preserve_step_io_t *ios, int32_t link,
+                          void *cuda_stream)
+{
+    if (!layers || !ios || n < 1 || n > 256)
+        return PRESERVE_EINVAL;
+    std::vector<StepPtrs> sps((size_t)n);
+    for (int i = 0; i < n; ++i) {
+        int rc = check_step(layers[i], &ios[i], &sps[i]);
+        if (rc)
+            return rc;
+        if (sps[i].batch != sps[0].batch)
+            return PRESERVE_ESHAPE;
+        if (link && i > 0) {
+            if (layers[i]->cfg.hidden != layers[0]->cfg.hidden)
+                return PRESERVE_ESHAPE;
+            sps[i].parts[0] = sps[i - 1].mlp_partial_out;
+            sps[i].residual_in = sps[i - 1].residual_out;
+        }
+    }
+    return run_steps(layers, sps.data(), n, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int preserve_decode_step_host(preserve_layer_t *L, const preserve_host_io_t *io, void *cuda_stream)
+{
+    if (!L || !io)
+        return PRESERVE_EINVAL;
+    const auto &c = L->cfg;
+    if (io->batch < 1 || io->batch > c.max_batch)
+        return PRESERVE_ESHAPE;
+    if (!io->ctx_len_host || !io->partials_in || !io->residual_in || !io->k_cache || !io->v_cache ||
+        !io->residual_out || !io->mlp_partial_out || (c.tp_degree > 1 && !io->attn_peer_partials))
+        return PRESERVE_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const size_t BH2 = (size_t)io->batch * c.hidden * 2;
+    const size_t slot = (size_t)c.max_batch * c.hidden * 2;
+    const void *dparts[kMaxParts], *dpeers[kMaxParts];
+    for (int i = 0; i < c.tp_degree; ++i) {
+        if (!io->partials_in[i])
+            return PRESERVE_EINVAL;
+        CK(L, cudaMemcpyAsync(L->stage_in + (size_t)i * slot, io->partials_in[i], BH2, cudaMemcpyHostToDevice, s));
+        dparts[i] = L->stage_in + (size_t)i * slot;
+    }
+    for (int i = 0; i + 1 < c.tp_degree; ++i) {
+        if (!io->attn_peer_partials[i])
+            return PRESERVE_EINVAL;
+        uint8_t *dst = L->stage_in + (size_t)(c.tp_degree + i) * slot;
+        CK(L, cudaMemcpyAsync(dst, io->attn_peer_partials[i], BH2, cudaMemcpyHostToDevice, s));
+        dpeers[i] = dst;
+    }
+    uint8_t *dres = L->stage_in + (size_t)(2 * c.tp_degree - 1) * slot;
+    CK(L, cudaMemcpyAsync(dres, io->residual_in, BH2, cudaMemcpyHostToDevice, s));
+    CK(L, cudaMemcpyAsync(L->ctx_dev, io->ctx_len_host, (size_t)io->batch * 4, cudaMemcpyHostToDevice, s));
+
+    preserve_step_io_t dio = {};
+    dio.batch = io->batch;
+    dio.ctx_len = L->ctx_dev;
+    dio.ctx_len_host = io->ctx_len_host;
+    dio.partials_in = dparts;
+    dio.attn_peer_partials = dpeers;
+    dio.residual_in = dres;
+    dio.k_cache = io->k_cache;
+    dio.v_cache = io->v_cache;
+    dio.residual_out = L->stage_out;
+    dio.mlp_partial_out = L->stage_out + slot;
+    dio.attn_partial_out = nullptr;
+    int rc = preserve_decode_step(L, &dio, cuda_stream);
+    if (rc)
+        return rc;
+    CK(L, cudaMemcpyAsync(io->residual_out, L->stage_out, BH2, cudaMemcpyDeviceToHost, s));
+    CK(L, cudaMemcpyAsync(io->mlp_partial_out, L->stage_out + slot, BH2, cudaMemcpyDeviceToHost, s));
+    return PRESERVE_OK;
+}
+
+int preserve_layer_get_info(const preserve_layer_t *L, preserve_info_t *info)
+{
+    if (!L || !info)
+        return PRESERVE_EINVAL;
+    memset(info, 0, sizeof(*info));
+    info->sm_count = L->sm_count;
+    info->l2_bytes = L->l2_bytes;
+    info->max_persisting_l2_bytes = L->max_persist;
+    info->max_access_window_bytes = L->max_window;
+    info->uses_tensor_path = L->tensor_path ? 1 : 0;
+    info->plan_mode = L->plan_mode;
+    info->prefetch_budget = L->budget;
+    for (int i = 0; i < 4; ++i)
+        info->weight_bytes[i] = L->wbytes[i];
+    info->kv_bytes = L->kv_bytes;
+    for (int i = 0; i < 2; ++i)
+        for (int j = 0; j < 3; ++j)
+            info->planned_bytes[i][j] = L->planned[i][j];
+    info->algorithmic_bytes = L->alg_bytes;
+    return PRESERVE_OK;
+}
+
+int preserve_last_status(preserve_layer_t *L)
+{
+    if (!L)
+        return PRESERVE_EINVAL;
+    CK(L, cudaSetDevice(L->dev));
+    CK(L, cudaDeviceSynchronize());
+    int st = 0;
+    CK(L, cudaMemcpy(&st, L->status, sizeof(int), cudaMemcpyDeviceToHost));
+    return st == 0 ? PRESERVE_OK : PRESERVE_ETIMEOUT;
+}
+
+int preserve_last_cuda_error(const preserve_layer_t *L) { return L ? L->last_cuda : 0; }
+
+int preserve_debug_copy(preserve_layer_t *L, int32_t which, void *dst, size_t bytes, void *cuda_stream)
+{
+    if (!L || !dst)
+        return PRESERVE_EINVAL;
+    const auto &c = L->cfg;
+    const size_t BH = (size_t)c.max_batch * c.hidden, Bq = (size_t)c.max_batch * c.n_q_heads * c.head_dim;
+    const void *src[6] = {L->h_f32, L->x, L->q, L->o, L->x2, L->a};
+    const size_t cap[6] = {BH * 4, BH * 2, Bq * 2, Bq * 2, BH * 2, (size_t)c.max_batch * c.ffn * 2};
+    if (which < 0 || which > 5 || bytes > cap[which])
+        return PRESERVE_EINVAL;
+    CK(L, cudaMemcpyAsync(dst, src[which], bytes, cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(cuda_stream)));
+    return PRESERVE_OK;
+}
+
+}  // extern "C"

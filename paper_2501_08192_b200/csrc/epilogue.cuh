@@ -1,0 +1,103 @@
+// Row orderings of the packed weights and the fused GEMM epilogues that rely on
+// them.  A skinny GEMM produces, for every batch row b, pairs of outputs
+// (v0, v1) that the epilogue needs together:
+//   PLAIN : two independent outputs;
+//   QKV   : head dims i and i + d/2 of one head (the rotary pair); q goes to the
+//           query buffer, k and v are appended to the cache at slot ctx_len[b];
+//   SWIGLU: gate_j and up_j  ->  silu(gate_j) * up_j.
+// Packed row orders:
+//   GEMV path  : 16-row blocks; rows r and r+8 (r < 8) of block rb are a pair.
+//   tensor path: rows 2m and 2m+1 are a pair.
+#pragma once
+#include "common.cuh"
+#include "kernels.h"
+
+namespace prsv {
+
+// Logical coordinates of pair `pair` (GEMV path: pair = rb * 8 + r; tensor path: pair = m).
+//   PLAIN : n0, n1 = output features of v0, v1
+//   QKV   : n0 = head index over [q | k | v], n1 = i (first dim of the rotary pair)
+//   SWIGLU: n0 = j
+__host__ __device__ inline void pair_coords(int kind, bool tensor_path, int pair, int &n0, int &n1)
+{
+    if (kind == EPI_PLAIN) {
+        if (tensor_path) { n0 = 2 * pair; n1 = 2 * pair + 1; }
+        else { n0 = (pair >> 3) * 16 + (pair & 7); n1 = n0 + 8; }
+    } else if (kind == EPI_QKV) {
+        n0 = pair >> 6;          // 64 pairs per 128-dim head in either path
+        n1 = pair & 63;
+    } else {
+        n0 = pair; n1 = 0;
+    }
+}
+
+// Source matrix and column of packed row p (used by the packers).
+// srcs are [K, cols_s] row-major; QKV: {w_q, w_k, w_v}; SWIGLU: {w_gate, w_up}; PLAIN: {w}.
+__host__ __device__ inline void packed_row_source(int kind, bool tensor_path, int p, const int *src_cols,
+                                                  int &src, int &col)
+{
+    int pair, member;
+    if (tensor_path) { pair = p >> 1; member = p & 1; }
+    else { pair = (p >> 4) * 8 + (p & 7); member = (p >> 3) & 1; }
+    int n0, n1;
+    pair_coords(kind, tensor_path, pair, n0, n1);
+    if (kind == EPI_PLAIN) {
+        src = 0; col = member ? n1 : n0;
+    } else if (kind == EPI_QKV) {
+        int f = n0 * kHeadDim + n1 + member * (kHeadDim / 2);
+        src = 0;
+        while (f >= src_cols[src]) { f -= src_cols[src]; ++src; }
+        col = f;
+    } else {
+        src = member; col = n0;
+    }
+}
+
+__device__ __forceinline__ void store_bf16(void *base, size_t idx, float v)
+{
+    reinterpret_cast<bf16 *>(base)[idx] = __float2bfloat16_rn(v);
+}
+
+// Apply the epilogue to one pair of fp32 results of batch row b.
+__device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, bool tensor_path, int N, int b, int pair,
+                                               float v0, float v1)
+{
+    int n0, n1;
+    pair_coords(e.kind, tensor_path, pair, n0, n1);
+    if (e.kind == EPI_PLAIN) {
+        store_bf16(e.out, (size_t)b * N + n0, v0);
+        store_bf16(e.out, (size_t)b * N + n1, v1);
+        if (e.out2) {
+            store_bf16(e.out2, (size_t)b * N + n0, v0);
+            store_bf16(e.out2, (size_t)b * N + n1, v1);
+        }
+    } else if (e.kind == EPI_SWIGLU) {
+        const float a = v0 / (1.f + __expf(-v0)) * v1;
+        store_bf16(e.out, (size_t)b * (N >> 1) + n0, a);
+    } else {
+        const int hd = n0, i = n1;
+        const int pos = e.ctx_len[b];
+        if (hd < e.nq + e.nkv && e.inv_freq) {
+            double s, c;
+            sincos((double)pos * e.inv_freq[i], &s, &c);
+            const float cf = (float)c, sf = (float)s;
+            const float r0 = v0 * cf - v1 * sf;
+            const float r1 = v1 * cf + v0 * sf;
+            v0 = r0; v1 = r1;
+        }
+        if (hd < e.nq) {
+            const size_t o = ((size_t)b * e.nq + hd) * kHeadDim + i;
+            store_bf16(e.q_out, o, v0);
+            store_bf16(e.q_out, o + kHeadDim / 2, v1);
+        } else {
+            const bool is_k = hd < e.nq + e.nkv;
+            const int kvh = is_k ? hd - e.nq : hd - e.nq - e.nkv;
+            const size_t o = (((size_t)b * e.nkv + kvh) * e.cap + pos) * kHeadDim + i;
+            void *dst = is_k ? e.k_cache : e.v_cache;
+            store_bf16(dst, o, v0);
+            store_bf16(dst, o + kHeadDim / 2, v1);
+        }
+    }
+}
+
+}  // namespace prsv

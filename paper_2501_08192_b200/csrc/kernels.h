@@ -1,0 +1,125 @@
+// Internal launch interface between the layer runtime (api.cu) and the kernels.
+// Every launcher is asynchronous on the given stream and returns the launch's
+// cudaError_t.  No launcher allocates.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace prsv {
+
+// Programmatic dependent launch: when non-zero, every kernel of the main stream is
+// launched with the programmatic-serialization attribute, so its prologue (index
+// setup, first weight loads) may overlap the previous kernel's tail.  Each kernel
+// executes griddepcontrol.wait before it touches anything another kernel wrote.
+extern int g_pdl;
+inline int pdl_attr(cudaLaunchAttribute *at)
+{
+    if (!g_pdl)
+        return 0;
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    return 1;
+}
+
+constexpr int kMaxParts = 16;   // most partial-sum buffers in one window
+constexpr int kHeadDim = 128;
+
+// ---- communication-window stand-in: h = resid + sum_p part_p ; x = RMSNorm(h) * gain
+struct WindowArgs {
+    const void *parts[kMaxParts];  // bf16 [B,H] each
+    int n_parts;
+    const void *resid;             // bf16 [B,H] or fp32 [B,H]
+    int resid_is_f32;
+    const void *gain;              // bf16 [H]
+    float eps;
+    float *h_f32;                  // optional fp32 [B,H]
+    void *h_bf16;                  // optional bf16 [B,H]
+    void *x_bf16;                  // bf16 [B,H]
+    int B, H;
+};
+cudaError_t launch_window(const WindowArgs &a, cudaStream_t s);
+
+// ---- skinny GEMM epilogues (shared by the GEMV and the tcgen05 paths)
+enum Epilogue : int { EPI_PLAIN = 0, EPI_QKV = 1, EPI_SWIGLU = 2 };
+struct EpilogueArgs {
+    int kind;
+    void *out;            // PLAIN: bf16 [B,N]; SWIGLU: bf16 [B,N/2]
+    void *out2;           // PLAIN: optional second copy of the output (bf16 [B,N])
+    // QKV: rows are heads [q | k | v] x head_dim; rotary embedding on q and k, k/v appended
+    void *q_out;          // bf16 [B,nq,d]
+    void *k_cache;        // bf16 [*,nkv,cap,d]
+    void *v_cache;
+    const int *ctx_len;   // device [B]
+    int nq, nkv, cap;
+    const double *inv_freq;  // device [d/2]: theta^(-2i/d); NULL disables the rotary embedding
+};
+
+// Packing kinds: how logical output features map to packed rows.
+//   GEMV path  : 16-row blocks; row r<8 and row r+8 of a block form an epilogue pair.
+//   tensor path: rows 2m and 2m+1 form a pair.
+// PLAIN has no pairing (identity order).  The packers and the epilogues agree through
+// packed_row_to_feature() in pack.cu / epilogue.cuh.
+cudaError_t launch_pack_gemv(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
+                             void *dst, cudaStream_t s);
+cudaError_t launch_pack_rows(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
+                             void *dst, cudaStream_t s);
+
+// ---- split-K GEMV (batch < 16): y[b,n] = sum_k x[b,k] W[n,k]; W in fragment-major tiles
+struct GemvArgs {
+    const void *w;        // packed weights (N*K bf16)
+    const void *x;        // bf16 [b0+B,K]
+    int B, N, K;          // B <= 16 batch rows starting at b0
+    int b0;
+    EpilogueArgs epi;
+};
+cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s);
+
+// ---- tcgen05 skinny GEMM (batch >= 16): W [N,K] K-major through TMA
+struct GemmTcArgs {
+    CUtensorMap w_map;    // dims (K, N), box (64, 128), 128B swizzle
+    CUtensorMap x_map;    // dims (K, max_batch), box (64, NB), 128B swizzle
+    int B, NB, N, K;
+    EpilogueArgs epi;
+    int *status;
+};
+cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s);
+
+// ---- split-KV decode attention + merge
+struct AttnArgs {
+    CUtensorMap k_map;    // dims (d, max_batch*nkv*cap), box (64, 64), 128B swizzle
+    CUtensorMap v_map;
+    const void *q;        // bf16 [B,nq,d]
+    const int *ctx_len;   // device [B]; keys attended = ctx_len[b] + 1
+    int B, nq, nkv, cap;
+    int grid;             // persistent CTAs
+    int tiles_per_item;   // 64-key tiles per work item
+    int max_items;        // capacity of the partial buffers
+    float *part_o;        // fp32 [max_items, G, d]
+    float *part_ml;       // fp32 [max_items, G, 2]
+    void *o_out;          // bf16 [B,nq,d]
+    int *status;
+};
+cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s);
+
+// ---- L2 prefetch (no arithmetic, writes nothing)
+struct PrefetchSeg {
+    const void *base;     // contiguous range, or the K cache when per_seq_tokens != 0
+    const void *base2;    // the V cache when per_seq_tokens != 0
+    uint64_t stride;      // KV: bytes between consecutive (sequence, kv head) runs
+    uint64_t bytes;       // bytes to prefetch from this segment (the planner's figure)
+    int count;            // KV: number of (sequence, kv head) runs
+    int per_seq_tokens;   // != 0: KV segment; run i holds ctx_len[i / ranges_per_seq] live tokens
+    int ranges_per_seq;   // KV heads per sequence
+    int token_bytes;      // bytes per token per run (head_dim * 2)
+};
+struct PrefetchArgs {
+    PrefetchSeg seg[6];
+    int n_segs;
+    const int *ctx_len;
+};
+void set_prefetch_kernel_mode(int mode, uint32_t chunk_bytes);
+cudaError_t launch_prefetch(const PrefetchArgs &a, int ctas, cudaStream_t s, const cudaLaunchAttribute *attrs,
+                            int n_attrs);
+
+}  // namespace prsv

@@ -1,0 +1,85 @@
+// Weight packing, run once at layer creation.  Sources are the caller's
+// [in, out] row-major matrices; destinations are laid out so that the GEMM
+// kernels stream them in address order with perfectly coalesced loads.
+//
+// GEMV path ("fragment-major"): the matrix is cut into tiles of 16 output rows
+// x 32 k; tile (rb, kc) occupies 1 KiB at ((rb * K/32) + kc) * 1024.  Inside a
+// tile lane L = 4g + t owns 32 contiguous bytes: 16 B of row g (k = 8t..8t+7)
+// then 16 B of row g + 8 (same k), which is exactly the A-operand fragment of two
+// m16n8k16 MMAs (up to a permutation of k shared with the activations).
+//
+// Tensor path: plain [N, K] K-major rows (the tcgen05 A operand, fetched by TMA
+// with a 128-byte swizzle).
+#include "epilogue.cuh"
+
+namespace prsv {
+
+struct PackParams {
+    const bf16 *src[3];
+    int cols[3];
+    int n_srcs;
+    int N, K, kind;
+    bf16 *dst;
+};
+
+template <bool TENSOR>
+__global__ void k_pack(const __grid_constant__ PackParams p)
+{
+    // one thread per (k, packed row); packed rows fastest so source reads coalesce
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t total = (size_t)p.N * p.K;
+    if (idx >= total)
+        return;
+    const int row = (int)(idx % p.N);
+    const int k = (int)(idx / p.N);
+    int src, col;
+    packed_row_source(p.kind, TENSOR, row, p.cols, src, col);
+    const bf16 v = p.src[src][(size_t)k * p.cols[src] + col];
+    size_t o;
+    if (TENSOR) {
+        o = (size_t)row * p.K + k;
+    } else {
+        const int rb = row >> 4, r = row & 15, g = r & 7, hi = r >> 3;
+        const int kc = k >> 5, t = (k & 31) >> 3, e = k & 7;
+        o = ((size_t)rb * (p.K >> 5) + kc) * 512 + (size_t)(g * 4 + t) * 16 + hi * 8 + e;
+    }
+    p.dst[o] = v;
+}
+
+static cudaError_t launch_pack(bool tensor, const void *const *srcs, const int *src_cols, int n_srcs, int K,
+                               int kind, void *dst, cudaStream_t s)
+{
+    PackParams p = {};
+    int N = 0;
+    for (int i = 0; i < n_srcs; ++i) {
+        p.src[i] = reinterpret_cast<const bf16 *>(srcs[i]);
+        p.cols[i] = src_cols[i];
+        N += src_cols[i];
+    }
+    p.n_srcs = n_srcs;
+    p.N = N;
+    p.K = K;
+    p.kind = kind;
+    p.dst = reinterpret_cast<bf16 *>(dst);
+    const size_t total = (size_t)N * K;
+    const int threads = 256;
+    const unsigned blocks = (unsigned)((total + threads - 1) / threads);
+    if (tensor)
+        k_pack<true><<<blocks, threads, 0, s>>>(p);
+    else
+        k_pack<false><<<blocks, threads, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pack_gemv(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind, void *dst,
+                             cudaStream_t s)
+{
+    return launch_pack(false, srcs, src_cols, n_srcs, K, kind, dst, s);
+}
+cudaError_t launch_pack_rows(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind, void *dst,
+                             cudaStream_t s)
+{
+    return launch_pack(true, srcs, src_cols, n_srcs, K, kind, dst, s);
+}
+
+}  // namespace prsv

@@ -1,0 +1,131 @@
+// L2 prefetch of weights and KV-cache entries on the side stream (Section 3,
+// "Execution with the proposed method": the read-only operands of the operators
+// that follow a collective are fetched into on-chip cache while the collective
+// runs).  The kernel does no arithmetic and writes nothing: it only issues
+// prefetch hints over the planned byte ranges, in the order the consumer
+// kernels will read them (weights in address order of the packed arena; K then
+// V of each (sequence, kv head) in cache order).  It uses a handful of CTAs so
+// it does not take SMs away from the main stream.
+//
+// Modes:
+//   0  cp.async.bulk.prefetch.L2 : one instruction per `chunk` bytes
+//   1  prefetch.global.L2        : one instruction per 128-byte line
+//   2  plain 128-bit loads whose values are dropped (completion of the kernel
+//      then implies arrival in L2; kept as the control for modes 0 and 1)
+#include "common.cuh"
+#include "kernels.h"
+
+namespace prsv {
+
+constexpr int kPfThreads = 128;
+constexpr int kPfMaxRanges = 1024 + 8;   // 512 (sequence, kv head) runs x {K, V} + weights
+
+struct PfRange { const uint8_t *ptr; uint64_t bytes; };
+
+struct PrefetchParams {
+    PrefetchArgs a;
+    int mode;
+    uint32_t chunk;
+};
+
+__global__ void __launch_bounds__(kPfThreads) k_prefetch_l2(const __grid_constant__ PrefetchParams p)
+{
+    __shared__ PfRange ranges[kPfMaxRanges];
+    __shared__ uint64_t range_first_chunk[kPfMaxRanges + 1];
+    __shared__ int n_ranges_s;
+
+    if (threadIdx.x == 0) {
+        // Flatten the segments into (ptr, bytes) ranges; every CTA builds the same table.
+        int n = 0;
+        uint64_t chunks = 0;
+        for (int si = 0; si < p.a.n_segs; ++si) {
+            const PrefetchSeg &sg = p.a.seg[si];
+            uint64_t left = sg.bytes;                    // budget of this segment
+            if (!sg.per_seq_tokens) {
+                if (left && n < kPfMaxRanges) {
+                    ranges[n].ptr = reinterpret_cast<const uint8_t *>(sg.base);
+                    ranges[n].bytes = left;
+                    range_first_chunk[n] = chunks;
+                    chunks += (left + p.chunk - 1) / p.chunk;
+                    ++n;
+                }
+                continue;
+            }
+            // KV: per (sequence, kv head) stream, K run then V run, each ctx_len * token_bytes long
+            const uint8_t *kb = reinterpret_cast<const uint8_t *>(sg.base);
+            const uint8_t *vb = reinterpret_cast<const uint8_t *>(sg.base2);
+            for (int st = 0; st < sg.count && left; ++st) {
+                const uint64_t live = (uint64_t)p.a.ctx_len[st / sg.ranges_per_seq] * sg.token_bytes;
+                for (int kv = 0; kv < 2 && left; ++kv) {
+                    const uint64_t take = (live < left ? live : left) & ~uint64_t(127);
+                    if (take && n < kPfMaxRanges) {
+                        ranges[n].ptr = (kv ? vb : kb) + (uint64_t)st * sg.stride;
+                        ranges[n].bytes = take;
+                        range_first_chunk[n] = chunks;
+                        chunks += (take + p.chunk - 1) / p.chunk;
+                        ++n;
+                    }
+                    left -= take;
+                    if (take < live)
+                        left = 0;           // budget ran out inside this run: stop here
+                }
+            }
+        }
+        range_first_chunk[n] = chunks;
+        n_ranges_s = n;
+    }
+    __syncthreads();
+    const int n_ranges = n_ranges_s;
+    if (n_ranges == 0)
+        return;
+    const uint64_t total_chunks = range_first_chunk[n_ranges];
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    int r = 0;
+    for (uint64_t c = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; c < total_chunks; c += stride) {
+        while (range_first_chunk[r + 1] <= c)
+            ++r;
+        const uint64_t off = (c - range_first_chunk[r]) * p.chunk;
+        const uint64_t left = ranges[r].bytes - off;
+        const uint32_t n = left < p.chunk ? (uint32_t)left : p.chunk;
+        const uint8_t *ptr = ranges[r].ptr + off;
+        if (p.mode == 0) {
+            bulk_prefetch_l2(ptr, n & ~15u);
+        } else if (p.mode == 1) {
+            for (uint32_t o = 0; o < n; o += 128)
+                line_prefetch_l2(ptr + o);
+        } else {
+            // the loads are volatile asm, so they are issued although their values are dropped;
+            // one 16-byte load per 32-byte sector brings in the whole line
+            for (uint32_t o = 0; o < n; o += 32)
+                (void)ld_stream(ptr + o);
+        }
+    }
+}
+
+static int g_pf_mode = 0;
+static uint32_t g_pf_chunk = 4096;
+
+void set_prefetch_kernel_mode(int mode, uint32_t chunk)
+{
+    g_pf_mode = mode;
+    if (chunk >= 128)
+        g_pf_chunk = chunk & ~127u;
+}
+
+cudaError_t launch_prefetch(const PrefetchArgs &a, int ctas, cudaStream_t s, const cudaLaunchAttribute *attrs,
+                            int n_attrs)
+{
+    PrefetchParams p;
+    p.a = a;
+    p.mode = g_pf_mode;
+    p.chunk = g_pf_chunk;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ctas);
+    cfg.blockDim = dim3(kPfThreads);
+    cfg.stream = s;
+    cfg.attrs = const_cast<cudaLaunchAttribute *>(attrs);
+    cfg.numAttrs = n_attrs;
+    return cudaLaunchKernelEx(&cfg, k_prefetch_l2, p);
+}
+
+}  // namespace prsv

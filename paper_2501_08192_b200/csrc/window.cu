@@ -1,0 +1,146 @@
+// Communication-window stand-in: what the allreduce plus its epilogue would
+// deliver on a tensor-parallel system (Section 2, "Multi-device inference";
+// Section 3, "Vanilla execution"): h = residual + sum of the P partial-sum
+// buffers, then x = RMSNorm(h) * gain.  One CTA per token row; 128-bit
+// coalesced loads; fp32 accumulation in the fixed order residual, part 0..P-1.
+// The kernel is deliberately narrow (B CTAs): during a real allreduce the SMs
+// idle, which is what leaves HBM bandwidth to the prefetch stream.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace prsv {
+
+constexpr int kWinMaxChunks = 2;   // 8-element chunks per thread; H <= 1024 * 8 * 2
+
+struct WindowParams {
+    const uint4 *parts[kMaxParts];
+    int n_parts;
+    const void *resid;
+    const uint4 *gain;
+    float eps;
+    float *h_f32;
+    uint4 *h_bf16;
+    uint4 *x_bf16;
+    int H;
+};
+
+template <bool RESID_F32>
+__global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_constant__ WindowParams p)
+{
+    const int row = blockIdx.x;
+    const int chunks = p.H >> 3;                 // uint4 chunks per row
+    const size_t row_off = (size_t)row * chunks;
+    float v[kWinMaxChunks][8];
+    float ss = 0.f;
+
+    pdl_wait();   // partial sums come from the preceding kernel in the stream
+
+#pragma unroll
+    for (int c = 0; c < kWinMaxChunks; ++c) {
+        const int ch = threadIdx.x + c * blockDim.x;
+        if (ch < chunks) {
+            if (RESID_F32) {
+                const float4 *r = reinterpret_cast<const float4 *>(p.resid) + (row_off + ch) * 2;
+                float4 a = r[0], b = r[1];
+                v[c][0] = a.x; v[c][1] = a.y; v[c][2] = a.z; v[c][3] = a.w;
+                v[c][4] = b.x; v[c][5] = b.y; v[c][6] = b.z; v[c][7] = b.w;
+            } else {
+                uint4 r = ld_stream(reinterpret_cast<const uint4 *>(p.resid) + row_off + ch);
+                v[c][0] = bf_lo(r.x); v[c][1] = bf_hi(r.x); v[c][2] = bf_lo(r.y); v[c][3] = bf_hi(r.y);
+                v[c][4] = bf_lo(r.z); v[c][5] = bf_hi(r.z); v[c][6] = bf_lo(r.w); v[c][7] = bf_hi(r.w);
+            }
+            for (int q = 0; q < p.n_parts; ++q) {
+                uint4 r = ld_stream(p.parts[q] + row_off + ch);
+                v[c][0] += bf_lo(r.x); v[c][1] += bf_hi(r.x); v[c][2] += bf_lo(r.y); v[c][3] += bf_hi(r.y);
+                v[c][4] += bf_lo(r.z); v[c][5] += bf_hi(r.z); v[c][6] += bf_lo(r.w); v[c][7] += bf_hi(r.w);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                ss += v[c][i] * v[c][i];
+        }
+    }
+
+    // block reduction of the sum of squares (fixed tree: bit-stable run to run)
+    __shared__ float warp_sums[32];
+    __shared__ float total;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+        ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0)
+        warp_sums[warp] = ss;
+    __syncthreads();
+    if (warp == 0) {
+        const int nw = (blockDim.x + 31) >> 5;
+        float t = lane < nw ? warp_sums[lane] : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+            t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (lane == 0)
+            total = t;
+    }
+    __syncthreads();
+    const float inv = rsqrtf(total / (float)p.H + p.eps);
+
+    pdl_launch_dependents();
+
+#pragma unroll
+    for (int c = 0; c < kWinMaxChunks; ++c) {
+        const int ch = threadIdx.x + c * blockDim.x;
+        if (ch < chunks) {
+            if (p.h_f32) {
+                float4 *o = reinterpret_cast<float4 *>(p.h_f32) + (row_off + ch) * 2;
+                o[0] = make_float4(v[c][0], v[c][1], v[c][2], v[c][3]);
+                o[1] = make_float4(v[c][4], v[c][5], v[c][6], v[c][7]);
+            }
+            if (p.h_bf16) {
+                uint4 o;
+                o.x = pack_bf16(v[c][0], v[c][1]); o.y = pack_bf16(v[c][2], v[c][3]);
+                o.z = pack_bf16(v[c][4], v[c][5]); o.w = pack_bf16(v[c][6], v[c][7]);
+                p.h_bf16[row_off + ch] = o;
+            }
+            uint4 g = ld_cached(p.gain + ch);
+            uint4 o;
+            o.x = pack_bf16(v[c][0] * inv * bf_lo(g.x), v[c][1] * inv * bf_hi(g.x));
+            o.y = pack_bf16(v[c][2] * inv * bf_lo(g.y), v[c][3] * inv * bf_hi(g.y));
+            o.z = pack_bf16(v[c][4] * inv * bf_lo(g.z), v[c][5] * inv * bf_hi(g.z));
+            o.w = pack_bf16(v[c][6] * inv * bf_lo(g.w), v[c][7] * inv * bf_hi(g.w));
+            p.x_bf16[row_off + ch] = o;
+        }
+    }
+}
+
+cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
+{
+    WindowParams p;
+    for (int i = 0; i < kMaxParts; ++i)
+        p.parts[i] = i < a.n_parts ? reinterpret_cast<const uint4 *>(a.parts[i]) : nullptr;
+    p.n_parts = a.n_parts;
+    p.resid = a.resid;
+    p.gain = reinterpret_cast<const uint4 *>(a.gain);
+    p.eps = a.eps;
+    p.h_f32 = a.h_f32;
+    p.h_bf16 = reinterpret_cast<uint4 *>(a.h_bf16);
+    p.x_bf16 = reinterpret_cast<uint4 *>(a.x_bf16);
+    p.H = a.H;
+    const int chunks = a.H / 8;
+    int threads = (chunks + kWinMaxChunks - 1) / kWinMaxChunks;
+    if (chunks <= 1024)
+        threads = chunks;
+    threads = ((threads + 31) / 32) * 32;
+    if (threads > 1024 || threads * kWinMaxChunks < chunks)
+        return cudaErrorInvalidValue;
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(a.B);
+    cfg.blockDim = dim3(threads);
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    cfg.attrs = at;
+    cfg.numAttrs = pdl_attr(at);
+    if (a.resid_is_f32)
+        return cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<true>, p);
+    return cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<false>, p);
+}
+
+}  // namespace prsv
