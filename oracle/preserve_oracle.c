@@ -31,8 +31,13 @@
  * Precision: inputs are bf16 bit patterns widened exactly to fp32; every
  * intermediate VALUE is stored as fp32 and is never rounded to bf16; every sum
  * (dot products, mean of squares, softmax denominator) is accumulated in
- * double so the result does not depend on summation order.  The new key and
- * value take part in attention unrounded.
+ * double so the result does not depend on summation order.  One rounding is part
+ * of the definition: the KV-cache is a bf16 array, the step writes the new key
+ * and value into it and the self-attention kernel reads the cache (Section 3,
+ * "Execution with the proposed method": the cache is read-only in decode except
+ * for the last entry, which the preceding projections update), so attention
+ * sees the new entry as stored, i.e. rounded to bf16 (nearest even).  k_new and
+ * v_new are reported unrounded.
  *
  * Pins (tests, CPU only): brute-force attention on tiny inputs, softmax rows
  * summing to one, uniform-key and dominant-key special cases, GQA == MHA with
@@ -80,6 +85,19 @@ static inline float bf16f(uint16_t b)
 {
     uint32_t u = (uint32_t)b << 16;
     float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+/* fp32 -> nearest-even bf16, returned widened to fp32 (the value a bf16 cache slot holds) */
+static inline float round_to_bf16(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7fffffffu) > 0x7f800000u)
+        return f;                       /* NaN stays NaN */
+    u += 0x7fffu + ((u >> 16) & 1u);
+    u &= 0xffff0000u;
     memcpy(&f, &u, 4);
     return f;
 }
@@ -248,8 +266,9 @@ int oracle_layer_step(const oracle_cfg_t *c, const uint16_t *w_q, const uint16_t
     float *o = falloc((size_t)B * nq * d), *ap = falloc(BH), *h2 = falloc(BH), *x2 = falloc(BH);
     float *gate = falloc((size_t)B * F), *up = falloc((size_t)B * F), *a = falloc((size_t)B * F);
     float *mp = falloc(BH), *parts2 = falloc((size_t)P * BH);
+    float *kn_c = falloc((size_t)B * nkv * d), *vn_c = falloc((size_t)B * nkv * d);
     int rc = -1;
-    if (!h || !x || !q || !kn || !vn || !o || !ap || !h2 || !x2 || !gate || !up || !a || !mp || !parts2)
+    if (!h || !x || !q || !kn || !vn || !o || !ap || !h2 || !x2 || !gate || !up || !a || !mp || !parts2 || !kn_c || !vn_c)
         goto done;
 
     /* window A: sum of the P partial buffers + residual, then RMSNorm */
@@ -263,8 +282,13 @@ int oracle_layer_step(const oracle_cfg_t *c, const uint16_t *w_q, const uint16_t
         oracle_rope(nq, d, ctx_len[b], c->rope_theta, q + (size_t)b * nq * d);
         oracle_rope(nkv, d, ctx_len[b], c->rope_theta, kn + (size_t)b * nkv * d);
     }
+    /* append: the new entry is stored in the bf16 cache; attention reads it from there */
+    for (size_t i = 0; i < (size_t)B * nkv * d; ++i) {
+        kn_c[i] = round_to_bf16(kn[i]);
+        vn_c[i] = round_to_bf16(vn[i]);
+    }
     /* self-attention over the cached entries plus the new one */
-    oracle_attention(B, nq, nkv, d, cap, ctx_len, q, kn, vn, k_cache, v_cache, o, NULL);
+    oracle_attention(B, nq, nkv, d, cap, ctx_len, q, kn_c, vn_c, k_cache, v_cache, o, NULL);
     /* output projection: this shard's partial sum */
     oracle_matmul(B, nq * d, H, o, w_o, ap);
     /* window B: own partial + the P-1 peers' partials + h, then RMSNorm */
@@ -295,6 +319,6 @@ int oracle_layer_step(const oracle_cfg_t *c, const uint16_t *w_q, const uint16_t
     rc = 0;
 done:
     free(h); free(x); free(q); free(kn); free(vn); free(o); free(ap); free(h2); free(x2);
-    free(gate); free(up); free(a); free(mp); free(parts2);
+    free(gate); free(up); free(a); free(mp); free(parts2); free(kn_c); free(vn_c);
     return rc;
 }

@@ -306,13 +306,14 @@ def torch_layer(shape, t, parts=None, resid=None, peers=None):
         return torch.cat([u1 * ang.cos() - u2 * ang.sin(), u2 * ang.cos() + u1 * ang.sin()], -1)
 
     q, k = rot(q), rot(k)
+    k_st, v_st = k.bfloat16().double(), v.bfloat16().double()     # the new entry as the bf16 cache stores it
     Kc, Vc = W("k_cache").clone(), W("v_cache").clone()
     o = torch.zeros(B, nq, d, dtype=torch.float64)
     G = nq // nkv
     for b in range(B):
         n = int(pos[b])
-        Kb = torch.cat([Kc[b, :, :n], k[b][:, None]], 1).repeat_interleave(G, 0)   # [nq,n+1,d]
-        Vb = torch.cat([Vc[b, :, :n], v[b][:, None]], 1).repeat_interleave(G, 0)
+        Kb = torch.cat([Kc[b, :, :n], k_st[b][:, None]], 1).repeat_interleave(G, 0)   # [nq,n+1,d]
+        Vb = torch.cat([Vc[b, :, :n], v_st[b][:, None]], 1).repeat_interleave(G, 0)
         p = torch.softmax(torch.einsum("hd,hjd->hj", q[b], Kb) / math.sqrt(d), -1)
         o[b] = torch.einsum("hj,hjd->hd", p, Vb)
     ap = o.reshape(B, nq * d) @ W("w_o")
@@ -380,6 +381,19 @@ def test_shard_sum_equals_unsharded_layer(oracle):
     np.testing.assert_allclose(r0["h2"], f["h2"], rtol=1e-5, atol=1e-5)
     np.testing.assert_allclose(r1["h2"], f["h2"], rtol=1e-5, atol=1e-5)
     np.testing.assert_allclose(r0["mlp_partial"] + r1["mlp_partial"], f["mlp_partial"], rtol=1e-4, atol=2e-5)
+
+
+def test_layer_attends_over_the_cache_as_stored(oracle):
+    """The new key/value enter attention as the bf16 cache holds them: the layer's o equals
+    the attention function applied to q and the nearest-even bf16 roundings of k_new, v_new."""
+    shape = I.small_shape(batch=2, ctx=40, seed=22)
+    t = I.make_layers(shape, 1)[0]
+    r = oracle.layer_step(shape, t)
+    kr, vr = widen(bits(r["k_new"])), widen(bits(r["v_new"]))
+    o = oracle.attention(r["q"], kr, vr, t["k_cache"], t["v_cache"], t["ctx_len"])
+    assert np.array_equal(o, r["o"])
+    o_unrounded = oracle.attention(r["q"], r["k_new"], r["v_new"], t["k_cache"], t["v_cache"], t["ctx_len"])
+    assert not np.array_equal(o_unrounded, r["o"])
 
 
 def test_layer_reads_only_live_cache_slots(oracle):
