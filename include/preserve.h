@@ -147,7 +147,9 @@ typedef struct {
     int32_t max_persisting_l2_bytes;  /* cudaDevAttrMaxPersistingL2CacheSize            */
     int32_t max_access_window_bytes;  /* cudaDevAttrMaxAccessPolicyWindowSize           */
     int32_t uses_tensor_path;         /* 1: tcgen05 GEMM (max_batch >= 16); 0: split-K GEMV */
+    int32_t activation_rows;          /* rows per plane of the internal split activations (see preserve_debug_copy) */
     int32_t plan_mode;
+    int32_t reserved;
     uint64_t prefetch_budget;         /* bytes per window                               */
     uint64_t weight_bytes[4];         /* Wqkv, Wo, Wgate|up, Wdown                      */
     uint64_t kv_bytes;                /* K+V bytes read by the last planned step        */
@@ -201,10 +203,12 @@ PRESERVE_API int preserve_last_status(preserve_layer_t *layer);
 PRESERVE_API int preserve_last_cuda_error(const preserve_layer_t *layer);
 
 /* Copy an intermediate of the last step into a caller's device buffer (for
- * kernel-level checks).  which: 0 h (fp32 [batch,hidden]), 1 x, 2 q (after the
- * rotary embedding, [batch,n_q_heads,head_dim]), 3 o (attention output, same
- * shape), 4 x2, 5 a ([batch,ffn]); 1..5 are bf16.  `bytes` must not exceed the
- * intermediate's size.  Asynchronous on `cuda_stream`. */
+ * kernel-level checks).  which: 0 h (fp32 [max_batch,hidden]); 1 x, 2 q (after the
+ * rotary embedding, [.., n_q_heads, head_dim]), 3 o (attention output, same shape),
+ * 4 x2, 5 a ([.., ffn]).  1..5 are kept internally as two bf16 planes, value =
+ * hi + lo, laid out [2][activation_rows][...] (activation_rows from
+ * preserve_layer_get_info); the copy delivers that layout as is.  `bytes` must
+ * not exceed the buffer's size.  Asynchronous on `cuda_stream`. */
 PRESERVE_API int preserve_debug_copy(preserve_layer_t *layer, int32_t which, void *dst_device, size_t bytes,
                         void *cuda_stream);
 

@@ -57,7 +57,8 @@ class HostIO(C.Structure):
 class Info(C.Structure):
     _fields_ = [("sm_count", C.c_int32), ("l2_bytes", C.c_int32), ("max_persisting_l2_bytes", C.c_int32),
                 ("max_access_window_bytes", C.c_int32), ("uses_tensor_path", C.c_int32),
-                ("plan_mode", C.c_int32), ("prefetch_budget", C.c_uint64),
+                ("activation_rows", C.c_int32), ("plan_mode", C.c_int32), ("reserved", C.c_int32),
+                ("prefetch_budget", C.c_uint64),
                 ("weight_bytes", C.c_uint64 * 4), ("kv_bytes", C.c_uint64),
                 ("planned_bytes", (C.c_uint64 * 3) * 2), ("algorithmic_bytes", C.c_uint64)]
 
@@ -147,7 +148,10 @@ class Layer:
     def __init__(self, cfg: LayerConfig, weights: dict):
         """weights: name -> CUDA bf16 tensor ([in,out] row-major) for w_q..w_down, g_attn, g_mlp."""
         self.cfg = cfg
-        w = LayerWeights(*[_ptr(weights[n].contiguous()) for n, _ in LayerWeights._fields_])
+        for n, _ in LayerWeights._fields_:
+            if not weights[n].is_contiguous():
+                raise ValueError(f"weight {n} must be contiguous")
+        w = LayerWeights(*[_ptr(weights[n]) for n, _ in LayerWeights._fields_])
         h = C.c_void_p()
         _check(lib().preserve_layer_init(C.byref(cfg), C.byref(w), C.byref(h)), "preserve_layer_init")
         self.handle = h

@@ -75,7 +75,8 @@ struct preserve_layer {
     double *inv_freq;
 
     float *h_f32;
-    void *x, *q, *o, *attn_partial, *x2, *a;
+    void *x, *q, *o, *attn_partial, *x2, *a;   // x, q, o, x2, a: split bf16 [2][rows][...] (hi + lo)
+    int rows;                                  // batch rows per plane (max_batch, padded to 16 on the tensor path)
     float *part_o, *part_ml;
     int max_items, attn_grid;
     int *status;
@@ -277,6 +278,7 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
         GemmTcArgs a;
         a.w_map = L->wmap[which];
         a.x_map = L->xmap[which];
+        (void)x;
         a.B = B; a.NB = L->nb_pad; a.N = d.n[which]; a.K = d.k[which];
         a.epi = epi;
         a.status = L->status;
@@ -287,6 +289,7 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
         GemvArgs a;
         a.w = L->arena + L->off[which];
         a.x = x;
+        a.x_plane = (size_t)L->rows * d.k[which];
         a.B = B - b0 < 16 ? B - b0 : 16;
         a.b0 = b0;
         a.N = d.n[which]; a.K = d.k[which];
@@ -372,6 +375,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         w.h_f32 = L->h_f32;
         w.h_bf16 = nullptr;
         w.x_bf16 = L->x;
+        w.x_plane_elems = (size_t)L->rows * H;
         w.B = B; w.H = H;
         CK(L, launch_window(w, s));
     }
@@ -380,6 +384,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         EpilogueArgs e = {};
         e.kind = EPI_QKV;
         e.q_out = L->q;
+        e.q_plane = (size_t)L->rows * c.n_q_heads * kHeadDim;
         e.k_cache = sp.k_cache;
         e.v_cache = sp.v_cache;
         e.ctx_len = sp.ctx_len;
@@ -395,6 +400,8 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         a.k_map = L->k_map;
         a.v_map = L->v_map;
         a.q = L->q;
+        a.q_plane = (size_t)L->rows * c.n_q_heads * kHeadDim;
+        a.o_plane = a.q_plane;
         a.ctx_len = sp.ctx_len;
         a.B = B; a.nq = c.n_q_heads; a.nkv = c.n_kv_heads; a.cap = cap;
         a.grid = L->attn_grid;
@@ -446,6 +453,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         w.h_f32 = nullptr;
         w.h_bf16 = sp.residual_out;
         w.x_bf16 = L->x2;
+        w.x_plane_elems = (size_t)L->rows * H;
         w.B = B; w.H = H;
         CK(L, launch_window(w, s));
     }
@@ -454,6 +462,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         EpilogueArgs e = {};
         e.kind = EPI_SWIGLU;
         e.out = L->a;
+        e.out_plane = (size_t)L->rows * c.ffn;
         int rc = launch_gemm(L, 2, L->x2, B, e, s);
         if (rc)
             return rc;
@@ -736,18 +745,23 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
         CKI(cudaMemcpy(L->inv_freq, f, sizeof(f), cudaMemcpyHostToDevice));
     }
     // workspaces
-    const size_t BH = (size_t)B * H, Bq = (size_t)B * c.n_q_heads * c.head_dim;
+    L->nb_pad = ((B + 15) / 16) * 16;
+    L->rows = L->tensor_path ? L->nb_pad : B;
+    const size_t BH = (size_t)B * H;
+    const size_t RH = (size_t)L->rows * H, Rq = (size_t)L->rows * c.n_q_heads * c.head_dim;
+    const size_t RF = (size_t)L->rows * c.ffn;
     CKI(cudaMalloc(&L->h_f32, BH * 4));
-    CKI(cudaMalloc(&L->x, BH * 2));
-    CKI(cudaMalloc(&L->q, Bq * 2));
-    CKI(cudaMalloc(&L->o, Bq * 2));
+    CKI(cudaMalloc(&L->x, 2 * RH * 2));
+    CKI(cudaMalloc(&L->q, 2 * Rq * 2));
+    CKI(cudaMalloc(&L->o, 2 * Rq * 2));
     CKI(cudaMalloc(&L->attn_partial, BH * 2));
-    CKI(cudaMalloc(&L->x2, BH * 2));
-    CKI(cudaMalloc(&L->a, (size_t)B * c.ffn * 2));
-    CKI(cudaMemset(L->x, 0, BH * 2));
-    CKI(cudaMemset(L->o, 0, Bq * 2));
-    CKI(cudaMemset(L->x2, 0, BH * 2));
-    CKI(cudaMemset(L->a, 0, (size_t)B * c.ffn * 2));
+    CKI(cudaMalloc(&L->x2, 2 * RH * 2));
+    CKI(cudaMalloc(&L->a, 2 * RF * 2));
+    CKI(cudaMemset(L->x, 0, 2 * RH * 2));
+    CKI(cudaMemset(L->q, 0, 2 * Rq * 2));
+    CKI(cudaMemset(L->o, 0, 2 * Rq * 2));
+    CKI(cudaMemset(L->x2, 0, 2 * RH * 2));
+    CKI(cudaMemset(L->a, 0, 2 * RF * 2));
     L->attn_grid = L->sm_count;
     L->max_items = L->attn_grid * 4 + B * c.n_kv_heads + 8;
     CKI(cudaMalloc(&L->part_o, (size_t)L->max_items * L->group * kHeadDim * 4));
@@ -760,11 +774,11 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     CKI(cudaMalloc(&L->ctx_dev, (size_t)B * 4));
 
     if (L->tensor_path) {
-        L->nb_pad = ((B + 15) / 16) * 16;
+        // activations as the B operand: [2 * nb_pad, K] = hi rows then lo rows, one box covers both
         const void *xb[4] = {L->x, L->o, L->x2, L->a};
         for (int i = 0; i < 4; ++i) {
             if (!make_map_2d(&L->wmap[i], L->arena + L->off[i], d.k[i], d.n[i], 64, 128) ||
-                !make_map_2d(&L->xmap[i], xb[i], d.k[i], B, 64, L->nb_pad > 256 ? 256 : L->nb_pad)) {
+                !make_map_2d(&L->xmap[i], xb[i], d.k[i], 2 * (uint64_t)L->nb_pad, 64, 2 * L->nb_pad)) {
                 preserve_layer_destroy(L);
                 return PRESERVE_EARCH;
             }
@@ -889,6 +903,7 @@ int preserve_layer_get_info(const preserve_layer_t *L, preserve_info_t *info)
     info->max_persisting_l2_bytes = L->max_persist;
     info->max_access_window_bytes = L->max_window;
     info->uses_tensor_path = L->tensor_path ? 1 : 0;
+    info->activation_rows = L->rows;
     info->plan_mode = L->plan_mode;
     info->prefetch_budget = L->budget;
     for (int i = 0; i < 4; ++i)
@@ -919,9 +934,10 @@ int preserve_debug_copy(preserve_layer_t *L, int32_t which, void *dst, size_t by
     if (!L || !dst)
         return PRESERVE_EINVAL;
     const auto &c = L->cfg;
-    const size_t BH = (size_t)c.max_batch * c.hidden, Bq = (size_t)c.max_batch * c.n_q_heads * c.head_dim;
+    const size_t BH = (size_t)c.max_batch * c.hidden;
+    const size_t RH = (size_t)L->rows * c.hidden, Rq = (size_t)L->rows * c.n_q_heads * c.head_dim;
     const void *src[6] = {L->h_f32, L->x, L->q, L->o, L->x2, L->a};
-    const size_t cap[6] = {BH * 4, BH * 2, Bq * 2, Bq * 2, BH * 2, (size_t)c.max_batch * c.ffn * 2};
+    const size_t cap[6] = {BH * 4, 2 * RH * 2, 2 * Rq * 2, 2 * Rq * 2, 2 * RH * 2, 2 * (size_t)L->rows * c.ffn * 2};
     if (which < 0 || which > 5 || bytes > cap[which])
         return PRESERVE_EINVAL;
     CK(L, cudaMemcpyAsync(dst, src[which], bytes, cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(cuda_stream)));

@@ -34,7 +34,8 @@ constexpr int kMaxStreams = 2048;                      // (sequence, kv head) pa
 struct AttnParams {
     CUtensorMap k_map;
     CUtensorMap v_map;
-    const bf16 *q;
+    const bf16 *q;          // hi plane; lo plane at q + q_plane (q = hi + lo)
+    size_t q_plane;
     const int *ctx_len;
     int B, nq, nkv, G, cap;
     int tiles_per_item;
@@ -42,7 +43,8 @@ struct AttnParams {
     float scale_log2;       // log2(e) / sqrt(d)
     float *part_o;
     float *part_ml;
-    bf16 *o_out;
+    bf16 *o_out;            // hi plane; lo plane at o_out + o_plane
+    size_t o_plane;
     int *status;
 };
 
@@ -149,16 +151,18 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_attn_decode_splitkv(const _
         const int t1 = min(nt, t0 + p.tiles_per_item);
 
         // Q fragments: rows = query heads of the group (zero beyond G)
-        uint32_t qa[8][4];
-        {
-            const bf16 *qb = p.q + ((size_t)b * p.nq + (size_t)kvh * p.G) * kHeadDim;
+        // (both bf16 planes of q: the scores are (q_hi + q_lo) . k)
+        uint32_t qa[2][8][4];
+#pragma unroll
+        for (int pl = 0; pl < 2; ++pl) {
+            const bf16 *qb = p.q + pl * p.q_plane + ((size_t)b * p.nq + (size_t)kvh * p.G) * kHeadDim;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
                 const int d0 = ks * 16 + 2 * t;
-                qa[ks][0] = g < p.G ? *reinterpret_cast<const uint32_t *>(qb + g * kHeadDim + d0) : 0u;
-                qa[ks][1] = g + 8 < p.G ? *reinterpret_cast<const uint32_t *>(qb + (g + 8) * kHeadDim + d0) : 0u;
-                qa[ks][2] = g < p.G ? *reinterpret_cast<const uint32_t *>(qb + g * kHeadDim + d0 + 8) : 0u;
-                qa[ks][3] = g + 8 < p.G ? *reinterpret_cast<const uint32_t *>(qb + (g + 8) * kHeadDim + d0 + 8) : 0u;
+                qa[pl][ks][0] = g < p.G ? *reinterpret_cast<const uint32_t *>(qb + g * kHeadDim + d0) : 0u;
+                qa[pl][ks][1] = g + 8 < p.G ? *reinterpret_cast<const uint32_t *>(qb + (g + 8) * kHeadDim + d0) : 0u;
+                qa[pl][ks][2] = g < p.G ? *reinterpret_cast<const uint32_t *>(qb + g * kHeadDim + d0 + 8) : 0u;
+                qa[pl][ks][3] = g + 8 < p.G ? *reinterpret_cast<const uint32_t *>(qb + (g + 8) * kHeadDim + d0 + 8) : 0u;
             }
         }
         float o[16][4];
@@ -206,8 +210,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_attn_decode_splitkv(const _
                     const uint32_t addr = rowaddr + (ks >> 2) * kHalfBytes + ((chunk16 ^ (key & 7)) << 4);
                     uint32_t r[4];
                     ldmatrix_x4(r, addr);
-                    mma_bf16_16816(s[0], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], r[0], r[1]);
-                    mma_bf16_16816(s[1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], r[2], r[3]);
+#pragma unroll
+                    for (int pl = 0; pl < 2; ++pl) {
+                        mma_bf16_16816(s[0], qa[pl][ks][0], qa[pl][ks][1], qa[pl][ks][2], qa[pl][ks][3], r[0], r[1]);
+                        mma_bf16_16816(s[1], qa[pl][ks][0], qa[pl][ks][1], qa[pl][ks][2], qa[pl][ks][3], r[2], r[3]);
+                    }
                 }
             }
             // scale, mask, online softmax (rows g and g + 8)
@@ -231,7 +238,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_attn_decode_splitkv(const _
                 m_run[r] = m_new;
                 l_run[r] *= corr[r];
             }
-            uint32_t pa[4];
+            uint32_t pa[4], pb[4];      // P as hi + lo bf16 planes
             {
                 float pv[2][4];
 #pragma unroll
@@ -242,10 +249,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_attn_decode_splitkv(const _
                         pv[i][j] = m == -INFINITY ? 0.f : exp2f(s[i][j] - m);
                         l_run[j >> 1] += pv[i][j];
                     }
-                pa[0] = pack_bf16(pv[0][0], pv[0][1]);
-                pa[1] = pack_bf16(pv[0][2], pv[0][3]);
-                pa[2] = pack_bf16(pv[1][0], pv[1][1]);
-                pa[3] = pack_bf16(pv[1][2], pv[1][3]);
+                split_bf16x2(pv[0][0], pv[0][1], pa[0], pb[0]);
+                split_bf16x2(pv[0][2], pv[0][3], pa[1], pb[1]);
+                split_bf16x2(pv[1][0], pv[1][1], pa[2], pb[2]);
+                split_bf16x2(pv[1][2], pv[1][3], pa[3], pb[3]);
             }
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
@@ -265,6 +272,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_attn_decode_splitkv(const _
                     ldmatrix_x4_trans(r, addr);
                     mma_bf16_16816(o[c], pa[0], pa[1], pa[2], pa[3], r[0], r[1]);
                     mma_bf16_16816(o[c + 1], pa[0], pa[1], pa[2], pa[3], r[2], r[3]);
+                    mma_bf16_16816(o[c], pb[0], pb[1], pb[2], pb[3], r[0], r[1]);
+                    mma_bf16_16816(o[c + 1], pb[0], pb[1], pb[2], pb[3], r[2], r[3]);
                 }
             }
             __syncwarp();
@@ -357,7 +366,11 @@ __global__ void __launch_bounds__(kHeadDim) k_attn_merge(const __grid_constant__
         acc += p.part_o[idx * kHeadDim + d] * w;
     }
     pdl_launch_dependents();
-    p.o_out[((size_t)b * p.nq + hq) * kHeadDim + d] = __float2bfloat16_rn(acc / L);
+    const float ov = acc / L;
+    const bf16 hi = __float2bfloat16_rn(ov);
+    const size_t oi = ((size_t)b * p.nq + hq) * kHeadDim + d;
+    p.o_out[oi] = hi;
+    p.o_out[p.o_plane + oi] = __float2bfloat16_rn(ov - __bfloat162float(hi));
 }
 
 cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
@@ -368,6 +381,8 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     p.k_map = a.k_map;
     p.v_map = a.v_map;
     p.q = reinterpret_cast<const bf16 *>(a.q);
+    p.q_plane = a.q_plane;
+    p.o_plane = a.o_plane;
     p.ctx_len = a.ctx_len;
     p.B = a.B; p.nq = a.nq; p.nkv = a.nkv; p.G = a.nq / a.nkv; p.cap = a.cap;
     p.tiles_per_item = a.tiles_per_item;

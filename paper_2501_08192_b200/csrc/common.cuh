@@ -25,6 +25,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&t);
 }
+// Split two fp32 values into bf16 hi and lo parts, v = hi + lo up to ~2^-17 relative.
+__device__ __forceinline__ void split_bf16x2(float a, float b, uint32_t &hi, uint32_t &lo)
+{
+    hi = pack_bf16(a, b);
+    lo = pack_bf16(a - bf_lo(hi), b - bf_hi(hi));
+}
 __device__ __forceinline__ uint16_t f2bf_bits(float v)
 {
     bf16 t = __float2bfloat16_rn(v);

@@ -57,6 +57,13 @@ __device__ __forceinline__ void store_bf16(void *base, size_t idx, float v)
 {
     reinterpret_cast<bf16 *>(base)[idx] = __float2bfloat16_rn(v);
 }
+// Activations that feed another GEMM are kept as hi + lo bf16 planes.
+__device__ __forceinline__ void store_split(void *base, size_t plane, size_t idx, float v)
+{
+    const bf16 hi = __float2bfloat16_rn(v);
+    reinterpret_cast<bf16 *>(base)[idx] = hi;
+    reinterpret_cast<bf16 *>(base)[plane + idx] = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
 
 // Apply the epilogue to one pair of fp32 results of batch row b.
 __device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, bool tensor_path, int N, int b, int pair,
@@ -72,8 +79,8 @@ __device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, bool tenso
             store_bf16(e.out2, (size_t)b * N + n1, v1);
         }
     } else if (e.kind == EPI_SWIGLU) {
-        const float a = v0 / (1.f + __expf(-v0)) * v1;
-        store_bf16(e.out, (size_t)b * (N >> 1) + n0, a);
+        const float a = v0 / (1.f + expf(-v0)) * v1;
+        store_split(e.out, e.out_plane, (size_t)b * (N >> 1) + n0, a);
     } else {
         const int hd = n0, i = n1;
         const int pos = e.ctx_len[b];
@@ -87,8 +94,8 @@ __device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, bool tenso
         }
         if (hd < e.nq) {
             const size_t o = ((size_t)b * e.nq + hd) * kHeadDim + i;
-            store_bf16(e.q_out, o, v0);
-            store_bf16(e.q_out, o + kHeadDim / 2, v1);
+            store_split(e.q_out, e.q_plane, o, v0);
+            store_split(e.q_out, e.q_plane, o + kHeadDim / 2, v1);
         } else {
             const bool is_k = hd < e.nq + e.nkv;
             const int kvh = is_k ? hd - e.nq : hd - e.nq - e.nkv;

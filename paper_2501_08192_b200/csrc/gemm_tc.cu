@@ -1,5 +1,306 @@
-// placeholder until the tcgen05 kernel lands
-#include "kernels.h"
+// Skinny GEMM on the 5th-generation tensor cores for decode batches >= 16:
+//     y[b, n] = sum_k x[b, k] * W[n, k]
+// computed "swapped": the weight tile is the M = 128 operand, the batch (padded
+// to a multiple of 16, and present twice: the hi and the lo bf16 plane of the
+// activations, x = hi + lo) is the N operand, so one tcgen05.mma per 16 k covers a
+// 128 x 16-k slab of weights for every batch row at once and the CUDA cores stay
+// out of the weight stream entirely.
+//
+// Per CTA: one 128-row tile of the packed weights x one slice of k.
+//   warp 0    : TMA producer - W tile (128 x 64, 128B swizzle) and x tile (NB x 64)
+//               into a multi-stage shared-memory ring, mbarrier full/empty
+//   warp 1    : allocates TMEM, issues tcgen05.mma (kind::f16, bf16 in, fp32
+//               accumulate in TMEM), tcgen05.commit frees ring slots
+//   warps 2-5 : epilogue - tcgen05.ld the accumulator (lane = output row), split-K
+//               reduction through distributed shared memory of the cluster in rank
+//               order, fused epilogue (epilogue.cuh)
+// Every mbarrier wait is bounded; a wait that gives up records a status code,
+// poisons the rest of the CTA's work, and the CTA still reaches every barrier
+// and frees its TMEM.
+#include <cooperative_groups.h>
+
+#include "epilogue.cuh"
+
+namespace cg = cooperative_groups;
+
 namespace prsv {
-cudaError_t launch_gemm_tc(const GemmTcArgs &, int, cudaStream_t) { return cudaErrorNotSupported; }
+
+constexpr int kTcMaxStages = 8;
+constexpr int kTcThreads = 192;
+constexpr int kTcBlockK = 64;
+constexpr int kTcTileM = 128;
+constexpr int kATileBytes = kTcTileM * kTcBlockK * 2;   // 16 KiB
+
+struct GemmTcParams {
+    CUtensorMap w_map;
+    CUtensorMap x_map;
+    int B, NB, N, K;
+    int kblocks;        // K / 64
+    int splits;         // cluster size along k
+    int stages;
+    int tmem_cols;
+    uint32_t idesc;
+    EpilogueArgs epi;
+    int *status;
+};
+
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr)
+{
+    // K-major operand, 128-byte swizzle: 8-row atoms of 1024 B (stride-byte-offset 1024),
+    // descriptor version 1, layout type 2 (SWIZZLE_128B)
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
+
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+                 "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16])
+{
+    uint32_t r[16];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+                   "=r"(r[15])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i)
+        v[i] = __uint_as_float(r[i]);
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_constant__ GemmTcParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ uint64_t full[kTcMaxStages], empty[kTcMaxStages], accum_bar;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ volatile int poisoned;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tile = blockIdx.x;
+    const int s = blockIdx.y;
+    const int stage_bytes = kATileBytes + 2 * p.NB * kTcBlockK * 2;
+    const int kb0 = (int)((long long)p.kblocks * s / p.splits);
+    const int kb1 = (int)((long long)p.kblocks * (s + 1) / p.splits);
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < p.stages; ++i) {
+            mbar_init(&full[i], 1);
+            mbar_init(&empty[i], 1);
+        }
+        mbar_init(&accum_bar, 1);
+        mbar_fence_init();
+        poisoned = 0;
+        tma_prefetch_desc(&p.w_map);
+        tma_prefetch_desc(&p.x_map);
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)),
+                     "r"((uint32_t)p.tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                const int st = it % p.stages;
+                const uint32_t ph = (it / p.stages) & 1;
+                if (!mbar_wait(&empty[st], ph ^ 1, p.status, ST_TIMEOUT_EMPTY)) { poisoned = 1; break; }
+                uint8_t *a_dst = smem + (size_t)st * stage_bytes;
+                mbar_expect_tx(&full[st], stage_bytes);
+                tma_load_2d(a_dst, &p.w_map, kb * kTcBlockK, tile * kTcTileM, &full[st]);
+                if (kb == kb0)
+                    pdl_wait();     // weights never depend on earlier kernels; the activations do
+                tma_load_2d(a_dst + kATileBytes, &p.x_map, kb * kTcBlockK, 0, &full[st]);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                const int st = it % p.stages;
+                const uint32_t ph = (it / p.stages) & 1;
+                if (!mbar_wait(&full[st], ph, p.status, ST_TIMEOUT_FULL)) { poisoned = 1; ok = false; break; }
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(smem + (size_t)st * stage_bytes);
+                const uint64_t adesc = make_smem_desc(a_addr);
+                const uint64_t bdesc = make_smem_desc(a_addr + kATileBytes);
+#pragma unroll
+                for (int k = 0; k < kTcBlockK / 16; ++k)
+                    tc_mma(tmem_base, adesc + 2 * k, bdesc + 2 * k, p.idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+                tc_commit(&empty[st]);      // slot is free once these MMAs have read it
+            }
+            if (ok)
+                tc_commit(&accum_bar);      // accumulator complete
+        }
+    }
+    __syncwarp();
+
+    // ---------------------------------------------------------------- epilogue
+    // Accumulator column b holds the hi-plane product of batch row b, column NB + b the
+    // lo-plane product; their sum is the result.  Handled 16 batch rows at a time.
+    const int lane_grp = warp & 3;          // TMEM lanes this warp may read: 32 * (warp % 4)
+    const int row = lane_grp * 32 + lane;   // row of the tile
+    const int nchunks = p.NB / 16;
+    bool have = false;
+    if (warp >= 2) {
+        have = mbar_wait(&accum_bar, 0, p.status, ST_TIMEOUT_MMA);
+        if (!have)
+            poisoned = 1;
+        tc_fence_after();
+    }
+    pdl_launch_dependents();
+    const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
+    float *red = reinterpret_cast<float *>(smem);      // [NB][128] fp32, reuses the ring
+
+    auto load_chunk = [&](int c, float (&v)[16]) {
+        if (have) {
+            float lo[16];
+            tc_ld16(t_lane + c * 16, v);
+            tc_ld16(t_lane + p.NB + c * 16, lo);
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                v[i] += lo[i];
+        } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                v[i] = 0.f;
+        }
+    };
+
+    if (p.splits > 1) {
+        cg::cluster_group cluster = cg::this_cluster();
+        if (warp >= 2 && s > 0) {
+            for (int c = 0; c < nchunks; ++c) {
+                float v[16];
+                load_chunk(c, v);
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    red[(c * 16 + i) * kTcTileM + row] = v[i];
+            }
+        }
+        cluster.sync();
+    }
+    if (warp >= 2 && s == 0) {
+        const int pair = (tile * kTcTileM + row) >> 1;
+        const int par = lane & 1;
+        for (int c = 0; c < nchunks; ++c) {
+            float v[16];
+            load_chunk(c, v);
+            if (p.splits > 1) {
+                cg::cluster_group cluster = cg::this_cluster();
+                for (int q = 1; q < p.splits; ++q) {
+                    const float *remote = cluster.map_shared_rank(red, q);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        v[i] += remote[(c * 16 + i) * kTcTileM + row];
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float mine = v[i];
+                const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
+                const int b = c * 16 + i;
+                if ((i & 1) == par && b < p.B && !poisoned)
+                    apply_epilogue(p.epi, true, p.N, b, pair, par ? other : mine, par ? mine : other);
+            }
+        }
+    }
+    if (p.splits > 1) {
+        cg::cluster_group cluster = cg::this_cluster();
+        cluster.sync();        // peers' shared memory must outlive rank 0's reads
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols)
+                     : "memory");
+    }
+}
+
+static int pow2_floor_i(int v)
+{
+    int r = 1;
+    while (r * 2 <= v)
+        r *= 2;
+    return r;
+}
+
+cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
+{
+    if (a.NB < 16 || a.NB > 128 || a.NB % 16 || a.N % kTcTileM || a.K % kTcBlockK || a.B > a.NB)
+        return cudaErrorInvalidValue;
+    GemmTcParams p;
+    p.w_map = a.w_map;
+    p.x_map = a.x_map;
+    p.B = a.B; p.NB = a.NB; p.N = a.N; p.K = a.K;
+    p.kblocks = a.K / kTcBlockK;
+    p.epi = a.epi;
+    p.status = a.status;
+    const int tiles = a.N / kTcTileM;
+    int splits = pow2_floor_i((2 * sm_count) / tiles > 0 ? (2 * sm_count) / tiles : 1);
+    if (splits > 8) splits = 8;
+    while (splits > 1 && p.kblocks / splits < 2) splits /= 2;
+    p.splits = splits;
+    const int stage_bytes = kATileBytes + 2 * a.NB * kTcBlockK * 2;
+    int stages = (200 * 1024) / stage_bytes;
+    if (stages > kTcMaxStages) stages = kTcMaxStages;
+    // two CTAs per SM when the ring is small enough, so one CTA's ramp-up overlaps another's stream
+    if (stages * stage_bytes > 100 * 1024 && (100 * 1024) / stage_bytes >= 4)
+        stages = (100 * 1024) / stage_bytes;
+    p.stages = stages;
+    int cols = 32;
+    while (cols < 2 * a.NB) cols *= 2;
+    p.tmem_cols = cols;
+    p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * a.NB) >> 3) << 17) | ((uint32_t)(kTcTileM >> 4) << 24);
+
+    size_t smem = (size_t)stages * stage_bytes + 1024;
+    const size_t red_bytes = (size_t)a.NB * kTcTileM * 4 + 1024;
+    if (smem < red_bytes) smem = red_bytes;
+    static size_t attr_smem = 0;
+    if (smem > attr_smem) {
+        cudaError_t e = cudaFuncSetAttribute(k_gemm_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess)
+            return e;
+        attr_smem = smem;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(tiles, splits, 1);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[2];
+    int n = pdl_attr(at);
+    if (splits > 1) {
+        at[n].id = cudaLaunchAttributeClusterDimension;
+        at[n].val.clusterDim.x = 1;
+        at[n].val.clusterDim.y = splits;
+        at[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = at;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, k_gemm_tcgen05, p);
+}
+
+}  // namespace prsv

@@ -29,7 +29,8 @@ constexpr int kGemvUnroll = 4;
 
 struct GemvParams {
     const uint4 *w;
-    const uint4 *x;
+    const uint4 *x;      // hi plane; lo plane at x + x_plane
+    size_t x_plane;      // in uint4 units
     int B, N, K;
     int b0;              // first batch row handled by this launch (x, outputs and ctx_len are indexed b0 + b)
     int row_blocks;      // N / 16
@@ -42,7 +43,8 @@ struct GemvParams {
 template <int NB, bool MMA>
 __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_constant__ GemvParams p)
 {
-    constexpr int NT = MMA ? NB / 8 : 1;
+    constexpr int NTB = MMA ? NB / 8 : 1;   // n-tiles that cover the batch
+    constexpr int NT = 2 * NTB;             // hi planes then lo planes of the activations
     __shared__ float red[kGemvWarps][16][NB];      // per-warp partials
     __shared__ float cta_part[kGemvWarps][16][NB];  // per-row-block CTA partials (read by cluster rank 0)
 
@@ -74,7 +76,7 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
     pdl_wait();   // x is produced by the previous kernel of the stream
 
     if (active) {
-        auto compute = [&](const uint4 &wl, const uint4 &wh, const uint4 (&xq)[MMA ? NT : NB]) {
+        auto compute = [&](const uint4 &wl, const uint4 &wh, const uint4 (&xq)[MMA ? NT : 2 * NB]) {
             if constexpr (MMA) {
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
@@ -88,8 +90,11 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
                 const float h4 = bf_lo(wh.z), h5 = bf_hi(wh.z), h6 = bf_lo(wh.w), h7 = bf_hi(wh.w);
 #pragma unroll
                 for (int b = 0; b < NB; ++b) {
-                    const float x0 = bf_lo(xq[b].x), x1 = bf_hi(xq[b].x), x2 = bf_lo(xq[b].y), x3 = bf_hi(xq[b].y);
-                    const float x4 = bf_lo(xq[b].z), x5 = bf_hi(xq[b].z), x6 = bf_lo(xq[b].w), x7 = bf_hi(xq[b].w);
+                    const uint4 &xh = xq[b], &xl = xq[NB + b];     // x = hi + lo, exact in fp32
+                    const float x0 = bf_lo(xh.x) + bf_lo(xl.x), x1 = bf_hi(xh.x) + bf_hi(xl.x);
+                    const float x2 = bf_lo(xh.y) + bf_lo(xl.y), x3 = bf_hi(xh.y) + bf_hi(xl.y);
+                    const float x4 = bf_lo(xh.z) + bf_lo(xl.z), x5 = bf_hi(xh.z) + bf_hi(xl.z);
+                    const float x6 = bf_lo(xh.w) + bf_lo(xl.w), x7 = bf_hi(xh.w) + bf_hi(xl.w);
                     float a = acc[2 * b][0], c = acc[2 * b + 1][0];
                     a = fmaf(l0, x0, a); a = fmaf(l1, x1, a); a = fmaf(l2, x2, a); a = fmaf(l3, x3, a);
                     a = fmaf(l4, x4, a); a = fmaf(l5, x5, a); a = fmaf(l6, x6, a); a = fmaf(l7, x7, a);
@@ -99,24 +104,28 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
                 }
             }
         };
-        auto load_x = [&](int c, uint4 (&xq)[MMA ? NT : NB]) {
+        auto load_x = [&](int c, uint4 (&xq)[MMA ? NT : 2 * NB]) {
             if constexpr (MMA) {
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
-                    const int b = nt * 8 + g;
-                    xq[nt] = b < p.B ? ld_cached(p.x + (size_t)(p.b0 + b) * xrow + c * 4 + t) : make_uint4(0, 0, 0, 0);
+                    const int b = (nt % NTB) * 8 + g;
+                    const uint4 *plane = p.x + (nt >= NTB ? p.x_plane : 0);
+                    xq[nt] = b < p.B ? ld_cached(plane + (size_t)(p.b0 + b) * xrow + c * 4 + t) : make_uint4(0, 0, 0, 0);
                 }
             } else {
 #pragma unroll
-                for (int b = 0; b < NB; ++b)
+                for (int b = 0; b < NB; ++b) {
                     xq[b] = b < p.B ? ld_cached(p.x + (size_t)(p.b0 + b) * xrow + c * 4 + t) : make_uint4(0, 0, 0, 0);
+                    xq[NB + b] = b < p.B ? ld_cached(p.x + p.x_plane + (size_t)(p.b0 + b) * xrow + c * 4 + t)
+                                         : make_uint4(0, 0, 0, 0);
+                }
             }
         };
 
         int c = c_begin;
         for (; c + kGemvUnroll <= c_end; c += kGemvUnroll) {
             uint4 wl[kGemvUnroll], wh[kGemvUnroll];
-            uint4 xq[kGemvUnroll][MMA ? NT : NB];
+            uint4 xq[kGemvUnroll][MMA ? NT : 2 * NB];
 #pragma unroll
             for (int u = 0; u < kGemvUnroll; ++u) {
                 wl[u] = ld_stream(wp + (size_t)(c + u) * 64);
@@ -130,7 +139,7 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
                 compute(wl[u], wh[u], xq[u]);
         }
         for (; c < c_end; ++c) {
-            uint4 xq[MMA ? NT : NB];
+            uint4 xq[MMA ? NT : 2 * NB];
             const uint4 wl = ld_stream(wp + (size_t)c * 64);
             const uint4 wh = ld_stream(wp + (size_t)c * 64 + 1);
             load_x(c, xq);
@@ -143,11 +152,11 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
     // ---- warp partial -> shared memory: red[warp][row][b]
     if constexpr (MMA) {
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            red[warp][g][nt * 8 + 2 * t] = acc[nt][0];
-            red[warp][g][nt * 8 + 2 * t + 1] = acc[nt][1];
-            red[warp][g + 8][nt * 8 + 2 * t] = acc[nt][2];
-            red[warp][g + 8][nt * 8 + 2 * t + 1] = acc[nt][3];
+        for (int nt = 0; nt < NTB; ++nt) {
+            red[warp][g][nt * 8 + 2 * t] = acc[nt][0] + acc[NTB + nt][0];
+            red[warp][g][nt * 8 + 2 * t + 1] = acc[nt][1] + acc[NTB + nt][1];
+            red[warp][g + 8][nt * 8 + 2 * t] = acc[nt][2] + acc[NTB + nt][2];
+            red[warp][g + 8][nt * 8 + 2 * t + 1] = acc[nt][3] + acc[NTB + nt][3];
         }
     } else {
 #pragma unroll
@@ -238,6 +247,7 @@ cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s)
     GemvParams p;
     p.w = reinterpret_cast<const uint4 *>(a.w);
     p.x = reinterpret_cast<const uint4 *>(a.x);
+    p.x_plane = a.x_plane / 8;
     p.B = a.B; p.N = a.N; p.K = a.K; p.b0 = a.b0;
     p.row_blocks = a.N / 16;
     p.kchunks = a.K / 32;

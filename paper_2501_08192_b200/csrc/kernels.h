@@ -35,7 +35,8 @@ struct WindowArgs {
     float eps;
     float *h_f32;                  // optional fp32 [B,H]
     void *h_bf16;                  // optional bf16 [B,H]
-    void *x_bf16;                  // bf16 [B,H]
+    void *x_bf16;                  // bf16 [2][rows][H]: hi plane then lo plane (x = hi + lo)
+    size_t x_plane_elems;          // elements between the planes
     int B, H;
 };
 cudaError_t launch_window(const WindowArgs &a, cudaStream_t s);
@@ -44,10 +45,12 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s);
 enum Epilogue : int { EPI_PLAIN = 0, EPI_QKV = 1, EPI_SWIGLU = 2 };
 struct EpilogueArgs {
     int kind;
-    void *out;            // PLAIN: bf16 [B,N]; SWIGLU: bf16 [B,N/2]
+    void *out;            // PLAIN: bf16 [B,N]; SWIGLU: split bf16 [2][rows][N/2]
+    size_t out_plane;     // SWIGLU: elements between the hi and lo planes of out
     void *out2;           // PLAIN: optional second copy of the output (bf16 [B,N])
     // QKV: rows are heads [q | k | v] x head_dim; rotary embedding on q and k, k/v appended
-    void *q_out;          // bf16 [B,nq,d]
+    void *q_out;          // split bf16 [2][rows][nq,d]
+    size_t q_plane;       // elements between the hi and lo planes of q_out
     void *k_cache;        // bf16 [*,nkv,cap,d]
     void *v_cache;
     const int *ctx_len;   // device [B]
@@ -68,7 +71,8 @@ cudaError_t launch_pack_rows(const void *const *srcs, const int *src_cols, int n
 // ---- split-K GEMV (batch < 16): y[b,n] = sum_k x[b,k] W[n,k]; W in fragment-major tiles
 struct GemvArgs {
     const void *w;        // packed weights (N*K bf16)
-    const void *x;        // bf16 [b0+B,K]
+    const void *x;        // split bf16 [2][rows][K]
+    size_t x_plane;       // elements between the hi and lo planes
     int B, N, K;          // B <= 16 batch rows starting at b0
     int b0;
     EpilogueArgs epi;
@@ -78,8 +82,8 @@ cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s);
 // ---- tcgen05 skinny GEMM (batch >= 16): W [N,K] K-major through TMA
 struct GemmTcArgs {
     CUtensorMap w_map;    // dims (K, N), box (64, 128), 128B swizzle
-    CUtensorMap x_map;    // dims (K, max_batch), box (64, NB), 128B swizzle
-    int B, NB, N, K;
+    CUtensorMap x_map;    // dims (K, 2*NB): hi rows then lo rows; box (64, 2*NB), 128B swizzle
+    int B, NB, N, K;      // NB = batch rows per plane (multiple of 16)
     EpilogueArgs epi;
     int *status;
 };
@@ -89,7 +93,8 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s);
 struct AttnArgs {
     CUtensorMap k_map;    // dims (d, max_batch*nkv*cap), box (64, 64), 128B swizzle
     CUtensorMap v_map;
-    const void *q;        // bf16 [B,nq,d]
+    const void *q;        // split bf16 [2][rows][nq,d]
+    size_t q_plane;
     const int *ctx_len;   // device [B]; keys attended = ctx_len[b] + 1
     int B, nq, nkv, cap;
     int grid;             // persistent CTAs
@@ -97,7 +102,8 @@ struct AttnArgs {
     int max_items;        // capacity of the partial buffers
     float *part_o;        // fp32 [max_items, G, d]
     float *part_ml;       // fp32 [max_items, G, 2]
-    void *o_out;          // bf16 [B,nq,d]
+    void *o_out;          // split bf16 [2][rows][nq,d]
+    size_t o_plane;
     int *status;
 };
 cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s);

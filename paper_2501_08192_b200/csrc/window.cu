@@ -20,7 +20,8 @@ struct WindowParams {
     float eps;
     float *h_f32;
     uint4 *h_bf16;
-    uint4 *x_bf16;
+    uint4 *x_bf16;       // hi plane; the lo plane follows at x_plane uint4s
+    size_t x_plane;
     int H;
 };
 
@@ -99,13 +100,21 @@ __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_con
                 o.z = pack_bf16(v[c][4], v[c][5]); o.w = pack_bf16(v[c][6], v[c][7]);
                 p.h_bf16[row_off + ch] = o;
             }
+            // x is kept as a pair of bf16 planes, x = hi + lo, so the GEMM that consumes it
+            // sees ~16 mantissa bits although its operands are bf16
             uint4 g = ld_cached(p.gain + ch);
-            uint4 o;
-            o.x = pack_bf16(v[c][0] * inv * bf_lo(g.x), v[c][1] * inv * bf_hi(g.x));
-            o.y = pack_bf16(v[c][2] * inv * bf_lo(g.y), v[c][3] * inv * bf_hi(g.y));
-            o.z = pack_bf16(v[c][4] * inv * bf_lo(g.z), v[c][5] * inv * bf_hi(g.z));
-            o.w = pack_bf16(v[c][6] * inv * bf_lo(g.w), v[c][7] * inv * bf_hi(g.w));
-            p.x_bf16[row_off + ch] = o;
+            float xv[8];
+            xv[0] = v[c][0] * inv * bf_lo(g.x); xv[1] = v[c][1] * inv * bf_hi(g.x);
+            xv[2] = v[c][2] * inv * bf_lo(g.y); xv[3] = v[c][3] * inv * bf_hi(g.y);
+            xv[4] = v[c][4] * inv * bf_lo(g.z); xv[5] = v[c][5] * inv * bf_hi(g.z);
+            xv[6] = v[c][6] * inv * bf_lo(g.w); xv[7] = v[c][7] * inv * bf_hi(g.w);
+            uint4 hi, lo;
+            split_bf16x2(xv[0], xv[1], hi.x, lo.x);
+            split_bf16x2(xv[2], xv[3], hi.y, lo.y);
+            split_bf16x2(xv[4], xv[5], hi.z, lo.z);
+            split_bf16x2(xv[6], xv[7], hi.w, lo.w);
+            p.x_bf16[row_off + ch] = hi;
+            p.x_bf16[p.x_plane + row_off + ch] = lo;
         }
     }
 }
@@ -122,6 +131,7 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
     p.h_f32 = a.h_f32;
     p.h_bf16 = reinterpret_cast<uint4 *>(a.h_bf16);
     p.x_bf16 = reinterpret_cast<uint4 *>(a.x_bf16);
+    p.x_plane = a.x_plane_elems / 8;
     p.H = a.H;
     const int chunks = a.H / 8;
     int threads = (chunks + kWinMaxChunks - 1) / kWinMaxChunks;

@@ -86,18 +86,21 @@ class DeviceLayer:
                 "attn_partial": cuda_to_bits(self.attn_out.t)}
 
     def intermediates(self) -> Dict[str, np.ndarray]:
+        """h, x, q, o, x2, a of the last step as fp32 (split activations are summed hi + lo)."""
         s = self.shape
         B, H, nq, d, F = s.batch, s.hidden, s.n_q_heads, s.head_dim, s.ffn
-        mb = self.cfg.max_batch
-        spec = {"h": (0, (mb, H), torch.float32), "x": (1, (mb, H), torch.bfloat16),
-                "q": (2, (mb, nq, d), torch.bfloat16), "o": (3, (mb, nq, d), torch.bfloat16),
-                "x2": (4, (mb, H), torch.bfloat16), "a": (5, (mb, F), torch.bfloat16)}
+        rows = int(self.layer.get_info().activation_rows)
         out = {}
-        for name, (which, shp, dt) in spec.items():
-            buf = torch.empty(shp, dtype=dt, device="cuda")
+        buf = torch.empty((self.cfg.max_batch, H), dtype=torch.float32, device="cuda")
+        self.layer.debug_copy(0, buf)
+        torch.cuda.synchronize()
+        out["h"] = buf[:B].cpu().numpy()
+        spec = {"x": (1, (H,)), "q": (2, (nq, d)), "o": (3, (nq, d)), "x2": (4, (H,)), "a": (5, (F,))}
+        for name, (which, tail) in spec.items():
+            buf = torch.empty((2, rows) + tail, dtype=torch.bfloat16, device="cuda")
             self.layer.debug_copy(which, buf)
             torch.cuda.synchronize()
-            out[name] = buf[:B].float().cpu().numpy()
+            out[name] = (buf[0, :B].double() + buf[1, :B].double()).float().cpu().numpy()
         return out
 
     def appended_kv(self):
