@@ -182,15 +182,41 @@ PRESERVE_API int preserve_set_plan_mode(preserve_layer_t *layer, int mode);
 PRESERVE_API int preserve_decode_step(preserve_layer_t *layer, const preserve_step_io_t *io, void *cuda_stream);
 
 /* Queue n layers back to back (a chain): ios[i] describes layer i's buffers as
- * given; when link != 0, layer i+1's partials_in[0] and residual_in are taken
- * from layer i's mlp_partial_out and residual_out instead of ios[i+1]'s.  All
- * layers must share batch.  The whole chain is replayed as one CUDA graph. */
+ * given; when link != 0, layer i+1's partials_in[0] and residual_in are layer
+ * i's MLP partial sum and residual, handed over inside the library unrounded
+ * (fp32) instead of ios[i+1]'s pointers; layer i's bf16 outputs are still
+ * written.  All layers must share batch and hidden.  The whole chain is replayed
+ * as one CUDA graph. */
 PRESERVE_API int preserve_decode_chain(preserve_layer_t *const *layers, int32_t n, const preserve_step_io_t *ios,
                           int32_t link, void *cuda_stream);
 
 /* The step with host activation buffers (see preserve_host_io_t).  Host
  * buffers should be pinned for the copies to be asynchronous. */
 PRESERVE_API int preserve_decode_step_host(preserve_layer_t *layer, const preserve_host_io_t *io, void *cuda_stream);
+
+/* Per-kernel device times of one step.  Runs the step with direct launches on
+ * `cuda_stream` (prefetch on the side stream as usual), with CUDA events recorded
+ * on that stream around each main-stream kernel, waits for the stream, and writes
+ * PRESERVE_N_KERNELS durations in milliseconds: window A, QKV projection, split-KV
+ * attention, attention merge, output projection, window B, gate/up projection,
+ * down projection.  Results of the step are the same as preserve_decode_step's. */
+#define PRESERVE_N_KERNELS 8
+PRESERVE_API int preserve_profile_step(preserve_layer_t *layer, const preserve_step_io_t *io, void *cuda_stream,
+                                       float *kernel_ms);
+
+/* Queue ONE main-stream kernel of the step (index as in preserve_profile_step) with the
+ * step's arguments, directly on `cuda_stream`, without prefetch.  For benchmarks that time a
+ * kernel on its own; the buffers it reads must hold the results of an earlier full step. */
+PRESERVE_API int preserve_run_kernel(preserve_layer_t *layer, const preserve_step_io_t *io, int32_t which,
+                                     void *cuda_stream);
+
+/* Timeline trace (diagnostics).  While on, every main-stream kernel of a step records, over all
+ * its CTAs, {earliest start, earliest and latest return from the wait on the previous kernel,
+ * latest end} in nanoseconds of the GPU's global timer.  preserve_read_trace synchronises the
+ * device, copies PRESERVE_N_KERNELS x 4 values (kernel order as in preserve_profile_step) to
+ * `out` (host) and clears the slots.  Results of the step do not change. */
+PRESERVE_API int preserve_set_trace(preserve_layer_t *layer, int32_t on);
+PRESERVE_API int preserve_read_trace(preserve_layer_t *layer, int64_t *out);
 
 /* Sizes, device attributes and the last plan. */
 PRESERVE_API int preserve_layer_get_info(const preserve_layer_t *layer, preserve_info_t *info);

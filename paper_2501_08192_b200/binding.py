@@ -23,8 +23,11 @@ EXPORTS = (
     "preserve_layer_init", "preserve_set_prefetch_bytes", "preserve_set_plan_mode", "preserve_decode_step",
     "preserve_decode_chain", "preserve_decode_step_host", "preserve_layer_get_info", "preserve_last_status",
     "preserve_last_cuda_error", "preserve_debug_copy", "preserve_layer_destroy", "preserve_strerror",
-    "preserve_plan_window", "preserve_algorithmic_bytes",
+    "preserve_plan_window", "preserve_algorithmic_bytes", "preserve_profile_step",
+    "preserve_run_kernel", "preserve_set_trace", "preserve_read_trace",
 )
+KERNEL_NAMES = ("window_a", "qkv_proj", "attn_splitkv", "attn_merge", "o_proj", "window_b", "gate_up_proj",
+                "down_proj")
 
 
 class LayerConfig(C.Structure):
@@ -81,6 +84,10 @@ def lib() -> C.CDLL:
         L.preserve_decode_chain.argtypes = [C.POINTER(C.c_void_p), C.c_int32, C.POINTER(StepIO), C.c_int32,
                                             C.c_void_p]
         L.preserve_decode_step_host.argtypes = [C.c_void_p, C.POINTER(HostIO), C.c_void_p]
+        L.preserve_profile_step.argtypes = [C.c_void_p, C.POINTER(StepIO), C.c_void_p, C.POINTER(C.c_float)]
+        L.preserve_run_kernel.argtypes = [C.c_void_p, C.POINTER(StepIO), C.c_int32, C.c_void_p]
+        L.preserve_set_trace.argtypes = [C.c_void_p, C.c_int32]
+        L.preserve_read_trace.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
         L.preserve_layer_get_info.argtypes = [C.c_void_p, C.POINTER(Info)]
         L.preserve_last_status.argtypes = [C.c_void_p]
         L.preserve_last_cuda_error.argtypes = [C.c_void_p]
@@ -193,6 +200,25 @@ class Layer:
     def decode_step_host(self, io: HostIO, stream=None) -> None:
         _check(lib().preserve_decode_step_host(self.handle, C.byref(io), _stream_ptr(stream)),
                "preserve_decode_step_host")
+
+    def profile_step(self, io: StepIO, stream=None) -> List[float]:
+        """Per-kernel milliseconds of one step (order: KERNEL_NAMES); synchronises the stream."""
+        ms = (C.c_float * len(KERNEL_NAMES))()
+        _check(lib().preserve_profile_step(self.handle, C.byref(io), _stream_ptr(stream), ms),
+               "preserve_profile_step")
+        return [float(v) for v in ms]
+
+    def run_kernel(self, io: StepIO, which: int, stream=None) -> None:
+        _check(lib().preserve_run_kernel(self.handle, C.byref(io), which, _stream_ptr(stream)), "preserve_run_kernel")
+
+    def set_trace(self, on: bool) -> None:
+        _check(lib().preserve_set_trace(self.handle, 1 if on else 0), "preserve_set_trace")
+
+    def read_trace(self):
+        """[(start, first_wait_return, last_wait_return, end)] per kernel, ns of the GPU global timer."""
+        buf = (C.c_int64 * (4 * len(KERNEL_NAMES)))()
+        _check(lib().preserve_read_trace(self.handle, buf), "preserve_read_trace")
+        return [tuple(int(buf[4 * k + i]) for i in range(4)) for k in range(len(KERNEL_NAMES))]
 
     def get_info(self) -> Info:
         info = Info()

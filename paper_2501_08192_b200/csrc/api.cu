@@ -74,7 +74,9 @@ struct preserve_layer {
     void *g_attn, *g_mlp;
     double *inv_freq;
 
-    float *h_f32;
+    float *h_f32;                              // window A sum (residual for window B)
+    float *attn_f32, *h2_f32, *mlp_f32;        // unrounded copies: own attention partial (window B input),
+                                               // and the two outputs (handed to the next layer of a linked chain)
     void *x, *q, *o, *attn_partial, *x2, *a;   // x, q, o, x2, a: split bf16 [2][rows][...] (hi + lo)
     int rows;                                  // batch rows per plane (max_batch, padded to 16 on the tensor path)
     float *part_o, *part_ml;
@@ -106,6 +108,13 @@ struct preserve_layer {
 
     std::vector<GraphEntry> graphs;
     uint64_t stamp;
+
+    // per-kernel timing (preserve_profile_step): events around the main-stream kernels
+    long long *trace_buf;        // device [PRESERVE_N_KERNELS][4] timeline slots, used when tracing
+    bool tracing;
+    int only;                    // >= 0: enqueue_step launches only this kernel (preserve_run_kernel)
+    bool profiling;
+    cudaEvent_t prof[PRESERVE_N_KERNELS + 1];
 };
 
 namespace {
@@ -219,6 +228,7 @@ struct StepPtrs {
     const void *parts[kMaxParts];
     const void *peers[kMaxParts];
     const void *residual_in;
+    int resid_f32, part0_f32;      // linked chain: residual_in / parts[0] are the previous layer's fp32 copies
     void *k_cache, *v_cache;
     void *residual_out, *mlp_partial_out, *attn_partial_out;
 };
@@ -271,7 +281,8 @@ int check_step(preserve_layer *L, const preserve_step_io_t *io, StepPtrs *sp)
     return PRESERVE_OK;
 }
 
-int launch_gemm(preserve_layer *L, int which, const void *x, int B, const EpilogueArgs &epi, cudaStream_t s)
+int launch_gemm(preserve_layer *L, int which, const void *x, int B, const EpilogueArgs &epi, cudaStream_t s,
+                long long *trace)
 {
     const Dims d = layer_dims(L->cfg);
     if (L->tensor_path) {
@@ -282,6 +293,7 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
         a.B = B; a.NB = L->nb_pad; a.N = d.n[which]; a.K = d.k[which];
         a.epi = epi;
         a.status = L->status;
+        a.trace = trace;
         CK(L, launch_gemm_tc(a, L->sm_count, s));
         return PRESERVE_OK;
     }
@@ -294,6 +306,8 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
         a.b0 = b0;
         a.N = d.n[which]; a.K = d.k[which];
         a.epi = epi;
+        a.status = L->status;
+        a.trace = trace;
         CK(L, launch_gemv(a, L->sm_count, s));
     }
     return PRESERVE_OK;
@@ -319,8 +333,10 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
     plan_window(nodes_b, 2, L->budget, L->plan_mode, L->planned[1]);
     L->planned[1][2] = 0;
     L->alg_bytes = L->wbytes[0] + L->wbytes[1] + L->wbytes[2] + L->wbytes[3] + L->kv_bytes + activation_bytes(c, B);
-    const bool pf_a = L->planned[0][0] + L->planned[0][1] + L->planned[0][2] > 0;
-    const bool pf_b = L->planned[1][0] + L->planned[1][1] > 0;
+    const bool pf_a = L->only < 0 && L->planned[0][0] + L->planned[0][1] + L->planned[0][2] > 0;
+    const bool pf_b = L->only < 0 && L->planned[1][0] + L->planned[1][1] > 0;
+#define WANT(k) (L->only < 0 || L->only == (k))
+#define TRACE(k) (L->tracing ? L->trace_buf + 4 * (k) : nullptr)
 
     // ---- K/V tensor maps
     if (sp.k_cache != L->k_ptr || sp.v_cache != L->v_ptr) {
@@ -331,6 +347,13 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         L->k_ptr = sp.k_cache;
         L->v_ptr = sp.v_cache;
     }
+
+    int mark = 0;
+#define MARK()                                                   \
+    do {                                                         \
+        if (L->profiling)                                        \
+            CK(L, cudaEventRecord(L->prof[mark++], s));          \
+    } while (0)
 
     // ---- window A  ||  prefetch {Wqkv, K/V, Wo}
     if (pf_a) {
@@ -363,13 +386,15 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         pa.n_segs = n;
         CK(L, launch_prefetch(pa, L->prefetch_ctas, L->side, nullptr, 0));
     }
-    {
+    MARK();   // 0: window A starts
+    if (WANT(0)) {
         WindowArgs w = {};
         for (int i = 0; i < c.tp_degree; ++i)
             w.parts[i] = sp.parts[i];
         w.n_parts = c.tp_degree;
         w.resid = sp.residual_in;
-        w.resid_is_f32 = 0;
+        w.resid_is_f32 = sp.resid_f32;
+        w.part0_is_f32 = sp.part0_f32;
         w.gain = L->g_attn;
         w.eps = c.rms_eps;
         w.h_f32 = L->h_f32;
@@ -377,10 +402,12 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         w.x_bf16 = L->x;
         w.x_plane_elems = (size_t)L->rows * H;
         w.B = B; w.H = H;
+        w.trace = TRACE(0);
         CK(L, launch_window(w, s));
     }
     // ---- QKV projection + rotary embedding + KV append
-    {
+    MARK();   // 1
+    if (WANT(1)) {
         EpilogueArgs e = {};
         e.kind = EPI_QKV;
         e.q_out = L->q;
@@ -390,13 +417,16 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         e.ctx_len = sp.ctx_len;
         e.nq = c.n_q_heads; e.nkv = c.n_kv_heads; e.cap = cap;
         e.inv_freq = c.rope_theta > 0.f ? L->inv_freq : nullptr;
-        int rc = launch_gemm(L, 0, L->x, B, e, s);
+        int rc = launch_gemm(L, 0, L->x, B, e, s, TRACE(1));
         if (rc)
             return rc;
     }
     // ---- attention
-    {
+    MARK();   // 2
+    if (WANT(2) || WANT(3)) {
         AttnArgs a = {};
+        a.phases = (WANT(2) ? 1 : 0) | (WANT(3) ? 2 : 0);
+        a.mid_event = L->profiling ? L->prof[mark++] : nullptr;   // 3: merge starts
         a.k_map = L->k_map;
         a.v_map = L->v_map;
         a.q = L->q;
@@ -405,22 +435,30 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         a.ctx_len = sp.ctx_len;
         a.B = B; a.nq = c.n_q_heads; a.nkv = c.n_kv_heads; a.cap = cap;
         a.grid = L->attn_grid;
-        uint64_t tpi = (total_tiles + (uint64_t)L->attn_grid * 4 - 1) / ((uint64_t)L->attn_grid * 4);
+        // Work items = runs of 64-key tiles.  Aim at one item per CTA when the whole cache is small
+        // (per-item overhead dominates) and at up to four per CTA when it is large (balance under
+        // ragged lengths); depends only on the lengths and the SM count.
+        uint64_t mult = total_tiles / ((uint64_t)L->attn_grid * 4);
+        mult = mult < 1 ? 1 : (mult > 4 ? 4 : mult);
+        uint64_t tpi = (total_tiles + (uint64_t)L->attn_grid * mult - 1) / ((uint64_t)L->attn_grid * mult);
         a.tiles_per_item = tpi < 1 ? 1 : (int)tpi;
         a.max_items = L->max_items;
         a.part_o = L->part_o;
         a.part_ml = L->part_ml;
         a.o_out = L->o;
         a.status = L->status;
+        a.trace = TRACE(2);
         CK(L, launch_attention(a, s));
     }
     // ---- output projection -> this shard's attention partial sum
-    {
+    MARK();   // 4
+    if (WANT(4)) {
         EpilogueArgs e = {};
         e.kind = EPI_PLAIN;
-        e.out = L->attn_partial;
+        e.out = nullptr;
         e.out2 = sp.attn_partial_out;
-        int rc = launch_gemm(L, 1, L->o, B, e, s);
+        e.out_f32 = L->attn_f32;
+        int rc = launch_gemm(L, 1, L->o, B, e, s, TRACE(4));
         if (rc)
             return rc;
     }
@@ -440,9 +478,11 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         pa.n_segs = n;
         CK(L, launch_prefetch(pa, L->prefetch_ctas, L->side, nullptr, 0));
     }
-    {
+    MARK();   // 5: window B starts
+    if (WANT(5)) {
         WindowArgs w = {};
-        w.parts[0] = L->attn_partial;
+        w.parts[0] = L->attn_f32;
+        w.part0_is_f32 = 1;
         for (int i = 0; i + 1 < c.tp_degree; ++i)
             w.parts[i + 1] = sp.peers[i];
         w.n_parts = c.tp_degree;
@@ -450,31 +490,39 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         w.resid_is_f32 = 1;
         w.gain = L->g_mlp;
         w.eps = c.rms_eps;
-        w.h_f32 = nullptr;
+        w.h_f32 = L->h2_f32;
         w.h_bf16 = sp.residual_out;
         w.x_bf16 = L->x2;
         w.x_plane_elems = (size_t)L->rows * H;
         w.B = B; w.H = H;
+        w.trace = TRACE(5);
         CK(L, launch_window(w, s));
     }
     // ---- gate/up projection + SwiGLU, down projection
-    {
+    MARK();   // 6
+    if (WANT(6)) {
         EpilogueArgs e = {};
         e.kind = EPI_SWIGLU;
         e.out = L->a;
         e.out_plane = (size_t)L->rows * c.ffn;
-        int rc = launch_gemm(L, 2, L->x2, B, e, s);
+        int rc = launch_gemm(L, 2, L->x2, B, e, s, TRACE(6));
         if (rc)
             return rc;
     }
-    {
+    MARK();   // 7
+    if (WANT(7)) {
         EpilogueArgs e = {};
         e.kind = EPI_PLAIN;
         e.out = sp.mlp_partial_out;
-        int rc = launch_gemm(L, 3, L->a, B, e, s);
+        e.out_f32 = L->mlp_f32;
+        int rc = launch_gemm(L, 3, L->a, B, e, s, TRACE(7));
         if (rc)
             return rc;
     }
+    MARK();   // 8: end of the last kernel
+#undef MARK
+#undef WANT
+#undef TRACE
     // ---- join the side stream
     if (pf_a || pf_b) {
         CK(L, cudaEventRecord(L->ev_join, L->side));
@@ -497,6 +545,9 @@ uint64_t step_key(const preserve_layer *L, const StepPtrs &sp, uint64_t h)
     h = fnv1a(h, ptrs, sizeof(ptrs));
     h = fnv1a(h, &L->budget, sizeof(L->budget));
     h = fnv1a(h, &L->plan_mode, sizeof(int));
+    h = fnv1a(h, &sp.resid_f32, 2 * sizeof(int));
+    const int tr = L->tracing ? 1 : 0;
+    h = fnv1a(h, &tr, sizeof(int));
     return h;
 }
 
@@ -624,11 +675,14 @@ void preserve_layer_destroy(preserve_layer_t *L)
     if (L->side)
         cudaStreamSynchronize(L->side);
     drop_graphs(L);
-    void *ptrs[] = {L->arena, L->inv_freq, L->h_f32, L->x, L->q, L->o, L->attn_partial, L->x2, L->a,
+    void *ptrs[] = {L->trace_buf, L->attn_f32, L->h2_f32, L->mlp_f32, L->arena, L->inv_freq, L->h_f32, L->x, L->q, L->o, L->attn_partial, L->x2, L->a,
                     L->part_o, L->part_ml, L->status, L->stage_in, L->stage_out, L->ctx_dev};
     for (void *p : ptrs)
         if (p)
             cudaFree(p);
+    for (cudaEvent_t e : L->prof)
+        if (e)
+            cudaEventDestroy(e);
     if (L->ev_a) cudaEventDestroy(L->ev_a);
     if (L->ev_b) cudaEventDestroy(L->ev_b);
     if (L->ev_join) cudaEventDestroy(L->ev_join);
@@ -670,6 +724,7 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     if (!L)
         return PRESERVE_ENOMEM;
     L->cfg = *cfg;
+    L->only = -1;
     L->dev = dev;
     L->sm_count = prop.multiProcessorCount;
     L->l2_bytes = prop.l2CacheSize;
@@ -677,7 +732,9 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     L->max_window = prop.accessPolicyMaxWindowSize;
     L->group = cfg->n_q_heads / cfg->n_kv_heads;
     const char *force = getenv("PRESERVE_FORCE_GEMV");
-    L->tensor_path = cfg->max_batch >= 16 && !(force && force[0] == '1');
+    const char *force_tc = getenv("PRESERVE_FORCE_TENSOR");
+    L->tensor_path = (cfg->max_batch >= 16 && !(force && force[0] == '1')) ||
+                     (force_tc && force_tc[0] == '1' && cfg->ffn % 128 == 0);
     const char *pdl = getenv("PRESERVE_PDL");
     if (pdl)
         g_pdl = pdl[0] == '1';
@@ -751,6 +808,9 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     const size_t RH = (size_t)L->rows * H, Rq = (size_t)L->rows * c.n_q_heads * c.head_dim;
     const size_t RF = (size_t)L->rows * c.ffn;
     CKI(cudaMalloc(&L->h_f32, BH * 4));
+    CKI(cudaMalloc(&L->attn_f32, BH * 4));
+    CKI(cudaMalloc(&L->h2_f32, BH * 4));
+    CKI(cudaMalloc(&L->mlp_f32, BH * 4));
     CKI(cudaMalloc(&L->x, 2 * RH * 2));
     CKI(cudaMalloc(&L->q, 2 * Rq * 2));
     CKI(cudaMalloc(&L->o, 2 * Rq * 2));
@@ -764,14 +824,15 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     CKI(cudaMemset(L->a, 0, 2 * RF * 2));
     L->attn_grid = L->sm_count;
     L->max_items = L->attn_grid * 4 + B * c.n_kv_heads + 8;
-    CKI(cudaMalloc(&L->part_o, (size_t)L->max_items * L->group * kHeadDim * 4));
-    CKI(cudaMalloc(&L->part_ml, (size_t)L->max_items * L->group * 2 * 4));
+    CKI(cudaMalloc(&L->part_o, (size_t)L->max_items * 4 * L->group * kHeadDim * 4));
+    CKI(cudaMalloc(&L->part_ml, (size_t)L->max_items * 4 * L->group * 2 * 4));
     CKI(cudaMalloc(&L->status, 256));
     CKI(cudaMemset(L->status, 0, 256));
     const size_t n_in = (size_t)(2 * c.tp_degree) * BH * 2;
     CKI(cudaMalloc(&L->stage_in, n_in));
     CKI(cudaMalloc(&L->stage_out, 2 * BH * 2));
     CKI(cudaMalloc(&L->ctx_dev, (size_t)B * 4));
+    CKI(cudaMalloc(&L->trace_buf, sizeof(long long) * 4 * PRESERVE_N_KERNELS));
 
     if (L->tensor_path) {
         // activations as the B operand: [2 * nb_pad, K] = hi rows then lo rows, one box covers both
@@ -788,6 +849,8 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     CKI(cudaEventCreateWithFlags(&L->ev_a, cudaEventDisableTiming));
     CKI(cudaEventCreateWithFlags(&L->ev_b, cudaEventDisableTiming));
     CKI(cudaEventCreateWithFlags(&L->ev_join, cudaEventDisableTiming));
+    for (int i = 0; i <= PRESERVE_N_KERNELS; ++i)
+        CKI(cudaEventCreate(&L->prof[i]));
     CKI(cudaDeviceSynchronize());
 #undef CKI
     *out = L;
@@ -835,8 +898,11 @@ int preserve_decode_chain(preserve_layer_t *const *layers, int32_t n, const pres
         if (link && i > 0) {
             if (layers[i]->cfg.hidden != layers[0]->cfg.hidden)
                 return PRESERVE_ESHAPE;
-            sps[i].parts[0] = sps[i - 1].mlp_partial_out;
-            sps[i].residual_in = sps[i - 1].residual_out;
+            // hand the previous layer's results over unrounded (fp32); its bf16 outputs are written too
+            sps[i].parts[0] = layers[i - 1]->mlp_f32;
+            sps[i].part0_f32 = 1;
+            sps[i].residual_in = layers[i - 1]->h2_f32;
+            sps[i].resid_f32 = 1;
         }
     }
     return run_steps(layers, sps.data(), n, static_cast<cudaStream_t>(cuda_stream));
@@ -891,6 +957,68 @@ int preserve_decode_step_host(preserve_layer_t *L, const preserve_host_io_t *io,
     CK(L, cudaMemcpyAsync(io->residual_out, L->stage_out, BH2, cudaMemcpyDeviceToHost, s));
     CK(L, cudaMemcpyAsync(io->mlp_partial_out, L->stage_out + slot, BH2, cudaMemcpyDeviceToHost, s));
     return PRESERVE_OK;
+}
+
+int preserve_profile_step(preserve_layer_t *L, const preserve_step_io_t *io, void *cuda_stream, float *kernel_ms)
+{
+    if (!kernel_ms)
+        return PRESERVE_EINVAL;
+    StepPtrs sp = {};
+    int rc = check_step(L, io, &sp);
+    if (rc)
+        return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    L->profiling = true;
+    rc = enqueue_step(L, sp, s);
+    L->profiling = false;
+    if (rc)
+        return rc;
+    CK(L, cudaStreamSynchronize(s));
+    for (int i = 0; i < PRESERVE_N_KERNELS; ++i)
+        CK(L, cudaEventElapsedTime(&kernel_ms[i], L->prof[i], L->prof[i + 1]));
+    return PRESERVE_OK;
+}
+
+int preserve_run_kernel(preserve_layer_t *L, const preserve_step_io_t *io, int32_t which, void *cuda_stream)
+{
+    if (which < 0 || which >= PRESERVE_N_KERNELS)
+        return PRESERVE_EINVAL;
+    StepPtrs sp = {};
+    int rc = check_step(L, io, &sp);
+    if (rc)
+        return rc;
+    L->only = which;
+    rc = enqueue_step(L, sp, static_cast<cudaStream_t>(cuda_stream));
+    L->only = -1;
+    return rc;
+}
+
+static int reset_trace(preserve_layer *L)
+{
+    long long init[PRESERVE_N_KERNELS][4];
+    for (auto &r : init) {
+        r[0] = r[1] = 0x7fffffffffffffffll;
+        r[2] = r[3] = 0;
+    }
+    CK(L, cudaMemcpy(L->trace_buf, init, sizeof(init), cudaMemcpyHostToDevice));
+    return PRESERVE_OK;
+}
+
+int preserve_set_trace(preserve_layer_t *L, int32_t on)
+{
+    if (!L)
+        return PRESERVE_EINVAL;
+    L->tracing = on != 0;
+    return on ? reset_trace(L) : PRESERVE_OK;
+}
+
+int preserve_read_trace(preserve_layer_t *L, int64_t *out)
+{
+    if (!L || !out)
+        return PRESERVE_EINVAL;
+    CK(L, cudaDeviceSynchronize());
+    CK(L, cudaMemcpy(out, L->trace_buf, sizeof(long long) * 4 * PRESERVE_N_KERNELS, cudaMemcpyDeviceToHost));
+    return reset_trace(L);
 }
 
 int preserve_layer_get_info(const preserve_layer_t *L, preserve_info_t *info)

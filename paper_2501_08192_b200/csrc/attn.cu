@@ -14,9 +14,8 @@
 // full/empty mbarriers (all waits bounded).  Warps 0-3 each own 16 of a tile's
 // 64 keys: S = Q K^T with mma.sync (Q rows = query heads padded to 16, from
 // registers; K via ldmatrix), online softmax in fp32 with exp2, O += P V (V via
-// ldmatrix.trans).  At the end of an item the four warps' (max, sum, O) are
-// combined through shared memory and written as an fp32 partial; k_attn_merge
-// combines the partials of a sequence in fixed order and writes bf16 output.
+// ldmatrix.trans).  At the end of an item every warp writes its (max, sum, O) as an
+// fp32 partial; k_attn_merge combines the partials of a sequence in fixed order.
 // Nothing depends on timing, so results are bit-stable.
 #include "common.cuh"
 #include "kernels.h"
@@ -46,13 +45,11 @@ struct AttnParams {
     bf16 *o_out;            // hi plane; lo plane at o_out + o_plane
     size_t o_plane;
     int *status;
+    long long *trace;
 };
 
 struct AttnSmem {
     alignas(1024) uint8_t stage[kStages][kStageBytes];
-    float merge_o[kConsumerWarps][16][kHeadDim];
-    float merge_m[kConsumerWarps][16];
-    float merge_l[kConsumerWarps][16];
     uint64_t full[kStages];
     uint64_t empty[kStages];
     int item_base[kMaxStreams + 1];
@@ -60,19 +57,33 @@ struct AttnSmem {
 
 __device__ __forceinline__ int tiles_of(int ctx) { return (ctx + 1 + kTileKeys - 1) / kTileKeys; }
 
-// First item index of every stream, computed identically by every CTA.
+// First item index of every stream, computed identically by every CTA: the lengths are
+// fetched by all threads at once (one memory round trip), then warp 0 scans them.
 __device__ __forceinline__ void build_item_table(const AttnParams &p, int *item_base)
 {
-    // serial prefix over at most kMaxStreams entries by one thread; tiny next to the KV stream
-    if (threadIdx.x == 0) {
-        int acc = 0;
-        const int streams = p.B * p.nkv;
-        for (int sidx = 0; sidx < streams; ++sidx) {
-            item_base[sidx] = acc;
-            const int nt = tiles_of(p.ctx_len[sidx / p.nkv]);
-            acc += (nt + p.tiles_per_item - 1) / p.tiles_per_item;
+    const int streams = p.B * p.nkv;
+    for (int i = threadIdx.x; i < streams; i += blockDim.x) {
+        const int nt = tiles_of(p.ctx_len[i / p.nkv]);
+        item_base[i + 1] = (nt + p.tiles_per_item - 1) / p.tiles_per_item;
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        int carry = 0;
+        for (int base = 0; base < streams; base += 32) {
+            const int i = base + threadIdx.x;
+            int v = i < streams ? item_base[i + 1] : 0;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int n = __shfl_up_sync(0xffffffffu, v, o);
+                if ((int)threadIdx.x >= o)
+                    v += n;
+            }
+            if (i < streams)
+                item_base[i + 1] = carry + v;
+            carry += __shfl_sync(0xffffffffu, v, 31);
         }
-        item_base[streams] = acc;
+        if (threadIdx.x == 0)
+            item_base[0] = 0;
     }
 }
 
@@ -102,16 +113,20 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_attn_decode_splitkv(const _
         tma_prefetch_desc(&p.k_map);
         tma_prefetch_desc(&p.v_map);
     }
-    pdl_wait();    // q and the appended k/v come from the QKV projection
-    build_item_table(p, sm.item_base);
+    trace_start(p.trace);
+    pdl_launch_dependents();
+    build_item_table(p, sm.item_base);       // sequence lengths are inputs of the step: no dependency
     __syncthreads();
     const int total_items = sm.item_base[streams];
 
     if (warp == kConsumerWarps) {
         // ------------------------------------------------------------ producer
         if (lane == 0) {
+            // Cached keys and values are read-only during the step, so their tiles are fetched
+            // right away, even while the QKV projection is still running; only a sequence's last
+            // tile (it holds the entry appended by that projection) has to wait for it.
             uint32_t it = 0;
-            bool ok = true;
+            bool ok = true, waited = false;
             for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
                 const int sidx = find_stream(sm.item_base, streams, item);
                 const int chunk = item - sm.item_base[sidx];
@@ -122,6 +137,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_attn_decode_splitkv(const _
                     const int st = it % kStages;
                     const uint32_t ph = (it / kStages) & 1;
                     if (!mbar_wait(&sm.empty[st], ph ^ 1, p.status, ST_TIMEOUT_EMPTY)) { ok = false; break; }
+                    if (tile == nt - 1 && !waited) {
+                        pdl_wait();
+                        waited = true;
+                    }
                     mbar_expect_tx(&sm.full[st], kStageBytes);
                     const int row = sidx * p.cap + tile * kTileKeys;
                     uint8_t *dst = sm.stage[st];
@@ -141,6 +160,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_attn_decode_splitkv(const _
     const int g = lane >> 2, t = lane & 3;
     uint32_t it = 0;
     bool ok = true;
+    pdl_wait();    // q comes from the QKV projection
+    trace_waited(p.trace);
     for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
         const int sidx = find_stream(sm.item_base, streams, item);
         const int b = sidx / p.nkv, kvh = sidx % p.nkv;
@@ -280,97 +301,123 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_attn_decode_splitkv(const _
             if (lane == 0)
                 mbar_arrive(&sm.empty[st]);
         }
-        // ---- combine the four warps and write the item's partial
+        // ---- every warp writes its own partial (max, sum, O) for its 16-key share of the item's
+        // tiles; k_attn_merge combines them.  No cross-warp traffic inside the stream loop.
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
             l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
             l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
         }
-        if (t == 0) {
-            sm.merge_m[warp][g] = m_run[0];
-            sm.merge_m[warp][g + 8] = m_run[1];
-        }
-        asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
-        float scale[2];
+        const size_t ebase = ((size_t)item * kConsumerWarps + warp) * p.G;
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
             const int row = g + 8 * r;
-            float M = sm.merge_m[0][row];
+            if (row < p.G) {
+                float *po = p.part_o + (ebase + row) * kHeadDim + 2 * t;
 #pragma unroll
-            for (int w = 1; w < kConsumerWarps; ++w)
-                M = fmaxf(M, sm.merge_m[w][row]);
-            scale[r] = m_run[r] == -INFINITY ? 0.f : exp2f(m_run[r] - M);
-        }
-        if (t == 0) {
-            sm.merge_l[warp][g] = l_run[0] * scale[0];
-            sm.merge_l[warp][g + 8] = l_run[1] * scale[1];
-        }
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            *reinterpret_cast<float2 *>(&sm.merge_o[warp][g][i * 8 + 2 * t]) =
-                make_float2(o[i][0] * scale[0], o[i][1] * scale[0]);
-            *reinterpret_cast<float2 *>(&sm.merge_o[warp][g + 8][i * 8 + 2 * t]) =
-                make_float2(o[i][2] * scale[1], o[i][3] * scale[1]);
-        }
-        asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
-        {
-            // 128 threads: thread = head dim; loop over the group's rows
-            const int d = threadIdx.x;
-            for (int row = 0; row < p.G; ++row) {
-                float acc = 0.f;
-#pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w)
-                    acc += sm.merge_o[w][row][d];
-                p.part_o[((size_t)item * p.G + row) * kHeadDim + d] = acc;
-                if (d == 0) {
-                    float M = sm.merge_m[0][row], L = 0.f;
-#pragma unroll
-                    for (int w = 1; w < kConsumerWarps; ++w)
-                        M = fmaxf(M, sm.merge_m[w][row]);
-#pragma unroll
-                    for (int w = 0; w < kConsumerWarps; ++w)
-                        L += sm.merge_l[w][row];
-                    p.part_ml[((size_t)item * p.G + row) * 2] = M;
-                    p.part_ml[((size_t)item * p.G + row) * 2 + 1] = L;
-                }
+                for (int i = 0; i < 16; ++i)
+                    *reinterpret_cast<float2 *>(po + i * 8) = make_float2(o[i][2 * r], o[i][2 * r + 1]);
+                if (t == 0)
+                    *reinterpret_cast<float2 *>(p.part_ml + (ebase + row) * 2) = make_float2(m_run[r], l_run[r]);
             }
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
     }
-    pdl_launch_dependents();
+    trace_end(p.trace);
 }
 
-// Merge the partials of one (sequence, query head) in item order; thread = head dim.
-__global__ void __launch_bounds__(kHeadDim) k_attn_merge(const __grid_constant__ AttnParams p)
+// Merge the partials of one (sequence, query head).  512 threads = 16 entry groups x 32
+// lanes of 4 head dims; group eg sums entries eg, eg + 16, ... (independent 128-bit loads, all
+// in flight together), then the 16 group sums are added in fixed order, so the result does
+// not depend on scheduling.
+constexpr int kMergeGroups = 16;
+constexpr int kMergeThreads = kMergeGroups * 32;
+constexpr int kMergeChunk = 1024;          // entries whose weights are staged in shared memory at a time
+__global__ void __launch_bounds__(kMergeThreads) k_attn_merge(const __grid_constant__ AttnParams p)
 {
+    __shared__ float w_s[kMergeChunk];
+    __shared__ float red_s[kMergeThreads / 32];
+    __shared__ int cnt_s[kMergeThreads / 32];
+    __shared__ float4 acc_s[kMergeGroups][32];
+    __shared__ float l_s[kMergeGroups];
     const int b = blockIdx.x / p.nq, hq = blockIdx.x % p.nq;
     const int kvh = hq / p.G, row = hq % p.G;
-    const int d = threadIdx.x;
-    pdl_wait();
-    int base = 0;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int sidx = b * p.nkv + kvh;
-    for (int s2 = 0; s2 < sidx; ++s2) {
-        const int nt = tiles_of(p.ctx_len[s2 / p.nkv]);
-        base += (nt + p.tiles_per_item - 1) / p.tiles_per_item;
-    }
-    const int n_items = (tiles_of(p.ctx_len[b]) + p.tiles_per_item - 1) / p.tiles_per_item;
-    float M = -INFINITY;
-    for (int j = 0; j < n_items; ++j)
-        M = fmaxf(M, p.part_ml[((size_t)(base + j) * p.G + row) * 2]);
-    float L = 0.f, acc = 0.f;
-    for (int j = 0; j < n_items; ++j) {
-        const size_t idx = (size_t)(base + j) * p.G + row;
-        const float m = p.part_ml[idx * 2];
-        const float w = m == -INFINITY ? 0.f : exp2f(m - M);
-        L += p.part_ml[idx * 2 + 1] * w;
-        acc += p.part_o[idx * kHeadDim + d] * w;
-    }
+    long long *tr = p.trace ? p.trace + 4 : nullptr;
+    trace_start(tr);
     pdl_launch_dependents();
-    const float ov = acc / L;
-    const bf16 hi = __float2bfloat16_rn(ov);
-    const size_t oi = ((size_t)b * p.nq + hq) * kHeadDim + d;
-    p.o_out[oi] = hi;
-    p.o_out[p.o_plane + oi] = __float2bfloat16_rn(ov - __bfloat162float(hi));
+    // first item of this stream: parallel count over the streams before it
+    int cnt = 0;
+    for (int s2 = tid; s2 < sidx; s2 += kMergeThreads) {
+        const int nt = tiles_of(p.ctx_len[s2 / p.nkv]);
+        cnt += (nt + p.tiles_per_item - 1) / p.tiles_per_item;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+        cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    if (lane == 0)
+        cnt_s[warp] = cnt;
+    const int n_items = (tiles_of(p.ctx_len[b]) + p.tiles_per_item - 1) / p.tiles_per_item;
+    __syncthreads();
+    int base = 0;
+#pragma unroll
+    for (int i = 0; i < kMergeThreads / 32; ++i)
+        base += cnt_s[i];
+    pdl_wait();    // the partials come from the split-KV kernel
+    trace_waited(tr);
+    const int n_ent = n_items * kConsumerWarps;                 // entry e = item * 4 + consumer warp
+    const size_t stride_ml = (size_t)p.G * 2, stride_o = (size_t)p.G * kHeadDim;
+    const float *ml = p.part_ml + ((size_t)base * kConsumerWarps * p.G + row) * 2;
+    const float *po = p.part_o + ((size_t)base * kConsumerWarps * p.G + row) * kHeadDim + 4 * lane;
+    float M = -INFINITY;
+    for (int e = tid; e < n_ent; e += kMergeThreads)
+        M = fmaxf(M, ml[e * stride_ml]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+        M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    if (lane == 0)
+        red_s[warp] = M;
+    __syncthreads();
+    M = red_s[0];
+#pragma unroll
+    for (int i = 1; i < kMergeThreads / 32; ++i)
+        M = fmaxf(M, red_s[i]);
+    float L = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int e0 = 0; e0 < n_ent; e0 += kMergeChunk) {
+        const int ne = min(kMergeChunk, n_ent - e0);
+        __syncthreads();
+        for (int e = tid; e < ne; e += kMergeThreads) {
+            const float m = ml[(e0 + e) * stride_ml];
+            w_s[e] = m == -INFINITY ? 0.f : exp2f(m - M);
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int e = warp; e < ne; e += kMergeGroups) {
+            const float w = w_s[e];
+            const float4 v = *reinterpret_cast<const float4 *>(po + (e0 + e) * stride_o);
+            L += ml[(e0 + e) * stride_ml + 1] * w;
+            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+        }
+    }
+    acc_s[warp][lane] = acc;
+    if (lane == 0)
+        l_s[warp] = L;
+    __syncthreads();
+    if (tid < kHeadDim) {
+        float a = 0.f, l = 0.f;
+#pragma unroll
+        for (int w = 0; w < kMergeGroups; ++w) {
+            a += reinterpret_cast<const float *>(&acc_s[w][0])[tid];
+            l += l_s[w];
+        }
+        const float ov = a / l;
+        const bf16 hi = __float2bfloat16_rn(ov);
+        const size_t oi = ((size_t)b * p.nq + hq) * kHeadDim + tid;
+        p.o_out[oi] = hi;
+        p.o_out[p.o_plane + oi] = __float2bfloat16_rn(ov - __bfloat162float(hi));
+    }
+    trace_end(tr);
 }
 
 cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
@@ -392,6 +439,7 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     p.part_ml = a.part_ml;
     p.o_out = reinterpret_cast<bf16 *>(a.o_out);
     p.status = a.status;
+    p.trace = a.trace;
 
     const size_t smem = sizeof(AttnSmem) + 1024;
     static bool attr_set = false;
@@ -410,15 +458,25 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     cfg.stream = s;
     cfg.attrs = at;
     cfg.numAttrs = pdl_attr(at);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, k_attn_decode_splitkv, p);
+    const int phases = a.phases ? a.phases : 3;
+    cudaError_t e = cudaSuccess;
+    if (phases & 1)
+        e = cudaLaunchKernelEx(&cfg, k_attn_decode_splitkv, p);
     if (e != cudaSuccess)
         return e;
+    if (a.mid_event) {
+        e = cudaEventRecord(a.mid_event, s);
+        if (e != cudaSuccess)
+            return e;
+    }
     cudaLaunchConfig_t cfg2 = {};
     cfg2.gridDim = dim3(a.B * a.nq);
-    cfg2.blockDim = dim3(kHeadDim);
+    cfg2.blockDim = dim3(kMergeThreads);
     cfg2.stream = s;
     cfg2.attrs = at;
     cfg2.numAttrs = pdl_attr(at);
+    if (!(phases & 2))
+        return cudaSuccess;
     return cudaLaunchKernelEx(&cfg2, k_attn_merge, p);
 }
 

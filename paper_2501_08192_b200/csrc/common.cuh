@@ -123,6 +123,14 @@ __device__ __forceinline__ void tma_load_2d_hint(void *smem_dst, const CUtensorM
                  "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy)
                  : "memory");
 }
+// 1-D bulk async copy global -> shared (16-byte aligned, size a multiple of 16), completing on `bar`.
+__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(smem_dst)),
+                 "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -162,6 +170,33 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t sad
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                  : "r"(saddr));
+}
+
+// Optional timeline trace: per kernel slot, {earliest start, earliest wait-return, latest
+// wait-return, latest end} in nanoseconds of the global timer, over all CTAs (thread 0 each).
+__device__ __forceinline__ long long gtime()
+{
+    long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void trace_start(long long *t)
+{
+    if (t && threadIdx.x == 0)
+        atomicMin(t, gtime());
+}
+__device__ __forceinline__ void trace_waited(long long *t)
+{
+    if (t && threadIdx.x == 0) {
+        const long long v = gtime();
+        atomicMin(t + 1, v);
+        atomicMax(t + 2, v);
+    }
+}
+__device__ __forceinline__ void trace_end(long long *t)
+{
+    if (t && threadIdx.x == 0)
+        atomicMax(t + 3, gtime());
 }
 
 // Programmatic dependent launch: wait for the producer grid's memory to be

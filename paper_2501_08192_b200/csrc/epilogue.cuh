@@ -72,11 +72,17 @@ __device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, bool tenso
     int n0, n1;
     pair_coords(e.kind, tensor_path, pair, n0, n1);
     if (e.kind == EPI_PLAIN) {
-        store_bf16(e.out, (size_t)b * N + n0, v0);
-        store_bf16(e.out, (size_t)b * N + n1, v1);
+        if (e.out) {
+            store_bf16(e.out, (size_t)b * N + n0, v0);
+            store_bf16(e.out, (size_t)b * N + n1, v1);
+        }
         if (e.out2) {
             store_bf16(e.out2, (size_t)b * N + n0, v0);
             store_bf16(e.out2, (size_t)b * N + n1, v1);
+        }
+        if (e.out_f32) {
+            e.out_f32[(size_t)b * N + n0] = v0;
+            e.out_f32[(size_t)b * N + n1] = v1;
         }
     } else if (e.kind == EPI_SWIGLU) {
         const float a = v0 / (1.f + expf(-v0)) * v1;
@@ -85,9 +91,13 @@ __device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, bool tenso
         const int hd = n0, i = n1;
         const int pos = e.ctx_len[b];
         if (hd < e.nq + e.nkv && e.inv_freq) {
-            double s, c;
-            sincos((double)pos * e.inv_freq[i], &s, &c);
-            const float cf = (float)c, sf = (float)s;
+            // angle = pos * theta^(-2i/d): the product and its reduction mod 2 pi need more than
+            // fp32 (angles reach tens of thousands of radians); the reduced angle does not
+            const double ang = (double)pos * e.inv_freq[i];
+            const double turns = rint(ang * 0.15915494309189535);
+            const float red = (float)fma(-turns, 6.283185307179586, ang);
+            float sf, cf;
+            sincosf(red, &sf, &cf);
             const float r0 = v0 * cf - v1 * sf;
             const float r1 = v1 * cf + v0 * sf;
             v0 = r0; v1 = r1;

@@ -42,6 +42,7 @@ struct GemmTcParams {
     uint32_t idesc;
     EpilogueArgs epi;
     int *status;
+    long long *trace;
 };
 
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr)
@@ -94,6 +95,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
     const int kb0 = (int)((long long)p.kblocks * s / p.splits);
     const int kb1 = (int)((long long)p.kblocks * (s + 1) / p.splits);
 
+    trace_start(p.trace);
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.stages; ++i) {
             mbar_init(&full[i], 1);
@@ -119,16 +122,27 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t it = 0;
-            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+            // Weights never depend on earlier kernels, the activations do: fill the whole ring
+            // with weight tiles first (they stream in while the previous kernel finishes), then
+            // wait for the previous kernel and add the activation tiles.
+            const int n_kb = kb1 - kb0;
+            const int pre = n_kb < p.stages ? n_kb : p.stages;
+            for (int i = 0; i < pre; ++i) {
+                mbar_expect_tx(&full[i], stage_bytes);
+                tma_load_2d(smem + (size_t)i * stage_bytes, &p.w_map, (kb0 + i) * kTcBlockK, tile * kTcTileM, &full[i]);
+            }
+            pdl_wait();
+            trace_waited(p.trace);
+            for (int i = 0; i < pre; ++i)
+                tma_load_2d(smem + (size_t)i * stage_bytes + kATileBytes, &p.x_map, (kb0 + i) * kTcBlockK, 0, &full[i]);
+            uint32_t it = pre;
+            for (int kb = kb0 + pre; kb < kb1; ++kb, ++it) {
                 const int st = it % p.stages;
                 const uint32_t ph = (it / p.stages) & 1;
                 if (!mbar_wait(&empty[st], ph ^ 1, p.status, ST_TIMEOUT_EMPTY)) { poisoned = 1; break; }
                 uint8_t *a_dst = smem + (size_t)st * stage_bytes;
                 mbar_expect_tx(&full[st], stage_bytes);
                 tma_load_2d(a_dst, &p.w_map, kb * kTcBlockK, tile * kTcTileM, &full[st]);
-                if (kb == kb0)
-                    pdl_wait();     // weights never depend on earlier kernels; the activations do
                 tma_load_2d(a_dst + kATileBytes, &p.x_map, kb * kTcBlockK, 0, &full[st]);
             }
         }
@@ -169,7 +183,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
             poisoned = 1;
         tc_fence_after();
     }
-    pdl_launch_dependents();
     const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
     float *red = reinterpret_cast<float *>(smem);      // [NB][128] fp32, reuses the ring
 
@@ -236,6 +249,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols)
                      : "memory");
     }
+    trace_end(p.trace);
 }
 
 static int pow2_floor_i(int v)
@@ -257,6 +271,7 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     p.kblocks = a.K / kTcBlockK;
     p.epi = a.epi;
     p.status = a.status;
+    p.trace = a.trace;
     const int tiles = a.N / kTcTileM;
     int splits = pow2_floor_i((2 * sm_count) / tiles > 0 ? (2 * sm_count) / tiles : 1);
     if (splits > 8) splits = 8;

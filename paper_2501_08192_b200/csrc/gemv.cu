@@ -2,18 +2,31 @@
 //
 // The projection layers of the decode phase reuse each weight only `batch`
 // times (Section 2, "LLM decoding is memory BW-limited"), so the kernel is a
-// pure weight stream: every warp walks a contiguous run of 1 KiB fragment-major
-// tiles (16 output rows x 32 k, see pack.cu) with two 128-bit loads per lane per
-// tile and no shared-memory staging.  Two arithmetic variants share the loop:
+// pure weight stream.  The packed weights are 1 KiB fragment-major tiles (16
+// output rows x 32 k, see pack.cu), contiguous along k within a 16-row block.
+//
+// Persistent CTAs of 8 warps.  A CTA (or a cluster of up to 8 CTAs) owns one
+// group of 16-row blocks at a time; the k range is split over the warps of the
+// CTA and the CTAs of the cluster, so every warp streams ONE contiguous run of
+// tiles.  Each warp is its own producer and consumer: lane 0 keeps a private ring
+// of four 2 KiB slots filled with bulk async copies (cp.async.bulk -> shared
+// memory, completion on per-slot mbarriers, all waits bounded) and refills a slot
+// as soon as the warp has consumed it.  The first four copies are issued before
+// the programmatic-dependent-launch wait, so weights are already streaming while
+// the previous kernel finishes; only the small activation fragments are loaded
+// after the wait.  Grids never exceed what is co-resident, so there is no second
+// wave.
+// Two arithmetic variants:
 //   - CUDA cores (batch <= 4): 2 x batch fp32 accumulators per lane, finished by
 //     a warp-shuffle reduction over the four lanes that share a row;
 //   - mma.sync m16n8k16 (5 <= batch <= 15): at batch 8 the fp32 FMA pipe would
 //     need ~8 FMAs per weight and co-limit the stream, so the 16x32 tile feeds
-//     two warp MMAs with the batch as the n = 8 operand.
-// Split-K: the k range is divided over the warps of a CTA (summed through
-// shared memory) and over the CTAs of a thread-block cluster (summed by rank 0
-// through distributed shared memory), always in a fixed order, so results are
-// bit-stable.  Rank 0 applies the fused epilogue (epilogue.cuh).
+//     warp MMAs with the batch as the n = 8 operand.
+// Activations arrive as hi + lo bf16 planes (x = hi + lo).
+// Split-K partial sums are added in a fixed order (warps through shared memory,
+// cluster ranks through distributed shared memory, each rank finishing its share
+// of the outputs), so results are bit-stable.  The fused epilogues live in
+// epilogue.cuh.
 #include <cooperative_groups.h>
 
 #include "epilogue.cuh"
@@ -22,10 +35,12 @@ namespace cg = cooperative_groups;
 
 namespace prsv {
 
-int g_pdl = 0;
+int g_pdl = 1;
 
 constexpr int kGemvWarps = 8;
-constexpr int kGemvUnroll = 4;
+constexpr int kRingSlots = 4;
+constexpr int kUnitChunks = 2;                       // tiles per ring slot (2 KiB)
+constexpr int kGemvSmemBytes = kGemvWarps * kRingSlots * kUnitChunks * 1024;
 
 struct GemvParams {
     const uint4 *w;
@@ -37,6 +52,9 @@ struct GemvParams {
     int kchunks;         // K / 32
     int warps_k;         // warps of a CTA that split k (1, 2, 4, 8)
     int splits;          // cluster size along k
+    int groups;          // row-block groups = row_blocks / (8 / warps_k)
+    int *status;
+    long long *trace;
     EpilogueArgs epi;
 };
 
@@ -45,38 +63,92 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
 {
     constexpr int NTB = MMA ? NB / 8 : 1;   // n-tiles that cover the batch
     constexpr int NT = 2 * NTB;             // hi planes then lo planes of the activations
-    __shared__ float red[kGemvWarps][16][NB];      // per-warp partials
-    __shared__ float cta_part[kGemvWarps][16][NB];  // per-row-block CTA partials (read by cluster rank 0)
+    constexpr int NX = MMA ? NT : 2 * NB;   // activation fragments (uint4) per tile
+    __shared__ float red[kGemvWarps][16][NB];       // per-warp partials
+    __shared__ float cta_part[kGemvWarps][16][NB];  // per-row-block CTA partials (read across the cluster)
+    __shared__ uint64_t bars[kGemvWarps][kRingSlots];
+    extern __shared__ uint8_t gemv_smem_raw[];
+    uint8_t *wsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(gemv_smem_raw) + 127) & ~uintptr_t(127));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
     const int rbs_per_cta = kGemvWarps / p.warps_k;
     const int rbl = warp / p.warps_k, wk = warp % p.warps_k;
-    const int rb = blockIdx.x * rbs_per_cta + rbl;
     const int s = blockIdx.y;                        // == cluster rank along k
-    const bool active = rb < p.row_blocks;
 
-    // k-chunk range of this CTA, then of this warp
-    const int cta_lo = (int)((long long)p.kchunks * s / p.splits);
-    const int cta_hi = (int)((long long)p.kchunks * (s + 1) / p.splits);
-    const int span = cta_hi - cta_lo;
-    const int c_begin = cta_lo + (int)((long long)span * wk / p.warps_k);
-    const int c_end = cta_lo + (int)((long long)span * (wk + 1) / p.warps_k);
+    // this warp's run of k-chunks: part ki of ks = splits * warps_k equal parts (same for every group)
+    const int ks = p.splits * p.warps_k, ki = s * p.warps_k + wk;
+    const int c_begin = (int)((long long)p.kchunks * ki / ks);
+    const int c_end = (int)((long long)p.kchunks * (ki + 1) / ks);
+    uint8_t *ring = wsm + (size_t)warp * (kRingSlots * kUnitChunks * 1024);
 
-    float acc[MMA ? NT : 2 * NB][MMA ? 4 : 1];
+    trace_start(p.trace);
+    pdl_launch_dependents();    // the next kernel may start its own weight fetch right away
+
+    // ---- producer side of this warp's ring (lane 0 only)
+    int p_grp = blockIdx.x, p_c = c_begin;           // next unit to fetch
+    uint32_t n_issued = 0;
+    auto issue_next = [&]() {
+        if (p_grp >= p.groups || c_begin >= c_end)
+            return;
+        const int n = min(kUnitChunks, c_end - p_c);
+        const int slot = n_issued % kRingSlots;
+        const size_t rb = (size_t)p_grp * rbs_per_cta + rbl;
+        const uint32_t bytes = (uint32_t)n * 1024u;
+        mbar_expect_tx(&bars[warp][slot], bytes);
+        bulk_load(ring + slot * (kUnitChunks * 1024), reinterpret_cast<const uint8_t *>(p.w) + (rb * p.kchunks + p_c) * 1024,
+                  bytes, &bars[warp][slot]);
+        ++n_issued;
+        p_c += kUnitChunks;
+        if (p_c >= c_end) {
+            p_c = c_begin;
+            p_grp += gridDim.x;
+        }
+    };
+    if (lane == 0) {
 #pragma unroll
-    for (int i = 0; i < (MMA ? NT : 2 * NB); ++i)
+        for (int i = 0; i < kRingSlots; ++i)
+            mbar_init(&bars[warp][i], 1);
+        mbar_fence_init();
 #pragma unroll
-        for (int j = 0; j < (MMA ? 4 : 1); ++j)
-            acc[i][j] = 0.f;
+        for (int i = 0; i < kRingSlots; ++i)
+            issue_next();
+    }
+    __syncwarp();
 
-    const uint4 *wp = p.w + (size_t)rb * p.kchunks * 64 + lane * 2;
     const int xrow = p.K >> 3;                       // uint4 per activation row
+    auto load_x = [&](int c, uint4 (&xq)[NX]) {
+        if constexpr (MMA) {
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                const int b = (nt % NTB) * 8 + g;
+                const uint4 *plane = p.x + (nt >= NTB ? p.x_plane : 0);
+                xq[nt] = b < p.B ? ld_cached(plane + (size_t)(p.b0 + b) * xrow + c * 4 + t) : make_uint4(0, 0, 0, 0);
+            }
+        } else {
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                xq[b] = b < p.B ? ld_cached(p.x + (size_t)(p.b0 + b) * xrow + c * 4 + t) : make_uint4(0, 0, 0, 0);
+                xq[NB + b] = b < p.B ? ld_cached(p.x + p.x_plane + (size_t)(p.b0 + b) * xrow + c * 4 + t)
+                                     : make_uint4(0, 0, 0, 0);
+            }
+        }
+    };
 
     pdl_wait();   // x is produced by the previous kernel of the stream
+    trace_waited(p.trace);
 
-    if (active) {
-        auto compute = [&](const uint4 &wl, const uint4 &wh, const uint4 (&xq)[MMA ? NT : 2 * NB]) {
+    uint32_t n_consumed = 0;
+    bool ok = true;
+    for (int grp = blockIdx.x; grp < p.groups; grp += gridDim.x) {
+        float acc[MMA ? NT : 2 * NB][MMA ? 4 : 1];
+#pragma unroll
+        for (int i = 0; i < (MMA ? NT : 2 * NB); ++i)
+#pragma unroll
+            for (int j = 0; j < (MMA ? 4 : 1); ++j)
+                acc[i][j] = 0.f;
+
+        auto compute = [&](const uint4 &wl, const uint4 &wh, const uint4 (&xq)[NX]) {
             if constexpr (MMA) {
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
@@ -104,119 +176,134 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
                 }
             }
         };
-        auto load_x = [&](int c, uint4 (&xq)[MMA ? NT : 2 * NB]) {
-            if constexpr (MMA) {
+
+        // ---- stream this warp's run through its ring.  The activation fragments of up to 8 tiles
+        // are requested in one burst, so their L2 latency is paid once per burst.
+        constexpr int kBurst = NX <= 2 ? 8 : (NX <= 4 ? 4 : 2);     // tiles per burst: <= 64 registers of x
+        constexpr int kBurstUnits = kBurst / kUnitChunks;
+        for (int c0 = c_begin; ok && c0 < c_end; c0 += kBurst) {
+            const int nb = min(kBurst, c_end - c0);
+            uint4 xq[kBurst][NX];
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const int b = (nt % NTB) * 8 + g;
-                    const uint4 *plane = p.x + (nt >= NTB ? p.x_plane : 0);
-                    xq[nt] = b < p.B ? ld_cached(plane + (size_t)(p.b0 + b) * xrow + c * 4 + t) : make_uint4(0, 0, 0, 0);
-                }
-            } else {
+            for (int u = 0; u < kBurst; ++u)
+                if (u < nb)
+                    load_x(c0 + u, xq[u]);
 #pragma unroll
-                for (int b = 0; b < NB; ++b) {
-                    xq[b] = b < p.B ? ld_cached(p.x + (size_t)(p.b0 + b) * xrow + c * 4 + t) : make_uint4(0, 0, 0, 0);
-                    xq[NB + b] = b < p.B ? ld_cached(p.x + p.x_plane + (size_t)(p.b0 + b) * xrow + c * 4 + t)
-                                         : make_uint4(0, 0, 0, 0);
+            for (int uu = 0; uu < kBurstUnits; ++uu) {
+                if (uu * kUnitChunks < nb && ok) {
+                    const int slot = n_consumed % kRingSlots;
+                    const uint32_t ph = (n_consumed / kRingSlots) & 1;
+                    ok = mbar_wait(&bars[warp][slot], ph, p.status, ST_TIMEOUT_FULL);
+                    if (ok) {
+                        const uint4 *wtile =
+                            reinterpret_cast<const uint4 *>(ring + slot * (kUnitChunks * 1024)) + lane * 2;
+#pragma unroll
+                        for (int u = 0; u < kUnitChunks; ++u)
+                            if (uu * kUnitChunks + u < nb) {
+                                const uint4 wl = wtile[u * 64], wh = wtile[u * 64 + 1];
+                                compute(wl, wh, xq[uu * kUnitChunks + u]);
+                            }
+                    }
+                    ++n_consumed;
+                    __syncwarp();
+                    if (lane == 0 && ok)
+                        issue_next();       // the slot just read is free again
                 }
             }
-        };
+        }
 
-        int c = c_begin;
-        for (; c + kGemvUnroll <= c_end; c += kGemvUnroll) {
-            uint4 wl[kGemvUnroll], wh[kGemvUnroll];
-            uint4 xq[kGemvUnroll][MMA ? NT : 2 * NB];
+        // ---- warp partial -> shared memory: red[warp][row][b]
+        if constexpr (MMA) {
 #pragma unroll
-            for (int u = 0; u < kGemvUnroll; ++u) {
-                wl[u] = ld_stream(wp + (size_t)(c + u) * 64);
-                wh[u] = ld_stream(wp + (size_t)(c + u) * 64 + 1);
+            for (int nt = 0; nt < NTB; ++nt) {
+                red[warp][g][nt * 8 + 2 * t] = acc[nt][0] + acc[NTB + nt][0];
+                red[warp][g][nt * 8 + 2 * t + 1] = acc[nt][1] + acc[NTB + nt][1];
+                red[warp][g + 8][nt * 8 + 2 * t] = acc[nt][2] + acc[NTB + nt][2];
+                red[warp][g + 8][nt * 8 + 2 * t + 1] = acc[nt][3] + acc[NTB + nt][3];
             }
+        } else {
 #pragma unroll
-            for (int u = 0; u < kGemvUnroll; ++u)
-                load_x(c + u, xq[u]);
+            for (int i = 0; i < 2 * NB; ++i) {
+                float v = acc[i][0];
+                v += __shfl_xor_sync(0xffffffffu, v, 1);
+                v += __shfl_xor_sync(0xffffffffu, v, 2);
+                if (t == 0)
+                    red[warp][g + 8 * (i & 1)][i >> 1] = v;
+            }
+        }
+        __syncthreads();
+
+        // ---- sum over the warps that split k (fixed order) -> cta_part[rbl][row][b]
+        for (int i = threadIdx.x; i < rbs_per_cta * 16 * NB; i += blockDim.x) {
+            const int b = i % NB, row = (i / NB) % 16, rl = i / (16 * NB);
+            float v = 0.f;
+            for (int k = 0; k < p.warps_k; ++k)
+                v += red[rl * p.warps_k + k][row][b];
+            cta_part[rl][row][b] = v;
+        }
+
+        // ---- sum over the cluster ranks (fixed order); every rank finishes its share of the outputs
+        const int n_out = rbs_per_cta * 8 * NB;          // (row block, pair, batch row) triples of the group
+        if (p.splits > 1) {
+            cg::cluster_group cluster = cg::this_cluster();
+            cluster.sync();
+            const float *remote[8];
 #pragma unroll
-            for (int u = 0; u < kGemvUnroll; ++u)
-                compute(wl[u], wh[u], xq[u]);
-        }
-        for (; c < c_end; ++c) {
-            uint4 xq[MMA ? NT : 2 * NB];
-            const uint4 wl = ld_stream(wp + (size_t)c * 64);
-            const uint4 wh = ld_stream(wp + (size_t)c * 64 + 1);
-            load_x(c, xq);
-            compute(wl, wh, xq);
-        }
-    }
-
-    pdl_launch_dependents();
-
-    // ---- warp partial -> shared memory: red[warp][row][b]
-    if constexpr (MMA) {
-#pragma unroll
-        for (int nt = 0; nt < NTB; ++nt) {
-            red[warp][g][nt * 8 + 2 * t] = acc[nt][0] + acc[NTB + nt][0];
-            red[warp][g][nt * 8 + 2 * t + 1] = acc[nt][1] + acc[NTB + nt][1];
-            red[warp][g + 8][nt * 8 + 2 * t] = acc[nt][2] + acc[NTB + nt][2];
-            red[warp][g + 8][nt * 8 + 2 * t + 1] = acc[nt][3] + acc[NTB + nt][3];
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 2 * NB; ++i) {
-            float v = acc[i][0];
-            v += __shfl_xor_sync(0xffffffffu, v, 1);
-            v += __shfl_xor_sync(0xffffffffu, v, 2);
-            if (t == 0)
-                red[warp][g + 8 * (i & 1)][i >> 1] = v;
-        }
-    }
-    __syncthreads();
-
-    // ---- sum over the warps that split k (fixed order) -> cta_part[rbl][row][b]
-    for (int i = threadIdx.x; i < rbs_per_cta * 16 * NB; i += blockDim.x) {
-        const int b = i % NB, row = (i / NB) % 16, rl = i / (16 * NB);
-        float v = 0.f;
-        for (int k = 0; k < p.warps_k; ++k)
-            v += red[rl * p.warps_k + k][row][b];
-        cta_part[rl][row][b] = v;
-    }
-
-    if (p.splits > 1) {
-        cg::cluster_group cluster = cg::this_cluster();
-        cluster.sync();
-        if (s == 0) {
-            for (int i = threadIdx.x; i < rbs_per_cta * 8 * NB; i += blockDim.x) {
+            for (int q = 0; q < 8; ++q)
+                remote[q] = cluster.map_shared_rank(&cta_part[0][0][0], q < p.splits ? q : 0);
+            for (int i = threadIdx.x * p.splits + s; i < n_out; i += blockDim.x * p.splits) {
                 const int b = i % NB, r = (i / NB) % 8, rl = i / (8 * NB);
-                const int rbg = blockIdx.x * rbs_per_cta + rl;
-                if (rbg >= p.row_blocks || b >= p.B)
+                if (b >= p.B)
                     continue;
                 float v0 = 0.f, v1 = 0.f;
-                for (int q = 0; q < p.splits; ++q) {
-                    const float *remote = cluster.map_shared_rank(&cta_part[0][0][0], q);
-                    v0 += remote[(rl * 16 + r) * NB + b];
-                    v1 += remote[(rl * 16 + r + 8) * NB + b];
-                }
-                apply_epilogue(p.epi, false, p.N, p.b0 + b, rbg * 8 + r, v0, v1);
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (q < p.splits) {
+                        v0 += remote[q][(rl * 16 + r) * NB + b];
+                        v1 += remote[q][(rl * 16 + r + 8) * NB + b];
+                    }
+                apply_epilogue(p.epi, false, p.N, p.b0 + b, (grp * rbs_per_cta + rl) * 8 + r, v0, v1);
             }
-        }
-        cluster.sync();   // peers' shared memory must outlive rank 0's reads
-    } else {
-        __syncthreads();
-        for (int i = threadIdx.x; i < rbs_per_cta * 8 * NB; i += blockDim.x) {
-            const int b = i % NB, r = (i / NB) % 8, rl = i / (8 * NB);
-            const int rbg = blockIdx.x * rbs_per_cta + rl;
-            if (rbg >= p.row_blocks || b >= p.B)
-                continue;
-            apply_epilogue(p.epi, false, p.N, p.b0 + b, rbg * 8 + r, cta_part[rl][r][b], cta_part[rl][r + 8][b]);
+            cluster.sync();   // peers' shared memory must outlive the reads; also fences red/cta_part reuse
+        } else {
+            __syncthreads();
+            for (int i = threadIdx.x; i < n_out; i += blockDim.x) {
+                const int b = i % NB, r = (i / NB) % 8, rl = i / (8 * NB);
+                if (b >= p.B)
+                    continue;
+                apply_epilogue(p.epi, false, p.N, p.b0 + b, (grp * rbs_per_cta + rl) * 8 + r, cta_part[rl][r][b],
+                               cta_part[rl][r + 8][b]);
+            }
+            __syncthreads();
         }
     }
+    trace_end(p.trace);
 }
 
 template <int NB, bool MMA>
-static cudaError_t launch_variant(const GemvParams &p, cudaStream_t s)
+static cudaError_t launch_variant(GemvParams &p, int sm_count, cudaStream_t s)
 {
-    const int rbs_per_cta = kGemvWarps / p.warps_k;
+    static int ctas_per_sm = 0;
+    if (!ctas_per_sm) {
+        cudaError_t e = cudaFuncSetAttribute(k_gemv_splitk<NB, MMA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kGemvSmemBytes + 128);
+        if (e != cudaSuccess)
+            return e;
+        int n = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_gemv_splitk<NB, MMA>, kGemvWarps * 32,
+                                                          kGemvSmemBytes + 128);
+        if (e != cudaSuccess)
+            return e;
+        ctas_per_sm = n < 1 ? 1 : n;
+    }
+    // one wave at most: clusters beyond what is co-resident become extra loop iterations
+    int clusters = (sm_count * ctas_per_sm) / p.splits;
+    if (clusters > p.groups) clusters = p.groups;
+    if (clusters < 1) clusters = 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((p.row_blocks + rbs_per_cta - 1) / rbs_per_cta, p.splits, 1);
+    cfg.gridDim = dim3(clusters, p.splits, 1);
     cfg.blockDim = dim3(kGemvWarps * 32);
+    cfg.dynamicSmemBytes = kGemvSmemBytes + 128;
     cfg.stream = s;
     cudaLaunchAttribute at[2];
     int n = pdl_attr(at);
@@ -232,14 +319,6 @@ static cudaError_t launch_variant(const GemvParams &p, cudaStream_t s)
     return cudaLaunchKernelEx(&cfg, k_gemv_splitk<NB, MMA>, p);
 }
 
-static int pow2_floor(int v)
-{
-    int r = 1;
-    while (r * 2 <= v)
-        r *= 2;
-    return r;
-}
-
 cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s)
 {
     if (a.B < 1 || a.B > 16 || a.N % 16 || a.K % 32)
@@ -252,27 +331,27 @@ cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s)
     p.row_blocks = a.N / 16;
     p.kchunks = a.K / 32;
     p.epi = a.epi;
+    p.status = a.status;
+    p.trace = a.trace;
 
-    // Split k so that about 16 warps per SM each own a few tiles.  The choice depends
-    // only on the shapes and the SM count, never on the prefetch setting.
-    const long long tiles = (long long)p.row_blocks * p.kchunks;
-    const long long target_warps = (long long)sm_count * 16;
-    long long per_warp = tiles / target_warps;
-    if (per_warp < 2) per_warp = 2;
-    if (per_warp > 16) per_warp = 16;
-    int ks = (int)(p.kchunks / per_warp);
-    if (ks < 1) ks = 1;
-    ks = pow2_floor(ks);
-    if (ks > 64) ks = 64;
-    p.warps_k = ks < kGemvWarps ? ks : kGemvWarps;
-    p.splits = ks / p.warps_k;
-    if (p.splits < 1) p.splits = 1;
+    // Mapping: k is split over the 8 warps of a CTA while every warp still gets at least two
+    // tiles (otherwise fewer warps split k and the others take further row blocks); cluster ranks
+    // add splits only while there are fewer row-block groups than SMs.  Larger clusters are
+    // avoided: they fragment the co-resident capacity and cause a second wave.  Depends only on
+    // the shapes and the SM count, never on the prefetch setting.
+    int wk = kGemvWarps;
+    while (wk > 1 && p.kchunks / wk < 2 && p.row_blocks % (2 * kGemvWarps / wk) == 0) wk /= 2;
+    p.warps_k = wk;
+    p.groups = p.row_blocks / (kGemvWarps / wk);
+    int splits = 1;
+    while (splits < 8 && p.groups * splits < sm_count && p.kchunks / (wk * splits * 2) >= 2) splits *= 2;
+    p.splits = splits;
 
-    if (a.B == 1) return launch_variant<1, false>(p, s);
-    if (a.B == 2) return launch_variant<2, false>(p, s);
-    if (a.B <= 4) return launch_variant<4, false>(p, s);
-    if (a.B <= 8) return launch_variant<8, true>(p, s);
-    return launch_variant<16, true>(p, s);
+    if (a.B == 1) return launch_variant<1, false>(p, sm_count, s);
+    if (a.B == 2) return launch_variant<2, false>(p, sm_count, s);
+    if (a.B <= 4) return launch_variant<4, false>(p, sm_count, s);
+    if (a.B <= 8) return launch_variant<8, true>(p, sm_count, s);
+    return launch_variant<16, true>(p, sm_count, s);
 }
 
 }  // namespace prsv

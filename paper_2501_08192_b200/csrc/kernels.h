@@ -27,8 +27,9 @@ constexpr int kHeadDim = 128;
 
 // ---- communication-window stand-in: h = resid + sum_p part_p ; x = RMSNorm(h) * gain
 struct WindowArgs {
-    const void *parts[kMaxParts];  // bf16 [B,H] each
+    const void *parts[kMaxParts];  // bf16 [B,H] each (parts[0] fp32 when part0_is_f32)
     int n_parts;
+    int part0_is_f32;
     const void *resid;             // bf16 [B,H] or fp32 [B,H]
     int resid_is_f32;
     const void *gain;              // bf16 [H]
@@ -38,6 +39,7 @@ struct WindowArgs {
     void *x_bf16;                  // bf16 [2][rows][H]: hi plane then lo plane (x = hi + lo)
     size_t x_plane_elems;          // elements between the planes
     int B, H;
+    long long *trace;              // optional timeline slot (4 values), see common.cuh
 };
 cudaError_t launch_window(const WindowArgs &a, cudaStream_t s);
 
@@ -48,6 +50,7 @@ struct EpilogueArgs {
     void *out;            // PLAIN: bf16 [B,N]; SWIGLU: split bf16 [2][rows][N/2]
     size_t out_plane;     // SWIGLU: elements between the hi and lo planes of out
     void *out2;           // PLAIN: optional second copy of the output (bf16 [B,N])
+    float *out_f32;       // PLAIN: optional unrounded copy (fp32 [B,N])
     // QKV: rows are heads [q | k | v] x head_dim; rotary embedding on q and k, k/v appended
     void *q_out;          // split bf16 [2][rows][nq,d]
     size_t q_plane;       // elements between the hi and lo planes of q_out
@@ -76,6 +79,8 @@ struct GemvArgs {
     int B, N, K;          // B <= 16 batch rows starting at b0
     int b0;
     EpilogueArgs epi;
+    int *status;
+    long long *trace;
 };
 cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s);
 
@@ -86,6 +91,7 @@ struct GemmTcArgs {
     int B, NB, N, K;      // NB = batch rows per plane (multiple of 16)
     EpilogueArgs epi;
     int *status;
+    long long *trace;
 };
 cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s);
 
@@ -100,11 +106,14 @@ struct AttnArgs {
     int grid;             // persistent CTAs
     int tiles_per_item;   // 64-key tiles per work item
     int max_items;        // capacity of the partial buffers
-    float *part_o;        // fp32 [max_items, G, d]
-    float *part_ml;       // fp32 [max_items, G, 2]
+    float *part_o;        // fp32 [max_items, 4 consumer warps, G, d]
+    float *part_ml;       // fp32 [max_items, 4, G, 2]
     void *o_out;          // split bf16 [2][rows][nq,d]
     size_t o_plane;
     int *status;
+    cudaEvent_t mid_event; // optional: recorded between the split-KV kernel and the merge kernel
+    int phases;            // bit 0: split-KV kernel, bit 1: merge kernel (0 = both)
+    long long *trace;      // optional: two consecutive timeline slots (split-KV, merge)
 };
 cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s);
 

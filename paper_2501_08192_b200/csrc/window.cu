@@ -2,7 +2,8 @@
 // deliver on a tensor-parallel system (Section 2, "Multi-device inference";
 // Section 3, "Vanilla execution"): h = residual + sum of the P partial-sum
 // buffers, then x = RMSNorm(h) * gain.  One CTA per token row; 128-bit
-// coalesced loads; fp32 accumulation in the fixed order residual, part 0..P-1.
+// coalesced loads; fp32 accumulation in the fixed order residual, part 0..P-1
+// (part 0 may be fp32: this shard's own result, or the previous layer's in a chain).
 // The kernel is deliberately narrow (B CTAs): during a real allreduce the SMs
 // idle, which is what leaves HBM bandwidth to the prefetch stream.
 #include "common.cuh"
@@ -23,18 +24,30 @@ struct WindowParams {
     uint4 *x_bf16;       // hi plane; the lo plane follows at x_plane uint4s
     size_t x_plane;
     int H;
+    long long *trace;
 };
 
-template <bool RESID_F32>
+template <bool RESID_F32, bool PART0_F32>
 __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_constant__ WindowParams p)
 {
     const int row = blockIdx.x;
     const int chunks = p.H >> 3;                 // uint4 chunks per row
     const size_t row_off = (size_t)row * chunks;
     float v[kWinMaxChunks][8];
+    uint4 gn[kWinMaxChunks];
     float ss = 0.f;
 
-    pdl_wait();   // partial sums come from the preceding kernel in the stream
+    // the gain does not depend on the previous kernel: fetch it before waiting
+#pragma unroll
+    for (int c = 0; c < kWinMaxChunks; ++c) {
+        const int ch = threadIdx.x + c * blockDim.x;
+        gn[c] = ch < chunks ? ld_cached(p.gain + ch) : make_uint4(0, 0, 0, 0);
+    }
+
+    trace_start(p.trace);
+    pdl_launch_dependents();   // the next kernel may start fetching its weights now
+    pdl_wait();                // partial sums come from the preceding kernel in the stream
+    trace_waited(p.trace);
 
 #pragma unroll
     for (int c = 0; c < kWinMaxChunks; ++c) {
@@ -50,10 +63,26 @@ __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_con
                 v[c][0] = bf_lo(r.x); v[c][1] = bf_hi(r.x); v[c][2] = bf_lo(r.y); v[c][3] = bf_hi(r.y);
                 v[c][4] = bf_lo(r.z); v[c][5] = bf_hi(r.z); v[c][6] = bf_lo(r.w); v[c][7] = bf_hi(r.w);
             }
-            for (int q = 0; q < p.n_parts; ++q) {
-                uint4 r = ld_stream(p.parts[q] + row_off + ch);
-                v[c][0] += bf_lo(r.x); v[c][1] += bf_hi(r.x); v[c][2] += bf_lo(r.y); v[c][3] += bf_hi(r.y);
-                v[c][4] += bf_lo(r.z); v[c][5] += bf_hi(r.z); v[c][6] += bf_lo(r.w); v[c][7] += bf_hi(r.w);
+            if (PART0_F32) {     // partial 0 handed over in fp32 (own result / previous layer of a chain)
+                const float4 *r = reinterpret_cast<const float4 *>(p.parts[0]) + (row_off + ch) * 2;
+                float4 a = r[0], b = r[1];
+                v[c][0] += a.x; v[c][1] += a.y; v[c][2] += a.z; v[c][3] += a.w;
+                v[c][4] += b.x; v[c][5] += b.y; v[c][6] += b.z; v[c][7] += b.w;
+            }
+            // issue the loads of up to 8 partial buffers before the first add, so the row is
+            // fetched in one or two memory round trips instead of one per buffer
+            for (int q0 = 0; q0 < p.n_parts; q0 += 8) {
+                uint4 r[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (q0 + j < p.n_parts)
+                        r[j] = PART0_F32 && q0 + j == 0 ? make_uint4(0, 0, 0, 0) : ld_stream(p.parts[q0 + j] + row_off + ch);
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (q0 + j < p.n_parts && !(PART0_F32 && q0 + j == 0)) {
+                        v[c][0] += bf_lo(r[j].x); v[c][1] += bf_hi(r[j].x); v[c][2] += bf_lo(r[j].y); v[c][3] += bf_hi(r[j].y);
+                        v[c][4] += bf_lo(r[j].z); v[c][5] += bf_hi(r[j].z); v[c][6] += bf_lo(r[j].w); v[c][7] += bf_hi(r[j].w);
+                    }
             }
 #pragma unroll
             for (int i = 0; i < 8; ++i)
@@ -83,8 +112,6 @@ __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_con
     __syncthreads();
     const float inv = rsqrtf(total / (float)p.H + p.eps);
 
-    pdl_launch_dependents();
-
 #pragma unroll
     for (int c = 0; c < kWinMaxChunks; ++c) {
         const int ch = threadIdx.x + c * blockDim.x;
@@ -102,7 +129,7 @@ __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_con
             }
             // x is kept as a pair of bf16 planes, x = hi + lo, so the GEMM that consumes it
             // sees ~16 mantissa bits although its operands are bf16
-            uint4 g = ld_cached(p.gain + ch);
+            const uint4 g = gn[c];
             float xv[8];
             xv[0] = v[c][0] * inv * bf_lo(g.x); xv[1] = v[c][1] * inv * bf_hi(g.x);
             xv[2] = v[c][2] * inv * bf_lo(g.y); xv[3] = v[c][3] * inv * bf_hi(g.y);
@@ -117,6 +144,7 @@ __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_con
             p.x_bf16[p.x_plane + row_off + ch] = lo;
         }
     }
+    trace_end(p.trace);
 }
 
 cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
@@ -133,6 +161,7 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
     p.x_bf16 = reinterpret_cast<uint4 *>(a.x_bf16);
     p.x_plane = a.x_plane_elems / 8;
     p.H = a.H;
+    p.trace = a.trace;
     const int chunks = a.H / 8;
     int threads = (chunks + kWinMaxChunks - 1) / kWinMaxChunks;
     if (chunks <= 1024)
@@ -149,8 +178,10 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
     cfg.attrs = at;
     cfg.numAttrs = pdl_attr(at);
     if (a.resid_is_f32)
-        return cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<true>, p);
-    return cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<false>, p);
+        return a.part0_is_f32 ? cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<true, true>, p)
+                              : cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<true, false>, p);
+    return a.part0_is_f32 ? cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<false, true>, p)
+                          : cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<false, false>, p);
 }
 
 }  // namespace prsv

@@ -1,0 +1,226 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on
+the same seeded inputs.  Tolerance (written in gpu_util.tolerance_ok):
+|gpu - ref| <= 2e-2 * min(1, rms(ref)) + 1e-2 * |ref| per element."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2501_08192_b200 import binding as P
+from paper_2501_08192_b200 import inputs as I
+
+import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+def full_check(oracle, shape, flags=0, budget=None):
+    t = I.make_layers(shape, 1)[0]
+    ref = oracle.layer_step(shape, t)
+    dl = G.DeviceLayer(shape, t, flags=flags)
+    try:
+        if budget is not None:
+            dl.layer.set_prefetch_bytes(budget)
+        k_before, v_before = G.cuda_to_bits(dl.k_cache), G.cuda_to_bits(dl.v_cache)
+        dl.run()
+        assert dl.layer.last_status() == P.PRESERVE_OK
+        out, inter = dl.outputs(), dl.intermediates()
+        k_new, v_new = dl.appended_kv()
+        for name in ("h", "x", "q", "o", "x2", "a"):
+            G.assert_close(inter[name], ref[name], f"{shape.name}:{name}")
+        G.assert_close(k_new, ref["k_new"], f"{shape.name}:k_new")
+        G.assert_close(v_new, ref["v_new"], f"{shape.name}:v_new")
+        for name in ("attn_partial", "h2", "mlp_partial"):
+            G.assert_close(out[name], ref[name], f"{shape.name}:{name}")
+        for g in (dl.residual_out, dl.mlp_out, dl.attn_out):
+            assert g.guards_intact(), "write outside an output buffer"
+        # append: exactly one slot per (sequence, kv head) changed in each cache
+        k_after, v_after = G.cuda_to_bits(dl.k_cache), G.cuda_to_bits(dl.v_cache)
+        mask = np.ones(k_before.shape, bool)
+        for b in range(shape.batch):
+            mask[b, :, int(t["ctx_len"][b])] = False
+        assert np.array_equal(k_before[mask], k_after[mask]) and np.array_equal(v_before[mask], v_after[mask])
+        assert not np.isnan(I.bf16_bits_to_f32(k_after[~mask])).any()
+        return dl.output_bits()
+    finally:
+        dl.close()
+
+
+SMALL = [
+    I.small_shape(name="b1_mha", batch=1, tp_degree=1, ctx=37, n_q_heads=2, n_kv_heads=2, seed=12),
+    I.small_shape(name="b2", batch=2, ctx=64, seed=40),
+    I.small_shape(name="b3", batch=3, ctx=200, seed=11),
+    I.small_shape(name="b4_g4", batch=4, ctx=63, n_q_heads=4, n_kv_heads=1, seed=41),
+    I.small_shape(name="b5", batch=5, ctx=127, seed=42),
+    I.small_shape(name="b8_ragged", batch=8, ctx=300, ctx_min=10, tp_degree=4, seed=13),
+    I.small_shape(name="b12_g8", batch=12, ctx=130, n_q_heads=8, n_kv_heads=1, seed=14),
+    I.small_shape(name="b15_g16", batch=15, ctx=65, n_q_heads=16, n_kv_heads=1, tp_degree=16, seed=43),
+    I.small_shape(name="b16", batch=16, ctx=100, seed=15),
+    I.small_shape(name="b33_ragged_g8", batch=33, ctx=300, ctx_min=1, n_q_heads=8, n_kv_heads=1, tp_degree=3, seed=16),
+    I.small_shape(name="b64", batch=64, hidden=1024, ffn=1152, ctx=64, seed=17),
+    I.small_shape(name="b128", batch=128, hidden=256, ffn=128, ctx=20, n_q_heads=2, n_kv_heads=2, seed=44),
+    I.small_shape(name="no_rope", batch=3, ctx=90, rope_theta=0.0, seed=45),
+    I.small_shape(name="ctx0", batch=2, ctx=0, seed=46),
+    I.small_shape(name="ctx63", batch=2, ctx=63, seed=47),     # 64 keys: exactly one tile
+    I.small_shape(name="long_multi_tile_items", batch=2, n_q_heads=4, n_kv_heads=2, ctx=20000, seed=18),
+]
+
+
+@pytest.mark.parametrize("shape", SMALL, ids=[s.name for s in SMALL])
+def test_small_shapes_match_oracle(oracle, shape):
+    full_check(oracle, shape)
+
+
+@pytest.mark.parametrize("idx", [0, 1, 3, 4])
+def test_benchmark_configs_match_oracle(oracle, idx):
+    full_check(oracle, I.CONFIGS[idx])
+
+
+def test_config3_chain_of_four_matches_oracle(oracle):
+    shape = I.CONFIGS[2]
+    layers = I.make_layers(shape)
+    refs = oracle.layer_chain(shape, layers)
+    dls = [G.DeviceLayer(shape, t) for t in layers]
+    try:
+        P.preserve_decode_chain([d.layer for d in dls], [d.io for d in dls], link=True)
+        for i, (dl, ref) in enumerate(zip(dls, refs)):
+            assert dl.layer.last_status() == P.PRESERVE_OK
+            out = dl.outputs()
+            for name in ("attn_partial", "h2", "mlp_partial"):
+                G.assert_close(out[name], ref[name], f"chain layer {i}:{name}")
+    finally:
+        for d in dls:
+            d.close()
+
+
+def test_prefetch_never_changes_results(oracle):
+    """Outputs are bit-identical across prefetch off, on, every swept budget, both planning
+    modes, graph replay vs direct launches, and repeated runs."""
+    for shape in (I.small_shape(name="det_gemv", batch=8, ctx=500, ctx_min=20, seed=50),
+                  I.small_shape(name="det_tc", batch=32, ctx=700, ctx_min=5, hidden=1024, ffn=512, seed=51),
+                  I.CONFIGS[1]):
+        t = I.make_layers(shape, 1)[0]
+        base = None
+        for flags in (0, P.FLAG_NO_GRAPH):
+            dl = G.DeviceLayer(shape, t, flags=flags)
+            try:
+                l2 = int(dl.layer.get_info().l2_bytes)
+                for mode in (P.PLAN_TRUNCATE, P.PLAN_WHOLE_NODE):
+                    dl.layer.set_plan_mode(mode)
+                    for frac in (0.0, 1 / 16, 1 / 4, 1 / 2, 1.0, 2.0):
+                        dl.layer.set_prefetch_bytes(int(frac * l2))
+                        for _ in range(2):
+                            dl.run()
+                            bits = dl.output_bits()
+                            if base is None:
+                                base = bits
+                            for k in base:
+                                assert np.array_equal(base[k], bits[k]), (shape.name, flags, mode, frac, k)
+            finally:
+                dl.close()
+
+
+def test_host_buffer_entry_point_matches_device_path(oracle):
+    shape = I.small_shape(name="host_io", batch=6, ctx=150, ctx_min=3, seed=52)
+    t = I.make_layers(shape, 1)[0]
+    dl = G.DeviceLayer(shape, t)
+    try:
+        dl.run()
+        want = dl.output_bits()
+        # restore the caches (the step appended), then run from pinned host buffers
+        dl.k_cache.copy_(G.bits_to_cuda(t["k_cache"]))
+        dl.v_cache.copy_(G.bits_to_cuda(t["v_cache"]))
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
+        parts = [pin(t["partials_in"][p]) for p in range(shape.tp_degree)]
+        peers = [pin(t["attn_peer_partials"][p]) for p in range(shape.tp_degree - 1)]
+        resid = pin(t["residual_in"])
+        r_out = torch.zeros((shape.batch, shape.hidden), dtype=torch.int16).pin_memory()
+        m_out = torch.zeros((shape.batch, shape.hidden), dtype=torch.int16).pin_memory()
+        hio = P.make_host_io(dl.cfg, shape.batch, dl.ctx_host, parts, peers, resid, dl.k_cache, dl.v_cache,
+                             r_out, m_out)
+        dl.layer.decode_step_host(hio)
+        torch.cuda.synchronize()
+        assert np.array_equal(r_out.numpy().view(np.uint16), want["h2"])
+        assert np.array_equal(m_out.numpy().view(np.uint16), want["mlp_partial"])
+    finally:
+        dl.close()
+
+
+def test_smaller_batch_than_max_batch(oracle):
+    shape = I.small_shape(name="b5_of_12", batch=5, ctx=77, seed=53)
+    t = I.make_layers(shape, 1)[0]
+    ref = oracle.layer_step(shape, t)
+    for max_batch in (12, 40):                     # GEMV path and tensor path
+        dl = G.DeviceLayer(shape, t, max_batch=max_batch)
+        try:
+            # caches are [max_batch, ...] for the library: rebuild them at that size
+            cap, d, nkv = shape.kv_capacity, shape.head_dim, shape.n_kv_heads
+            kc = torch.zeros((max_batch, nkv, cap, d), dtype=torch.bfloat16, device="cuda")
+            vc = torch.zeros_like(kc)
+            kc[:shape.batch] = G.bits_to_cuda(t["k_cache"])
+            vc[:shape.batch] = G.bits_to_cuda(t["v_cache"])
+            dl.k_cache, dl.v_cache = kc, vc
+            dl.io = dl.layer.make_io(shape.batch, dl.ctx_dev, dl.ctx_host, dl.partials, dl.peers, dl.residual,
+                                     kc, vc, dl.residual_out.t, dl.mlp_out.t, dl.attn_out.t)
+            dl.run()
+            assert dl.layer.last_status() == P.PRESERVE_OK
+            out = dl.outputs()
+            for name in ("attn_partial", "h2", "mlp_partial"):
+                G.assert_close(out[name], ref[name], f"max_batch {max_batch}:{name}")
+        finally:
+            dl.close()
+
+
+def test_argument_validation_on_device():
+    shape = I.small_shape(name="args", batch=2, ctx=10, seed=54)
+    t = I.make_layers(shape, 1)[0]
+    dl = G.DeviceLayer(shape, t)
+    try:
+        import ctypes as C
+        lib = P.lib()
+        io = dl.io
+        good_batch = io.batch
+        io.batch = 3                                     # > max_batch
+        assert lib.preserve_decode_step(dl.layer.handle, C.byref(io), 0) == P.PRESERVE_ESHAPE
+        io.batch = good_batch
+        keep = io.residual_in
+        io.residual_in = keep + 2                        # misaligned
+        assert lib.preserve_decode_step(dl.layer.handle, C.byref(io), 0) == P.PRESERVE_EALIGN
+        io.residual_in = None
+        assert lib.preserve_decode_step(dl.layer.handle, C.byref(io), 0) == P.PRESERVE_EINVAL
+        io.residual_in = keep
+        bad_ctx = np.array([5, shape.ctx + 1], np.int32)  # beyond max_ctx
+        old = io.ctx_len_host
+        io.ctx_len_host = bad_ctx.ctypes.data
+        assert lib.preserve_decode_step(dl.layer.handle, C.byref(io), 0) == P.PRESERVE_ESHAPE
+        io.ctx_len_host = old
+        assert lib.preserve_decode_step(None, C.byref(io), 0) == P.PRESERVE_EINVAL
+        dl.run()                                         # still usable afterwards
+        assert dl.layer.last_status() == P.PRESERVE_OK
+    finally:
+        dl.close()
+    for bad in (replace(shape, head_dim=64), replace(shape, hidden=520), replace(shape, ffn=100),
+                replace(shape, n_q_heads=3), replace(shape, tp_degree=17)):
+        with pytest.raises(P.PreserveError) as e:
+            G.DeviceLayer(bad, t)
+        assert e.value.code == P.PRESERVE_ESHAPE
+
+
+def test_info_reports_plan_and_bytes():
+    shape = I.CONFIGS[1]
+    t = I.make_layers(shape, 1)[0]
+    dl = G.DeviceLayer(shape, t)
+    try:
+        dl.layer.set_plan_mode(P.PLAN_WHOLE_NODE)
+        dl.layer.set_prefetch_bytes(32 << 20)
+        dl.run()
+        torch.cuda.synchronize()
+        info = dl.layer.get_info()
+        assert list(info.weight_bytes) == [6291456, 4194304, 29360128, 14680064]
+        assert info.kv_bytes == 16777216
+        assert [list(r) for r in info.planned_bytes] == [[6291456, 16777216, 4194304], [29360128, 0, 0]]
+        assert info.algorithmic_bytes == P.preserve_algorithmic_bytes(dl.cfg, shape.batch, shape.batch * shape.ctx)
+        assert info.sm_count > 0 and info.l2_bytes > 0 and info.uses_tensor_path == 0
+    finally:
+        dl.close()
