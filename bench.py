@@ -203,37 +203,67 @@ def run_ours(args):
     alg = int(P.preserve_algorithmic_bytes(cfg, shape.batch, sum_ctx))
     assert alg > 0
 
+    def set_delay(ns):
+        for L in layers:
+            L.set_window_delay_ns(ns)
+
     # ---- headline: default prefetch setting, with clocks sampled during the timed region
     sampler = ClockSampler(local_rank)
     sampler.start()
     set_budget(default_budget)
     ms_on, per_on = time_steps(chain_step, args.steps, args.warmup)
     clocks = sampler.summary()
-    # ---- prefetch off, and the sweep over the budget (fewer steps each)
+    # ---- prefetch off (vanilla execution), early launch only (budget of one byte: nothing planned for
+    # L2), and the sweep over the L2 budget (fewer steps each)
     set_budget(0)
     ms_off, per_off = time_steps(chain_step, args.steps, args.warmup)
+    set_budget(1)
+    ms_early, _ = time_steps(chain_step, max(10, args.steps // 2), 3)
     sweep = []
     if not args.no_sweep:
         for f in SWEEP_FRACS:
             set_budget(int(f * l2))
             ms, _ = time_steps(chain_step, max(10, args.steps // 4), 3)
             sweep.append({"frac_of_l2": round(f, 4), "us_per_layer": round(ms * 1e3 / R, 3)})
+    # ---- modelled communication latency added to every window (the single-GPU stand-in has none)
+    modelled = []
+    if not args.no_sweep:
+        for delay_us in (10, 20):
+            set_delay(delay_us * 1000)
+            row = {"window_delay_us": delay_us}
+            for name, b in (("off", 0), ("early_launch_only", 1), ("on", default_budget)):
+                set_budget(b)
+                ms, _ = time_steps(chain_step, max(10, args.steps // 4), 3)
+                row[name + "_us_per_layer"] = round(ms * 1e3 / R, 3)
+            modelled.append(row)
+        set_delay(0)
     # ---- end to end through the host-buffer entry point
     set_budget(default_budget)
     ms_e2e, _ = time_steps(host_step, args.steps, args.warmup)
     h2d = (2 * shape.tp_degree) * shape.batch * shape.hidden * 2 + shape.batch * 4
     d2h = 2 * shape.batch * shape.hidden * 2
-    # ---- per-kernel times (direct launches with events on the launching stream), cold L2 by rotation
+    # ---- per-kernel times: each main-stream kernel alone, launched back to back over the R layer
+    # instances (cold L2 by rotation) from a captured graph, CUDA events on the launching stream
+    # around many replays.  Launches of one kernel are independent of each other, so this is the
+    # kernel's own duration including its launch hand-over, not a dependency chain.
     kms = np.zeros(len(P.KERNEL_NAMES))
-    reps = 0
     with torch.cuda.stream(stream):
-        for rep in range(1 + args.profile_reps):
+        chain_step()
+        torch.cuda.synchronize()
+    for k in range(len(P.KERNEL_NAMES)):
+        def one():
             for L, io in zip(layers, ios):
-                ms = L.profile_step(io, stream)
-                if rep > 0:
-                    kms += np.array(ms)
-                    reps += 1
-    kms /= max(reps, 1)
+                L.run_kernel(io, k, stream)
+        with torch.cuda.stream(stream):
+            one()
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for _ in range(4):
+                    one()
+        ms, _ = time_steps(lambda: g.replay(), 10, 3)
+        kms[k] = ms / (4 * R)
+        del g
     status = max(L.last_status() for L in layers)
 
     peak, peak_src = load_peaks()
@@ -243,7 +273,9 @@ def run_ours(args):
     gbs = lambda ms: alg * R / (ms * 1e-3) / 1e9
     us = lambda ms: ms * 1e3 / R
     best = min(sweep, key=lambda e: e["us_per_layer"]) if sweep else None
-    launches_per_layer = len(P.KERNEL_NAMES) + (2 if default_budget > 0 else 0)
+    info = layers[0].get_info()
+    n_pf = sum(1 for w in range(2) if sum(info.planned_bytes[w]) > 0)
+    launches_per_layer = len(P.KERNEL_NAMES) + n_pf
     out = {
         "metric": METRIC, "value": round(gbs(ms_on) * world, 2), "unit": "GB/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_on, 5),
@@ -263,20 +295,26 @@ def run_ours(args):
         "frac_of_nominal_8TBs": round(gbs(ms_on) / 8000.0, 4),
         "frac_of_measured_copy_bw": round(gbs(ms_on) / peak, 4),
         "prefetch": {"on_us_per_layer": round(us(ms_on), 3), "off_us_per_layer": round(us(ms_off), 3),
+                     "early_launch_only_us_per_layer": round(us(ms_early), 3),
                      "on_gbs": round(gbs(ms_on), 1), "off_gbs": round(gbs(ms_off), 1),
                      "speedup_on_vs_off": round(ms_off / ms_on, 4),
                      "p10_p50_p90_on_us": [round(float(np.percentile(per_on, q)) * 1e3 / R, 3) for q in (10, 50, 90)],
                      "p10_p50_p90_off_us": [round(float(np.percentile(per_off, q)) * 1e3 / R, 3) for q in (10, 50, 90)],
-                     "sweep": sweep, "best": best,
+                     "meaning": "off = vanilla execution (budget 0: no early launch, no side stream); "
+                                "early_launch_only = consumer kernels stage operands in shared memory during "
+                                "the window; on = that plus the L2 prefetch kernel at the default budget",
+                     "sweep": sweep, "best": best, "modelled_window": modelled,
                      "paper_context": "up to 1.6x end to end on 8x Ascend 910B, int8 (another machine; not a target)"},
         "e2e": {"value": round(gbs(ms_e2e) * world, 2), "unit": "GB/s", "us_per_layer": round(us(ms_e2e), 3),
                 "h2d_bytes_per_step": h2d * R, "d2h_bytes_per_step": d2h * R},
         "gpu_launches": launches_per_layer * R * args.steps,
         "kernels_us": {n: round(float(v) * 1e3, 3) for n, v in zip(P.KERNEL_NAMES, kms)},
+        "kernels_gbs": {n: round(kb[i] / (float(kms[i]) * 1e-3) / 1e9, 1) for i, n in enumerate(P.KERNEL_NAMES)},
         "roofline": {"bound": "hbm", "kernel": P.KERNEL_NAMES[dom], "achieved": round(achieved, 1),
                      "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
                      "traffic": NCU_TRAFFIC.get((P.KERNEL_NAMES[dom], args.config)), "peak_source": peak_src,
-                     "algorithmic_bytes_per_launch": kb[dom]},
+                     "algorithmic_bytes_per_launch": kb[dom],
+                     "how": "kernel launched alone, back to back over the rotation, from a captured graph"},
         "clocks": clocks, "device_status": status,
     }
     if rank == 0:
@@ -361,7 +399,6 @@ def main():
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--config", type=int, default=1, help="index into the five benchmark configurations")
     ap.add_argument("--rotation", type=int, default=0, help="layer instances per step (0 = sized from L2)")
-    ap.add_argument("--profile-reps", type=int, default=3)
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     args = ap.parse_args()

@@ -73,6 +73,8 @@ extern "C" {
 /* flags for preserve_layer_config_t.flags */
 #define PRESERVE_FLAG_NO_GRAPH   1u /* launch kernels directly instead of replaying a CUDA graph     */
 #define PRESERVE_FLAG_PERSIST_L2 2u /* mark prefetched lines as persisting (access-policy window)    */
+#define PRESERVE_FLAG_NO_EARLY_LAUNCH 4u /* ablation: prefetch into L2 only; consumer kernels are not
+                                       launched early to stage operands in shared memory              */
 
 typedef struct preserve_layer preserve_layer_t;   /* opaque, owned by the library */
 
@@ -161,14 +163,27 @@ typedef struct {
  * arena laid out in the order the kernels consume them, allocates workspaces,
  * a side stream and events on the CURRENT device.  The weight pointers may be
  * freed after the call returns.  *out is NULL on failure.
- * The prefetch budget starts at the device's L2 size, mode PRESERVE_PLAN_TRUNCATE. */
+ * The prefetch budget starts at a quarter of the device's L2 size, mode PRESERVE_PLAN_TRUNCATE. */
 PRESERVE_API int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer_weights_t *w,
                         preserve_layer_t **out);
 
 /* Upper limit, in bytes, on what one window's prefetch may bring into L2
- * (Algorithm 1's C; Section 3 "L2 capacity requirements").  0 switches the
- * prefetch off entirely: no side-stream work is queued. */
+ * (Algorithm 1's C; Section 3 "L2 capacity requirements").
+ * 0 = vanilla execution (Section 3, "Vanilla execution"): nothing is fetched ahead of
+ * the data dependency - no side-stream work, and every kernel starts only after its
+ * predecessor has completed.
+ * > 0 = the read-only operands of the operators after a window are brought on chip
+ * while the window runs, in two tiers: (1) the consumer kernels are launched early
+ * (programmatic dependent launch) and stage the leading part of their weights / cached
+ * K and V in shared memory before they wait for the window's result; (2) a side-stream
+ * kernel prefetches the planned byte ranges, up to this limit per window, into L2. */
 PRESERVE_API int preserve_set_prefetch_bytes(preserve_layer_t *layer, size_t bytes_per_window);
+
+/* Modelled communication latency: every window kernel additionally waits (bounded, on
+ * the GPU's global timer) until `ns` nanoseconds after its start before it delivers its
+ * result, standing in for the network time of a real allreduce, which the single-GPU
+ * stand-in does not have.  0 (default) = no added wait.  At most 1,000,000. */
+PRESERVE_API int preserve_set_window_delay_ns(preserve_layer_t *layer, int32_t ns);
 
 /* PRESERVE_PLAN_WHOLE_NODE (Algorithm 1 as printed) or PRESERVE_PLAN_TRUNCATE. */
 PRESERVE_API int preserve_set_plan_mode(preserve_layer_t *layer, int mode);

@@ -17,7 +17,7 @@ PRESERVE_OK = 0
 PRESERVE_EINVAL, PRESERVE_EALIGN, PRESERVE_ESHAPE, PRESERVE_ENOMEM = -1, -2, -3, -4
 PRESERVE_ECUDA, PRESERVE_EARCH, PRESERVE_ETIMEOUT = -5, -6, -7
 PLAN_WHOLE_NODE, PLAN_TRUNCATE = 0, 1
-FLAG_NO_GRAPH, FLAG_PERSIST_L2 = 1, 2
+FLAG_NO_GRAPH, FLAG_PERSIST_L2, FLAG_NO_EARLY_LAUNCH = 1, 2, 4
 
 EXPORTS = (
     "preserve_layer_init", "preserve_set_prefetch_bytes", "preserve_set_plan_mode", "preserve_decode_step",
@@ -25,6 +25,7 @@ EXPORTS = (
     "preserve_last_cuda_error", "preserve_debug_copy", "preserve_layer_destroy", "preserve_strerror",
     "preserve_plan_window", "preserve_algorithmic_bytes", "preserve_profile_step",
     "preserve_run_kernel", "preserve_set_trace", "preserve_read_trace",
+    "preserve_set_window_delay_ns",
 )
 KERNEL_NAMES = ("window_a", "qkv_proj", "attn_splitkv", "attn_merge", "o_proj", "window_b", "gate_up_proj",
                 "down_proj")
@@ -80,6 +81,7 @@ def lib() -> C.CDLL:
         L.preserve_layer_init.argtypes = [C.POINTER(LayerConfig), C.POINTER(LayerWeights), C.POINTER(C.c_void_p)]
         L.preserve_set_prefetch_bytes.argtypes = [C.c_void_p, C.c_size_t]
         L.preserve_set_plan_mode.argtypes = [C.c_void_p, C.c_int]
+        L.preserve_set_window_delay_ns.argtypes = [C.c_void_p, C.c_int32]
         L.preserve_decode_step.argtypes = [C.c_void_p, C.POINTER(StepIO), C.c_void_p]
         L.preserve_decode_chain.argtypes = [C.POINTER(C.c_void_p), C.c_int32, C.POINTER(StepIO), C.c_int32,
                                             C.c_void_p]
@@ -177,6 +179,9 @@ class Layer:
 
     def set_prefetch_bytes(self, n: int) -> None:
         _check(lib().preserve_set_prefetch_bytes(self.handle, n), "preserve_set_prefetch_bytes")
+
+    def set_window_delay_ns(self, ns: int) -> None:
+        _check(lib().preserve_set_window_delay_ns(self.handle, ns), "preserve_set_window_delay_ns")
 
     def set_plan_mode(self, mode: int) -> None:
         _check(lib().preserve_set_plan_mode(self.handle, mode), "preserve_set_plan_mode")

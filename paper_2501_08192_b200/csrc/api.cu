@@ -98,6 +98,10 @@ struct preserve_layer {
 
     cudaStream_t side;
     cudaEvent_t ev_a, ev_b, ev_join;
+    bool side_pending;           // prefetch work queued on the side stream and not yet joined
+    bool no_early;               // ablation: prefetch into L2 only, no early launch of the consumer kernels
+    int window_delay_ns;         // modelled extra duration of each communication window
+    bool pdl_env;                // PRESERVE_PDL=0 switches programmatic dependent launch off entirely
 
     size_t budget;
     int plan_mode;
@@ -333,6 +337,9 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
     plan_window(nodes_b, 2, L->budget, L->plan_mode, L->planned[1]);
     L->planned[1][2] = 0;
     L->alg_bytes = L->wbytes[0] + L->wbytes[1] + L->wbytes[2] + L->wbytes[3] + L->kv_bytes + activation_bytes(c, B);
+    // budget 0 = vanilla execution: every kernel starts after its predecessor has completed and
+    // nothing is fetched ahead of the dependency
+    g_pdl = (L->budget > 0 && !L->no_early && L->pdl_env) ? 1 : 0;
     const bool pf_a = L->only < 0 && L->planned[0][0] + L->planned[0][1] + L->planned[0][2] > 0;
     const bool pf_b = L->only < 0 && L->planned[1][0] + L->planned[1][1] > 0;
 #define WANT(k) (L->only < 0 || L->only == (k))
@@ -403,6 +410,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         w.x_plane_elems = (size_t)L->rows * H;
         w.B = B; w.H = H;
         w.trace = TRACE(0);
+        w.delay_ns = L->window_delay_ns;
         CK(L, launch_window(w, s));
     }
     // ---- QKV projection + rotary embedding + KV append
@@ -438,7 +446,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         // Work items = runs of 64-key tiles.  Aim at one item per CTA when the whole cache is small
         // (per-item overhead dominates) and at up to four per CTA when it is large (balance under
         // ragged lengths); depends only on the lengths and the SM count.
-        uint64_t mult = total_tiles / ((uint64_t)L->attn_grid * 4);
+        uint64_t mult = total_tiles / ((uint64_t)L->attn_grid * 3);
         mult = mult < 1 ? 1 : (mult > 4 ? 4 : mult);
         uint64_t tpi = (total_tiles + (uint64_t)L->attn_grid * mult - 1) / ((uint64_t)L->attn_grid * mult);
         a.tiles_per_item = tpi < 1 ? 1 : (int)tpi;
@@ -496,6 +504,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         w.x_plane_elems = (size_t)L->rows * H;
         w.B = B; w.H = H;
         w.trace = TRACE(5);
+        w.delay_ns = L->window_delay_ns;
         CK(L, launch_window(w, s));
     }
     // ---- gate/up projection + SwiGLU, down projection
@@ -523,12 +532,24 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
 #undef MARK
 #undef WANT
 #undef TRACE
-    // ---- join the side stream
-    if (pf_a || pf_b) {
+    // ---- the side stream is joined once, after the last layer of the call (the prefetch kernels only
+    // read, so nothing on the main stream has to wait for them earlier)
+    if (pf_a || pf_b)
+        L->side_pending = true;       // joined by run_steps after the last layer
+    (void)d;
+    return PRESERVE_OK;
+}
+
+int join_side_streams(preserve_layer *const *layers, int n, cudaStream_t s)
+{
+    for (int i = 0; i < n; ++i) {
+        preserve_layer *L = layers[i];
+        if (!L->side_pending)
+            continue;
         CK(L, cudaEventRecord(L->ev_join, L->side));
         CK(L, cudaStreamWaitEvent(s, L->ev_join, 0));
+        L->side_pending = false;
     }
-    (void)d;
     return PRESERVE_OK;
 }
 
@@ -548,6 +569,7 @@ uint64_t step_key(const preserve_layer *L, const StepPtrs &sp, uint64_t h)
     h = fnv1a(h, &sp.resid_f32, 2 * sizeof(int));
     const int tr = L->tracing ? 1 : 0;
     h = fnv1a(h, &tr, sizeof(int));
+    h = fnv1a(h, &L->window_delay_ns, sizeof(int));
     return h;
 }
 
@@ -562,7 +584,7 @@ int run_steps(preserve_layer *const *layers, const StepPtrs *sps, int n, cudaStr
             if (rc)
                 return rc;
         }
-        return PRESERVE_OK;
+        return join_side_streams(layers, n, s);
     }
     uint64_t key = 1469598103934665603ull;
     for (int i = 0; i < n; ++i)
@@ -584,12 +606,14 @@ int run_steps(preserve_layer *const *layers, const StepPtrs *sps, int n, cudaStr
             if (rc)
                 return rc;
         }
-        return PRESERVE_OK;
+        return join_side_streams(layers, n, s);
     }
     CK(L0, cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal));
     int rc = PRESERVE_OK;
     for (int i = 0; i < n && rc == PRESERVE_OK; ++i)
         rc = enqueue_step(layers[i], sps[i], s);
+    if (rc == PRESERVE_OK)
+        rc = join_side_streams(layers, n, s);
     cudaGraph_t graph = nullptr;
     cudaError_t e = cudaStreamEndCapture(s, &graph);
     if (rc != PRESERVE_OK) {
@@ -736,17 +760,17 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     L->tensor_path = (cfg->max_batch >= 16 && !(force && force[0] == '1')) ||
                      (force_tc && force_tc[0] == '1' && cfg->ffn % 128 == 0);
     const char *pdl = getenv("PRESERVE_PDL");
-    if (pdl)
-        g_pdl = pdl[0] == '1';
+    L->pdl_env = !(pdl && pdl[0] == '0');
+    L->no_early = (cfg->flags & PRESERVE_FLAG_NO_EARLY_LAUNCH) != 0;
     const char *pfm = getenv("PRESERVE_PREFETCH_MODE");
     const char *pfc = getenv("PRESERVE_PREFETCH_CHUNK");
     if (pfm || pfc)
-        set_prefetch_kernel_mode(pfm ? atoi(pfm) : 0, pfc ? (uint32_t)atoi(pfc) : 4096u);
+        set_prefetch_kernel_mode(pfm ? atoi(pfm) : 2, pfc ? (uint32_t)atoi(pfc) : 4096u);
     const char *pfn = getenv("PRESERVE_PREFETCH_CTAS");
-    L->prefetch_ctas = pfn ? atoi(pfn) : 8;
+    L->prefetch_ctas = pfn ? atoi(pfn) : 64;
     if (L->prefetch_ctas < 1)
         L->prefetch_ctas = 1;
-    L->budget = (size_t)L->l2_bytes;
+    L->budget = (size_t)L->l2_bytes / 4;
     L->plan_mode = PRESERVE_PLAN_TRUNCATE;
 
 #define CKI(expr)                                   \
@@ -822,7 +846,7 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     CKI(cudaMemset(L->o, 0, 2 * Rq * 2));
     CKI(cudaMemset(L->x2, 0, 2 * RH * 2));
     CKI(cudaMemset(L->a, 0, 2 * RF * 2));
-    L->attn_grid = L->sm_count;
+    L->attn_grid = 2 * L->sm_count;      // two persistent attention CTAs per SM
     L->max_items = L->attn_grid * 4 + B * c.n_kv_heads + 8;
     CKI(cudaMalloc(&L->part_o, (size_t)L->max_items * 4 * L->group * kHeadDim * 4));
     CKI(cudaMalloc(&L->part_ml, (size_t)L->max_items * 4 * L->group * 2 * 4));
@@ -862,6 +886,14 @@ int preserve_set_prefetch_bytes(preserve_layer_t *L, size_t bytes_per_window)
     if (!L)
         return PRESERVE_EINVAL;
     L->budget = bytes_per_window;
+    return PRESERVE_OK;
+}
+
+int preserve_set_window_delay_ns(preserve_layer_t *L, int32_t ns)
+{
+    if (!L || ns < 0 || ns > 1000000)
+        return PRESERVE_EINVAL;
+    L->window_delay_ns = ns;
     return PRESERVE_OK;
 }
 
@@ -973,6 +1005,12 @@ int preserve_profile_step(preserve_layer_t *L, const preserve_step_io_t *io, voi
     L->profiling = false;
     if (rc)
         return rc;
+    {
+        preserve_layer *one[1] = {L};
+        rc = join_side_streams(one, 1, s);
+        if (rc)
+            return rc;
+    }
     CK(L, cudaStreamSynchronize(s));
     for (int i = 0; i < PRESERVE_N_KERNELS; ++i)
         CK(L, cudaEventElapsedTime(&kernel_ms[i], L->prof[i], L->prof[i + 1]));

@@ -8,9 +8,9 @@
 // (sequence, kv head) is one contiguous run and a tile of 64 keys is two TMA
 // boxes of 64 x 64 bf16 (128-byte swizzle) per tensor.
 //
-// Persistent CTAs (one per SM) walk a static list of work items = (sequence,
+// Persistent CTAs (two per SM) walk a static list of work items = (sequence,
 // kv head, run of `tiles_per_item` tiles) in address order.  Warp 4 is the
-// producer: one lane issues the TMA loads into a 4-stage ring guarded by
+// producer: one lane issues the TMA loads into a 3-stage ring guarded by
 // full/empty mbarriers (all waits bounded).  Warps 0-3 each own 16 of a tile's
 // 64 keys: S = Q K^T with mma.sync (Q rows = query heads padded to 16, from
 // registers; K via ldmatrix), online softmax in fp32 with exp2, O += P V (V via
@@ -23,7 +23,7 @@
 namespace prsv {
 
 constexpr int kTileKeys = 64;
-constexpr int kStages = 4;
+constexpr int kStages = 3;                            // 96 KiB ring: two CTAs per SM
 constexpr int kConsumerWarps = 4;
 constexpr int kAttnThreads = (kConsumerWarps + 1) * 32;
 constexpr int kHalfBytes = kTileKeys * 128;            // one 64x64 bf16 box
@@ -97,7 +97,7 @@ __device__ __forceinline__ int find_stream(const int *item_base, int streams, in
     return lo;
 }
 
-__global__ void __launch_bounds__(kAttnThreads, 1) k_attn_decode_splitkv(const __grid_constant__ AttnParams p)
+__global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const __grid_constant__ AttnParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     AttnSmem &sm = *reinterpret_cast<AttnSmem *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -125,6 +125,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_attn_decode_splitkv(const _
             // Cached keys and values are read-only during the step, so their tiles are fetched
             // right away, even while the QKV projection is still running; only a sequence's last
             // tile (it holds the entry appended by that projection) has to wait for it.
+            const uint64_t pol = policy_evict_first();   // each cached byte is read once per step
             uint32_t it = 0;
             bool ok = true, waited = false;
             for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
@@ -144,10 +145,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_attn_decode_splitkv(const _
                     mbar_expect_tx(&sm.full[st], kStageBytes);
                     const int row = sidx * p.cap + tile * kTileKeys;
                     uint8_t *dst = sm.stage[st];
-                    tma_load_2d(dst, &p.k_map, 0, row, &sm.full[st]);
-                    tma_load_2d(dst + kHalfBytes, &p.k_map, 64, row, &sm.full[st]);
-                    tma_load_2d(dst + 2 * kHalfBytes, &p.v_map, 0, row, &sm.full[st]);
-                    tma_load_2d(dst + 3 * kHalfBytes, &p.v_map, 64, row, &sm.full[st]);
+                    tma_load_2d_hint(dst, &p.k_map, 0, row, &sm.full[st], pol);
+                    tma_load_2d_hint(dst + kHalfBytes, &p.k_map, 64, row, &sm.full[st], pol);
+                    tma_load_2d_hint(dst + 2 * kHalfBytes, &p.v_map, 0, row, &sm.full[st], pol);
+                    tma_load_2d_hint(dst + 3 * kHalfBytes, &p.v_map, 64, row, &sm.full[st], pol);
                 }
             }
         }

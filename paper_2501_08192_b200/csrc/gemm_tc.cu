@@ -125,11 +125,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
             // Weights never depend on earlier kernels, the activations do: fill the whole ring
             // with weight tiles first (they stream in while the previous kernel finishes), then
             // wait for the previous kernel and add the activation tiles.
+            const uint64_t pol = policy_evict_first();   // every weight byte is read once per step
             const int n_kb = kb1 - kb0;
             const int pre = n_kb < p.stages ? n_kb : p.stages;
             for (int i = 0; i < pre; ++i) {
                 mbar_expect_tx(&full[i], stage_bytes);
-                tma_load_2d(smem + (size_t)i * stage_bytes, &p.w_map, (kb0 + i) * kTcBlockK, tile * kTcTileM, &full[i]);
+                tma_load_2d_hint(smem + (size_t)i * stage_bytes, &p.w_map, (kb0 + i) * kTcBlockK, tile * kTcTileM,
+                                 &full[i], pol);
             }
             pdl_wait();
             trace_waited(p.trace);
@@ -142,7 +144,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
                 if (!mbar_wait(&empty[st], ph ^ 1, p.status, ST_TIMEOUT_EMPTY)) { poisoned = 1; break; }
                 uint8_t *a_dst = smem + (size_t)st * stage_bytes;
                 mbar_expect_tx(&full[st], stage_bytes);
-                tma_load_2d(a_dst, &p.w_map, kb * kTcBlockK, tile * kTcTileM, &full[st]);
+                tma_load_2d_hint(a_dst, &p.w_map, kb * kTcBlockK, tile * kTcTileM, &full[st], pol);
                 tma_load_2d(a_dst + kATileBytes, &p.x_map, kb * kTcBlockK, 0, &full[st]);
             }
         }

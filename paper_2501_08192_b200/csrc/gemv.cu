@@ -88,6 +88,7 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
     // ---- producer side of this warp's ring (lane 0 only)
     int p_grp = blockIdx.x, p_c = c_begin;           // next unit to fetch
     uint32_t n_issued = 0;
+    const uint64_t pol = policy_evict_first();       // every weight byte is read once per step
     auto issue_next = [&]() {
         if (p_grp >= p.groups || c_begin >= c_end)
             return;
@@ -96,8 +97,8 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
         const size_t rb = (size_t)p_grp * rbs_per_cta + rbl;
         const uint32_t bytes = (uint32_t)n * 1024u;
         mbar_expect_tx(&bars[warp][slot], bytes);
-        bulk_load(ring + slot * (kUnitChunks * 1024), reinterpret_cast<const uint8_t *>(p.w) + (rb * p.kchunks + p_c) * 1024,
-                  bytes, &bars[warp][slot]);
+        bulk_load_hint(ring + slot * (kUnitChunks * 1024),
+                       reinterpret_cast<const uint8_t *>(p.w) + (rb * p.kchunks + p_c) * 1024, bytes, &bars[warp][slot], pol);
         ++n_issued;
         p_c += kUnitChunks;
         if (p_c >= c_end) {

@@ -40,6 +40,7 @@ struct WindowArgs {
     size_t x_plane_elems;          // elements between the planes
     int B, H;
     long long *trace;              // optional timeline slot (4 values), see common.cuh
+    int delay_ns;                  // modelled communication latency added to the window (0 = none)
 };
 cudaError_t launch_window(const WindowArgs &a, cudaStream_t s);
 

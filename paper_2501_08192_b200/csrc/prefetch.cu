@@ -102,7 +102,8 @@ __global__ void __launch_bounds__(kPfThreads) k_prefetch_l2(const __grid_constan
     }
 }
 
-static int g_pf_mode = 0;
+static int g_pf_mode = 2;   // measured: the fire-and-forget hints (modes 0, 1) flood the memory system and
+                            // delay the main stream's demand loads; plain loads are flow-controlled
 static uint32_t g_pf_chunk = 4096;
 
 void set_prefetch_kernel_mode(int mode, uint32_t chunk)

@@ -25,6 +25,7 @@ struct WindowParams {
     size_t x_plane;
     int H;
     long long *trace;
+    int delay_ns;
 };
 
 template <bool RESID_F32, bool PART0_F32>
@@ -48,6 +49,7 @@ __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_con
     pdl_launch_dependents();   // the next kernel may start fetching its weights now
     pdl_wait();                // partial sums come from the preceding kernel in the stream
     trace_waited(p.trace);
+    const long long t_begin = p.delay_ns ? gtime() : 0;   // the modelled collective starts when its inputs exist
 
 #pragma unroll
     for (int c = 0; c < kWinMaxChunks; ++c) {
@@ -112,6 +114,14 @@ __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_con
     __syncthreads();
     const float inv = rsqrtf(total / (float)p.H + p.eps);
 
+    // modelled network time of the allreduce this kernel stands in for: hold the result back until
+    // delay_ns after its inputs were complete (bounded by the delay itself)
+    if (p.delay_ns) {
+        while (gtime() - t_begin < (long long)p.delay_ns) {
+            __nanosleep(200);
+        }
+    }
+
 #pragma unroll
     for (int c = 0; c < kWinMaxChunks; ++c) {
         const int ch = threadIdx.x + c * blockDim.x;
@@ -162,6 +172,7 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
     p.x_plane = a.x_plane_elems / 8;
     p.H = a.H;
     p.trace = a.trace;
+    p.delay_ns = a.delay_ns;
     const int chunks = a.H / 8;
     int threads = (chunks + kWinMaxChunks - 1) / kWinMaxChunks;
     if (chunks <= 1024)
