@@ -64,6 +64,7 @@ extern "C" {
 #define PRESERVE_ECUDA    (-5)  /* a CUDA call failed; see preserve_last_cuda_error */
 #define PRESERVE_EARCH    (-6)  /* no sm_100 device / driver entry point missing    */
 #define PRESERVE_ETIMEOUT (-7)  /* a bounded device-side wait gave up               */
+#define PRESERVE_ETOOBIG  (-8)  /* problem larger than a fixed-capacity entry point  */
 
 /* Prefetch planning modes. */
 #define PRESERVE_PLAN_WHOLE_NODE 0  /* Algorithm 1: a tensor is prefetched whole or not at all      */
@@ -252,6 +253,46 @@ PRESERVE_API int preserve_last_cuda_error(const preserve_layer_t *layer);
  * not exceed the buffer's size.  Asynchronous on `cuda_stream`. */
 PRESERVE_API int preserve_debug_copy(preserve_layer_t *layer, int32_t which, void *dst_device, size_t bytes,
                         void *cuda_stream);
+
+/* Decode attention that allocates nothing.  (The paper has no counterpart to this
+ * entry point; it exists for callers of this library.)
+ *
+ * Who it is for: code that must not, or cannot, call cudaMalloc at the moment it needs
+ * attention - a step that runs inside a memory-frozen region of a serving process, a
+ * plug-in that is handed device buffers by its host and has no allocator of its own, a
+ * caller that is already capturing a stream (allocation is illegal during capture).
+ * preserve_layer_init allocates workspaces; this call never does, and needs no handle.
+ *
+ * What it computes: for every sequence b and query head h, softmax(q . K^T / sqrt(128)) V
+ * over cache slots 0..ctx_len[b] (ctx_len[b] + 1 keys: the newest entry must already be
+ * in the cache), grouped-query layout as in preserve_step_io_t, by the same split-KV
+ * kernel and merge kernel as the layer path.  The split-KV partial results live in a
+ * fixed PRESERVE_STATIC_SCRATCH_BYTES array that is part of the library image: every
+ * GPU that loads the library holds that much memory until the process exits.
+ *
+ * Arguments: q_hi/q_lo and o_hi/o_lo are device bf16 [batch, n_q_heads, 128]; a value is
+ * hi + lo (pass a zero-filled q_lo for plain bf16 queries; o_lo receives the rounding
+ * remainder of the output).  k_cache/v_cache are device bf16
+ * [batch, n_kv_heads, kv_capacity, 128].  ctx_len is a device array, ctx_len_host the same
+ * values on the host; each 0..kv_capacity-1.  At most 16 query heads per KV head.
+ *
+ * Limits and errors: the partials of (2 x SM count + batch x n_kv_heads) work items must
+ * fit in the scratch array, else PRESERVE_ETOOBIG is returned and nothing is queued; other
+ * bad arguments return PRESERVE_EINVAL / _EALIGN / _ESHAPE.
+ *
+ * Sharing: all calls on one GPU use the same array, and it keeps whatever the previous
+ * call left there (the call clears the one word that must start at zero).  Two calls that
+ * overlap on the GPU - different streams, or different threads - race on it; serialise them.
+ *
+ * First call: the first call on each device looks up the array's device address and sets
+ * the kernels' shared-memory limit, which are synchronous set-up steps; make that first
+ * call outside any stream capture.  Later calls only queue work on `cuda_stream`. */
+#define PRESERVE_STATIC_SCRATCH_BYTES (8u << 20)
+PRESERVE_API int preserve_attention_static(const void *q_hi, const void *q_lo, const void *k_cache,
+                                           const void *v_cache, const int32_t *ctx_len,
+                                           const int32_t *ctx_len_host, int32_t batch, int32_t n_q_heads,
+                                           int32_t n_kv_heads, int32_t kv_capacity, void *o_hi, void *o_lo,
+                                           void *cuda_stream);
 
 /* Frees everything the library allocated for the handle (NULL is allowed). */
 PRESERVE_API void preserve_layer_destroy(preserve_layer_t *layer);

@@ -15,7 +15,8 @@ LIB_PATH = os.path.join(_HERE, "libpreserve.so")
 
 PRESERVE_OK = 0
 PRESERVE_EINVAL, PRESERVE_EALIGN, PRESERVE_ESHAPE, PRESERVE_ENOMEM = -1, -2, -3, -4
-PRESERVE_ECUDA, PRESERVE_EARCH, PRESERVE_ETIMEOUT = -5, -6, -7
+PRESERVE_ECUDA, PRESERVE_EARCH, PRESERVE_ETIMEOUT, PRESERVE_ETOOBIG = -5, -6, -7, -8
+STATIC_SCRATCH_BYTES = 8 << 20
 PLAN_WHOLE_NODE, PLAN_TRUNCATE = 0, 1
 FLAG_NO_GRAPH, FLAG_PERSIST_L2, FLAG_NO_EARLY_LAUNCH = 1, 2, 4
 
@@ -25,7 +26,7 @@ EXPORTS = (
     "preserve_last_cuda_error", "preserve_debug_copy", "preserve_layer_destroy", "preserve_strerror",
     "preserve_plan_window", "preserve_algorithmic_bytes", "preserve_profile_step",
     "preserve_run_kernel", "preserve_set_trace", "preserve_read_trace",
-    "preserve_set_window_delay_ns",
+    "preserve_set_window_delay_ns", "preserve_attention_static",
 )
 KERNEL_NAMES = ("window_a", "qkv_proj", "attn_splitkv", "attn_merge", "o_proj", "window_b", "gate_up_proj",
                 "down_proj")
@@ -90,6 +91,7 @@ def lib() -> C.CDLL:
         L.preserve_run_kernel.argtypes = [C.c_void_p, C.POINTER(StepIO), C.c_int32, C.c_void_p]
         L.preserve_set_trace.argtypes = [C.c_void_p, C.c_int32]
         L.preserve_read_trace.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
+        L.preserve_attention_static.argtypes = [C.c_void_p] * 6 + [C.c_int32] * 4 + [C.c_void_p] * 3
         L.preserve_layer_get_info.argtypes = [C.c_void_p, C.POINTER(Info)]
         L.preserve_last_status.argtypes = [C.c_void_p]
         L.preserve_last_cuda_error.argtypes = [C.c_void_p]
@@ -239,6 +241,18 @@ class Layer:
     def debug_copy(self, which: int, dst, stream=None) -> None:
         _check(lib().preserve_debug_copy(self.handle, which, _ptr(dst), dst.numel() * dst.element_size(),
                                          _stream_ptr(stream)), "preserve_debug_copy")
+
+
+def preserve_attention_static(q_hi, q_lo, k_cache, v_cache, ctx_len_dev, ctx_len_host, n_q_heads: int,
+                              n_kv_heads: int, o_hi, o_lo, stream=None) -> int:
+    """Allocation-free decode attention; returns the PRESERVE_* code (see preserve.h).
+
+    Tensors: q_hi/q_lo/o_hi/o_lo CUDA bf16 [batch, n_q_heads, 128]; caches CUDA bf16
+    [batch, n_kv_heads, capacity, 128]; ctx_len_dev CUDA int32 [batch]; ctx_len_host int32 numpy array."""
+    batch, _, cap, _ = k_cache.shape
+    return int(lib().preserve_attention_static(_ptr(q_hi), _ptr(q_lo), _ptr(k_cache), _ptr(v_cache),
+                                               _ptr(ctx_len_dev), ctx_len_host.ctypes.data, batch, n_q_heads,
+                                               n_kv_heads, cap, _ptr(o_hi), _ptr(o_lo), _stream_ptr(stream)))
 
 
 def preserve_decode_chain(layers: Sequence[Layer], ios: Sequence[StepIO], link: bool, stream=None) -> None:

@@ -61,6 +61,14 @@ struct GraphEntry {
 
 }  // namespace
 
+namespace prsv {
+bool encode_bf16_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_cols,
+                        uint32_t box_rows)
+{
+    return make_map_2d(m, base, cols, rows, box_cols, box_rows);
+}
+}  // namespace prsv
+
 struct preserve_layer {
     preserve_layer_config_t cfg;
     int dev, sm_count, l2_bytes, max_persist, max_window;
@@ -664,6 +672,7 @@ const char *preserve_strerror(int code)
     case PRESERVE_ECUDA: return "CUDA call failed";
     case PRESERVE_EARCH: return "needs an sm_100 device";
     case PRESERVE_ETIMEOUT: return "a bounded device-side wait gave up";
+    case PRESERVE_ETOOBIG: return "problem exceeds the fixed scratch capacity of the allocation-free entry point";
     default: return "unknown error";
     }
 }

@@ -17,6 +17,7 @@
 // ldmatrix.trans).  At the end of an item every warp writes its (max, sum, O) as an
 // fp32 partial; k_attn_merge combines the partials of a sequence in fixed order.
 // Nothing depends on timing, so results are bit-stable.
+#include "../../include/preserve.h"
 #include "common.cuh"
 #include "kernels.h"
 
@@ -482,3 +483,111 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
 }
 
 }  // namespace prsv
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free decode attention.  Some callers cannot allocate device memory when they
+// need attention (see the declaration in preserve.h), so the split-KV partials of this
+// variant live in an array that is part of the library image instead of a cudaMalloc'd
+// workspace.  In host code the array's name is only a handle for the runtime - not a device
+// address - so the address is looked up once per device with cudaGetSymbolAddress and that
+// pointer is what the kernels receive.
+static __device__ __align__(256) unsigned char g_static_scratch[PRESERVE_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void *g_scratch_addr[kMaxDevices];      // per device, filled by the first call on that device
+int g_scratch_sms[kMaxDevices];
+}  // namespace
+
+extern "C" int preserve_attention_static(const void *q_hi, const void *q_lo, const void *k_cache,
+                                         const void *v_cache, const int32_t *ctx_len,
+                                         const int32_t *ctx_len_host, int32_t batch, int32_t n_q_heads,
+                                         int32_t n_kv_heads, int32_t kv_capacity, void *o_hi, void *o_lo,
+                                         void *cuda_stream)
+{
+    using namespace prsv;
+    if (!q_hi || !q_lo || !k_cache || !v_cache || !ctx_len || !ctx_len_host || !o_hi || !o_lo)
+        return PRESERVE_EINVAL;
+    const void *ptrs[] = {q_hi, q_lo, k_cache, v_cache, o_hi, o_lo};
+    for (const void *p : ptrs)
+        if (reinterpret_cast<uintptr_t>(p) & 15)
+            return PRESERVE_EALIGN;
+    if (batch < 1 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads || n_q_heads / n_kv_heads > 16 ||
+        kv_capacity < 1 || (long long)batch * n_kv_heads > kMaxStreams ||
+        (long long)batch * n_kv_heads * kv_capacity > 0x7fffffffll)
+        return PRESERVE_ESHAPE;
+    uint64_t total_tiles = 0;
+    for (int b = 0; b < batch; ++b) {
+        if (ctx_len_host[b] < 0 || ctx_len_host[b] >= kv_capacity)
+            return PRESERVE_ESHAPE;
+        total_tiles += (uint64_t)n_kv_heads * ((ctx_len_host[b] + 1 + kTileKeys - 1) / kTileKeys);
+    }
+
+    // ---- once per device: the array's device address (with that device current)
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return PRESERVE_EARCH;
+    }
+    if (!g_scratch_addr[dev]) {
+        void *addr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&addr, g_static_scratch);
+        if (e != cudaSuccess || !addr) {
+            (void)cudaGetLastError();
+            return PRESERVE_ECUDA;
+        }
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+            (void)cudaGetLastError();
+            return PRESERVE_ECUDA;
+        }
+        if (cudaFuncSetAttribute(k_attn_decode_splitkv, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(sizeof(AttnSmem) + 1024)) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return PRESERVE_ECUDA;
+        }
+        g_scratch_sms[dev] = sms;
+        g_scratch_addr[dev] = addr;
+    }
+
+    // ---- carve the array: [status word, 256 B][partial O][partial (max, sum)]
+    const int G = n_q_heads / n_kv_heads;
+    const int grid = 2 * g_scratch_sms[dev];
+    const uint64_t tpi = (total_tiles + grid - 1) / grid;            // about one work item per CTA
+    const uint64_t max_items = (uint64_t)grid + (uint64_t)batch * n_kv_heads;
+    const uint64_t o_bytes = max_items * kConsumerWarps * G * kHeadDim * sizeof(float);
+    const uint64_t ml_bytes = max_items * kConsumerWarps * G * 2 * sizeof(float);
+    if (256 + o_bytes + ml_bytes > PRESERVE_STATIC_SCRATCH_BYTES)
+        return PRESERVE_ETOOBIG;
+    unsigned char *base = static_cast<unsigned char *>(g_scratch_addr[dev]);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+
+    AttnArgs a = {};
+    const uint64_t rows = (uint64_t)batch * n_kv_heads * kv_capacity;
+    if (!encode_bf16_map_2d(&a.k_map, k_cache, kHeadDim, rows, 64, 64) ||
+        !encode_bf16_map_2d(&a.v_map, v_cache, kHeadDim, rows, 64, 64))
+        return PRESERVE_EARCH;
+    // the status word is the only part of the array that must start at zero
+    if (cudaMemsetAsync(base, 0, 256, s) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return PRESERVE_ECUDA;
+    }
+    a.q = q_hi;
+    a.q_plane = (size_t)(static_cast<const bf16 *>(q_lo) - static_cast<const bf16 *>(q_hi));
+    a.ctx_len = ctx_len;
+    a.B = batch; a.nq = n_q_heads; a.nkv = n_kv_heads; a.cap = kv_capacity;
+    a.grid = grid;
+    a.tiles_per_item = tpi < 1 ? 1 : (int)tpi;
+    a.max_items = (int)max_items;
+    a.part_o = reinterpret_cast<float *>(base + 256);
+    a.part_ml = reinterpret_cast<float *>(base + 256 + o_bytes);
+    a.o_out = o_hi;
+    a.o_plane = (size_t)(static_cast<bf16 *>(o_lo) - static_cast<bf16 *>(o_hi));
+    a.status = reinterpret_cast<int *>(base);
+    if (launch_attention(a, s) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return PRESERVE_ECUDA;
+    }
+    return PRESERVE_OK;
+}
+

@@ -118,6 +118,10 @@ struct AttnArgs {
 };
 cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s);
 
+// 2-D bf16 tensor map (rows x cols, cols contiguous), box (box_cols x box_rows), 128-byte swizzle.
+bool encode_bf16_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_cols,
+                        uint32_t box_rows);
+
 // ---- L2 prefetch (no arithmetic, writes nothing)
 struct PrefetchSeg {
     const void *base;     // contiguous range, or the K cache when per_seq_tokens != 0
