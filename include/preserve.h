@@ -164,7 +164,7 @@ typedef struct {
  * arena laid out in the order the kernels consume them, allocates workspaces,
  * a side stream and events on the CURRENT device.  The weight pointers may be
  * freed after the call returns.  *out is NULL on failure.
- * The prefetch budget starts at a quarter of the device's L2 size, mode PRESERVE_PLAN_TRUNCATE. */
+ * The prefetch budget starts at one sixteenth of the device's L2 size, mode PRESERVE_PLAN_TRUNCATE. */
 PRESERVE_API int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer_weights_t *w,
                         preserve_layer_t **out);
 

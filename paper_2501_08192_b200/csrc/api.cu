@@ -376,6 +376,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         CK(L, cudaStreamWaitEvent(L->side, L->ev_a, 0));
         PrefetchArgs pa = {};
         pa.ctx_len = sp.ctx_len;
+        pa.sink = L->status + 8;
         int n = 0;
         if (L->planned[0][0]) {
             pa.seg[n].base = L->arena + L->off[0];
@@ -484,6 +485,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         CK(L, cudaStreamWaitEvent(L->side, L->ev_b, 0));
         PrefetchArgs pa = {};
         pa.ctx_len = sp.ctx_len;
+        pa.sink = L->status + 8;
         int n = 0;
         for (int i = 0; i < 2; ++i)
             if (L->planned[1][i]) {
@@ -774,12 +776,12 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     const char *pfm = getenv("PRESERVE_PREFETCH_MODE");
     const char *pfc = getenv("PRESERVE_PREFETCH_CHUNK");
     if (pfm || pfc)
-        set_prefetch_kernel_mode(pfm ? atoi(pfm) : 2, pfc ? (uint32_t)atoi(pfc) : 4096u);
+        set_prefetch_kernel_mode(pfm ? atoi(pfm) : 0, pfc ? (uint32_t)atoi(pfc) : 4096u);
     const char *pfn = getenv("PRESERVE_PREFETCH_CTAS");
-    L->prefetch_ctas = pfn ? atoi(pfn) : 64;
+    L->prefetch_ctas = pfn ? atoi(pfn) : 128;
     if (L->prefetch_ctas < 1)
         L->prefetch_ctas = 1;
-    L->budget = (size_t)L->l2_bytes / 4;
+    L->budget = (size_t)L->l2_bytes / 16;
     L->plan_mode = PRESERVE_PLAN_TRUNCATE;
 
 #define CKI(expr)                                   \

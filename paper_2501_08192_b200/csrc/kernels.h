@@ -137,6 +137,7 @@ struct PrefetchArgs {
     PrefetchSeg seg[6];
     int n_segs;
     const int *ctx_len;
+    int *sink;            // scratch word for the load variant (practically never written)
 };
 void set_prefetch_kernel_mode(int mode, uint32_t chunk_bytes);
 cudaError_t launch_prefetch(const PrefetchArgs &a, int ctas, cudaStream_t s, const cudaLaunchAttribute *attrs,

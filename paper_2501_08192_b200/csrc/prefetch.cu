@@ -26,6 +26,7 @@ struct PrefetchParams {
     PrefetchArgs a;
     int mode;
     uint32_t chunk;
+    int *sink;      // never written in practice (see mode 2)
 };
 
 __global__ void __launch_bounds__(kPfThreads) k_prefetch_l2(const __grid_constant__ PrefetchParams p)
@@ -79,6 +80,33 @@ __global__ void __launch_bounds__(kPfThreads) k_prefetch_l2(const __grid_constan
     if (n_ranges == 0)
         return;
     const uint64_t total_chunks = range_first_chunk[n_ranges];
+    if (p.mode == 2) {
+        // load variant: a warp takes a chunk and reads it with coalesced accesses - lane l touches
+        // the 32-byte sector l of each KiB (one 16-byte load per sector brings in the whole line).
+        // The values are folded into a word that is stored only if it equals a magic number, which
+        // keeps the assembler from dropping the loads; in practice nothing is ever written.
+        const int lane = threadIdx.x & 31;
+        const uint64_t warp_id = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+        const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+        uint32_t fold = 0;
+        int r = 0;
+        for (uint64_t c = warp_id; c < total_chunks; c += n_warps) {
+            while (range_first_chunk[r + 1] <= c)
+                ++r;
+            const uint64_t off = (c - range_first_chunk[r]) * p.chunk;
+            const uint64_t left = ranges[r].bytes - off;
+            const uint32_t n = left < p.chunk ? (uint32_t)left : p.chunk;
+            const uint8_t *ptr = ranges[r].ptr + off + lane * 32;
+#pragma unroll 4
+            for (uint32_t o = lane * 32; o < n; o += 1024, ptr += 1024) {
+                const uint4 v = ld_stream(ptr);
+                fold ^= v.x ^ v.y ^ v.z ^ v.w;
+            }
+        }
+        if (fold == 0x5eed1234u && p.sink)
+            *p.sink = (int)fold;
+        return;
+    }
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
     int r = 0;
     for (uint64_t c = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; c < total_chunks; c += stride) {
@@ -90,20 +118,15 @@ __global__ void __launch_bounds__(kPfThreads) k_prefetch_l2(const __grid_constan
         const uint8_t *ptr = ranges[r].ptr + off;
         if (p.mode == 0) {
             bulk_prefetch_l2(ptr, n & ~15u);
-        } else if (p.mode == 1) {
+        } else {
             for (uint32_t o = 0; o < n; o += 128)
                 line_prefetch_l2(ptr + o);
-        } else {
-            // the loads are volatile asm, so they are issued although their values are dropped;
-            // one 16-byte load per 32-byte sector brings in the whole line
-            for (uint32_t o = 0; o < n; o += 32)
-                (void)ld_stream(ptr + o);
         }
     }
 }
 
-static int g_pf_mode = 2;   // measured: the fire-and-forget hints (modes 0, 1) flood the memory system and
-                            // delay the main stream's demand loads; plain loads are flow-controlled
+static int g_pf_mode = 0;   // measured on config 2: bulk L2 prefetch from 128 CTAs disturbs the main stream
+                            // least; per-line hints and plain loads cost more issue slots and time
 static uint32_t g_pf_chunk = 4096;
 
 void set_prefetch_kernel_mode(int mode, uint32_t chunk)
@@ -120,6 +143,7 @@ cudaError_t launch_prefetch(const PrefetchArgs &a, int ctas, cudaStream_t s, con
     p.a = a;
     p.mode = g_pf_mode;
     p.chunk = g_pf_chunk;
+    p.sink = a.sink;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ctas);
     cfg.blockDim = dim3(kPfThreads);
