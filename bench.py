@@ -36,7 +36,11 @@ SWEEP_FRACS = (0.0, 1 / 16, 1 / 8, 1 / 4, 3 / 8, 1 / 2, 5 / 8, 3 / 4, 7 / 8, 1.0
 
 # DRAM traffic per launch of the dominant kernel from an ncu capture (bytes), keyed by
 # (kernel, workload); see profiles/.  None where no capture exists.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # profiles/ncu_full_gemv_attn_window_config1_small.md (dram__bytes_read.sum + dram__bytes_write.sum)
+    ("gate_up_proj", 1): 29533952, ("down_proj", 1): 14780160, ("qkv_proj", 1): 6466048, ("o_proj", 1): 4253440,
+    ("attn_splitkv", 1): 16964352, ("attn_merge", 1): 2233856, ("window_a", 1): 618496, ("window_b", 1): 749312,
+}
 
 
 def load_peaks():
