@@ -203,9 +203,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
         }
     };
 
+    const int pair = (tile * kTcTileM + row) >> 1;
+    const int par = lane & 1;
     if (p.splits > 1) {
+        // Split-K across the cluster, reduce-scatter style: every rank publishes its partial tile in
+        // its own shared memory, then finishes NB / splits of the batch columns - reading that slice
+        // from all ranks in rank order (independent loads) - so the reduction and the epilogue work
+        // are spread over the whole cluster.
         cg::cluster_group cluster = cg::this_cluster();
-        if (warp >= 2 && s > 0) {
+        if (warp >= 2) {
             for (int c = 0; c < nchunks; ++c) {
                 float v[16];
                 load_chunk(c, v);
@@ -215,22 +221,34 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
             }
         }
         cluster.sync();
-    }
-    if (warp >= 2 && s == 0) {
-        const int pair = (tile * kTcTileM + row) >> 1;
-        const int par = lane & 1;
+        if (warp >= 2) {
+            const float *remote[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                remote[q] = cluster.map_shared_rank(red, q < p.splits ? q : 0) + row;
+            const int cols = p.NB / p.splits;             // columns finished by this rank (>= 2, even)
+            for (int b0 = s * cols; b0 < (s + 1) * cols; b0 += 2) {
+                float mine[2] = {0.f, 0.f};
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (q < p.splits) {
+                        mine[0] += remote[q][(b0 + 0) * kTcTileM];
+                        mine[1] += remote[q][(b0 + 1) * kTcTileM];
+                    }
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const float other = __shfl_xor_sync(0xffffffffu, mine[i], 1);
+                    const int b = b0 + i;
+                    if (i == par && b < p.B && !poisoned)
+                        apply_epilogue(p.epi, true, p.N, b, pair, par ? other : mine[i], par ? mine[i] : other);
+                }
+            }
+        }
+        cluster.sync();        // peers' shared memory must outlive the reads
+    } else if (warp >= 2) {
         for (int c = 0; c < nchunks; ++c) {
             float v[16];
             load_chunk(c, v);
-            if (p.splits > 1) {
-                cg::cluster_group cluster = cg::this_cluster();
-                for (int q = 1; q < p.splits; ++q) {
-                    const float *remote = cluster.map_shared_rank(red, q);
-#pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        v[i] += remote[(c * 16 + i) * kTcTileM + row];
-                }
-            }
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const float mine = v[i];
@@ -240,10 +258,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
                     apply_epilogue(p.epi, true, p.N, b, pair, par ? other : mine, par ? mine : other);
             }
         }
-    }
-    if (p.splits > 1) {
-        cg::cluster_group cluster = cg::this_cluster();
-        cluster.sync();        // peers' shared memory must outlive rank 0's reads
     }
     tc_fence_before();
     __syncthreads();
@@ -275,17 +289,24 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     p.status = a.status;
     p.trace = a.trace;
     const int tiles = a.N / kTcTileM;
-    int splits = pow2_floor_i((2 * sm_count) / tiles > 0 ? (2 * sm_count) / tiles : 1);
-    if (splits > 8) splits = 8;
-    while (splits > 1 && p.kblocks / splits < 2) splits /= 2;
-    p.splits = splits;
     const int stage_bytes = kATileBytes + 2 * a.NB * kTcBlockK * 2;
     int stages = (200 * 1024) / stage_bytes;
     if (stages > kTcMaxStages) stages = kTcMaxStages;
     // two CTAs per SM when the ring is small enough, so one CTA's ramp-up overlaps another's stream
-    if (stages * stage_bytes > 100 * 1024 && (100 * 1024) / stage_bytes >= 4)
+    int per_sm = 1;
+    if (stages * stage_bytes > 100 * 1024 && (100 * 1024) / stage_bytes >= 4) {
         stages = (100 * 1024) / stage_bytes;
+        per_sm = 2;
+    } else if (stages * stage_bytes <= 100 * 1024) {
+        per_sm = 2;
+    }
     p.stages = stages;
+    // One wave: the grid (tiles x cluster ranks) must fit the co-resident slots, else the second
+    // wave doubles the kernel.  Splits are a power of two <= 8 and leave every rank >= 2 k-blocks.
+    const int slots = sm_count * per_sm;
+    int splits = 1;
+    while (splits < 8 && tiles * splits * 2 <= slots && p.kblocks / (splits * 2) >= 2) splits *= 2;
+    p.splits = splits;
     int cols = 32;
     while (cols < 2 * a.NB) cols *= 2;
     p.tmem_cols = cols;
