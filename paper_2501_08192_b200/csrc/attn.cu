@@ -333,10 +333,8 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
 // not depend on scheduling.
 constexpr int kMergeGroups = 16;
 constexpr int kMergeThreads = kMergeGroups * 32;
-constexpr int kMergeChunk = 1024;          // entries whose weights are staged in shared memory at a time
 __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(const __grid_constant__ AttnParams p)
 {
-    __shared__ float w_s[kMergeChunk];
     __shared__ float red_s[kMergeThreads / 32];
     __shared__ int cnt_s[kMergeThreads / 32];
     __shared__ float4 acc_s[kMergeGroups][32];
@@ -371,47 +369,56 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(const __grid_const
     const size_t stride_ml = (size_t)p.G * 2, stride_o = (size_t)p.G * kHeadDim;
     const float *ml = p.part_ml + ((size_t)base * kConsumerWarps * p.G + row) * 2;
     const float *po = p.part_o + ((size_t)base * kConsumerWarps * p.G + row) * kHeadDim + 4 * lane;
-    float M = -INFINITY;
-    for (int e = tid; e < n_ent; e += kMergeThreads)
-        M = fmaxf(M, ml[e * stride_ml]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1)
-        M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-    if (lane == 0)
-        red_s[warp] = M;
-    __syncthreads();
-    M = red_s[0];
-#pragma unroll
-    for (int i = 1; i < kMergeThreads / 32; ++i)
-        M = fmaxf(M, red_s[i]);
-    float L = 0.f;
+    // One pass: group `warp` takes entries warp, warp + 16, ... in bursts of 8 (all loads of a burst
+    // are independent), keeping a running maximum like the attention kernel does, so every partial
+    // is read exactly once and the reads are a single memory round trip for <= 128 entries.
+    float Mg = -INFINITY, L = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int e0 = 0; e0 < n_ent; e0 += kMergeChunk) {
-        const int ne = min(kMergeChunk, n_ent - e0);
-        __syncthreads();
-        for (int e = tid; e < ne; e += kMergeThreads) {
-            const float m = ml[(e0 + e) * stride_ml];
-            w_s[e] = m == -INFINITY ? 0.f : exp2f(m - M);
+    for (int e0 = warp; e0 < n_ent; e0 += kMergeGroups * 8) {
+        float2 mlv[8];
+        float4 ov[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int e = e0 + u * kMergeGroups;
+            if (e < n_ent) {
+                mlv[u] = *reinterpret_cast<const float2 *>(ml + e * stride_ml);
+                ov[u] = *reinterpret_cast<const float4 *>(po + e * stride_o);
+            } else {
+                mlv[u] = make_float2(-INFINITY, 0.f);
+                ov[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
         }
-        __syncthreads();
-#pragma unroll 8
-        for (int e = warp; e < ne; e += kMergeGroups) {
-            const float w = w_s[e];
-            const float4 v = *reinterpret_cast<const float4 *>(po + (e0 + e) * stride_o);
-            L += ml[(e0 + e) * stride_ml + 1] * w;
-            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+        float mb = Mg;
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            mb = fmaxf(mb, mlv[u].x);
+        const float c = mb == -INFINITY ? 1.f : exp2f(Mg - mb);
+        L *= c; acc.x *= c; acc.y *= c; acc.z *= c; acc.w *= c;
+        Mg = mb;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const float w = mlv[u].x == -INFINITY ? 0.f : exp2f(mlv[u].x - Mg);
+            L += mlv[u].y * w;
+            acc.x += ov[u].x * w; acc.y += ov[u].y * w; acc.z += ov[u].z * w; acc.w += ov[u].w * w;
         }
     }
     acc_s[warp][lane] = acc;
-    if (lane == 0)
+    if (lane == 0) {
         l_s[warp] = L;
+        red_s[warp] = Mg;
+    }
     __syncthreads();
     if (tid < kHeadDim) {
+        float M = red_s[0];
+#pragma unroll
+        for (int w = 1; w < kMergeGroups; ++w)
+            M = fmaxf(M, red_s[w]);
         float a = 0.f, l = 0.f;
 #pragma unroll
         for (int w = 0; w < kMergeGroups; ++w) {
-            a += reinterpret_cast<const float *>(&acc_s[w][0])[tid];
-            l += l_s[w];
+            const float c = red_s[w] == -INFINITY ? 0.f : exp2f(red_s[w] - M);
+            a += reinterpret_cast<const float *>(&acc_s[w][0])[tid] * c;
+            l += l_s[w] * c;
         }
         const float ov = a / l;
         const bf16 hi = __float2bfloat16_rn(ov);
