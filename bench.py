@@ -225,7 +225,6 @@ def run_ours(args):
     sampler.start()
     set_budget(default_budget)
     ms_on, per_on = time_steps(chain_step, args.steps, args.warmup)
-    clocks = sampler.summary()
     # ---- prefetch off (vanilla execution), early launch only (budget of one byte: nothing planned for
     # L2), and the sweep over the L2 budget (fewer steps each)
     set_budget(0)
@@ -278,6 +277,7 @@ def run_ours(args):
         kms[k] = ms / (4 * R)
         del g
     status = max(L.last_status() for L in layers)
+    clocks = sampler.summary()      # sampled from before the first timed region to after the last
 
     peak, peak_src = load_peaks()
     kb = kernel_bytes(shape, sum_ctx)

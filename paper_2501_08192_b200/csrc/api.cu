@@ -333,10 +333,12 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
     const Dims d = layer_dims(c);
 
     // ---- plan (host): Algorithm 1 per window over {Wqkv, KV, Wo} and {Wgate|up, Wdown}
-    uint64_t sum_ctx = 0, total_tiles = 0;
+    uint64_t sum_ctx = 0, total_tiles = 0, max_tiles_seq = 0;
     for (int b = 0; b < B; ++b) {
         sum_ctx += (uint64_t)sp.ctx_len_host[b];
-        total_tiles += (uint64_t)c.n_kv_heads * ((sp.ctx_len_host[b] + 1 + 63) / 64);
+        const uint64_t nt = (uint64_t)(sp.ctx_len_host[b] + 1 + 63) / 64;
+        total_tiles += (uint64_t)c.n_kv_heads * nt;
+        max_tiles_seq = nt > max_tiles_seq ? nt : max_tiles_seq;
     }
     L->kv_bytes = 2 * sum_ctx * c.n_kv_heads * c.head_dim * 2;
     const uint64_t nodes_a[3] = {L->wbytes[0], L->kv_bytes, L->wbytes[1]};
@@ -459,6 +461,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         mult = mult < 1 ? 1 : (mult > 4 ? 4 : mult);
         uint64_t tpi = (total_tiles + (uint64_t)L->attn_grid * mult - 1) / ((uint64_t)L->attn_grid * mult);
         a.tiles_per_item = tpi < 1 ? 1 : (int)tpi;
+        a.max_entries_per_stream = 4 * (int)((max_tiles_seq + a.tiles_per_item - 1) / a.tiles_per_item);
         a.max_items = L->max_items;
         a.part_o = L->part_o;
         a.part_ml = L->part_ml;

@@ -327,10 +327,10 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
     trace_end(p.trace);
 }
 
-// Merge the partials of one (sequence, query head).  512 threads = 16 entry groups x 32
-// lanes of 4 head dims; group eg sums entries eg, eg + 16, ... (independent 128-bit loads, all
-// in flight together), then the 16 group sums are added in fixed order, so the result does
-// not depend on scheduling.
+// Merge the partials of one (sequence, query head).  A CTA is 4..16 entry groups (one warp
+// each, chosen from the number of partials per sequence) x 32 lanes of 4 head dims; group g sums
+// entries g, g + groups, ... (independent 128-bit loads, all in flight together), then the group
+// sums are added in fixed order, so the result does not depend on scheduling.
 constexpr int kMergeGroups = 16;
 constexpr int kMergeThreads = kMergeGroups * 32;
 __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(const __grid_constant__ AttnParams p)
@@ -342,13 +342,14 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(const __grid_const
     const int b = blockIdx.x / p.nq, hq = blockIdx.x % p.nq;
     const int kvh = hq / p.G, row = hq % p.G;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_groups = blockDim.x >> 5, n_threads = blockDim.x;
     const int sidx = b * p.nkv + kvh;
     long long *tr = p.trace ? p.trace + 4 : nullptr;
     trace_start(tr);
     pdl_launch_dependents();
     // first item of this stream: parallel count over the streams before it
     int cnt = 0;
-    for (int s2 = tid; s2 < sidx; s2 += kMergeThreads) {
+    for (int s2 = tid; s2 < sidx; s2 += n_threads) {
         const int nt = tiles_of(p.ctx_len[s2 / p.nkv]);
         cnt += (nt + p.tiles_per_item - 1) / p.tiles_per_item;
     }
@@ -360,8 +361,7 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(const __grid_const
     const int n_items = (tiles_of(p.ctx_len[b]) + p.tiles_per_item - 1) / p.tiles_per_item;
     __syncthreads();
     int base = 0;
-#pragma unroll
-    for (int i = 0; i < kMergeThreads / 32; ++i)
+    for (int i = 0; i < n_groups; ++i)
         base += cnt_s[i];
     pdl_wait();    // the partials come from the split-KV kernel
     trace_waited(tr);
@@ -374,12 +374,12 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(const __grid_const
     // is read exactly once and the reads are a single memory round trip for <= 128 entries.
     float Mg = -INFINITY, L = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int e0 = warp; e0 < n_ent; e0 += kMergeGroups * 8) {
+    for (int e0 = warp; e0 < n_ent; e0 += n_groups * 8) {
         float2 mlv[8];
         float4 ov[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            const int e = e0 + u * kMergeGroups;
+            const int e = e0 + u * n_groups;
             if (e < n_ent) {
                 mlv[u] = *reinterpret_cast<const float2 *>(ml + e * stride_ml);
                 ov[u] = *reinterpret_cast<const float4 *>(po + e * stride_o);
@@ -410,12 +410,10 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(const __grid_const
     __syncthreads();
     if (tid < kHeadDim) {
         float M = red_s[0];
-#pragma unroll
-        for (int w = 1; w < kMergeGroups; ++w)
+        for (int w = 1; w < n_groups; ++w)
             M = fmaxf(M, red_s[w]);
         float a = 0.f, l = 0.f;
-#pragma unroll
-        for (int w = 0; w < kMergeGroups; ++w) {
+        for (int w = 0; w < n_groups; ++w) {
             const float c = red_s[w] == -INFINITY ? 0.f : exp2f(red_s[w] - M);
             a += reinterpret_cast<const float *>(&acc_s[w][0])[tid] * c;
             l += l_s[w] * c;
@@ -480,7 +478,10 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     }
     cudaLaunchConfig_t cfg2 = {};
     cfg2.gridDim = dim3(a.B * a.nq);
-    cfg2.blockDim = dim3(kMergeThreads);
+    // merge groups: enough warps that each reads its share of a sequence's partials in one burst of 8
+    int merge_groups = (a.max_entries_per_stream + 7) / 8;
+    merge_groups = merge_groups < 4 ? 4 : (merge_groups > kMergeGroups ? kMergeGroups : merge_groups);
+    cfg2.blockDim = dim3(merge_groups * 32);
     cfg2.stream = s;
     cfg2.attrs = at;
     cfg2.numAttrs = pdl_attr(at);
@@ -523,11 +524,13 @@ extern "C" int preserve_attention_static(const void *q_hi, const void *q_lo, con
         kv_capacity < 1 || (long long)batch * n_kv_heads > kMaxStreams ||
         (long long)batch * n_kv_heads * kv_capacity > 0x7fffffffll)
         return PRESERVE_ESHAPE;
-    uint64_t total_tiles = 0;
+    uint64_t total_tiles = 0, max_tiles_seq = 0;
     for (int b = 0; b < batch; ++b) {
         if (ctx_len_host[b] < 0 || ctx_len_host[b] >= kv_capacity)
             return PRESERVE_ESHAPE;
-        total_tiles += (uint64_t)n_kv_heads * ((ctx_len_host[b] + 1 + kTileKeys - 1) / kTileKeys);
+        const uint64_t nt = (uint64_t)(ctx_len_host[b] + 1 + kTileKeys - 1) / kTileKeys;
+        total_tiles += (uint64_t)n_kv_heads * nt;
+        max_tiles_seq = nt > max_tiles_seq ? nt : max_tiles_seq;
     }
 
     // ---- once per device: the array's device address (with that device current)
@@ -586,6 +589,7 @@ extern "C" int preserve_attention_static(const void *q_hi, const void *q_lo, con
     a.grid = grid;
     a.tiles_per_item = tpi < 1 ? 1 : (int)tpi;
     a.max_items = (int)max_items;
+    a.max_entries_per_stream = kConsumerWarps * (int)((max_tiles_seq + a.tiles_per_item - 1) / a.tiles_per_item);
     a.part_o = reinterpret_cast<float *>(base + 256);
     a.part_ml = reinterpret_cast<float *>(base + 256 + o_bytes);
     a.o_out = o_hi;

@@ -107,6 +107,7 @@ struct AttnArgs {
     int grid;             // persistent CTAs
     int tiles_per_item;   // 64-key tiles per work item
     int max_items;        // capacity of the partial buffers
+    int max_entries_per_stream;  // 4 x work items of the longest sequence (sizes the merge CTAs; 0 = unknown)
     float *part_o;        // fp32 [max_items, 4 consumer warps, G, d]
     float *part_ml;       // fp32 [max_items, 4, G, 2]
     void *o_out;          // split bf16 [2][rows][nq,d]

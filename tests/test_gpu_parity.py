@@ -121,6 +121,57 @@ def test_prefetch_never_changes_results(oracle):
                 dl.close()
 
 
+def test_schedule_variants_do_not_change_results(oracle):
+    """Early launch off (ablation flag), a modelled window latency and the timeline trace change
+    when kernels run, never what they compute."""
+    shape = I.small_shape(name="sched", batch=7, ctx=400, ctx_min=9, seed=55)
+    t = I.make_layers(shape, 1)[0]
+    ref = oracle.layer_step(shape, t)
+    base = None
+    for flags in (0, P.FLAG_NO_EARLY_LAUNCH, P.FLAG_NO_GRAPH | P.FLAG_NO_EARLY_LAUNCH):
+        dl = G.DeviceLayer(shape, t, flags=flags)
+        try:
+            for delay, trace in ((0, False), (5000, False), (0, True)):
+                dl.layer.set_window_delay_ns(delay)
+                dl.layer.set_trace(trace)
+                dl.run()
+                bits = dl.output_bits()
+                if base is None:
+                    base = bits
+                    for name in ("attn_partial", "h2", "mlp_partial"):
+                        G.assert_close(dl.outputs()[name], ref[name], name)
+                for k in base:
+                    assert np.array_equal(base[k], bits[k]), (flags, delay, trace, k)
+                if trace:
+                    tr = dl.layer.read_trace()
+                    assert len(tr) == len(P.KERNEL_NAMES)
+                    ends = [e for (_, _, _, e) in tr]
+                    assert all(s <= w1 <= w2 <= e for (s, w1, w2, e) in tr)
+                    assert ends == sorted(ends)            # the main-stream kernels finish in order
+            assert dl.layer.last_status() == P.PRESERVE_OK
+        finally:
+            dl.close()
+
+
+def test_single_kernel_entry_point_reproduces_the_step(oracle):
+    shape = I.small_shape(name="single", batch=4, ctx=120, seed=56)
+    t = I.make_layers(shape, 1)[0]
+    dl = G.DeviceLayer(shape, t)
+    try:
+        dl.run()
+        want = dl.output_bits()
+        dl.mlp_out.t.zero_()
+        for k in range(len(P.KERNEL_NAMES)):
+            dl.layer.run_kernel(dl.io, k)
+        got = dl.output_bits()
+        for name in want:
+            assert np.array_equal(want[name], got[name]), name
+        ms = dl.layer.profile_step(dl.io)
+        assert len(ms) == len(P.KERNEL_NAMES) and all(v >= 0 for v in ms)
+    finally:
+        dl.close()
+
+
 def test_host_buffer_entry_point_matches_device_path(oracle):
     shape = I.small_shape(name="host_io", batch=6, ctx=150, ctx_min=3, seed=52)
     t = I.make_layers(shape, 1)[0]
