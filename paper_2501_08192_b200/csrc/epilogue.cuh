@@ -65,9 +65,27 @@ __device__ __forceinline__ void store_split(void *base, size_t plane, size_t idx
     reinterpret_cast<bf16 *>(base)[plane + idx] = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
-// Apply the epilogue to one pair of fp32 results of batch row b.
-__device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, bool tensor_path, int N, int b, int pair,
-                                               float v0, float v1)
+// The QKV epilogue needs, per output, the sequence position and the rotary frequency of the pair.
+// Both are inputs of the step (not results of earlier kernels), so a kernel copies them to shared
+// memory once, before it waits for its predecessor, instead of chasing them through global memory
+// for every output.
+struct EpilogueTables {
+    int pos[128];              // ctx_len[b0 + b], b < batch handled by the launch (at most 128)
+    double inv_freq[kHeadDim / 2];
+};
+__device__ __forceinline__ void load_epilogue_tables(const EpilogueArgs &e, EpilogueTables &t, int b0, int nb)
+{
+    if (e.kind != EPI_QKV)
+        return;
+    for (int i = threadIdx.x; i < nb && i < 128; i += blockDim.x)
+        t.pos[i] = e.ctx_len[b0 + i];
+    for (int i = threadIdx.x; i < kHeadDim / 2; i += blockDim.x)
+        t.inv_freq[i] = e.inv_freq ? e.inv_freq[i] : 0.0;
+}
+
+// Apply the epilogue to one pair of fp32 results of batch row b (b_local = b - b0 indexes the tables).
+__device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, const EpilogueTables &tab, int b_local,
+                                               bool tensor_path, int N, int b, int pair, float v0, float v1)
 {
     int n0, n1;
     pair_coords(e.kind, tensor_path, pair, n0, n1);
@@ -89,11 +107,11 @@ __device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, bool tenso
         store_split(e.out, e.out_plane, (size_t)b * (N >> 1) + n0, a);
     } else {
         const int hd = n0, i = n1;
-        const int pos = e.ctx_len[b];
+        const int pos = tab.pos[b_local];
         if (hd < e.nq + e.nkv && e.inv_freq) {
             // angle = pos * theta^(-2i/d): the product and its reduction mod 2 pi need more than
             // fp32 (angles reach tens of thousands of radians); the reduced angle does not
-            const double ang = (double)pos * e.inv_freq[i];
+            const double ang = (double)pos * tab.inv_freq[i];
             const double turns = rint(ang * 0.15915494309189535);
             const float red = (float)fma(-turns, 6.283185307179586, ang);
             float sf, cf;

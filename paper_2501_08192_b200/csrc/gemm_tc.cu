@@ -87,6 +87,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
     __shared__ uint64_t full[kTcMaxStages], empty[kTcMaxStages], accum_bar;
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile int poisoned;
+    __shared__ EpilogueTables tabs;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile = blockIdx.x;
@@ -97,6 +98,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
 
     trace_start(p.trace);
     pdl_launch_dependents();
+    load_epilogue_tables(p.epi, tabs, 0, p.B);   // inputs of the step: safe before the wait
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.stages; ++i) {
             mbar_init(&full[i], 1);
@@ -240,7 +242,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
                     const float other = __shfl_xor_sync(0xffffffffu, mine[i], 1);
                     const int b = b0 + i;
                     if (i == par && b < p.B && !poisoned)
-                        apply_epilogue(p.epi, true, p.N, b, pair, par ? other : mine[i], par ? mine[i] : other);
+                        apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? other : mine[i], par ? mine[i] : other);
                 }
             }
         }
@@ -255,7 +257,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
                 const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
                 const int b = c * 16 + i;
                 if ((i & 1) == par && b < p.B && !poisoned)
-                    apply_epilogue(p.epi, true, p.N, b, pair, par ? other : mine, par ? mine : other);
+                    apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? other : mine, par ? mine : other);
             }
         }
     }

@@ -67,6 +67,7 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
     __shared__ float red[kGemvWarps][16][NB];       // per-warp partials
     __shared__ float cta_part[kGemvWarps][16][NB];  // per-row-block CTA partials (read across the cluster)
     __shared__ uint64_t bars[kGemvWarps][kRingSlots];
+    __shared__ EpilogueTables tabs;
     extern __shared__ uint8_t gemv_smem_raw[];
     uint8_t *wsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(gemv_smem_raw) + 127) & ~uintptr_t(127));
 
@@ -117,6 +118,7 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
     }
     __syncwarp();
 
+    load_epilogue_tables(p.epi, tabs, p.b0, p.B);    // inputs of the step: safe before the wait
     const int xrow = p.K >> 3;                       // uint4 per activation row
     auto load_x = [&](int c, uint4 (&xq)[NX]) {
         if constexpr (MMA) {
@@ -263,7 +265,7 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
                         v0 += remote[q][(rl * 16 + r) * NB + b];
                         v1 += remote[q][(rl * 16 + r + 8) * NB + b];
                     }
-                apply_epilogue(p.epi, false, p.N, p.b0 + b, (grp * rbs_per_cta + rl) * 8 + r, v0, v1);
+                apply_epilogue(p.epi, tabs, b, false, p.N, p.b0 + b, (grp * rbs_per_cta + rl) * 8 + r, v0, v1);
             }
             cluster.sync();   // peers' shared memory must outlive the reads; also fences red/cta_part reuse
         } else {
@@ -272,8 +274,8 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
                 const int b = i % NB, r = (i / NB) % 8, rl = i / (8 * NB);
                 if (b >= p.B)
                     continue;
-                apply_epilogue(p.epi, false, p.N, p.b0 + b, (grp * rbs_per_cta + rl) * 8 + r, cta_part[rl][r][b],
-                               cta_part[rl][r + 8][b]);
+                apply_epilogue(p.epi, tabs, b, false, p.N, p.b0 + b, (grp * rbs_per_cta + rl) * 8 + r,
+                               cta_part[rl][r][b], cta_part[rl][r + 8][b]);
             }
             __syncthreads();
         }
