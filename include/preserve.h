@@ -206,8 +206,11 @@ PRESERVE_API int preserve_decode_step(preserve_layer_t *layer, const preserve_st
 PRESERVE_API int preserve_decode_chain(preserve_layer_t *const *layers, int32_t n, const preserve_step_io_t *ios,
                           int32_t link, void *cuda_stream);
 
-/* The step with host activation buffers (see preserve_host_io_t).  Host
- * buffers should be pinned for the copies to be asynchronous. */
+/* The step with host activation buffers (see preserve_host_io_t).  When every
+ * input buffer is pinned (page-locked) host memory, the window kernels read the
+ * inputs directly from host memory (that read is the host-to-device transfer);
+ * otherwise the inputs are first copied into a device staging area.  The two
+ * outputs are copied back from device memory at the end. */
 PRESERVE_API int preserve_decode_step_host(preserve_layer_t *layer, const preserve_host_io_t *io, void *cuda_stream);
 
 /* Per-kernel device times of one step.  Runs the step with direct launches on

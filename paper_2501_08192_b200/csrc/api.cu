@@ -968,26 +968,58 @@ int preserve_decode_step_host(preserve_layer_t *L, const preserve_host_io_t *io,
     const size_t BH2 = (size_t)io->batch * c.hidden * 2;
     const size_t slot = (size_t)c.max_batch * c.hidden * 2;
     const void *dparts[kMaxParts], *dpeers[kMaxParts];
-    for (int i = 0; i < c.tp_degree; ++i) {
+    for (int i = 0; i < c.tp_degree; ++i)
         if (!io->partials_in[i])
             return PRESERVE_EINVAL;
-        CK(L, cudaMemcpyAsync(L->stage_in + (size_t)i * slot, io->partials_in[i], BH2, cudaMemcpyHostToDevice, s));
-        dparts[i] = L->stage_in + (size_t)i * slot;
-    }
-    for (int i = 0; i + 1 < c.tp_degree; ++i) {
+    for (int i = 0; i + 1 < c.tp_degree; ++i)
         if (!io->attn_peer_partials[i])
             return PRESERVE_EINVAL;
-        uint8_t *dst = L->stage_in + (size_t)(c.tp_degree + i) * slot;
-        CK(L, cudaMemcpyAsync(dst, io->attn_peer_partials[i], BH2, cudaMemcpyHostToDevice, s));
-        dpeers[i] = dst;
+
+    // Pinned (page-locked) host buffers are visible to the device: the window kernels then read the
+    // step's inputs straight from host memory - that read IS the host-to-device transfer - instead
+    // of 2P + 1 separate copy calls followed by a second read from device memory.  Pageable buffers
+    // take the staged path.
+    auto device_view = [](const void *hp) -> const void * {
+        cudaPointerAttributes at;
+        if (cudaPointerGetAttributes(&at, hp) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        if (at.type != cudaMemoryTypeHost || !at.devicePointer ||
+            (reinterpret_cast<uintptr_t>(at.devicePointer) & 15))
+            return nullptr;
+        return at.devicePointer;
+    };
+    bool direct = true;
+    for (int i = 0; i < c.tp_degree && direct; ++i)
+        direct = (dparts[i] = device_view(io->partials_in[i])) != nullptr;
+    for (int i = 0; i + 1 < c.tp_degree && direct; ++i)
+        direct = (dpeers[i] = device_view(io->attn_peer_partials[i])) != nullptr;
+    const void *dres = direct ? device_view(io->residual_in) : nullptr;
+    const void *dctx = direct && dres ? device_view(io->ctx_len_host) : nullptr;
+    direct = direct && dres;
+    if (!direct) {
+        for (int i = 0; i < c.tp_degree; ++i) {
+            CK(L, cudaMemcpyAsync(L->stage_in + (size_t)i * slot, io->partials_in[i], BH2, cudaMemcpyHostToDevice, s));
+            dparts[i] = L->stage_in + (size_t)i * slot;
+        }
+        for (int i = 0; i + 1 < c.tp_degree; ++i) {
+            uint8_t *dst = L->stage_in + (size_t)(c.tp_degree + i) * slot;
+            CK(L, cudaMemcpyAsync(dst, io->attn_peer_partials[i], BH2, cudaMemcpyHostToDevice, s));
+            dpeers[i] = dst;
+        }
+        uint8_t *dst = L->stage_in + (size_t)(2 * c.tp_degree - 1) * slot;
+        CK(L, cudaMemcpyAsync(dst, io->residual_in, BH2, cudaMemcpyHostToDevice, s));
+        dres = dst;
     }
-    uint8_t *dres = L->stage_in + (size_t)(2 * c.tp_degree - 1) * slot;
-    CK(L, cudaMemcpyAsync(dres, io->residual_in, BH2, cudaMemcpyHostToDevice, s));
-    CK(L, cudaMemcpyAsync(L->ctx_dev, io->ctx_len_host, (size_t)io->batch * 4, cudaMemcpyHostToDevice, s));
+    if (!dctx || (reinterpret_cast<uintptr_t>(dctx) & 3)) {
+        CK(L, cudaMemcpyAsync(L->ctx_dev, io->ctx_len_host, (size_t)io->batch * 4, cudaMemcpyHostToDevice, s));
+        dctx = L->ctx_dev;
+    }
 
     preserve_step_io_t dio = {};
     dio.batch = io->batch;
-    dio.ctx_len = L->ctx_dev;
+    dio.ctx_len = static_cast<const int32_t *>(dctx);
     dio.ctx_len_host = io->ctx_len_host;
     dio.partials_in = dparts;
     dio.attn_peer_partials = dpeers;
