@@ -97,6 +97,8 @@ struct preserve_layer {
 
     // tensor path
     CUtensorMap wmap[4];
+    CUtensorMap wmap256[4];      // box of 256 rows (valid when has256[i])
+    bool has256[4];
     CUtensorMap xmap[4];         // x, o, x2, a as B operands
     int nb_pad;
 
@@ -300,6 +302,7 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
     if (L->tensor_path) {
         GemmTcArgs a;
         a.w_map = L->wmap[which];
+        a.w_map256 = L->has256[which] ? &L->wmap256[which] : nullptr;
         a.x_map = L->xmap[which];
         (void)x;
         a.B = B; a.NB = L->nb_pad; a.N = d.n[which]; a.K = d.k[which];
@@ -881,6 +884,8 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
                 preserve_layer_destroy(L);
                 return PRESERVE_EARCH;
             }
+            L->has256[i] = d.n[i] % 256 == 0 &&
+                           make_map_2d(&L->wmap256[i], L->arena + L->off[i], d.k[i], d.n[i], 64, 256);
         }
     }
     CKI(cudaStreamCreateWithFlags(&L->side, cudaStreamNonBlocking));

@@ -6,8 +6,9 @@
 // 128 x 16-k slab of weights for every batch row at once and the CUDA cores stay
 // out of the weight stream entirely.
 //
-// Per CTA: one 128-row tile of the packed weights x one slice of k.
-//   warp 0    : TMA producer - W tile (128 x 64, 128B swizzle) and x tile (NB x 64)
+// Per CTA: one 128-row tile of the packed weights (two for wide batches, sharing one activation
+// tile) x one slice of k.
+//   warp 0    : TMA producer - W tile (128 or 256 rows x 64, 128B swizzle) and x tile (2 NB x 64)
 //               into a multi-stage shared-memory ring, mbarrier full/empty
 //   warp 1    : allocates TMEM, issues tcgen05.mma (kind::f16, bf16 in, fp32
 //               accumulate in TMEM), tcgen05.commit frees ring slots
@@ -25,7 +26,7 @@ namespace cg = cooperative_groups;
 
 namespace prsv {
 
-constexpr int kTcMaxStages = 8;
+constexpr int kTcMaxStages = 12;
 constexpr int kTcThreads = 192;
 constexpr int kTcBlockK = 64;
 constexpr int kTcTileM = 128;
@@ -35,6 +36,7 @@ struct GemmTcParams {
     CUtensorMap w_map;
     CUtensorMap x_map;
     int B, NB, N, K;
+    int mt;             // 128-row weight tiles per CTA (1 or 2): two tiles share one activation tile
     int kblocks;        // K / 64
     int splits;         // cluster size along k
     int stages;
@@ -92,7 +94,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile = blockIdx.x;
     const int s = blockIdx.y;
-    const int stage_bytes = kATileBytes + 2 * p.NB * kTcBlockK * 2;
+    const int a_bytes = p.mt * kATileBytes;
+    const int stage_bytes = a_bytes + 2 * p.NB * kTcBlockK * 2;
     const int kb0 = (int)((long long)p.kblocks * s / p.splits);
     const int kb1 = (int)((long long)p.kblocks * (s + 1) / p.splits);
 
@@ -132,13 +135,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
             const int pre = n_kb < p.stages ? n_kb : p.stages;
             for (int i = 0; i < pre; ++i) {
                 mbar_expect_tx(&full[i], stage_bytes);
-                tma_load_2d_hint(smem + (size_t)i * stage_bytes, &p.w_map, (kb0 + i) * kTcBlockK, tile * kTcTileM,
-                                 &full[i], pol);
+                tma_load_2d_hint(smem + (size_t)i * stage_bytes, &p.w_map, (kb0 + i) * kTcBlockK,
+                                 tile * p.mt * kTcTileM, &full[i], pol);
             }
             pdl_wait();
             trace_waited(p.trace);
             for (int i = 0; i < pre; ++i)
-                tma_load_2d(smem + (size_t)i * stage_bytes + kATileBytes, &p.x_map, (kb0 + i) * kTcBlockK, 0, &full[i]);
+                tma_load_2d(smem + (size_t)i * stage_bytes + a_bytes, &p.x_map, (kb0 + i) * kTcBlockK, 0, &full[i]);
             uint32_t it = pre;
             for (int kb = kb0 + pre; kb < kb1; ++kb, ++it) {
                 const int st = it % p.stages;
@@ -146,8 +149,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
                 if (!mbar_wait(&empty[st], ph ^ 1, p.status, ST_TIMEOUT_EMPTY)) { poisoned = 1; break; }
                 uint8_t *a_dst = smem + (size_t)st * stage_bytes;
                 mbar_expect_tx(&full[st], stage_bytes);
-                tma_load_2d_hint(a_dst, &p.w_map, kb * kTcBlockK, tile * kTcTileM, &full[st], pol);
-                tma_load_2d(a_dst + kATileBytes, &p.x_map, kb * kTcBlockK, 0, &full[st]);
+                tma_load_2d_hint(a_dst, &p.w_map, kb * kTcBlockK, tile * p.mt * kTcTileM, &full[st], pol);
+                tma_load_2d(a_dst + a_bytes, &p.x_map, kb * kTcBlockK, 0, &full[st]);
             }
         }
     } else if (warp == 1) {
@@ -161,11 +164,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
                 if (!mbar_wait(&full[st], ph, p.status, ST_TIMEOUT_FULL)) { poisoned = 1; ok = false; break; }
                 tc_fence_after();
                 const uint32_t a_addr = smem_u32(smem + (size_t)st * stage_bytes);
-                const uint64_t adesc = make_smem_desc(a_addr);
-                const uint64_t bdesc = make_smem_desc(a_addr + kATileBytes);
+                const uint64_t bdesc = make_smem_desc(a_addr + a_bytes);
+                for (int m = 0; m < p.mt; ++m) {
+                    // each 128-row weight tile has its own accumulator (2 * NB TMEM columns)
+                    const uint64_t adesc = make_smem_desc(a_addr + m * kATileBytes);
 #pragma unroll
-                for (int k = 0; k < kTcBlockK / 16; ++k)
-                    tc_mma(tmem_base, adesc + 2 * k, bdesc + 2 * k, p.idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+                    for (int k = 0; k < kTcBlockK / 16; ++k)
+                        tc_mma(tmem_base + m * 2 * p.NB, adesc + 2 * k, bdesc + 2 * k, p.idesc,
+                               (kb > kb0 || k > 0) ? 1u : 0u);
+                }
                 tc_commit(&empty[st]);      // slot is free once these MMAs have read it
             }
             if (ok)
@@ -188,13 +195,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
         tc_fence_after();
     }
     const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
-    float *red = reinterpret_cast<float *>(smem);      // [NB][128] fp32, reuses the ring
+    float *red = reinterpret_cast<float *>(smem);      // [mt][NB][128] fp32, reuses the ring
 
-    auto load_chunk = [&](int c, float (&v)[16]) {
+    auto load_chunk = [&](int m, int c, float (&v)[16]) {
         if (have) {
             float lo[16];
-            tc_ld16(t_lane + c * 16, v);
-            tc_ld16(t_lane + p.NB + c * 16, lo);
+            tc_ld16(t_lane + m * 2 * p.NB + c * 16, v);
+            tc_ld16(t_lane + m * 2 * p.NB + p.NB + c * 16, lo);
 #pragma unroll
             for (int i = 0; i < 16; ++i)
                 v[i] += lo[i];
@@ -205,22 +212,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
         }
     };
 
-    const int pair = (tile * kTcTileM + row) >> 1;
     const int par = lane & 1;
     if (p.splits > 1) {
-        // Split-K across the cluster, reduce-scatter style: every rank publishes its partial tile in
+        // Split-K across the cluster, reduce-scatter style: every rank publishes its partial tiles in
         // its own shared memory, then finishes NB / splits of the batch columns - reading that slice
-        // from all ranks in rank order (independent loads) - so the reduction and the epilogue work
-        // are spread over the whole cluster.
+        // from all ranks in rank order - so the reduction and the epilogue work are spread over the
+        // whole cluster.
         cg::cluster_group cluster = cg::this_cluster();
         if (warp >= 2) {
-            for (int c = 0; c < nchunks; ++c) {
-                float v[16];
-                load_chunk(c, v);
+            for (int m = 0; m < p.mt; ++m)
+                for (int c = 0; c < nchunks; ++c) {
+                    float v[16];
+                    load_chunk(m, c, v);
 #pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    red[(c * 16 + i) * kTcTileM + row] = v[i];
-            }
+                    for (int i = 0; i < 16; ++i)
+                        red[((size_t)m * p.NB + c * 16 + i) * kTcTileM + row] = v[i];
+                }
         }
         cluster.sync();
         if (warp >= 2) {
@@ -229,13 +236,32 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
             for (int q = 0; q < 8; ++q)
                 remote[q] = cluster.map_shared_rank(red, q < p.splits ? q : 0) + row;
             const int cols = p.NB / p.splits;             // columns finished by this rank (>= 2, even)
-            for (int b0 = s * cols; b0 < (s + 1) * cols; b0 += 2) {
+            const int n_pairs = p.mt * cols / 2;
+            // Remote loads of the next column pair are issued before the current pair is finished
+            // (its stores would otherwise fence them off), hiding most of the ~800-cycle latency of
+            // distributed shared memory.
+            auto fetch = [&](int it, float (&t)[2][8]) {
+                const int m = it / (cols / 2), b0 = s * cols + 2 * (it % (cols / 2));
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (q < p.splits) {
+                        t[0][q] = remote[q][((size_t)m * p.NB + b0 + 0) * kTcTileM];
+                        t[1][q] = remote[q][((size_t)m * p.NB + b0 + 1) * kTcTileM];
+                    }
+            };
+            float cur[2][8], nxt[2][8];
+            fetch(0, cur);
+            for (int it = 0; it < n_pairs; ++it) {
+                if (it + 1 < n_pairs)
+                    fetch(it + 1, nxt);
+                const int m = it / (cols / 2), b0 = s * cols + 2 * (it % (cols / 2));
+                const int pair = ((tile * p.mt + m) * kTcTileM + row) >> 1;
                 float mine[2] = {0.f, 0.f};
 #pragma unroll
                 for (int q = 0; q < 8; ++q)
                     if (q < p.splits) {
-                        mine[0] += remote[q][(b0 + 0) * kTcTileM];
-                        mine[1] += remote[q][(b0 + 1) * kTcTileM];
+                        mine[0] += cur[0][q];
+                        mine[1] += cur[1][q];
                     }
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
@@ -244,20 +270,28 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
                     if (i == par && b < p.B && !poisoned)
                         apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? other : mine[i], par ? mine[i] : other);
                 }
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    cur[0][q] = nxt[0][q];
+                    cur[1][q] = nxt[1][q];
+                }
             }
         }
         cluster.sync();        // peers' shared memory must outlive the reads
     } else if (warp >= 2) {
-        for (int c = 0; c < nchunks; ++c) {
-            float v[16];
-            load_chunk(c, v);
+        for (int m = 0; m < p.mt; ++m) {
+            const int pair = ((tile * p.mt + m) * kTcTileM + row) >> 1;
+            for (int c = 0; c < nchunks; ++c) {
+                float v[16];
+                load_chunk(m, c, v);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const float mine = v[i];
-                const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
-                const int b = c * 16 + i;
-                if ((i & 1) == par && b < p.B && !poisoned)
-                    apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? other : mine, par ? mine : other);
+                for (int i = 0; i < 16; ++i) {
+                    const float mine = v[i];
+                    const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
+                    const int b = c * 16 + i;
+                    if ((i & 1) == par && b < p.B && !poisoned)
+                        apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? other : mine, par ? mine : other);
+                }
             }
         }
     }
@@ -290,32 +324,40 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     p.epi = a.epi;
     p.status = a.status;
     p.trace = a.trace;
-    const int tiles = a.N / kTcTileM;
-    const int stage_bytes = kATileBytes + 2 * a.NB * kTcBlockK * 2;
-    int stages = (200 * 1024) / stage_bytes;
-    if (stages > kTcMaxStages) stages = kTcMaxStages;
-    // two CTAs per SM when the ring is small enough, so one CTA's ramp-up overlaps another's stream
-    int per_sm = 1;
-    if (stages * stage_bytes > 100 * 1024 && (100 * 1024) / stage_bytes >= 4) {
+    // Two 128-row weight tiles per CTA share one activation tile when the batch is wide enough for
+    // the activation tile (2 * NB rows) to weigh as much as a weight tile: halves the L2->SM traffic
+    // of the activations, which every CTA re-reads.
+    const int mt = (a.NB >= 48 && a.N % (2 * kTcTileM) == 0 && a.w_map256) ? 2 : 1;
+    p.mt = mt;
+    if (mt == 2)
+        p.w_map = *a.w_map256;
+    const int tiles = a.N / (kTcTileM * mt);
+    const int stage_bytes = mt * kATileBytes + 2 * a.NB * kTcBlockK * 2;
+    // Ring depth, CTAs per SM and cluster splits.  Two CTAs per SM (rings <= 100 KiB) whenever that
+    // leaves >= 4 stages: measured better than one CTA with a ring twice as deep, because the second
+    // CTA streams while the first is in its epilogue.  The grid (tiles x splits) must fit the
+    // co-resident slots (a second wave doubles the kernel); splits are a power of two <= 8 that leave
+    // every rank >= 2 k-blocks.
+    int stages = (200 * 1024) / stage_bytes, per_sm = 1;
+    if ((100 * 1024) / stage_bytes >= 4) {
         stages = (100 * 1024) / stage_bytes;
         per_sm = 2;
-    } else if (stages * stage_bytes <= 100 * 1024) {
-        per_sm = 2;
     }
-    p.stages = stages;
-    // One wave: the grid (tiles x cluster ranks) must fit the co-resident slots, else the second
-    // wave doubles the kernel.  Splits are a power of two <= 8 and leave every rank >= 2 k-blocks.
+    if (stages > kTcMaxStages) stages = kTcMaxStages;
+    if (stages < 2)
+        return cudaErrorInvalidValue;
     const int slots = sm_count * per_sm;
     int splits = 1;
     while (splits < 8 && tiles * splits * 2 <= slots && p.kblocks / (splits * 2) >= 2) splits *= 2;
+    p.stages = stages;
     p.splits = splits;
     int cols = 32;
-    while (cols < 2 * a.NB) cols *= 2;
+    while (cols < mt * 2 * a.NB) cols *= 2;
     p.tmem_cols = cols;
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * a.NB) >> 3) << 17) | ((uint32_t)(kTcTileM >> 4) << 24);
 
     size_t smem = (size_t)stages * stage_bytes + 1024;
-    const size_t red_bytes = (size_t)a.NB * kTcTileM * 4 + 1024;
+    const size_t red_bytes = (size_t)mt * a.NB * kTcTileM * 4 + 1024;
     if (smem < red_bytes) smem = red_bytes;
     static size_t attr_smem = 0;
     if (smem > attr_smem) {

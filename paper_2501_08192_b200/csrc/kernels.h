@@ -88,6 +88,7 @@ cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s);
 // ---- tcgen05 skinny GEMM (batch >= 16): W [N,K] K-major through TMA
 struct GemmTcArgs {
     CUtensorMap w_map;    // dims (K, N), box (64, 128), 128B swizzle
+    const CUtensorMap *w_map256;  // optional: same tensor with box (64, 256), for two weight tiles per CTA
     CUtensorMap x_map;    // dims (K, 2*NB): hi rows then lo rows; box (64, 2*NB), 128B swizzle
     int B, NB, N, K;      // NB = batch rows per plane (multiple of 16)
     EpilogueArgs epi;
