@@ -277,6 +277,12 @@ def run_ours(args):
         kms[k] = ms / (4 * R)
         del g
     status = max(L.last_status() for L in layers)
+    # ---- the read roofline of this GPU, measured live: a pure 128-bit read stream over 1 GiB (HBM)
+    # and over 32 MiB read repeatedly (L2)
+    big = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
+    read_bw = {"hbm_read_gbs": round(P.preserve_measure_read_bandwidth(big, 5, stream), 1),
+               "l2_read_gbs": round(P.preserve_measure_read_bandwidth(big[: 32 << 20], 50, stream), 1)}
+    del big
     clocks = sampler.summary()      # sampled from before the first timed region to after the last
 
     peak, peak_src = load_peaks()
@@ -328,6 +334,7 @@ def run_ours(args):
                      "traffic": NCU_TRAFFIC.get((P.KERNEL_NAMES[dom], args.config)), "peak_source": peak_src,
                      "algorithmic_bytes_per_launch": kb[dom],
                      "how": "kernel launched alone, back to back over the rotation, from a captured graph"},
+        "read_bandwidth": read_bw, "frac_of_measured_read_bw": round(gbs(ms_on) / read_bw["hbm_read_gbs"], 4),
         "clocks": clocks, "device_status": status,
     }
     if rank == 0:

@@ -73,7 +73,9 @@ extern "C" {
 
 /* flags for preserve_layer_config_t.flags */
 #define PRESERVE_FLAG_NO_GRAPH   1u /* launch kernels directly instead of replaying a CUDA graph     */
-#define PRESERVE_FLAG_PERSIST_L2 2u /* mark prefetched lines as persisting (access-policy window)    */
+#define PRESERVE_FLAG_PERSIST_L2 2u /* prefetch kernels run with a persisting access-policy window over the
+                                       planned weight range; sets this process's persisting-L2 limit to
+                                       3/4 of cudaDevAttrMaxPersistingL2CacheSize at init (off by default) */
 #define PRESERVE_FLAG_NO_EARLY_LAUNCH 4u /* ablation: prefetch into L2 only; consumer kernels are not
                                        launched early to stage operands in shared memory              */
 
@@ -296,6 +298,14 @@ PRESERVE_API int preserve_attention_static(const void *q_hi, const void *q_lo, c
                                            const int32_t *ctx_len_host, int32_t batch, int32_t n_q_heads,
                                            int32_t n_kv_heads, int32_t kv_capacity, void *o_hi, void *o_lo,
                                            void *cuda_stream);
+
+/* Read-bandwidth microbenchmark (the read roofline next to the copy-bandwidth figure): streams
+ * `bytes` (>= 1 MiB, 16-byte aligned) of the caller's device buffer `reps` times (1..1000) with
+ * 128-bit loads from 4 CTAs per SM and writes GB/s to *gbs_out.  A buffer several times larger
+ * than L2 measures HBM; a buffer well inside L2 measures L2.  Synchronises `cuda_stream`;
+ * allocates nothing. */
+PRESERVE_API int preserve_measure_read_bandwidth(const void *device_buffer, size_t bytes, int32_t reps,
+                                                 void *cuda_stream, float *gbs_out);
 
 /* Frees everything the library allocated for the handle (NULL is allowed). */
 PRESERVE_API void preserve_layer_destroy(preserve_layer_t *layer);

@@ -27,6 +27,7 @@ EXPORTS = (
     "preserve_plan_window", "preserve_algorithmic_bytes", "preserve_profile_step",
     "preserve_run_kernel", "preserve_set_trace", "preserve_read_trace",
     "preserve_set_window_delay_ns", "preserve_attention_static",
+    "preserve_measure_read_bandwidth",
 )
 KERNEL_NAMES = ("window_a", "qkv_proj", "attn_splitkv", "attn_merge", "o_proj", "window_b", "gate_up_proj",
                 "down_proj")
@@ -92,6 +93,8 @@ def lib() -> C.CDLL:
         L.preserve_set_trace.argtypes = [C.c_void_p, C.c_int32]
         L.preserve_read_trace.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
         L.preserve_attention_static.argtypes = [C.c_void_p] * 6 + [C.c_int32] * 4 + [C.c_void_p] * 3
+        L.preserve_measure_read_bandwidth.argtypes = [C.c_void_p, C.c_size_t, C.c_int32, C.c_void_p,
+                                                      C.POINTER(C.c_float)]
         L.preserve_layer_get_info.argtypes = [C.c_void_p, C.POINTER(Info)]
         L.preserve_last_status.argtypes = [C.c_void_p]
         L.preserve_last_cuda_error.argtypes = [C.c_void_p]
@@ -253,6 +256,15 @@ def preserve_attention_static(q_hi, q_lo, k_cache, v_cache, ctx_len_dev, ctx_len
     return int(lib().preserve_attention_static(_ptr(q_hi), _ptr(q_lo), _ptr(k_cache), _ptr(v_cache),
                                                _ptr(ctx_len_dev), ctx_len_host.ctypes.data, batch, n_q_heads,
                                                n_kv_heads, cap, _ptr(o_hi), _ptr(o_lo), _stream_ptr(stream)))
+
+
+def preserve_measure_read_bandwidth(buf, reps: int = 10, stream=None) -> float:
+    """GB/s of a pure 128-bit read stream over the CUDA tensor `buf` (see preserve.h)."""
+    out = C.c_float()
+    _check(lib().preserve_measure_read_bandwidth(_ptr(buf), buf.numel() * buf.element_size(), reps,
+                                                 _stream_ptr(stream), C.byref(out)),
+           "preserve_measure_read_bandwidth")
+    return float(out.value)
 
 
 def preserve_decode_chain(layers: Sequence[Layer], ios: Sequence[StepIO], link: bool, stream=None) -> None:

@@ -375,6 +375,23 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
             CK(L, cudaEventRecord(L->prof[mark++], s));          \
     } while (0)
 
+    // Optional: mark the prefetched weight range as persisting in L2 (access-policy window on the
+    // prefetch kernel).  Only the weight arena can be covered (one contiguous window per launch).
+    cudaLaunchAttribute pf_attr[1];
+    auto persist_window = [&](size_t first_off, uint64_t bytes) -> int {
+        if (!(c.flags & PRESERVE_FLAG_PERSIST_L2) || bytes == 0 || L->max_window <= 0)
+            return 0;
+        if (bytes > (uint64_t)L->max_window)
+            bytes = (uint64_t)L->max_window;
+        pf_attr[0].id = cudaLaunchAttributeAccessPolicyWindow;
+        pf_attr[0].val.accessPolicyWindow.base_ptr = L->arena + first_off;
+        pf_attr[0].val.accessPolicyWindow.num_bytes = (size_t)bytes;
+        pf_attr[0].val.accessPolicyWindow.hitRatio = 1.0f;
+        pf_attr[0].val.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
+        pf_attr[0].val.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
+        return 1;
+    };
+
     // ---- window A  ||  prefetch {Wqkv, K/V, Wo}
     if (pf_a) {
         CK(L, cudaEventRecord(L->ev_a, s));
@@ -405,7 +422,9 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
             ++n;
         }
         pa.n_segs = n;
-        CK(L, launch_prefetch(pa, L->prefetch_ctas, L->side, nullptr, 0));
+        // Wqkv and Wo are adjacent in the arena
+        const int na = persist_window(L->off[0], L->planned[0][2] ? L->wbytes[0] + L->planned[0][2] : L->planned[0][0]);
+        CK(L, launch_prefetch(pa, L->prefetch_ctas, L->side, na ? pf_attr : nullptr, na));
     }
     MARK();   // 0: window A starts
     if (WANT(0)) {
@@ -500,7 +519,8 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
                 ++n;
             }
         pa.n_segs = n;
-        CK(L, launch_prefetch(pa, L->prefetch_ctas, L->side, nullptr, 0));
+        const int nb_attr = persist_window(L->off[2], L->planned[1][0] + L->planned[1][1]);
+        CK(L, launch_prefetch(pa, L->prefetch_ctas, L->side, nb_attr ? pf_attr : nullptr, nb_attr));
     }
     MARK();   // 5: window B starts
     if (WANT(5)) {
@@ -887,6 +907,10 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
             L->has256[i] = d.n[i] % 256 == 0 &&
                            make_map_2d(&L->wmap256[i], L->arena + L->off[i], d.k[i], d.n[i], 64, 256);
         }
+    }
+    if ((c.flags & PRESERVE_FLAG_PERSIST_L2) && L->max_persist > 0) {
+        // a context-wide limit of this process: reserve up to 3/4 of what the device allows
+        CKI(cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, (size_t)L->max_persist / 4 * 3));
     }
     CKI(cudaStreamCreateWithFlags(&L->side, cudaStreamNonBlocking));
     CKI(cudaEventCreateWithFlags(&L->ev_a, cudaEventDisableTiming));
