@@ -176,7 +176,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     stream = torch.cuda.Stream()
     info = layers[0].get_info()
-    default_budget = int(info.prefetch_budget)
+    default_budget = int(info.prefetch_budget) if args.budget_bytes < 0 else args.budget_bytes
 
     def barrier():
         torch.cuda.synchronize()
@@ -421,6 +421,7 @@ def main():
     ap.add_argument("--rotation", type=int, default=0, help="layer instances per step (0 = sized from L2)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-kernels", action="store_true", help="skip the isolated per-kernel timing")
+    ap.add_argument("--budget-bytes", type=int, default=-1, help="prefetch budget per window (default: the library's)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
