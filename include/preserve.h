@@ -232,10 +232,13 @@ PRESERVE_API int preserve_run_kernel(preserve_layer_t *layer, const preserve_ste
                                      void *cuda_stream);
 
 /* Timeline trace (diagnostics).  While on, every main-stream kernel of a step records, over all
- * its CTAs, {earliest start, earliest and latest return from the wait on the previous kernel,
- * latest end} in nanoseconds of the GPU's global timer.  preserve_read_trace synchronises the
- * device, copies PRESERVE_N_KERNELS x 4 values (kernel order as in preserve_profile_step) to
- * `out` (host) and clears the slots.  Results of the step do not change. */
+ * its CTAs, PRESERVE_TRACE_SLOTS values in nanoseconds of the GPU's global timer: {earliest
+ * start, earliest and latest return from the wait on the previous kernel, latest end, latest
+ * start, latest end of the operand-streaming loop (0 where a kernel has none), earliest end,
+ * unused}.  preserve_read_trace synchronises the device, copies PRESERVE_N_KERNELS x
+ * PRESERVE_TRACE_SLOTS values (kernel order as in preserve_profile_step) to `out` (host) and
+ * clears the slots.  Results of the step do not change. */
+#define PRESERVE_TRACE_SLOTS 8
 PRESERVE_API int preserve_set_trace(preserve_layer_t *layer, int32_t on);
 PRESERVE_API int preserve_read_trace(preserve_layer_t *layer, int64_t *out);
 

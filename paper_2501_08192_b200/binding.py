@@ -29,6 +29,7 @@ EXPORTS = (
     "preserve_set_window_delay_ns", "preserve_attention_static",
     "preserve_measure_read_bandwidth",
 )
+TRACE_SLOTS = 8
 KERNEL_NAMES = ("window_a", "qkv_proj", "attn_splitkv", "attn_merge", "o_proj", "window_b", "gate_up_proj",
                 "down_proj")
 
@@ -225,10 +226,11 @@ class Layer:
         _check(lib().preserve_set_trace(self.handle, 1 if on else 0), "preserve_set_trace")
 
     def read_trace(self):
-        """[(start, first_wait_return, last_wait_return, end)] per kernel, ns of the GPU global timer."""
-        buf = (C.c_int64 * (4 * len(KERNEL_NAMES)))()
+        """Per kernel: (first start, first wait-return, last wait-return, last end, last start,
+        last end of the streaming loop, first end, unused), ns of the GPU global timer."""
+        buf = (C.c_int64 * (TRACE_SLOTS * len(KERNEL_NAMES)))()
         _check(lib().preserve_read_trace(self.handle, buf), "preserve_read_trace")
-        return [tuple(int(buf[4 * k + i]) for i in range(4)) for k in range(len(KERNEL_NAMES))]
+        return [tuple(int(buf[TRACE_SLOTS * k + i]) for i in range(TRACE_SLOTS)) for k in range(len(KERNEL_NAMES))]
 
     def get_info(self) -> Info:
         info = Info()

@@ -124,7 +124,7 @@ struct preserve_layer {
     uint64_t stamp;
 
     // per-kernel timing (preserve_profile_step): events around the main-stream kernels
-    long long *trace_buf;        // device [PRESERVE_N_KERNELS][4] timeline slots, used when tracing
+    long long *trace_buf;        // device [PRESERVE_N_KERNELS][PRESERVE_TRACE_SLOTS] timeline slots, used when tracing
     bool tracing;
     int only;                    // >= 0: enqueue_step launches only this kernel (preserve_run_kernel)
     bool profiling;
@@ -356,7 +356,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
     const bool pf_a = L->only < 0 && L->planned[0][0] + L->planned[0][1] + L->planned[0][2] > 0;
     const bool pf_b = L->only < 0 && L->planned[1][0] + L->planned[1][1] > 0;
 #define WANT(k) (L->only < 0 || L->only == (k))
-#define TRACE(k) (L->tracing ? L->trace_buf + 4 * (k) : nullptr)
+#define TRACE(k) (L->tracing ? L->trace_buf + PRESERVE_TRACE_SLOTS * (k) : nullptr)
 
     // ---- K/V tensor maps
     if (sp.k_cache != L->k_ptr || sp.v_cache != L->v_ptr) {
@@ -893,7 +893,7 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     CKI(cudaMalloc(&L->stage_in, n_in));
     CKI(cudaMalloc(&L->stage_out, 2 * BH * 2));
     CKI(cudaMalloc(&L->ctx_dev, (size_t)B * 4));
-    CKI(cudaMalloc(&L->trace_buf, sizeof(long long) * 4 * PRESERVE_N_KERNELS));
+    CKI(cudaMalloc(&L->trace_buf, sizeof(long long) * PRESERVE_TRACE_SLOTS * PRESERVE_N_KERNELS));
 
     if (L->tensor_path) {
         // activations as the B operand: [2 * nb_pad, K] = hi rows then lo rows, one box covers both
@@ -1108,10 +1108,11 @@ int preserve_run_kernel(preserve_layer_t *L, const preserve_step_io_t *io, int32
 
 static int reset_trace(preserve_layer *L)
 {
-    long long init[PRESERVE_N_KERNELS][4];
+    long long init[PRESERVE_N_KERNELS][PRESERVE_TRACE_SLOTS];
     for (auto &r : init) {
-        r[0] = r[1] = 0x7fffffffffffffffll;
-        r[2] = r[3] = 0;
+        for (auto &v : r)
+            v = 0;
+        r[0] = r[1] = r[6] = 0x7fffffffffffffffll;     // the slots that take a minimum
     }
     CK(L, cudaMemcpy(L->trace_buf, init, sizeof(init), cudaMemcpyHostToDevice));
     return PRESERVE_OK;
@@ -1130,7 +1131,7 @@ int preserve_read_trace(preserve_layer_t *L, int64_t *out)
     if (!L || !out)
         return PRESERVE_EINVAL;
     CK(L, cudaDeviceSynchronize());
-    CK(L, cudaMemcpy(out, L->trace_buf, sizeof(long long) * 4 * PRESERVE_N_KERNELS, cudaMemcpyDeviceToHost));
+    CK(L, cudaMemcpy(out, L->trace_buf, sizeof(long long) * PRESERVE_TRACE_SLOTS * PRESERVE_N_KERNELS, cudaMemcpyDeviceToHost));
     return reset_trace(L);
 }
 

@@ -303,6 +303,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
             if (lane == 0)
                 mbar_arrive(&sm.empty[st]);
         }
+        trace_streamed(p.trace, threadIdx.x == 0);
         // ---- every warp writes its own partial (max, sum, O) for its 16-key share of the item's
         // tiles; k_attn_merge combines them.  No cross-warp traffic inside the stream loop.
 #pragma unroll
@@ -344,7 +345,7 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(const __grid_const
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_groups = blockDim.x >> 5, n_threads = blockDim.x;
     const int sidx = b * p.nkv + kvh;
-    long long *tr = p.trace ? p.trace + 4 : nullptr;
+    long long *tr = p.trace ? p.trace + kTraceSlots : nullptr;
     trace_start(tr);
     pdl_launch_dependents();
     // first item of this stream: parallel count over the streams before it

@@ -188,8 +188,10 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t sad
                  : "r"(saddr));
 }
 
-// Optional timeline trace: per kernel slot, {earliest start, earliest wait-return, latest
-// wait-return, latest end} in nanoseconds of the global timer, over all CTAs (thread 0 each).
+// Optional timeline trace: per kernel, kTraceSlots values in nanoseconds of the global timer,
+// over all CTAs (thread 0 each): {earliest start, earliest wait-return, latest wait-return,
+// latest end, latest start, latest end of the streaming loop, earliest end, unused}.
+constexpr int kTraceSlots = 8;
 __device__ __forceinline__ long long gtime()
 {
     long long t;
@@ -198,8 +200,16 @@ __device__ __forceinline__ long long gtime()
 }
 __device__ __forceinline__ void trace_start(long long *t)
 {
-    if (t && threadIdx.x == 0)
-        atomicMin(t, gtime());
+    if (t && threadIdx.x == 0) {
+        const long long v = gtime();
+        atomicMin(t, v);
+        atomicMax(t + 4, v);
+    }
+}
+__device__ __forceinline__ void trace_streamed(long long *t, bool elected)
+{
+    if (t && elected)
+        atomicMax(t + 5, gtime());
 }
 __device__ __forceinline__ void trace_waited(long long *t)
 {
@@ -211,8 +221,11 @@ __device__ __forceinline__ void trace_waited(long long *t)
 }
 __device__ __forceinline__ void trace_end(long long *t)
 {
-    if (t && threadIdx.x == 0)
-        atomicMax(t + 3, gtime());
+    if (t && threadIdx.x == 0) {
+        const long long v = gtime();
+        atomicMax(t + 3, v);
+        atomicMin(t + 6, v);
+    }
 }
 
 // Programmatic dependent launch: wait for the producer grid's memory to be

@@ -193,6 +193,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
         if (!have)
             poisoned = 1;
         tc_fence_after();
+        trace_streamed(p.trace, threadIdx.x == 64);
     }
     const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
     float *red = reinterpret_cast<float *>(smem);      // [mt][NB][128] fp32, reuses the ring

@@ -215,6 +215,7 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
             }
         }
 
+        trace_streamed(p.trace, threadIdx.x == 0);
         // ---- warp partial -> shared memory: red[warp][row][b]
         if constexpr (MMA) {
 #pragma unroll

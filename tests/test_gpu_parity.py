@@ -145,8 +145,10 @@ def test_schedule_variants_do_not_change_results(oracle):
                 if trace:
                     tr = dl.layer.read_trace()
                     assert len(tr) == len(P.KERNEL_NAMES)
-                    ends = [e for (_, _, _, e) in tr]
-                    assert all(s <= w1 <= w2 <= e for (s, w1, w2, e) in tr)
+                    assert all(len(r) == P.TRACE_SLOTS for r in tr)
+                    ends = [r[3] for r in tr]
+                    assert all(s <= w1 <= w2 <= e and s <= s2 <= e and e1 <= e
+                               for (s, w1, w2, e, s2, _, e1, _) in tr)
                     assert ends == sorted(ends)            # the main-stream kernels finish in order
             assert dl.layer.last_status() == P.PRESERVE_OK
         finally:
