@@ -88,7 +88,7 @@ struct preserve_layer {
     void *x, *q, *o, *attn_partial, *x2, *a;   // x, q, o, x2, a: split bf16 [2][rows][...] (hi + lo)
     int rows;                                  // batch rows per plane (max_batch, padded to 16 on the tensor path)
     float *part_o, *part_ml;
-    int max_items, attn_grid;
+    int max_items;
     int *status;
 
     // staging for the host-buffer entry point
@@ -475,15 +475,8 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         a.o_plane = a.q_plane;
         a.ctx_len = sp.ctx_len;
         a.B = B; a.nq = c.n_q_heads; a.nkv = c.n_kv_heads; a.cap = cap;
-        a.grid = L->attn_grid;
-        // Work items = runs of 64-key tiles.  Aim at one item per CTA when the whole cache is small
-        // (per-item overhead dominates) and at up to four per CTA when it is large (balance under
-        // ragged lengths); depends only on the lengths and the SM count.
-        uint64_t mult = total_tiles / ((uint64_t)L->attn_grid * 3);
-        mult = mult < 1 ? 1 : (mult > 4 ? 4 : mult);
-        uint64_t tpi = (total_tiles + (uint64_t)L->attn_grid * mult - 1) / ((uint64_t)L->attn_grid * mult);
-        a.tiles_per_item = tpi < 1 ? 1 : (int)tpi;
-        a.max_entries_per_stream = 4 * (int)((max_tiles_seq + a.tiles_per_item - 1) / a.tiles_per_item);
+        plan_attention(total_tiles, L->sm_count, &a.grid, &a.tiles_per_item);
+        a.max_items_per_stream = (int)((max_tiles_seq + a.tiles_per_item - 1) / a.tiles_per_item);
         a.max_items = L->max_items;
         a.part_o = L->part_o;
         a.part_ml = L->part_ml;
@@ -883,10 +876,11 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     CKI(cudaMemset(L->o, 0, 2 * Rq * 2));
     CKI(cudaMemset(L->x2, 0, 2 * RH * 2));
     CKI(cudaMemset(L->a, 0, 2 * RF * 2));
-    L->attn_grid = 2 * L->sm_count;      // two persistent attention CTAs per SM
-    L->max_items = L->attn_grid * 4 + B * c.n_kv_heads + 8;
-    CKI(cudaMalloc(&L->part_o, (size_t)L->max_items * 4 * L->group * kHeadDim * 4));
-    CKI(cudaMalloc(&L->part_ml, (size_t)L->max_items * 4 * L->group * 2 * 4));
+    // work items of the attention kernel: at most 2 CTAs per SM x 4 items each, plus one short
+    // item per (sequence, kv head) from rounding up
+    L->max_items = L->sm_count * 8 + B * c.n_kv_heads + 8;
+    CKI(cudaMalloc(&L->part_o, (size_t)L->max_items * L->group * kHeadDim * 4));
+    CKI(cudaMalloc(&L->part_ml, (size_t)L->max_items * L->group * 2 * 4));
     CKI(cudaMalloc(&L->status, 256));
     CKI(cudaMemset(L->status, 0, 256));
     const size_t n_in = (size_t)(2 * c.tp_degree) * BH * 2;

@@ -8,15 +8,18 @@
 // (sequence, kv head) is one contiguous run and a tile of 64 keys is two TMA
 // boxes of 64 x 64 bf16 (128-byte swizzle) per tensor.
 //
-// Persistent CTAs (two per SM) walk a static list of work items = (sequence,
-// kv head, run of `tiles_per_item` tiles) in address order.  Warp 4 is the
-// producer: one lane issues the TMA loads into a 3-stage ring guarded by
-// full/empty mbarriers (all waits bounded).  Warps 0-3 each own 16 of a tile's
-// 64 keys: S = Q K^T with mma.sync (Q rows = query heads padded to 16, from
-// registers; K via ldmatrix), online softmax in fp32 with exp2, O += P V (V via
-// ldmatrix.trans).  At the end of an item every warp writes its (max, sum, O) as an
-// fp32 partial; k_attn_merge combines the partials of a sequence in fixed order.
-// Nothing depends on timing, so results are bit-stable.
+// Persistent CTAs (one per SM while the whole cache fits a few ring fills, so that
+// the kernels before and after can be co-resident; two per SM for long caches) walk
+// a static list of work items = (sequence, kv head, run of `tiles_per_item` tiles)
+// in address order.  Warp 4 is the producer: one lane issues the TMA loads into a
+// 3-stage ring guarded by full/empty mbarriers (all waits bounded).  Warps 0-3 each
+// own 16 of a tile's 64 keys: S = Q K^T with mma.sync (Q rows = query heads padded
+// to 16, from registers; K via ldmatrix), online softmax in fp32 with exp2,
+// O += P V (V via ldmatrix.trans).  At the end of an item the four warps combine
+// their (max, sum, O) through the ring stage they consumed last and the CTA writes
+// ONE fp32 partial per item (or the final o when the item is the whole sequence).
+// k_attn_merge then combines the partials of a sequence in fixed order.  Nothing
+// depends on timing, so results are bit-stable.
 #include "../../include/preserve.h"
 #include "common.cuh"
 #include "kernels.h"
@@ -41,8 +44,8 @@ struct AttnParams {
     int tiles_per_item;
     int max_items;
     float scale_log2;       // log2(e) / sqrt(d)
-    float *part_o;
-    float *part_ml;
+    float *part_o;          // [item][G][d] CTA partials (unnormalised, relative to the item's max)
+    float *part_ml;         // [item][G][2] (max, sum)
     bf16 *o_out;            // hi plane; lo plane at o_out + o_plane
     size_t o_plane;
     int *status;
@@ -53,8 +56,25 @@ struct AttnSmem {
     alignas(1024) uint8_t stage[kStages][kStageBytes];
     uint64_t full[kStages];
     uint64_t empty[kStages];
-    int item_base[kMaxStreams + 1];
+    float comb_ml[kConsumerWarps][16][2];
+    int item_base[kMaxStreams + 1];      // last: the launch only asks for the entries it needs
 };
+
+__device__ __forceinline__ void consumer_barrier()
+{
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
+}
+
+// Where consumer warp w keeps row r (a query head of the group) of its O partial inside a ring
+// stage: in the 16 key rows of each 64x64 box that only this warp reads, so no other warp can
+// still be reading the bytes it overwrites.  512 B per row, four rows per box slice.
+__device__ __forceinline__ float *comb_row(uint8_t *stage, int w, int r)
+{
+    return reinterpret_cast<float *>(stage + (r >> 2) * kHalfBytes + w * 2048 + (r & 3) * 512);
+}
+// float2 slot of head dims (2c, 2c + 1) within a row: XOR swizzle so that the fragment stores
+// (eight rows x four column pairs per instruction) and the row reads are both conflict-free
+__device__ __forceinline__ int comb_col2(int r, int c) { return c ^ ((r & 3) << 2); }
 
 __device__ __forceinline__ int tiles_of(int ctx) { return (ctx + 1 + kTileKeys - 1) / kTileKeys; }
 
@@ -300,57 +320,88 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
                 }
             }
             __syncwarp();
-            if (lane == 0)
-                mbar_arrive(&sm.empty[st]);
+            if (tile + 1 < t1 && lane == 0)
+                mbar_arrive(&sm.empty[st]);      // the item's last stage is kept for the combine below
         }
         trace_streamed(p.trace, threadIdx.x == 0);
-        // ---- every warp writes its own partial (max, sum, O) for its 16-key share of the item's
-        // tiles; k_attn_merge combines them.  No cross-warp traffic inside the stream loop.
+
+        // ---- combine the four warps' partials through the stage consumed last
+        uint8_t *stage_last = sm.stage[(it + kStages - 1) % kStages];
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
             l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
             l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
-        }
-        const size_t ebase = ((size_t)item * kConsumerWarps + warp) * p.G;
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
             const int row = g + 8 * r;
             if (row < p.G) {
-                float *po = p.part_o + (ebase + row) * kHeadDim + 2 * t;
+                float2 *dst = reinterpret_cast<float2 *>(comb_row(stage_last, warp, row));
 #pragma unroll
                 for (int i = 0; i < 16; ++i)
-                    *reinterpret_cast<float2 *>(po + i * 8) = make_float2(o[i][2 * r], o[i][2 * r + 1]);
-                if (t == 0)
-                    *reinterpret_cast<float2 *>(p.part_ml + (ebase + row) * 2) = make_float2(m_run[r], l_run[r]);
+                    dst[comb_col2(row, i * 4 + t)] = make_float2(o[i][2 * r], o[i][2 * r + 1]);
+                if (t == 0) {
+                    sm.comb_ml[warp][row][0] = m_run[r];
+                    sm.comb_ml[warp][row][1] = l_run[r];
+                }
             }
         }
+        consumer_barrier();
+        const int n_items_stream = sm.item_base[sidx + 1] - sm.item_base[sidx];
+        const int d = threadIdx.x;                       // one head dim per consumer thread
+        for (int r = 0; r < p.G; ++r) {
+            float M = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kConsumerWarps; ++w)
+                M = fmaxf(M, sm.comb_ml[w][r][0]);
+            float acc = 0.f, lsum = 0.f;
+#pragma unroll
+            for (int w = 0; w < kConsumerWarps; ++w) {
+                const float mw = sm.comb_ml[w][r][0];
+                const float c = mw == -INFINITY ? 0.f : exp2f(mw - M);
+                acc += comb_row(stage_last, w, r)[2 * comb_col2(r, d >> 1) + (d & 1)] * c;
+                lsum += sm.comb_ml[w][r][1] * c;
+            }
+            if (n_items_stream == 1) {
+                // the item is the whole sequence: finish here
+                const float ov = acc / lsum;
+                const bf16 hi = __float2bfloat16_rn(ov);
+                const size_t oi = ((size_t)b * p.nq + (size_t)kvh * p.G + r) * kHeadDim + d;
+                p.o_out[oi] = hi;
+                p.o_out[p.o_plane + oi] = __float2bfloat16_rn(ov - __bfloat162float(hi));
+            } else {
+                p.part_o[((size_t)item * p.G + r) * kHeadDim + d] = acc;
+                if (d == 0)
+                    *reinterpret_cast<float2 *>(p.part_ml + ((size_t)item * p.G + r) * 2) = make_float2(M, lsum);
+            }
+        }
+        consumer_barrier();
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0)
+            mbar_arrive(&sm.empty[(it + kStages - 1) % kStages]);
     }
     trace_end(p.trace);
 }
 
-// Merge the partials of one (sequence, query head).  A CTA is 4..16 entry groups (one warp
-// each, chosen from the number of partials per sequence) x 32 lanes of 4 head dims; group g sums
-// entries g, g + groups, ... (independent 128-bit loads, all in flight together), then the group
-// sums are added in fixed order, so the result does not depend on scheduling.
-constexpr int kMergeGroups = 16;
-constexpr int kMergeThreads = kMergeGroups * 32;
-__global__ void __launch_bounds__(kMergeThreads) k_attn_merge(const __grid_constant__ AttnParams p)
+// Merge the item partials of one (sequence, query head).  One warp per partial (each lane four
+// head dims, a single 16-byte load in flight per thread: a read spread over many warps returns in
+// one L2 round trip, the same bytes requested by few warps take several times longer), then the
+// warps' results are added in warp order, so the result does not depend on scheduling.
+constexpr int kMergeMaxWarps = 32;
+__global__ void __launch_bounds__(kMergeMaxWarps * 32) k_attn_merge(const __grid_constant__ AttnParams p)
 {
-    __shared__ float red_s[kMergeThreads / 32];
-    __shared__ int cnt_s[kMergeThreads / 32];
-    __shared__ float4 acc_s[kMergeGroups][32];
-    __shared__ float l_s[kMergeGroups];
+    __shared__ int cnt_s[kMergeMaxWarps];
+    __shared__ float m_s[kMergeMaxWarps], l_s[kMergeMaxWarps];
+    __shared__ float acc_s[kMergeMaxWarps][kHeadDim];
     const int b = blockIdx.x / p.nq, hq = blockIdx.x % p.nq;
     const int kvh = hq / p.G, row = hq % p.G;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n_groups = blockDim.x >> 5, n_threads = blockDim.x;
+    const int n_warps = blockDim.x >> 5;
     const int sidx = b * p.nkv + kvh;
     long long *tr = p.trace ? p.trace + kTraceSlots : nullptr;
     trace_start(tr);
     pdl_launch_dependents();
-    // first item of this stream: parallel count over the streams before it
+    // first item of this stream: parallel count over the streams before it (lengths are inputs)
     int cnt = 0;
-    for (int s2 = tid; s2 < sidx; s2 += n_threads) {
+    for (int s2 = tid; s2 < sidx; s2 += blockDim.x) {
         const int nt = tiles_of(p.ctx_len[s2 / p.nkv]);
         cnt += (nt + p.tiles_per_item - 1) / p.tiles_per_item;
     }
@@ -362,70 +413,70 @@ __global__ void __launch_bounds__(kMergeThreads) k_attn_merge(const __grid_const
     const int n_items = (tiles_of(p.ctx_len[b]) + p.tiles_per_item - 1) / p.tiles_per_item;
     __syncthreads();
     int base = 0;
-    for (int i = 0; i < n_groups; ++i)
+    for (int i = 0; i < n_warps; ++i)
         base += cnt_s[i];
-    pdl_wait();    // the partials come from the split-KV kernel
+    pdl_wait();    // the partials come from the split-KV kernel (every CTA waits, also those with nothing to do)
     trace_waited(tr);
-    const int n_ent = n_items * kConsumerWarps;                 // entry e = item * 4 + consumer warp
-    const size_t stride_ml = (size_t)p.G * 2, stride_o = (size_t)p.G * kHeadDim;
-    const float *ml = p.part_ml + ((size_t)base * kConsumerWarps * p.G + row) * 2;
-    const float *po = p.part_o + ((size_t)base * kConsumerWarps * p.G + row) * kHeadDim + 4 * lane;
-    // One pass: group `warp` takes entries warp, warp + 16, ... in bursts of 8 (all loads of a burst
-    // are independent), keeping a running maximum like the attention kernel does, so every partial
-    // is read exactly once and the reads are a single memory round trip for <= 128 entries.
-    float Mg = -INFINITY, L = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int e0 = warp; e0 < n_ent; e0 += n_groups * 8) {
-        float2 mlv[8];
-        float4 ov[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int e = e0 + u * n_groups;
-            if (e < n_ent) {
-                mlv[u] = *reinterpret_cast<const float2 *>(ml + e * stride_ml);
-                ov[u] = *reinterpret_cast<const float4 *>(po + e * stride_o);
-            } else {
-                mlv[u] = make_float2(-INFINITY, 0.f);
-                ov[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (n_items > 1) {          // a single item was finished by the split-KV kernel itself
+        float Mg = -INFINITY, L = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int e = warp; e < n_items; e += n_warps) {
+            const size_t ent = (size_t)(base + e) * p.G + row;
+            const float2 ml = *reinterpret_cast<const float2 *>(p.part_ml + ent * 2);
+            const float4 ov = *(reinterpret_cast<const float4 *>(p.part_o + ent * kHeadDim) + lane);
+            const float mb = fmaxf(Mg, ml.x);
+            const float c = mb == -INFINITY ? 1.f : exp2f(Mg - mb);
+            const float w = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mb);
+            L = L * c + ml.y * w;
+            acc.x = acc.x * c + ov.x * w; acc.y = acc.y * c + ov.y * w;
+            acc.z = acc.z * c + ov.z * w; acc.w = acc.w * c + ov.w * w;
+            Mg = mb;
+        }
+        *reinterpret_cast<float4 *>(&acc_s[warp][4 * lane]) = acc;
+        if (lane == 0) {
+            m_s[warp] = Mg;
+            l_s[warp] = L;
+        }
+        __syncthreads();
+        if (tid < kHeadDim) {
+            float M = m_s[0];
+            for (int w = 1; w < n_warps; ++w)
+                M = fmaxf(M, m_s[w]);
+            float a = 0.f, l = 0.f;
+            for (int w = 0; w < n_warps; ++w) {
+                const float c = m_s[w] == -INFINITY ? 0.f : exp2f(m_s[w] - M);
+                a += acc_s[w][tid] * c;
+                l += l_s[w] * c;
             }
+            const float ov = a / l;
+            const bf16 hi = __float2bfloat16_rn(ov);
+            const size_t oi = ((size_t)b * p.nq + hq) * kHeadDim + tid;
+            p.o_out[oi] = hi;
+            p.o_out[p.o_plane + oi] = __float2bfloat16_rn(ov - __bfloat162float(hi));
         }
-        float mb = Mg;
-#pragma unroll
-        for (int u = 0; u < 8; ++u)
-            mb = fmaxf(mb, mlv[u].x);
-        const float c = mb == -INFINITY ? 1.f : exp2f(Mg - mb);
-        L *= c; acc.x *= c; acc.y *= c; acc.z *= c; acc.w *= c;
-        Mg = mb;
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const float w = mlv[u].x == -INFINITY ? 0.f : exp2f(mlv[u].x - Mg);
-            L += mlv[u].y * w;
-            acc.x += ov[u].x * w; acc.y += ov[u].y * w; acc.z += ov[u].z * w; acc.w += ov[u].w * w;
-        }
-    }
-    acc_s[warp][lane] = acc;
-    if (lane == 0) {
-        l_s[warp] = L;
-        red_s[warp] = Mg;
-    }
-    __syncthreads();
-    if (tid < kHeadDim) {
-        float M = red_s[0];
-        for (int w = 1; w < n_groups; ++w)
-            M = fmaxf(M, red_s[w]);
-        float a = 0.f, l = 0.f;
-        for (int w = 0; w < n_groups; ++w) {
-            const float c = red_s[w] == -INFINITY ? 0.f : exp2f(red_s[w] - M);
-            a += reinterpret_cast<const float *>(&acc_s[w][0])[tid] * c;
-            l += l_s[w] * c;
-        }
-        const float ov = a / l;
-        const bf16 hi = __float2bfloat16_rn(ov);
-        const size_t oi = ((size_t)b * p.nq + hq) * kHeadDim + tid;
-        p.o_out[oi] = hi;
-        p.o_out[p.o_plane + oi] = __float2bfloat16_rn(ov - __bfloat162float(hi));
     }
     trace_end(tr);
+}
+
+static size_t attn_smem_bytes(int streams)
+{
+    return offsetof(AttnSmem, item_base) + sizeof(int) * (size_t)(streams + 1) + 1024;
+}
+
+void plan_attention(uint64_t total_tiles, int sm_count, int *grid, int *tiles_per_item)
+{
+    // One CTA per SM while the whole cache is at most two ring fills per SM: the ring then holds
+    // most of the CTA's share before the queries exist, and half of every SM's shared memory stays
+    // free for the kernels before and after.  Longer caches are a steady stream: two CTAs per SM
+    // keep twice the bytes in flight.
+    const int g = total_tiles <= (uint64_t)2 * kStages * sm_count ? sm_count : 2 * sm_count;
+    // Work items = runs of 64-key tiles: one item per CTA when the cache is small (per-item overhead
+    // dominates), up to four per CTA when it is large (balance under ragged lengths).
+    uint64_t mult = total_tiles / ((uint64_t)g * 3);
+    mult = mult < 1 ? 1 : (mult > 4 ? 4 : mult);
+    const uint64_t tpi = (total_tiles + (uint64_t)g * mult - 1) / ((uint64_t)g * mult);
+    *grid = g;
+    *tiles_per_item = tpi < 1 ? 1 : (int)tpi;
 }
 
 cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
@@ -449,11 +500,11 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     p.status = a.status;
     p.trace = a.trace;
 
-    const size_t smem = sizeof(AttnSmem) + 1024;
+    const size_t smem = attn_smem_bytes(a.B * a.nkv);
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(k_attn_decode_splitkv, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem);
+                                             (int)attn_smem_bytes(kMaxStreams));
         if (e != cudaSuccess)
             return e;
         attr_set = true;
@@ -477,17 +528,17 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
         if (e != cudaSuccess)
             return e;
     }
+    if (!(phases & 2))
+        return cudaSuccess;
+    // one warp per item partial of the longest sequence (at least the four that write the head dims)
+    int warps = a.max_items_per_stream < 4 ? 4 : (a.max_items_per_stream > kMergeMaxWarps ? kMergeMaxWarps
+                                                                                          : a.max_items_per_stream);
     cudaLaunchConfig_t cfg2 = {};
     cfg2.gridDim = dim3(a.B * a.nq);
-    // merge groups: enough warps that each reads its share of a sequence's partials in one burst of 8
-    int merge_groups = (a.max_entries_per_stream + 7) / 8;
-    merge_groups = merge_groups < 4 ? 4 : (merge_groups > kMergeGroups ? kMergeGroups : merge_groups);
-    cfg2.blockDim = dim3(merge_groups * 32);
+    cfg2.blockDim = dim3(warps * 32);
     cfg2.stream = s;
     cfg2.attrs = at;
     cfg2.numAttrs = pdl_attr(at);
-    if (!(phases & 2))
-        return cudaSuccess;
     return cudaLaunchKernelEx(&cfg2, k_attn_merge, p);
 }
 
@@ -525,13 +576,11 @@ extern "C" int preserve_attention_static(const void *q_hi, const void *q_lo, con
         kv_capacity < 1 || (long long)batch * n_kv_heads > kMaxStreams ||
         (long long)batch * n_kv_heads * kv_capacity > 0x7fffffffll)
         return PRESERVE_ESHAPE;
-    uint64_t total_tiles = 0, max_tiles_seq = 0;
+    uint64_t total_tiles = 0;
     for (int b = 0; b < batch; ++b) {
         if (ctx_len_host[b] < 0 || ctx_len_host[b] >= kv_capacity)
             return PRESERVE_ESHAPE;
-        const uint64_t nt = (uint64_t)(ctx_len_host[b] + 1 + kTileKeys - 1) / kTileKeys;
-        total_tiles += (uint64_t)n_kv_heads * nt;
-        max_tiles_seq = nt > max_tiles_seq ? nt : max_tiles_seq;
+        total_tiles += (uint64_t)n_kv_heads * ((uint64_t)(ctx_len_host[b] + 1 + kTileKeys - 1) / kTileKeys);
     }
 
     // ---- once per device: the array's device address (with that device current)
@@ -552,22 +601,23 @@ extern "C" int preserve_attention_static(const void *q_hi, const void *q_lo, con
             (void)cudaGetLastError();
             return PRESERVE_ECUDA;
         }
-        if (cudaFuncSetAttribute(k_attn_decode_splitkv, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(sizeof(AttnSmem) + 1024)) != cudaSuccess) {
-            (void)cudaGetLastError();
-            return PRESERVE_ECUDA;
-        }
         g_scratch_sms[dev] = sms;
         g_scratch_addr[dev] = addr;
     }
 
     // ---- carve the array: [status word, 256 B][partial O][partial (max, sum)]
     const int G = n_q_heads / n_kv_heads;
-    const int grid = 2 * g_scratch_sms[dev];
-    const uint64_t tpi = (total_tiles + grid - 1) / grid;            // about one work item per CTA
-    const uint64_t max_items = (uint64_t)grid + (uint64_t)batch * n_kv_heads;
-    const uint64_t o_bytes = max_items * kConsumerWarps * G * kHeadDim * sizeof(float);
-    const uint64_t ml_bytes = max_items * kConsumerWarps * G * 2 * sizeof(float);
+    int grid = 0, tpi = 1;
+    plan_attention(total_tiles, g_scratch_sms[dev], &grid, &tpi);
+    uint64_t n_items = 0, max_items_seq = 0;
+    for (int b = 0; b < batch; ++b) {
+        const uint64_t nt = (uint64_t)(ctx_len_host[b] + 1 + kTileKeys - 1) / kTileKeys;
+        const uint64_t ni = (nt + tpi - 1) / tpi;
+        n_items += (uint64_t)n_kv_heads * ni;
+        max_items_seq = ni > max_items_seq ? ni : max_items_seq;
+    }
+    const uint64_t o_bytes = n_items * G * kHeadDim * sizeof(float);
+    const uint64_t ml_bytes = n_items * G * 2 * sizeof(float);
     if (256 + o_bytes + ml_bytes > PRESERVE_STATIC_SCRATCH_BYTES)
         return PRESERVE_ETOOBIG;
     unsigned char *base = static_cast<unsigned char *>(g_scratch_addr[dev]);
@@ -588,9 +638,9 @@ extern "C" int preserve_attention_static(const void *q_hi, const void *q_lo, con
     a.ctx_len = ctx_len;
     a.B = batch; a.nq = n_q_heads; a.nkv = n_kv_heads; a.cap = kv_capacity;
     a.grid = grid;
-    a.tiles_per_item = tpi < 1 ? 1 : (int)tpi;
-    a.max_items = (int)max_items;
-    a.max_entries_per_stream = kConsumerWarps * (int)((max_tiles_seq + a.tiles_per_item - 1) / a.tiles_per_item);
+    a.tiles_per_item = tpi;
+    a.max_items = (int)n_items;
+    a.max_items_per_stream = (int)max_items_seq;
     a.part_o = reinterpret_cast<float *>(base + 256);
     a.part_ml = reinterpret_cast<float *>(base + 256 + o_bytes);
     a.o_out = o_hi;

@@ -108,9 +108,9 @@ struct AttnArgs {
     int grid;             // persistent CTAs
     int tiles_per_item;   // 64-key tiles per work item
     int max_items;        // capacity of the partial buffers
-    int max_entries_per_stream;  // 4 x work items of the longest sequence (sizes the merge CTAs; 0 = unknown)
-    float *part_o;        // fp32 [max_items, 4 consumer warps, G, d]
-    float *part_ml;       // fp32 [max_items, 4, G, 2]
+    float *part_o;        // fp32 [max_items, G, d]: one partial per work item
+    float *part_ml;       // fp32 [max_items, G, 2]
+    int max_items_per_stream;   // work items of the longest sequence (sizes the merge CTAs)
     void *o_out;          // split bf16 [2][rows][nq,d]
     size_t o_plane;
     int *status;
@@ -119,6 +119,9 @@ struct AttnArgs {
     long long *trace;      // optional: two consecutive timeline slots (split-KV, merge)
 };
 cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s);
+// Grid size (persistent CTAs) and tiles per work item for a cache of `total_tiles` 64-key tiles;
+// depends only on the lengths and the SM count.
+void plan_attention(uint64_t total_tiles, int sm_count, int *grid, int *tiles_per_item);
 
 // 2-D bf16 tensor map (rows x cols, cols contiguous), box (box_cols x box_rows), 128-byte swizzle.
 bool encode_bf16_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_cols,
