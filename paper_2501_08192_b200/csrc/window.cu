@@ -1,17 +1,27 @@
 // Communication-window stand-in: what the allreduce plus its epilogue would
 // deliver on a tensor-parallel system (Section 2, "Multi-device inference";
 // Section 3, "Vanilla execution"): h = residual + sum of the P partial-sum
-// buffers, then x = RMSNorm(h) * gain.  One CTA per token row; 128-bit
-// coalesced loads; fp32 accumulation in the fixed order residual, part 0..P-1
-// (part 0 may be fp32: this shard's own result, or the previous layer's in a chain).
-// The kernel is deliberately narrow (B CTAs): during a real allreduce the SMs
-// idle, which is what leaves HBM bandwidth to the prefetch stream.
+// buffers, then x = RMSNorm(h) * gain.  One cluster of up to 8 CTAs per token
+// row, each CTA a slice of the row with one thread per 8 elements: the P + 1
+// 128-bit loads of a thread are all in flight together, and a row's bytes are
+// requested by many warps on several SMs (the same bytes requested by the few
+// warps of one SM take several times longer).  The slices' sums of squares meet
+// through distributed shared memory and are added in rank order.  fp32
+// accumulation in the fixed order residual, part 0..P-1 (part 0 may be fp32: this
+// shard's own result, or the previous layer's in a chain).
+// The kernel stays narrow (at most 8 B small CTAs): during a real allreduce the
+// SMs idle, which is what leaves HBM bandwidth to the prefetch stream.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 #include "kernels.h"
 
+namespace cg = cooperative_groups;
+
 namespace prsv {
 
-constexpr int kWinMaxChunks = 2;   // 8-element chunks per thread; H <= 1024 * 8 * 2
+constexpr int kWinMaxChunks = 2;   // 8-element chunks per thread
+constexpr int kWinMaxCluster = 8;  // CTAs per row
 
 struct WindowParams {
     const uint4 *parts[kMaxParts];
@@ -24,6 +34,7 @@ struct WindowParams {
     uint4 *x_bf16;       // hi plane; the lo plane follows at x_plane uint4s
     size_t x_plane;
     int H;
+    int cluster;         // CTAs per row
     long long *trace;
     int delay_ns;
 };
@@ -31,9 +42,10 @@ struct WindowParams {
 template <bool RESID_F32, bool PART0_F32>
 __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_constant__ WindowParams p)
 {
-    const int row = blockIdx.x;
-    const int chunks = p.H >> 3;                 // uint4 chunks per row
-    const size_t row_off = (size_t)row * chunks;
+    const int row = blockIdx.x / p.cluster, rank = blockIdx.x % p.cluster;
+    const int chunks = (p.H >> 3) / p.cluster;   // uint4 chunks of this CTA's slice of the row
+    const size_t row_off = (size_t)row * (p.H >> 3) + (size_t)rank * chunks;
+    const int gain_off = rank * chunks;
     float v[kWinMaxChunks][8];
     uint4 gn[kWinMaxChunks];
     float ss = 0.f;
@@ -42,7 +54,7 @@ __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_con
 #pragma unroll
     for (int c = 0; c < kWinMaxChunks; ++c) {
         const int ch = threadIdx.x + c * blockDim.x;
-        gn[c] = ch < chunks ? ld_cached(p.gain + ch) : make_uint4(0, 0, 0, 0);
+        gn[c] = ch < chunks ? ld_cached(p.gain + gain_off + ch) : make_uint4(0, 0, 0, 0);
     }
 
     trace_start(p.trace);
@@ -95,6 +107,7 @@ __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_con
     // block reduction of the sum of squares (fixed tree: bit-stable run to run)
     __shared__ float warp_sums[32];
     __shared__ float total;
+    __shared__ float slice_sum;      // this CTA's part, read by the other CTAs of the row
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1)
         ss += __shfl_xor_sync(0xffffffffu, ss, o);
@@ -108,11 +121,23 @@ __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_con
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1)
             t += __shfl_xor_sync(0xffffffffu, t, o);
-        if (lane == 0)
+        if (lane == 0) {
             total = t;
+            slice_sum = t;
+        }
     }
     __syncthreads();
-    const float inv = rsqrtf(total / (float)p.H + p.eps);
+    float row_total = total;
+    if (p.cluster > 1) {
+        // sum of the slices in rank order (the same order in every CTA of the row)
+        cg::cluster_group cluster = cg::this_cluster();
+        cluster.sync();
+        row_total = 0.f;
+        for (int q = 0; q < p.cluster; ++q)
+            row_total += *cluster.map_shared_rank(&slice_sum, q);
+        cluster.sync();      // peers' shared memory must outlive the reads
+    }
+    const float inv = rsqrtf(row_total / (float)p.H + p.eps);
 
     // modelled network time of the allreduce this kernel stands in for: hold the result back until
     // delay_ns after its inputs were complete (bounded by the delay itself)
@@ -173,7 +198,13 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
     p.H = a.H;
     p.trace = a.trace;
     p.delay_ns = a.delay_ns;
-    const int chunks = a.H / 8;
+    // CTAs per row: as many (a power of two, at most 8) as leave every CTA at least 128 threads of
+    // one 8-element chunk each
+    int cl = 1;
+    while (cl < kWinMaxCluster && (a.H / 8) % (cl * 2) == 0 && (a.H / 8) / (cl * 2) >= 128)
+        cl *= 2;
+    p.cluster = cl;
+    const int chunks = a.H / 8 / cl;
     int threads = (chunks + kWinMaxChunks - 1) / kWinMaxChunks;
     if (chunks <= 1024)
         threads = chunks;
@@ -182,12 +213,20 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
         return cudaErrorInvalidValue;
 
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(a.B);
+    cfg.gridDim = dim3(a.B * cl);
     cfg.blockDim = dim3(threads);
     cfg.stream = s;
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     cfg.attrs = at;
-    cfg.numAttrs = pdl_attr(at);
+    int n_attr = pdl_attr(at);
+    if (cl > 1) {
+        at[n_attr].id = cudaLaunchAttributeClusterDimension;
+        at[n_attr].val.clusterDim.x = cl;
+        at[n_attr].val.clusterDim.y = 1;
+        at[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
+    }
+    cfg.numAttrs = n_attr;
     if (a.resid_is_f32)
         return a.part0_is_f32 ? cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<true, true>, p)
                               : cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<true, false>, p);
