@@ -53,6 +53,7 @@ struct GemvParams {
     int warps_k;         // warps of a CTA that split k (1, 2, 4, 8)
     int splits;          // cluster size along k
     int groups;          // row-block groups = row_blocks / (8 / warps_k)
+    int slots;           // ring slots per warp actually used (1, 2 or 4): no more than the warp's run needs
     int *status;
     long long *trace;
     EpilogueArgs epi;
@@ -81,7 +82,8 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
     const int ks = p.splits * p.warps_k, ki = s * p.warps_k + wk;
     const int c_begin = (int)((long long)p.kchunks * ki / ks);
     const int c_end = (int)((long long)p.kchunks * (ki + 1) / ks);
-    uint8_t *ring = wsm + (size_t)warp * (kRingSlots * kUnitChunks * 1024);
+    uint8_t *ring = wsm + (size_t)warp * (p.slots * kUnitChunks * 1024);
+    const uint32_t slot_mask = (uint32_t)p.slots - 1;
 
     trace_start(p.trace);
     pdl_launch_dependents();    // the next kernel may start its own weight fetch right away
@@ -94,7 +96,7 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
         if (p_grp >= p.groups || c_begin >= c_end)
             return;
         const int n = min(kUnitChunks, c_end - p_c);
-        const int slot = n_issued % kRingSlots;
+        const int slot = n_issued & slot_mask;
         const size_t rb = (size_t)p_grp * rbs_per_cta + rbl;
         const uint32_t bytes = (uint32_t)n * 1024u;
         mbar_expect_tx(&bars[warp][slot], bytes);
@@ -112,8 +114,7 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
         for (int i = 0; i < kRingSlots; ++i)
             mbar_init(&bars[warp][i], 1);
         mbar_fence_init();
-#pragma unroll
-        for (int i = 0; i < kRingSlots; ++i)
+        for (int i = 0; i < p.slots; ++i)
             issue_next();
     }
     __syncwarp();
@@ -194,8 +195,8 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
 #pragma unroll
             for (int uu = 0; uu < kBurstUnits; ++uu) {
                 if (uu * kUnitChunks < nb && ok) {
-                    const int slot = n_consumed % kRingSlots;
-                    const uint32_t ph = (n_consumed / kRingSlots) & 1;
+                    const int slot = n_consumed & slot_mask;
+                    const uint32_t ph = (n_consumed >> (p.slots == 4 ? 2 : p.slots - 1)) & 1;
                     ok = mbar_wait(&bars[warp][slot], ph, p.status, ST_TIMEOUT_FULL);
                     if (ok) {
                         const uint4 *wtile =
@@ -304,10 +305,16 @@ static cudaError_t launch_variant(GemvParams &p, int sm_count, cudaStream_t s)
     int clusters = (sm_count * ctas_per_sm) / p.splits;
     if (clusters > p.groups) clusters = p.groups;
     if (clusters < 1) clusters = 1;
+    // ring depth: no deeper than a warp's whole run, so that a small projection leaves the shared
+    // memory to the kernels it shares the SM with
+    const int groups_per_cta = (p.groups + clusters - 1) / clusters;
+    const int chunks_per_warp = (p.kchunks + p.splits * p.warps_k - 1) / (p.splits * p.warps_k);
+    const int units = groups_per_cta * ((chunks_per_warp + kUnitChunks - 1) / kUnitChunks);
+    p.slots = units >= 4 ? 4 : (units >= 2 ? 2 : 1);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(clusters, p.splits, 1);
     cfg.blockDim = dim3(kGemvWarps * 32);
-    cfg.dynamicSmemBytes = kGemvSmemBytes + 128;
+    cfg.dynamicSmemBytes = (size_t)kGemvWarps * p.slots * kUnitChunks * 1024 + 128;
     cfg.stream = s;
     cudaLaunchAttribute at[2];
     int n = pdl_attr(at);

@@ -9,6 +9,9 @@
 // through distributed shared memory and are added in rank order.  fp32
 // accumulation in the fixed order residual, part 0..P-1 (part 0 may be fp32: this
 // shard's own result, or the previous layer's in a chain).
+// Loads of buffers that are inputs of the step are issued before the
+// programmatic-dependent-launch wait; only what an earlier kernel of the step
+// produces (this shard's own partial sum, the fp32 residual) is read after it.
 // The kernel stays narrow (at most 8 B small CTAs): during a real allreduce the
 // SMs idle, which is what leaves HBM bandwidth to the prefetch stream.
 #include <cooperative_groups.h>
@@ -40,7 +43,7 @@ struct WindowParams {
 };
 
 template <bool RESID_F32, bool PART0_F32>
-__global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_constant__ WindowParams p)
+__global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_constant__ WindowParams p)
 {
     const int row = blockIdx.x / p.cluster, rank = blockIdx.x % p.cluster;
     const int chunks = (p.H >> 3) / p.cluster;   // uint4 chunks of this CTA's slice of the row
@@ -59,7 +62,26 @@ __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_con
 
     trace_start(p.trace);
     pdl_launch_dependents();   // the next kernel may start fetching its weights now
-    pdl_wait();                // partial sums come from the preceding kernel in the stream
+
+    // Buffers that are inputs of the step (the peers' partial sums, and the residual / partial 0
+    // unless they are handed over in fp32 by an earlier kernel of the step) do not depend on the
+    // previous kernel either: their loads - the only ones that go to HBM - are issued before the
+    // wait, up to 8 partial buffers per chunk.
+    uint4 pre[kWinMaxChunks][8], pre_res[kWinMaxChunks];
+#pragma unroll
+    for (int c = 0; c < kWinMaxChunks; ++c) {
+        const int ch = threadIdx.x + c * blockDim.x;
+        if (ch < chunks) {
+            if (!RESID_F32)
+                pre_res[c] = ld_stream(reinterpret_cast<const uint4 *>(p.resid) + row_off + ch);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (j < p.n_parts && !(PART0_F32 && j == 0))
+                    pre[c][j] = ld_stream(p.parts[j] + row_off + ch);
+        }
+    }
+
+    pdl_wait();                // this shard's own partial sum comes from the preceding kernel in the stream
     trace_waited(p.trace);
     const long long t_begin = p.delay_ns ? gtime() : 0;   // the modelled collective starts when its inputs exist
 
@@ -73,7 +95,7 @@ __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_con
                 v[c][0] = a.x; v[c][1] = a.y; v[c][2] = a.z; v[c][3] = a.w;
                 v[c][4] = b.x; v[c][5] = b.y; v[c][6] = b.z; v[c][7] = b.w;
             } else {
-                uint4 r = ld_stream(reinterpret_cast<const uint4 *>(p.resid) + row_off + ch);
+                const uint4 r = pre_res[c];
                 v[c][0] = bf_lo(r.x); v[c][1] = bf_hi(r.x); v[c][2] = bf_lo(r.y); v[c][3] = bf_hi(r.y);
                 v[c][4] = bf_lo(r.z); v[c][5] = bf_hi(r.z); v[c][6] = bf_lo(r.w); v[c][7] = bf_hi(r.w);
             }
@@ -83,17 +105,23 @@ __global__ void __launch_bounds__(1024) k_window_reduce_rmsnorm(const __grid_con
                 v[c][0] += a.x; v[c][1] += a.y; v[c][2] += a.z; v[c][3] += a.w;
                 v[c][4] += b.x; v[c][5] += b.y; v[c][6] += b.z; v[c][7] += b.w;
             }
-            // issue the loads of up to 8 partial buffers before the first add, so the row is
-            // fetched in one or two memory round trips instead of one per buffer
-            for (int q0 = 0; q0 < p.n_parts; q0 += 8) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (j < p.n_parts && !(PART0_F32 && j == 0)) {
+                    const uint4 r = pre[c][j];
+                    v[c][0] += bf_lo(r.x); v[c][1] += bf_hi(r.x); v[c][2] += bf_lo(r.y); v[c][3] += bf_hi(r.y);
+                    v[c][4] += bf_lo(r.z); v[c][5] += bf_hi(r.z); v[c][6] += bf_lo(r.w); v[c][7] += bf_hi(r.w);
+                }
+            // (more than 8 partial buffers: the rest in bursts of 8)
+            for (int q0 = 8; q0 < p.n_parts; q0 += 8) {
                 uint4 r[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     if (q0 + j < p.n_parts)
-                        r[j] = PART0_F32 && q0 + j == 0 ? make_uint4(0, 0, 0, 0) : ld_stream(p.parts[q0 + j] + row_off + ch);
+                        r[j] = ld_stream(p.parts[q0 + j] + row_off + ch);
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
-                    if (q0 + j < p.n_parts && !(PART0_F32 && q0 + j == 0)) {
+                    if (q0 + j < p.n_parts) {
                         v[c][0] += bf_lo(r[j].x); v[c][1] += bf_hi(r[j].x); v[c][2] += bf_lo(r[j].y); v[c][3] += bf_hi(r[j].y);
                         v[c][4] += bf_lo(r[j].z); v[c][5] += bf_hi(r[j].z); v[c][6] += bf_lo(r[j].w); v[c][7] += bf_hi(r[j].w);
                     }
@@ -206,10 +234,10 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
     p.cluster = cl;
     const int chunks = a.H / 8 / cl;
     int threads = (chunks + kWinMaxChunks - 1) / kWinMaxChunks;
-    if (chunks <= 1024)
+    if (chunks <= 512)
         threads = chunks;
     threads = ((threads + 31) / 32) * 32;
-    if (threads > 1024 || threads * kWinMaxChunks < chunks)
+    if (threads > 512 || threads * kWinMaxChunks < chunks)
         return cudaErrorInvalidValue;
 
     cudaLaunchConfig_t cfg = {};
