@@ -59,14 +59,17 @@ struct GemvParams {
     EpilogueArgs epi;
 };
 
-template <int NB, bool MMA>
-__global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_constant__ GemvParams p)
+// RB = 16-row blocks per warp: with two, every activation fragment a warp loads is used for two
+// weight tiles, which halves the activation traffic from L2 (for batch 8 it is otherwise as large
+// as the weight stream itself, and an SM takes in only ~50 GB/s in total).
+template <int NB, bool MMA, int RB>
+__global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid_constant__ GemvParams p)
 {
     constexpr int NTB = MMA ? NB / 8 : 1;   // n-tiles that cover the batch
     constexpr int NT = 2 * NTB;             // hi planes then lo planes of the activations
     constexpr int NX = MMA ? NT : 2 * NB;   // activation fragments (uint4) per tile
-    __shared__ float red[kGemvWarps][16][NB];       // per-warp partials
-    __shared__ float cta_part[kGemvWarps][16][NB];  // per-row-block CTA partials (read across the cluster)
+    __shared__ float red[kGemvWarps][RB * 16][NB];       // per-warp partials
+    __shared__ float cta_part[kGemvWarps * RB][16][NB];  // per-row-block CTA partials (read across the cluster)
     __shared__ uint64_t bars[kGemvWarps][kRingSlots];
     __shared__ EpilogueTables tabs;
     extern __shared__ uint8_t gemv_smem_raw[];
@@ -74,8 +77,8 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
-    const int rbs_per_cta = kGemvWarps / p.warps_k;
-    const int rbl = warp / p.warps_k, wk = warp % p.warps_k;
+    const int rbs_per_cta = kGemvWarps / p.warps_k * RB;
+    const int rbl = warp / p.warps_k * RB, wk = warp % p.warps_k;   // rbl: first of this warp's row blocks in the group
     const int s = blockIdx.y;                        // == cluster rank along k
 
     // this warp's run of k-chunks: part ki of ks = splits * warps_k equal parts (same for every group)
@@ -88,25 +91,40 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
     trace_start(p.trace);
     pdl_launch_dependents();    // the next kernel may start its own weight fetch right away
 
-    // ---- producer side of this warp's ring (lane 0 only)
-    int p_grp = blockIdx.x, p_c = c_begin;           // next unit to fetch
+    // The activation fragments of kBurst tiles are requested in one burst (their L2 latency is paid
+    // once per burst) and used for the warp's RB row blocks: <= 64 registers of fragments.
+    constexpr int kBurstBase = NX <= 2 ? 8 : (NX <= 4 ? 4 : 2);
+    constexpr int kBurst = kBurstBase / RB >= kUnitChunks ? kBurstBase / RB : kUnitChunks;
+    constexpr int kBurstUnits = kBurst / kUnitChunks;
+
+    // ---- producer side of this warp's ring (lane 0 only): units in consumption order - per burst of
+    // k, the units of row block 0, then those of row block 1
+    int p_grp = blockIdx.x, p_c0 = c_begin, p_r = 0, p_u = 0;   // next unit: burst start, row block, unit in burst
     uint32_t n_issued = 0;
     const uint64_t pol = policy_evict_first();       // every weight byte is read once per step
     auto issue_next = [&]() {
         if (p_grp >= p.groups || c_begin >= c_end)
             return;
+        const int p_c = p_c0 + p_u * kUnitChunks;
         const int n = min(kUnitChunks, c_end - p_c);
         const int slot = n_issued & slot_mask;
-        const size_t rb = (size_t)p_grp * rbs_per_cta + rbl;
+        const size_t rb = (size_t)p_grp * rbs_per_cta + rbl + p_r;
         const uint32_t bytes = (uint32_t)n * 1024u;
         mbar_expect_tx(&bars[warp][slot], bytes);
         bulk_load_hint(ring + slot * (kUnitChunks * 1024),
                        reinterpret_cast<const uint8_t *>(p.w) + (rb * p.kchunks + p_c) * 1024, bytes, &bars[warp][slot], pol);
         ++n_issued;
-        p_c += kUnitChunks;
-        if (p_c >= c_end) {
-            p_c = c_begin;
-            p_grp += gridDim.x;
+        ++p_u;
+        if (p_u == kBurstUnits || p_c0 + p_u * kUnitChunks >= c_end) {
+            p_u = 0;
+            if (++p_r == RB) {
+                p_r = 0;
+                p_c0 += kBurst;
+                if (p_c0 >= c_end) {
+                    p_c0 = c_begin;
+                    p_grp += gridDim.x;
+                }
+            }
         }
     };
     if (lane == 0) {
@@ -145,19 +163,21 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
     uint32_t n_consumed = 0;
     bool ok = true;
     for (int grp = blockIdx.x; grp < p.groups; grp += gridDim.x) {
-        float acc[MMA ? NT : 2 * NB][MMA ? 4 : 1];
+        float acc[RB][MMA ? NT : 2 * NB][MMA ? 4 : 1];
 #pragma unroll
-        for (int i = 0; i < (MMA ? NT : 2 * NB); ++i)
+        for (int r = 0; r < RB; ++r)
 #pragma unroll
-            for (int j = 0; j < (MMA ? 4 : 1); ++j)
-                acc[i][j] = 0.f;
+            for (int i = 0; i < (MMA ? NT : 2 * NB); ++i)
+#pragma unroll
+                for (int j = 0; j < (MMA ? 4 : 1); ++j)
+                    acc[r][i][j] = 0.f;
 
-        auto compute = [&](const uint4 &wl, const uint4 &wh, const uint4 (&xq)[NX]) {
+        auto compute = [&](float (&a_)[MMA ? NT : 2 * NB][MMA ? 4 : 1], const uint4 &wl, const uint4 &wh, const uint4 (&xq)[NX]) {
             if constexpr (MMA) {
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
-                    mma_bf16_16816(acc[nt], wl.x, wh.x, wl.y, wh.y, xq[nt].x, xq[nt].y);
-                    mma_bf16_16816(acc[nt], wl.z, wh.z, wl.w, wh.w, xq[nt].z, xq[nt].w);
+                    mma_bf16_16816(a_[nt], wl.x, wh.x, wl.y, wh.y, xq[nt].x, xq[nt].y);
+                    mma_bf16_16816(a_[nt], wl.z, wh.z, wl.w, wh.w, xq[nt].z, xq[nt].w);
                 }
             } else {
                 const float l0 = bf_lo(wl.x), l1 = bf_hi(wl.x), l2 = bf_lo(wl.y), l3 = bf_hi(wl.y);
@@ -171,20 +191,17 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
                     const float x2 = bf_lo(xh.y) + bf_lo(xl.y), x3 = bf_hi(xh.y) + bf_hi(xl.y);
                     const float x4 = bf_lo(xh.z) + bf_lo(xl.z), x5 = bf_hi(xh.z) + bf_hi(xl.z);
                     const float x6 = bf_lo(xh.w) + bf_lo(xl.w), x7 = bf_hi(xh.w) + bf_hi(xl.w);
-                    float a = acc[2 * b][0], c = acc[2 * b + 1][0];
+                    float a = a_[2 * b][0], c = a_[2 * b + 1][0];
                     a = fmaf(l0, x0, a); a = fmaf(l1, x1, a); a = fmaf(l2, x2, a); a = fmaf(l3, x3, a);
                     a = fmaf(l4, x4, a); a = fmaf(l5, x5, a); a = fmaf(l6, x6, a); a = fmaf(l7, x7, a);
                     c = fmaf(h0, x0, c); c = fmaf(h1, x1, c); c = fmaf(h2, x2, c); c = fmaf(h3, x3, c);
                     c = fmaf(h4, x4, c); c = fmaf(h5, x5, c); c = fmaf(h6, x6, c); c = fmaf(h7, x7, c);
-                    acc[2 * b][0] = a; acc[2 * b + 1][0] = c;
+                    a_[2 * b][0] = a; a_[2 * b + 1][0] = c;
                 }
             }
         };
 
-        // ---- stream this warp's run through its ring.  The activation fragments of up to 8 tiles
-        // are requested in one burst, so their L2 latency is paid once per burst.
-        constexpr int kBurst = NX <= 2 ? 8 : (NX <= 4 ? 4 : 2);     // tiles per burst: <= 64 registers of x
-        constexpr int kBurstUnits = kBurst / kUnitChunks;
+        // ---- stream this warp's run through its ring
         for (int c0 = c_begin; ok && c0 < c_end; c0 += kBurst) {
             const int nb = min(kBurst, c_end - c0);
             uint4 xq[kBurst][NX];
@@ -193,47 +210,53 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
                 if (u < nb)
                     load_x(c0 + u, xq[u]);
 #pragma unroll
-            for (int uu = 0; uu < kBurstUnits; ++uu) {
-                if (uu * kUnitChunks < nb && ok) {
-                    const int slot = n_consumed & slot_mask;
-                    const uint32_t ph = (n_consumed >> (p.slots == 4 ? 2 : p.slots - 1)) & 1;
-                    ok = mbar_wait(&bars[warp][slot], ph, p.status, ST_TIMEOUT_FULL);
-                    if (ok) {
-                        const uint4 *wtile =
-                            reinterpret_cast<const uint4 *>(ring + slot * (kUnitChunks * 1024)) + lane * 2;
+            for (int r = 0; r < RB; ++r) {
 #pragma unroll
-                        for (int u = 0; u < kUnitChunks; ++u)
-                            if (uu * kUnitChunks + u < nb) {
-                                const uint4 wl = wtile[u * 64], wh = wtile[u * 64 + 1];
-                                compute(wl, wh, xq[uu * kUnitChunks + u]);
-                            }
+                for (int uu = 0; uu < kBurstUnits; ++uu) {
+                    if (uu * kUnitChunks < nb && ok) {
+                        const int slot = n_consumed & slot_mask;
+                        const uint32_t ph = (n_consumed >> (p.slots == 4 ? 2 : p.slots - 1)) & 1;
+                        ok = mbar_wait(&bars[warp][slot], ph, p.status, ST_TIMEOUT_FULL);
+                        if (ok) {
+                            const uint4 *wtile =
+                                reinterpret_cast<const uint4 *>(ring + slot * (kUnitChunks * 1024)) + lane * 2;
+#pragma unroll
+                            for (int u = 0; u < kUnitChunks; ++u)
+                                if (uu * kUnitChunks + u < nb) {
+                                    const uint4 wl = wtile[u * 64], wh = wtile[u * 64 + 1];
+                                    compute(acc[r], wl, wh, xq[uu * kUnitChunks + u]);
+                                }
+                        }
+                        ++n_consumed;
+                        __syncwarp();
+                        if (lane == 0 && ok)
+                            issue_next();       // the slot just read is free again
                     }
-                    ++n_consumed;
-                    __syncwarp();
-                    if (lane == 0 && ok)
-                        issue_next();       // the slot just read is free again
                 }
             }
         }
 
         trace_streamed(p.trace, threadIdx.x == 0);
-        // ---- warp partial -> shared memory: red[warp][row][b]
-        if constexpr (MMA) {
+        // ---- warp partial -> shared memory: red[warp][row block of the warp * 16 + row][b]
 #pragma unroll
-            for (int nt = 0; nt < NTB; ++nt) {
-                red[warp][g][nt * 8 + 2 * t] = acc[nt][0] + acc[NTB + nt][0];
-                red[warp][g][nt * 8 + 2 * t + 1] = acc[nt][1] + acc[NTB + nt][1];
-                red[warp][g + 8][nt * 8 + 2 * t] = acc[nt][2] + acc[NTB + nt][2];
-                red[warp][g + 8][nt * 8 + 2 * t + 1] = acc[nt][3] + acc[NTB + nt][3];
-            }
-        } else {
+        for (int r = 0; r < RB; ++r) {
+            if constexpr (MMA) {
 #pragma unroll
-            for (int i = 0; i < 2 * NB; ++i) {
-                float v = acc[i][0];
-                v += __shfl_xor_sync(0xffffffffu, v, 1);
-                v += __shfl_xor_sync(0xffffffffu, v, 2);
-                if (t == 0)
-                    red[warp][g + 8 * (i & 1)][i >> 1] = v;
+                for (int nt = 0; nt < NTB; ++nt) {
+                    red[warp][r * 16 + g][nt * 8 + 2 * t] = acc[r][nt][0] + acc[r][NTB + nt][0];
+                    red[warp][r * 16 + g][nt * 8 + 2 * t + 1] = acc[r][nt][1] + acc[r][NTB + nt][1];
+                    red[warp][r * 16 + g + 8][nt * 8 + 2 * t] = acc[r][nt][2] + acc[r][NTB + nt][2];
+                    red[warp][r * 16 + g + 8][nt * 8 + 2 * t + 1] = acc[r][nt][3] + acc[r][NTB + nt][3];
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 2 * NB; ++i) {
+                    float v = acc[r][i][0];
+                    v += __shfl_xor_sync(0xffffffffu, v, 1);
+                    v += __shfl_xor_sync(0xffffffffu, v, 2);
+                    if (t == 0)
+                        red[warp][r * 16 + g + 8 * (i & 1)][i >> 1] = v;
+                }
             }
         }
         __syncthreads();
@@ -241,9 +264,10 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
         // ---- sum over the warps that split k (fixed order) -> cta_part[rbl][row][b]
         for (int i = threadIdx.x; i < rbs_per_cta * 16 * NB; i += blockDim.x) {
             const int b = i % NB, row = (i / NB) % 16, rl = i / (16 * NB);
+            const int wrow = rl / RB, r = rl % RB;       // warp row of the CTA, row block of that warp
             float v = 0.f;
             for (int k = 0; k < p.warps_k; ++k)
-                v += red[rl * p.warps_k + k][row][b];
+                v += red[wrow * p.warps_k + k][r * 16 + row][b];
             cta_part[rl][row][b] = v;
         }
 
@@ -285,31 +309,41 @@ __global__ void __launch_bounds__(kGemvWarps * 32) k_gemv_splitk(const __grid_co
     trace_end(p.trace);
 }
 
-template <int NB, bool MMA>
+template <int NB, bool MMA, int RB>
 static cudaError_t launch_variant(GemvParams &p, int sm_count, cudaStream_t s)
 {
-    static int ctas_per_sm = 0;
-    if (!ctas_per_sm) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemv_splitk<NB, MMA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(k_gemv_splitk<NB, MMA, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kGemvSmemBytes + 128);
         if (e != cudaSuccess)
             return e;
-        int n = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_gemv_splitk<NB, MMA>, kGemvWarps * 32,
-                                                          kGemvSmemBytes + 128);
-        if (e != cudaSuccess)
-            return e;
-        ctas_per_sm = n < 1 ? 1 : n;
+        attr_done = true;
     }
-    // one wave at most: clusters beyond what is co-resident become extra loop iterations
-    int clusters = (sm_count * ctas_per_sm) / p.splits;
+    // Mapping: k is split over the 8 warps of a CTA while every warp still gets at least two
+    // tiles (otherwise fewer warps split k and the others take further row blocks); cluster ranks
+    // add splits only while the grid stays within the co-resident CTAs; groups beyond the grid
+    // become further loop iterations.  Depends only on the shapes and the SM count, never on the
+    // prefetch setting.
+    int wk = kGemvWarps;
+    while (wk > 1 && p.kchunks / wk < 2 && p.row_blocks % (2 * RB * kGemvWarps / wk) == 0) wk /= 2;
+    p.warps_k = wk;
+    p.groups = p.row_blocks / (kGemvWarps / wk * RB);
+    // CTAs per SM: one when a ring per SM holds the whole matrix (it is then in shared memory before
+    // the activations exist, and the rest of the SM stays free for the kernels around); two for
+    // larger matrices, which are a steady stream that needs twice the bytes in flight per SM.
+    const int per_sm = (size_t)p.N * p.K * 2 <= (size_t)sm_count * kGemvSmemBytes ? 1 : 2;
+    int splits = 1;
+    while (splits < 8 && p.groups * splits * 2 <= sm_count * per_sm && p.kchunks / (wk * splits * 2) >= 2) splits *= 2;
+    p.splits = splits;
+    int clusters = sm_count * per_sm / p.splits;
     if (clusters > p.groups) clusters = p.groups;
     if (clusters < 1) clusters = 1;
     // ring depth: no deeper than a warp's whole run, so that a small projection leaves the shared
     // memory to the kernels it shares the SM with
     const int groups_per_cta = (p.groups + clusters - 1) / clusters;
     const int chunks_per_warp = (p.kchunks + p.splits * p.warps_k - 1) / (p.splits * p.warps_k);
-    const int units = groups_per_cta * ((chunks_per_warp + kUnitChunks - 1) / kUnitChunks);
+    const int units = groups_per_cta * RB * ((chunks_per_warp + kUnitChunks - 1) / kUnitChunks);
     p.slots = units >= 4 ? 4 : (units >= 2 ? 2 : 1);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(clusters, p.splits, 1);
@@ -327,7 +361,7 @@ static cudaError_t launch_variant(GemvParams &p, int sm_count, cudaStream_t s)
     }
     cfg.attrs = at;
     cfg.numAttrs = n;
-    return cudaLaunchKernelEx(&cfg, k_gemv_splitk<NB, MMA>, p);
+    return cudaLaunchKernelEx(&cfg, k_gemv_splitk<NB, MMA, RB>, p);
 }
 
 cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s)
@@ -345,24 +379,13 @@ cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s)
     p.status = a.status;
     p.trace = a.trace;
 
-    // Mapping: k is split over the 8 warps of a CTA while every warp still gets at least two
-    // tiles (otherwise fewer warps split k and the others take further row blocks); cluster ranks
-    // add splits only while there are fewer row-block groups than SMs.  Larger clusters are
-    // avoided: they fragment the co-resident capacity and cause a second wave.  Depends only on
-    // the shapes and the SM count, never on the prefetch setting.
-    int wk = kGemvWarps;
-    while (wk > 1 && p.kchunks / wk < 2 && p.row_blocks % (2 * kGemvWarps / wk) == 0) wk /= 2;
-    p.warps_k = wk;
-    p.groups = p.row_blocks / (kGemvWarps / wk);
-    int splits = 1;
-    while (splits < 8 && p.groups * splits < sm_count && p.kchunks / (wk * splits * 2) >= 2) splits *= 2;
-    p.splits = splits;
-
-    if (a.B == 1) return launch_variant<1, false>(p, sm_count, s);
-    if (a.B == 2) return launch_variant<2, false>(p, sm_count, s);
-    if (a.B <= 4) return launch_variant<4, false>(p, sm_count, s);
-    if (a.B <= 8) return launch_variant<8, true>(p, sm_count, s);
-    return launch_variant<16, true>(p, sm_count, s);
+    // two row blocks per warp whenever the matrix has enough row blocks to still fill the SMs
+    const bool two = p.row_blocks % 2 == 0 && p.row_blocks >= 32;
+    if (a.B == 1) return two ? launch_variant<1, false, 2>(p, sm_count, s) : launch_variant<1, false, 1>(p, sm_count, s);
+    if (a.B == 2) return two ? launch_variant<2, false, 2>(p, sm_count, s) : launch_variant<2, false, 1>(p, sm_count, s);
+    if (a.B <= 4) return two ? launch_variant<4, false, 2>(p, sm_count, s) : launch_variant<4, false, 1>(p, sm_count, s);
+    if (a.B <= 8) return two ? launch_variant<8, true, 2>(p, sm_count, s) : launch_variant<8, true, 1>(p, sm_count, s);
+    return two ? launch_variant<16, true, 2>(p, sm_count, s) : launch_variant<16, true, 1>(p, sm_count, s);
 }
 
 }  // namespace prsv
