@@ -12,13 +12,15 @@
 //               into a multi-stage shared-memory ring, mbarrier full/empty
 //   warp 1    : allocates TMEM, issues tcgen05.mma (kind::f16, bf16 in, fp32
 //               accumulate in TMEM), tcgen05.commit frees ring slots
-//   warps 2-5 : epilogue - tcgen05.ld the accumulator (lane = output row), split-K
+//   warps 2.. : epilogue (8 or 16 warps) - tcgen05.ld the accumulator (lane = output row; the warps of
+//               a TMEM lane group share the columns), split-K
 //               reduction through distributed shared memory of the cluster in rank
 //               order, fused epilogue (epilogue.cuh)
 // Every mbarrier wait is bounded; a wait that gives up records a status code,
 // poisons the rest of the CTA's work, and the CTA still reaches every barrier
 // and frees its TMEM.
 #include <cooperative_groups.h>
+#include <type_traits>
 
 #include "epilogue.cuh"
 
@@ -27,7 +29,9 @@ namespace cg = cooperative_groups;
 namespace prsv {
 
 constexpr int kTcMaxStages = 12;
-constexpr int kTcThreads = 192;
+constexpr int kTcMaxEpiWarps = 16;        // 2-4 per TMEM lane group: the epilogue is a chain of short dependent
+                                          // operations per output, so its speed is set by how many warps run it
+constexpr int kTcMaxThreads = (2 + kTcMaxEpiWarps) * 32;
 constexpr int kTcBlockK = 64;
 constexpr int kTcTileM = 128;
 constexpr int kATileBytes = kTcTileM * kTcBlockK * 2;   // 16 KiB
@@ -82,7 +86,7 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16])
         v[i] = __uint_as_float(r[i]);
 }
 
-__global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_constant__ GemmTcParams p)
+__global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_constant__ GemmTcParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -187,6 +191,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
     const int lane_grp = warp & 3;          // TMEM lanes this warp may read: 32 * (warp % 4)
     const int row = lane_grp * 32 + lane;   // row of the tile
     const int nchunks = p.NB / 16;
+    const int sub = warp >= 2 ? (warp - 2) >> 2 : 0;     // which of the lane group's warps this is
+    const int kSubs = ((int)blockDim.x / 32 - 2) / 4;    // warps per lane group
     bool have = false;
     if (warp >= 2) {
         have = mbar_wait(&accum_bar, 0, p.status, ST_TIMEOUT_MMA);
@@ -221,14 +227,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
         // whole cluster.
         cg::cluster_group cluster = cg::this_cluster();
         if (warp >= 2) {
-            for (int m = 0; m < p.mt; ++m)
-                for (int c = 0; c < nchunks; ++c) {
-                    float v[16];
-                    load_chunk(m, c, v);
+            for (int j = sub; j < p.mt * nchunks; j += kSubs) {      // the lane group's warps share the chunks
+                const int m = j / nchunks, c = j % nchunks;
+                float v[16];
+                load_chunk(m, c, v);
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        red[((size_t)m * p.NB + c * 16 + i) * kTcTileM + row] = v[i];
-                }
+                for (int i = 0; i < 16; ++i)
+                    red[((size_t)m * p.NB + c * 16 + i) * kTcTileM + row] = v[i];
+            }
         }
         cluster.sync();
         if (warp >= 2) {
@@ -238,61 +244,73 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tcgen05(const __grid_con
                 remote[q] = cluster.map_shared_rank(red, q < p.splits ? q : 0) + row;
             const int cols = p.NB / p.splits;             // columns finished by this rank (>= 2, even)
             const int n_pairs = p.mt * cols / 2;
-            // Remote loads of the next column pair are issued before the current pair is finished
-            // (its stores would otherwise fence them off), hiding most of the ~800-cycle latency of
-            // distributed shared memory.
-            auto fetch = [&](int it, float (&t)[2][8]) {
-                const int m = it / (cols / 2), b0 = s * cols + 2 * (it % (cols / 2));
+            // The remote loads of a block of column pairs (16 values per rank slot in flight) are
+            // issued before the first pair of the block is finished: distributed shared memory has a
+            // latency of ~800 cycles, so a thread that fetched pair by pair would spend that long on
+            // each of its mt * cols / 2 pairs.
+            auto run = [&](auto sp_tag) {
+                constexpr int SP = decltype(sp_tag)::value;
+                constexpr int D = 16 / SP;                 // pairs per block
+                // (this warp's pairs: sub, sub + kSubs, ...)
+                for (int it0 = sub; it0 < n_pairs; it0 += D * kSubs) {
+                    float buf[D][2][SP];
 #pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    if (q < p.splits) {
-                        t[0][q] = remote[q][((size_t)m * p.NB + b0 + 0) * kTcTileM];
-                        t[1][q] = remote[q][((size_t)m * p.NB + b0 + 1) * kTcTileM];
+                    for (int d = 0; d < D; ++d) {
+                        const int it = it0 + d * kSubs;
+                        if (it < n_pairs) {
+                            const int m = it / (cols / 2), b0 = s * cols + 2 * (it % (cols / 2));
+#pragma unroll
+                            for (int q = 0; q < SP; ++q) {
+                                buf[d][0][q] = remote[q][((size_t)m * p.NB + b0 + 0) * kTcTileM];
+                                buf[d][1][q] = remote[q][((size_t)m * p.NB + b0 + 1) * kTcTileM];
+                            }
+                        }
                     }
+#pragma unroll
+                    for (int d = 0; d < D; ++d) {
+                        const int it = it0 + d * kSubs;
+                        if (it < n_pairs) {
+                            const int m = it / (cols / 2), b0 = s * cols + 2 * (it % (cols / 2));
+                            const int pair = ((tile * p.mt + m) * kTcTileM + row) >> 1;
+                            float mine[2] = {0.f, 0.f};
+#pragma unroll
+                            for (int q = 0; q < SP; ++q) {       // rank order
+                                mine[0] += buf[d][0][q];
+                                mine[1] += buf[d][1][q];
+                            }
+#pragma unroll
+                            for (int i = 0; i < 2; ++i) {
+                                const float other = __shfl_xor_sync(0xffffffffu, mine[i], 1);
+                                const int b = b0 + i;
+                                if (i == par && b < p.B && !poisoned)
+                                    apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? other : mine[i],
+                                                   par ? mine[i] : other);
+                            }
+                        }
+                    }
+                }
             };
-            float cur[2][8], nxt[2][8];
-            fetch(0, cur);
-            for (int it = 0; it < n_pairs; ++it) {
-                if (it + 1 < n_pairs)
-                    fetch(it + 1, nxt);
-                const int m = it / (cols / 2), b0 = s * cols + 2 * (it % (cols / 2));
-                const int pair = ((tile * p.mt + m) * kTcTileM + row) >> 1;
-                float mine[2] = {0.f, 0.f};
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    if (q < p.splits) {
-                        mine[0] += cur[0][q];
-                        mine[1] += cur[1][q];
-                    }
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const float other = __shfl_xor_sync(0xffffffffu, mine[i], 1);
-                    const int b = b0 + i;
-                    if (i == par && b < p.B && !poisoned)
-                        apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? other : mine[i], par ? mine[i] : other);
-                }
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    cur[0][q] = nxt[0][q];
-                    cur[1][q] = nxt[1][q];
-                }
-            }
+            if (p.splits == 2)
+                run(std::integral_constant<int, 2>());
+            else if (p.splits == 4)
+                run(std::integral_constant<int, 4>());
+            else
+                run(std::integral_constant<int, 8>());
         }
         cluster.sync();        // peers' shared memory must outlive the reads
     } else if (warp >= 2) {
-        for (int m = 0; m < p.mt; ++m) {
+        for (int j = sub; j < p.mt * nchunks; j += kSubs) {
+            const int m = j / nchunks, c = j % nchunks;
             const int pair = ((tile * p.mt + m) * kTcTileM + row) >> 1;
-            for (int c = 0; c < nchunks; ++c) {
-                float v[16];
-                load_chunk(m, c, v);
+            float v[16];
+            load_chunk(m, c, v);
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float mine = v[i];
-                    const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
-                    const int b = c * 16 + i;
-                    if ((i & 1) == par && b < p.B && !poisoned)
-                        apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? other : mine, par ? mine : other);
-                }
+            for (int i = 0; i < 16; ++i) {
+                const float mine = v[i];
+                const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
+                const int b = c * 16 + i;
+                if ((i & 1) == par && b < p.B && !poisoned)
+                    apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? other : mine, par ? mine : other);
             }
         }
     }
@@ -369,7 +387,10 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(tiles, splits, 1);
-    cfg.blockDim = dim3(kTcThreads);
+    // epilogue warps: 16 when the CTA has the SM to itself and enough column pairs per thread to share,
+    // else 8 (two CTAs per SM must share the registers)
+    const int epi_warps = (per_sm == 1 && mt * (a.NB / splits) / 2 >= 8) ? 16 : 8;
+    cfg.blockDim = dim3((2 + epi_warps) * 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cudaLaunchAttribute at[2];
