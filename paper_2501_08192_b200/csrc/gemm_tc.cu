@@ -278,14 +278,13 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                                 mine[0] += buf[d][0][q];
                                 mine[1] += buf[d][1][q];
                             }
-#pragma unroll
-                            for (int i = 0; i < 2; ++i) {
-                                const float other = __shfl_xor_sync(0xffffffffu, mine[i], 1);
-                                const int b = b0 + i;
-                                if (i == par && b < p.B && !poisoned)
-                                    apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? other : mine[i],
-                                                   par ? mine[i] : other);
-                            }
+                            // rows 2r and 2r + 1 (adjacent lanes) form the output pair: the even lane finishes
+                            // column b0, the odd lane column b0 + 1, each with one value from its neighbour -
+                            // one exchange and one epilogue call for the whole warp
+                            const float recv = __shfl_xor_sync(0xffffffffu, par ? mine[0] : mine[1], 1);
+                            const int b = b0 + par;
+                            if (b < p.B && !poisoned)
+                                apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? recv : mine[0], par ? mine[1] : recv);
                         }
                     }
                 }
@@ -305,12 +304,12 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             float v[16];
             load_chunk(m, c, v);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const float mine = v[i];
-                const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
-                const int b = c * 16 + i;
-                if ((i & 1) == par && b < p.B && !poisoned)
-                    apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? other : mine, par ? mine : other);
+            for (int i = 0; i < 16; i += 2) {
+                // (as above: the even lane of a row pair finishes column i, the odd lane column i + 1)
+                const float recv = __shfl_xor_sync(0xffffffffu, par ? v[i] : v[i + 1], 1);
+                const int b = c * 16 + i + par;
+                if (b < p.B && !poisoned)
+                    apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? recv : v[i], par ? v[i + 1] : recv);
             }
         }
     }
