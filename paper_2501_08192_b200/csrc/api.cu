@@ -475,7 +475,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         a.o_plane = a.q_plane;
         a.ctx_len = sp.ctx_len;
         a.B = B; a.nq = c.n_q_heads; a.nkv = c.n_kv_heads; a.cap = cap;
-        plan_attention(total_tiles, L->sm_count, &a.grid, &a.tiles_per_item);
+        plan_attention(sp.ctx_len_host, B, c.n_kv_heads, L->sm_count, &a.grid, &a.tiles_per_item);
         a.max_items_per_stream = (int)((max_tiles_seq + a.tiles_per_item - 1) / a.tiles_per_item);
         a.max_items = L->max_items;
         a.part_o = L->part_o;

@@ -20,6 +20,8 @@
 // ONE fp32 partial per item (or the final o when the item is the whole sequence).
 // k_attn_merge then combines the partials of a sequence in fixed order.  Nothing
 // depends on timing, so results are bit-stable.
+#include <cstdlib>
+
 #include "../../include/preserve.h"
 #include "common.cuh"
 #include "kernels.h"
@@ -463,20 +465,44 @@ static size_t attn_smem_bytes(int streams)
     return offsetof(AttnSmem, item_base) + sizeof(int) * (size_t)(streams + 1) + 1024;
 }
 
-void plan_attention(uint64_t total_tiles, int sm_count, int *grid, int *tiles_per_item)
+void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_count, int *grid, int *tiles_per_item)
 {
+    uint64_t total_tiles = 0;
+    int longest = 1;
+    for (int b = 0; b < batch; ++b) {
+        const int nt = (ctx_len_host[b] + 1 + kTileKeys - 1) / kTileKeys;
+        total_tiles += (uint64_t)nkv * nt;
+        longest = nt > longest ? nt : longest;
+    }
     // One CTA per SM while the whole cache is at most two ring fills per SM: the ring then holds
     // most of the CTA's share before the queries exist, and half of every SM's shared memory stays
     // free for the kernels before and after.  Longer caches are a steady stream: two CTAs per SM
     // keep twice the bytes in flight.
     const int g = total_tiles <= (uint64_t)2 * kStages * sm_count ? sm_count : 2 * sm_count;
-    // Work items = runs of 64-key tiles: one item per CTA when the cache is small (per-item overhead
-    // dominates), up to four per CTA when it is large (balance under ragged lengths).
-    uint64_t mult = total_tiles / ((uint64_t)g * 3);
-    mult = mult < 1 ? 1 : (mult > 4 ? 4 : mult);
-    const uint64_t tpi = (total_tiles + (uint64_t)g * mult - 1) / ((uint64_t)g * mult);
+    // Work items = runs of `tpi` 64-key tiles of one sequence, dealt to the CTAs round-robin.  The
+    // kernel lasts about rounds x (tpi + the per-item cost of combining and writing a partial,
+    // worth ~1.5 tiles), rounds = items / CTAs rounded up: take the tpi that minimises that, between
+    // a quarter of an even share (at most four items per CTA) and a whole share.
+    const int tpi_hi = (int)((total_tiles + g - 1) / g) + 1;
+    int tpi_lo = (int)((total_tiles + 4ull * g - 1) / (4ull * g));
+    tpi_lo = tpi_lo < 1 ? 1 : tpi_lo;
+    int best = tpi_lo;
+    double best_cost = -1.0;
+    for (int tpi = tpi_lo; tpi <= tpi_hi && tpi <= longest + 1; ++tpi) {
+        uint64_t items = 0;
+        for (int b = 0; b < batch; ++b) {
+            const int nt = (ctx_len_host[b] + 1 + kTileKeys - 1) / kTileKeys;
+            items += (uint64_t)nkv * ((nt + tpi - 1) / tpi);
+        }
+        const uint64_t rounds = (items + g - 1) / g;
+        const double cost = (double)rounds * (tpi + 1.5);
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            best = tpi;
+        }
+    }
     *grid = g;
-    *tiles_per_item = tpi < 1 ? 1 : (int)tpi;
+    *tiles_per_item = best;
 }
 
 cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
@@ -608,7 +634,7 @@ extern "C" int preserve_attention_static(const void *q_hi, const void *q_lo, con
     // ---- carve the array: [status word, 256 B][partial O][partial (max, sum)]
     const int G = n_q_heads / n_kv_heads;
     int grid = 0, tpi = 1;
-    plan_attention(total_tiles, g_scratch_sms[dev], &grid, &tpi);
+    plan_attention(ctx_len_host, batch, n_kv_heads, g_scratch_sms[dev], &grid, &tpi);
     uint64_t n_items = 0, max_items_seq = 0;
     for (int b = 0; b < batch; ++b) {
         const uint64_t nt = (uint64_t)(ctx_len_host[b] + 1 + kTileKeys - 1) / kTileKeys;

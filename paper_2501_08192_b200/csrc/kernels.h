@@ -119,9 +119,9 @@ struct AttnArgs {
     long long *trace;      // optional: two consecutive timeline slots (split-KV, merge)
 };
 cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s);
-// Grid size (persistent CTAs) and tiles per work item for a cache of `total_tiles` 64-key tiles;
+// Grid size (persistent CTAs) and tiles per work item for the given sequence lengths (host array);
 // depends only on the lengths and the SM count.
-void plan_attention(uint64_t total_tiles, int sm_count, int *grid, int *tiles_per_item);
+void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_count, int *grid, int *tiles_per_item);
 
 // 2-D bf16 tensor map (rows x cols, cols contiguous), box (box_cols x box_rows), 128-byte swizzle.
 bool encode_bf16_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_cols,
