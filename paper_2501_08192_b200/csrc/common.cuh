@@ -188,6 +188,24 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t sad
                  : "r"(saddr));
 }
 
+// Address of `smem_ptr`'s counterpart in CTA `rank` of the cluster (shared::cluster window).
+__device__ __forceinline__ uint32_t cluster_map(const void *smem_ptr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(smem_ptr)), "r"(rank));
+    return r;
+}
+// 16-byte store into another CTA's shared memory that also signals 16 bytes on that CTA's mbarrier
+// (both given as shared::cluster addresses): a one-sided hand-over, no cluster barrier needed.
+__device__ __forceinline__ void st_async_v4(uint32_t dst_cluster_addr, float4 v, uint32_t bar_cluster_addr)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(
+                     dst_cluster_addr),
+                 "r"(__float_as_uint(v.x)), "r"(__float_as_uint(v.y)), "r"(__float_as_uint(v.z)), "r"(__float_as_uint(v.w)),
+                 "r"(bar_cluster_addr)
+                 : "memory");
+}
+
 // Optional timeline trace: per kernel, kTraceSlots values in nanoseconds of the global timer,
 // over all CTAs (thread 0 each): {earliest start, earliest wait-return, latest wait-return,
 // latest end, latest start, latest end of the streaming loop, earliest end, unused}.

@@ -54,6 +54,8 @@ struct GemvParams {
     int splits;          // cluster size along k
     int groups;          // row-block groups = row_blocks / (8 / warps_k)
     int slots;           // ring slots per warp actually used (1, 2 or 4): no more than the warp's run needs
+    int push;            // cluster reduction by one-sided hand-over to rank 0 (else every rank reads all ranks)
+    int recv_off;        // push: offset of rank 0's receive area in dynamic shared memory
     int *status;
     long long *trace;
     EpilogueArgs epi;
@@ -71,6 +73,7 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
     __shared__ float red[kGemvWarps][RB * 16][NB];       // per-warp partials
     __shared__ float cta_part[kGemvWarps * RB][16][NB];  // per-row-block CTA partials (read across the cluster)
     __shared__ uint64_t bars[kGemvWarps][kRingSlots];
+    __shared__ uint64_t push_bar;
     __shared__ EpilogueTables tabs;
     extern __shared__ uint8_t gemv_smem_raw[];
     uint8_t *wsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(gemv_smem_raw) + 127) & ~uintptr_t(127));
@@ -137,6 +140,17 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
     }
     __syncwarp();
 
+    const int part_floats = rbs_per_cta * 16 * NB;   // one rank's partial sums of a group
+    if (p.push) {
+        // rank 0 will receive the other ranks' partial sums: its barrier must exist (and expect them)
+        // before anybody sends - a cluster barrier here, where it overlaps the weight fetch
+        if (s == 0 && threadIdx.x == 0) {
+            mbar_init(&push_bar, 1);
+            mbar_fence_init();
+            mbar_expect_tx(&push_bar, (uint32_t)(p.splits - 1) * part_floats * 4u);
+        }
+        cg::this_cluster().sync();
+    }
     load_epilogue_tables(p.epi, tabs, p.b0, p.B);    // inputs of the step: safe before the wait
     const int xrow = p.K >> 3;                       // uint4 per activation row
     auto load_x = [&](int c, uint4 (&xq)[NX]) {
@@ -271,9 +285,36 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
             cta_part[rl][row][b] = v;
         }
 
-        // ---- sum over the cluster ranks (fixed order); every rank finishes its share of the outputs
+        // ---- sum over the cluster ranks (fixed order)
         const int n_out = rbs_per_cta * 8 * NB;          // (row block, pair, batch row) triples of the group
-        if (p.splits > 1) {
+        if (p.splits > 1 && p.push) {
+            // One-sided: ranks 1.. store their partial sums into rank 0's shared memory, signalling its
+            // barrier with the bytes, and are done; rank 0 waits for all the bytes and finishes every
+            // output.  No cluster barrier on the critical path.  (One group per CTA in this mode.)
+            __syncthreads();
+            float *recv = reinterpret_cast<float *>(wsm + p.recv_off);
+            if (s != 0) {
+                const uint32_t dst = cluster_map(recv + (size_t)(s - 1) * part_floats, 0);
+                const uint32_t bar = cluster_map(&push_bar, 0);
+                const float4 *src = reinterpret_cast<const float4 *>(&cta_part[0][0][0]);
+                for (int i = threadIdx.x; i < part_floats / 4; i += blockDim.x)
+                    st_async_v4(dst + i * 16, src[i], bar);
+            } else {
+                ok = mbar_wait(&push_bar, 0, p.status, ST_TIMEOUT_FULL) && ok;
+                for (int i = threadIdx.x; i < n_out; i += blockDim.x) {
+                    const int b = i % NB, r = (i / NB) % 8, rl = i / (8 * NB);
+                    if (b >= p.B)
+                        continue;
+                    float v0 = cta_part[rl][r][b], v1 = cta_part[rl][r + 8][b];
+                    for (int q = 1; q < p.splits; ++q) {
+                        v0 += recv[(size_t)(q - 1) * part_floats + (rl * 16 + r) * NB + b];
+                        v1 += recv[(size_t)(q - 1) * part_floats + (rl * 16 + r + 8) * NB + b];
+                    }
+                    apply_epilogue(p.epi, tabs, b, false, p.N, p.b0 + b, (grp * rbs_per_cta + rl) * 8 + r, v0, v1);
+                }
+            }
+        } else if (p.splits > 1) {
+            // every rank finishes its share of the outputs, reading all ranks' partial sums
             cg::cluster_group cluster = cg::this_cluster();
             cluster.sync();
             const float *remote[8];
@@ -315,7 +356,7 @@ static cudaError_t launch_variant(GemvParams &p, int sm_count, cudaStream_t s)
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(k_gemv_splitk<NB, MMA, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kGemvSmemBytes + 128);
+                                             kGemvSmemBytes + 32 * 1024 + 128);
         if (e != cudaSuccess)
             return e;
         attr_done = true;
@@ -345,10 +386,15 @@ static cudaError_t launch_variant(GemvParams &p, int sm_count, cudaStream_t s)
     const int chunks_per_warp = (p.kchunks + p.splits * p.warps_k - 1) / (p.splits * p.warps_k);
     const int units = groups_per_cta * RB * ((chunks_per_warp + kUnitChunks - 1) / kUnitChunks);
     p.slots = units >= 4 ? 4 : (units >= 2 ? 2 : 1);
+    // one-sided cluster reduction when every CTA has a single group and rank 0's receive area is small
+    const size_t ring_bytes = (size_t)kGemvWarps * p.slots * kUnitChunks * 1024;
+    const size_t recv_bytes = (size_t)(p.splits - 1) * (kGemvWarps / p.warps_k * RB) * 16 * NB * 4;
+    p.push = p.splits > 1 && groups_per_cta == 1 && recv_bytes <= 32 * 1024;
+    p.recv_off = (int)ring_bytes;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(clusters, p.splits, 1);
     cfg.blockDim = dim3(kGemvWarps * 32);
-    cfg.dynamicSmemBytes = (size_t)kGemvWarps * p.slots * kUnitChunks * 1024 + 128;
+    cfg.dynamicSmemBytes = ring_bytes + (p.push ? recv_bytes : 0) + 128;
     cfg.stream = s;
     cudaLaunchAttribute at[2];
     int n = pdl_attr(at);
