@@ -206,6 +206,13 @@ __device__ __forceinline__ void st_async_v4(uint32_t dst_cluster_addr, float4 v,
                  : "memory");
 }
 
+__device__ __forceinline__ void st_async_v2(uint32_t dst_cluster_addr, float2 v, uint32_t bar_cluster_addr)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.b32 [%0], {%1, %2}, [%3];" ::"r"(dst_cluster_addr),
+                 "r"(__float_as_uint(v.x)), "r"(__float_as_uint(v.y)), "r"(bar_cluster_addr)
+                 : "memory");
+}
+
 // Optional timeline trace: per kernel, kTraceSlots values in nanoseconds of the global timer,
 // over all CTAs (thread 0 each): {earliest start, earliest wait-return, latest wait-return,
 // latest end, latest start, latest end of the streaming loop, earliest end, unused}.

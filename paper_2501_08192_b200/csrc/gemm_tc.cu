@@ -44,6 +44,8 @@ struct GemmTcParams {
     int kblocks;        // K / 64
     int splits;         // cluster size along k
     int stages;
+    int push;           // split-K reduction by one-sided hand-over (else every rank reads all ranks)
+    int recv_off;       // push: offset of the receive area behind the ring
     int tmem_cols;
     uint32_t idesc;
     EpilogueArgs epi;
@@ -90,7 +92,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    __shared__ uint64_t full[kTcMaxStages], empty[kTcMaxStages], accum_bar;
+    __shared__ uint64_t full[kTcMaxStages], empty[kTcMaxStages], accum_bar, push_bar;
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile int poisoned;
     __shared__ EpilogueTables tabs;
@@ -123,8 +125,16 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    if (p.push && threadIdx.x == 0) {
+        // this rank will receive NB / splits columns of every other rank's partial tile
+        mbar_init(&push_bar, 1);
+        mbar_fence_init();
+        mbar_expect_tx(&push_bar, (uint32_t)(p.splits - 1) * p.mt * kTcTileM * (p.NB / p.splits) * 4u);
+    }
     tc_fence_before();
     __syncthreads();
+    if (p.push)
+        cg::this_cluster().sync();      // every rank's barrier exists before anybody sends; overlaps the weight fetch
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
 
@@ -220,7 +230,62 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     };
 
     const int par = lane & 1;
-    if (p.splits > 1) {
+    if (p.splits > 1 && p.push) {
+        // Split-K across the cluster, one-sided reduce-scatter: rank q finishes columns [q * cols,
+        // (q + 1) * cols).  Every rank stores those columns of its partial tile into rank q's receive
+        // area [source rank][m][row][cols] (st.async, signalling q's barrier with the bytes; its own
+        // share with plain stores), then waits until its own area is complete and sums the sources in
+        // rank order.  No cluster barrier and no remote loads on the critical path.
+        const int cols = p.NB / p.splits;
+        float *recv = reinterpret_cast<float *>(smem + p.recv_off);
+        const size_t src_stride = (size_t)p.mt * kTcTileM * cols;          // floats per source rank
+        if (warp >= 2) {
+            for (int j = sub; j < p.mt * nchunks; j += kSubs) {
+                const int m = j / nchunks, c = j % nchunks;
+                float v[16];
+                load_chunk(m, c, v);
+                const size_t off = (size_t)s * src_stride + ((size_t)m * kTcTileM + row) * cols;   // my slot, my row
+#pragma unroll
+                for (int i = 0; i < 16; i += 2) {
+                    const int col = c * 16 + i, q = col / cols, cl = col % cols;
+                    if (cols % 4 == 0) {
+                        if (i % 4 == 0) {
+                            const float4 val = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                            if (q == s)
+                                *reinterpret_cast<float4 *>(recv + off + cl) = val;
+                            else
+                                st_async_v4(cluster_map(recv + off + cl, q), val, cluster_map(&push_bar, q));
+                        }
+                    } else {
+                        const float2 val = make_float2(v[i], v[i + 1]);
+                        if (q == s)
+                            *reinterpret_cast<float2 *>(recv + off + cl) = val;
+                        else
+                            st_async_v2(cluster_map(recv + off + cl, q), val, cluster_map(&push_bar, q));
+                    }
+                }
+            }
+            asm volatile("bar.sync 1, %0;" ::"r"(kSubs * 128) : "memory");    // own share stored by all epilogue warps
+            if (!mbar_wait(&push_bar, 0, p.status, ST_TIMEOUT_MMA))
+                poisoned = 1;
+            const int n_pairs = p.mt * cols / 2;
+            for (int it = sub; it < n_pairs; it += kSubs) {
+                const int m = it / (cols / 2), cl = 2 * (it % (cols / 2));
+                const int pair = ((tile * p.mt + m) * kTcTileM + row) >> 1;
+                float mine[2] = {0.f, 0.f};
+                for (int q = 0; q < p.splits; ++q) {       // rank order
+                    const float2 t2 = *reinterpret_cast<const float2 *>(recv + (size_t)q * src_stride +
+                                                                        ((size_t)m * kTcTileM + row) * cols + cl);
+                    mine[0] += t2.x;
+                    mine[1] += t2.y;
+                }
+                const float got = __shfl_xor_sync(0xffffffffu, par ? mine[0] : mine[1], 1);
+                const int b = s * cols + cl + par;
+                if (b < p.B && !poisoned)
+                    apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? got : mine[0], par ? mine[1] : got);
+            }
+        }
+    } else if (p.splits > 1) {
         // Split-K across the cluster, reduce-scatter style: every rank publishes its partial tiles in
         // its own shared memory, then finishes NB / splits of the batch columns - reading that slice
         // from all ranks in rank order - so the reduction and the epilogue work are spread over the
@@ -374,7 +439,23 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     p.tmem_cols = cols;
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * a.NB) >> 3) << 17) | ((uint32_t)(kTcTileM >> 4) << 24);
 
-    size_t smem = (size_t)stages * stage_bytes + 1024;
+    // one-sided split-K reduction when the receive area (one partial tile per CTA) is small - every
+    // thread then hands over one or two 16-byte pieces per owner; wide batches keep the pull form,
+    // whose remote accesses are full 128-byte rows - and fits behind the ring
+    const size_t recv_bytes = (size_t)mt * a.NB * kTcTileM * 4;
+    const size_t smem_cap = (per_sm == 2 ? 108 : 222) * 1024;
+    p.push = 0;
+    if (splits > 1 && recv_bytes <= 16 * 1024) {
+        int st = stages;
+        while (st > 3 && (size_t)st * stage_bytes + recv_bytes + 1024 > smem_cap) --st;
+        if ((size_t)st * stage_bytes + recv_bytes + 1024 <= smem_cap) {
+            stages = st;
+            p.stages = st;
+            p.push = 1;
+        }
+    }
+    p.recv_off = stages * stage_bytes;
+    size_t smem = (size_t)stages * stage_bytes + (p.push ? recv_bytes : 0) + 1024;
     const size_t red_bytes = (size_t)mt * a.NB * kTcTileM * 4 + 1024;
     if (smem < red_bytes) smem = red_bytes;
     static size_t attr_smem = 0;
