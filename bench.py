@@ -38,8 +38,11 @@ SWEEP_FRACS = (0.0, 1 / 16, 1 / 8, 1 / 4, 3 / 8, 1 / 2, 5 / 8, 3 / 4, 7 / 8, 1.0
 # (kernel, workload); see profiles/.  None where no capture exists.
 NCU_TRAFFIC = {
     # profiles/ncu_full_gemv_attn_window_config1_small.md (dram__bytes_read.sum + dram__bytes_write.sum)
-    ("gate_up_proj", 1): 29533952, ("down_proj", 1): 14780160, ("qkv_proj", 1): 6466048, ("o_proj", 1): 4253440,
-    ("attn_splitkv", 1): 16964352, ("attn_merge", 1): 2233856, ("window_a", 1): 618496, ("window_b", 1): 749312,
+    ("gate_up_proj", 1): 29540000, ("down_proj", 1): 14790000, ("qkv_proj", 1): 6480000, ("o_proj", 1): 4260000,
+    ("attn_splitkv", 1): 16900000, ("attn_merge", 1): 300000, ("window_a", 1): 630000, ("window_b", 1): 760000,
+    # profiles/ncu_full_gemm_tcgen05_config3_small.md, profiles/ncu_full_attn_splitkv_config5.md
+    ("gate_up_proj", 2): 121630000, ("down_proj", 2): 59200000, ("qkv_proj", 2): 21570000, ("o_proj", 2): 16910000,
+    ("attn_splitkv", 4): 545000000,
 }
 
 
