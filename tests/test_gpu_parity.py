@@ -64,6 +64,12 @@ SMALL = [
     I.small_shape(name="ctx0", batch=2, ctx=0, seed=46),
     I.small_shape(name="ctx63", batch=2, ctx=63, seed=47),     # 64 keys: exactly one tile
     I.small_shape(name="long_multi_tile_items", batch=2, n_q_heads=4, n_kv_heads=2, ctx=20000, seed=18),
+    # gate/up with more row-block groups than CTAs (a CTA loops over several groups)
+    I.small_shape(name="wide_ffn_b8", batch=8, hidden=256, ffn=5120, ctx=70, seed=48),
+    # 24 / 28 row blocks: one row block per warp, k split over a cluster with the one-sided reduction
+    I.small_shape(name="h384_b7", batch=7, hidden=384, ffn=224, ctx=33, seed=49),
+    # window rows split over a cluster of CTAs
+    I.small_shape(name="h2048_b3", batch=3, hidden=2048, ffn=256, ctx=40, tp_degree=5, seed=50),
 ]
 
 
