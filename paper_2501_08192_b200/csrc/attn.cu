@@ -120,6 +120,8 @@ __device__ __forceinline__ int find_stream(const int *item_base, int streams, in
     return lo;
 }
 
+// NARROW: groups of up to 8 query heads (keys as MMA rows in the QK product), else up to 16.
+template <bool NARROW>
 __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const __grid_constant__ AttnParams p)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -195,6 +197,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
         const int t0 = chunk * p.tiles_per_item;
         const int t1 = min(nt, t0 + p.tiles_per_item);
 
+        constexpr bool narrow = NARROW;
         // Q fragments: rows = query heads of the group (zero beyond G)
         // (both bf16 planes of q: the scores are (q_hi + q_lo) . k)
         uint32_t qa[2][8][4];
@@ -205,9 +208,9 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
             for (int ks = 0; ks < 8; ++ks) {
                 const int d0 = ks * 16 + 2 * t;
                 qa[pl][ks][0] = g < p.G ? *reinterpret_cast<const uint32_t *>(qb + g * kHeadDim + d0) : 0u;
-                qa[pl][ks][1] = g + 8 < p.G ? *reinterpret_cast<const uint32_t *>(qb + (g + 8) * kHeadDim + d0) : 0u;
+                qa[pl][ks][1] = (!narrow && g + 8 < p.G) ? *reinterpret_cast<const uint32_t *>(qb + (g + 8) * kHeadDim + d0) : 0u;
                 qa[pl][ks][2] = g < p.G ? *reinterpret_cast<const uint32_t *>(qb + g * kHeadDim + d0 + 8) : 0u;
-                qa[pl][ks][3] = g + 8 < p.G ? *reinterpret_cast<const uint32_t *>(qb + (g + 8) * kHeadDim + d0 + 8) : 0u;
+                qa[pl][ks][3] = (!narrow && g + 8 < p.G) ? *reinterpret_cast<const uint32_t *>(qb + (g + 8) * kHeadDim + d0 + 8) : 0u;
             }
         }
         float o[16][4];
@@ -240,6 +243,61 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
                 __syncwarp();
             }
 
+            float corr[2];
+            uint32_t pa[4];
+            if constexpr (narrow) {
+                // ---- up to 8 query heads: S^T = K Q^T, keys as the 16 MMA rows, heads as the 8 columns -
+                // half the MMAs of the other orientation.  Lane (g, t) holds keys g and g + 8 for the
+                // heads 2t and 2t + 1.
+                float sT[4] = {0.f, 0.f, 0.f, 0.f};
+                {
+                    const int key = warp * 16 + ((lane >> 4) << 3) + (lane & 7);
+                    const uint32_t rowaddr = kbase + key * 128;
+                    const int csel = (lane >> 3) & 1;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const int chunk16 = ((ks & 3) << 1) + csel;
+                        const uint32_t addr = rowaddr + (ks >> 2) * kHalfBytes + ((chunk16 ^ (key & 7)) << 4);
+                        uint32_t r[4];
+                        ldmatrix_x4(r, addr);        // [keys 0-7 | 8-15] x [d 0-7 | 8-15] of this 16 x 16 block
+#pragma unroll
+                        for (int pl = 0; pl < 2; ++pl)
+                            mma_bf16_16816(sT, r[0], r[2], r[1], r[3], qa[pl][ks][0], qa[pl][ks][2]);
+                    }
+                }
+                // scale, mask, online softmax per head (a column: its 16 keys sit in the lanes of equal t)
+                float v[4], mx[2];
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    v[j] = (g + 8 * (j >> 1)) < valid ? sT[j] * p.scale_log2 : -INFINITY;
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    mx[j] = fmaxf(v[j], v[2 + j]);
+                    mx[j] = fmaxf(mx[j], __shfl_xor_sync(0xffffffffu, mx[j], 4));
+                    mx[j] = fmaxf(mx[j], __shfl_xor_sync(0xffffffffu, mx[j], 8));
+                    mx[j] = fmaxf(mx[j], __shfl_xor_sync(0xffffffffu, mx[j], 16));
+                    const float m_new = fmaxf(m_run[j], mx[j]);
+                    corr[j] = m_new == -INFINITY ? 1.f : exp2f(m_run[j] - m_new);
+                    m_run[j] = m_new;                       // (narrow: m_run / l_run belong to heads 2t, 2t + 1;
+                    l_run[j] *= corr[j];                    //  l_run is this lane's share, summed at the end)
+                }
+                float ph[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float m = m_run[j & 1];
+                    ph[j] = m == -INFINITY ? 0.f : exp2f(v[j] - m);
+                    l_run[j & 1] += ph[j];
+                }
+                // P^T (keys x heads) -> the A fragment of P (heads x keys): two 8 x 8 transposes
+                const uint32_t x0 = pack_bf16(ph[0], ph[1]), x1 = pack_bf16(ph[2], ph[3]);
+                asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pa[0]) : "r"(x0));
+                asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pa[2]) : "r"(x1));
+                pa[1] = pa[3] = 0u;
+                // the accumulator rows are heads g: fetch head g's correction from the lane that holds it
+                const float ce = __shfl_sync(0xffffffffu, corr[0], g >> 1), co = __shfl_sync(0xffffffffu, corr[1], g >> 1);
+                corr[0] = (g & 1) ? co : ce;
+                corr[1] = 1.f;
+            } else {
             // S = Q K^T for this warp's 16 keys
             float s[2][4];
 #pragma unroll
@@ -273,7 +331,6 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
                     s[i][j] = v;
                     mx[j >> 1] = fmaxf(mx[j >> 1], v);
                 }
-            float corr[2];
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
                 mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
@@ -286,7 +343,6 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
             // P as one bf16 plane: the weights lie in [0, 1] and enter a sum of products with V, so
             // their 2^-9 relative rounding stays within a quarter of the tolerance on o (measured on
             // all five configs); q, whose rounding is amplified by the softmax, keeps both planes
-            uint32_t pa[4];
             {
                 float pv[2][4];
 #pragma unroll
@@ -301,6 +357,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
                 pa[1] = pack_bf16(pv[0][2], pv[0][3]);
                 pa[2] = pack_bf16(pv[1][0], pv[1][1]);
                 pa[3] = pack_bf16(pv[1][2], pv[1][3]);
+            }
             }
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
@@ -330,20 +387,37 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
 
         // ---- combine the four warps' partials through the stage consumed last
         uint8_t *stage_last = sm.stage[(it + kStages - 1) % kStages];
+        if constexpr (narrow) {
+            // (max, sum) of heads 2t and 2t + 1: add the lanes' shares of the sum, lanes g == 0 write
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                l_run[j] += __shfl_xor_sync(0xffffffffu, l_run[j], 4);
+                l_run[j] += __shfl_xor_sync(0xffffffffu, l_run[j], 8);
+                l_run[j] += __shfl_xor_sync(0xffffffffu, l_run[j], 16);
+                if (g == 0 && 2 * t + j < p.G) {
+                    sm.comb_ml[warp][2 * t + j][0] = m_run[j];
+                    sm.comb_ml[warp][2 * t + j][1] = l_run[j];
+                }
+            }
+        } else {
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
+                l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+                if (t == 0 && g + 8 * r < p.G) {
+                    sm.comb_ml[warp][g + 8 * r][0] = m_run[r];
+                    sm.comb_ml[warp][g + 8 * r][1] = l_run[r];
+                }
+            }
+        }
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
-            l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
-            l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
             const int row = g + 8 * r;
             if (row < p.G) {
                 float2 *dst = reinterpret_cast<float2 *>(comb_row(stage_last, warp, row));
 #pragma unroll
                 for (int i = 0; i < 16; ++i)
                     dst[comb_col2(row, i * 4 + t)] = make_float2(o[i][2 * r], o[i][2 * r + 1]);
-                if (t == 0) {
-                    sm.comb_ml[warp][row][0] = m_run[r];
-                    sm.comb_ml[warp][row][1] = l_run[r];
-                }
             }
         }
         consumer_barrier();
@@ -530,8 +604,11 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     const size_t smem = attn_smem_bytes(a.B * a.nkv);
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_attn_decode_splitkv, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(k_attn_decode_splitkv<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)attn_smem_bytes(kMaxStreams));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(k_attn_decode_splitkv<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)attn_smem_bytes(kMaxStreams));
         if (e != cudaSuccess)
             return e;
         attr_set = true;
@@ -547,7 +624,8 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     const int phases = a.phases ? a.phases : 3;
     cudaError_t e = cudaSuccess;
     if (phases & 1)
-        e = cudaLaunchKernelEx(&cfg, k_attn_decode_splitkv, p);
+        e = p.G <= 8 ? cudaLaunchKernelEx(&cfg, k_attn_decode_splitkv<true>, p)
+                     : cudaLaunchKernelEx(&cfg, k_attn_decode_splitkv<false>, p);
     if (e != cudaSuccess)
         return e;
     if (a.mid_event) {
