@@ -213,9 +213,12 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
                 qa[pl][ks][3] = (!narrow && g + 8 < p.G) ? *reinterpret_cast<const uint32_t *>(qb + (g + 8) * kHeadDim + d0 + 8) : 0u;
             }
         }
-        float o[16][4];
+        // accumulators: O (heads x d) as 16 n-tiles of 8 head dims, or, for narrow groups, O^T (d x heads)
+        // as 8 m-tiles of 16 head dims (lane (g, t): dims 16 i + g and 16 i + g + 8, heads 2t and 2t + 1)
+        constexpr int kOT = narrow ? 8 : 16;
+        float o[kOT][4];
 #pragma unroll
-        for (int i = 0; i < 16; ++i)
+        for (int i = 0; i < kOT; ++i)
             o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
         float m_run[2] = {-INFINITY, -INFINITY};
         float l_run[2] = {0.f, 0.f};
@@ -288,15 +291,11 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
                     ph[j] = m == -INFINITY ? 0.f : exp2f(v[j] - m);
                     l_run[j & 1] += ph[j];
                 }
-                // P^T (keys x heads) -> the A fragment of P (heads x keys): two 8 x 8 transposes
+                // P^T (keys x heads) -> (heads x keys), the B fragment of P^T in O^T = V^T P^T: two 8 x 8 transposes
                 const uint32_t x0 = pack_bf16(ph[0], ph[1]), x1 = pack_bf16(ph[2], ph[3]);
                 asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pa[0]) : "r"(x0));
                 asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pa[2]) : "r"(x1));
                 pa[1] = pa[3] = 0u;
-                // the accumulator rows are heads g: fetch head g's correction from the lane that holds it
-                const float ce = __shfl_sync(0xffffffffu, corr[0], g >> 1), co = __shfl_sync(0xffffffffu, corr[1], g >> 1);
-                corr[0] = (g & 1) ? co : ce;
-                corr[1] = 1.f;
             } else {
             // S = Q K^T for this warp's 16 keys
             float s[2][4];
@@ -360,11 +359,16 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
             }
             }
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                o[i][0] *= corr[0]; o[i][1] *= corr[0];
-                o[i][2] *= corr[1]; o[i][3] *= corr[1];
+            for (int i = 0; i < kOT; ++i) {
+                if constexpr (narrow) {          // columns = heads 2t, 2t + 1
+                    o[i][0] *= corr[0]; o[i][1] *= corr[1];
+                    o[i][2] *= corr[0]; o[i][3] *= corr[1];
+                } else {                         // rows = heads g, g + 8
+                    o[i][0] *= corr[0]; o[i][1] *= corr[0];
+                    o[i][2] *= corr[1]; o[i][3] *= corr[1];
+                }
             }
-            // O += P V
+            // O += P V  (narrow: O^T += V^T P^T, the 16 head dims of a tile as MMA rows)
             {
                 const int key = warp * 16 + (((lane >> 3) & 1) << 3) + (lane & 7);
                 const uint32_t rowaddr = vbase + key * 128;
@@ -373,10 +377,14 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
                 for (int c = 0; c < 16; c += 2) {
                     const int cc = (c & 7) + csel;
                     const uint32_t addr = rowaddr + (c >> 3) * kHalfBytes + ((cc ^ (key & 7)) << 4);
-                    uint32_t r[4];
+                    uint32_t r[4];     // transposed 8 x 8 blocks [keys 0-7 | 8-15] x [dims 0-7 | 8-15] of 16 head dims
                     ldmatrix_x4_trans(r, addr);
-                    mma_bf16_16816(o[c], pa[0], pa[1], pa[2], pa[3], r[0], r[1]);
-                    mma_bf16_16816(o[c + 1], pa[0], pa[1], pa[2], pa[3], r[2], r[3]);
+                    if constexpr (narrow) {
+                        mma_bf16_16816(o[c >> 1], r[0], r[2], r[1], r[3], pa[0], pa[2]);
+                    } else {
+                        mma_bf16_16816(o[c], pa[0], pa[1], pa[2], pa[3], r[0], r[1]);
+                        mma_bf16_16816(o[c + 1], pa[0], pa[1], pa[2], pa[3], r[2], r[3]);
+                    }
                 }
             }
             __syncwarp();
@@ -410,14 +418,30 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
                 }
             }
         }
+        if constexpr (narrow) {
 #pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            const int row = g + 8 * r;
-            if (row < p.G) {
-                float2 *dst = reinterpret_cast<float2 *>(comb_row(stage_last, warp, row));
+            for (int j = 0; j < 2; ++j) {
+                const int row = 2 * t + j;              // head
+                if (row < p.G) {
+                    float *dst = comb_row(stage_last, warp, row);
 #pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    dst[comb_col2(row, i * 4 + t)] = make_float2(o[i][2 * r], o[i][2 * r + 1]);
+                    for (int i = 0; i < 8; ++i) {
+                        const int d0 = 16 * i + g, d1 = d0 + 8;
+                        dst[2 * comb_col2(row, d0 >> 1) + (d0 & 1)] = o[i][j];
+                        dst[2 * comb_col2(row, d1 >> 1) + (d1 & 1)] = o[i][2 + j];
+                    }
+                }
+            }
+        } else {
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const int row = g + 8 * r;
+                if (row < p.G) {
+                    float2 *dst = reinterpret_cast<float2 *>(comb_row(stage_last, warp, row));
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        dst[comb_col2(row, i * 4 + t)] = make_float2(o[i][2 * r], o[i][2 * r + 1]);
+                }
             }
         }
         consumer_barrier();
