@@ -85,7 +85,7 @@ struct preserve_layer {
     float *h_f32;                              // window A sum (residual for window B)
     float *attn_f32, *h2_f32, *mlp_f32;        // unrounded copies: own attention partial (window B input),
                                                // and the two outputs (handed to the next layer of a linked chain)
-    void *x, *q, *o, *attn_partial, *x2, *a;   // x, q, o, x2, a: split bf16 [2][rows][...] (hi + lo)
+    void *x, *q, *o, *x2, *a;                  // split bf16 [2][rows][...] (hi + lo)
     int rows;                                  // batch rows per plane (max_batch, padded to 16 on the tensor path)
     float *part_o, *part_ml;
     int max_items;
@@ -336,11 +336,10 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
     const Dims d = layer_dims(c);
 
     // ---- plan (host): Algorithm 1 per window over {Wqkv, KV, Wo} and {Wgate|up, Wdown}
-    uint64_t sum_ctx = 0, total_tiles = 0, max_tiles_seq = 0;
+    uint64_t sum_ctx = 0, max_tiles_seq = 0;
     for (int b = 0; b < B; ++b) {
         sum_ctx += (uint64_t)sp.ctx_len_host[b];
         const uint64_t nt = (uint64_t)(sp.ctx_len_host[b] + 1 + 63) / 64;
-        total_tiles += (uint64_t)c.n_kv_heads * nt;
         max_tiles_seq = nt > max_tiles_seq ? nt : max_tiles_seq;
     }
     L->kv_bytes = 2 * sum_ctx * c.n_kv_heads * c.head_dim * 2;
@@ -729,7 +728,7 @@ void preserve_layer_destroy(preserve_layer_t *L)
     if (L->side)
         cudaStreamSynchronize(L->side);
     drop_graphs(L);
-    void *ptrs[] = {L->trace_buf, L->attn_f32, L->h2_f32, L->mlp_f32, L->arena, L->inv_freq, L->h_f32, L->x, L->q, L->o, L->attn_partial, L->x2, L->a,
+    void *ptrs[] = {L->trace_buf, L->attn_f32, L->h2_f32, L->mlp_f32, L->arena, L->inv_freq, L->h_f32, L->x, L->q, L->o, L->x2, L->a,
                     L->part_o, L->part_ml, L->status, L->stage_in, L->stage_out, L->ctx_dev};
     for (void *p : ptrs)
         if (p)
@@ -868,7 +867,6 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     CKI(cudaMalloc(&L->x, 2 * RH * 2));
     CKI(cudaMalloc(&L->q, 2 * Rq * 2));
     CKI(cudaMalloc(&L->o, 2 * Rq * 2));
-    CKI(cudaMalloc(&L->attn_partial, BH * 2));
     CKI(cudaMalloc(&L->x2, 2 * RH * 2));
     CKI(cudaMalloc(&L->a, 2 * RF * 2));
     CKI(cudaMemset(L->x, 0, 2 * RH * 2));

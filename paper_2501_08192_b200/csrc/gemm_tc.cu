@@ -387,14 +387,6 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     trace_end(p.trace);
 }
 
-static int pow2_floor_i(int v)
-{
-    int r = 1;
-    while (r * 2 <= v)
-        r *= 2;
-    return r;
-}
-
 cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
 {
     if (a.NB < 16 || a.NB > 128 || a.NB % 16 || a.N % kTcTileM || a.K % kTcBlockK || a.B > a.NB)
