@@ -284,8 +284,9 @@ PRESERVE_API int preserve_debug_copy(preserve_layer_t *layer, int32_t which, voi
  * [batch, n_kv_heads, kv_capacity, 128].  ctx_len is a device array, ctx_len_host the same
  * values on the host; each 0..kv_capacity-1.  At most 16 query heads per KV head.
  *
- * Limits and errors: the partials of (2 x SM count + batch x n_kv_heads) work items must
- * fit in the scratch array, else PRESERVE_ETOOBIG is returned and nothing is queued; other
+ * Limits and errors: the partials of the call's work items (runs of 64-key tiles of one
+ * sequence and KV head; at most 8 x SM count + batch x n_kv_heads of them, 520 bytes per query
+ * head of the group each) must fit in the scratch array, else PRESERVE_ETOOBIG is returned and nothing is queued; other
  * bad arguments return PRESERVE_EINVAL / _EALIGN / _ESHAPE.
  *
  * Sharing: all calls on one GPU use the same array, and it keeps whatever the previous

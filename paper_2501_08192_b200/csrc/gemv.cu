@@ -5,17 +5,20 @@
 // pure weight stream.  The packed weights are 1 KiB fragment-major tiles (16
 // output rows x 32 k, see pack.cu), contiguous along k within a 16-row block.
 //
-// Persistent CTAs of 8 warps.  A CTA (or a cluster of up to 8 CTAs) owns one
-// group of 16-row blocks at a time; the k range is split over the warps of the
-// CTA and the CTAs of the cluster, so every warp streams ONE contiguous run of
-// tiles.  Each warp is its own producer and consumer: lane 0 keeps a private ring
-// of four 2 KiB slots filled with bulk async copies (cp.async.bulk -> shared
-// memory, completion on per-slot mbarriers, all waits bounded) and refills a slot
-// as soon as the warp has consumed it.  The first four copies are issued before
-// the programmatic-dependent-launch wait, so weights are already streaming while
-// the previous kernel finishes; only the small activation fragments are loaded
-// after the wait.  Grids never exceed what is co-resident, so there is no second
-// wave.
+// CTAs of 8 warps.  A CTA (or a cluster of up to 8 CTAs) owns one group of
+// 16-row blocks at a time (further groups are loop iterations); the k range is
+// split over the warps of the CTA and the CTAs of the cluster, so every warp
+// streams ONE contiguous run of tiles per row block - for one or (RB = 2) two row
+// blocks, which then share every activation fragment the warp loads.  Each warp is
+// its own producer and consumer: lane 0 keeps a private ring of up to four 2 KiB
+// slots filled with bulk async copies (cp.async.bulk -> shared memory, completion
+// on per-slot mbarriers, all waits bounded) and refills a slot as soon as the warp
+// has consumed it.  The ring is filled before the programmatic-dependent-launch
+// wait, so weights are already streaming while the previous kernel finishes; only
+// the small activation fragments are loaded after the wait (in bursts, so that
+// their L2 latency is paid once per burst).  Grids never exceed what is
+// co-resident: one CTA per SM when a ring per SM holds the whole matrix, two for
+// larger matrices.
 // Two arithmetic variants:
 //   - CUDA cores (batch <= 4): 2 x batch fp32 accumulators per lane, finished by
 //     a warp-shuffle reduction over the four lanes that share a row;
@@ -23,10 +26,12 @@
 //     need ~8 FMAs per weight and co-limit the stream, so the 16x32 tile feeds
 //     warp MMAs with the batch as the n = 8 operand.
 // Activations arrive as hi + lo bf16 planes (x = hi + lo).
-// Split-K partial sums are added in a fixed order (warps through shared memory,
-// cluster ranks through distributed shared memory, each rank finishing its share
-// of the outputs), so results are bit-stable.  The fused epilogues live in
-// epilogue.cuh.
+// Split-K partial sums are added in a fixed order, so results are bit-stable: warps
+// through shared memory; cluster ranks one-sidedly - ranks 1.. store their sums
+// into rank 0's shared memory (st.async + mbarrier complete_tx) and rank 0
+// finishes the outputs - or, when a CTA handles several groups, through
+// distributed shared memory with every rank finishing its share of the outputs.
+// The fused epilogues live in epilogue.cuh.
 #include <cooperative_groups.h>
 
 #include "epilogue.cuh"
