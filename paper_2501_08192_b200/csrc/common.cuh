@@ -206,6 +206,48 @@ __device__ __forceinline__ void st_async_v4(uint32_t dst_cluster_addr, float4 v,
                  : "memory");
 }
 
+// Shared-memory loads by 32-bit shared address (a generic pointer costs address conversion and
+// the slower generic path).
+__device__ __forceinline__ float lds_f32(uint32_t addr)
+{
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float2 lds_f32x2(uint32_t addr)
+{
+    float2 v;
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+    return v;
+}
+// Cluster barrier split in two; the arrive carries no data (it only keeps shared memory alive), so
+// it needs no release.
+__device__ __forceinline__ void cluster_arrive_relaxed()
+{
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait()
+{
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// Bulk copy from this CTA's shared memory into another CTA's of the cluster; the bytes are signalled
+// on the destination CTA's mbarrier.  Addresses 16-byte aligned, size a multiple of 16.  The source
+// must stay valid until the destination's barrier has completed.
+__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster_addr, uint32_t src_cta_addr, uint32_t bytes,
+                                                     uint32_t bar_cluster_addr)
+{
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     dst_cluster_addr),
+                 "r"(src_cta_addr), "r"(bytes), "r"(bar_cluster_addr)
+                 : "memory");
+}
+// Orders this thread's earlier generic-proxy writes to shared memory before later async-proxy reads.
+__device__ __forceinline__ void fence_proxy_async_smem()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
 __device__ __forceinline__ void st_async_v2(uint32_t dst_cluster_addr, float2 v, uint32_t bar_cluster_addr)
 {
     asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.b32 [%0], {%1, %2}, [%3];" ::"r"(dst_cluster_addr),

@@ -103,7 +103,9 @@ __device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, const Epil
             e.out_f32[(size_t)b * N + n1] = v1;
         }
     } else if (e.kind == EPI_SWIGLU) {
-        const float a = v0 / (1.f + expf(-v0)) * v1;
+        // silu by the fast exponential and division (a few ulp; for v0 < -87 the quotient flushes to 0,
+        // its true size being < 1e-36)
+        const float a = __fdividef(v0, 1.f + __expf(-v0)) * v1;
         store_split(e.out, e.out_plane, (size_t)b * (N >> 1) + n0, a);
     } else {
         const int hd = n0, i = n1;

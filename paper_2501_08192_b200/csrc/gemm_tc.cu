@@ -44,7 +44,7 @@ struct GemmTcParams {
     int kblocks;        // K / 64
     int splits;         // cluster size along k
     int stages;
-    int push;           // split-K reduction by one-sided hand-over (else every rank reads all ranks)
+    int push;           // split-K reduction by one-sided hand-over: 1 = st.async, 2 = bulk copies (0: every rank reads all ranks)
     int recv_off;       // push: offset of the receive area behind the ring
     int tmem_cols;
     uint32_t idesc;
@@ -230,7 +230,84 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     };
 
     const int par = lane & 1;
-    if (p.splits > 1 && p.push) {
+    if (p.splits > 1 && p.push == 2) {
+        // Split-K across the cluster for wide batches, one-sided reduce-scatter by bulk copies: every
+        // rank lays its partial tiles out in its own (idle) ring as [m][column][row], then one bulk
+        // copy per (owner, m) moves the owner's columns - a contiguous slice - into the owner's receive
+        // area [source slot][m][column][row], signalling the owner's barrier with the bytes.  The owner
+        // waits for its area, sums the sources in rank order (its own share straight from its ring)
+        // and applies the epilogue.  The cluster barrier that keeps the senders' shared memory alive
+        // until the copies have landed is split: arrive once this rank's area is complete, wait at
+        // the very end, so its latency hides behind the epilogue.
+        cg::cluster_group cluster = cg::this_cluster();
+        const int cols = p.NB / p.splits;
+        float *recv = reinterpret_cast<float *>(smem + p.recv_off);
+        if (warp >= 2) {
+            for (int j = sub; j < p.mt * nchunks; j += kSubs) {
+                const int m = j / nchunks, c = j % nchunks;
+                float v[16];
+                load_chunk(m, c, v);
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    red[((size_t)m * p.NB + c * 16 + i) * kTcTileM + row] = v[i];
+            }
+            fence_proxy_async_smem();
+            asm volatile("bar.sync 1, %0;" ::"r"(kSubs * 128) : "memory");
+            const int e = (int)threadIdx.x - 64;
+            if (e < (p.splits - 1) * p.mt) {
+                const int slot_q = e / p.mt, m = e % p.mt;
+                const int q = slot_q < s ? slot_q : slot_q + 1;      // owner
+                const int my_slot = s < q ? s : s - 1;               // where the owner keeps this rank's share
+                bulk_copy_to_cluster(cluster_map(recv + ((size_t)(my_slot * p.mt + m) * cols) * kTcTileM, q),
+                                     smem_u32(red + ((size_t)m * p.NB + q * cols) * kTcTileM),
+                                     (uint32_t)cols * kTcTileM * 4u, cluster_map(&push_bar, q));
+            }
+            if (!mbar_wait(&push_bar, 0, p.status, ST_TIMEOUT_MMA))
+                poisoned = 1;
+        }
+        cluster_arrive_relaxed();
+        if (warp >= 2) {
+            const uint32_t red_a = smem_u32(red) + (uint32_t)(s * cols * kTcTileM + row) * 4u;
+            const uint32_t recv_a = smem_u32(recv) + (uint32_t)row * 4u;
+            const bool bad = poisoned;
+            auto finish = [&](auto sp_tag) {
+                constexpr int SP = decltype(sp_tag)::value;
+                // per source rank: address of (m = 0, column 0, this row) and the stride between m
+                uint32_t base[SP], mstr[SP];
+#pragma unroll
+                for (int q = 0; q < SP; ++q) {
+                    base[q] = q == s ? red_a : recv_a + (uint32_t)((q < s ? q : q - 1) * p.mt * cols) * (kTcTileM * 4u);
+                    mstr[q] = (uint32_t)(q == s ? p.NB : cols) * (kTcTileM * 4u);
+                }
+                const int hp = cols / 2;                   // column pairs per m
+                int m = 0, c2 = sub;
+                while (c2 >= hp) { c2 -= hp; ++m; }
+                while (m < p.mt) {
+                    float mine[2] = {0.f, 0.f};
+#pragma unroll
+                    for (int q = 0; q < SP; ++q) {         // rank order
+                        const uint32_t a = base[q] + m * mstr[q] + (uint32_t)c2 * (2u * kTcTileM * 4u);
+                        mine[0] += lds_f32(a);
+                        mine[1] += lds_f32(a + kTcTileM * 4u);
+                    }
+                    const float got = __shfl_xor_sync(0xffffffffu, par ? mine[0] : mine[1], 1);
+                    const int b = s * cols + 2 * c2 + par;
+                    const int pair = ((tile * p.mt + m) * kTcTileM + row) >> 1;
+                    if (b < p.B && !bad)
+                        apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? got : mine[0], par ? mine[1] : got);
+                    c2 += kSubs;
+                    while (c2 >= hp) { c2 -= hp; ++m; }
+                }
+            };
+            if (p.splits == 2)
+                finish(std::integral_constant<int, 2>());
+            else if (p.splits == 4)
+                finish(std::integral_constant<int, 4>());
+            else
+                finish(std::integral_constant<int, 8>());
+        }
+        cluster_wait();
+    } else if (p.splits > 1 && p.push) {
         // Split-K across the cluster, one-sided reduce-scatter: rank q finishes columns [q * cols,
         // (q + 1) * cols).  Every rank stores those columns of its partial tile into rank q's receive
         // area [source rank][m][row][cols] (st.async, signalling q's barrier with the bytes; its own
@@ -435,7 +512,7 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     // thread then hands over one or two 16-byte pieces per owner; wide batches keep the pull form,
     // whose remote accesses are full 128-byte rows - and fits behind the ring
     const size_t recv_bytes = (size_t)mt * a.NB * kTcTileM * 4;
-    const size_t smem_cap = (per_sm == 2 ? 108 : 222) * 1024;
+    const size_t smem_cap = (per_sm == 2 ? 108 : 225) * 1024;
     p.push = 0;
     if (splits > 1 && recv_bytes <= 16 * 1024) {
         int st = stages;
@@ -446,8 +523,21 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
             p.push = 1;
         }
     }
+    // wide batches: the same by bulk copies (receive area: the other ranks' shares of this rank's columns)
+    size_t recv_alloc = p.push ? recv_bytes : 0;
+    if (splits > 1 && !p.push) {
+        const size_t need = recv_bytes / splits * (splits - 1);
+        int st = stages;
+        while (st > 3 && (size_t)st * stage_bytes + need + 1024 > smem_cap) --st;
+        if ((size_t)st * stage_bytes + need + 1024 <= smem_cap) {
+            stages = st;
+            p.stages = st;
+            p.push = 2;
+            recv_alloc = need;
+        }
+    }
     p.recv_off = stages * stage_bytes;
-    size_t smem = (size_t)stages * stage_bytes + (p.push ? recv_bytes : 0) + 1024;
+    size_t smem = (size_t)stages * stage_bytes + recv_alloc + 1024;
     const size_t red_bytes = (size_t)mt * a.NB * kTcTileM * 4 + 1024;
     if (smem < red_bytes) smem = red_bytes;
     static size_t attr_smem = 0;
