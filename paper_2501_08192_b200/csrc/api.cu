@@ -443,6 +443,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         w.B = B; w.H = H;
         w.trace = TRACE(0);
         w.delay_ns = L->window_delay_ns;
+        w.status = L->status;
         CK(L, launch_window(w, s));
     }
     // ---- QKV projection + rotary embedding + KV append
@@ -533,6 +534,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         w.B = B; w.H = H;
         w.trace = TRACE(5);
         w.delay_ns = L->window_delay_ns;
+        w.status = L->status;
         CK(L, launch_window(w, s));
     }
     // ---- gate/up projection + SwiGLU, down projection

@@ -195,6 +195,12 @@ __device__ __forceinline__ uint32_t cluster_map(const void *smem_ptr, uint32_t r
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(smem_ptr)), "r"(rank));
     return r;
 }
+__device__ __forceinline__ uint32_t cluster_map_addr(uint32_t smem_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
 // 16-byte store into another CTA's shared memory that also signals 16 bytes on that CTA's mbarrier
 // (both given as shared::cluster addresses): a one-sided hand-over, no cluster barrier needed.
 __device__ __forceinline__ void st_async_v4(uint32_t dst_cluster_addr, float4 v, uint32_t bar_cluster_addr)
@@ -211,14 +217,26 @@ __device__ __forceinline__ void st_async_v4(uint32_t dst_cluster_addr, float4 v,
 __device__ __forceinline__ float lds_f32(uint32_t addr)
 {
     float v;
-    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
     return v;
 }
 __device__ __forceinline__ float2 lds_f32x2(uint32_t addr)
 {
     float2 v;
-    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
     return v;
+}
+__device__ __forceinline__ void sts_f32(uint32_t addr, float v)
+{
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void sts_f32x4(uint32_t addr, float4 v)
+{
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void sts_f32x2(uint32_t addr, float2 v)
+{
+    asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(v.x), "f"(v.y) : "memory");
 }
 // Cluster barrier split in two; the arrive carries no data (it only keeps shared memory alive), so
 // it needs no release.
@@ -248,6 +266,12 @@ __device__ __forceinline__ void fence_proxy_async_smem()
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+__device__ __forceinline__ void st_async_f32(uint32_t dst_cluster_addr, float v, uint32_t bar_cluster_addr)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(dst_cluster_addr),
+                 "r"(__float_as_uint(v)), "r"(bar_cluster_addr)
+                 : "memory");
+}
 __device__ __forceinline__ void st_async_v2(uint32_t dst_cluster_addr, float2 v, uint32_t bar_cluster_addr)
 {
     asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.b32 [%0], {%1, %2}, [%3];" ::"r"(dst_cluster_addr),

@@ -74,18 +74,25 @@ __device__ __forceinline__ void tc_commit(uint64_t *bar)
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16])
+// TMEM -> registers, 16 consecutive columns of this thread's lane.  The load is asynchronous: the
+// registers are valid after tc_ld_wait, which names them so that no use can move above it.
+__device__ __forceinline__ void tc_ld16_issue(uint32_t taddr, uint32_t (&r)[16])
 {
-    uint32_t r[16];
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
                    "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
                    "=r"(r[15])
                  : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 16; ++i)
-        v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tc_ld_wait(uint32_t (&a)[16], uint32_t (&b)[16])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]),
+                   "+r"(a[8]), "+r"(a[9]), "+r"(a[10]), "+r"(a[11]), "+r"(a[12]), "+r"(a[13]), "+r"(a[14]), "+r"(a[15]),
+                   "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7]),
+                   "+r"(b[8]), "+r"(b[9]), "+r"(b[10]), "+r"(b[11]), "+r"(b[12]), "+r"(b[13]), "+r"(b[14]), "+r"(b[15])
+                 :
+                 : "memory");
 }
 
 __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_constant__ GemmTcParams p)
@@ -214,14 +221,16 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
     float *red = reinterpret_cast<float *>(smem);      // [mt][NB][128] fp32, reuses the ring
 
+    // hi- and lo-plane columns are fetched together, one wait for both
     auto load_chunk = [&](int m, int c, float (&v)[16]) {
         if (have) {
-            float lo[16];
-            tc_ld16(t_lane + m * 2 * p.NB + c * 16, v);
-            tc_ld16(t_lane + m * 2 * p.NB + p.NB + c * 16, lo);
+            uint32_t hi[16], lo[16];
+            tc_ld16_issue(t_lane + m * 2 * p.NB + c * 16, hi);
+            tc_ld16_issue(t_lane + m * 2 * p.NB + p.NB + c * 16, lo);
+            tc_ld_wait(hi, lo);
 #pragma unroll
             for (int i = 0; i < 16; ++i)
-                v[i] += lo[i];
+                v[i] = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
         } else {
 #pragma unroll
             for (int i = 0; i < 16; ++i)
@@ -247,9 +256,10 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 const int m = j / nchunks, c = j % nchunks;
                 float v[16];
                 load_chunk(m, c, v);
+                const uint32_t a = smem_u32(red) + (uint32_t)((m * p.NB + c * 16) * kTcTileM + row) * 4u;
 #pragma unroll
                 for (int i = 0; i < 16; ++i)
-                    red[((size_t)m * p.NB + c * 16 + i) * kTcTileM + row] = v[i];
+                    sts_f32(a + i * (kTcTileM * 4), v[i]);
             }
             fence_proxy_async_smem();
             asm volatile("bar.sync 1, %0;" ::"r"(kSubs * 128) : "memory");
@@ -314,14 +324,14 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         // share with plain stores), then waits until its own area is complete and sums the sources in
         // rank order.  No cluster barrier and no remote loads on the critical path.
         const int cols = p.NB / p.splits;
-        float *recv = reinterpret_cast<float *>(smem + p.recv_off);
-        const size_t src_stride = (size_t)p.mt * kTcTileM * cols;          // floats per source rank
+        const uint32_t recv_a = smem_u32(smem + p.recv_off);
+        const uint32_t src_stride = (uint32_t)p.mt * kTcTileM * cols * 4u;          // bytes per source rank
         if (warp >= 2) {
             for (int j = sub; j < p.mt * nchunks; j += kSubs) {
                 const int m = j / nchunks, c = j % nchunks;
                 float v[16];
                 load_chunk(m, c, v);
-                const size_t off = (size_t)s * src_stride + ((size_t)m * kTcTileM + row) * cols;   // my slot, my row
+                const uint32_t off = recv_a + s * src_stride + (uint32_t)((m * kTcTileM + row) * cols) * 4u;   // my slot, my row
 #pragma unroll
                 for (int i = 0; i < 16; i += 2) {
                     const int col = c * 16 + i, q = col / cols, cl = col % cols;
@@ -329,38 +339,54 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                         if (i % 4 == 0) {
                             const float4 val = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
                             if (q == s)
-                                *reinterpret_cast<float4 *>(recv + off + cl) = val;
+                                sts_f32x4(off + cl * 4, val);
                             else
-                                st_async_v4(cluster_map(recv + off + cl, q), val, cluster_map(&push_bar, q));
+                                st_async_v4(cluster_map_addr(off + cl * 4, q), val, cluster_map(&push_bar, q));
                         }
                     } else {
                         const float2 val = make_float2(v[i], v[i + 1]);
                         if (q == s)
-                            *reinterpret_cast<float2 *>(recv + off + cl) = val;
+                            sts_f32x2(off + cl * 4, val);
                         else
-                            st_async_v2(cluster_map(recv + off + cl, q), val, cluster_map(&push_bar, q));
+                            st_async_v2(cluster_map_addr(off + cl * 4, q), val, cluster_map(&push_bar, q));
                     }
                 }
             }
             asm volatile("bar.sync 1, %0;" ::"r"(kSubs * 128) : "memory");    // own share stored by all epilogue warps
             if (!mbar_wait(&push_bar, 0, p.status, ST_TIMEOUT_MMA))
                 poisoned = 1;
-            const int n_pairs = p.mt * cols / 2;
-            for (int it = sub; it < n_pairs; it += kSubs) {
-                const int m = it / (cols / 2), cl = 2 * (it % (cols / 2));
-                const int pair = ((tile * p.mt + m) * kTcTileM + row) >> 1;
-                float mine[2] = {0.f, 0.f};
-                for (int q = 0; q < p.splits; ++q) {       // rank order
-                    const float2 t2 = *reinterpret_cast<const float2 *>(recv + (size_t)q * src_stride +
-                                                                        ((size_t)m * kTcTileM + row) * cols + cl);
-                    mine[0] += t2.x;
-                    mine[1] += t2.y;
+            const bool bad = poisoned;
+            const uint32_t row_a = recv_a + (uint32_t)(row * cols) * 4u;
+            const uint32_t mstr = (uint32_t)(kTcTileM * cols) * 4u;
+            auto finish = [&](auto sp_tag) {
+                constexpr int SP = decltype(sp_tag)::value;
+                const int hp = cols / 2;                   // column pairs per m
+                int m = 0, c2 = sub;
+                while (c2 >= hp) { c2 -= hp; ++m; }
+                while (m < p.mt) {
+                    const uint32_t a = row_a + m * mstr + c2 * 8u;
+                    float mine[2] = {0.f, 0.f};
+#pragma unroll
+                    for (int q = 0; q < SP; ++q) {         // rank order
+                        const float2 t2 = lds_f32x2(a + q * src_stride);
+                        mine[0] += t2.x;
+                        mine[1] += t2.y;
+                    }
+                    const float got = __shfl_xor_sync(0xffffffffu, par ? mine[0] : mine[1], 1);
+                    const int b = s * cols + 2 * c2 + par;
+                    const int pair = ((tile * p.mt + m) * kTcTileM + row) >> 1;
+                    if (b < p.B && !bad)
+                        apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? got : mine[0], par ? mine[1] : got);
+                    c2 += kSubs;
+                    while (c2 >= hp) { c2 -= hp; ++m; }
                 }
-                const float got = __shfl_xor_sync(0xffffffffu, par ? mine[0] : mine[1], 1);
-                const int b = s * cols + cl + par;
-                if (b < p.B && !poisoned)
-                    apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? got : mine[0], par ? mine[1] : got);
-            }
+            };
+            if (p.splits == 2)
+                finish(std::integral_constant<int, 2>());
+            else if (p.splits == 4)
+                finish(std::integral_constant<int, 4>());
+            else
+                finish(std::integral_constant<int, 8>());
         }
     } else if (p.splits > 1) {
         // Split-K across the cluster, reduce-scatter style: every rank publishes its partial tiles in

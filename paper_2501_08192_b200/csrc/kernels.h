@@ -41,6 +41,7 @@ struct WindowArgs {
     int B, H;
     long long *trace;              // optional timeline slot (4 values), see common.cuh
     int delay_ns;                  // modelled communication latency added to the window (0 = none)
+    int *status;                   // device error word (bounded waits report here)
 };
 cudaError_t launch_window(const WindowArgs &a, cudaStream_t s);
 

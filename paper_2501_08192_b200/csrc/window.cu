@@ -6,7 +6,7 @@
 // 128-bit loads of a thread are all in flight together, and a row's bytes are
 // requested by many warps on several SMs (the same bytes requested by the few
 // warps of one SM take several times longer).  The slices' sums of squares meet
-// through distributed shared memory and are added in rank order.  fp32
+// by one-sided stores into each peer's shared memory and are added in rank order.  fp32
 // accumulation in the fixed order residual, part 0..P-1 (part 0 may be fp32: this
 // shard's own result, or the previous layer's in a chain).
 // Loads of buffers that are inputs of the step are issued before the
@@ -40,6 +40,7 @@ struct WindowParams {
     int cluster;         // CTAs per row
     long long *trace;
     int delay_ns;
+    int *status;
 };
 
 template <bool RESID_F32, bool PART0_F32>
@@ -63,6 +64,19 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
     trace_start(p.trace);
     pdl_launch_dependents();   // the next kernel may start fetching its weights now
 
+    // The slices' sums of squares are handed over one-sidedly: every CTA of the row stores its sum
+    // into each peer's recv[] slot, signalling the peer's barrier.  The barriers must exist before
+    // anybody sends: one cluster barrier here, long before the data it guards.
+    __shared__ uint64_t recv_bar;
+    __shared__ float recv[kWinMaxCluster];
+    if (p.cluster > 1) {
+        if (threadIdx.x == 0) {
+            mbar_init(&recv_bar, 1);
+            mbar_fence_init();
+            mbar_expect_tx(&recv_bar, (uint32_t)(p.cluster - 1) * 4u);
+        }
+    }
+
     // Buffers that are inputs of the step (the peers' partial sums, and the residual / partial 0
     // unless they are handed over in fp32 by an earlier kernel of the step) do not depend on the
     // previous kernel either: their loads - the only ones that go to HBM - are issued before the
@@ -80,6 +94,9 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
                     pre[c][j] = ld_stream(p.parts[j] + row_off + ch);
         }
     }
+
+    if (p.cluster > 1)
+        cg::this_cluster().sync();      // (the loads above are in flight meanwhile)
 
     pdl_wait();                // this shard's own partial sum comes from the preceding kernel in the stream
     trace_waited(p.trace);
@@ -135,7 +152,6 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
     // block reduction of the sum of squares (fixed tree: bit-stable run to run)
     __shared__ float warp_sums[32];
     __shared__ float total;
-    __shared__ float slice_sum;      // this CTA's part, read by the other CTAs of the row
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1)
         ss += __shfl_xor_sync(0xffffffffu, ss, o);
@@ -148,22 +164,24 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
         float t = lane < nw ? warp_sums[lane] : 0.f;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1)
-            t += __shfl_xor_sync(0xffffffffu, t, o);
-        if (lane == 0) {
+            t += __shfl_xor_sync(0xffffffffu, t, o);      // every lane holds the CTA's sum
+        if (lane == 0)
             total = t;
-            slice_sum = t;
+        if (p.cluster > 1 && lane < p.cluster) {
+            if (lane == rank)
+                recv[rank] = t;
+            else
+                st_async_f32(cluster_map(&recv[rank], lane), t, cluster_map(&recv_bar, lane));
         }
     }
     __syncthreads();
     float row_total = total;
     if (p.cluster > 1) {
         // sum of the slices in rank order (the same order in every CTA of the row)
-        cg::cluster_group cluster = cg::this_cluster();
-        cluster.sync();
         row_total = 0.f;
-        for (int q = 0; q < p.cluster; ++q)
-            row_total += *cluster.map_shared_rank(&slice_sum, q);
-        cluster.sync();      // peers' shared memory must outlive the reads
+        if (mbar_wait(&recv_bar, 0, p.status, ST_TIMEOUT_FULL))
+            for (int q = 0; q < p.cluster; ++q)
+                row_total += recv[q];
     }
     const float inv = rsqrtf(row_total / (float)p.H + p.eps);
 
@@ -226,6 +244,7 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
     p.H = a.H;
     p.trace = a.trace;
     p.delay_ns = a.delay_ns;
+    p.status = a.status;
     // CTAs per row: as many (a power of two, at most 8) as leave every CTA at least 128 threads of
     // one 8-element chunk each
     int cl = 1;
