@@ -83,6 +83,46 @@ __device__ __forceinline__ void load_epilogue_tables(const EpilogueArgs &e, Epil
         t.inv_freq[i] = e.inv_freq ? e.inv_freq[i] : 0.0;
 }
 
+// Rotary factors (cos, sin) of rotary pair i at sequence position pos; (1, 0) for heads that are
+// not rotated (values) and when the layer has no rotary embedding.
+__device__ __forceinline__ float2 rope_trig(const EpilogueArgs &e, const EpilogueTables &tab, int pos, int hd, int i)
+{
+    if (!(hd < e.nq + e.nkv && e.inv_freq))
+        return make_float2(1.f, 0.f);
+    // angle = pos * theta^(-2i/d): the product and its reduction mod 2 pi need more than
+    // fp32 (angles reach tens of thousands of radians); the reduced angle does not
+    const double ang = (double)pos * tab.inv_freq[i];
+    const double turns = rint(ang * 0.15915494309189535);
+    const float red = (float)fma(-turns, 6.283185307179586, ang);
+    float sf, cf;
+    sincosf(red, &sf, &cf);
+    return make_float2(cf, sf);
+}
+
+// The QKV epilogue of one rotary pair with its factors given: rotate, then q to the query planes,
+// k and v to the cache at slot pos.
+__device__ __forceinline__ void epilogue_qkv(const EpilogueArgs &e, int pos, int b, int hd, int i, float v0, float v1,
+                                             float2 cs)
+{
+    if (hd < e.nq + e.nkv && e.inv_freq) {
+        const float r0 = v0 * cs.x - v1 * cs.y;
+        const float r1 = v1 * cs.x + v0 * cs.y;
+        v0 = r0; v1 = r1;
+    }
+    if (hd < e.nq) {
+        const size_t o = ((size_t)b * e.nq + hd) * kHeadDim + i;
+        store_split(e.q_out, e.q_plane, o, v0);
+        store_split(e.q_out, e.q_plane, o + kHeadDim / 2, v1);
+    } else {
+        const bool is_k = hd < e.nq + e.nkv;
+        const int kvh = is_k ? hd - e.nq : hd - e.nq - e.nkv;
+        const size_t o = (((size_t)b * e.nkv + kvh) * e.cap + pos) * kHeadDim + i;
+        void *dst = is_k ? e.k_cache : e.v_cache;
+        store_bf16(dst, o, v0);
+        store_bf16(dst, o + kHeadDim / 2, v1);
+    }
+}
+
 // Apply the epilogue to one pair of fp32 results of batch row b (b_local = b - b0 indexes the tables).
 __device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, const EpilogueTables &tab, int b_local,
                                                bool tensor_path, int N, int b, int pair, float v0, float v1)
@@ -90,6 +130,17 @@ __device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, const Epil
     int n0, n1;
     pair_coords(e.kind, tensor_path, pair, n0, n1);
     if (e.kind == EPI_PLAIN) {
+        if (tensor_path) {
+            // the pair's outputs are neighbours: one store per buffer
+            const size_t o = (size_t)b * N + n0;
+            if (e.out)
+                *reinterpret_cast<uint32_t *>(reinterpret_cast<bf16 *>(e.out) + o) = pack_bf16(v0, v1);
+            if (e.out2)
+                *reinterpret_cast<uint32_t *>(reinterpret_cast<bf16 *>(e.out2) + o) = pack_bf16(v0, v1);
+            if (e.out_f32)
+                *reinterpret_cast<float2 *>(e.out_f32 + o) = make_float2(v0, v1);
+            return;
+        }
         if (e.out) {
             store_bf16(e.out, (size_t)b * N + n0, v0);
             store_bf16(e.out, (size_t)b * N + n1, v1);
@@ -108,31 +159,63 @@ __device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, const Epil
         const float a = __fdividef(v0, 1.f + __expf(-v0)) * v1;
         store_split(e.out, e.out_plane, (size_t)b * (N >> 1) + n0, a);
     } else {
-        const int hd = n0, i = n1;
         const int pos = tab.pos[b_local];
+        epilogue_qkv(e, pos, b, n0, n1, v0, v1, rope_trig(e, tab, pos, n0, n1));
+    }
+}
+
+// Tensor path, two neighbouring pairs (pair0 even, and pair0 + 1) of batch row b at once:
+// v = (v0, v1) of pair0 then (v0, v1) of pair0 + 1.  Their outputs are neighbours in every output
+// buffer, so each buffer takes one vector store.  cs0 / cs1: the pairs' rotary factors when
+// have_trig (QKV only), else computed here.
+__device__ __forceinline__ void apply_epilogue_quad(const EpilogueArgs &e, const EpilogueTables &tab, int N, int b,
+                                                    int pair0, float4 v, bool have_trig, float2 cs0, float2 cs1)
+{
+    if (e.kind == EPI_PLAIN) {
+        const size_t o = (size_t)b * N + 2 * (size_t)pair0;
+        const uint2 packed = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
+        if (e.out)
+            *reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(e.out) + o) = packed;
+        if (e.out2)
+            *reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(e.out2) + o) = packed;
+        if (e.out_f32)
+            *reinterpret_cast<float4 *>(e.out_f32 + o) = v;
+    } else if (e.kind == EPI_SWIGLU) {
+        const float a0 = __fdividef(v.x, 1.f + __expf(-v.x)) * v.y;
+        const float a1 = __fdividef(v.z, 1.f + __expf(-v.z)) * v.w;
+        uint32_t hi, lo;
+        split_bf16x2(a0, a1, hi, lo);
+        const size_t o = (size_t)b * (N >> 1) + pair0;
+        *reinterpret_cast<uint32_t *>(reinterpret_cast<bf16 *>(e.out) + o) = hi;
+        *reinterpret_cast<uint32_t *>(reinterpret_cast<bf16 *>(e.out) + e.out_plane + o) = lo;
+    } else {
+        const int pos = tab.pos[b], hd = pair0 >> 6, i = pair0 & 63;
+        if (!have_trig) {
+            cs0 = rope_trig(e, tab, pos, hd, i);
+            cs1 = rope_trig(e, tab, pos, hd, i + 1);
+        }
+        float a0 = v.x, a1 = v.y, c0 = v.z, c1 = v.w;     // dims i, i + d/2 and i + 1, i + 1 + d/2
         if (hd < e.nq + e.nkv && e.inv_freq) {
-            // angle = pos * theta^(-2i/d): the product and its reduction mod 2 pi need more than
-            // fp32 (angles reach tens of thousands of radians); the reduced angle does not
-            const double ang = (double)pos * tab.inv_freq[i];
-            const double turns = rint(ang * 0.15915494309189535);
-            const float red = (float)fma(-turns, 6.283185307179586, ang);
-            float sf, cf;
-            sincosf(red, &sf, &cf);
-            const float r0 = v0 * cf - v1 * sf;
-            const float r1 = v1 * cf + v0 * sf;
-            v0 = r0; v1 = r1;
+            a0 = v.x * cs0.x - v.y * cs0.y; a1 = v.y * cs0.x + v.x * cs0.y;
+            c0 = v.z * cs1.x - v.w * cs1.y; c1 = v.w * cs1.x + v.z * cs1.y;
         }
         if (hd < e.nq) {
             const size_t o = ((size_t)b * e.nq + hd) * kHeadDim + i;
-            store_split(e.q_out, e.q_plane, o, v0);
-            store_split(e.q_out, e.q_plane, o + kHeadDim / 2, v1);
+            bf16 *q = reinterpret_cast<bf16 *>(e.q_out);
+            uint32_t hi, lo;
+            split_bf16x2(a0, c0, hi, lo);
+            *reinterpret_cast<uint32_t *>(q + o) = hi;
+            *reinterpret_cast<uint32_t *>(q + e.q_plane + o) = lo;
+            split_bf16x2(a1, c1, hi, lo);
+            *reinterpret_cast<uint32_t *>(q + o + kHeadDim / 2) = hi;
+            *reinterpret_cast<uint32_t *>(q + e.q_plane + o + kHeadDim / 2) = lo;
         } else {
             const bool is_k = hd < e.nq + e.nkv;
             const int kvh = is_k ? hd - e.nq : hd - e.nq - e.nkv;
             const size_t o = (((size_t)b * e.nkv + kvh) * e.cap + pos) * kHeadDim + i;
-            void *dst = is_k ? e.k_cache : e.v_cache;
-            store_bf16(dst, o, v0);
-            store_bf16(dst, o + kHeadDim / 2, v1);
+            bf16 *dst = reinterpret_cast<bf16 *>(is_k ? e.k_cache : e.v_cache);
+            *reinterpret_cast<uint32_t *>(dst + o) = pack_bf16(a0, c0);
+            *reinterpret_cast<uint32_t *>(dst + o + kHeadDim / 2) = pack_bf16(a1, c1);
         }
     }
 }

@@ -210,6 +210,47 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     const int nchunks = p.NB / 16;
     const int sub = warp >= 2 ? (warp - 2) >> 2 : 0;     // which of the lane group's warps this is
     const int kSubs = ((int)blockDim.x / 32 - 2) / 4;    // warps per lane group
+    const int par = lane & 1;
+    // Rotary factors of this thread's first two finish iterations of a one-sided split-K reduction
+    // (the iteration order is fixed: column pairs sub, sub + kSubs, ... of this rank's columns):
+    // computed here, while the weights stream, instead of in the tail.
+    float2 trig[2] = {make_float2(1.f, 0.f), make_float2(1.f, 0.f)};
+    if (warp >= 2 && p.epi.kind == EPI_QKV && p.splits > 1 && p.push == 2) {
+        // (bulk form: a warp's first item is column warp - 2 of this rank's mt * cols (m, column)
+        // items, a lane's two pairs are rows 4 * lane .. 4 * lane + 3)
+        const int cols = p.NB / p.splits;
+        int m = 0, cl = warp - 2;
+        while (cl >= cols) { cl -= cols; ++m; }
+        const int b = s * cols + cl;
+        if (m < p.mt && b < p.B) {
+            trig[0] = rope_trig(p.epi, tabs, tabs.pos[b], tile * p.mt + m, 2 * lane);
+            trig[1] = rope_trig(p.epi, tabs, tabs.pos[b], tile * p.mt + m, 2 * lane + 1);
+        }
+    } else if (warp >= 2 && p.epi.kind == EPI_QKV && p.splits > 1 && p.push) {
+        const int cols = p.NB / p.splits, hp = cols / 2;
+        int m = 0, c2 = sub;
+        while (c2 >= hp) { c2 -= hp; ++m; }
+#pragma unroll
+        for (int k = 0; k < 2; ++k)
+            if (m < p.mt) {
+                const int b = s * cols + 2 * c2 + par;
+                if (b < p.B)
+                    trig[k] = rope_trig(p.epi, tabs, tabs.pos[b], tile * p.mt + m, row >> 1);
+                c2 += kSubs;
+                while (c2 >= hp) { c2 -= hp; ++m; }
+            }
+    }
+    // one finished pair of iteration k (k < 2 uses the factors above)
+    auto finish_pair = [&](int k, int m, int b, float v0, float v1) {
+        const int pair = ((tile * p.mt + m) * kTcTileM + row) >> 1;
+        if (p.epi.kind == EPI_QKV) {
+            const int pos = tabs.pos[b], hd = pair >> 6, i = pair & 63;
+            const float2 cs = k == 0 ? trig[0] : (k == 1 ? trig[1] : rope_trig(p.epi, tabs, pos, hd, i));
+            epilogue_qkv(p.epi, pos, b, hd, i, v0, v1, cs);
+        } else {
+            apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, v0, v1);
+        }
+    };
     bool have = false;
     if (warp >= 2) {
         have = mbar_wait(&accum_bar, 0, p.status, ST_TIMEOUT_MMA);
@@ -238,7 +279,6 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         }
     };
 
-    const int par = lane & 1;
     if (p.splits > 1 && p.push == 2) {
         // Split-K across the cluster for wide batches, one-sided reduce-scatter by bulk copies: every
         // rank lays its partial tiles out in its own (idle) ring as [m][column][row], then one bulk
@@ -277,36 +317,36 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         }
         cluster_arrive_relaxed();
         if (warp >= 2) {
-            const uint32_t red_a = smem_u32(red) + (uint32_t)(s * cols * kTcTileM + row) * 4u;
-            const uint32_t recv_a = smem_u32(recv) + (uint32_t)row * 4u;
+            // finish this rank's columns: one (m, column) item per warp and iteration, a lane takes
+            // rows 4 * lane .. 4 * lane + 3 - two complete output pairs - with one 16-byte load per rank
+            const int n_ew = kSubs * 4;
+            const uint32_t red_a = smem_u32(red) + (uint32_t)(s * cols * kTcTileM) * 4u + lane * 16u;
+            const uint32_t recv_a = smem_u32(recv) + lane * 16u;
             const bool bad = poisoned;
             auto finish = [&](auto sp_tag) {
                 constexpr int SP = decltype(sp_tag)::value;
-                // per source rank: address of (m = 0, column 0, this row) and the stride between m
+                // per source rank: address of (m = 0, column 0, this lane's rows) and the stride between m
                 uint32_t base[SP], mstr[SP];
 #pragma unroll
                 for (int q = 0; q < SP; ++q) {
                     base[q] = q == s ? red_a : recv_a + (uint32_t)((q < s ? q : q - 1) * p.mt * cols) * (kTcTileM * 4u);
                     mstr[q] = (uint32_t)(q == s ? p.NB : cols) * (kTcTileM * 4u);
                 }
-                const int hp = cols / 2;                   // column pairs per m
-                int m = 0, c2 = sub;
-                while (c2 >= hp) { c2 -= hp; ++m; }
-                while (m < p.mt) {
-                    float mine[2] = {0.f, 0.f};
+                int m = 0, cl = warp - 2;
+                while (cl >= cols) { cl -= cols; ++m; }
+                for (int k = 0; m < p.mt; ++k) {
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                     for (int q = 0; q < SP; ++q) {         // rank order
-                        const uint32_t a = base[q] + m * mstr[q] + (uint32_t)c2 * (2u * kTcTileM * 4u);
-                        mine[0] += lds_f32(a);
-                        mine[1] += lds_f32(a + kTcTileM * 4u);
+                        const float4 t4 = lds_f32x4(base[q] + m * mstr[q] + (uint32_t)cl * (kTcTileM * 4u));
+                        acc.x += t4.x; acc.y += t4.y; acc.z += t4.z; acc.w += t4.w;
                     }
-                    const float got = __shfl_xor_sync(0xffffffffu, par ? mine[0] : mine[1], 1);
-                    const int b = s * cols + 2 * c2 + par;
-                    const int pair = ((tile * p.mt + m) * kTcTileM + row) >> 1;
+                    const int b = s * cols + cl;
                     if (b < p.B && !bad)
-                        apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? got : mine[0], par ? mine[1] : got);
-                    c2 += kSubs;
-                    while (c2 >= hp) { c2 -= hp; ++m; }
+                        apply_epilogue_quad(p.epi, tabs, p.N, b, (tile * p.mt + m) * (kTcTileM / 2) + 2 * lane, acc, k == 0,
+                                            trig[0], trig[1]);
+                    cl += n_ew;
+                    while (cl >= cols) { cl -= cols; ++m; }
                 }
             };
             if (p.splits == 2)
@@ -363,7 +403,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 const int hp = cols / 2;                   // column pairs per m
                 int m = 0, c2 = sub;
                 while (c2 >= hp) { c2 -= hp; ++m; }
-                while (m < p.mt) {
+                for (int k = 0; m < p.mt; ++k) {
                     const uint32_t a = row_a + m * mstr + c2 * 8u;
                     float mine[2] = {0.f, 0.f};
 #pragma unroll
@@ -374,9 +414,8 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                     }
                     const float got = __shfl_xor_sync(0xffffffffu, par ? mine[0] : mine[1], 1);
                     const int b = s * cols + 2 * c2 + par;
-                    const int pair = ((tile * p.mt + m) * kTcTileM + row) >> 1;
                     if (b < p.B && !bad)
-                        apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? got : mine[0], par ? mine[1] : got);
+                        finish_pair(k, m, b, par ? got : mine[0], par ? mine[1] : got);
                     c2 += kSubs;
                     while (c2 >= hp) { c2 -= hp; ++m; }
                 }

@@ -63,6 +63,9 @@ struct GemvParams {
     int recv_off;        // push: offset of rank 0's receive area in dynamic shared memory
     int *status;
     long long *trace;
+    const uint8_t *next_w;
+    uint32_t next_slice;   // bytes of next_w each CTA prefetches
+    size_t next_bytes;
     EpilogueArgs epi;
 };
 
@@ -256,6 +259,15 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
         }
 
         trace_streamed(p.trace, threadIdx.x == 0);
+        if (p.next_slice && grp + (int)gridDim.x >= p.groups && threadIdx.x == 32) {
+            // this CTA's stream is over: HBM would idle until the next kernel's late CTAs start -
+            // pull its slice of that kernel's weights into L2 meanwhile
+            const size_t o = (size_t)(blockIdx.y * gridDim.x + blockIdx.x) * p.next_slice;
+            if (o < p.next_bytes) {
+                const size_t left = p.next_bytes - o;
+                bulk_prefetch_l2(p.next_w + o, (uint32_t)(left < p.next_slice ? left : p.next_slice) & ~15u);
+            }
+        }
         // ---- warp partial -> shared memory: red[warp][row block of the warp * 16 + row][b]
 #pragma unroll
         for (int r = 0; r < RB; ++r) {
@@ -396,6 +408,11 @@ static cudaError_t launch_variant(GemvParams &p, int sm_count, cudaStream_t s)
     const size_t recv_bytes = (size_t)(p.splits - 1) * (kGemvWarps / p.warps_k * RB) * 16 * NB * 4;
     p.push = p.splits > 1 && groups_per_cta == 1 && recv_bytes <= 32 * 1024;
     p.recv_off = (int)ring_bytes;
+    p.next_slice = 0;
+    if (p.next_w && p.next_bytes) {
+        const size_t n_ctas = (size_t)clusters * p.splits;
+        p.next_slice = (uint32_t)(((p.next_bytes + n_ctas - 1) / n_ctas + 127) & ~size_t(127));
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(clusters, p.splits, 1);
     cfg.blockDim = dim3(kGemvWarps * 32);
@@ -429,6 +446,8 @@ cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s)
     p.epi = a.epi;
     p.status = a.status;
     p.trace = a.trace;
+    p.next_w = reinterpret_cast<const uint8_t *>(a.next_w);
+    p.next_bytes = a.next_bytes;
 
     // two row blocks per warp whenever the matrix has enough row blocks to still fill the SMs
     const bool two = p.row_blocks % 2 == 0 && p.row_blocks >= 32;

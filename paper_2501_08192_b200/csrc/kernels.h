@@ -83,6 +83,8 @@ struct GemvArgs {
     EpilogueArgs epi;
     int *status;
     long long *trace;
+    const void *next_w;   // optional: weights of the kernel that follows, prefetched to L2 once this one has streamed its own
+    size_t next_bytes;
 };
 cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s);
 
