@@ -84,6 +84,20 @@ __device__ __forceinline__ void tc_ld16_issue(uint32_t taddr, uint32_t (&r)[16])
                    "=r"(r[15])
                  : "r"(taddr));
 }
+__device__ __forceinline__ void tc_ld_wait4(uint32_t (&a)[16], uint32_t (&b)[16], uint32_t (&c)[16], uint32_t (&d)[16])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]),
+                   "+r"(a[8]), "+r"(a[9]), "+r"(a[10]), "+r"(a[11]), "+r"(a[12]), "+r"(a[13]), "+r"(a[14]), "+r"(a[15]),
+                   "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7]),
+                   "+r"(b[8]), "+r"(b[9]), "+r"(b[10]), "+r"(b[11]), "+r"(b[12]), "+r"(b[13]), "+r"(b[14]), "+r"(b[15]),
+                   "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3]), "+r"(c[4]), "+r"(c[5]), "+r"(c[6]), "+r"(c[7]),
+                   "+r"(c[8]), "+r"(c[9]), "+r"(c[10]), "+r"(c[11]), "+r"(c[12]), "+r"(c[13]), "+r"(c[14]), "+r"(c[15]),
+                   "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]), "+r"(d[4]), "+r"(d[5]), "+r"(d[6]), "+r"(d[7]),
+                   "+r"(d[8]), "+r"(d[9]), "+r"(d[10]), "+r"(d[11]), "+r"(d[12]), "+r"(d[13]), "+r"(d[14]), "+r"(d[15])
+                 :
+                 : "memory");
+}
 __device__ __forceinline__ void tc_ld_wait(uint32_t (&a)[16], uint32_t (&b)[16])
 {
     asm volatile("tcgen05.wait::ld.sync.aligned;"
@@ -292,18 +306,42 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         const int cols = p.NB / p.splits;
         float *recv = reinterpret_cast<float *>(smem + p.recv_off);
         if (warp >= 2) {
-            for (int j = sub; j < p.mt * nchunks; j += kSubs) {
-                const int m = j / nchunks, c = j % nchunks;
-                float v[16];
-                load_chunk(m, c, v);
-                const uint32_t a = smem_u32(red) + (uint32_t)((m * p.NB + c * 16) * kTcTileM + row) * 4u;
+            // two chunks (four TMEM loads) in flight per wait
+            const uint32_t red_row = smem_u32(red) + (uint32_t)row * 4u;
+            for (int j = sub; j < p.mt * nchunks; j += 2 * kSubs) {
+                const int j1 = j + kSubs;
+                const bool two = j1 < p.mt * nchunks;
+                const int m0 = j / nchunks, c0 = j % nchunks;
+                const int m1 = two ? j1 / nchunks : m0, c1 = two ? j1 % nchunks : c0;
+                uint32_t h0[16], l0[16], h1[16], l1[16];
+                if (have) {
+                    tc_ld16_issue(t_lane + m0 * 2 * p.NB + c0 * 16, h0);
+                    tc_ld16_issue(t_lane + m0 * 2 * p.NB + p.NB + c0 * 16, l0);
+                    tc_ld16_issue(t_lane + m1 * 2 * p.NB + c1 * 16, h1);
+                    tc_ld16_issue(t_lane + m1 * 2 * p.NB + p.NB + c1 * 16, l1);
+                    tc_ld_wait4(h0, l0, h1, l1);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        h0[i] = l0[i] = h1[i] = l1[i] = 0u;
+                }
+                const uint32_t a0 = red_row + (uint32_t)((m0 * p.NB + c0 * 16) * kTcTileM) * 4u;
 #pragma unroll
                 for (int i = 0; i < 16; ++i)
-                    sts_f32(a + i * (kTcTileM * 4), v[i]);
+                    sts_f32(a0 + i * (kTcTileM * 4), __uint_as_float(h0[i]) + __uint_as_float(l0[i]));
+                if (two) {
+                    const uint32_t a1 = red_row + (uint32_t)((m1 * p.NB + c1 * 16) * kTcTileM) * 4u;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        sts_f32(a1 + i * (kTcTileM * 4), __uint_as_float(h1[i]) + __uint_as_float(l1[i]));
+                }
             }
             fence_proxy_async_smem();
             asm volatile("bar.sync 1, %0;" ::"r"(kSubs * 128) : "memory");
-            const int e = (int)threadIdx.x - 64;
+            // copy e is issued by lane e / n_warps of epilogue warp e % n_warps: spread over the warps,
+            // the (splits - 1) * mt copies go out side by side
+            const int n_ewarps = kSubs * 4;
+            const int e = lane < 8 ? (warp - 2) + lane * n_ewarps : 1 << 30;
             if (e < (p.splits - 1) * p.mt) {
                 const int slot_q = e / p.mt, m = e % p.mt;
                 const int q = slot_q < s ? slot_q : slot_q + 1;      // owner
