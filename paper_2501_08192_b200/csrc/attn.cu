@@ -446,30 +446,35 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
         }
         consumer_barrier();
         const int n_items_stream = sm.item_base[sidx + 1] - sm.item_base[sidx];
-        const int d = threadIdx.x;                       // one head dim per consumer thread
-        for (int r = 0; r < p.G; ++r) {
+        // two head dims per consumer thread, the heads of one parity per half of the threads
+        const int d2 = threadIdx.x & 63;
+        for (int r = threadIdx.x >> 6; r < p.G; r += 2) {
             float M = -INFINITY;
 #pragma unroll
             for (int w = 0; w < kConsumerWarps; ++w)
                 M = fmaxf(M, sm.comb_ml[w][r][0]);
-            float acc = 0.f, lsum = 0.f;
+            float2 acc = make_float2(0.f, 0.f);
+            float lsum = 0.f;
 #pragma unroll
             for (int w = 0; w < kConsumerWarps; ++w) {
                 const float mw = sm.comb_ml[w][r][0];
                 const float c = mw == -INFINITY ? 0.f : exp2f(mw - M);
-                acc += comb_row(stage_last, w, r)[2 * comb_col2(r, d >> 1) + (d & 1)] * c;
+                const float2 v = reinterpret_cast<const float2 *>(comb_row(stage_last, w, r))[comb_col2(r, d2)];
+                acc.x += v.x * c;
+                acc.y += v.y * c;
                 lsum += sm.comb_ml[w][r][1] * c;
             }
             if (n_items_stream == 1) {
                 // the item is the whole sequence: finish here
-                const float ov = acc / lsum;
-                const bf16 hi = __float2bfloat16_rn(ov);
-                const size_t oi = ((size_t)b * p.nq + (size_t)kvh * p.G + r) * kHeadDim + d;
-                p.o_out[oi] = hi;
-                p.o_out[p.o_plane + oi] = __float2bfloat16_rn(ov - __bfloat162float(hi));
+                const float o0 = acc.x / lsum, o1 = acc.y / lsum;
+                uint32_t hi, lo;
+                split_bf16x2(o0, o1, hi, lo);
+                const size_t oi = ((size_t)b * p.nq + (size_t)kvh * p.G + r) * kHeadDim + 2 * d2;
+                *reinterpret_cast<uint32_t *>(p.o_out + oi) = hi;
+                *reinterpret_cast<uint32_t *>(p.o_out + p.o_plane + oi) = lo;
             } else {
-                p.part_o[((size_t)item * p.G + r) * kHeadDim + d] = acc;
-                if (d == 0)
+                *reinterpret_cast<float2 *>(p.part_o + ((size_t)item * p.G + r) * kHeadDim + 2 * d2) = acc;
+                if (d2 == 0)
                     *reinterpret_cast<float2 *>(p.part_ml + ((size_t)item * p.G + r) * 2) = make_float2(M, lsum);
             }
         }
@@ -572,6 +577,24 @@ void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_coun
         const int nt = (ctx_len_host[b] + 1 + kTileKeys - 1) / kTileKeys;
         total_tiles += (uint64_t)nkv * nt;
         longest = nt > longest ? nt : longest;
+    }
+    // A short cache fits the CTAs' rings whole: items of at most kStages tiles, one per CTA, are then
+    // all in shared memory before the queries exist, and what remains after the wait is arithmetic.
+    // The shortest such items that leave a (sequence, head) at most one partial per merge warp.
+    for (int tpi = 1; tpi <= kStages; ++tpi) {
+        uint64_t items = 0;
+        int per_stream = 0;
+        for (int b = 0; b < batch; ++b) {
+            const int nt = (ctx_len_host[b] + 1 + kTileKeys - 1) / kTileKeys;
+            const int n = (nt + tpi - 1) / tpi;
+            items += (uint64_t)nkv * n;
+            per_stream = n > per_stream ? n : per_stream;
+        }
+        if (items <= (uint64_t)2 * sm_count && per_stream <= 32) {
+            *grid = items <= (uint64_t)sm_count ? sm_count : 2 * sm_count;
+            *tiles_per_item = tpi;
+            return;
+        }
     }
     // One CTA per SM while the whole cache is at most two ring fills per SM: the ring then holds
     // most of the CTA's share before the queries exist, and half of every SM's shared memory stays
