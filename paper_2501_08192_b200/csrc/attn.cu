@@ -538,21 +538,24 @@ __global__ void __launch_bounds__(kMergeMaxWarps * 32) k_attn_merge(const __grid
             acc.z = acc.z * c + ov.z * w; acc.w = acc.w * c + ov.w * w;
             Mg = mb;
         }
-        *reinterpret_cast<float4 *>(&acc_s[warp][4 * lane]) = acc;
-        if (lane == 0) {
+        if (lane == 0)
             m_s[warp] = Mg;
-            l_s[warp] = L;
-        }
+        __syncthreads();
+        // every warp rescales its own result to the common maximum (so the final sum is plain adds)
+        float M = lane < n_warps ? m_s[lane] : -INFINITY;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+            M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        const float cw = Mg == -INFINITY ? 0.f : exp2f(Mg - M);
+        *reinterpret_cast<float4 *>(&acc_s[warp][4 * lane]) = make_float4(acc.x * cw, acc.y * cw, acc.z * cw, acc.w * cw);
+        if (lane == 0)
+            l_s[warp] = L * cw;
         __syncthreads();
         if (tid < kHeadDim) {
-            float M = m_s[0];
-            for (int w = 1; w < n_warps; ++w)
-                M = fmaxf(M, m_s[w]);
             float a = 0.f, l = 0.f;
-            for (int w = 0; w < n_warps; ++w) {
-                const float c = m_s[w] == -INFINITY ? 0.f : exp2f(m_s[w] - M);
-                a += acc_s[w][tid] * c;
-                l += l_s[w] * c;
+            for (int w = 0; w < n_warps; ++w) {          // warp order
+                a += acc_s[w][tid];
+                l += l_s[w];
             }
             const float ov = a / l;
             const bf16 hi = __float2bfloat16_rn(ov);
