@@ -123,13 +123,16 @@ __device__ __forceinline__ void epilogue_qkv(const EpilogueArgs &e, int pos, int
     }
 }
 
-// Apply the epilogue to one pair of fp32 results of batch row b (b_local = b - b0 indexes the tables).
-__device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, const EpilogueTables &tab, int b_local,
-                                               bool tensor_path, int N, int b, int pair, float v0, float v1)
+// Apply the epilogue KIND to one pair of fp32 results of batch row b (b_local = b - b0 indexes the
+// tables).  The kind is a template argument so that a kernel instantiated for one kind carries only
+// that kind's instructions.
+template <int KIND>
+__device__ __forceinline__ void apply_epilogue_t(const EpilogueArgs &e, const EpilogueTables &tab, int b_local,
+                                                 bool tensor_path, int N, int b, int pair, float v0, float v1)
 {
     int n0, n1;
-    pair_coords(e.kind, tensor_path, pair, n0, n1);
-    if (e.kind == EPI_PLAIN) {
+    pair_coords(KIND, tensor_path, pair, n0, n1);
+    if constexpr (KIND == EPI_PLAIN) {
         if (tensor_path) {
             // the pair's outputs are neighbours: one store per buffer
             const size_t o = (size_t)b * N + n0;
@@ -153,7 +156,7 @@ __device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, const Epil
             e.out_f32[(size_t)b * N + n0] = v0;
             e.out_f32[(size_t)b * N + n1] = v1;
         }
-    } else if (e.kind == EPI_SWIGLU) {
+    } else if constexpr (KIND == EPI_SWIGLU) {
         // silu by the fast exponential and division (a few ulp; for v0 < -87 the quotient flushes to 0,
         // its true size being < 1e-36)
         const float a = __fdividef(v0, 1.f + __expf(-v0)) * v1;
@@ -163,15 +166,27 @@ __device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, const Epil
         epilogue_qkv(e, pos, b, n0, n1, v0, v1, rope_trig(e, tab, pos, n0, n1));
     }
 }
+// The same with the kind read from the arguments.
+__device__ __forceinline__ void apply_epilogue(const EpilogueArgs &e, const EpilogueTables &tab, int b_local,
+                                               bool tensor_path, int N, int b, int pair, float v0, float v1)
+{
+    if (e.kind == EPI_PLAIN)
+        apply_epilogue_t<EPI_PLAIN>(e, tab, b_local, tensor_path, N, b, pair, v0, v1);
+    else if (e.kind == EPI_SWIGLU)
+        apply_epilogue_t<EPI_SWIGLU>(e, tab, b_local, tensor_path, N, b, pair, v0, v1);
+    else
+        apply_epilogue_t<EPI_QKV>(e, tab, b_local, tensor_path, N, b, pair, v0, v1);
+}
 
 // Tensor path, two neighbouring pairs (pair0 even, and pair0 + 1) of batch row b at once:
 // v = (v0, v1) of pair0 then (v0, v1) of pair0 + 1.  Their outputs are neighbours in every output
 // buffer, so each buffer takes one vector store.  cs0 / cs1: the pairs' rotary factors when
 // have_trig (QKV only), else computed here.
-__device__ __forceinline__ void apply_epilogue_quad(const EpilogueArgs &e, const EpilogueTables &tab, int N, int b,
-                                                    int pair0, float4 v, bool have_trig, float2 cs0, float2 cs1)
+template <int KIND>
+__device__ __forceinline__ void apply_epilogue_quad_t(const EpilogueArgs &e, const EpilogueTables &tab, int N, int b,
+                                                      int pair0, float4 v, bool have_trig, float2 cs0, float2 cs1)
 {
-    if (e.kind == EPI_PLAIN) {
+    if constexpr (KIND == EPI_PLAIN) {
         const size_t o = (size_t)b * N + 2 * (size_t)pair0;
         const uint2 packed = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
         if (e.out)
@@ -180,7 +195,7 @@ __device__ __forceinline__ void apply_epilogue_quad(const EpilogueArgs &e, const
             *reinterpret_cast<uint2 *>(reinterpret_cast<bf16 *>(e.out2) + o) = packed;
         if (e.out_f32)
             *reinterpret_cast<float4 *>(e.out_f32 + o) = v;
-    } else if (e.kind == EPI_SWIGLU) {
+    } else if constexpr (KIND == EPI_SWIGLU) {
         const float a0 = __fdividef(v.x, 1.f + __expf(-v.x)) * v.y;
         const float a1 = __fdividef(v.z, 1.f + __expf(-v.z)) * v.w;
         uint32_t hi, lo;

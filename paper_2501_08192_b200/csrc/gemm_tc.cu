@@ -109,6 +109,9 @@ __device__ __forceinline__ void tc_ld_wait(uint32_t (&a)[16], uint32_t (&b)[16])
                  : "memory");
 }
 
+// KIND: the epilogue; PUSH: the split-K hand-over (0 pull, 1 st.async, 2 bulk copies) - template
+// arguments, so that each instantiation carries a single tail and its instructions stay close together.
+template <int KIND, int PUSH>
 __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_constant__ GemmTcParams p)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -146,7 +149,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    if (p.push && threadIdx.x == 0) {
+    if (PUSH && p.splits > 1 && threadIdx.x == 0) {
         // this rank will receive NB / splits columns of every other rank's partial tile
         mbar_init(&push_bar, 1);
         mbar_fence_init();
@@ -154,7 +157,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     }
     tc_fence_before();
     __syncthreads();
-    if (p.push)
+    if (PUSH && p.splits > 1)
         cg::this_cluster().sync();      // every rank's barrier exists before anybody sends; overlaps the weight fetch
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
@@ -229,7 +232,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     // (the iteration order is fixed: column pairs sub, sub + kSubs, ... of this rank's columns):
     // computed here, while the weights stream, instead of in the tail.
     float2 trig[2] = {make_float2(1.f, 0.f), make_float2(1.f, 0.f)};
-    if (warp >= 2 && p.epi.kind == EPI_QKV && p.splits > 1 && p.push == 2) {
+    if (warp >= 2 && KIND == EPI_QKV && p.splits > 1 && PUSH == 2) {
         // (bulk form: a warp's first item is column warp - 2 of this rank's mt * cols (m, column)
         // items, a lane's two pairs are rows 4 * lane .. 4 * lane + 3)
         const int cols = p.NB / p.splits;
@@ -240,7 +243,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             trig[0] = rope_trig(p.epi, tabs, tabs.pos[b], tile * p.mt + m, 2 * lane);
             trig[1] = rope_trig(p.epi, tabs, tabs.pos[b], tile * p.mt + m, 2 * lane + 1);
         }
-    } else if (warp >= 2 && p.epi.kind == EPI_QKV && p.splits > 1 && p.push) {
+    } else if (warp >= 2 && KIND == EPI_QKV && p.splits > 1 && PUSH == 1) {
         const int cols = p.NB / p.splits, hp = cols / 2;
         int m = 0, c2 = sub;
         while (c2 >= hp) { c2 -= hp; ++m; }
@@ -257,12 +260,12 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     // one finished pair of iteration k (k < 2 uses the factors above)
     auto finish_pair = [&](int k, int m, int b, float v0, float v1) {
         const int pair = ((tile * p.mt + m) * kTcTileM + row) >> 1;
-        if (p.epi.kind == EPI_QKV) {
+        if constexpr (KIND == EPI_QKV) {
             const int pos = tabs.pos[b], hd = pair >> 6, i = pair & 63;
             const float2 cs = k == 0 ? trig[0] : (k == 1 ? trig[1] : rope_trig(p.epi, tabs, pos, hd, i));
             epilogue_qkv(p.epi, pos, b, hd, i, v0, v1, cs);
         } else {
-            apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, v0, v1);
+            apply_epilogue_t<KIND>(p.epi, tabs, b, true, p.N, b, pair, v0, v1);
         }
     };
     bool have = false;
@@ -293,7 +296,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         }
     };
 
-    if (p.splits > 1 && p.push == 2) {
+    if (PUSH == 2 && p.splits > 1) {
         // Split-K across the cluster for wide batches, one-sided reduce-scatter by bulk copies: every
         // rank lays its partial tiles out in its own (idle) ring as [m][column][row], then one bulk
         // copy per (owner, m) moves the owner's columns - a contiguous slice - into the owner's receive
@@ -381,7 +384,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                     }
                     const int b = s * cols + cl;
                     if (b < p.B && !bad)
-                        apply_epilogue_quad(p.epi, tabs, p.N, b, (tile * p.mt + m) * (kTcTileM / 2) + 2 * lane, acc, k == 0,
+                        apply_epilogue_quad_t<KIND>(p.epi, tabs, p.N, b, (tile * p.mt + m) * (kTcTileM / 2) + 2 * lane, acc, k == 0,
                                             trig[0], trig[1]);
                     cl += n_ew;
                     while (cl >= cols) { cl -= cols; ++m; }
@@ -395,7 +398,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 finish(std::integral_constant<int, 8>());
         }
         cluster_wait();
-    } else if (p.splits > 1 && p.push) {
+    } else if (PUSH == 1 && p.splits > 1) {
         // Split-K across the cluster, one-sided reduce-scatter: rank q finishes columns [q * cols,
         // (q + 1) * cols).  Every rank stores those columns of its partial tile into rank q's receive
         // area [source rank][m][row][cols] (st.async, signalling q's barrier with the bytes; its own
@@ -465,7 +468,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             else
                 finish(std::integral_constant<int, 8>());
         }
-    } else if (p.splits > 1) {
+    } else if (PUSH == 0 && p.splits > 1) {
         // Split-K across the cluster, reduce-scatter style: every rank publishes its partial tiles in
         // its own shared memory, then finishes NB / splits of the batch columns - reading that slice
         // from all ranks in rank order - so the reduction and the epilogue work are spread over the
@@ -529,7 +532,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                             const float recv = __shfl_xor_sync(0xffffffffu, par ? mine[0] : mine[1], 1);
                             const int b = b0 + par;
                             if (b < p.B && !poisoned)
-                                apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? recv : mine[0], par ? mine[1] : recv);
+                                apply_epilogue_t<KIND>(p.epi, tabs, b, true, p.N, b, pair, par ? recv : mine[0], par ? mine[1] : recv);
                         }
                     }
                 }
@@ -554,7 +557,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 const float recv = __shfl_xor_sync(0xffffffffu, par ? v[i] : v[i + 1], 1);
                 const int b = c * 16 + i + par;
                 if (b < p.B && !poisoned)
-                    apply_epilogue(p.epi, tabs, b, true, p.N, b, pair, par ? recv : v[i], par ? v[i + 1] : recv);
+                    apply_epilogue_t<KIND>(p.epi, tabs, b, true, p.N, b, pair, par ? recv : v[i], par ? v[i + 1] : recv);
             }
         }
     }
@@ -565,6 +568,19 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                      : "memory");
     }
     trace_end(p.trace);
+}
+
+template <int KIND, int PUSH>
+static cudaError_t launch_instance(cudaLaunchConfig_t &cfg, const GemmTcParams &p, size_t smem)
+{
+    static size_t attr_smem = 0;        // per instantiation
+    if (smem > attr_smem) {
+        cudaError_t e = cudaFuncSetAttribute(k_gemm_tcgen05<KIND, PUSH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess)
+            return e;
+        attr_smem = smem;
+    }
+    return cudaLaunchKernelEx(&cfg, k_gemm_tcgen05<KIND, PUSH>, p);
 }
 
 cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
@@ -643,13 +659,6 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     size_t smem = (size_t)stages * stage_bytes + recv_alloc + 1024;
     const size_t red_bytes = (size_t)mt * a.NB * kTcTileM * 4 + 1024;
     if (smem < red_bytes) smem = red_bytes;
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemm_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess)
-            return e;
-        attr_smem = smem;
-    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(tiles, splits, 1);
     // epilogue warps: 16 when the CTA has the SM to itself and enough column pairs per thread to share,
@@ -669,7 +678,15 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     }
     cfg.attrs = at;
     cfg.numAttrs = n;
-    return cudaLaunchKernelEx(&cfg, k_gemm_tcgen05, p);
+    const int push = splits > 1 ? p.push : 0;
+#define PRSV_TC_CASE(KIND, PUSH)                                   \
+    if (a.epi.kind == (KIND) && push == (PUSH))                    \
+        return launch_instance<KIND, PUSH>(cfg, p, smem);
+    PRSV_TC_CASE(EPI_PLAIN, 0) PRSV_TC_CASE(EPI_PLAIN, 1) PRSV_TC_CASE(EPI_PLAIN, 2)
+    PRSV_TC_CASE(EPI_QKV, 0) PRSV_TC_CASE(EPI_QKV, 1) PRSV_TC_CASE(EPI_QKV, 2)
+    PRSV_TC_CASE(EPI_SWIGLU, 0) PRSV_TC_CASE(EPI_SWIGLU, 1) PRSV_TC_CASE(EPI_SWIGLU, 2)
+#undef PRSV_TC_CASE
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace prsv
