@@ -38,14 +38,17 @@ struct WindowParams {
     size_t x_plane;
     int H;
     int cluster;         // CTAs per row
+    int resid_f32, part0_f32;   // the residual / partial 0 are fp32 (handed over by an earlier kernel of the step)
     long long *trace;
     int delay_ns;
     int *status;
 };
 
-template <bool RESID_F32, bool PART0_F32>
+// (One instantiation for all four input forms: the two windows of a layer then run the same
+// instructions, which the second finds in the instruction caches.)
 __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_constant__ WindowParams p)
 {
+    const bool RESID_F32 = p.resid_f32 != 0, PART0_F32 = p.part0_f32 != 0;
     const int row = blockIdx.x / p.cluster, rank = blockIdx.x % p.cluster;
     const int chunks = (p.H >> 3) / p.cluster;   // uint4 chunks of this CTA's slice of the row
     const size_t row_off = (size_t)row * (p.H >> 3) + (size_t)rank * chunks;
@@ -274,11 +277,9 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
         ++n_attr;
     }
     cfg.numAttrs = n_attr;
-    if (a.resid_is_f32)
-        return a.part0_is_f32 ? cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<true, true>, p)
-                              : cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<true, false>, p);
-    return a.part0_is_f32 ? cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<false, true>, p)
-                          : cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<false, false>, p);
+    p.resid_f32 = a.resid_is_f32;
+    p.part0_f32 = a.part0_is_f32;
+    return cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm, p);
 }
 
 }  // namespace prsv
