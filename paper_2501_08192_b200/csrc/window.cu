@@ -46,8 +46,13 @@ struct WindowParams {
 
 // (One instantiation for all four input forms: the two windows of a layer then run the same
 // instructions, which the second finds in the instruction caches.)
+// LEAN, for big batches (hundreds of CTAs): one chunk per thread and the step's input buffers are only
+// hinted into L2 before the wait and loaded after it, so that a CTA holds few registers while it
+// waits - the grid then fits beside the early-launched GEMM CTAs in one wave instead of several.
+template <bool LEAN>
 __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_constant__ WindowParams p)
 {
+    constexpr int kWinMaxChunks = LEAN ? 1 : prsv::kWinMaxChunks;
     const bool RESID_F32 = p.resid_f32 != 0, PART0_F32 = p.part0_f32 != 0;
     const int row = blockIdx.x / p.cluster, rank = blockIdx.x % p.cluster;
     const int chunks = (p.H >> 3) / p.cluster;   // uint4 chunks of this CTA's slice of the row
@@ -85,17 +90,31 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
     // previous kernel either: their loads - the only ones that go to HBM - are issued before the
     // wait, up to 8 partial buffers per chunk.
     uint4 pre[kWinMaxChunks][8], pre_res[kWinMaxChunks];
+    auto load_inputs = [&]() {
 #pragma unroll
-    for (int c = 0; c < kWinMaxChunks; ++c) {
-        const int ch = threadIdx.x + c * blockDim.x;
-        if (ch < chunks) {
-            if (!RESID_F32)
-                pre_res[c] = ld_stream(reinterpret_cast<const uint4 *>(p.resid) + row_off + ch);
+        for (int c = 0; c < kWinMaxChunks; ++c) {
+            const int ch = threadIdx.x + c * blockDim.x;
+            if (ch < chunks) {
+                if (!RESID_F32)
+                    pre_res[c] = ld_stream(reinterpret_cast<const uint4 *>(p.resid) + row_off + ch);
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if (j < p.n_parts && !(PART0_F32 && j == 0))
-                    pre[c][j] = ld_stream(p.parts[j] + row_off + ch);
+                for (int j = 0; j < 8; ++j)
+                    if (j < p.n_parts && !(PART0_F32 && j == 0))
+                        pre[c][j] = ld_stream(p.parts[j] + row_off + ch);
+            }
         }
+    };
+    if constexpr (LEAN) {
+        // one hint per 128-byte line (8 threads share a line)
+        if ((threadIdx.x & 7) == 0 && (int)threadIdx.x < chunks) {
+            if (!RESID_F32)
+                line_prefetch_l2(reinterpret_cast<const uint4 *>(p.resid) + row_off + threadIdx.x);
+            for (int j = 0; j < p.n_parts; ++j)
+                if (!(PART0_F32 && j == 0))
+                    line_prefetch_l2(p.parts[j] + row_off + threadIdx.x);
+        }
+    } else {
+        load_inputs();
     }
 
     if (p.cluster > 1)
@@ -104,6 +123,8 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
     pdl_wait();                // this shard's own partial sum comes from the preceding kernel in the stream
     trace_waited(p.trace);
     const long long t_begin = p.delay_ns ? gtime() : 0;   // the modelled collective starts when its inputs exist
+    if constexpr (LEAN)
+        load_inputs();
 
 #pragma unroll
     for (int c = 0; c < kWinMaxChunks; ++c) {
@@ -255,6 +276,7 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
         cl *= 2;
     p.cluster = cl;
     const int chunks = a.H / 8 / cl;
+    const bool lean = a.B * cl > 256 && chunks <= 512;
     int threads = (chunks + kWinMaxChunks - 1) / kWinMaxChunks;
     if (chunks <= 512)
         threads = chunks;
@@ -279,7 +301,8 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
     cfg.numAttrs = n_attr;
     p.resid_f32 = a.resid_is_f32;
     p.part0_f32 = a.part0_is_f32;
-    return cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm, p);
+    return lean ? cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<true>, p)
+                : cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<false>, p);
 }
 
 }  // namespace prsv
