@@ -70,6 +70,10 @@ SMALL = [
     I.small_shape(name="h384_b7", batch=7, hidden=384, ffn=224, ctx=33, seed=49),
     # window rows split over a cluster of CTAs
     I.small_shape(name="h2048_b3", batch=3, hidden=2048, ffn=256, ctx=40, tp_degree=5, seed=50),
+    # 40 rows x 8 CTAs: the window kernel's big-batch form (inputs loaded after the wait); tensor path with a
+    # 48-column batch tile, two weight tiles per CTA and the bulk split-K hand-over
+    I.small_shape(name="h8192_b40", batch=40, hidden=8192, ffn=256, ctx=50, ctx_min=3, n_q_heads=2, n_kv_heads=2,
+                  tp_degree=3, seed=57),
 ]
 
 
