@@ -209,10 +209,16 @@ PRESERVE_API int preserve_decode_chain(preserve_layer_t *const *layers, int32_t 
                           int32_t link, void *cuda_stream);
 
 /* The step with host activation buffers (see preserve_host_io_t).  When every
- * input buffer is pinned (page-locked) host memory, the window kernels read the
- * inputs directly from host memory (that read is the host-to-device transfer);
- * otherwise the inputs are first copied into a device staging area.  The two
- * outputs are copied back from device memory at the end. */
+ * input buffer is pinned (page-locked) host memory, one gather kernel on a
+ * stream owned by the layer reads the inputs over PCIe into the layer's device
+ * staging area (that read is the host-to-device transfer) while whatever was
+ * queued on `cuda_stream` before this call is still running, and the step
+ * waits only for that gather; pinned output buffers are written directly by
+ * the kernels that produce the results.  Pageable buffers are copied with
+ * copy calls on `cuda_stream` instead.  As with every entry point the results
+ * are complete once the work queued on `cuda_stream` has completed.  Calls on
+ * one layer share its staging area: the gather of a call starts when the step
+ * of the previous call on that layer has finished. */
 PRESERVE_API int preserve_decode_step_host(preserve_layer_t *layer, const preserve_host_io_t *io, void *cuda_stream);
 
 /* Per-kernel device times of one step.  Runs the step with direct launches on

@@ -108,6 +108,9 @@ struct preserve_layer {
 
     cudaStream_t side;
     cudaEvent_t ev_a, ev_b, ev_join;
+    cudaStream_t xfer;           // host-buffer entry point: the stream the input gather runs on
+    cudaEvent_t ev_in_ready, ev_in_free;
+    bool in_free_valid;
     bool side_pending;           // prefetch work queued on the side stream and not yet joined
     bool no_early;               // ablation: prefetch into L2 only, no early launch of the consumer kernels
     int window_delay_ns;         // modelled extra duration of each communication window
@@ -751,6 +754,9 @@ void preserve_layer_destroy(preserve_layer_t *L)
     if (L->ev_b) cudaEventDestroy(L->ev_b);
     if (L->ev_join) cudaEventDestroy(L->ev_join);
     if (L->side) cudaStreamDestroy(L->side);
+    if (L->xfer) { cudaStreamSynchronize(L->xfer); cudaStreamDestroy(L->xfer); }
+    if (L->ev_in_ready) cudaEventDestroy(L->ev_in_ready);
+    if (L->ev_in_free) cudaEventDestroy(L->ev_in_free);
     delete L;
 }
 
@@ -919,6 +925,15 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     CKI(cudaEventCreateWithFlags(&L->ev_a, cudaEventDisableTiming));
     CKI(cudaEventCreateWithFlags(&L->ev_b, cudaEventDisableTiming));
     CKI(cudaEventCreateWithFlags(&L->ev_join, cudaEventDisableTiming));
+    {
+        // highest priority: its few CTAs take the first slots that free up beside the main stream's kernels
+        int prio_lo = 0, prio_hi = 0;
+        CKI(cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi));
+        CKI(cudaStreamCreateWithPriority(&L->xfer, cudaStreamNonBlocking, prio_hi));
+    }
+    CKI(cudaEventCreateWithFlags(&L->ev_in_ready, cudaEventDisableTiming));
+    CKI(cudaEventCreateWithFlags(&L->ev_in_free, cudaEventDisableTiming));
+    L->in_free_valid = false;
     for (int i = 0; i <= PRESERVE_N_KERNELS; ++i)
         CKI(cudaEventCreate(&L->prof[i]));
     CKI(cudaDeviceSynchronize());
@@ -1007,10 +1022,12 @@ int preserve_decode_step_host(preserve_layer_t *L, const preserve_host_io_t *io,
         if (!io->attn_peer_partials[i])
             return PRESERVE_EINVAL;
 
-    // Pinned (page-locked) host buffers are visible to the device: the window kernels then read the
-    // step's inputs straight from host memory - that read IS the host-to-device transfer - instead
-    // of 2P + 1 separate copy calls followed by a second read from device memory.  Pageable buffers
-    // take the staged path.
+    // Pinned (page-locked) host buffers are visible to the device: one gather kernel on the layer's
+    // transfer stream reads them over PCIe into the staging area - that read IS the host-to-device
+    // transfer - while the kernels of the call before this one are still running on `s`; the step
+    // then reads device memory.  (2P + 1 separate copy calls would cost more host time than a small
+    // layer runs, and window kernels reading host memory themselves put the PCIe latency on the
+    // critical path.)  Pageable buffers take the copy-call path.
     auto device_view = [](const void *hp) -> const void * {
         cudaPointerAttributes at;
         if (cudaPointerGetAttributes(&at, hp) != cudaSuccess) {
@@ -1022,32 +1039,44 @@ int preserve_decode_step_host(preserve_layer_t *L, const preserve_host_io_t *io,
             return nullptr;
         return at.devicePointer;
     };
-    bool direct = true;
+    const int n_bufs = 2 * c.tp_degree;      // P partials, P - 1 peers, residual
+    const void *views[2 * kMaxParts + 1];
+    void *slots[2 * kMaxParts + 1];
+    bool direct = BH2 % 16 == 0;
+    for (int i = 0; i < n_bufs; ++i)
+        slots[i] = L->stage_in + (size_t)i * slot;
     for (int i = 0; i < c.tp_degree && direct; ++i)
-        direct = (dparts[i] = device_view(io->partials_in[i])) != nullptr;
+        direct = (views[i] = device_view(io->partials_in[i])) != nullptr;
     for (int i = 0; i + 1 < c.tp_degree && direct; ++i)
-        direct = (dpeers[i] = device_view(io->attn_peer_partials[i])) != nullptr;
-    const void *dres = direct ? device_view(io->residual_in) : nullptr;
-    const void *dctx = direct && dres ? device_view(io->ctx_len_host) : nullptr;
-    direct = direct && dres;
-    if (!direct) {
-        for (int i = 0; i < c.tp_degree; ++i) {
-            CK(L, cudaMemcpyAsync(L->stage_in + (size_t)i * slot, io->partials_in[i], BH2, cudaMemcpyHostToDevice, s));
-            dparts[i] = L->stage_in + (size_t)i * slot;
-        }
-        for (int i = 0; i + 1 < c.tp_degree; ++i) {
-            uint8_t *dst = L->stage_in + (size_t)(c.tp_degree + i) * slot;
-            CK(L, cudaMemcpyAsync(dst, io->attn_peer_partials[i], BH2, cudaMemcpyHostToDevice, s));
-            dpeers[i] = dst;
-        }
-        uint8_t *dst = L->stage_in + (size_t)(2 * c.tp_degree - 1) * slot;
-        CK(L, cudaMemcpyAsync(dst, io->residual_in, BH2, cudaMemcpyHostToDevice, s));
-        dres = dst;
+        direct = (views[c.tp_degree + i] = device_view(io->attn_peer_partials[i])) != nullptr;
+    if (direct)
+        direct = (views[2 * c.tp_degree - 1] = device_view(io->residual_in)) != nullptr;
+    const void *dctx_view = direct ? device_view(io->ctx_len_host) : nullptr;
+    if (dctx_view && (reinterpret_cast<uintptr_t>(dctx_view) & 3))
+        dctx_view = nullptr;
+    // the staging area is free again once the previous call's step has read it
+    if (L->in_free_valid)
+        CK(L, cudaStreamWaitEvent(direct ? L->xfer : s, L->ev_in_free, 0));
+    if (direct) {
+        CK(L, launch_stage_inputs(views, slots, n_bufs, BH2, static_cast<const int *>(dctx_view), L->ctx_dev,
+                                  dctx_view ? io->batch : 0, L->xfer));
+        CK(L, cudaEventRecord(L->ev_in_ready, L->xfer));
+        CK(L, cudaStreamWaitEvent(s, L->ev_in_ready, 0));
+    } else {
+        for (int i = 0; i < c.tp_degree; ++i)
+            CK(L, cudaMemcpyAsync(slots[i], io->partials_in[i], BH2, cudaMemcpyHostToDevice, s));
+        for (int i = 0; i + 1 < c.tp_degree; ++i)
+            CK(L, cudaMemcpyAsync(slots[c.tp_degree + i], io->attn_peer_partials[i], BH2, cudaMemcpyHostToDevice, s));
+        CK(L, cudaMemcpyAsync(slots[2 * c.tp_degree - 1], io->residual_in, BH2, cudaMemcpyHostToDevice, s));
     }
-    if (!dctx || (reinterpret_cast<uintptr_t>(dctx) & 3)) {
+    if (!direct || !dctx_view)
         CK(L, cudaMemcpyAsync(L->ctx_dev, io->ctx_len_host, (size_t)io->batch * 4, cudaMemcpyHostToDevice, s));
-        dctx = L->ctx_dev;
-    }
+    for (int i = 0; i < c.tp_degree; ++i)
+        dparts[i] = slots[i];
+    for (int i = 0; i + 1 < c.tp_degree; ++i)
+        dpeers[i] = slots[c.tp_degree + i];
+    const void *dres = slots[2 * c.tp_degree - 1];
+    const void *dctx = L->ctx_dev;
 
     preserve_step_io_t dio = {};
     dio.batch = io->batch;
@@ -1058,14 +1087,23 @@ int preserve_decode_step_host(preserve_layer_t *L, const preserve_host_io_t *io,
     dio.residual_in = dres;
     dio.k_cache = io->k_cache;
     dio.v_cache = io->v_cache;
-    dio.residual_out = L->stage_out;
-    dio.mlp_partial_out = L->stage_out + slot;
+    // Results go straight into the caller's pinned buffers when the device can address them (posted
+    // writes over PCIe from the kernels that produce them); copy calls otherwise.
+    void *out_res = direct ? const_cast<void *>(device_view(io->residual_out)) : nullptr;
+    void *out_mlp = direct ? const_cast<void *>(device_view(io->mlp_partial_out)) : nullptr;
+    const bool direct_out = out_res && out_mlp;
+    dio.residual_out = direct_out ? out_res : L->stage_out;
+    dio.mlp_partial_out = direct_out ? out_mlp : L->stage_out + slot;
     dio.attn_partial_out = nullptr;
     int rc = preserve_decode_step(L, &dio, cuda_stream);
     if (rc)
         return rc;
-    CK(L, cudaMemcpyAsync(io->residual_out, L->stage_out, BH2, cudaMemcpyDeviceToHost, s));
-    CK(L, cudaMemcpyAsync(io->mlp_partial_out, L->stage_out + slot, BH2, cudaMemcpyDeviceToHost, s));
+    CK(L, cudaEventRecord(L->ev_in_free, s));
+    L->in_free_valid = true;
+    if (!direct_out) {
+        CK(L, cudaMemcpyAsync(io->residual_out, L->stage_out, BH2, cudaMemcpyDeviceToHost, s));
+        CK(L, cudaMemcpyAsync(io->mlp_partial_out, L->stage_out + slot, BH2, cudaMemcpyDeviceToHost, s));
+    }
     return PRESERVE_OK;
 }
 

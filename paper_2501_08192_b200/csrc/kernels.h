@@ -147,6 +147,10 @@ struct PrefetchArgs {
     const int *ctx_len;
     int *sink;            // scratch word for the load variant (practically never written)
 };
+// ---- host-buffer entry point: gather of pinned host buffers (device views) into device memory
+cudaError_t launch_stage_inputs(const void *const *src, void *const *dst, int n, size_t bytes_each, const int *ctx_src,
+                                int *ctx_dst, int n_ctx, cudaStream_t s);
+
 void set_prefetch_kernel_mode(int mode, uint32_t chunk_bytes);
 cudaError_t launch_prefetch(const PrefetchArgs &a, int ctas, cudaStream_t s, const cudaLaunchAttribute *attrs,
                             int n_attrs);
