@@ -39,7 +39,7 @@ struct WindowArgs {
     void *x_bf16;                  // bf16 [2][rows][H]: hi plane then lo plane (x = hi + lo)
     size_t x_plane_elems;          // elements between the planes
     int B, H;
-    long long *trace;              // optional timeline slot (4 values), see common.cuh
+    long long *trace;              // optional timeline slot (kTraceSlots values), see common.cuh
     int delay_ns;                  // modelled communication latency added to the window (0 = none)
     int *status;                   // device error word (bounded waits report here)
 };
