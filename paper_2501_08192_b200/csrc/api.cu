@@ -331,7 +331,8 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
         // Prefetching on: the gate/up projection fills both CTA slots of most SMs, so most CTAs of the
         // down projection start only when it ends and would fetch their first tiles from idle HBM
         // after that; the gate/up CTAs request them into L2 as soon as their own stream is over.
-        if (which == 2 && L->budget > 0 && !L->no_early && L->wbytes[3] <= L->l2_bytes / 4) {
+        // (Not when a single kernel is run alone for timing: nothing would consume the bytes.)
+        if (which == 2 && L->only < 0 && L->budget > 0 && !L->no_early && L->wbytes[3] <= L->l2_bytes / 4) {
             a.next_w = L->arena + L->off[3];
             a.next_bytes = (size_t)L->wbytes[3];
         }
