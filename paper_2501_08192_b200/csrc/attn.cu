@@ -8,10 +8,11 @@
 // (sequence, kv head) is one contiguous run and a tile of 64 keys is two TMA
 // boxes of 64 x 64 bf16 (128-byte swizzle) per tensor.
 //
-// Persistent CTAs (one per SM while the whole cache fits a few ring fills, so that
-// the kernels before and after can be co-resident; two per SM for long caches) walk
-// a static list of work items = (sequence, kv head, run of `tiles_per_item` tiles)
-// in address order.  Warp 4 is the producer: one lane issues the TMA loads into a
+// Persistent CTAs walk a static list of work items = (sequence, kv head, run of
+// `tiles_per_item` tiles) in address order.  A short cache is cut into items of at most
+// one ring fill, one per CTA, so every tile is in shared memory before the queries exist;
+// otherwise one CTA per SM while the cache is a few ring fills (the kernels before and
+// after can then be co-resident), two per SM for long caches (plan_attention).  Warp 4 is the producer: one lane issues the TMA loads into a
 // 3-stage ring guarded by full/empty mbarriers (all waits bounded).  Warps 0-3 each
 // own 16 of a tile's 64 keys: S = Q K^T with mma.sync (Q rows = query heads padded
 // to 16, from registers; K via ldmatrix), online softmax in fp32 with exp2,

@@ -13,9 +13,13 @@
 //   warp 1    : allocates TMEM, issues tcgen05.mma (kind::f16, bf16 in, fp32
 //               accumulate in TMEM), tcgen05.commit frees ring slots
 //   warps 2.. : epilogue (8 or 16 warps) - tcgen05.ld the accumulator (lane = output row; the warps of
-//               a TMEM lane group share the columns), split-K
-//               reduction through distributed shared memory of the cluster in rank
-//               order, fused epilogue (epilogue.cuh)
+//               a TMEM lane group share the column chunks), split-K reduction across the cluster as a
+//               one-sided reduce-scatter in rank order (every rank finishes NB / splits columns:
+//               st.async pieces for narrow batches, bulk shared-memory copies for wide ones; reads
+//               through distributed shared memory only where the receive area does not fit), fused
+//               epilogue (epilogue.cuh)
+// The kernel is instantiated per (epilogue kind, hand-over form): the tail of one instantiation is
+// a few KB of instructions, which matters for a kernel that runs for microseconds.
 // Every mbarrier wait is bounded; a wait that gives up records a status code,
 // poisons the rest of the CTA's work, and the CTA still reaches every barrier
 // and frees its TMEM.
