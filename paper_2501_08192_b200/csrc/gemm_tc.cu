@@ -398,8 +398,10 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 finish(std::integral_constant<int, 2>());
             else if (p.splits == 4)
                 finish(std::integral_constant<int, 4>());
-            else
+            else if (p.splits == 8)
                 finish(std::integral_constant<int, 8>());
+            else
+                finish(std::integral_constant<int, 16>());
         }
         cluster_wait();
     } else if (PUSH == 1 && p.splits > 1) {
@@ -584,6 +586,15 @@ static cudaError_t launch_instance(cudaLaunchConfig_t &cfg, const GemmTcParams &
             return e;
         attr_smem = smem;
     }
+    if (p.splits > 8) {
+        static bool np_set = false;     // per instantiation
+        if (!np_set) {
+            cudaError_t e = cudaFuncSetAttribute(k_gemm_tcgen05<KIND, PUSH>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            if (e != cudaSuccess)
+                return e;
+            np_set = true;
+        }
+    }
     return cudaLaunchKernelEx(&cfg, k_gemm_tcgen05<KIND, PUSH>, p);
 }
 
@@ -624,6 +635,14 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     const int slots = sm_count * per_sm;
     int splits = 1;
     while (splits < 8 && tiles * splits * 2 <= slots && p.kblocks / (splits * 2) >= 2) splits *= 2;
+    // Sixteen ranks (a cluster size the device has to be asked for) when even eight leave half of the
+    // SMs without a CTA; only with the bulk hand-over, whose owners may hold a single column.
+    const size_t need16 = (size_t)mt * a.NB * kTcTileM * 4 / 16 * 15;
+    const bool sixteen = splits == 8 && tiles * 16 <= slots && tiles * 8 * 5 <= sm_count * 3 && p.kblocks / 16 >= 2 &&
+                         a.NB % 16 == 0 &&
+                         (size_t)3 * stage_bytes + need16 + 1024 <= (size_t)(per_sm == 2 ? 108 : 225) * 1024;
+    if (sixteen)
+        splits = 16;
     p.stages = stages;
     p.splits = splits;
     int cols = 32;
@@ -637,7 +656,7 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     const size_t recv_bytes = (size_t)mt * a.NB * kTcTileM * 4;
     const size_t smem_cap = (per_sm == 2 ? 108 : 225) * 1024;
     p.push = 0;
-    if (splits > 1 && recv_bytes <= 16 * 1024) {
+    if (splits > 1 && splits <= 8 && recv_bytes <= 16 * 1024) {
         int st = stages;
         while (st > 3 && (size_t)st * stage_bytes + recv_bytes + 1024 > smem_cap) --st;
         if ((size_t)st * stage_bytes + recv_bytes + 1024 <= smem_cap) {
