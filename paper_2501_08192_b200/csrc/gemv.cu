@@ -17,8 +17,8 @@
 // wait, so weights are already streaming while the previous kernel finishes; only
 // the small activation fragments are loaded after the wait (in bursts, so that
 // their L2 latency is paid once per burst).  Grids never exceed what is
-// co-resident: one CTA per SM when a ring per SM holds the whole matrix, two for
-// larger matrices.
+// co-resident (two CTAs per SM); a projection with few row-block groups is split
+// further along k, which shortens the activation slice every CTA reads after the wait.
 // Two arithmetic variants:
 //   - CUDA cores (batch <= 4): 2 x batch fp32 accumulators per lane, finished by
 //     a warp-shuffle reduction over the four lanes that share a row;
@@ -387,14 +387,15 @@ static cudaError_t launch_variant(GemvParams &p, int sm_count, cudaStream_t s)
     while (wk > 1 && p.kchunks / wk < 2 && p.row_blocks % (2 * RB * kGemvWarps / wk) == 0) wk /= 2;
     p.warps_k = wk;
     p.groups = p.row_blocks / (kGemvWarps / wk * RB);
-    // CTAs per SM: one when a ring per SM holds the whole matrix (it is then in shared memory before
-    // the activations exist, and the rest of the SM stays free for the kernels around); two for
-    // larger matrices, which are a steady stream that needs twice the bytes in flight per SM.
-    const int per_sm = (size_t)p.N * p.K * 2 <= (size_t)sm_count * kGemvSmemBytes ? 1 : 2;
+    // Two CTA slots per SM for every matrix (64 KiB rings, <= 128 registers).  A small projection whose
+    // rows alone give few groups is split further along k instead (QKV of an 8B shard: 24 groups x 8
+    // ranks): each CTA then reads a short slice of the activations after the wait, and that read - not
+    // the weights, which are in the rings by then - is what such a kernel's time consists of.
+    const int slots_total = 2 * sm_count;
     int splits = 1;
-    while (splits < 8 && p.groups * splits * 2 <= sm_count * per_sm && p.kchunks / (wk * splits * 2) >= 2) splits *= 2;
+    while (splits < 8 && p.groups * splits * 2 <= slots_total && p.kchunks / (wk * splits * 2) >= 2) splits *= 2;
     p.splits = splits;
-    int clusters = sm_count * per_sm / p.splits;
+    int clusters = slots_total / p.splits;
     if (clusters > p.groups) clusters = p.groups;
     if (clusters < 1) clusters = 1;
     // ring depth: no deeper than a warp's whole run, so that a small projection leaves the shared
