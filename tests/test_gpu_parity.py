@@ -206,6 +206,25 @@ def test_host_buffer_entry_point_matches_device_path(oracle):
         torch.cuda.synchronize()
         assert np.array_equal(r_out.numpy().view(np.uint16), want["h2"])
         assert np.array_equal(m_out.numpy().view(np.uint16), want["mlp_partial"])
+        # twice in a row on one layer (the second call's gather must wait for the first call's step),
+        # then from pageable buffers (copy calls instead of the gather kernel and the direct stores)
+        for pinned in (True, True, False):
+            dl.k_cache.copy_(G.bits_to_cuda(t["k_cache"]))
+            dl.v_cache.copy_(G.bits_to_cuda(t["v_cache"]))
+            mk = pin if pinned else (lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16).copy()))
+            parts2 = [mk(t["partials_in"][p]) for p in range(shape.tp_degree)]
+            peers2 = [mk(t["attn_peer_partials"][p]) for p in range(shape.tp_degree - 1)]
+            resid2 = mk(t["residual_in"])
+            r2 = torch.zeros((shape.batch, shape.hidden), dtype=torch.int16)
+            m2 = torch.zeros((shape.batch, shape.hidden), dtype=torch.int16)
+            if pinned:
+                r2, m2 = r2.pin_memory(), m2.pin_memory()
+            hio2 = P.make_host_io(dl.cfg, shape.batch, dl.ctx_host, parts2, peers2, resid2, dl.k_cache, dl.v_cache,
+                                  r2, m2)
+            dl.layer.decode_step_host(hio2)
+            torch.cuda.synchronize()
+            assert np.array_equal(r2.numpy().view(np.uint16), want["h2"]), f"pinned={pinned}"
+            assert np.array_equal(m2.numpy().view(np.uint16), want["mlp_partial"]), f"pinned={pinned}"
     finally:
         dl.close()
 
