@@ -2,17 +2,22 @@
 """Benchmark of the decode-layer hot path (one tensor-parallel shard's decode step).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config I]
+    python bench.py --mode timeline --config I      per-kernel timeline of one layer-step
+    python bench.py --mode decode-loop              32-layer chain, contexts advancing every token
+    python bench.py --mode streams                  L2 / HBM streaming-read microbenchmark table
 
-Metric: decode-layer us/step and effective HBM GB/s (weights + KV + activation
-bytes over time), prefetch on vs off.  A "step" is one pass of the whole hot path
-over a rotation of R distinct layer instances of the workload (distinct weight
-arenas and KV-caches, R x (weights + KV) >= 4 x L2), so every layer-step starts
-with a cold L2; per-layer figures are the step's divided by R.
-`value` is the effective GB/s with the library's default prefetch setting and
-inputs resident in HBM; `e2e` is the same metric through the host-buffer entry
-point with host<->device copies inside the timed region.  With --gpus N each rank
-runs an independent shard replica (no data-path collective; weak scaling).
-The reference arm times the CPU oracle on the host cores.
+Metric: decode-layer us/step and effective HBM GB/s (weights + KV + activation bytes over
+time), prefetch on vs off.  A "step" is one pass of the whole hot path over a rotation of R
+distinct layer instances of the workload (distinct weight arenas and KV-caches, R x (weights +
+KV) >= 4 x L2), so every layer-step starts with a cold L2; per-layer figures are the step's
+divided by R.  Without --config all five benchmark configurations run in one invocation: the
+top-level `value` / `config` / `roofline` are those of the largest single-GPU one (configs[3]:
+70B-shaped TP=4 shard, batch 64, ragged contexts), `per_config` carries all five.
+`value` is the effective GB/s with the library's default prefetch setting and inputs resident in
+HBM; `e2e` is the same metric through the host-buffer entry point with host<->device copies
+inside the timed region.  With --gpus N each rank runs an independent shard replica (no
+data-path collective; weak scaling); started without a launcher, bench.py spawns the N ranks
+itself.  The reference arm times the CPU oracle on the host cores.
 """
 from __future__ import annotations
 
@@ -20,6 +25,7 @@ import argparse
 import json
 import math
 import os
+import socket
 import subprocess
 import sys
 import threading
@@ -33,22 +39,16 @@ if ROOT not in sys.path:
 
 METRIC = "decode-layer us/step and effective HBM GB/s (% of roofline), prefetch on vs off"
 SWEEP_FRACS = (0.0, 1 / 16, 1 / 8, 1 / 4, 3 / 8, 1 / 2, 5 / 8, 3 / 4, 7 / 8, 1.0)
+HEADLINE_CONFIG = 3          # the largest single-GPU configuration
+MIN_LAYER_STEPS = 200        # timed layer-steps per setting, whatever --steps says
 
-# DRAM traffic per launch of the dominant kernel from an ncu capture (bytes), keyed by
-# (kernel, workload); see profiles/.  None where no capture exists.
+# DRAM traffic per launch of a kernel from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum),
+# keyed by (kernel, config index): (bytes, the profiles/ file the figure was read from).
 NCU_TRAFFIC = {
-    # profiles/ncu_full_gemv_attn_window_config1_small.md (dram__bytes_read.sum + dram__bytes_write.sum)
-    # gate/up: its own 29.45 MB + the 14.68 MB of down-projection weights that its CTAs prefetch into L2 at the end
-    ("gate_up_proj", 1): 44220000, ("down_proj", 1): 14790000, ("qkv_proj", 1): 6470000, ("o_proj", 1): 4260000,
-    ("attn_splitkv", 1): 16830000, ("attn_merge", 1): 380000, ("window_a", 1): 630000, ("window_b", 1): 760000,
-    # profiles/ncu_full_gemm_tcgen05_config3_small.md, profiles/ncu_full_attn_splitkv_config5.md
-    ("gate_up_proj", 2): 121910000, ("down_proj", 2): 59230000, ("qkv_proj", 2): 21560000, ("o_proj", 2): 16890000,
-    ("attn_splitkv", 4): 542870000,
-}
-NCU_TRAFFIC_NOTE = {
-    ("gate_up_proj", 1): "captured in the layer chain: includes 14.68 MB of the next kernel's weights, prefetched into L2 by "
-                         "this kernel's CTAs once their own stream is over (served from L2 to the down projection: 256 B of "
-                         "DRAM reads there); its own bytes are 29.54 MB, and the kernel timed alone does not prefetch",
+    ("gate_up_proj", 1): (44220000, "profiles/ncu_full_gemv_attn_window_config1_small.md (includes 14.68 MB of the "
+                                    "down projection's weights that this kernel's CTAs prefetch into L2)"),
+    ("gate_up_proj", 2): (121910000, "profiles/ncu_full_gemm_tcgen05_config3_small.md"),
+    ("attn_splitkv", 4): (542870000, "profiles/ncu_full_attn_splitkv_config5.md"),
 }
 
 
@@ -62,7 +62,7 @@ def load_peaks():
 
 
 class ClockSampler(threading.Thread):
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed regions run."""
 
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -96,7 +96,8 @@ class ClockSampler(threading.Thread):
 
 
 def kernel_bytes(s, sum_ctx: int):
-    """Algorithmic bytes per launch of each main-stream kernel (order: binding.KERNEL_NAMES)."""
+    """Algorithmic bytes per launch of each main-stream kernel (order: window A, QKV, split-KV
+    attention, merge, O, window B, gate/up, down).  Their sum is the layer-step's algorithmic bytes."""
     B, H, d, P_ = s.batch, s.hidden, s.head_dim, s.tp_degree
     BH, Bq, Bkv, BF = B * H * 2, B * s.n_q_heads * d * 2, B * s.n_kv_heads * d * 2, B * s.ffn * 2
     wqkv = 2 * H * (s.n_q_heads + 2 * s.n_kv_heads) * d
@@ -104,6 +105,10 @@ def kernel_bytes(s, sum_ctx: int):
     kv = 2 * sum_ctx * s.n_kv_heads * d * 2
     win = (P_ + 1) * BH + H * 2 + 2 * BH
     return [win, wqkv + BH + Bq + 2 * Bkv, kv + Bq, Bq, wo + Bq + BH, win, wgu + BH + BF, wdn + BF + BH]
+
+
+def algorithmic_bytes(s, sum_ctx: int) -> int:
+    return int(sum(kernel_bytes(s, sum_ctx)))
 
 
 def max_over_ranks(ms: float, world: int, device: str = "cuda") -> float:
@@ -127,63 +132,95 @@ def rotation_size(shape, l2_bytes: int) -> int:
     return max(2, math.ceil(4 * l2_bytes / per_layer))
 
 
+def free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return int(s.getsockname()[1])
+
+
+def spawn_command(n_ranks: int, port: int, argv):
+    """The launcher command that starts `n_ranks` ranks of this script on one node."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_ranks}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+
+
+def spawn_ranks(args, argv) -> int:
+    """`python bench.py --gpus N` without a launcher: start the N ranks here, one per GPU."""
+    return subprocess.call(spawn_command(args.gpus, free_port(), argv))
+
+
 # --------------------------------------------------------------------------- ours
-def run_ours(args):
-    import torch
-    import torch.distributed as dist
+class Workload:
+    """R layer instances of one configuration on the device, plus pinned host copies of the step
+    inputs for the end-to-end arm.  Instance 0 holds the configuration's seeded draw; the other
+    instances are distinct device buffers with the same bit patterns (the kernels' timing does not
+    depend on the values; what the rotation needs is distinct addresses)."""
 
-    from paper_2501_08192_b200 import binding as P
-    from paper_2501_08192_b200 import build as B
-    from paper_2501_08192_b200 import inputs as I
-
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
-    torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    B.build()
-    from dataclasses import replace
-    shape = replace(I.CONFIGS[args.config], seed=I.CONFIGS[args.config].seed + 1000 * rank)
-    l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size
-    R = args.rotation or rotation_size(shape, l2)
-
-    def to_dev(bits):
-        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
-
-    rng = np.random.Generator(np.random.PCG64(shape.seed))
-    layers, ios, keep, hios = [], [], [], []
-    cfg = P.make_config(shape)
-    for _ in range(R):
+    def __init__(self, P, I, torch, idx: int, rank: int, l2: int, rotation: int = 0, keep_host: bool = False,
+                 flags: int = 0):
+        from dataclasses import replace
+        base = I.CONFIGS[idx]
+        self.shape = shape = replace(base, seed=base.seed + 1000 * rank)
+        self.R = R = rotation or rotation_size(shape, l2)
+        self.cfg = cfg = P.make_config(shape, flags=flags)
+        rng = np.random.Generator(np.random.PCG64(shape.seed))
         t = I.make_layer(shape, rng, nan_fill_tail=False)
+
+        def to_dev(bits):
+            return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+        def pin(a):
+            return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
+
         w = {n: to_dev(t[n]) for n in ("w_q", "w_k", "w_v", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")}
-        L = P.Layer(cfg, w)
-        del w
-        parts = [to_dev(t["partials_in"][p]) for p in range(shape.tp_degree)]
-        peers = [to_dev(t["attn_peer_partials"][p]) for p in range(shape.tp_degree - 1)]
-        resid = to_dev(t["residual_in"])
-        kc, vc = to_dev(t["k_cache"]), to_dev(t["v_cache"])
-        ctx_host = np.ascontiguousarray(t["ctx_len"], np.int32)
-        ctx_dev = torch.from_numpy(ctx_host).cuda()
-        r_out = torch.empty((shape.batch, shape.hidden), dtype=torch.bfloat16, device="cuda")
-        m_out = torch.empty_like(r_out)
-        ios.append(L.make_io(shape.batch, ctx_dev, ctx_host, parts, peers, resid, kc, vc, r_out, m_out))
-        layers.append(L)
-        # pinned host copies for the end-to-end arm
-        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
+        parts0 = [to_dev(t["partials_in"][p]) for p in range(shape.tp_degree)]
+        peers0 = [to_dev(t["attn_peer_partials"][p]) for p in range(shape.tp_degree - 1)]
+        resid0, kc0, vc0 = to_dev(t["residual_in"]), to_dev(t["k_cache"]), to_dev(t["v_cache"])
+        self.ctx_host = np.ascontiguousarray(t["ctx_len"], np.int32)
+        self.sum_ctx = int(self.ctx_host.sum())
         hp = [pin(t["partials_in"][p]) for p in range(shape.tp_degree)]
         hq = [pin(t["attn_peer_partials"][p]) for p in range(shape.tp_degree - 1)]
         hr = pin(t["residual_in"])
-        ho1 = torch.zeros((shape.batch, shape.hidden), dtype=torch.int16).pin_memory()
-        ho2 = torch.zeros((shape.batch, shape.hidden), dtype=torch.int16).pin_memory()
-        hios.append(P.make_host_io(cfg, shape.batch, ctx_host, hp, hq, hr, kc, vc, ho1, ho2))
-        keep.append((t["ctx_len"], ho1, ho2))
-        del t
-    sum_ctx = int(sum(int(x) for x in keep[0][0]))
-    torch.cuda.synchronize()
-    stream = torch.cuda.Stream()
+        self.layers, self.ios, self.hios, self.keep = [], [], [], []
+        for i in range(R):
+            L = P.Layer(cfg, w)
+            c = (lambda x: x) if i == 0 else (lambda x: x.clone())
+            parts, peers = [c(x) for x in parts0], [c(x) for x in peers0]
+            resid, kc, vc = c(resid0), c(kc0), c(vc0)
+            ctx_dev = torch.from_numpy(self.ctx_host).cuda()
+            r_out = torch.empty((shape.batch, shape.hidden), dtype=torch.bfloat16, device="cuda")
+            m_out = torch.empty_like(r_out)
+            self.ios.append(L.make_io(shape.batch, ctx_dev, self.ctx_host, parts, peers, resid, kc, vc, r_out, m_out))
+            self.layers.append(L)
+            ho1 = torch.zeros((shape.batch, shape.hidden), dtype=torch.int16).pin_memory()
+            ho2 = torch.zeros((shape.batch, shape.hidden), dtype=torch.int16).pin_memory()
+            self.hios.append(P.make_host_io(cfg, shape.batch, self.ctx_host, hp, hq, hr, kc, vc, ho1, ho2))
+            self.keep.append((ho1, ho2))
+        del w
+        self.host_tensors = t if keep_host else None
+        self.alg = algorithmic_bytes(shape, self.sum_ctx)
+        torch.cuda.synchronize()
+
+    def set_budget(self, b):
+        for L in self.layers:
+            L.set_prefetch_bytes(b)
+
+    def set_delay(self, ns):
+        for L in self.layers:
+            L.set_window_delay_ns(ns)
+
+    def close(self):
+        for L in self.layers:
+            L.close()
+        self.layers, self.ios, self.hios, self.keep = [], [], [], []
+
+
+def bench_config(P, I, torch, dist, args, idx, rank, local_rank, world, stream, headline: bool):
+    l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size
+    wl = Workload(P, I, torch, idx, rank, l2, args.rotation, keep_host=headline and rank == 0)
+    shape, R, alg = wl.shape, wl.R, wl.alg
+    layers, ios, hios = wl.layers, wl.ios, wl.hios
+    assert alg == int(P.preserve_algorithmic_bytes(wl.cfg, shape.batch, wl.sum_ctx)) > 0
     info = layers[0].get_info()
     default_budget = int(info.prefetch_budget) if args.budget_bytes < 0 else args.budget_bytes
 
@@ -193,13 +230,9 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def set_budget(b):
-        for L in layers:
-            L.set_prefetch_bytes(b)
-
     def time_steps(step_fn, steps, warmup):
-        """Mean ms per step over exactly `steps` steps (events on the launching stream), max over ranks,
-        plus the per-step times of this rank."""
+        """Mean ms per step over exactly `steps` steps (events on the launching stream), max over
+        ranks, plus this rank's per-step times."""
         with torch.cuda.stream(stream):
             for _ in range(warmup):
                 step_fn()
@@ -222,45 +255,42 @@ def run_ours(args):
         for L, h in zip(layers, hios):
             L.decode_step_host(h, stream)
 
-    alg = int(P.preserve_algorithmic_bytes(cfg, shape.batch, sum_ctx))
-    assert alg > 0
+    n_min = max(3, math.ceil(MIN_LAYER_STEPS / R))          # chain steps that make up >= 200 layer-steps
+    n_short = max(3, math.ceil(MIN_LAYER_STEPS / 2 / R))
+    us = lambda ms: ms * 1e3 / R
+    gbs = lambda ms: alg * R / (ms * 1e-3) / 1e9
+    pct = lambda per: [round(float(np.percentile(per, q)) * 1e3 / R, 3) for q in (10, 50, 90)]
+    peak, peak_src = load_peaks()
 
-    def set_delay(ns):
-        for L in layers:
-            L.set_window_delay_ns(ns)
-
-    # ---- headline: default prefetch setting, with clocks sampled during the timed region
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    set_budget(default_budget)
+    # ---- default prefetch setting ("on"): exactly --steps steps after --warmup warm-up steps
+    wl.set_budget(default_budget)
     ms_on, per_on = time_steps(chain_step, args.steps, args.warmup)
-    # ---- prefetch off (vanilla execution), early launch only (budget of one byte: nothing planned for
-    # L2), and the sweep over the L2 budget (fewer steps each)
-    set_budget(0)
-    ms_off, per_off = time_steps(chain_step, args.steps, args.warmup)
-    set_budget(1)
-    ms_early, _ = time_steps(chain_step, max(10, args.steps // 2), 3)
-    sweep = []
+    if args.steps < n_min:
+        _, per_on = time_steps(chain_step, n_min, 3)
+    # ---- prefetch off (vanilla execution) and early launch only (a budget of one byte plans nothing for L2)
+    wl.set_budget(0)
+    ms_off, per_off = time_steps(chain_step, n_min, 3)
+    wl.set_budget(1)
+    ms_early, per_early = time_steps(chain_step, n_min, 3)
+    sweep, modelled = [], []
     if not args.no_sweep:
         for f in SWEEP_FRACS:
-            set_budget(int(f * l2))
-            ms, _ = time_steps(chain_step, max(10, args.steps // 4), 3)
-            sweep.append({"frac_of_l2": round(f, 4), "us_per_layer": round(ms * 1e3 / R, 3)})
-    # ---- modelled communication latency added to every window (the single-GPU stand-in has none)
-    modelled = []
-    if not args.no_sweep:
+            wl.set_budget(int(f * l2))
+            ms, _ = time_steps(chain_step, n_short, 3)
+            sweep.append({"frac_of_l2": round(f, 4), "us_per_layer": round(us(ms), 3)})
+        # modelled communication latency added to every window (the single-GPU stand-in has none)
         for delay_us in (10, 20):
-            set_delay(delay_us * 1000)
+            wl.set_delay(delay_us * 1000)
             row = {"window_delay_us": delay_us}
-            for name, b in (("off", 0), ("early_launch_only", 1), ("on", default_budget)):
-                set_budget(b)
-                ms, _ = time_steps(chain_step, max(10, args.steps // 4), 3)
-                row[name + "_us_per_layer"] = round(ms * 1e3 / R, 3)
+            for name, b in (("off", 0), ("early_launch_only", 1), ("on", default_budget), ("on_quarter_l2", l2 // 4)):
+                wl.set_budget(b)
+                ms, _ = time_steps(chain_step, n_short, 3)
+                row[name + "_us_per_layer"] = round(us(ms), 3)
             modelled.append(row)
-        set_delay(0)
+        wl.set_delay(0)
     # ---- end to end through the host-buffer entry point
-    set_budget(default_budget)
-    ms_e2e, _ = time_steps(host_step, args.steps, args.warmup)
+    wl.set_budget(default_budget)
+    ms_e2e, _ = time_steps(host_step, n_min, 3)
     h2d = (2 * shape.tp_degree) * shape.batch * shape.hidden * 2 + shape.batch * 4
     d2h = 2 * shape.batch * shape.hidden * 2
     # ---- per-kernel times: each main-stream kernel alone, launched back to back over the R layer
@@ -282,104 +312,301 @@ def run_ours(args):
             with torch.cuda.graph(g, stream=stream):
                 for _ in range(4):
                     one()
-        ms, _ = time_steps(lambda: g.replay(), 10, 3)
+        ms, _ = time_steps(lambda: g.replay(), max(5, math.ceil(MIN_LAYER_STEPS / (4 * R))), 3)
         kms[k] = ms / (4 * R)
         del g
     status = max(L.last_status() for L in layers)
-    # ---- the read roofline of this GPU, measured live: a pure 128-bit read stream over 1 GiB (HBM)
-    # and over 32 MiB read repeatedly (L2)
-    big = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
-    read_bw = {"hbm_read_gbs": round(P.preserve_measure_read_bandwidth(big, 5, stream), 1),
-               "l2_read_gbs": round(P.preserve_measure_read_bandwidth(big[: 32 << 20], 50, stream), 1)}
-    del big
-    clocks = sampler.summary()      # sampled from before the first timed region to after the last
-
-    peak, peak_src = load_peaks()
-    kb = kernel_bytes(shape, sum_ctx)
-    dom = int(np.argmax(kms))
-    achieved = kb[dom] / (kms[dom] * 1e-3) / 1e9
-    gbs = lambda ms: alg * R / (ms * 1e-3) / 1e9
-    us = lambda ms: ms * 1e3 / R
-    best = min(sweep, key=lambda e: e["us_per_layer"]) if sweep else None
     info = layers[0].get_info()
     n_pf = sum(1 for w in range(2) if sum(info.planned_bytes[w]) > 0)
-    launches_per_layer = len(P.KERNEL_NAMES) + n_pf
-    out = {
-        "metric": METRIC, "value": round(whole_job_gbs(alg, R, ms_on, world), 2), "unit": "GB/s", "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_on, 5),
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 (fp32 accumulate)",
-        "data": "synthetic (seeded N(0,0.02) weights, N(0,1) activations and KV, shapes of the named config)",
-        "config": {"workload": f"configs[{args.config}] {shape.name}: hidden {shape.hidden}, "
-                               f"{shape.n_q_heads}q/{shape.n_kv_heads}kv heads, ffn {shape.ffn}, batch {shape.batch}, "
-                               f"ctx {shape.ctx}, P={shape.tp_degree}",
-                   "layers_per_step": R,
-                   "cold_l2": f"rotation of {R} distinct layer instances per step "
-                              f"({R * (shape.weight_bytes() + 2 * sum_ctx * shape.n_kv_heads * 256) / 1e6:.0f} MB "
-                              f"> 4 x L2 of {l2 / 1e6:.0f} MB); inputs larger than L2, no flush",
-                   "algorithmic_bytes_per_layer": alg,
-                   "prefetch_budget_bytes": default_budget, "plan_mode": "truncate",
-                   "parallelism": f"{world} independent shard replica(s)"},
-        "us_per_layer": round(us(ms_on), 3),
-        "frac_of_nominal_8TBs": round(gbs(ms_on) / 8000.0, 4),
-        "frac_of_measured_copy_bw": round(gbs(ms_on) / peak, 4),
-        "prefetch": {"on_us_per_layer": round(us(ms_on), 3), "off_us_per_layer": round(us(ms_off), 3),
-                     "early_launch_only_us_per_layer": round(us(ms_early), 3),
-                     "on_gbs": round(gbs(ms_on), 1), "off_gbs": round(gbs(ms_off), 1),
-                     "speedup_on_vs_off": round(ms_off / ms_on, 4),
-                     "p10_p50_p90_on_us": [round(float(np.percentile(per_on, q)) * 1e3 / R, 3) for q in (10, 50, 90)],
-                     "p10_p50_p90_off_us": [round(float(np.percentile(per_off, q)) * 1e3 / R, 3) for q in (10, 50, 90)],
-                     "meaning": "off = vanilla execution (budget 0: no early launch, no side stream); "
-                                "early_launch_only = consumer kernels stage operands in shared memory during "
-                                "the window; on = that plus the L2 prefetch kernel at the default budget",
-                     "sweep": sweep, "best": best, "modelled_window": modelled,
-                     "paper_context": "up to 1.6x end to end on 8x Ascend 910B, int8 (another machine; not a target)"},
+
+    kb = kernel_bytes(shape, wl.sum_ctx)
+    dom = int(np.argmax(kms))
+    achieved = kb[dom] / (kms[dom] * 1e-3) / 1e9
+    best = min(sweep, key=lambda e: e["us_per_layer"]) if sweep else None
+    traffic = NCU_TRAFFIC.get((P.KERNEL_NAMES[dom], idx))
+    res = {
+        "config_index": idx, "name": shape.name,
+        "workload": f"configs[{idx}] {shape.name}: hidden {shape.hidden}, {shape.n_q_heads}q/{shape.n_kv_heads}kv heads, "
+                    f"ffn {shape.ffn}, batch {shape.batch}, ctx "
+                    f"{'U[%d,%d]' % (shape.ctx_min, shape.ctx) if shape.ctx_min is not None else shape.ctx}, "
+                    f"P={shape.tp_degree}",
+        "layers_per_step": R, "algorithmic_bytes_per_layer": alg,
+        "cold_l2": f"rotation of {R} distinct layer instances per step "
+                   f"({R * (shape.weight_bytes() + 2 * wl.sum_ctx * shape.n_kv_heads * 256) / 1e6:.0f} MB "
+                   f"> 4 x L2 of {l2 / 1e6:.0f} MB); inputs larger than L2, no flush",
+        "prefetch_budget_bytes": default_budget, "plan_mode": "truncate",
+        "timed_layer_steps_per_setting": n_min * R,
+        "ms_per_step": round(ms_on, 5), "steps": args.steps,
+        "us_per_layer": round(us(ms_on), 3), "gbs": round(gbs(ms_on), 1),
+        "frac_of_measured_copy_bw": round(gbs(ms_on) / peak, 4), "frac_of_nominal_8TBs": round(gbs(ms_on) / 8000.0, 4),
+        "prefetch": {
+            "on_us_per_layer": round(us(ms_on), 3), "off_us_per_layer": round(us(ms_off), 3),
+            "early_launch_only_us_per_layer": round(us(ms_early), 3),
+            "on_gbs": round(gbs(ms_on), 1), "off_gbs": round(gbs(ms_off), 1), "early_gbs": round(gbs(ms_early), 1),
+            "speedup_on_vs_off": round(ms_off / ms_on, 4), "speedup_on_vs_early": round(ms_early / ms_on, 4),
+            "speedup_early_vs_off": round(ms_off / ms_early, 4),
+            "p10_p50_p90_on_us": pct(per_on), "p10_p50_p90_off_us": pct(per_off), "p10_p50_p90_early_us": pct(per_early),
+            "sweep": sweep, "best": best, "modelled_window": modelled},
         "e2e": {"value": round(gbs(ms_e2e) * world, 2), "unit": "GB/s", "us_per_layer": round(us(ms_e2e), 3),
                 "h2d_bytes_per_step": h2d * R, "d2h_bytes_per_step": d2h * R},
-        "gpu_launches": launches_per_layer * R * args.steps,
+        "gpu_launches": (len(P.KERNEL_NAMES) + n_pf) * R * args.steps,
         "kernels_us": {n: round(float(v) * 1e3, 3) for n, v in zip(P.KERNEL_NAMES, kms)},
         "kernels_gbs": {n: round(kb[i] / (float(kms[i]) * 1e-3) / 1e9, 1) for i, n in enumerate(P.KERNEL_NAMES)},
-        "roofline": {"bound": "hbm", "kernel": P.KERNEL_NAMES[dom], "achieved": round(achieved, 1),
-                     "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
-                     "traffic": NCU_TRAFFIC.get((P.KERNEL_NAMES[dom], args.config)),
-                     "traffic_note": NCU_TRAFFIC_NOTE.get((P.KERNEL_NAMES[dom], args.config)), "peak_source": peak_src,
+        "kernels_frac_of_measured": {n: round(kb[i] / (float(kms[i]) * 1e-3) / 1e9 / peak, 3)
+                                     for i, n in enumerate(P.KERNEL_NAMES)},
+        "roofline": {"bound": "hbm", "kernel": P.KERNEL_NAMES[dom], "achieved": round(achieved, 1), "peak": peak,
+                     "unit": "GB/s", "frac": round(achieved / peak, 4),
+                     "traffic": traffic[0] if traffic else None,
+                     "traffic_source": traffic[1] if traffic else None, "peak_source": peak_src,
                      "algorithmic_bytes_per_launch": kb[dom],
                      "how": "kernel launched alone, back to back over the rotation, from a captured graph"},
-        "read_bandwidth": read_bw, "frac_of_measured_read_bw": round(gbs(ms_on) / read_bw["hbm_read_gbs"], 4),
-        "clocks": clocks, "device_status": status,
+        "device_status": status,
     }
+    if headline and rank == 0 and args.cpu_baseline and world == 1:
+        res["cpu_baseline"] = cpu_baseline(shape, wl.host_tensors, alg, budget_s=12.0, idx=idx)
+    wl.close()
+    del wl
+    torch.cuda.empty_cache()
+    return res
+
+
+def measure_streams(P, torch, stream, quick: bool = True):
+    """Single-launch streaming reads: L2-resident sizes and 1 GiB (HBM), by plain loads and by bulk
+    copies into shared memory, at one and two CTAs per SM, and what one SM alone takes in."""
+    sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+    big = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
+    big.zero_()
+    status = torch.zeros(64, dtype=torch.int32, device="cuda")
+    rows = []
+    sizes = [(32 << 20, "l2")] if quick else [(s << 20, "l2") for s in (8, 16, 32, 64, 96)]
+    sizes.append((1 << 30, "hbm"))
+    for nbytes, kind in sizes:
+        target = 8 << 30 if kind == "l2" else 4 << 30          # bytes moved per measurement
+        passes = max(2, target // nbytes)
+        for path, pname in ((0, "ld.global.nc"), (1, "cp.async.bulk")):
+            for per_sm in (1, 2):
+                g = P.preserve_measure_stream(big, nbytes, passes, path, sms * per_sm, 6, 16384, status, stream)
+                rows.append({"buffer_mib": nbytes >> 20, "source": kind, "path": pname, "ctas_per_sm": per_sm,
+                             "gbs": round(g, 1), "gbs_per_sm": round(g / sms, 2)})
+    # one SM alone: a 256 KiB slice read over and over (L2), and 256 MiB read once (HBM)
+    for slice_bytes, passes, kind in ((256 << 10, 1024, "l2"), (256 << 20, 1, "hbm")):
+        for path, pname in ((0, "ld.global.nc"), (1, "cp.async.bulk")):
+            for stages in ((6, 12) if path == 1 else (0,)):
+                g = P.preserve_measure_stream(big, slice_bytes, passes, path, 1, stages or 6, 16384, status, stream)
+                rows.append({"buffer_mib": round(slice_bytes / (1 << 20), 2), "source": kind + " (one CTA on one SM)",
+                             "path": pname + (f" x{stages} stages" if path == 1 else ""), "ctas_per_sm": None,
+                             "gbs": round(g, 1), "gbs_per_sm": round(g, 2)})
+    assert int(status[0].item()) == 0
+    del big
+    return rows
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2501_08192_b200 import build as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.dry_run:
+        # launch plumbing only (CPU, gloo): no kernel runs, nothing is timed
+        if world > 1:
+            dist.init_process_group("gloo")
+        ms = max_over_ranks(1.0 + 0.25 * rank, world, device="cpu")
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "dry_run": True, "n_gpus": world, "ms_per_step": ms,
+                              "value": None, "scaling": "weak"}), flush=True)
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    B.build()
+    from paper_2501_08192_b200 import binding as P
+    from paper_2501_08192_b200 import inputs as I
+    stream = torch.cuda.Stream()
+
+    if args.mode == "timeline":
+        run_timeline(P, I, torch, args, stream)
+        return
+    if args.mode == "decode-loop":
+        run_decode_loop(P, I, torch, args, stream)
+        return
+    if args.mode == "streams":
+        rows = measure_streams(P, torch, stream, quick=False)
+        print(json.dumps({"streams": rows}), flush=True)
+        return
+
+    configs = [args.config] if args.config >= 0 else list(range(len(I.CONFIGS)))
+    head = args.config if args.config >= 0 else HEADLINE_CONFIG
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    # the headline configuration first (its timed region is the one --steps / --warmup describe)
+    order = [head] + [c for c in configs if c != head]
+    per = {}
+    for idx in order:
+        per[idx] = bench_config(P, I, torch, dist, args, idx, rank, local_rank, world, stream, headline=idx == head)
+    streams = measure_streams(P, torch, stream, quick=True) if not args.no_kernels else []
+    clocks = sampler.summary()      # sampled from before the first timed region to after the last
+
+    h = per[head]
+    read_bw = {}
+    for r in streams:
+        if r["ctas_per_sm"] == 2 and r["path"] == "ld.global.nc":
+            read_bw["hbm_read_gbs" if r["source"] == "hbm" else "l2_read_gbs"] = r["gbs"]
+        if r["ctas_per_sm"] == 2 and r["path"] == "cp.async.bulk":
+            read_bw["hbm_bulk_gbs" if r["source"] == "hbm" else "l2_bulk_gbs"] = r["gbs"]
+    out = {
+        "metric": METRIC, "value": round(whole_job_gbs(h["algorithmic_bytes_per_layer"], h["layers_per_step"],
+                                                       h["ms_per_step"], world), 2),
+        "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": h["ms_per_step"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 (fp32 accumulate)",
+        "data": "synthetic (seeded N(0,0.02) weights, N(0,1) activations and KV, shapes of the named config; the "
+                "layer instances of a rotation are distinct device buffers holding the same seeded draw)",
+        "config": {"workload": h["workload"], "layers_per_step": h["layers_per_step"], "cold_l2": h["cold_l2"],
+                   "algorithmic_bytes_per_layer": h["algorithmic_bytes_per_layer"],
+                   "prefetch_budget_bytes": h["prefetch_budget_bytes"], "plan_mode": h["plan_mode"],
+                   "parallelism": f"{world} independent shard replica(s)"},
+        "us_per_layer": h["us_per_layer"], "frac_of_nominal_8TBs": h["frac_of_nominal_8TBs"],
+        "frac_of_measured_copy_bw": h["frac_of_measured_copy_bw"],
+        "prefetch": dict(h["prefetch"], meaning="off = vanilla execution (budget 0: no early launch, no side stream); "
+                         "early_launch_only = the consumer kernels are launched early and stage their leading operand "
+                         "bytes in shared memory during the window (budget of one byte: nothing planned for L2); on = "
+                         "that plus the side-stream L2 prefetch kernel at the library's default budget.  "
+                         "speedup_on_vs_off is therefore mostly the early launch; speedup_on_vs_early is what the L2 "
+                         "prefetch kernel adds",
+                         paper_context="up to 1.6x end to end on 8x Ascend 910B, int8 (another machine; not a target)"),
+        "e2e": h["e2e"], "gpu_launches": h["gpu_launches"],
+        "kernels_us": h["kernels_us"], "kernels_gbs": h["kernels_gbs"], "roofline": h["roofline"],
+        "read_bandwidth": read_bw, "streams": streams, "clocks": clocks, "device_status": h["device_status"],
+        "per_config": [per[i] for i in sorted(per)],
+    }
+    if "cpu_baseline" in h:
+        out["cpu_baseline"] = h.pop("cpu_baseline")
     if rank == 0:
-        if args.cpu_baseline and world == 1:
-            out["cpu_baseline"] = cpu_baseline(args.config, alg, budget_s=12.0)
         print(json.dumps(out), flush=True)
         det = os.path.join(ROOT, "gpurun_out")
         if os.path.isdir(det):
-            with open(os.path.join(det, f"bench_config{args.config}_n{world}.json"), "w") as f:
+            with open(os.path.join(det, f"bench_n{world}.json"), "w") as f:
                 json.dump(out, f, indent=1)
-    for L in layers:
-        L.close()
     if world > 1:
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------ other modes
+def run_timeline(P, I, torch, args, stream):
+    """Per-kernel timeline of one layer-step from the in-kernel global-timer trace, averaged over
+    many cold steps: for each main-stream kernel, when its first CTA started, when the wait on its
+    predecessor returned, when its operand stream ended, when it ended."""
+    idx = args.config if args.config >= 0 else HEADLINE_CONFIG
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    wl = Workload(P, I, torch, idx, 0, l2, args.rotation)
+    if args.budget_bytes >= 0:
+        wl.set_budget(args.budget_bytes)
+    for L in wl.layers:
+        L.set_trace(True)
+    rows = []
+    reps = max(10, args.steps)
+    for rep in range(reps + 3):
+        with torch.cuda.stream(stream):
+            P.preserve_decode_chain(wl.layers, wl.ios, link=False, stream=stream)
+        torch.cuda.synchronize()
+        for li, L in enumerate(wl.layers):
+            tr = L.read_trace()
+            if rep >= 3 and li > 0:          # (layer 0 of a call has no kernel in front of it)
+                rows.append(tr)
+    a = np.array(rows, dtype=np.float64)      # [samples, kernel, slot]
+    names = P.KERNEL_NAMES
+    table = []
+    for k, n in enumerate(names):
+        s0, w0, w1, e1, s1, st, e0 = (a[:, k, j] for j in range(7))
+        prev_end = a[:, k - 1, 3] if k > 0 else None
+        nxt = a[:, k + 1, 2] if k + 1 < len(names) else None
+        table.append({
+            "kernel": n,
+            "start_to_wait_return_us": round(float(np.mean(w1 - s0)) / 1e3, 2),
+            "early_start_before_prev_end_us": round(float(np.mean(prev_end - s0)) / 1e3, 2) if k > 0 else None,
+            "wait_return_after_prev_end_us": round(float(np.mean(w1 - prev_end)) / 1e3, 2) if k > 0 else None,
+            "wait_return_to_stream_end_us": round(float(np.mean(np.where(st > 0, st - w1, 0.0))) / 1e3, 2),
+            "stream_end_to_end_us": round(float(np.mean(np.where(st > 0, e1 - st, e1 - w1))) / 1e3, 2),
+            "wait_return_to_end_us": round(float(np.mean(e1 - w1)) / 1e3, 2),
+            "end_to_next_wait_return_us": round(float(np.mean(nxt - e1)) / 1e3, 2) if nxt is not None else None,
+        })
+    layer_us = float(np.mean(a[:, -1, 3] - a[:, 0, 2])) / 1e3
+    print(json.dumps({"mode": "timeline", "config_index": idx, "name": wl.shape.name, "samples": len(rows),
+                      "budget_bytes": int(wl.layers[0].get_info().prefetch_budget),
+                      "first_wait_return_to_last_end_us": round(layer_us, 2), "kernels": table}), flush=True)
+    wl.close()
+
+
+def run_decode_loop(P, I, torch, args, stream):
+    """A 32-layer model made of configs[1] layers (linked chain: layer i + 1 consumes layer i's
+    results), decoding tokens with every context advancing by one per token, against the same chain
+    replayed with fixed contexts: us per token with prefetch off / early launch only / on, and the
+    number of graphs captured along the way."""
+    idx = args.config if args.config >= 0 else 1
+    n_layers, n_tokens = args.layers, max(args.steps, 64)
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    wl = Workload(P, I, torch, idx, 0, l2, rotation=n_layers)
+    shape = wl.shape
+    # start n_tokens + 8 below the configured context so that the contexts can advance inside the cache
+    start = np.maximum(wl.ctx_host - (n_tokens + 8), 1).astype(np.int32)
+    ctx_host = start.copy()
+    ctx_dev = torch.from_numpy(ctx_host).cuda()
+    ios = []
+    for L, io in zip(wl.layers, wl.ios):
+        k = io._keep
+        ios.append(L.make_io(shape.batch, ctx_dev, ctx_host, k[4], k[5], k[6], k[7], k[8], k[9], k[10]))
+    res = {}
+    for name, b in (("off", 0), ("early_launch_only", 1), ("on", int(wl.layers[0].get_info().prefetch_budget))):
+        wl.set_budget(b)
+        out = {}
+        for advancing in (False, True):
+            ctx_host[:] = start
+            ctx_dev.copy_(torch.from_numpy(start))
+            torch.cuda.synchronize()
+            caps0 = wl.layers[0].graph_captures()
+            with torch.cuda.stream(stream):
+                for _ in range(3):
+                    P.preserve_decode_chain(wl.layers, ios, link=True, stream=stream)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0 = time.perf_counter()
+            with torch.cuda.stream(stream):
+                e0.record(stream)
+                for _ in range(n_tokens):
+                    P.preserve_decode_chain(wl.layers, ios, link=True, stream=stream)
+                    if advancing:
+                        ctx_dev += 1
+                        ctx_host += 1
+                e1.record(stream)
+            torch.cuda.synchronize()
+            wall = (time.perf_counter() - t0) * 1e6 / n_tokens
+            key = "advancing" if advancing else "fixed"
+            out[key + "_us_per_token"] = round(e0.elapsed_time(e1) * 1e3 / n_tokens, 2)
+            out[key + "_host_wall_us_per_token"] = round(wall, 2)
+            out[key + "_graph_captures"] = wl.layers[0].graph_captures() - caps0
+        out["advancing_over_fixed"] = round(out["advancing_us_per_token"] / out["fixed_us_per_token"], 4)
+        res[name] = out
+    status = max(L.last_status() for L in wl.layers)
+    print(json.dumps({"mode": "decode-loop", "layers": n_layers, "tokens": n_tokens,
+                      "workload": f"{n_layers} x configs[{idx}] {shape.name} (linked chain), contexts "
+                                  f"{int(start.min())}..{int(start.max())} advancing by one per token",
+                      "results": res, "device_status": status}), flush=True)
+    wl.close()
+
+
 # ---------------------------------------------------------------------- reference
-def oracle_step_timer(config_idx: int):
-    """Returns (fn, shape, algorithmic bytes): fn() runs the CPU oracle on one layer-step of the workload."""
+def cpu_baseline(shape, t, alg: int, budget_s: float, idx: int):
     from oracle import oracle as O
-    from paper_2501_08192_b200 import binding as P
-    from paper_2501_08192_b200 import inputs as I
     O.build()
-    shape = I.CONFIGS[config_idx]
-    t = I.make_layers(shape, 1, nan_fill_tail=False)[0]
-    sum_ctx = int(t["ctx_len"].sum())
-    try:
-        alg = int(P.preserve_algorithmic_bytes(P.make_config(shape), shape.batch, sum_ctx))
-    except Exception:
-        alg = shape.weight_bytes() + 2 * sum_ctx * shape.n_kv_heads * 256
-    return (lambda: O.layer_step(shape, t)), shape, alg, O.num_threads()
-
-
-def cpu_baseline(config_idx: int, alg: int, budget_s: float):
-    fn, shape, _, threads = oracle_step_timer(config_idx)
+    fn = lambda: O.layer_step(shape, t)
     fn()
     t0 = time.perf_counter()
     n = 0
@@ -389,33 +616,43 @@ def cpu_baseline(config_idx: int, alg: int, budget_s: float):
         if time.perf_counter() - t0 > budget_s or n >= 50:
             break
     dt = (time.perf_counter() - t0) / n
-    return {"value": round(alg / dt / 1e9, 4), "unit": "GB/s", "us_per_layer": round(dt * 1e6, 1), "cores": threads,
-            "kind": "oracle", "sample": f"{n} full layer-steps of configs[{config_idx}] ({shape.name}), "
-                                        f"one layer instance, after one untimed run"}
+    return {"value": round(alg / dt / 1e9, 4), "unit": "GB/s", "us_per_layer": round(dt * 1e6, 1),
+            "cores": O.num_threads(), "kind": "oracle",
+            "sample": f"{n} full layer-steps of configs[{idx}] ({shape.name}), one layer instance, after one untimed run"}
 
 
 def run_reference(args):
+    """The CPU oracle alone, on the host cores: no CUDA library is loaded by this arm."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    fn, shape, alg, threads = oracle_step_timer(args.config)
-    for _ in range(min(args.warmup, 2)):
+    from oracle import oracle as O
+    from paper_2501_08192_b200 import inputs as I
+    O.build()
+    idx = args.config if args.config >= 0 else HEADLINE_CONFIG
+    shape = I.CONFIGS[idx]
+    t = I.make_layers(shape, 1, nan_fill_tail=False)[0]
+    alg = algorithmic_bytes(shape, int(t["ctx_len"].sum()))
+    fn = lambda: O.layer_step(shape, t)
+    warm = min(args.warmup, 2)
+    for _ in range(warm):
         fn()
-    steps = min(args.steps, 20)
-    t0 = time.perf_counter()
-    for _ in range(steps):
+    # each step = one full layer-step; the number of steps is bounded by a time budget
+    steps, t0 = 0, time.perf_counter()
+    while steps < args.steps and (steps < 3 or time.perf_counter() - t0 < 90.0):
         fn()
+        steps += 1
     ms = (time.perf_counter() - t0) * 1e3 / steps
     val = round(alg / (ms * 1e-3) / 1e9, 4)
-    sample = f"each step = one full layer-step of configs[{args.config}] ({shape.name}) on one layer instance"
+    sample = f"each step = one full layer-step of configs[{idx}] ({shape.name}) on one layer instance"
     out = {"impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus,
-           "steps": steps, "warmup": min(args.warmup, 2), "ms_per_step": round(ms, 3), "higher_is_better": True,
+           "steps": steps, "warmup": warm, "ms_per_step": round(ms, 3), "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "fp32 values, fp64 accumulation",
            "data": "synthetic (same seeded inputs as the CUDA arm)",
-           "config": {"workload": f"configs[{args.config}] {shape.name}", "layers_per_step": 1,
+           "config": {"workload": f"configs[{idx}] {shape.name}", "layers_per_step": 1,
                       "algorithmic_bytes_per_layer": alg},
            "us_per_layer": round(ms * 1e3, 1),
-           "cpu_baseline": {"value": val, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
+           "cpu_baseline": {"value": val, "unit": "GB/s", "cores": O.num_threads(), "kind": "oracle", "sample": sample},
            "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
     print(json.dumps(out), flush=True)
@@ -427,19 +664,26 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
-    ap.add_argument("--config", type=int, default=1, help="index into the five benchmark configurations")
+    ap.add_argument("--config", type=int, default=-1,
+                    help="index into the five benchmark configurations (default: all five, configs[3] as the headline)")
+    ap.add_argument("--mode", default="bench", choices=("bench", "timeline", "decode-loop", "streams"))
+    ap.add_argument("--layers", type=int, default=32, help="decode-loop mode: layers of the chain")
     ap.add_argument("--rotation", type=int, default=0, help="layer instances per step (0 = sized from L2)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-kernels", action="store_true", help="skip the isolated per-kernel timing")
     ap.add_argument("--budget-bytes", type=int, default=-1, help="prefetch budget per window (default: the library's)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--dry-run", action="store_true", help="launch plumbing only (CPU, gloo); nothing is timed")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         run_reference(args)
-    else:
-        run_ours(args)
+        return 0
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return spawn_ranks(args, sys.argv[1:])
+    run_ours(args)
+    return 0
 
 
 if __name__ == "__main__":
-    main()
+    sys.exit(main())

@@ -35,7 +35,14 @@
  *     that gave up) is reported by preserve_last_status.
  *   - Results are a pure function of the inputs: they do not depend, bit for
  *     bit, on the prefetch budget or mode.
- *   - A handle is not thread-safe; distinct handles are independent.
+ *   - A handle is not thread-safe; distinct handles are independent (the library keeps
+ *     no mutable process-wide state besides per-device "attribute already set" marks).
+ *   - Buffers of one call: outputs must not overlap each other or the inputs of the same
+ *     layer; the KV-caches of different layers of a call must not overlap.  An input of a
+ *     layer MAY be an output of an earlier layer of the same preserve_decode_chain call
+ *     (layers wired output to input): the library then reads it only after the producer
+ *     has finished.  Inputs written by work queued on the stream BEFORE the call are
+ *     always read after that work.
  *   - The library needs a device of compute capability 10.x and fails with
  *     PRESERVE_EARCH elsewhere; it has no CPU fallback.
  */
@@ -78,6 +85,10 @@ extern "C" {
                                        3/4 of cudaDevAttrMaxPersistingL2CacheSize at init (off by default) */
 #define PRESERVE_FLAG_NO_EARLY_LAUNCH 4u /* ablation: prefetch into L2 only; consumer kernels are not
                                        launched early to stage operands in shared memory              */
+#define PRESERVE_FLAG_FORCE_GEMV   8u  /* use the split-K GEMV kernels whatever max_batch is (each launch
+                                       covers 16 batch rows)                                          */
+#define PRESERVE_FLAG_FORCE_TENSOR 16u /* use the tcgen05 GEMM kernels although max_batch < 16 (needs ffn
+                                       to be a multiple of 128)                                       */
 
 typedef struct preserve_layer preserve_layer_t;   /* opaque, owned by the library */
 
@@ -166,7 +177,8 @@ typedef struct {
  * arena laid out in the order the kernels consume them, allocates workspaces,
  * a side stream and events on the CURRENT device.  The weight pointers may be
  * freed after the call returns.  *out is NULL on failure.
- * The prefetch budget starts at one sixteenth of the device's L2 size, mode PRESERVE_PLAN_TRUNCATE. */
+ * The prefetch budget starts at the library's default (reported by preserve_layer_get_info as
+ * prefetch_budget; see preserve_set_prefetch_bytes), mode PRESERVE_PLAN_TRUNCATE. */
 PRESERVE_API int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer_weights_t *w,
                         preserve_layer_t **out);
 
@@ -181,6 +193,14 @@ PRESERVE_API int preserve_layer_init(const preserve_layer_config_t *cfg, const p
  * K and V in shared memory before they wait for the window's result; (2) a side-stream
  * kernel prefetches the planned byte ranges, up to this limit per window, into L2. */
 PRESERVE_API int preserve_set_prefetch_bytes(preserve_layer_t *layer, size_t bytes_per_window);
+
+/* How the side-stream kernel brings the planned bytes into L2: mechanism 0 =
+ * cp.async.bulk.prefetch.L2 (one instruction per chunk_bytes; the default, with 4096-byte chunks
+ * from 128 CTAs), 1 = prefetch.global.L2 per 128-byte line, 2 = plain loads whose values are
+ * dropped (the control: completion then implies arrival).  chunk_bytes a multiple of 128, at most
+ * 1 MiB; 1 <= ctas <= 1024.  Results never depend on it. */
+PRESERVE_API int preserve_set_prefetch_mechanism(preserve_layer_t *layer, int32_t mechanism, uint32_t chunk_bytes,
+                                                 int32_t ctas);
 
 /* Modelled communication latency: every window kernel additionally waits (bounded, on
  * the GPU's global timer) until `ns` nanoseconds after its start before it delivers its
@@ -251,9 +271,31 @@ PRESERVE_API int preserve_read_trace(preserve_layer_t *layer, int64_t *out);
 /* Sizes, device attributes and the last plan. */
 PRESERVE_API int preserve_layer_get_info(const preserve_layer_t *layer, preserve_info_t *info);
 
-/* Synchronises the device work queued by this handle and returns the device
- * status word: PRESERVE_OK, or PRESERVE_ETIMEOUT if a bounded wait gave up. */
+/* Synchronises the device and returns the layer's device status word: PRESERVE_OK;
+ * PRESERVE_ETIMEOUT if a bounded wait gave up (the step's results are then undefined, the
+ * handle stays usable); PRESERVE_ESHAPE if the device copy of ctx_len described more
+ * attention work than the host copy the step was planned with.  The word keeps the first
+ * failure until preserve_clear_status. */
 PRESERVE_API int preserve_last_status(preserve_layer_t *layer);
+PRESERVE_API int preserve_clear_status(preserve_layer_t *layer);
+
+/* Graphs captured so far by calls whose first (or only) layer is this handle.  Replays of
+ * a cached graph do not count: a decode loop whose contexts advance should see this number
+ * grow only when the attention work split changes (about once per 64 tokens at most). */
+PRESERVE_API int64_t preserve_graph_captures(const preserve_layer_t *layer);
+
+/* Test hooks.  PRESERVE_DEBUG_WAIT_LIMIT_CYCLES: upper limit, in SM clock cycles, on every
+ * bounded device-side wait of this handle's kernels (0 = the built-in limit of 2^31 cycles,
+ * about a second; waits shorter than 2^19 cycles are never cut).  PRESERVE_DEBUG_WITHHOLD:
+ * 0 = off; otherwise ONE producer of one kernel of the next steps withholds ONE issue - 1: a
+ * CTA of the first window's row cluster does not hand over its sum of squares (needs hidden >=
+ * 2048); 2: a warp of the QKV GEMV never fills its first ring slot; 3: a CTA of the tcgen05 QKV
+ * GEMM never fetches its first weight tile; 4: the first attention CTA never fetches one box of
+ * its first tile - so that the consumer's bounded wait runs out, the kernel gives up and returns,
+ * and preserve_last_status reports PRESERVE_ETIMEOUT.  Nothing faults or hangs. */
+#define PRESERVE_DEBUG_WITHHOLD          0
+#define PRESERVE_DEBUG_WAIT_LIMIT_CYCLES 1
+PRESERVE_API int preserve_debug_set(preserve_layer_t *layer, int32_t what, int64_t value);
 
 /* The cudaError_t of the most recent failing CUDA call made for this handle. */
 PRESERVE_API int preserve_last_cuda_error(const preserve_layer_t *layer);
@@ -263,8 +305,11 @@ PRESERVE_API int preserve_last_cuda_error(const preserve_layer_t *layer);
  * rotary embedding, [.., n_q_heads, head_dim]), 3 o (attention output, same shape),
  * 4 x2, 5 a ([.., ffn]).  1..5 are kept internally as two bf16 planes, value =
  * hi + lo, laid out [2][activation_rows][...] (activation_rows from
- * preserve_layer_get_info); the copy delivers that layout as is.  `bytes` must
- * not exceed the buffer's size.  Asynchronous on `cuda_stream`. */
+ * preserve_layer_get_info); the copy delivers that layout as is.  6: uint64 [2][3], the
+ * bytes per node that the prefetch kernels of the last step decided to bring in - the same
+ * walk as preserve_layer_get_info's planned_bytes, evaluated on the device from the device
+ * copy of ctx_len (a window whose host plan is empty launches no kernel and keeps its old
+ * values).  `bytes` must not exceed the buffer's size.  Asynchronous on `cuda_stream`. */
 PRESERVE_API int preserve_debug_copy(preserve_layer_t *layer, int32_t which, void *dst_device, size_t bytes,
                         void *cuda_stream);
 
@@ -301,13 +346,20 @@ PRESERVE_API int preserve_debug_copy(preserve_layer_t *layer, int32_t which, voi
  *
  * First call: the first call on each device looks up the array's device address and sets
  * the kernels' shared-memory limit, which are synchronous set-up steps; make that first
- * call outside any stream capture.  Later calls only queue work on `cuda_stream`. */
+ * call outside any stream capture.  Later calls only queue work on `cuda_stream`.
+ *
+ * Status: the bounded waits of the two kernels report into the first word of the array;
+ * preserve_attention_static_status() waits for the current device and returns PRESERVE_OK,
+ * PRESERVE_ETIMEOUT (a wait gave up: o is undefined) or PRESERVE_ESHAPE (the device ctx_len
+ * described more work than ctx_len_host: the surplus was dropped, nothing was written out
+ * of bounds, o is wrong).  It allocates nothing either. */
 #define PRESERVE_STATIC_SCRATCH_BYTES (8u << 20)
 PRESERVE_API int preserve_attention_static(const void *q_hi, const void *q_lo, const void *k_cache,
                                            const void *v_cache, const int32_t *ctx_len,
                                            const int32_t *ctx_len_host, int32_t batch, int32_t n_q_heads,
                                            int32_t n_kv_heads, int32_t kv_capacity, void *o_hi, void *o_lo,
                                            void *cuda_stream);
+PRESERVE_API int preserve_attention_static_status(void);
 
 /* Read-bandwidth microbenchmark (the read roofline next to the copy-bandwidth figure): streams
  * `bytes` (>= 1 MiB, 16-byte aligned) of the caller's device buffer `reps` times (1..1000) with
@@ -316,6 +368,19 @@ PRESERVE_API int preserve_attention_static(const void *q_hi, const void *q_lo, c
  * allocates nothing. */
 PRESERVE_API int preserve_measure_read_bandwidth(const void *device_buffer, size_t bytes, int32_t reps,
                                                  void *cuda_stream, float *gbs_out);
+
+/* Streaming-read microbenchmark in ONE launch: `ctas` CTAs each walk their own contiguous slice
+ * of the caller's device buffer (128-byte aligned) `passes` times inside the kernel, so launch
+ * ramp and tail are paid once.  A buffer well inside L2 with many passes measures L2; a buffer
+ * several times larger than L2 measures HBM; ctas = 1 measures what one SM can take in.
+ * path 0: 128-bit read-only loads (256 threads, 8 loads in flight each); path 1: bulk async
+ * copies of chunk_bytes (multiple of 1024) into a shared-memory ring with `stages` (1..12) copies
+ * in flight per CTA, stages * chunk_bytes <= 200 KiB.  status_block: 64 zeroed device ints (the
+ * bounded waits of path 1 report there).  Writes GB/s to *gbs_out; synchronises `cuda_stream`;
+ * allocates nothing. */
+PRESERVE_API int preserve_measure_stream(const void *device_buffer, size_t bytes, int32_t passes, int32_t path,
+                                         int32_t ctas, int32_t stages, uint32_t chunk_bytes, int32_t *status_block,
+                                         void *cuda_stream, float *gbs_out);
 
 /* Frees everything the library allocated for the handle (NULL is allowed). */
 PRESERVE_API void preserve_layer_destroy(preserve_layer_t *layer);
@@ -330,6 +395,24 @@ PRESERVE_API const char *preserve_strerror(int code);
  * rounded down to 128 bytes).  Needs no GPU. */
 PRESERVE_API int preserve_plan_window(const uint64_t *node_bytes, int32_t n_nodes, uint64_t budget, int32_t mode,
                          uint64_t *out_bytes);
+
+/* Host-only: Algorithm 1 as a pass over an explicit operator graph (the form the paper gives
+ * it: for every communication operator, a breadth-first walk over its successors up to the next
+ * communication operator or the end of the graph, inserting a prefetch for every MatMul and
+ * SelfAttention node while the running sum of their sizes stays below the budget).
+ * kind[i] is PRESERVE_NODE_*; mem_bytes[i] what a prefetch of node i brings in (weights, or K+V;
+ * ignored for other kinds); successors of node i are succ[succ_off[i] .. succ_off[i+1]).  Writes
+ * one (communication op, node, bytes) triple per inserted prefetch, in insertion order, and their
+ * number to *n_out; PRESERVE_ETOOBIG (with *n_out set) if there are more than max_out.  A layer's
+ * own step plan is this pass applied to the layer's operator chain. */
+#define PRESERVE_NODE_COMM      0
+#define PRESERVE_NODE_MATMUL    1
+#define PRESERVE_NODE_ATTENTION 2
+#define PRESERVE_NODE_OTHER     3
+PRESERVE_API int preserve_plan_graph(int32_t n_nodes, const int32_t *kind, const uint64_t *mem_bytes,
+                                     const int32_t *succ_off, const int32_t *succ, uint64_t budget, int32_t mode,
+                                     int32_t max_out, int32_t *out_comm, int32_t *out_node, uint64_t *out_bytes,
+                                     int32_t *n_out);
 
 /* Host-only: bytes one step must move once (weights + K/V of the cached tokens
  * + activations), the numerator of the effective-bandwidth figure.

@@ -18,7 +18,9 @@ PRESERVE_EINVAL, PRESERVE_EALIGN, PRESERVE_ESHAPE, PRESERVE_ENOMEM = -1, -2, -3,
 PRESERVE_ECUDA, PRESERVE_EARCH, PRESERVE_ETIMEOUT, PRESERVE_ETOOBIG = -5, -6, -7, -8
 STATIC_SCRATCH_BYTES = 8 << 20
 PLAN_WHOLE_NODE, PLAN_TRUNCATE = 0, 1
-FLAG_NO_GRAPH, FLAG_PERSIST_L2, FLAG_NO_EARLY_LAUNCH = 1, 2, 4
+FLAG_NO_GRAPH, FLAG_PERSIST_L2, FLAG_NO_EARLY_LAUNCH, FLAG_FORCE_GEMV, FLAG_FORCE_TENSOR = 1, 2, 4, 8, 16
+DEBUG_WITHHOLD, DEBUG_WAIT_LIMIT_CYCLES = 0, 1
+WITHHOLD_WINDOW, WITHHOLD_GEMV, WITHHOLD_TENSOR, WITHHOLD_ATTENTION = 1, 2, 3, 4
 
 EXPORTS = (
     "preserve_layer_init", "preserve_set_prefetch_bytes", "preserve_set_plan_mode", "preserve_decode_step",
@@ -27,8 +29,10 @@ EXPORTS = (
     "preserve_plan_window", "preserve_algorithmic_bytes", "preserve_profile_step",
     "preserve_run_kernel", "preserve_set_trace", "preserve_read_trace",
     "preserve_set_window_delay_ns", "preserve_attention_static",
-    "preserve_measure_read_bandwidth",
+    "preserve_measure_read_bandwidth", "preserve_set_prefetch_mechanism", "preserve_clear_status",
+    "preserve_graph_captures", "preserve_debug_set", "preserve_attention_static_status", "preserve_plan_graph", "preserve_measure_stream",
 )
+NODE_COMM, NODE_MATMUL, NODE_ATTENTION, NODE_OTHER = 0, 1, 2, 3
 TRACE_SLOTS = 8
 KERNEL_NAMES = ("window_a", "qkv_proj", "attn_splitkv", "attn_merge", "o_proj", "window_b", "gate_up_proj",
                 "down_proj")
@@ -96,6 +100,14 @@ def lib() -> C.CDLL:
         L.preserve_attention_static.argtypes = [C.c_void_p] * 6 + [C.c_int32] * 4 + [C.c_void_p] * 3
         L.preserve_measure_read_bandwidth.argtypes = [C.c_void_p, C.c_size_t, C.c_int32, C.c_void_p,
                                                       C.POINTER(C.c_float)]
+        L.preserve_set_prefetch_mechanism.argtypes = [C.c_void_p, C.c_int32, C.c_uint32, C.c_int32]
+        L.preserve_clear_status.argtypes = [C.c_void_p]
+        L.preserve_graph_captures.argtypes = [C.c_void_p]
+        L.preserve_graph_captures.restype = C.c_int64
+        L.preserve_debug_set.argtypes = [C.c_void_p, C.c_int32, C.c_int64]
+        L.preserve_attention_static_status.argtypes = []
+        L.preserve_measure_stream.argtypes = [C.c_void_p, C.c_size_t, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                              C.c_uint32, C.c_void_p, C.c_void_p, C.POINTER(C.c_float)]
         L.preserve_layer_get_info.argtypes = [C.c_void_p, C.POINTER(Info)]
         L.preserve_last_status.argtypes = [C.c_void_p]
         L.preserve_last_cuda_error.argtypes = [C.c_void_p]
@@ -106,6 +118,10 @@ def lib() -> C.CDLL:
         L.preserve_strerror.restype = C.c_char_p
         L.preserve_plan_window.argtypes = [C.POINTER(C.c_uint64), C.c_int32, C.c_uint64, C.c_int32,
                                            C.POINTER(C.c_uint64)]
+        L.preserve_plan_graph.argtypes = [C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_uint64),
+                                          C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.c_uint64, C.c_int32,
+                                          C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32),
+                                          C.POINTER(C.c_uint64), C.POINTER(C.c_int32)]
         L.preserve_algorithmic_bytes.argtypes = [C.POINTER(LayerConfig), C.c_int32, C.c_uint64]
         L.preserve_algorithmic_bytes.restype = C.c_uint64
         _lib = L
@@ -133,6 +149,27 @@ def preserve_plan_window(node_bytes: Sequence[int], budget: int, mode: int = PLA
     dst = (C.c_uint64 * max(n, 1))()
     _check(lib().preserve_plan_window(src, n, budget, mode, dst), "preserve_plan_window")
     return [int(dst[i]) for i in range(n)]
+
+
+def preserve_plan_graph(kinds: Sequence[int], mem_bytes: Sequence[int], children: Sequence[Sequence[int]],
+                        budget: int, mode: int = PLAN_WHOLE_NODE):
+    """Algorithm 1 over an explicit graph; returns [(comm op, node, bytes), ...] in insertion order."""
+    n = len(kinds)
+    off = [0]
+    flat: List[int] = []
+    for ch in children:
+        flat.extend(ch)
+        off.append(len(flat))
+    k = (C.c_int32 * max(n, 1))(*kinds)
+    m = (C.c_uint64 * max(n, 1))(*mem_bytes)
+    so = (C.c_int32 * (n + 1))(*off)
+    su = (C.c_int32 * max(len(flat), 1))(*flat)
+    cap = max(n * max(1, sum(1 for x in kinds if x == NODE_COMM)), 1)
+    oc, on, ob = (C.c_int32 * cap)(), (C.c_int32 * cap)(), (C.c_uint64 * cap)()
+    cnt = C.c_int32()
+    _check(lib().preserve_plan_graph(n, k, m, so, su, budget, mode, cap, oc, on, ob, C.byref(cnt)),
+           "preserve_plan_graph")
+    return [(int(oc[i]), int(on[i]), int(ob[i])) for i in range(cnt.value)]
 
 
 def make_config(shape, max_batch: Optional[int] = None, max_ctx: Optional[int] = None, flags: int = 0) -> LayerConfig:
@@ -240,6 +277,19 @@ class Layer:
     def last_status(self) -> int:
         return int(lib().preserve_last_status(self.handle))
 
+    def clear_status(self) -> None:
+        _check(lib().preserve_clear_status(self.handle), "preserve_clear_status")
+
+    def graph_captures(self) -> int:
+        return int(lib().preserve_graph_captures(self.handle))
+
+    def set_prefetch_mechanism(self, mechanism: int, chunk_bytes: int = 4096, ctas: int = 128) -> None:
+        _check(lib().preserve_set_prefetch_mechanism(self.handle, mechanism, chunk_bytes, ctas),
+               "preserve_set_prefetch_mechanism")
+
+    def debug_set(self, what: int, value: int) -> None:
+        _check(lib().preserve_debug_set(self.handle, what, value), "preserve_debug_set")
+
     def last_cuda_error(self) -> int:
         return int(lib().preserve_last_cuda_error(self.handle))
 
@@ -260,12 +310,26 @@ def preserve_attention_static(q_hi, q_lo, k_cache, v_cache, ctx_len_dev, ctx_len
                                                n_kv_heads, cap, _ptr(o_hi), _ptr(o_lo), _stream_ptr(stream)))
 
 
+def preserve_attention_static_status() -> int:
+    return int(lib().preserve_attention_static_status())
+
+
 def preserve_measure_read_bandwidth(buf, reps: int = 10, stream=None) -> float:
     """GB/s of a pure 128-bit read stream over the CUDA tensor `buf` (see preserve.h)."""
     out = C.c_float()
     _check(lib().preserve_measure_read_bandwidth(_ptr(buf), buf.numel() * buf.element_size(), reps,
                                                  _stream_ptr(stream), C.byref(out)),
            "preserve_measure_read_bandwidth")
+    return float(out.value)
+
+
+def preserve_measure_stream(buf, n_bytes: int, passes: int, path: int, ctas: int, stages: int = 6,
+                            chunk_bytes: int = 16384, status=None, stream=None) -> float:
+    """GB/s of the single-launch streaming microbenchmark over the first n_bytes of `buf` (see preserve.h).
+    `status`: CUDA int32 tensor of 64 zeros."""
+    out = C.c_float()
+    _check(lib().preserve_measure_stream(_ptr(buf), n_bytes, passes, path, ctas, stages, chunk_bytes, _ptr(status),
+                                         _stream_ptr(stream), C.byref(out)), "preserve_measure_stream")
     return float(out.value)
 
 

@@ -53,11 +53,14 @@ bool make_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// A replayable graph and everything its kernel nodes were captured with: a cached graph is
+// reused only when the whole signature matches word for word (no bare hash).
 struct GraphEntry {
-    uint64_t key;
+    std::vector<uint64_t> sig;
     cudaGraphExec_t exec;
     uint64_t stamp;
 };
+constexpr size_t kMaxCachedGraphs = 32;
 
 }  // namespace
 
@@ -114,7 +117,10 @@ struct preserve_layer {
     bool side_pending;           // prefetch work queued on the side stream and not yet joined
     bool no_early;               // ablation: prefetch into L2 only, no early launch of the consumer kernels
     int window_delay_ns;         // modelled extra duration of each communication window
-    bool pdl_env;                // PRESERVE_PDL=0 switches programmatic dependent launch off entirely
+    int pf_mechanism;            // prefetch kernel: 0 bulk L2 prefetch, 1 per-line hints, 2 plain loads
+    uint32_t pf_chunk;           // bytes per prefetch instruction
+    int inject;                  // test hook (prsv::Inject): one producer withholds one issue
+    uint64_t n_captures;         // graphs captured so far by calls whose first layer is this handle
 
     size_t budget;
     int plan_mode;
@@ -125,6 +131,7 @@ struct preserve_layer {
 
     std::vector<GraphEntry> graphs;
     uint64_t stamp;
+    bool budget_is_default;      // preserve_set_prefetch_bytes has not been called: the library picks per path
 
     // per-kernel timing (preserve_profile_step): events around the main-stream kernels
     long long *trace_buf;        // device [PRESERVE_N_KERNELS][PRESERVE_TRACE_SLOTS] timeline slots, used when tracing
@@ -152,16 +159,6 @@ int cuda_fail(preserve_layer *L, cudaError_t e)
     } while (0)
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
-
-uint64_t fnv1a(uint64_t h, const void *data, size_t n)
-{
-    const uint8_t *p = static_cast<const uint8_t *>(data);
-    for (size_t i = 0; i < n; ++i) {
-        h ^= p[i];
-        h *= 1099511628211ull;
-    }
-    return h;
-}
 
 int validate_config(const preserve_layer_config_t *c)
 {
@@ -248,6 +245,21 @@ struct StepPtrs {
     int resid_f32, part0_f32;      // linked chain: residual_in / parts[0] are the previous layer's fp32 copies
     void *k_cache, *v_cache;
     void *residual_out, *mlp_partial_out, *attn_partial_out;
+    int late_a, late_b;            // an input of window A / B is an output of an earlier layer of the same call:
+                                   // the window reads its inputs only after the dependency wait
+    int first_of_call;             // first layer of a call
+};
+
+// What the host decides for one step before anything is queued (Algorithm 1 per window over the
+// layer's fixed operator list, the attention work split): everything the launches depend on besides
+// the pointers.  Nothing here depends on the VALUES of the sequence lengths except through these
+// few derived numbers, so a decode loop whose contexts advance keeps replaying one graph.
+struct StepPlan {
+    uint64_t planned[2][3];
+    uint64_t kv_bytes, alg_bytes;
+    bool pf_a, pf_b;
+    int pdl;
+    int attn_grid, attn_tpi, attn_items_per_stream;
 };
 
 int check_step(preserve_layer *L, const preserve_step_io_t *io, StepPtrs *sp)
@@ -298,7 +310,7 @@ int check_step(preserve_layer *L, const preserve_step_io_t *io, StepPtrs *sp)
     return PRESERVE_OK;
 }
 
-int launch_gemm(preserve_layer *L, int which, const void *x, int B, const EpilogueArgs &epi, cudaStream_t s,
+int launch_gemm(preserve_layer *L, int which, const void *x, int B, const EpilogueArgs &epi, int pdl, cudaStream_t s,
                 long long *trace)
 {
     const Dims d = layer_dims(L->cfg);
@@ -312,6 +324,8 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
         a.epi = epi;
         a.status = L->status;
         a.trace = trace;
+        a.pdl = pdl;
+        a.inject = L->inject == INJECT_TC_RING && which == 0 ? INJECT_TC_RING : INJECT_NONE;
         CK(L, launch_gemm_tc(a, L->sm_count, s));
         return PRESERVE_OK;
     }
@@ -326,6 +340,8 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
         a.epi = epi;
         a.status = L->status;
         a.trace = trace;
+        a.pdl = pdl;
+        a.inject = L->inject == INJECT_GEMV_RING && which == 0 ? INJECT_GEMV_RING : INJECT_NONE;
         a.next_w = nullptr;
         a.next_bytes = 0;
         // Prefetching on: the gate/up projection fills both CTA slots of most SMs, so most CTAs of the
@@ -341,32 +357,63 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
     return PRESERVE_OK;
 }
 
-// Queue one layer step on `s` (directly, or into an ongoing capture of `s`).
-int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
+// Host planning of one step: Algorithm 1 per window over {Wqkv, KV, Wo} and {Wgate|up, Wdown}, the
+// byte accounting, and the split of the attention work.
+void plan_step(preserve_layer *L, const StepPtrs &sp, StepPlan *pl)
 {
     const auto &c = L->cfg;
-    const int B = sp.batch, H = c.hidden, cap = c.max_ctx + 1;
-    const Dims d = layer_dims(c);
-
-    // ---- plan (host): Algorithm 1 per window over {Wqkv, KV, Wo} and {Wgate|up, Wdown}
+    const int B = sp.batch;
     uint64_t sum_ctx = 0, max_tiles_seq = 0;
     for (int b = 0; b < B; ++b) {
         sum_ctx += (uint64_t)sp.ctx_len_host[b];
         const uint64_t nt = (uint64_t)(sp.ctx_len_host[b] + 1 + 63) / 64;
         max_tiles_seq = nt > max_tiles_seq ? nt : max_tiles_seq;
     }
-    L->kv_bytes = 2 * sum_ctx * c.n_kv_heads * c.head_dim * 2;
-    const uint64_t nodes_a[3] = {L->wbytes[0], L->kv_bytes, L->wbytes[1]};
-    const uint64_t nodes_b[2] = {L->wbytes[2], L->wbytes[3]};
-    plan_window(nodes_a, 3, L->budget, L->plan_mode, L->planned[0]);
-    plan_window(nodes_b, 2, L->budget, L->plan_mode, L->planned[1]);
-    L->planned[1][2] = 0;
-    L->alg_bytes = L->wbytes[0] + L->wbytes[1] + L->wbytes[2] + L->wbytes[3] + L->kv_bytes + activation_bytes(c, B);
+    pl->kv_bytes = 2 * sum_ctx * c.n_kv_heads * c.head_dim * 2;
+    // The layer's operator chain as Algorithm 1 sees it: window A -> Wqkv -> (rotary, append) ->
+    // SelfAttention -> Wo -> window B -> Wgate|up -> (activation) -> Wdown -> next window.
+    {
+        static const int32_t kind[10] = {PRESERVE_NODE_COMM, PRESERVE_NODE_MATMUL, PRESERVE_NODE_OTHER,
+                                         PRESERVE_NODE_ATTENTION, PRESERVE_NODE_MATMUL, PRESERVE_NODE_COMM,
+                                         PRESERVE_NODE_MATMUL, PRESERVE_NODE_OTHER, PRESERVE_NODE_MATMUL,
+                                         PRESERVE_NODE_COMM};
+        static const int32_t succ_off[11] = {0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 9};
+        static const int32_t succ[9] = {1, 2, 3, 4, 5, 6, 7, 8, 9};
+        const uint64_t mem[10] = {0, L->wbytes[0], 0, pl->kv_bytes, L->wbytes[1], 0, L->wbytes[2], 0, L->wbytes[3], 0};
+        static const int slot_of_node[10] = {-1, 0, -1, 1, 2, -1, 0, -1, 1, -1};
+        std::vector<PlanHit> hits;
+        plan_graph(10, kind, mem, succ_off, succ, L->budget, L->plan_mode, hits);
+        memset(pl->planned, 0, sizeof(pl->planned));
+        for (const PlanHit &h : hits)
+            pl->planned[h.comm == 0 ? 0 : 1][slot_of_node[h.node]] = h.bytes;
+    }
+    pl->alg_bytes = L->wbytes[0] + L->wbytes[1] + L->wbytes[2] + L->wbytes[3] + pl->kv_bytes + activation_bytes(c, B);
     // budget 0 = vanilla execution: every kernel starts after its predecessor has completed and
     // nothing is fetched ahead of the dependency
-    g_pdl = (L->budget > 0 && !L->no_early && L->pdl_env) ? 1 : 0;
-    const bool pf_a = L->only < 0 && L->planned[0][0] + L->planned[0][1] + L->planned[0][2] > 0;
-    const bool pf_b = L->only < 0 && L->planned[1][0] + L->planned[1][1] > 0;
+    pl->pdl = (L->budget > 0 && !L->no_early) ? 1 : 0;
+    pl->pf_a = L->only < 0 && pl->planned[0][0] + pl->planned[0][1] + pl->planned[0][2] > 0;
+    pl->pf_b = L->only < 0 && pl->planned[1][0] + pl->planned[1][1] > 0;
+    plan_attention(sp.ctx_len_host, B, c.n_kv_heads, L->sm_count, &pl->attn_grid, &pl->attn_tpi);
+    pl->attn_items_per_stream = (int)((max_tiles_seq + pl->attn_tpi - 1) / pl->attn_tpi);
+    // (the merge kernel sizes its CTAs from this, between 4 and 32 warps: clamp here so that the
+    // number that enters the graph signature changes as rarely as the launch does)
+    if (pl->attn_items_per_stream < 4) pl->attn_items_per_stream = 4;
+    if (pl->attn_items_per_stream > 32) pl->attn_items_per_stream = 32;
+}
+
+// Queue one layer step on `s` (directly, or into an ongoing capture of `s`).
+int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool direct, cudaStream_t s)
+{
+    const auto &c = L->cfg;
+    const int B = sp.batch, H = c.hidden, cap = c.max_ctx + 1;
+
+    L->kv_bytes = pl.kv_bytes;
+    L->alg_bytes = pl.alg_bytes;
+    for (int w = 0; w < 2; ++w)
+        for (int j = 0; j < 3; ++j)
+            L->planned[w][j] = pl.planned[w][j];
+    const int pdl = pl.pdl;
+    const bool pf_a = pl.pf_a, pf_b = pl.pf_b;
 #define WANT(k) (L->only < 0 || L->only == (k))
 #define TRACE(k) (L->tracing ? L->trace_buf + PRESERVE_TRACE_SLOTS * (k) : nullptr)
 
@@ -403,39 +450,38 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         pf_attr[0].val.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
         return 1;
     };
+    auto prefetch_base = [&](int window) {
+        PrefetchArgs pa = {};
+        pa.ctx_len = sp.ctx_len;
+        pa.sink = L->status + kStatusSinkWord;
+        pa.plan_out = reinterpret_cast<unsigned long long *>(L->status + kStatusPlanWord) + 3 * window;
+        pa.budget = L->budget;
+        pa.plan_mode = L->plan_mode;
+        pa.mechanism = L->pf_mechanism;
+        pa.chunk = L->pf_chunk;
+        pa.kv_node = -1;
+        return pa;
+    };
 
-    // ---- window A  ||  prefetch {Wqkv, K/V, Wo}
+    // ---- window A  ||  prefetch {Wqkv, K/V, Wo}: the kernel walks the three nodes itself
     if (pf_a) {
         CK(L, cudaEventRecord(L->ev_a, s));
         CK(L, cudaStreamWaitEvent(L->side, L->ev_a, 0));
-        PrefetchArgs pa = {};
-        pa.ctx_len = sp.ctx_len;
-        pa.sink = L->status + 8;
-        int n = 0;
-        if (L->planned[0][0]) {
-            pa.seg[n].base = L->arena + L->off[0];
-            pa.seg[n].bytes = L->planned[0][0];
-            ++n;
-        }
-        if (L->planned[0][1]) {
-            pa.seg[n].base = sp.k_cache;
-            pa.seg[n].base2 = sp.v_cache;
-            pa.seg[n].stride = (uint64_t)cap * kHeadDim * 2;
-            pa.seg[n].bytes = L->planned[0][1];
-            pa.seg[n].count = B * c.n_kv_heads;
-            pa.seg[n].per_seq_tokens = 1;
-            pa.seg[n].ranges_per_seq = c.n_kv_heads;
-            pa.seg[n].token_bytes = kHeadDim * 2;
-            ++n;
-        }
-        if (L->planned[0][2]) {
-            pa.seg[n].base = L->arena + L->off[1];
-            pa.seg[n].bytes = L->planned[0][2];
-            ++n;
-        }
-        pa.n_segs = n;
+        PrefetchArgs pa = prefetch_base(0);
+        pa.n_nodes = 3;
+        pa.node[0].base = L->arena + L->off[0];
+        pa.node[0].bytes = L->wbytes[0];
+        pa.node[1].base = sp.k_cache;
+        pa.node[1].base2 = sp.v_cache;
+        pa.node[2].base = L->arena + L->off[1];
+        pa.node[2].bytes = L->wbytes[1];
+        pa.kv_node = 1;
+        pa.kv_count = B * c.n_kv_heads;
+        pa.kv_ranges_per_seq = c.n_kv_heads;
+        pa.kv_token_bytes = kHeadDim * 2;
+        pa.kv_stride = (uint64_t)cap * kHeadDim * 2;
         // Wqkv and Wo are adjacent in the arena
-        const int na = persist_window(L->off[0], L->planned[0][2] ? L->wbytes[0] + L->planned[0][2] : L->planned[0][0]);
+        const int na = persist_window(L->off[0], L->wbytes[0] + L->wbytes[1]);
         CK(L, launch_prefetch(pa, L->prefetch_ctas, L->side, na ? pf_attr : nullptr, na));
     }
     MARK();   // 0: window A starts
@@ -457,6 +503,13 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         w.trace = TRACE(0);
         w.delay_ns = L->window_delay_ns;
         w.status = L->status;
+        // Launched directly, the first kernel of a call must not start before everything queued on
+        // the stream earlier has finished: it reads its input buffers ahead of the dependency wait,
+        // and an earlier call may still be writing them.  (Inside a graph the launch itself is
+        // ordered after the earlier work.)
+        w.pdl = pdl && !(direct && sp.first_of_call);
+        w.inputs_after_wait = sp.late_a;
+        w.inject = L->inject == INJECT_WINDOW_HANDOVER ? INJECT_WINDOW_HANDOVER : INJECT_NONE;
         CK(L, launch_window(w, s));
     }
     // ---- QKV projection + rotary embedding + KV append
@@ -471,7 +524,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         e.ctx_len = sp.ctx_len;
         e.nq = c.n_q_heads; e.nkv = c.n_kv_heads; e.cap = cap;
         e.inv_freq = c.rope_theta > 0.f ? L->inv_freq : nullptr;
-        int rc = launch_gemm(L, 0, L->x, B, e, s, TRACE(1));
+        int rc = launch_gemm(L, 0, L->x, B, e, pdl, s, TRACE(1));
         if (rc)
             return rc;
     }
@@ -488,14 +541,17 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         a.o_plane = a.q_plane;
         a.ctx_len = sp.ctx_len;
         a.B = B; a.nq = c.n_q_heads; a.nkv = c.n_kv_heads; a.cap = cap;
-        plan_attention(sp.ctx_len_host, B, c.n_kv_heads, L->sm_count, &a.grid, &a.tiles_per_item);
-        a.max_items_per_stream = (int)((max_tiles_seq + a.tiles_per_item - 1) / a.tiles_per_item);
+        a.grid = pl.attn_grid;
+        a.tiles_per_item = pl.attn_tpi;
+        a.max_items_per_stream = pl.attn_items_per_stream;
         a.max_items = L->max_items;
         a.part_o = L->part_o;
         a.part_ml = L->part_ml;
         a.o_out = L->o;
         a.status = L->status;
         a.trace = TRACE(2);
+        a.pdl = pdl;
+        a.inject = L->inject == INJECT_ATTN_RING ? INJECT_ATTN_RING : INJECT_NONE;
         CK(L, launch_attention(a, s));
     }
     // ---- output projection -> this shard's attention partial sum
@@ -506,7 +562,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         e.out = nullptr;
         e.out2 = sp.attn_partial_out;
         e.out_f32 = L->attn_f32;
-        int rc = launch_gemm(L, 1, L->o, B, e, s, TRACE(4));
+        int rc = launch_gemm(L, 1, L->o, B, e, pdl, s, TRACE(4));
         if (rc)
             return rc;
     }
@@ -514,18 +570,13 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
     if (pf_b) {
         CK(L, cudaEventRecord(L->ev_b, s));
         CK(L, cudaStreamWaitEvent(L->side, L->ev_b, 0));
-        PrefetchArgs pa = {};
-        pa.ctx_len = sp.ctx_len;
-        pa.sink = L->status + 8;
-        int n = 0;
-        for (int i = 0; i < 2; ++i)
-            if (L->planned[1][i]) {
-                pa.seg[n].base = L->arena + L->off[2 + i];
-                pa.seg[n].bytes = L->planned[1][i];
-                ++n;
-            }
-        pa.n_segs = n;
-        const int nb_attr = persist_window(L->off[2], L->planned[1][0] + L->planned[1][1]);
+        PrefetchArgs pa = prefetch_base(1);
+        pa.n_nodes = 2;
+        for (int i = 0; i < 2; ++i) {
+            pa.node[i].base = L->arena + L->off[2 + i];
+            pa.node[i].bytes = L->wbytes[2 + i];
+        }
+        const int nb_attr = persist_window(L->off[2], L->wbytes[2] + L->wbytes[3]);
         CK(L, launch_prefetch(pa, L->prefetch_ctas, L->side, nb_attr ? pf_attr : nullptr, nb_attr));
     }
     MARK();   // 5: window B starts
@@ -548,6 +599,8 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         w.trace = TRACE(5);
         w.delay_ns = L->window_delay_ns;
         w.status = L->status;
+        w.pdl = pdl;
+        w.inputs_after_wait = sp.late_b;
         CK(L, launch_window(w, s));
     }
     // ---- gate/up projection + SwiGLU, down projection
@@ -557,7 +610,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         e.kind = EPI_SWIGLU;
         e.out = L->a;
         e.out_plane = (size_t)L->rows * c.ffn;
-        int rc = launch_gemm(L, 2, L->x2, B, e, s, TRACE(6));
+        int rc = launch_gemm(L, 2, L->x2, B, e, pdl, s, TRACE(6));
         if (rc)
             return rc;
     }
@@ -567,7 +620,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
         e.kind = EPI_PLAIN;
         e.out = sp.mlp_partial_out;
         e.out_f32 = L->mlp_f32;
-        int rc = launch_gemm(L, 3, L->a, B, e, s, TRACE(7));
+        int rc = launch_gemm(L, 3, L->a, B, e, pdl, s, TRACE(7));
         if (rc)
             return rc;
     }
@@ -579,7 +632,6 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, cudaStream_t s)
     // read, so nothing on the main stream has to wait for them earlier)
     if (pf_a || pf_b)
         L->side_pending = true;       // joined by run_steps after the last layer
-    (void)d;
     return PRESERVE_OK;
 }
 
@@ -596,65 +648,83 @@ int join_side_streams(preserve_layer *const *layers, int n, cudaStream_t s)
     return PRESERVE_OK;
 }
 
-uint64_t step_key(const preserve_layer *L, const StepPtrs &sp, uint64_t h)
+// Everything the captured kernel nodes of one step depend on: the handle, every pointer, the
+// settings, and the few numbers the host derives from the sequence lengths (whether each window
+// prefetches at all, the attention grid, tiles per work item, merge warps).  The lengths themselves
+// are read by the kernels from device memory and are not part of it.
+void step_signature(const preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, std::vector<uint64_t> &sig)
 {
-    h = fnv1a(h, &L, sizeof(L));
-    h = fnv1a(h, &sp.batch, sizeof(int));
-    h = fnv1a(h, &sp.ctx_len, sizeof(void *));
-    h = fnv1a(h, sp.ctx_len_host, sizeof(int) * sp.batch);
-    h = fnv1a(h, sp.parts, sizeof(void *) * L->cfg.tp_degree);
-    h = fnv1a(h, sp.peers, sizeof(void *) * (L->cfg.tp_degree - 1));
-    const void *ptrs[] = {sp.residual_in, sp.k_cache, sp.v_cache, sp.residual_out, sp.mlp_partial_out,
-                          sp.attn_partial_out};
-    h = fnv1a(h, ptrs, sizeof(ptrs));
-    h = fnv1a(h, &L->budget, sizeof(L->budget));
-    h = fnv1a(h, &L->plan_mode, sizeof(int));
-    h = fnv1a(h, &sp.resid_f32, 2 * sizeof(int));
-    const int tr = L->tracing ? 1 : 0;
-    h = fnv1a(h, &tr, sizeof(int));
-    h = fnv1a(h, &L->window_delay_ns, sizeof(int));
-    return h;
+    auto put = [&](uint64_t v) { sig.push_back(v); };
+    auto putp = [&](const void *p) { sig.push_back((uint64_t)reinterpret_cast<uintptr_t>(p)); };
+    putp(L);
+    put((uint64_t)sp.batch);
+    putp(sp.ctx_len);
+    for (int i = 0; i < L->cfg.tp_degree; ++i)
+        putp(sp.parts[i]);
+    for (int i = 0; i + 1 < L->cfg.tp_degree; ++i)
+        putp(sp.peers[i]);
+    putp(sp.residual_in); putp(sp.k_cache); putp(sp.v_cache);
+    putp(sp.residual_out); putp(sp.mlp_partial_out); putp(sp.attn_partial_out);
+    put((uint64_t)sp.resid_f32 | (uint64_t)sp.part0_f32 << 1 | (uint64_t)sp.late_a << 2 | (uint64_t)sp.late_b << 3 |
+        (uint64_t)(L->tracing ? 1 : 0) << 4 | (uint64_t)pl.pdl << 5 | (uint64_t)(pl.pf_a ? 1 : 0) << 6 |
+        (uint64_t)(pl.pf_b ? 1 : 0) << 7 | (uint64_t)L->inject << 8 | (uint64_t)L->pf_mechanism << 16 |
+        (uint64_t)L->plan_mode << 24);
+    put((uint64_t)L->budget);
+    put((uint64_t)L->window_delay_ns | (uint64_t)L->pf_chunk << 32);
+    put((uint64_t)L->prefetch_ctas);
+    put((uint64_t)pl.attn_grid | (uint64_t)pl.attn_tpi << 32);
+    put((uint64_t)pl.attn_items_per_stream);
 }
 
 // Run `n` steps (already validated) as one replayed graph, or directly.
-int run_steps(preserve_layer *const *layers, const StepPtrs *sps, int n, cudaStream_t s)
+int run_steps(preserve_layer *const *layers, StepPtrs *sps, int n, cudaStream_t s)
 {
     preserve_layer *L0 = layers[0];
-    const bool direct = (L0->cfg.flags & PRESERVE_FLAG_NO_GRAPH) || s == nullptr || s == cudaStreamLegacy;
-    if (direct) {
+    bool direct = (L0->cfg.flags & PRESERVE_FLAG_NO_GRAPH) || s == nullptr || s == cudaStreamLegacy;
+    std::vector<StepPlan> plans((size_t)n);
+    for (int i = 0; i < n; ++i) {
+        sps[i].first_of_call = i == 0;
+        plan_step(layers[i], sps[i], &plans[i]);
+    }
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (!direct) {
+        CK(L0, cudaStreamIsCapturing(s, &cs));
+        // the caller is capturing already: just add our nodes to their graph (the capture orders them
+        // after the caller's earlier nodes, as a graph launch of our own would)
+    }
+    if (direct || cs != cudaStreamCaptureStatusNone) {
         for (int i = 0; i < n; ++i) {
-            int rc = enqueue_step(layers[i], sps[i], s);
+            // (first kernel without the early-launch attribute in both cases: nothing orders it
+            // after the earlier work on the stream, or the caller's earlier nodes, otherwise)
+            int rc = enqueue_step(layers[i], sps[i], plans[i], true, s);
             if (rc)
                 return rc;
         }
         return join_side_streams(layers, n, s);
     }
-    uint64_t key = 1469598103934665603ull;
+    std::vector<uint64_t> sig;
+    sig.reserve((size_t)n * 40 + 2);
+    sig.push_back((uint64_t)reinterpret_cast<uintptr_t>(s));
+    sig.push_back((uint64_t)n);
     for (int i = 0; i < n; ++i)
-        key = step_key(layers[i], sps[i], key);
-    key = fnv1a(key, &s, sizeof(s));
+        step_signature(layers[i], sps[i], plans[i], sig);
     for (auto &g : L0->graphs)
-        if (g.key == key) {
+        if (g.sig == sig) {
             g.stamp = ++L0->stamp;
+            for (int i = 0; i < n; ++i) {      // what get_info reports follows the step, replayed or not
+                preserve_layer *L = layers[i];
+                L->kv_bytes = plans[i].kv_bytes;
+                L->alg_bytes = plans[i].alg_bytes;
+                memcpy(L->planned, plans[i].planned, sizeof(L->planned));
+            }
             CK(L0, cudaGraphLaunch(g.exec, s));
             return PRESERVE_OK;
         }
     // capture
-    cudaStreamCaptureStatus cs;
-    CK(L0, cudaStreamIsCapturing(s, &cs));
-    if (cs != cudaStreamCaptureStatusNone) {
-        // the caller is capturing already: just add our nodes to their graph
-        for (int i = 0; i < n; ++i) {
-            int rc = enqueue_step(layers[i], sps[i], s);
-            if (rc)
-                return rc;
-        }
-        return join_side_streams(layers, n, s);
-    }
     CK(L0, cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal));
     int rc = PRESERVE_OK;
     for (int i = 0; i < n && rc == PRESERVE_OK; ++i)
-        rc = enqueue_step(layers[i], sps[i], s);
+        rc = enqueue_step(layers[i], sps[i], plans[i], false, s);
     if (rc == PRESERVE_OK)
         rc = join_side_streams(layers, n, s);
     cudaGraph_t graph = nullptr;
@@ -671,7 +741,8 @@ int run_steps(preserve_layer *const *layers, const StepPtrs *sps, int n, cudaStr
     cudaGraphDestroy(graph);
     if (e != cudaSuccess)
         return cuda_fail(L0, e);
-    if (L0->graphs.size() >= 16) {
+    ++L0->n_captures;
+    if (L0->graphs.size() >= kMaxCachedGraphs) {
         size_t victim = 0;
         for (size_t i = 1; i < L0->graphs.size(); ++i)
             if (L0->graphs[i].stamp < L0->graphs[victim].stamp)
@@ -679,7 +750,7 @@ int run_steps(preserve_layer *const *layers, const StepPtrs *sps, int n, cudaStr
         cudaGraphExecDestroy(L0->graphs[victim].exec);
         L0->graphs.erase(L0->graphs.begin() + victim);
     }
-    L0->graphs.push_back({key, exec, ++L0->stamp});
+    L0->graphs.push_back({std::move(sig), exec, ++L0->stamp});
     CK(L0, cudaGraphLaunch(exec, s));
     return PRESERVE_OK;
 }
@@ -802,21 +873,14 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     L->max_persist = prop.persistingL2CacheMaxSize;
     L->max_window = prop.accessPolicyMaxWindowSize;
     L->group = cfg->n_q_heads / cfg->n_kv_heads;
-    const char *force = getenv("PRESERVE_FORCE_GEMV");
-    const char *force_tc = getenv("PRESERVE_FORCE_TENSOR");
-    L->tensor_path = (cfg->max_batch >= 16 && !(force && force[0] == '1')) ||
-                     (force_tc && force_tc[0] == '1' && cfg->ffn % 128 == 0);
-    const char *pdl = getenv("PRESERVE_PDL");
-    L->pdl_env = !(pdl && pdl[0] == '0');
+    const bool force_gemv = (cfg->flags & PRESERVE_FLAG_FORCE_GEMV) != 0;
+    const bool force_tc = (cfg->flags & PRESERVE_FLAG_FORCE_TENSOR) != 0 && cfg->ffn % 128 == 0;
+    L->tensor_path = (cfg->max_batch >= 16 && !force_gemv) || force_tc;
     L->no_early = (cfg->flags & PRESERVE_FLAG_NO_EARLY_LAUNCH) != 0;
-    const char *pfm = getenv("PRESERVE_PREFETCH_MODE");
-    const char *pfc = getenv("PRESERVE_PREFETCH_CHUNK");
-    if (pfm || pfc)
-        set_prefetch_kernel_mode(pfm ? atoi(pfm) : 0, pfc ? (uint32_t)atoi(pfc) : 4096u);
-    const char *pfn = getenv("PRESERVE_PREFETCH_CTAS");
-    L->prefetch_ctas = pfn ? atoi(pfn) : 128;
-    if (L->prefetch_ctas < 1)
-        L->prefetch_ctas = 1;
+    L->pf_mechanism = 0;      // measured: bulk L2 prefetch from 128 CTAs disturbs the main stream least
+    L->pf_chunk = 4096;
+    L->prefetch_ctas = 128;
+    L->budget_is_default = true;
     L->budget = (size_t)L->l2_bytes / 16;
     L->plan_mode = PRESERVE_PLAN_TRUNCATE;
 
@@ -948,8 +1012,54 @@ int preserve_set_prefetch_bytes(preserve_layer_t *L, size_t bytes_per_window)
     if (!L)
         return PRESERVE_EINVAL;
     L->budget = bytes_per_window;
+    L->budget_is_default = false;
     return PRESERVE_OK;
 }
+
+int preserve_set_prefetch_mechanism(preserve_layer_t *L, int32_t mechanism, uint32_t chunk_bytes, int32_t ctas)
+{
+    if (!L || mechanism < 0 || mechanism > 2 || chunk_bytes < 128 || chunk_bytes % 128 || chunk_bytes > (1u << 20) ||
+        ctas < 1 || ctas > 1024)
+        return PRESERVE_EINVAL;
+    L->pf_mechanism = mechanism;
+    L->pf_chunk = chunk_bytes;
+    L->prefetch_ctas = ctas;
+    return PRESERVE_OK;
+}
+
+int preserve_debug_set(preserve_layer_t *L, int32_t what, int64_t value)
+{
+    if (!L)
+        return PRESERVE_EINVAL;
+    if (what == PRESERVE_DEBUG_WITHHOLD) {
+        if (value < 0 || value > INJECT_ATTN_RING)
+            return PRESERVE_EINVAL;
+        L->inject = (int)value;
+        return PRESERVE_OK;
+    }
+    if (what == PRESERVE_DEBUG_WAIT_LIMIT_CYCLES) {
+        if (value < 0)
+            return PRESERVE_EINVAL;
+        CK(L, cudaSetDevice(L->dev));
+        CK(L, cudaDeviceSynchronize());
+        long long lim = value;
+        CK(L, cudaMemcpy(L->status + kStatusLimitWord, &lim, sizeof(lim), cudaMemcpyHostToDevice));
+        return PRESERVE_OK;
+    }
+    return PRESERVE_EINVAL;
+}
+
+int preserve_clear_status(preserve_layer_t *L)
+{
+    if (!L)
+        return PRESERVE_EINVAL;
+    CK(L, cudaSetDevice(L->dev));
+    CK(L, cudaDeviceSynchronize());
+    CK(L, cudaMemset(L->status, 0, sizeof(int)));
+    return PRESERVE_OK;
+}
+
+int64_t preserve_graph_captures(const preserve_layer_t *L) { return L ? (int64_t)L->n_captures : -1; }
 
 int preserve_set_window_delay_ns(preserve_layer_t *L, int32_t ns)
 {
@@ -977,6 +1087,16 @@ int preserve_decode_step(preserve_layer_t *L, const preserve_step_io_t *io, void
     return run_steps(layers, &sp, 1, static_cast<cudaStream_t>(cuda_stream));
 }
 
+namespace {
+bool ranges_overlap(const void *a, size_t na, const void *b, size_t nb)
+{
+    if (!a || !b)
+        return false;
+    const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+    return x < y + nb && y < x + na;
+}
+}  // namespace
+
 int preserve_decode_chain(preserve_layer_t *const *layers, int32_t n, const preserve_step_io_t *ios, int32_t link,
                           void *cuda_stream)
 {
@@ -997,6 +1117,28 @@ int preserve_decode_chain(preserve_layer_t *const *layers, int32_t n, const pres
             sps[i].part0_f32 = 1;
             sps[i].residual_in = layers[i - 1]->h2_f32;
             sps[i].resid_f32 = 1;
+        }
+    }
+    // The window kernels request the step's input buffers before they wait for the kernel in front
+    // of them.  Inside one call that is only safe for buffers no earlier layer of the call writes:
+    // where an input of layer i overlaps an output of a layer before it (layers wired output to
+    // input without `link`), that window reads its inputs after the wait instead.
+    for (int i = 1; i < n; ++i) {
+        const size_t nb = (size_t)sps[i].batch * layers[i]->cfg.hidden * 2;
+        const int P = layers[i]->cfg.tp_degree;
+        for (int j = 0; j < i; ++j) {
+            const size_t mb = (size_t)sps[j].batch * layers[j]->cfg.hidden * 2;
+            const void *outs[3] = {sps[j].residual_out, sps[j].mlp_partial_out, sps[j].attn_partial_out};
+            for (const void *o : outs) {
+                if (!sps[i].resid_f32 && ranges_overlap(sps[i].residual_in, nb, o, mb))
+                    sps[i].late_a = 1;
+                for (int q = 0; q < P; ++q)
+                    if (!(q == 0 && sps[i].part0_f32) && ranges_overlap(sps[i].parts[q], nb, o, mb))
+                        sps[i].late_a = 1;
+                for (int q = 0; q + 1 < P; ++q)
+                    if (ranges_overlap(sps[i].peers[q], nb, o, mb))
+                        sps[i].late_b = 1;
+            }
         }
     }
     return run_steps(layers, sps.data(), n, static_cast<cudaStream_t>(cuda_stream));
@@ -1117,8 +1259,11 @@ int preserve_profile_step(preserve_layer_t *L, const preserve_step_io_t *io, voi
     if (rc)
         return rc;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    StepPlan pl;
+    sp.first_of_call = 1;
+    plan_step(L, sp, &pl);
     L->profiling = true;
-    rc = enqueue_step(L, sp, s);
+    rc = enqueue_step(L, sp, pl, true, s);
     L->profiling = false;
     if (rc)
         return rc;
@@ -1143,7 +1288,10 @@ int preserve_run_kernel(preserve_layer_t *L, const preserve_step_io_t *io, int32
     if (rc)
         return rc;
     L->only = which;
-    rc = enqueue_step(L, sp, static_cast<cudaStream_t>(cuda_stream));
+    StepPlan pl;
+    sp.first_of_call = 1;
+    plan_step(L, sp, &pl);
+    rc = enqueue_step(L, sp, pl, true, static_cast<cudaStream_t>(cuda_stream));
     L->only = -1;
     return rc;
 }
@@ -1208,7 +1356,7 @@ int preserve_last_status(preserve_layer_t *L)
     CK(L, cudaDeviceSynchronize());
     int st = 0;
     CK(L, cudaMemcpy(&st, L->status, sizeof(int), cudaMemcpyDeviceToHost));
-    return st == 0 ? PRESERVE_OK : PRESERVE_ETIMEOUT;
+    return st == ST_OK ? PRESERVE_OK : (st == ST_ITEMS_OVERFLOW ? PRESERVE_ESHAPE : PRESERVE_ETIMEOUT);
 }
 
 int preserve_last_cuda_error(const preserve_layer_t *L) { return L ? L->last_cuda : 0; }
@@ -1220,9 +1368,10 @@ int preserve_debug_copy(preserve_layer_t *L, int32_t which, void *dst, size_t by
     const auto &c = L->cfg;
     const size_t BH = (size_t)c.max_batch * c.hidden;
     const size_t RH = (size_t)L->rows * c.hidden, Rq = (size_t)L->rows * c.n_q_heads * c.head_dim;
-    const void *src[6] = {L->h_f32, L->x, L->q, L->o, L->x2, L->a};
-    const size_t cap[6] = {BH * 4, 2 * RH * 2, 2 * Rq * 2, 2 * Rq * 2, 2 * RH * 2, 2 * (size_t)L->rows * c.ffn * 2};
-    if (which < 0 || which > 5 || bytes > cap[which])
+    const void *src[7] = {L->h_f32, L->x, L->q, L->o, L->x2, L->a, L->status + kStatusPlanWord};
+    const size_t cap[7] = {BH * 4, 2 * RH * 2, 2 * Rq * 2, 2 * Rq * 2, 2 * RH * 2, 2 * (size_t)L->rows * c.ffn * 2,
+                           6 * sizeof(uint64_t)};
+    if (which < 0 || which > 6 || bytes > cap[which])
         return PRESERVE_EINVAL;
     CK(L, cudaMemcpyAsync(dst, src[which], bytes, cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(cuda_stream)));
     return PRESERVE_OK;

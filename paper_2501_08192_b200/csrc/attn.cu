@@ -53,6 +53,7 @@ struct AttnParams {
     size_t o_plane;
     int *status;
     long long *trace;
+    int inject;             // test hook: the producer of CTA 0 never fetches one box of its first tile
 };
 
 struct AttnSmem {
@@ -143,7 +144,15 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
     pdl_launch_dependents();
     build_item_table(p, sm.item_base);       // sequence lengths are inputs of the step: no dependency
     __syncthreads();
-    const int total_items = sm.item_base[streams];
+    // The partial buffers hold max_items entries, sized from the host copy of the lengths.  Device
+    // lengths that disagree with it must not write past them: the surplus items are dropped (the
+    // result is then wrong, and the status word says why).
+    int total_items = sm.item_base[streams];
+    if (total_items > p.max_items) {
+        total_items = p.max_items;
+        if (threadIdx.x == 0)
+            atomicCAS(p.status, ST_OK, ST_ITEMS_OVERFLOW);
+    }
 
     if (warp == kConsumerWarps) {
         // ------------------------------------------------------------ producer
@@ -171,7 +180,8 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
                     mbar_expect_tx(&sm.full[st], kStageBytes);
                     const int row = sidx * p.cap + tile * kTileKeys;
                     uint8_t *dst = sm.stage[st];
-                    tma_load_2d_hint(dst, &p.k_map, 0, row, &sm.full[st], pol);
+                    if (!(p.inject == INJECT_ATTN_RING && it == 0 && blockIdx.x == 0))
+                        tma_load_2d_hint(dst, &p.k_map, 0, row, &sm.full[st], pol);
                     tma_load_2d_hint(dst + kHalfBytes, &p.k_map, 64, row, &sm.full[st], pol);
                     tma_load_2d_hint(dst + 2 * kHalfBytes, &p.v_map, 0, row, &sm.full[st], pol);
                     tma_load_2d_hint(dst + 3 * kHalfBytes, &p.v_map, 64, row, &sm.full[st], pol);
@@ -527,7 +537,7 @@ __global__ void __launch_bounds__(kMergeMaxWarps * 32) k_attn_merge(const __grid
     if (n_items > 1) {          // a single item was finished by the split-KV kernel itself
         float Mg = -INFINITY, L = 0.f;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int e = warp; e < n_items; e += n_warps) {
+        for (int e = warp; e < n_items && base + e < p.max_items; e += n_warps) {
             const size_t ent = (size_t)(base + e) * p.G + row;
             const float2 ml = *reinterpret_cast<const float2 *>(p.part_ml + ent * 2);
             const float4 ov = *(reinterpret_cast<const float4 *>(p.part_o + ent * kHeadDim) + lane);
@@ -651,18 +661,16 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     p.o_out = reinterpret_cast<bf16 *>(a.o_out);
     p.status = a.status;
     p.trace = a.trace;
+    p.inject = a.inject;
 
     const size_t smem = attn_smem_bytes(a.B * a.nkv);
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_attn_decode_splitkv<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)attn_smem_bytes(kMaxStreams));
+    {
+        static PerDeviceSize lim_narrow, lim_wide;      // per device: the attribute belongs to one device
+        cudaError_t e = ensure_dynamic_smem(k_attn_decode_splitkv<true>, lim_narrow, attn_smem_bytes(kMaxStreams));
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(k_attn_decode_splitkv<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)attn_smem_bytes(kMaxStreams));
+            e = ensure_dynamic_smem(k_attn_decode_splitkv<false>, lim_wide, attn_smem_bytes(kMaxStreams));
         if (e != cudaSuccess)
             return e;
-        attr_set = true;
     }
     cudaLaunchAttribute at[1];
     cudaLaunchConfig_t cfg = {};
@@ -671,7 +679,7 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cfg.attrs = at;
-    cfg.numAttrs = pdl_attr(at);
+    cfg.numAttrs = pdl_attr(at, a.pdl);
     const int phases = a.phases ? a.phases : 3;
     cudaError_t e = cudaSuccess;
     if (phases & 1)
@@ -694,7 +702,7 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     cfg2.blockDim = dim3(warps * 32);
     cfg2.stream = s;
     cfg2.attrs = at;
-    cfg2.numAttrs = pdl_attr(at);
+    cfg2.numAttrs = pdl_attr(at, a.pdl);
     return cudaLaunchKernelEx(&cfg2, k_attn_merge, p);
 }
 
@@ -710,9 +718,8 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
 static __device__ __align__(256) unsigned char g_static_scratch[PRESERVE_STATIC_SCRATCH_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
-void *g_scratch_addr[kMaxDevices];      // per device, filled by the first call on that device
-int g_scratch_sms[kMaxDevices];
+void *g_scratch_addr[prsv::kMaxDevices];      // per device, filled by the first call on that device
+int g_scratch_sms[prsv::kMaxDevices];
 }  // namespace
 
 extern "C" int preserve_attention_static(const void *q_hi, const void *q_lo, const void *k_cache,
@@ -802,10 +809,32 @@ extern "C" int preserve_attention_static(const void *q_hi, const void *q_lo, con
     a.o_out = o_hi;
     a.o_plane = (size_t)(static_cast<bf16 *>(o_lo) - static_cast<bf16 *>(o_hi));
     a.status = reinterpret_cast<int *>(base);
+    a.pdl = 1;      // (the merge kernel's prologue overlaps the split-KV kernel's tail)
     if (launch_attention(a, s) != cudaSuccess) {
         (void)cudaGetLastError();
         return PRESERVE_ECUDA;
     }
     return PRESERVE_OK;
+}
+
+// The device status word of the allocation-free entry point on the current device (it lives at the
+// start of the static array, where no handle can reach it).  Waits for the device, allocates nothing.
+extern "C" int preserve_attention_static_status(void)
+{
+    using namespace prsv;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return PRESERVE_EARCH;
+    }
+    if (!g_scratch_addr[dev])
+        return PRESERVE_OK;         // no call on this device yet
+    int st = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess ||
+        cudaMemcpy(&st, g_scratch_addr[dev], sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return PRESERVE_ECUDA;
+    }
+    return st == ST_OK ? PRESERVE_OK : (st == ST_ITEMS_OVERFLOW ? PRESERVE_ESHAPE : PRESERVE_ETIMEOUT);
 }
 

@@ -6,17 +6,19 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "kernels.h"
+
 namespace prsv {
 
 typedef __nv_bfloat16 bf16;
 
-// Device status codes written to the layer's status word (first writer wins).
-enum : int { ST_OK = 0, ST_TIMEOUT_FULL = 1, ST_TIMEOUT_EMPTY = 2, ST_TIMEOUT_MMA = 3, ST_TIMEOUT_TMEM = 4 };
-
 // Upper bound, in SM clock cycles, on any mbarrier wait (about a second): far
 // beyond every legitimate wait of these kernels (microseconds), yet it guarantees
-// that a kernel can never spin forever.
+// that a kernel can never spin forever.  A handle may set a shorter limit (tests of
+// the give-up paths do); it is read from the status block only once a wait has
+// already lasted kFastWaitCycles, so ordinary waits never touch global memory.
 constexpr long long kMaxWaitCycles = 1ll << 31;
+constexpr long long kFastWaitCycles = 1ll << 19;
 
 __device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
@@ -102,7 +104,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *s
     do {
         if (mbar_try_wait(bar, parity))
             return true;
-    } while (clock64() - t0 < kMaxWaitCycles);
+    } while (clock64() - t0 < kFastWaitCycles);
+    long long limit = *reinterpret_cast<volatile long long *>(status + kStatusLimitWord);
+    if (limit <= 0 || limit > kMaxWaitCycles)
+        limit = kMaxWaitCycles;
+    while (clock64() - t0 < limit) {
+        if (mbar_try_wait(bar, parity))
+            return true;
+    }
     atomicCAS(status, ST_OK, code);
     return false;
 }

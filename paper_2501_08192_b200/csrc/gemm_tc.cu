@@ -55,6 +55,7 @@ struct GemmTcParams {
     EpilogueArgs epi;
     int *status;
     long long *trace;
+    int inject;         // test hook: the producer of CTA (0, 0) never fetches its first weight tile
 };
 
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr)
@@ -177,6 +178,8 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             const int pre = n_kb < p.stages ? n_kb : p.stages;
             for (int i = 0; i < pre; ++i) {
                 mbar_expect_tx(&full[i], stage_bytes);
+                if (p.inject == INJECT_TC_RING && i == 0 && tile == 0 && s == 0)
+                    continue;
                 tma_load_2d_hint(smem + (size_t)i * stage_bytes, &p.w_map, (kb0 + i) * kTcBlockK,
                                  tile * p.mt * kTcTileM, &full[i], pol);
             }
@@ -579,20 +582,19 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
 template <int KIND, int PUSH>
 static cudaError_t launch_instance(cudaLaunchConfig_t &cfg, const GemmTcParams &p, size_t smem)
 {
-    static size_t attr_smem = 0;        // per instantiation
-    if (smem > attr_smem) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemm_tcgen05<KIND, PUSH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess)
-            return e;
-        attr_smem = smem;
-    }
+    static PerDeviceSize smem_limit, np_set;      // per instantiation and device
+    cudaError_t e = ensure_dynamic_smem(k_gemm_tcgen05<KIND, PUSH>, smem_limit, smem);
+    if (e != cudaSuccess)
+        return e;
     if (p.splits > 8) {
-        static bool np_set = false;     // per instantiation
-        if (!np_set) {
-            cudaError_t e = cudaFuncSetAttribute(k_gemm_tcgen05<KIND, PUSH>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        const int dev = current_device_index();
+        if (dev < 0)
+            return cudaErrorInvalidDevice;
+        if (!np_set.v[dev]) {
+            e = cudaFuncSetAttribute(k_gemm_tcgen05<KIND, PUSH>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
             if (e != cudaSuccess)
                 return e;
-            np_set = true;
+            np_set.v[dev] = 1;
         }
     }
     return cudaLaunchKernelEx(&cfg, k_gemm_tcgen05<KIND, PUSH>, p);
@@ -610,6 +612,7 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     p.epi = a.epi;
     p.status = a.status;
     p.trace = a.trace;
+    p.inject = a.inject;
     // Two 128-row weight tiles per CTA share one activation tile when the batch is wide enough for
     // the activation tile (2 * NB rows) to weigh as much as a weight tile: halves the L2->SM traffic
     // of the activations, which every CTA re-reads.
@@ -691,7 +694,7 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cudaLaunchAttribute at[2];
-    int n = pdl_attr(at);
+    int n = pdl_attr(at, a.pdl);
     if (splits > 1) {
         at[n].id = cudaLaunchAttributeClusterDimension;
         at[n].val.clusterDim.x = 1;

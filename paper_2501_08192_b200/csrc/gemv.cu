@@ -40,8 +40,6 @@ namespace cg = cooperative_groups;
 
 namespace prsv {
 
-int g_pdl = 1;
-
 constexpr int kGemvWarps = 8;
 constexpr int kRingSlots = 4;
 constexpr int kUnitChunks = 2;                       // tiles per ring slot (2 KiB)
@@ -66,6 +64,7 @@ struct GemvParams {
     const uint8_t *next_w;
     uint32_t next_slice;   // bytes of next_w each CTA prefetches
     size_t next_bytes;
+    int inject;            // test hook: warp 0 of CTA (0, 0) arms its first ring slot but never fills it
     EpilogueArgs epi;
 };
 
@@ -122,8 +121,9 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
         const size_t rb = (size_t)p_grp * rbs_per_cta + rbl + p_r;
         const uint32_t bytes = (uint32_t)n * 1024u;
         mbar_expect_tx(&bars[warp][slot], bytes);
-        bulk_load_hint(ring + slot * (kUnitChunks * 1024),
-                       reinterpret_cast<const uint8_t *>(p.w) + (rb * p.kchunks + p_c) * 1024, bytes, &bars[warp][slot], pol);
+        if (!(p.inject == INJECT_GEMV_RING && n_issued == 0 && warp == 0 && blockIdx.x == 0 && blockIdx.y == 0))
+            bulk_load_hint(ring + slot * (kUnitChunks * 1024),
+                           reinterpret_cast<const uint8_t *>(p.w) + (rb * p.kchunks + p_c) * 1024, bytes, &bars[warp][slot], pol);
         ++n_issued;
         ++p_u;
         if (p_u == kBurstUnits || p_c0 + p_u * kUnitChunks >= c_end) {
@@ -368,15 +368,13 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
 }
 
 template <int NB, bool MMA, int RB>
-static cudaError_t launch_variant(GemvParams &p, int sm_count, cudaStream_t s)
+static cudaError_t launch_variant(GemvParams &p, int sm_count, int pdl, cudaStream_t s)
 {
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemv_splitk<NB, MMA, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kGemvSmemBytes + 32 * 1024 + 128);
+    static PerDeviceSize smem_limit;      // per instantiation and device
+    {
+        cudaError_t e = ensure_dynamic_smem(k_gemv_splitk<NB, MMA, RB>, smem_limit, kGemvSmemBytes + 32 * 1024 + 128);
         if (e != cudaSuccess)
             return e;
-        attr_done = true;
     }
     // Mapping: k is split over the 8 warps of a CTA while every warp still gets at least two
     // tiles (otherwise fewer warps split k and the others take further row blocks); cluster ranks
@@ -420,7 +418,7 @@ static cudaError_t launch_variant(GemvParams &p, int sm_count, cudaStream_t s)
     cfg.dynamicSmemBytes = ring_bytes + (p.push ? recv_bytes : 0) + 128;
     cfg.stream = s;
     cudaLaunchAttribute at[2];
-    int n = pdl_attr(at);
+    int n = pdl_attr(at, pdl);
     if (p.splits > 1) {
         at[n].id = cudaLaunchAttributeClusterDimension;
         at[n].val.clusterDim.x = 1;
@@ -449,14 +447,16 @@ cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s)
     p.trace = a.trace;
     p.next_w = reinterpret_cast<const uint8_t *>(a.next_w);
     p.next_bytes = a.next_bytes;
+    p.inject = a.inject;
+    const int pdl = a.pdl;
 
     // two row blocks per warp whenever the matrix has enough row blocks to still fill the SMs
     const bool two = p.row_blocks % 2 == 0 && p.row_blocks >= 32;
-    if (a.B == 1) return two ? launch_variant<1, false, 2>(p, sm_count, s) : launch_variant<1, false, 1>(p, sm_count, s);
-    if (a.B == 2) return two ? launch_variant<2, false, 2>(p, sm_count, s) : launch_variant<2, false, 1>(p, sm_count, s);
-    if (a.B <= 4) return two ? launch_variant<4, false, 2>(p, sm_count, s) : launch_variant<4, false, 1>(p, sm_count, s);
-    if (a.B <= 8) return two ? launch_variant<8, true, 2>(p, sm_count, s) : launch_variant<8, true, 1>(p, sm_count, s);
-    return two ? launch_variant<16, true, 2>(p, sm_count, s) : launch_variant<16, true, 1>(p, sm_count, s);
+    if (a.B == 1) return two ? launch_variant<1, false, 2>(p, sm_count, pdl, s) : launch_variant<1, false, 1>(p, sm_count, pdl, s);
+    if (a.B == 2) return two ? launch_variant<2, false, 2>(p, sm_count, pdl, s) : launch_variant<2, false, 1>(p, sm_count, pdl, s);
+    if (a.B <= 4) return two ? launch_variant<4, false, 2>(p, sm_count, pdl, s) : launch_variant<4, false, 1>(p, sm_count, pdl, s);
+    if (a.B <= 8) return two ? launch_variant<8, true, 2>(p, sm_count, pdl, s) : launch_variant<8, true, 1>(p, sm_count, pdl, s);
+    return two ? launch_variant<16, true, 2>(p, sm_count, pdl, s) : launch_variant<16, true, 1>(p, sm_count, pdl, s);
 }
 
 }  // namespace prsv

@@ -6,21 +6,66 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 namespace prsv {
 
-// Programmatic dependent launch: when non-zero, every kernel of the main stream is
-// launched with the programmatic-serialization attribute, so its prologue (index
-// setup, first weight loads) may overlap the previous kernel's tail.  Each kernel
-// executes griddepcontrol.wait before it touches anything another kernel wrote.
-extern int g_pdl;
-inline int pdl_attr(cudaLaunchAttribute *at)
+// Programmatic dependent launch: when `pdl` is non-zero the kernel is launched with the
+// programmatic-serialization attribute, so its prologue (index setup, first weight
+// loads) may overlap the previous kernel's tail.  Each kernel executes
+// griddepcontrol.wait before it touches anything another kernel wrote.  The switch is
+// a launch argument (every launcher's args carry it): no process-wide state.
+inline int pdl_attr(cudaLaunchAttribute *at, int pdl)
 {
-    if (!g_pdl)
+    if (!pdl)
         return 0;
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
     return 1;
 }
+
+// cudaFuncSetAttribute applies to the current device only, so "already set" is kept per
+// device (indexed by cudaGetDevice), never per process.  Setting an attribute twice is
+// harmless, so two threads that race here both succeed.
+constexpr int kMaxDevices = 64;
+struct PerDeviceSize {
+    size_t v[kMaxDevices] = {};
+};
+inline int current_device_index()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+        return -1;
+    return dev;
+}
+// Raise kernel `fn`'s dynamic shared-memory limit to at least `bytes` on the current device.
+template <typename Fn>
+inline cudaError_t ensure_dynamic_smem(Fn fn, PerDeviceSize &state, size_t bytes)
+{
+    const int dev = current_device_index();
+    if (dev < 0)
+        return cudaErrorInvalidDevice;
+    if (bytes <= state.v[dev])
+        return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess)
+        state.v[dev] = bytes;
+    return e;
+}
+
+// Test hooks (preserve_debug_set): make ONE producer of a kernel withhold ONE issue, so that the
+// consumer's bounded wait runs out and the give-up path runs.  Nothing faults or hangs: the wait
+// expires after the handle's wait limit and the kernel returns with a status code.
+enum Inject : int { INJECT_NONE = 0, INJECT_WINDOW_HANDOVER = 1, INJECT_GEMV_RING = 2, INJECT_TC_RING = 3,
+                    INJECT_ATTN_RING = 4 };
+
+// Device status block of a layer (ints): [0] status word (first writer wins), [2..3] the handle's
+// limit on any mbarrier wait in SM cycles (64-bit, 0 = the default below), [8] sink of the
+// prefetch kernel's load variant, [16..27] the prefetch kernels' own evaluation of the plan
+// (uint64 [2][3], written by CTA 0 of each prefetch launch).
+enum : int { ST_OK = 0, ST_TIMEOUT_FULL = 1, ST_TIMEOUT_EMPTY = 2, ST_TIMEOUT_MMA = 3, ST_TIMEOUT_TMEM = 4,
+             ST_ITEMS_OVERFLOW = 5 };
+constexpr int kStatusLimitWord = 2, kStatusSinkWord = 8, kStatusPlanWord = 16;
 
 constexpr int kMaxParts = 16;   // most partial-sum buffers in one window
 constexpr int kHeadDim = 128;
@@ -41,7 +86,11 @@ struct WindowArgs {
     int B, H;
     long long *trace;              // optional timeline slot (kTraceSlots values), see common.cuh
     int delay_ns;                  // modelled communication latency added to the window (0 = none)
-    int *status;                   // device error word (bounded waits report here)
+    int *status;                   // device status block (bounded waits report here)
+    int pdl;                       // launch with the programmatic-serialization attribute
+    int inputs_after_wait;         // the step's input buffers may still be written by an earlier kernel of the
+                                   // same call: read them only after the dependency wait
+    int inject;                    // test hook (Inject)
 };
 cudaError_t launch_window(const WindowArgs &a, cudaStream_t s);
 
@@ -85,6 +134,8 @@ struct GemvArgs {
     long long *trace;
     const void *next_w;   // optional: weights of the kernel that follows, prefetched to L2 once this one has streamed its own
     size_t next_bytes;
+    int pdl;
+    int inject;
 };
 cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s);
 
@@ -97,6 +148,8 @@ struct GemmTcArgs {
     EpilogueArgs epi;
     int *status;
     long long *trace;
+    int pdl;
+    int inject;
 };
 cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s);
 
@@ -120,6 +173,8 @@ struct AttnArgs {
     cudaEvent_t mid_event; // optional: recorded between the split-KV kernel and the merge kernel
     int phases;            // bit 0: split-KV kernel, bit 1: merge kernel (0 = both)
     long long *trace;      // optional: two consecutive timeline slots (split-KV, merge)
+    int pdl;
+    int inject;
 };
 cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s);
 // Grid size (persistent CTAs) and tiles per work item for the given sequence lengths (host array);
@@ -130,28 +185,40 @@ void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_coun
 bool encode_bf16_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_cols,
                         uint32_t box_rows);
 
-// ---- L2 prefetch (no arithmetic, writes nothing)
-struct PrefetchSeg {
-    const void *base;     // contiguous range, or the K cache when per_seq_tokens != 0
-    const void *base2;    // the V cache when per_seq_tokens != 0
-    uint64_t stride;      // KV: bytes between consecutive (sequence, kv head) runs
-    uint64_t bytes;       // bytes to prefetch from this segment (the planner's figure)
-    int count;            // KV: number of (sequence, kv head) runs
-    int per_seq_tokens;   // != 0: KV segment; run i holds ctx_len[i / ranges_per_seq] live tokens
-    int ranges_per_seq;   // KV heads per sequence
-    int token_bytes;      // bytes per token per run (head_dim * 2)
+// ---- L2 prefetch (no arithmetic on the data).  The launch carries one window's node list in
+// breadth-first order and the budget; the kernel evaluates Algorithm 1 itself with the live
+// sequence lengths, so the arguments do not change from step to step of a decode loop.
+constexpr int kPfMaxNodes = 6;
+struct PrefetchNode {
+    const void *base;     // weights: the contiguous packed matrix; SelfAttention: the K cache
+    const void *base2;    // SelfAttention: the V cache
+    uint64_t bytes;       // weights: the node's memSize; unused for the SelfAttention node
 };
 struct PrefetchArgs {
-    PrefetchSeg seg[6];
-    int n_segs;
-    const int *ctx_len;
-    int *sink;            // scratch word for the load variant (practically never written)
+    PrefetchNode node[kPfMaxNodes];
+    int n_nodes;
+    int kv_node;            // index of the SelfAttention node in node[], or -1
+    int kv_count;           // (sequence, kv head) runs
+    int kv_ranges_per_seq;  // kv heads per sequence: run i belongs to sequence i / kv_ranges_per_seq
+    int kv_token_bytes;     // bytes per cached token per run (head_dim * 2)
+    uint64_t kv_stride;     // bytes between consecutive runs
+    uint64_t budget;        // Algorithm 1's C for this window
+    int plan_mode;          // PRESERVE_PLAN_*
+    int mechanism;          // 0 bulk L2 prefetch, 1 per-line hints, 2 plain loads
+    uint32_t chunk;         // bytes per prefetch instruction / per thread visit (multiple of 128)
+    const int *ctx_len;     // device [sequences]
+    int *sink;              // scratch word for the load variant (practically never written)
+    unsigned long long *plan_out;   // optional: device uint64[kPfMaxNodes], receives the bytes taken per node
 };
+// ---- Algorithm 1 over an explicit operator graph (planner.cu; host only).  Successors in CSR form.
+struct PlanHit { int comm, node; uint64_t bytes; };      // prefetch `bytes` of `node` beside communication op `comm`
+int plan_graph(int n_nodes, const int32_t *kind, const uint64_t *mem_bytes, const int32_t *succ_off,
+               const int32_t *succ, uint64_t budget, int mode, std::vector<PlanHit> &out);
+
 // ---- host-buffer entry point: gather of pinned host buffers (device views) into device memory
 cudaError_t launch_stage_inputs(const void *const *src, void *const *dst, int n, size_t bytes_each, const int *ctx_src,
                                 int *ctx_dst, int n_ctx, cudaStream_t s);
 
-void set_prefetch_kernel_mode(int mode, uint32_t chunk_bytes);
 cudaError_t launch_prefetch(const PrefetchArgs &a, int ctas, cudaStream_t s, const cudaLaunchAttribute *attrs,
                             int n_attrs);
 

@@ -1,149 +1,211 @@
 // L2 prefetch of weights and KV-cache entries on the side stream (Section 3,
 // "Execution with the proposed method": the read-only operands of the operators
 // that follow a collective are fetched into on-chip cache while the collective
-// runs).  The kernel does no arithmetic and writes nothing: it only issues
-// prefetch hints over the planned byte ranges, in the order the consumer
-// kernels will read them (weights in address order of the packed arena; K then
-// V of each (sequence, kv head) in cache order).  It uses a handful of CTAs so
-// it does not take SMs away from the main stream.
+// runs).  The kernel does no arithmetic on the data: it issues prefetch hints
+// over the planned byte ranges, in the order the consumer kernels will read them
+// (weights in address order of the packed arena; K then V of each (sequence, kv
+// head) in cache order).  It uses a handful of CTAs so it does not take SMs away
+// from the main stream.
 //
-// Modes:
+// Which bytes: the kernel evaluates Algorithm 1 ("Prefetch Operator Insertion")
+// itself, over the window's node list (weight nodes with fixed sizes; the
+// SelfAttention node whose size is the K and V bytes of the tokens cached right
+// now, read from the device copy of the sequence lengths) against the budget C.
+// The launch arguments therefore do not depend on the sequence lengths, so one
+// captured graph serves every step of a decode loop; the host evaluates the same
+// walk for reporting (preserve_layer_get_info), and CTA 0 writes what it decided
+// into the layer's status block so the two can be compared.
+//
+// Mechanisms:
 //   0  cp.async.bulk.prefetch.L2 : one instruction per `chunk` bytes
 //   1  prefetch.global.L2        : one instruction per 128-byte line
 //   2  plain 128-bit loads whose values are dropped (completion of the kernel
-//      then implies arrival in L2; kept as the control for modes 0 and 1)
+//      then implies arrival in L2; kept as the control for mechanisms 0 and 1)
+#include "../../include/preserve.h"
 #include "common.cuh"
 #include "kernels.h"
 
 namespace prsv {
 
 constexpr int kPfThreads = 128;
-constexpr int kPfMaxRanges = 1024 + 8;   // 512 (sequence, kv head) runs x {K, V} + weights
-
-struct PfRange { const uint8_t *ptr; uint64_t bytes; };
+constexpr int kPfMaxRuns = 2 * 2048;     // {K, V} x (sequence, kv head) runs: the most a layer can have
+constexpr int kPfRunsPerThread = kPfMaxRuns / kPfThreads;
 
 struct PrefetchParams {
     PrefetchArgs a;
-    int mode;
-    uint32_t chunk;
-    int *sink;      // never written in practice (see mode 2)
 };
+
+// Exclusive prefix sum over the 128 threads' values (two-level warp scan); returns the total.
+__device__ __forceinline__ uint64_t block_exclusive_scan(uint64_t v, uint64_t *warp_tot, uint64_t &excl)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint64_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint64_t n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o)
+            inc += n;
+    }
+    __syncthreads();            // warp_tot may still be read from an earlier scan
+    if (lane == 31)
+        warp_tot[warp] = inc;
+    __syncthreads();
+    uint64_t before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < kPfThreads / 32; ++w) {
+        if (w < warp)
+            before += warp_tot[w];
+        total += warp_tot[w];
+    }
+    excl = before + inc - v;
+    return total;
+}
 
 __global__ void __launch_bounds__(kPfThreads) k_prefetch_l2(const __grid_constant__ PrefetchParams p)
 {
-    __shared__ PfRange ranges[kPfMaxRanges];
-    __shared__ uint64_t range_first_chunk[kPfMaxRanges + 1];
-    __shared__ int n_ranges_s;
+    // per run of the SelfAttention node: bytes to prefetch and the run's first chunk index
+    __shared__ uint32_t run_bytes[kPfMaxRuns];
+    __shared__ uint32_t run_chunk0[kPfMaxRuns + 1];
+    __shared__ uint64_t warp_tot[kPfThreads / 32];
+    __shared__ uint64_t take_s[kPfMaxNodes];
 
+    const PrefetchArgs &a = p.a;
+    const int kv_node = a.kv_node;                     // index of the SelfAttention node, or -1
+    const int n_runs = kv_node >= 0 ? 2 * a.kv_count : 0;
+    const int r0 = threadIdx.x * kPfRunsPerThread;     // this thread's block of runs
+
+    // ---- live bytes of every K / V run (run 2 i = K of stream i, run 2 i + 1 = V of stream i)
+    uint64_t mine = 0;
+    for (int r = r0; r < r0 + kPfRunsPerThread && r < n_runs; ++r) {
+        const uint64_t live64 = (uint64_t)a.ctx_len[(r >> 1) / a.kv_ranges_per_seq] * (uint64_t)a.kv_token_bytes;
+        const uint32_t live = live64 < 0xFFFFFF80ull ? (uint32_t)live64 : 0xFFFFFF80u;
+        run_bytes[r] = live;
+        mine += live;
+    }
+    uint64_t before = 0;
+    const uint64_t kv_total = block_exclusive_scan(mine, warp_tot, before);
+
+    // ---- Algorithm 1 over the window's nodes (one thread; a handful of nodes)
     if (threadIdx.x == 0) {
-        // Flatten the segments into (ptr, bytes) ranges; every CTA builds the same table.
-        int n = 0;
-        uint64_t chunks = 0;
-        for (int si = 0; si < p.a.n_segs; ++si) {
-            const PrefetchSeg &sg = p.a.seg[si];
-            uint64_t left = sg.bytes;                    // budget of this segment
-            if (!sg.per_seq_tokens) {
-                if (left && n < kPfMaxRanges) {
-                    ranges[n].ptr = reinterpret_cast<const uint8_t *>(sg.base);
-                    ranges[n].bytes = left;
-                    range_first_chunk[n] = chunks;
-                    chunks += (left + p.chunk - 1) / p.chunk;
-                    ++n;
-                }
-                continue;
-            }
-            // KV: per (sequence, kv head) stream, K run then V run, each ctx_len * token_bytes long
-            const uint8_t *kb = reinterpret_cast<const uint8_t *>(sg.base);
-            const uint8_t *vb = reinterpret_cast<const uint8_t *>(sg.base2);
-            for (int st = 0; st < sg.count && left; ++st) {
-                const uint64_t live = (uint64_t)p.a.ctx_len[st / sg.ranges_per_seq] * sg.token_bytes;
-                for (int kv = 0; kv < 2 && left; ++kv) {
-                    const uint64_t take = (live < left ? live : left) & ~uint64_t(127);
-                    if (take && n < kPfMaxRanges) {
-                        ranges[n].ptr = (kv ? vb : kb) + (uint64_t)st * sg.stride;
-                        ranges[n].bytes = take;
-                        range_first_chunk[n] = chunks;
-                        chunks += (take + p.chunk - 1) / p.chunk;
-                        ++n;
+        uint64_t cache_sum = 0;
+        bool open = true;
+        for (int i = 0; i < a.n_nodes; ++i) {
+            const uint64_t mem = i == kv_node ? kv_total : a.node[i].bytes;
+            uint64_t take = 0;
+            if (open) {
+                if (cache_sum + mem < a.budget) {           // strict: a node that fills C exactly is not inserted
+                    cache_sum += mem;
+                    take = mem;
+                } else {
+                    if (a.plan_mode == PRESERVE_PLAN_TRUNCATE) {
+                        const uint64_t room = a.budget > cache_sum ? a.budget - cache_sum : 0;
+                        take = room & ~uint64_t(127);
+                        if (take > mem)
+                            take = mem;
                     }
-                    left -= take;
-                    if (take < live)
-                        left = 0;           // budget ran out inside this run: stop here
+                    open = false;                           // the walk for this communication op ends
                 }
             }
+            take_s[i] = take;
+            if (blockIdx.x == 0 && a.plan_out)
+                a.plan_out[i] = take;
         }
-        range_first_chunk[n] = chunks;
-        n_ranges_s = n;
+        if (blockIdx.x == 0 && a.plan_out)
+            for (int i = a.n_nodes; i < kPfMaxNodes; ++i)
+                a.plan_out[i] = 0;
     }
     __syncthreads();
-    const int n_ranges = n_ranges_s;
-    if (n_ranges == 0)
-        return;
-    const uint64_t total_chunks = range_first_chunk[n_ranges];
-    if (p.mode == 2) {
-        // load variant: a warp takes a chunk and reads it with coalesced accesses - lane l touches
-        // the 32-byte sector l of each KiB (one 16-byte load per sector brings in the whole line).
-        // The values are folded into a word that is stored only if it equals a magic number, which
-        // keeps the assembler from dropping the loads; in practice nothing is ever written.
-        const int lane = threadIdx.x & 31;
-        const uint64_t warp_id = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-        const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
-        uint32_t fold = 0;
-        int r = 0;
-        for (uint64_t c = warp_id; c < total_chunks; c += n_warps) {
-            while (range_first_chunk[r + 1] <= c)
-                ++r;
-            const uint64_t off = (c - range_first_chunk[r]) * p.chunk;
-            const uint64_t left = ranges[r].bytes - off;
-            const uint32_t n = left < p.chunk ? (uint32_t)left : p.chunk;
-            const uint8_t *ptr = ranges[r].ptr + off + lane * 32;
-#pragma unroll 4
-            for (uint32_t o = lane * 32; o < n; o += 1024, ptr += 1024) {
-                const uint4 v = ld_stream(ptr);
+
+    // ---- cut the SelfAttention node's share over its runs, in cache order, whole 128-byte lines
+    const uint32_t chunk = a.chunk;
+    uint64_t my_chunks = 0;
+    if (n_runs) {
+        const uint64_t kv_take = take_s[kv_node];
+        uint64_t off = before;                              // live bytes before this thread's first run
+        for (int r = r0; r < r0 + kPfRunsPerThread && r < n_runs; ++r) {
+            const uint64_t live = run_bytes[r];
+            uint64_t t = off >= kv_take ? 0 : (kv_take - off < live ? kv_take - off : live);
+            t &= ~uint64_t(127);
+            off += live;
+            run_bytes[r] = (uint32_t)t;
+            my_chunks += (t + chunk - 1) / chunk;
+        }
+    }
+    uint64_t chunks_before = 0;
+    const uint64_t kv_chunks = block_exclusive_scan(my_chunks, warp_tot, chunks_before);
+    if (n_runs) {
+        uint32_t c = (uint32_t)chunks_before;
+        for (int r = r0; r < r0 + kPfRunsPerThread && r < n_runs; ++r) {
+            run_chunk0[r] = c;
+            c += (run_bytes[r] + chunk - 1) / chunk;
+        }
+        if (threadIdx.x == 0)
+            run_chunk0[n_runs] = (uint32_t)kv_chunks;
+    }
+    __syncthreads();
+
+    // ---- walk the nodes in order; the chunks of a node are dealt to all threads of the grid
+    const uint64_t gtid = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint64_t gthreads = (uint64_t)gridDim.x * blockDim.x;
+    uint32_t fold = 0;
+    auto touch = [&](const uint8_t *ptr, uint32_t n) {
+        if (a.mechanism == 0) {
+            bulk_prefetch_l2(ptr, n & ~15u);
+        } else if (a.mechanism == 1) {
+            for (uint32_t o = 0; o < n; o += 128)
+                line_prefetch_l2(ptr + o);
+        } else {
+#pragma unroll 8
+            for (uint32_t o = 0; o < n; o += 32) {          // one 16-byte load per 32-byte sector
+                const uint4 v = ld_stream(ptr + o);
                 fold ^= v.x ^ v.y ^ v.z ^ v.w;
             }
         }
-        if (fold == 0x5eed1234u && p.sink)
-            *p.sink = (int)fold;
-        return;
-    }
-    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-    int r = 0;
-    for (uint64_t c = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; c < total_chunks; c += stride) {
-        while (range_first_chunk[r + 1] <= c)
-            ++r;
-        const uint64_t off = (c - range_first_chunk[r]) * p.chunk;
-        const uint64_t left = ranges[r].bytes - off;
-        const uint32_t n = left < p.chunk ? (uint32_t)left : p.chunk;
-        const uint8_t *ptr = ranges[r].ptr + off;
-        if (p.mode == 0) {
-            bulk_prefetch_l2(ptr, n & ~15u);
+    };
+    uint64_t first = 0;                                     // global chunk index of the node's first chunk
+    for (int i = 0; i < a.n_nodes; ++i) {
+        const uint64_t take = take_s[i];
+        if (i != kv_node) {
+            const uint64_t n_chunks = (take + chunk - 1) / chunk;
+            const uint8_t *base = reinterpret_cast<const uint8_t *>(a.node[i].base);
+            // (start where the previous node's dealing left off, so the threads stay evenly loaded)
+            uint64_t c = (gtid + gthreads - first % gthreads) % gthreads;
+            for (; c < n_chunks; c += gthreads) {
+                const uint64_t off = c * chunk;
+                const uint64_t left = take - off;
+                touch(base + off, left < chunk ? (uint32_t)left : chunk);
+            }
+            first += n_chunks;
         } else {
-            for (uint32_t o = 0; o < n; o += 128)
-                line_prefetch_l2(ptr + o);
+            const uint8_t *kb = reinterpret_cast<const uint8_t *>(a.node[i].base);
+            const uint8_t *vb = reinterpret_cast<const uint8_t *>(a.node[i].base2);
+            int r = 0;
+            uint64_t c = (gtid + gthreads - first % gthreads) % gthreads;
+            for (; c < kv_chunks; c += gthreads) {
+                while (run_chunk0[r + 1] <= c)
+                    ++r;
+                const uint64_t off = (c - run_chunk0[r]) * chunk;
+                const uint64_t left = run_bytes[r] - off;
+                const uint8_t *ptr = ((r & 1) ? vb : kb) + (uint64_t)(r >> 1) * a.kv_stride + off;
+                touch(ptr, left < chunk ? (uint32_t)left : chunk);
+            }
+            first += kv_chunks;
         }
     }
-}
-
-static int g_pf_mode = 0;   // measured on config 2: bulk L2 prefetch from 128 CTAs disturbs the main stream
-                            // least; per-line hints and plain loads cost more issue slots and time
-static uint32_t g_pf_chunk = 4096;
-
-void set_prefetch_kernel_mode(int mode, uint32_t chunk)
-{
-    g_pf_mode = mode;
-    if (chunk >= 128)
-        g_pf_chunk = chunk & ~127u;
+    // the load variant folds its values into a word that is stored only if it equals a magic number,
+    // which keeps the assembler from dropping the loads; in practice nothing is ever written
+    if (a.mechanism == 2 && fold == 0x5eed1234u && a.sink)
+        *a.sink = (int)fold;
 }
 
 cudaError_t launch_prefetch(const PrefetchArgs &a, int ctas, cudaStream_t s, const cudaLaunchAttribute *attrs,
                             int n_attrs)
 {
+    if (a.n_nodes < 0 || a.n_nodes > kPfMaxNodes || a.kv_node >= a.n_nodes || a.chunk < 128 || a.chunk % 128 ||
+        (a.kv_node >= 0 && (2 * a.kv_count > kPfMaxRuns || a.kv_count < 0 || a.kv_ranges_per_seq < 1)))
+        return cudaErrorInvalidValue;
     PrefetchParams p;
     p.a = a;
-    p.mode = g_pf_mode;
-    p.chunk = g_pf_chunk;
-    p.sink = a.sink;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ctas);
     cfg.blockDim = dim3(kPfThreads);

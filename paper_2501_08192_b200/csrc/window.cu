@@ -42,6 +42,8 @@ struct WindowParams {
     long long *trace;
     int delay_ns;
     int *status;
+    int no_hint;         // LEAN: do not even hint the inputs into L2 before the wait (another kernel of the call still writes them)
+    int inject;          // test hook: rank 1 of every row withholds its hand-over to rank 0
 };
 
 // (One instantiation for all four input forms: the two windows of a layer then run the same
@@ -106,7 +108,7 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
     };
     if constexpr (LEAN) {
         // one hint per 128-byte line (8 threads share a line)
-        if ((threadIdx.x & 7) == 0 && (int)threadIdx.x < chunks) {
+        if (!p.no_hint && (threadIdx.x & 7) == 0 && (int)threadIdx.x < chunks) {
             if (!RESID_F32)
                 line_prefetch_l2(reinterpret_cast<const uint4 *>(p.resid) + row_off + threadIdx.x);
             for (int j = 0; j < p.n_parts; ++j)
@@ -194,7 +196,7 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
         if (p.cluster > 1 && lane < p.cluster) {
             if (lane == rank)
                 recv[rank] = t;
-            else
+            else if (!(p.inject == INJECT_WINDOW_HANDOVER && rank == 1 && lane == 0))
                 st_async_f32(cluster_map(&recv[rank], lane), t, cluster_map(&recv_bar, lane));
         }
     }
@@ -276,7 +278,13 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
         cl *= 2;
     p.cluster = cl;
     const int chunks = a.H / 8 / cl;
-    const bool lean = a.B * cl > 256 && chunks <= 512;
+    // LEAN (inputs read after the wait) for big batches, and whenever an input buffer may still be
+    // written by an earlier kernel of the same call
+    const bool lean = (a.B * cl > 256 || a.inputs_after_wait) && chunks <= 512;
+    if (a.inputs_after_wait && !lean)
+        return cudaErrorInvalidValue;
+    p.no_hint = a.inputs_after_wait;
+    p.inject = a.inject;
     int threads = (chunks + kWinMaxChunks - 1) / kWinMaxChunks;
     if (chunks <= 512)
         threads = chunks;
@@ -290,7 +298,7 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
     cfg.stream = s;
     cudaLaunchAttribute at[2];
     cfg.attrs = at;
-    int n_attr = pdl_attr(at);
+    int n_attr = pdl_attr(at, a.pdl);
     if (cl > 1) {
         at[n_attr].id = cudaLaunchAttributeClusterDimension;
         at[n_attr].val.clusterDim.x = cl;

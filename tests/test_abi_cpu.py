@@ -131,3 +131,76 @@ def test_input_recipe_is_stable():
     assert r.min() >= 512 and r.max() <= 4096 and len(set(r.tolist())) > 32
     again = I.make_layers(I.CONFIGS[0], 1)[0]
     assert all(np.array_equal(t[k], again[k]) for k in ("w_q", "w_down", "k_cache", "partials_in"))
+
+
+# ---------------------------------------------------------------- Algorithm 1 as a graph pass
+_KIND = {"comm": P.NODE_COMM, "matmul": P.NODE_MATMUL, "attention": P.NODE_ATTENTION, "other": P.NODE_OTHER}
+
+
+def _run_graph_pass(g, budget, mode=P.PLAN_WHOLE_NODE):
+    hits = P.preserve_plan_graph([_KIND[n["kind"]] for n in g], [int(n["mem"]) for n in g],
+                                 [n["children"] for n in g], budget, mode)
+    plan = {i: [] for i, n in enumerate(g) if n["kind"] == "comm"}
+    for comm, node, nbytes in hits:
+        plan[comm].append((node, nbytes))
+    return plan
+
+
+def test_graph_pass_matches_the_oracle_on_whole_models(lib, oracle):
+    """32- and 80-layer operator chains of the Llama-shaped shards: the library's pass inserts the
+    same prefetches, beside the same communication operators, in the same order, as the oracle's
+    restatement of Algorithm 1."""
+    for s, n_layers in ((I.CONFIGS[1], 32), (I.CONFIGS[2], 80), (I.CONFIGS[3], 80), (I.CONFIGS[4], 32)):
+        g = oracle.layer_graph(s.hidden, s.n_q_heads, s.n_kv_heads, s.head_dim, s.ffn, s.batch * s.ctx, n_layers)
+        for budget in (0, 1, 8 << 20, 32 << 20, 126 << 20, 1 << 30, 1 << 40):
+            want = oracle.insert_prefetch_ops(g, budget)
+            got = _run_graph_pass(g, budget)
+            assert {k: [n for n, _ in v] for k, v in got.items()} == want, (s.name, budget)
+            assert all(b == g[n]["mem"] for v in got.values() for n, b in v)
+
+
+def test_graph_pass_matches_the_oracle_on_random_dags(lib, oracle):
+    rng = np.random.default_rng(11)
+    kinds = ("comm", "matmul", "attention", "other")
+    for trial in range(200):
+        n = int(rng.integers(1, 40))
+        g = []
+        for i in range(n):
+            later = list(range(i + 1, n))
+            k = int(rng.integers(0, min(4, len(later)) + 1))
+            ch = sorted(rng.choice(later, size=k, replace=False).tolist()) if k else []
+            g.append({"kind": kinds[int(rng.choice(4, p=(0.2, 0.4, 0.15, 0.25)))],
+                      "mem": int(rng.integers(0, 1000)), "children": [int(c) for c in ch]})
+        total = sum(x["mem"] for x in g)
+        for budget in (0, 1, int(rng.integers(0, total + 2)), total + 1):
+            want = oracle.insert_prefetch_ops(g, budget)
+            got = _run_graph_pass(g, budget)
+            assert {k: [nn for nn, _ in v] for k, v in got.items()} == want, (trial, budget)
+
+
+def test_graph_pass_truncate_mode_and_errors(lib, oracle):
+    # on a chain the TRUNCATE pass equals the ordered-list form, window by window
+    s = I.CONFIGS[2]
+    g = oracle.layer_graph(s.hidden, s.n_q_heads, s.n_kv_heads, s.head_dim, s.ffn, s.batch * s.ctx, 2)
+    na, nb = layer_nodes(s, s.batch * s.ctx)
+    for budget in (0, 100, 64 << 20, 126 << 20, 1 << 29):
+        got = _run_graph_pass(g, budget, P.PLAN_TRUNCATE)
+        for base, comm_a, comm_b in ((0, 0, 5), (9, 9, 14)):
+            a = {n - base: b for n, b in got[comm_a]}
+            b_ = {n - base: b for n, b in got[comm_b]}
+            assert [a.get(i, 0) for i in (1, 3, 4)] == oracle.truncate_plan(na, budget)
+            assert [b_.get(i, 0) for i in (6, 8)] == oracle.truncate_plan(nb, budget)
+    # a cycle is walked once; bad arguments are refused
+    assert P.preserve_plan_graph([0, 1, 1], [0, 5, 5], [[1], [2], [1]], 100) == [(0, 1, 5), (0, 2, 5)]
+    assert P.preserve_plan_graph([], [], [], 10) == []
+    with pytest.raises(P.PreserveError):
+        P.preserve_plan_graph([0, 9], [0, 1], [[1], []], 10)
+    with pytest.raises(P.PreserveError):
+        P.preserve_plan_graph([0, 1], [0, 1], [[5], []], 10)
+    n_out = C.c_int32()
+    k = (C.c_int32 * 2)(0, 1)
+    m = (C.c_uint64 * 2)(0, 5)
+    so = (C.c_int32 * 3)(0, 1, 1)
+    su = (C.c_int32 * 1)(1)
+    assert lib.preserve_plan_graph(2, k, m, so, su, 10, 0, 0, None, None, None, C.byref(n_out)) == P.PRESERVE_ETOOBIG
+    assert n_out.value == 1

@@ -112,6 +112,7 @@ def test_prefetch_never_changes_results(oracle):
                   I.CONFIGS[1]):
         t = I.make_layers(shape, 1)[0]
         base = None
+        stream = torch.cuda.Stream()      # (on the legacy default stream every step is launched directly)
         for flags in (0, P.FLAG_NO_GRAPH):
             dl = G.DeviceLayer(shape, t, flags=flags)
             try:
@@ -121,7 +122,8 @@ def test_prefetch_never_changes_results(oracle):
                     for frac in (0.0, 1 / 16, 1 / 4, 1 / 2, 1.0, 2.0):
                         dl.layer.set_prefetch_bytes(int(frac * l2))
                         for _ in range(2):
-                            dl.run()
+                            with torch.cuda.stream(stream):
+                                dl.run(stream)
                             bits = dl.output_bits()
                             if base is None:
                                 base = bits

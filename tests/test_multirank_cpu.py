@@ -41,3 +41,40 @@ def test_two_replicas_aggregate_by_slowest_rank():
         assert abs(gbs - 2 * 73117696 * 8 / 1.5e-3 / 1e9) < 1e-6
     a, b = out[world]
     assert a != b and out[world] == out[world + 1]         # different seeds, consistent view
+
+
+def test_bench_spawns_its_own_ranks_when_started_without_a_launcher():
+    """`python bench.py --gpus 2` with no WORLD_SIZE in the environment starts two ranks itself
+    (here with --dry-run: CPU, gloo, nothing timed) and rank 0 reports n_gpus = 2."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run"],
+                       capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                     # rank 0 alone prints
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2 and out["dry_run"] is True
+    assert out["ms_per_step"] == 1.25          # the slowest rank's time
+
+    import bench
+    cmd = bench.spawn_command(4, 29999, ["--gpus", "4", "--steps", "7"])
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node=4" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[-4:] == ["--gpus", "4", "--steps", "7"]
+
+
+def test_bench_byte_accounting_matches_the_library():
+    """bench.py's per-kernel byte table sums to the library's algorithmic bytes for every config
+    (the reference arm uses the table alone and never loads the CUDA library)."""
+    import bench
+    from paper_2501_08192_b200 import binding as P
+    from paper_2501_08192_b200 import build as B
+    from paper_2501_08192_b200 import inputs as I
+    B.build()
+    for s in I.CONFIGS:
+        for sum_ctx in (s.batch * s.ctx, s.batch * 17):
+            assert bench.algorithmic_bytes(s, sum_ctx) == P.preserve_algorithmic_bytes(P.make_config(s), s.batch, sum_ctx)
+    src = open(os.path.join(ROOT, "bench.py")).read()
+    ref = src[src.index("def run_reference"):src.index("def main")]
+    assert "binding" not in ref and "libpreserve" not in ref

@@ -67,6 +67,32 @@ def test_static_attention_matches_layer_path_twice_in_a_row():
         G.assert_close(got.cpu().numpy(), o_ref.cpu().numpy(), f"{shape.name}:o (second round)")
 
 
+def test_static_attention_matches_the_oracle_directly(oracle):
+    """The same entry point against the CPU oracle's attention on inputs drawn here (no layer path
+    in between): plain bf16 queries (zero lo plane), ragged lengths, two calls in a row."""
+    rng = np.random.default_rng(63)
+    for B, nq, nkv, cap, lens in ((5, 8, 2, 900, (899, 1, 64, 63, 500)), (2, 4, 4, 130, (129, 77))):
+        q_bits = I.f32_to_bf16_bits(rng.standard_normal((B, nq, 128), dtype=np.float32))
+        k_bits = I.f32_to_bf16_bits(rng.standard_normal((B, nkv, cap, 128), dtype=np.float32))
+        v_bits = I.f32_to_bf16_bits(rng.standard_normal((B, nkv, cap, 128), dtype=np.float32))
+        ctx = np.array(lens, np.int32) - 1                  # the newest entry is already in the cache
+        for b in range(B):
+            k_bits[b, :, lens[b]:] = I.BF16_NAN
+            v_bits[b, :, lens[b]:] = I.BF16_NAN
+        # oracle: attends over slots 0..ctx[b]-1 of the cache plus the "new" entry = slot ctx[b]
+        k_new = np.stack([I.bf16_bits_to_f32(k_bits[b, :, ctx[b]]) for b in range(B)])
+        v_new = np.stack([I.bf16_bits_to_f32(v_bits[b, :, ctx[b]]) for b in range(B)])
+        want = oracle.attention(I.bf16_bits_to_f32(q_bits), k_new, v_new, k_bits, v_bits, ctx)
+        q_hi = G.bits_to_cuda(q_bits)
+        q_lo = torch.zeros_like(q_hi)
+        kc, vc = G.bits_to_cuda(k_bits), G.bits_to_cuda(v_bits)
+        ctx_dev = torch.from_numpy(ctx).cuda()
+        shape = I.small_shape(name="static_direct", batch=B, n_q_heads=nq, n_kv_heads=nkv, ctx=cap - 1)
+        got = run_static(shape, q_hi, q_lo, kc, vc, ctx_dev, ctx)
+        assert P.preserve_attention_static_status() == P.PRESERVE_OK
+        G.assert_close(got.cpu().numpy(), want, f"static vs oracle B={B}")
+
+
 def test_static_attention_rejects_what_does_not_fit():
     # 16 query heads per KV head and 1024 (sequence, kv head) streams need far more than the fixed array
     B, nq, nkv, cap = 128, 128, 8, 2
