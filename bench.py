@@ -396,6 +396,26 @@ def measure_streams(P, torch, stream, quick: bool = True):
                 rows.append({"buffer_mib": round(slice_bytes / (1 << 20), 2), "source": kind + " (one CTA on one SM)",
                              "path": pname + (f" x{stages} stages" if path == 1 else ""), "ctas_per_sm": None,
                              "gbs": round(g, 1), "gbs_per_sm": round(g, 2)})
+    if not quick:
+        # what limits one CTA: bytes per copy and issuing threads per CTA (L2-resident 32 MiB and HBM)
+        for nbytes, kind in ((32 << 20, "l2"), (1 << 30, "hbm")):
+            passes = max(2, ((8 << 30) if kind == "l2" else (4 << 30)) // nbytes)
+            for chunk, stages, producers in ((4096, 12, 1), (8192, 12, 1), (32768, 6, 1), (65536, 3, 1),
+                                             (16384, 6, 2), (16384, 3, 4), (8192, 3, 8), (2048, 8, 8)):
+                for per_sm in (1, 2):
+                    if per_sm * stages * chunk * producers > 200 * 1024:
+                        continue
+                    g = P.preserve_measure_stream(big, nbytes, passes, 1, sms * per_sm, stages, chunk, status, stream,
+                                                  producers)
+                    rows.append({"buffer_mib": nbytes >> 20, "source": kind,
+                                 "path": f"cp.async.bulk {chunk} B x{stages} stages x{producers} threads",
+                                 "ctas_per_sm": per_sm, "gbs": round(g, 1), "gbs_per_sm": round(g / sms, 2)})
+            # issuing threads that are lanes of ONE warp
+            for chunk, stages, producers in ((16384, 3, 4), (8192, 3, 8)):
+                g = P.preserve_measure_stream(big, nbytes, passes, 2, sms, stages, chunk, status, stream, producers)
+                rows.append({"buffer_mib": nbytes >> 20, "source": kind,
+                             "path": f"cp.async.bulk {chunk} B x{stages} stages x{producers} lanes of one warp",
+                             "ctas_per_sm": 1, "gbs": round(g, 1), "gbs_per_sm": round(g / sms, 2)})
     assert int(status[0].item()) == 0
     del big
     return rows

@@ -374,13 +374,15 @@ PRESERVE_API int preserve_measure_read_bandwidth(const void *device_buffer, size
  * ramp and tail are paid once.  A buffer well inside L2 with many passes measures L2; a buffer
  * several times larger than L2 measures HBM; ctas = 1 measures what one SM can take in.
  * path 0: 128-bit read-only loads (256 threads, 8 loads in flight each); path 1: bulk async
- * copies of chunk_bytes (multiple of 1024) into a shared-memory ring with `stages` (1..12) copies
- * in flight per CTA, stages * chunk_bytes <= 200 KiB.  status_block: 64 zeroed device ints (the
+ * copies of chunk_bytes (multiple of 1024) issued by `producers` (1..8) threads per CTA, each
+ * keeping `stages` (1..12) copies in flight in its own shared-memory ring, stages * chunk_bytes *
+ * producers <= 200 KiB; path 2: the same with the issuing threads being lanes of one warp.
+ * status_block: 64 zeroed device ints (the
  * bounded waits of path 1 report there).  Writes GB/s to *gbs_out; synchronises `cuda_stream`;
  * allocates nothing. */
 PRESERVE_API int preserve_measure_stream(const void *device_buffer, size_t bytes, int32_t passes, int32_t path,
-                                         int32_t ctas, int32_t stages, uint32_t chunk_bytes, int32_t *status_block,
-                                         void *cuda_stream, float *gbs_out);
+                                         int32_t ctas, int32_t stages, uint32_t chunk_bytes, int32_t producers,
+                                         int32_t *status_block, void *cuda_stream, float *gbs_out);
 
 /* Frees everything the library allocated for the handle (NULL is allowed). */
 PRESERVE_API void preserve_layer_destroy(preserve_layer_t *layer);

@@ -107,7 +107,7 @@ def lib() -> C.CDLL:
         L.preserve_debug_set.argtypes = [C.c_void_p, C.c_int32, C.c_int64]
         L.preserve_attention_static_status.argtypes = []
         L.preserve_measure_stream.argtypes = [C.c_void_p, C.c_size_t, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
-                                              C.c_uint32, C.c_void_p, C.c_void_p, C.POINTER(C.c_float)]
+                                              C.c_uint32, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(C.c_float)]
         L.preserve_layer_get_info.argtypes = [C.c_void_p, C.POINTER(Info)]
         L.preserve_last_status.argtypes = [C.c_void_p]
         L.preserve_last_cuda_error.argtypes = [C.c_void_p]
@@ -324,12 +324,12 @@ def preserve_measure_read_bandwidth(buf, reps: int = 10, stream=None) -> float:
 
 
 def preserve_measure_stream(buf, n_bytes: int, passes: int, path: int, ctas: int, stages: int = 6,
-                            chunk_bytes: int = 16384, status=None, stream=None) -> float:
+                            chunk_bytes: int = 16384, status=None, stream=None, producers: int = 1) -> float:
     """GB/s of the single-launch streaming microbenchmark over the first n_bytes of `buf` (see preserve.h).
     `status`: CUDA int32 tensor of 64 zeros."""
     out = C.c_float()
-    _check(lib().preserve_measure_stream(_ptr(buf), n_bytes, passes, path, ctas, stages, chunk_bytes, _ptr(status),
-                                         _stream_ptr(stream), C.byref(out)), "preserve_measure_stream")
+    _check(lib().preserve_measure_stream(_ptr(buf), n_bytes, passes, path, ctas, stages, chunk_bytes, producers,
+                                         _ptr(status), _stream_ptr(stream), C.byref(out)), "preserve_measure_stream")
     return float(out.value)
 
 

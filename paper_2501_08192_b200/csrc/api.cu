@@ -1291,7 +1291,8 @@ int preserve_run_kernel(preserve_layer_t *L, const preserve_step_io_t *io, int32
     StepPlan pl;
     sp.first_of_call = 1;
     plan_step(L, sp, &pl);
-    rc = enqueue_step(L, sp, pl, true, static_cast<cudaStream_t>(cuda_stream));
+    // (early launch allowed: the buffers the kernel reads hold an earlier step's results by contract)
+    rc = enqueue_step(L, sp, pl, false, static_cast<cudaStream_t>(cuda_stream));
     L->only = -1;
     return rc;
 }

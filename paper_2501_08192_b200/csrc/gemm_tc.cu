@@ -8,8 +8,13 @@
 //
 // Per CTA: one 128-row tile of the packed weights (two for wide batches, sharing one activation
 // tile) x one slice of k.
-//   warp 0    : TMA producer - W tile (128 or 256 rows x 64, 128B swizzle) and x tile (2 NB x 64)
-//               into a multi-stage shared-memory ring, mbarrier full/empty
+//   warp 0 (+ lane 0 of the first one or two epilogue warps): TMA producers - W tile (128 or 256 rows
+//               x 64, 128B swizzle) and x tile (2 NB x 64) into a multi-stage shared-memory ring,
+//               mbarrier full/empty.  One thread can start a bulk copy only every ~0.4 us whatever
+//               its size (measured: a single issuing thread moves 43 GB/s in 16 KiB copies, 131 GB/s
+//               in 64 KiB copies, and threads of different warps add up), so one producer alone caps
+//               a CTA near 50-70 GB/s - below an SM's share of HBM; the ring's stage uses are
+//               therefore dealt round-robin to several issuing threads
 //   warp 1    : allocates TMEM, issues tcgen05.mma (kind::f16, bf16 in, fp32
 //               accumulate in TMEM), tcgen05.commit frees ring slots
 //   warps 2.. : epilogue (8 or 16 warps) - tcgen05.ld the accumulator (lane = output row; the warps of
@@ -35,6 +40,8 @@ namespace prsv {
 constexpr int kTcMaxStages = 12;
 constexpr int kTcMaxEpiWarps = 16;        // 2-4 per TMEM lane group: the epilogue is a chain of short dependent
                                           // operations per output, so its speed is set by how many warps run it
+constexpr int kTcMaxProducers = 3;        // issuing threads of the TMA ring: warp 0, and lane 0 of the first epilogue warps
+                                          // (which have nothing else to do until the accumulator is complete)
 constexpr int kTcMaxThreads = (2 + kTcMaxEpiWarps) * 32;
 constexpr int kTcBlockK = 64;
 constexpr int kTcTileM = 128;
@@ -56,6 +63,8 @@ struct GemmTcParams {
     int *status;
     long long *trace;
     int inject;         // test hook: the producer of CTA (0, 0) never fetches its first weight tile
+    int epi_warps;      // 8 or 16
+    int producers;      // 1..kTcMaxProducers threads that issue the ring's TMA loads (stage uses dealt round-robin)
 };
 
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr)
@@ -167,37 +176,46 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            // Weights never depend on earlier kernels, the activations do: fill the whole ring
-            // with weight tiles first (they stream in while the previous kernel finishes), then
-            // wait for the previous kernel and add the activation tiles.
-            const uint64_t pol = policy_evict_first();   // every weight byte is read once per step
-            const int n_kb = kb1 - kb0;
-            const int pre = n_kb < p.stages ? n_kb : p.stages;
-            for (int i = 0; i < pre; ++i) {
-                mbar_expect_tx(&full[i], stage_bytes);
-                if (p.inject == INJECT_TC_RING && i == 0 && tile == 0 && s == 0)
-                    continue;
-                tma_load_2d_hint(smem + (size_t)i * stage_bytes, &p.w_map, (kb0 + i) * kTcBlockK,
-                                 tile * p.mt * kTcTileM, &full[i], pol);
-            }
-            pdl_wait();
-            trace_waited(p.trace);
-            for (int i = 0; i < pre; ++i)
-                tma_load_2d(smem + (size_t)i * stage_bytes + a_bytes, &p.x_map, (kb0 + i) * kTcBlockK, 0, &full[i]);
-            uint32_t it = pre;
-            for (int kb = kb0 + pre; kb < kb1; ++kb, ++it) {
-                const int st = it % p.stages;
-                const uint32_t ph = (it / p.stages) & 1;
-                if (!mbar_wait(&empty[st], ph ^ 1, p.status, ST_TIMEOUT_EMPTY)) { poisoned = 1; break; }
-                uint8_t *a_dst = smem + (size_t)st * stage_bytes;
-                mbar_expect_tx(&full[st], stage_bytes);
-                tma_load_2d_hint(a_dst, &p.w_map, kb * kTcBlockK, tile * p.mt * kTcTileM, &full[st], pol);
-                tma_load_2d(a_dst + a_bytes, &p.x_map, kb * kTcBlockK, 0, &full[st]);
-            }
+    const bool is_epi = warp >= 2;
+    // ------------------------------------------------------------ TMA producers
+    // Weights never depend on earlier kernels, the activations do: fill the whole ring with
+    // weight tiles first (they stream in while the previous kernel finishes), then wait for the
+    // previous kernel and add the activation tiles.  Producer j of NP owns the stage uses
+    // it = j, j + NP, ...  (one thread each: lane 0 of warp 0, and of epilogue warps 2, 3).
+    auto run_producer = [&](int prod) {
+        const uint64_t pol = policy_evict_first();   // every weight byte is read once per step
+        const int NP = p.producers;
+        const int n_kb = kb1 - kb0;
+        const int pre = n_kb < p.stages ? n_kb : p.stages;
+        for (int i = prod; i < pre; i += NP) {
+            mbar_expect_tx(&full[i], stage_bytes);
+            if (p.inject == INJECT_TC_RING && i == 0 && tile == 0 && s == 0)
+                continue;
+            tma_load_2d_hint(smem + (size_t)i * stage_bytes, &p.w_map, (kb0 + i) * kTcBlockK,
+                             tile * p.mt * kTcTileM, &full[i], pol);
         }
+        pdl_wait();
+        if (prod == 0)
+            trace_waited(p.trace);
+        for (int i = prod; i < pre; i += NP)
+            tma_load_2d(smem + (size_t)i * stage_bytes + a_bytes, &p.x_map, (kb0 + i) * kTcBlockK, 0, &full[i]);
+        int it = prod;
+        while (it < pre)
+            it += NP;
+        for (; it < n_kb; it += NP) {
+            const int kb = kb0 + it;
+            const int st = it % p.stages;
+            const uint32_t ph = (uint32_t)(it / p.stages) & 1;
+            if (!mbar_wait(&empty[st], ph ^ 1, p.status, ST_TIMEOUT_EMPTY)) { poisoned = 1; break; }
+            uint8_t *a_dst = smem + (size_t)st * stage_bytes;
+            mbar_expect_tx(&full[st], stage_bytes);
+            tma_load_2d_hint(a_dst, &p.w_map, kb * kTcBlockK, tile * p.mt * kTcTileM, &full[st], pol);
+            tma_load_2d(a_dst + a_bytes, &p.x_map, kb * kTcBlockK, 0, &full[st]);
+        }
+    };
+    if (warp == 0) {
+        if (lane == 0)
+            run_producer(0);
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
@@ -232,14 +250,14 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     const int lane_grp = warp & 3;          // TMEM lanes this warp may read: 32 * (warp % 4)
     const int row = lane_grp * 32 + lane;   // row of the tile
     const int nchunks = p.NB / 16;
-    const int sub = warp >= 2 ? (warp - 2) >> 2 : 0;     // which of the lane group's warps this is
+    const int sub = is_epi ? (warp - 2) >> 2 : 0;        // which of the lane group's warps this is
     const int kSubs = ((int)blockDim.x / 32 - 2) / 4;    // warps per lane group
     const int par = lane & 1;
     // Rotary factors of this thread's first two finish iterations of a one-sided split-K reduction
     // (the iteration order is fixed: column pairs sub, sub + kSubs, ... of this rank's columns):
     // computed here, while the weights stream, instead of in the tail.
     float2 trig[2] = {make_float2(1.f, 0.f), make_float2(1.f, 0.f)};
-    if (warp >= 2 && KIND == EPI_QKV && p.splits > 1 && PUSH == 2) {
+    if (is_epi && KIND == EPI_QKV && p.splits > 1 && PUSH == 2) {
         // (bulk form: a warp's first item is column warp - 2 of this rank's mt * cols (m, column)
         // items, a lane's two pairs are rows 4 * lane .. 4 * lane + 3)
         const int cols = p.NB / p.splits;
@@ -250,7 +268,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             trig[0] = rope_trig(p.epi, tabs, tabs.pos[b], tile * p.mt + m, 2 * lane);
             trig[1] = rope_trig(p.epi, tabs, tabs.pos[b], tile * p.mt + m, 2 * lane + 1);
         }
-    } else if (warp >= 2 && KIND == EPI_QKV && p.splits > 1 && PUSH == 1) {
+    } else if (is_epi && KIND == EPI_QKV && p.splits > 1 && PUSH == 1) {
         const int cols = p.NB / p.splits, hp = cols / 2;
         int m = 0, c2 = sub;
         while (c2 >= hp) { c2 -= hp; ++m; }
@@ -275,8 +293,14 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             apply_epilogue_t<KIND>(p.epi, tabs, b, true, p.N, b, pair, v0, v1);
         }
     };
+    // the first epilogue warps lend their lane 0 to the ring (the warp reconverges behind the block)
+    if (is_epi && warp - 1 < p.producers) {
+        if (lane == 0)
+            run_producer(warp - 1);
+        __syncwarp();
+    }
     bool have = false;
-    if (warp >= 2) {
+    if (is_epi) {
         have = mbar_wait(&accum_bar, 0, p.status, ST_TIMEOUT_MMA);
         if (!have)
             poisoned = 1;
@@ -315,7 +339,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         cg::cluster_group cluster = cg::this_cluster();
         const int cols = p.NB / p.splits;
         float *recv = reinterpret_cast<float *>(smem + p.recv_off);
-        if (warp >= 2) {
+        if (is_epi) {
             // two chunks (four TMEM loads) in flight per wait
             const uint32_t red_row = smem_u32(red) + (uint32_t)row * 4u;
             for (int j = sub; j < p.mt * nchunks; j += 2 * kSubs) {
@@ -364,7 +388,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 poisoned = 1;
         }
         cluster_arrive_relaxed();
-        if (warp >= 2) {
+        if (is_epi) {
             // finish this rank's columns: one (m, column) item per warp and iteration, a lane takes
             // rows 4 * lane .. 4 * lane + 3 - two complete output pairs - with one 16-byte load per rank
             const int n_ew = kSubs * 4;
@@ -416,7 +440,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         const int cols = p.NB / p.splits;
         const uint32_t recv_a = smem_u32(smem + p.recv_off);
         const uint32_t src_stride = (uint32_t)p.mt * kTcTileM * cols * 4u;          // bytes per source rank
-        if (warp >= 2) {
+        if (is_epi) {
             for (int j = sub; j < p.mt * nchunks; j += kSubs) {
                 const int m = j / nchunks, c = j % nchunks;
                 float v[16];
@@ -483,7 +507,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         // from all ranks in rank order - so the reduction and the epilogue work are spread over the
         // whole cluster.
         cg::cluster_group cluster = cg::this_cluster();
-        if (warp >= 2) {
+        if (is_epi) {
             for (int j = sub; j < p.mt * nchunks; j += kSubs) {      // the lane group's warps share the chunks
                 const int m = j / nchunks, c = j % nchunks;
                 float v[16];
@@ -494,7 +518,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             }
         }
         cluster.sync();
-        if (warp >= 2) {
+        if (is_epi) {
             const float *remote[8];
 #pragma unroll
             for (int q = 0; q < 8; ++q)
@@ -554,7 +578,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 run(std::integral_constant<int, 8>());
         }
         cluster.sync();        // peers' shared memory must outlive the reads
-    } else if (warp >= 2) {
+    } else if (is_epi) {
         for (int j = sub; j < p.mt * nchunks; j += kSubs) {
             const int m = j / nchunks, c = j % nchunks;
             const int pair = ((tile * p.mt + m) * kTcTileM + row) >> 1;
@@ -690,6 +714,8 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     // epilogue warps: 16 when the CTA has the SM to itself and enough column pairs per thread to share,
     // else 8 (two CTAs per SM must share the registers)
     const int epi_warps = (per_sm == 1 && mt * (a.NB / splits) / 2 >= 8) ? 16 : 8;
+    p.epi_warps = epi_warps;
+    p.producers = stages < kTcMaxProducers ? stages : kTcMaxProducers;
     cfg.blockDim = dim3((2 + epi_warps) * 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;

@@ -41,6 +41,8 @@ struct StreamParams {
     int passes;
     uint32_t chunk;
     int stages;
+    int producers;       // path 1 / 2: issuing threads per CTA, each with its own ring and sub-slice
+    int same_warp;       // path 2: the issuing threads are lanes of one warp instead of lane 0 of several warps
     int *status;         // status block (bounded waits report here)
     unsigned *sink;
 };
@@ -71,30 +73,35 @@ __global__ void __launch_bounds__(256) k_stream_ld(const __grid_constant__ Strea
 }
 
 constexpr int kStreamMaxStages = 12;
-__global__ void __launch_bounds__(32) k_stream_bulk(const __grid_constant__ StreamParams p)
+constexpr int kStreamMaxProducers = 8;
+__global__ void __launch_bounds__(32 * kStreamMaxProducers) k_stream_bulk(const __grid_constant__ StreamParams p)
 {
     extern __shared__ uint8_t stream_smem_raw[];
-    uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(stream_smem_raw) + 127) & ~uintptr_t(127));
-    __shared__ uint64_t bars[kStreamMaxStages];
-    if (threadIdx.x != 0)
+    uint8_t *ring0 = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(stream_smem_raw) + 127) & ~uintptr_t(127));
+    __shared__ uint64_t bars[kStreamMaxProducers][kStreamMaxStages];
+    // issuing threads: lane 0 of `producers` warps, or (same_warp) lanes 0.. of warp 0
+    if (p.same_warp ? (int)threadIdx.x >= p.producers : (threadIdx.x & 31) != 0)
         return;
+    const int w = p.same_warp ? (int)threadIdx.x : (int)(threadIdx.x >> 5);
+    uint8_t *ring = ring0 + (size_t)w * p.stages * p.chunk;
     for (int i = 0; i < p.stages; ++i)
-        mbar_init(&bars[i], 1);
+        mbar_init(&bars[w][i], 1);
     mbar_fence_init();
-    const uint8_t *base = p.buf + (size_t)blockIdx.x * p.slice;
-    const size_t per_pass = p.slice / p.chunk;
+    const size_t sub = p.slice / p.producers;           // bytes per producer (multiple of chunk)
+    const uint8_t *base = p.buf + (size_t)blockIdx.x * p.slice + (size_t)w * sub;
+    const size_t per_pass = sub / p.chunk;
     const size_t total = per_pass * (size_t)p.passes;
     // keep `stages` copies in flight: wait for the oldest, issue the next into its slot
     for (size_t i = 0; i < total + p.stages; ++i) {
         const int st = (int)(i % p.stages);
         if (i >= (size_t)p.stages) {
             const uint32_t ph = (uint32_t)((i / p.stages - 1) & 1);
-            if (!mbar_wait(&bars[st], ph, p.status, ST_TIMEOUT_FULL))
+            if (!mbar_wait(&bars[w][st], ph, p.status, ST_TIMEOUT_FULL))
                 return;                                 // (copies in flight land in this CTA's memory at most)
         }
         if (i < total) {
-            mbar_expect_tx(&bars[st], p.chunk);
-            bulk_load(ring + (size_t)st * p.chunk, base + (i % per_pass) * p.chunk, p.chunk, &bars[st]);
+            mbar_expect_tx(&bars[w][st], p.chunk);
+            bulk_load(ring + (size_t)st * p.chunk, base + (i % per_pass) * p.chunk, p.chunk, &bars[w][st]);
         }
     }
 }
@@ -102,20 +109,24 @@ __global__ void __launch_bounds__(32) k_stream_bulk(const __grid_constant__ Stre
 }  // namespace prsv
 
 extern "C" int preserve_measure_stream(const void *device_buffer, size_t bytes, int32_t passes, int32_t path,
-                                       int32_t ctas, int32_t stages, uint32_t chunk_bytes, int32_t *status_block,
-                                       void *cuda_stream, float *gbs_out)
+                                       int32_t ctas, int32_t stages, uint32_t chunk_bytes, int32_t producers,
+                                       int32_t *status_block, void *cuda_stream, float *gbs_out)
 {
     using namespace prsv;
     if (!device_buffer || !gbs_out || !status_block || passes < 1 || passes > 100000 || ctas < 1 || ctas > 4096 ||
-        (path != 0 && path != 1) || (reinterpret_cast<uintptr_t>(device_buffer) & 127))
+        (path < 0 || path > 2) || (reinterpret_cast<uintptr_t>(device_buffer) & 127))
         return PRESERVE_EINVAL;
-    if (path == 1 && (stages < 1 || stages > kStreamMaxStages || chunk_bytes < 1024 || chunk_bytes % 1024 ||
-                      (size_t)stages * chunk_bytes > 200 * 1024))
+    if (path >= 1 && (stages < 1 || stages > kStreamMaxStages || chunk_bytes < 1024 || chunk_bytes % 1024 ||
+                      producers < 1 || producers > kStreamMaxProducers ||
+                      (size_t)stages * chunk_bytes * producers > 200 * 1024))
         return PRESERVE_EINVAL;
-    const uint32_t chunk = path == 1 ? chunk_bytes : 4096u;
+    const uint32_t chunk = path >= 1 ? chunk_bytes : 4096u;
+    const size_t unit = (size_t)chunk * (path >= 1 ? producers : 1);
     StreamParams p = {};
     p.buf = static_cast<const uint8_t *>(device_buffer);
-    p.slice = bytes / (size_t)ctas / chunk * chunk;
+    p.producers = path >= 1 ? producers : 1;
+    p.same_warp = path == 2;
+    p.slice = bytes / (size_t)ctas / unit * unit;
     if (p.slice == 0)
         return PRESERVE_EINVAL;
     p.passes = passes;
@@ -124,8 +135,8 @@ extern "C" int preserve_measure_stream(const void *device_buffer, size_t bytes, 
     p.status = status_block;
     p.sink = nullptr;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    const size_t smem = path == 1 ? (size_t)stages * chunk + 128 : 0;
-    if (path == 1) {
+    const size_t smem = path >= 1 ? (size_t)stages * chunk * producers + 128 : 0;
+    if (path >= 1) {
         static PerDeviceSize lim;
         if (ensure_dynamic_smem(k_stream_bulk, lim, smem) != cudaSuccess) {
             (void)cudaGetLastError();
@@ -143,7 +154,7 @@ extern "C" int preserve_measure_stream(const void *device_buffer, size_t bytes, 
         if (path == 0)
             k_stream_ld<<<ctas, 256, 0, s>>>(q);
         else
-            k_stream_bulk<<<ctas, 32, smem, s>>>(q);
+            k_stream_bulk<<<ctas, 32 * producers, smem, s>>>(q);
     };
     launch(1);                      // warm-up: brings a small buffer into L2, pages in the code
     cudaEventRecord(e0, s);

@@ -29,7 +29,6 @@ namespace prsv {
 
 constexpr int kPfThreads = 128;
 constexpr int kPfMaxRuns = 2 * 2048;     // {K, V} x (sequence, kv head) runs: the most a layer can have
-constexpr int kPfRunsPerThread = kPfMaxRuns / kPfThreads;
 
 struct PrefetchParams {
     PrefetchArgs a;
@@ -63,15 +62,19 @@ __device__ __forceinline__ uint64_t block_exclusive_scan(uint64_t v, uint64_t *w
 
 __global__ void __launch_bounds__(kPfThreads) k_prefetch_l2(const __grid_constant__ PrefetchParams p)
 {
-    // per run of the SelfAttention node: bytes to prefetch and the run's first chunk index
-    __shared__ uint32_t run_bytes[kPfMaxRuns];
-    __shared__ uint32_t run_chunk0[kPfMaxRuns + 1];
+    // per run of the SelfAttention node: bytes to prefetch and the run's first chunk index (dynamic
+    // shared memory sized to the launch's runs: a few hundred bytes for a small batch, so the CTAs
+    // fit beside the early-launched consumer kernels)
+    extern __shared__ uint32_t pf_smem[];
     __shared__ uint64_t warp_tot[kPfThreads / 32];
     __shared__ uint64_t take_s[kPfMaxNodes];
 
     const PrefetchArgs &a = p.a;
     const int kv_node = a.kv_node;                     // index of the SelfAttention node, or -1
     const int n_runs = kv_node >= 0 ? 2 * a.kv_count : 0;
+    uint32_t *run_bytes = pf_smem;
+    uint32_t *run_chunk0 = pf_smem + n_runs;
+    const int kPfRunsPerThread = (n_runs + kPfThreads - 1) / kPfThreads;
     const int r0 = threadIdx.x * kPfRunsPerThread;     // this thread's block of runs
 
     // ---- live bytes of every K / V run (run 2 i = K of stream i, run 2 i + 1 = V of stream i)
@@ -162,26 +165,21 @@ __global__ void __launch_bounds__(kPfThreads) k_prefetch_l2(const __grid_constan
             }
         }
     };
-    uint64_t first = 0;                                     // global chunk index of the node's first chunk
     for (int i = 0; i < a.n_nodes; ++i) {
         const uint64_t take = take_s[i];
         if (i != kv_node) {
             const uint64_t n_chunks = (take + chunk - 1) / chunk;
             const uint8_t *base = reinterpret_cast<const uint8_t *>(a.node[i].base);
-            // (start where the previous node's dealing left off, so the threads stay evenly loaded)
-            uint64_t c = (gtid + gthreads - first % gthreads) % gthreads;
-            for (; c < n_chunks; c += gthreads) {
+            for (uint64_t c = gtid; c < n_chunks; c += gthreads) {
                 const uint64_t off = c * chunk;
                 const uint64_t left = take - off;
                 touch(base + off, left < chunk ? (uint32_t)left : chunk);
             }
-            first += n_chunks;
         } else {
             const uint8_t *kb = reinterpret_cast<const uint8_t *>(a.node[i].base);
             const uint8_t *vb = reinterpret_cast<const uint8_t *>(a.node[i].base2);
             int r = 0;
-            uint64_t c = (gtid + gthreads - first % gthreads) % gthreads;
-            for (; c < kv_chunks; c += gthreads) {
+            for (uint64_t c = gtid; c < kv_chunks; c += gthreads) {
                 while (run_chunk0[r + 1] <= c)
                     ++r;
                 const uint64_t off = (c - run_chunk0[r]) * chunk;
@@ -189,7 +187,6 @@ __global__ void __launch_bounds__(kPfThreads) k_prefetch_l2(const __grid_constan
                 const uint8_t *ptr = ((r & 1) ? vb : kb) + (uint64_t)(r >> 1) * a.kv_stride + off;
                 touch(ptr, left < chunk ? (uint32_t)left : chunk);
             }
-            first += kv_chunks;
         }
     }
     // the load variant folds its values into a word that is stored only if it equals a magic number,
@@ -209,6 +206,7 @@ cudaError_t launch_prefetch(const PrefetchArgs &a, int ctas, cudaStream_t s, con
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ctas);
     cfg.blockDim = dim3(kPfThreads);
+    cfg.dynamicSmemBytes = a.kv_node >= 0 ? (size_t)(4 * a.kv_count + 1) * sizeof(uint32_t) : 0;
     cfg.stream = s;
     cfg.attrs = const_cast<cudaLaunchAttribute *>(attrs);
     cfg.numAttrs = n_attrs;
