@@ -458,6 +458,18 @@ def run_ours(args):
     if args.mode == "decode-loop":
         run_decode_loop(P, I, torch, args, stream)
         return
+    if args.mode == "real-window":
+        # the multi-GPU measurement alone (with one rank: a one-member group, which still runs every
+        # code path of it - exchange blocks, fused window, library all-reduce - on one GPU)
+        if world == 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", str(free_port()))
+            dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", local_rank))
+        out = bench_real_window(P, I, torch, dist, args, rank, local_rank, world, stream)
+        if rank == 0:
+            print(json.dumps({"mode": "real-window", "n_gpus": world, "real_window": out}), flush=True)
+        dist.destroy_process_group()
+        return
     if args.mode == "streams":
         rows = measure_streams(P, torch, stream, quick=False)
         print(json.dumps({"streams": rows}), flush=True)
@@ -509,6 +521,11 @@ def run_ours(args):
     }
     if "cpu_baseline" in h:
         out["cpu_baseline"] = h.pop("cpu_baseline")
+    if world > 1 and not args.no_real_window:
+        try:
+            out["real_window"] = bench_real_window(P, I, torch, dist, args, rank, local_rank, world, stream)
+        except Exception as e:      # noqa: BLE001  (the replicas' result above must survive)
+            out["real_window"] = {"error": f"{type(e).__name__}: {e}"}
     if rank == 0:
         print(json.dumps(out), flush=True)
         det = os.path.join(ROOT, "gpurun_out")
@@ -520,6 +537,152 @@ def run_ours(args):
 
 
 # ------------------------------------------------------------------------ other modes
+def bench_real_window(P, I, torch, dist, args, rank, local_rank, world, stream):
+    """N > 1: the communication window for real.  The ranks are the `world` shards of a
+    configs[1]-shaped layer (tp_degree = world) chained over a rotation of R layers; per layer-step
+    time with (a) the fused one-shot all-reduce window (peer reads in the window kernel), (b) the
+    library-collective baseline (NCCL all-reduce + a one-buffer window, kernels queued one by one)
+    and (c) the local stand-in, each with prefetch off / early launch only / on.  Every phase is
+    agreed on over a gloo control group first, so a rank that fails makes all ranks skip, not hang."""
+    from dataclasses import replace
+    from datetime import timedelta
+    from paper_2501_08192_b200 import comm as CM
+    ctrl = dist.new_group(backend="gloo", timeout=timedelta(seconds=120))
+
+    def all_ok(ok: bool) -> bool:
+        t = torch.tensor([1 if ok else 0], dtype=torch.int32)
+        dist.all_reduce(t, op=dist.ReduceOp.MIN, group=ctrl)
+        return bool(t.item())
+
+    res, err = {}, None
+    l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size
+    base = replace(I.CONFIGS[1], tp_degree=world, seed=I.CONFIGS[1].seed + 1000 * rank)
+    wl = wl1 = comm = None
+    try:
+        R = rotation_size(base, l2)
+        # (Workload indexes I.CONFIGS: build from a patched copy of configs[1])
+        saved = I.CONFIGS
+        I.CONFIGS = tuple(replace(c, tp_degree=world) if i == 1 else c for i, c in enumerate(saved))
+        try:
+            wl = Workload(P, I, torch, 1, rank, l2, R)
+            I.CONFIGS = tuple(replace(c, tp_degree=1) if i == 1 else c for i, c in enumerate(saved))
+            wl1 = Workload(P, I, torch, 1, rank, l2, R)
+        finally:
+            I.CONFIGS = saved
+        shape = wl.shape
+        comm = P.Comm(rank, world, shape.batch, shape.hidden)
+        handles = [None] * world
+        dist.all_gather_object(handles, (rank, comm.export_handle()), group=ctrl)
+        for r, h in handles:
+            if r != rank:
+                comm.import_handle(r, h)
+        comm.write(0, wl.ios[0]._keep[4][0])          # the first window A reads the exchange buffers
+        torch.cuda.synchronize()
+    except Exception as e:      # noqa: BLE001
+        err = f"setup: {type(e).__name__}: {e}"
+    if not all_ok(err is None):
+        return {"skipped": err or "another rank failed during setup"}
+
+    def timed(step_fn, steps):
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                step_fn()
+        torch.cuda.synchronize()
+        dist.barrier(group=ctrl)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for _ in range(steps):
+                step_fn()
+            e1.record(stream)
+        torch.cuda.synchronize()
+        dist.barrier(group=ctrl)
+        t = torch.tensor([e0.elapsed_time(e1) / steps], dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX, group=ctrl)
+        return float(t.item())
+
+    steps = max(3, math.ceil(MIN_LAYER_STEPS / wl.R))
+    default_budget = int(wl.layers[0].get_info().prefetch_budget)
+    settings = (("off", 0), ("early_launch_only", 1), ("on_l2_sixteenth", l2 // 16), ("on_l2_quarter", l2 // 4))
+
+    def fused_step():
+        P.preserve_decode_chain(wl.layers, wl.ios, link=False, stream=stream)
+
+    def standin_step():
+        P.preserve_decode_chain(wl.layers, wl.ios, link=False, stream=stream)
+
+    nccl_bufs = []
+
+    def nccl_step():
+        for L, io, (mlp_sum, attn_sum) in zip(wl1.layers, wl1.ios, nccl_bufs):
+            dist.all_reduce(mlp_sum)
+            for k in range(5):
+                L.run_kernel(io, k, stream)
+            dist.all_reduce(attn_sum)
+            for k in range(5, 8):
+                L.run_kernel(io, k, stream)
+
+    try:
+        # (c) the local stand-in first (no communication at all)
+        row = {}
+        for name, b in settings:
+            wl.set_budget(b)
+            row[name + "_us_per_layer"] = round(timed(standin_step, steps) * 1e3 / wl.R, 3)
+        res["local_stand_in"] = row
+        # (a) fused peer-read window
+        for L in wl.layers:
+            L.set_comm(comm)
+        row = {}
+        for name, b in settings:
+            wl.set_budget(b)
+            row[name + "_us_per_layer"] = round(timed(fused_step, steps) * 1e3 / wl.R, 3)
+        # measured length of the real window (wait return to end of the window kernels, traced)
+        for L in wl.layers:
+            L.set_trace(True)
+        wl.set_budget(1)
+        with torch.cuda.stream(stream):
+            fused_step()
+        torch.cuda.synchronize()
+        tr = [L.read_trace() for L in wl.layers[1:]]
+        row["window_a_us"] = round(float(np.mean([t_[0][3] - t_[0][2] for t_ in tr])) / 1e3, 2)
+        row["window_b_us"] = round(float(np.mean([t_[5][3] - t_[5][2] for t_ in tr])) / 1e3, 2)
+        for L in wl.layers:
+            L.set_trace(False)
+        row["device_status_code"] = max(L.last_status_code() for L in wl.layers)
+        res["fused_peer_read_window"] = row
+        for L in wl.layers:
+            L.set_comm(None)
+        # (b) NCCL all-reduce + one-buffer window: layer j's window A reads the all-reduced MLP partial
+        # sums of the layer before it in the rotation (reduced in place in that layer's output buffer),
+        # its window B the all-reduced attention partial sums (reduced in place in its own buffer)
+        n1 = len(wl1.layers)
+        attn_bufs = [torch.zeros_like(io._keep[10]) for io in wl1.ios]
+        new_ios = []
+        for j, (L, io) in enumerate(zip(wl1.layers, wl1.ios)):
+            mlp_sum = wl1.ios[(j - 1) % n1]._keep[10]       # mlp_partial_out of the previous layer
+            new_ios.append(L.make_io(wl1.shape.batch, io._keep[3], io._keep[2], [mlp_sum], [], io._keep[6],
+                                     io._keep[7], io._keep[8], io._keep[9], io._keep[10], attn_bufs[j]))
+            L.set_external_attention_sum(attn_bufs[j])
+            nccl_bufs.append((mlp_sum, attn_bufs[j]))
+        wl1.ios = new_ios
+        row = {}
+        for name, b in settings:
+            wl1.set_budget(b)
+            row[name + "_us_per_layer"] = round(timed(nccl_step, steps) * 1e3 / wl1.R, 3)
+        res["nccl_allreduce_window"] = row
+    except Exception as e:      # noqa: BLE001
+        err = f"{type(e).__name__}: {e}"
+        res["error"] = err
+    res["workload"] = (f"{world} shards of a configs[1]-shaped layer (tp_degree {world}), rotation of {wl.R} layers, "
+                       f"{steps * wl.R} layer-steps per setting, time = slowest rank")
+    for w_ in (wl, wl1):
+        if w_ is not None:
+            w_.close()
+    if comm is not None:
+        comm.close()
+    return res
+
+
 def run_timeline(P, I, torch, args, stream):
     """Per-kernel timeline of one layer-step from the in-kernel global-timer trace, averaged over
     many cold steps: for each main-stream kernel, when its first CTA started, when the wait on its
@@ -686,13 +849,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--config", type=int, default=-1,
                     help="index into the five benchmark configurations (default: all five, configs[3] as the headline)")
-    ap.add_argument("--mode", default="bench", choices=("bench", "timeline", "decode-loop", "streams"))
+    ap.add_argument("--mode", default="bench", choices=("bench", "timeline", "decode-loop", "streams", "real-window"))
     ap.add_argument("--layers", type=int, default=32, help="decode-loop mode: layers of the chain")
     ap.add_argument("--rotation", type=int, default=0, help="layer instances per step (0 = sized from L2)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-kernels", action="store_true", help="skip the isolated per-kernel timing")
     ap.add_argument("--budget-bytes", type=int, default=-1, help="prefetch budget per window (default: the library's)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--no-real-window", action="store_true",
+                    help="N > 1: skip the measurement of the real communication window")
     ap.add_argument("--dry-run", action="store_true", help="launch plumbing only (CPU, gloo); nothing is timed")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)

@@ -279,6 +279,12 @@ PRESERVE_API int preserve_layer_get_info(const preserve_layer_t *layer, preserve
 PRESERVE_API int preserve_last_status(preserve_layer_t *layer);
 PRESERVE_API int preserve_clear_status(preserve_layer_t *layer);
 
+/* The raw device status word behind preserve_last_status (synchronises the device): 0 ok;
+ * 1 a wait for operand bytes (TMA / bulk copy / cluster hand-over) gave up; 2 a wait for a free
+ * ring slot; 3 a wait for the tensor-core accumulator or a cluster reduction; 4 tensor memory;
+ * 5 device ctx_len beyond the host copy; 6 a peer rank never announced its exchange buffer. */
+PRESERVE_API int preserve_last_status_code(preserve_layer_t *layer);
+
 /* Graphs captured so far by calls whose first (or only) layer is this handle.  Replays of
  * a cached graph do not count: a decode loop whose contexts advance should see this number
  * grow only when the attention work split changes (about once per 64 tokens at most). */
@@ -360,6 +366,55 @@ PRESERVE_API int preserve_attention_static(const void *q_hi, const void *q_lo, c
                                            int32_t n_kv_heads, int32_t kv_capacity, void *o_hi, void *o_lo,
                                            void *cuda_stream);
 PRESERVE_API int preserve_attention_static_status(void);
+
+/* ---- The real communication window (one process per GPU; Section 2, "Multi-device inference":
+ * one all-reduce of a [batch, hidden] tensor per attention block and one per MLP block).
+ *
+ * A preserve_comm_t owns this rank's EXCHANGE BLOCK in device memory: its two partial-sum buffers
+ * (window A: what its down projection produced; window B: what its output projection produced),
+ * arrival flags and epoch counters.  preserve_comm_create allocates the block on the current
+ * device (n_ranks <= 8); the ranks then exchange 64-byte handles (preserve_comm_export on the
+ * owner, preserve_comm_import on every other rank; how the bytes travel is the caller's business -
+ * the Python layer uses torch.distributed), which maps every peer's block into this process (CUDA
+ * IPC, peer access enabled lazily).  Inside ONE process, preserve_comm_set_peer connects blocks
+ * directly.  All peers must be connected before preserve_layer_set_comm.
+ *
+ * With a comm attached (n_ranks must equal tp_degree), a step's two windows become one-shot
+ * all-reduces fused into the window kernel: the output / down projections also write this rank's
+ * bf16 partial sums into its exchange buffers; each window kernel, once its own buffer is complete,
+ * stores the window's epoch number into every peer's flag block, waits - bounded by the handle's
+ * wait limit, PRESERVE_ETIMEOUT / status code 6 if a peer never arrives - until every peer has done
+ * the same, then reads all n_ranks buffers through the peer mappings with plain 128-bit loads and
+ * adds them in rank order (identical bits on every rank), adds the residual and normalises.
+ * io->partials_in and io->attn_peer_partials are then ignored.  Window A of a step reads what the
+ * down projection of the step before wrote (for the very first step: what preserve_comm_write put
+ * there).  Every rank must queue the same sequence of steps.  Several layers may share one comm.
+ * No multicast and no bulk / TMA copy ever touches a peer's memory.
+ *
+ * preserve_comm_write: copy `bytes` of device data into this rank's own buffer of `window` (0 = A,
+ * 1 = B), asynchronously on the stream.  preserve_comm_epoch: windows of that kind this rank has
+ * completed (synchronises).  preserve_comm_debug_arrive (tests on one GPU, where no second rank
+ * runs): marks `from_rank` as having announced every window up to `epoch` in this rank's flag
+ * block, from the host. */
+typedef struct preserve_comm preserve_comm_t;
+PRESERVE_API int preserve_comm_create(int32_t rank, int32_t n_ranks, int32_t max_batch, int32_t hidden,
+                                      preserve_comm_t **out);
+PRESERVE_API int preserve_comm_export(const preserve_comm_t *comm, void *handle64);
+PRESERVE_API int preserve_comm_import(preserve_comm_t *comm, int32_t peer_rank, const void *handle64);
+PRESERVE_API int preserve_comm_set_peer(preserve_comm_t *comm, int32_t peer_rank, const preserve_comm_t *peer);
+PRESERVE_API int preserve_comm_write(preserve_comm_t *comm, int32_t window, const void *src_device, size_t bytes,
+                                     void *cuda_stream);
+PRESERVE_API int preserve_comm_debug_arrive(preserve_comm_t *comm, int32_t window, int32_t from_rank, uint32_t epoch);
+PRESERVE_API int64_t preserve_comm_epoch(preserve_comm_t *comm, int32_t window);
+PRESERVE_API void preserve_comm_destroy(preserve_comm_t *comm);
+PRESERVE_API int preserve_layer_set_comm(preserve_layer_t *layer, preserve_comm_t *comm_or_null);
+
+/* For a window whose all-reduce the CALLER performs (the library-collective baseline): window B
+ * then takes `reduced_attn_partial` (device bf16 [batch, hidden], e.g. the NCCL all-reduce of
+ * attn_partial_out) as its partial 0 instead of this shard's own result; NULL restores the
+ * default.  The caller runs the step kernel by kernel (preserve_run_kernel) and reduces between
+ * the output projection (4) and window B (5).  Not together with a comm. */
+PRESERVE_API int preserve_layer_set_external_attention_sum(preserve_layer_t *layer, const void *reduced_attn_partial);
 
 /* Read-bandwidth microbenchmark (the read roofline next to the copy-bandwidth figure): streams
  * `bytes` (>= 1 MiB, 16-byte aligned) of the caller's device buffer `reps` times (1..1000) with

@@ -31,6 +31,9 @@ EXPORTS = (
     "preserve_set_window_delay_ns", "preserve_attention_static",
     "preserve_measure_read_bandwidth", "preserve_set_prefetch_mechanism", "preserve_clear_status",
     "preserve_graph_captures", "preserve_debug_set", "preserve_attention_static_status", "preserve_plan_graph", "preserve_measure_stream",
+    "preserve_last_status_code", "preserve_comm_create", "preserve_comm_export", "preserve_comm_import",
+    "preserve_comm_set_peer", "preserve_comm_write", "preserve_comm_debug_arrive", "preserve_comm_epoch",
+    "preserve_comm_destroy", "preserve_layer_set_comm", "preserve_layer_set_external_attention_sum",
 )
 NODE_COMM, NODE_MATMUL, NODE_ATTENTION, NODE_OTHER = 0, 1, 2, 3
 TRACE_SLOTS = 8
@@ -108,6 +111,19 @@ def lib() -> C.CDLL:
         L.preserve_attention_static_status.argtypes = []
         L.preserve_measure_stream.argtypes = [C.c_void_p, C.c_size_t, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                               C.c_uint32, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(C.c_float)]
+        L.preserve_last_status_code.argtypes = [C.c_void_p]
+        L.preserve_comm_create.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_void_p)]
+        L.preserve_comm_export.argtypes = [C.c_void_p, C.c_void_p]
+        L.preserve_comm_import.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
+        L.preserve_comm_set_peer.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
+        L.preserve_comm_write.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.preserve_comm_debug_arrive.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_uint32]
+        L.preserve_comm_epoch.argtypes = [C.c_void_p, C.c_int32]
+        L.preserve_comm_epoch.restype = C.c_int64
+        L.preserve_comm_destroy.argtypes = [C.c_void_p]
+        L.preserve_comm_destroy.restype = None
+        L.preserve_layer_set_comm.argtypes = [C.c_void_p, C.c_void_p]
+        L.preserve_layer_set_external_attention_sum.argtypes = [C.c_void_p, C.c_void_p]
         L.preserve_layer_get_info.argtypes = [C.c_void_p, C.POINTER(Info)]
         L.preserve_last_status.argtypes = [C.c_void_p]
         L.preserve_last_cuda_error.argtypes = [C.c_void_p]
@@ -277,6 +293,19 @@ class Layer:
     def last_status(self) -> int:
         return int(lib().preserve_last_status(self.handle))
 
+    def last_status_code(self) -> int:
+        return int(lib().preserve_last_status_code(self.handle))
+
+    def set_comm(self, comm) -> None:
+        _check(lib().preserve_layer_set_comm(self.handle, comm.handle if comm is not None else None),
+               "preserve_layer_set_comm")
+        self._comm = comm
+
+    def set_external_attention_sum(self, t) -> None:
+        _check(lib().preserve_layer_set_external_attention_sum(self.handle, _ptr(t)),
+               "preserve_layer_set_external_attention_sum")
+        self._ext = t
+
     def clear_status(self) -> None:
         _check(lib().preserve_clear_status(self.handle), "preserve_clear_status")
 
@@ -308,6 +337,50 @@ def preserve_attention_static(q_hi, q_lo, k_cache, v_cache, ctx_len_dev, ctx_len
     return int(lib().preserve_attention_static(_ptr(q_hi), _ptr(q_lo), _ptr(k_cache), _ptr(v_cache),
                                                _ptr(ctx_len_dev), ctx_len_host.ctypes.data, batch, n_q_heads,
                                                n_kv_heads, cap, _ptr(o_hi), _ptr(o_lo), _stream_ptr(stream)))
+
+
+class Comm:
+    """Owns one preserve_comm_t: this rank's exchange block of the real communication window."""
+
+    def __init__(self, rank: int, n_ranks: int, max_batch: int, hidden: int):
+        h = C.c_void_p()
+        _check(lib().preserve_comm_create(rank, n_ranks, max_batch, hidden, C.byref(h)), "preserve_comm_create")
+        self.handle, self.rank, self.n_ranks = h, rank, n_ranks
+        self._peers = []
+
+    def export_handle(self) -> bytes:
+        buf = (C.c_uint8 * 64)()
+        _check(lib().preserve_comm_export(self.handle, buf), "preserve_comm_export")
+        return bytes(buf)
+
+    def import_handle(self, peer_rank: int, handle: bytes) -> None:
+        buf = (C.c_uint8 * 64)(*handle)
+        _check(lib().preserve_comm_import(self.handle, peer_rank, buf), "preserve_comm_import")
+
+    def set_peer(self, peer: "Comm") -> None:
+        _check(lib().preserve_comm_set_peer(self.handle, peer.rank, peer.handle), "preserve_comm_set_peer")
+        self._peers.append(peer)
+
+    def write(self, window: int, t, stream=None) -> None:
+        _check(lib().preserve_comm_write(self.handle, window, _ptr(t), t.numel() * t.element_size(),
+                                         _stream_ptr(stream)), "preserve_comm_write")
+
+    def debug_arrive(self, window: int, from_rank: int, epoch: int) -> None:
+        _check(lib().preserve_comm_debug_arrive(self.handle, window, from_rank, epoch), "preserve_comm_debug_arrive")
+
+    def epoch(self, window: int) -> int:
+        return int(lib().preserve_comm_epoch(self.handle, window))
+
+    def close(self) -> None:
+        if self.handle:
+            lib().preserve_comm_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def preserve_attention_static_status() -> int:

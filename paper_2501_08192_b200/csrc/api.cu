@@ -120,6 +120,8 @@ struct preserve_layer {
     int pf_mechanism;            // prefetch kernel: 0 bulk L2 prefetch, 1 per-line hints, 2 plain loads
     uint32_t pf_chunk;           // bytes per prefetch instruction
     int inject;                  // test hook (prsv::Inject): one producer withholds one issue
+    preserve_comm *comm;         // real communication window (NULL: the local stand-in)
+    const void *ext_attn_sum;    // window B's partial 0 comes from this caller-reduced buffer instead of the own result
     uint64_t n_captures;         // graphs captured so far by calls whose first layer is this handle
 
     size_t budget;
@@ -510,6 +512,23 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
         w.pdl = pdl && !(direct && sp.first_of_call);
         w.inputs_after_wait = sp.late_a;
         w.inject = L->inject == INJECT_WINDOW_HANDOVER ? INJECT_WINDOW_HANDOVER : INJECT_NONE;
+        w.comm_rank = -1;
+        if (L->comm) {
+            // the real window: the ranks' exchange buffers instead of the step's partial-sum inputs
+            CommView cv;
+            if (!comm_fill(L->comm, 0, &cv))
+                return PRESERVE_EINVAL;
+            for (int i = 0; i < cv.n_ranks; ++i) {
+                w.parts[i] = cv.buf[i];
+                w.comm_flags_peer[i] = cv.flags[i];
+            }
+            w.part0_is_f32 = 0;
+            w.comm_rank = cv.rank;
+            w.comm_window = 0;
+            w.comm_flags_local = cv.flags[cv.rank];
+            w.comm_epoch = cv.epoch;
+            w.comm_done = cv.done;
+        }
         CK(L, launch_window(w, s));
     }
     // ---- QKV projection + rotary embedding + KV append
@@ -562,6 +581,12 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
         e.out = nullptr;
         e.out2 = sp.attn_partial_out;
         e.out_f32 = L->attn_f32;
+        if (L->comm) {
+            CommView cv;
+            if (!comm_fill(L->comm, 1, &cv))
+                return PRESERVE_EINVAL;
+            e.out = cv.buf[cv.rank];      // this rank's attention partial sums, for every rank's window B
+        }
         int rc = launch_gemm(L, 1, L->o, B, e, pdl, s, TRACE(4));
         if (rc)
             return rc;
@@ -601,6 +626,26 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
         w.status = L->status;
         w.pdl = pdl;
         w.inputs_after_wait = sp.late_b;
+        w.comm_rank = -1;
+        if (L->ext_attn_sum) {
+            w.parts[0] = L->ext_attn_sum;     // reduced by the caller (e.g. a library all-reduce) beforehand
+            w.part0_is_f32 = 0;
+        }
+        if (L->comm) {
+            CommView cv;
+            if (!comm_fill(L->comm, 1, &cv))
+                return PRESERVE_EINVAL;
+            for (int i = 0; i < cv.n_ranks; ++i) {
+                w.parts[i] = cv.buf[i];
+                w.comm_flags_peer[i] = cv.flags[i];
+            }
+            w.part0_is_f32 = 0;
+            w.comm_rank = cv.rank;
+            w.comm_window = 1;
+            w.comm_flags_local = cv.flags[cv.rank];
+            w.comm_epoch = cv.epoch;
+            w.comm_done = cv.done;
+        }
         CK(L, launch_window(w, s));
     }
     // ---- gate/up projection + SwiGLU, down projection
@@ -620,6 +665,12 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
         e.kind = EPI_PLAIN;
         e.out = sp.mlp_partial_out;
         e.out_f32 = L->mlp_f32;
+        if (L->comm) {
+            CommView cv;
+            if (!comm_fill(L->comm, 0, &cv))
+                return PRESERVE_EINVAL;
+            e.out2 = cv.buf[cv.rank];     // this rank's MLP partial sums, for every rank's next window A
+        }
         int rc = launch_gemm(L, 3, L->a, B, e, pdl, s, TRACE(7));
         if (rc)
             return rc;
@@ -674,6 +725,8 @@ void step_signature(const preserve_layer *L, const StepPtrs &sp, const StepPlan 
     put((uint64_t)L->prefetch_ctas);
     put((uint64_t)pl.attn_grid | (uint64_t)pl.attn_tpi << 32);
     put((uint64_t)pl.attn_items_per_stream);
+    putp(L->comm);
+    putp(L->ext_attn_sum);
 }
 
 // Run `n` steps (already validated) as one replayed graph, or directly.
@@ -1059,6 +1112,34 @@ int preserve_clear_status(preserve_layer_t *L)
     return PRESERVE_OK;
 }
 
+int preserve_layer_set_comm(preserve_layer_t *L, preserve_comm_t *comm)
+{
+    if (!L)
+        return PRESERVE_EINVAL;
+    if (comm) {
+        CommView cv;
+        if (!comm_fill(comm, 0, &cv))
+            return PRESERVE_EINVAL;                 // not every peer connected
+        if (cv.n_ranks != L->cfg.tp_degree || comm_hidden(comm) != L->cfg.hidden ||
+            comm_max_batch(comm) < L->cfg.max_batch)
+            return PRESERVE_ESHAPE;
+        if (L->ext_attn_sum)
+            return PRESERVE_EINVAL;
+    }
+    L->comm = comm;
+    return PRESERVE_OK;
+}
+
+int preserve_layer_set_external_attention_sum(preserve_layer_t *L, const void *reduced_attn_partial)
+{
+    if (!L || (reduced_attn_partial && L->comm))
+        return PRESERVE_EINVAL;
+    if (reduced_attn_partial && !aligned16(reduced_attn_partial))
+        return PRESERVE_EALIGN;
+    L->ext_attn_sum = reduced_attn_partial;
+    return PRESERVE_OK;
+}
+
 int64_t preserve_graph_captures(const preserve_layer_t *L) { return L ? (int64_t)L->n_captures : -1; }
 
 int preserve_set_window_delay_ns(preserve_layer_t *L, int32_t ns)
@@ -1358,6 +1439,17 @@ int preserve_last_status(preserve_layer_t *L)
     int st = 0;
     CK(L, cudaMemcpy(&st, L->status, sizeof(int), cudaMemcpyDeviceToHost));
     return st == ST_OK ? PRESERVE_OK : (st == ST_ITEMS_OVERFLOW ? PRESERVE_ESHAPE : PRESERVE_ETIMEOUT);
+}
+
+int preserve_last_status_code(preserve_layer_t *L)
+{
+    if (!L)
+        return PRESERVE_EINVAL;
+    CK(L, cudaSetDevice(L->dev));
+    CK(L, cudaDeviceSynchronize());
+    int st = 0;
+    CK(L, cudaMemcpy(&st, L->status, sizeof(int), cudaMemcpyDeviceToHost));
+    return st;
 }
 
 int preserve_last_cuda_error(const preserve_layer_t *L) { return L ? L->last_cuda : 0; }

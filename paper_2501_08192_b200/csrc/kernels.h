@@ -64,7 +64,7 @@ enum Inject : int { INJECT_NONE = 0, INJECT_WINDOW_HANDOVER = 1, INJECT_GEMV_RIN
 // prefetch kernel's load variant, [16..27] the prefetch kernels' own evaluation of the plan
 // (uint64 [2][3], written by CTA 0 of each prefetch launch).
 enum : int { ST_OK = 0, ST_TIMEOUT_FULL = 1, ST_TIMEOUT_EMPTY = 2, ST_TIMEOUT_MMA = 3, ST_TIMEOUT_TMEM = 4,
-             ST_ITEMS_OVERFLOW = 5 };
+             ST_ITEMS_OVERFLOW = 5, ST_TIMEOUT_PEER = 6 };
 constexpr int kStatusLimitWord = 2, kStatusSinkWord = 8, kStatusPlanWord = 16;
 
 constexpr int kMaxParts = 16;   // most partial-sum buffers in one window
@@ -91,6 +91,16 @@ struct WindowArgs {
     int inputs_after_wait;         // the step's input buffers may still be written by an earlier kernel of the
                                    // same call: read them only after the dependency wait
     int inject;                    // test hook (Inject)
+    // Real communication window (one process per GPU): parts[] are the ranks' exchange buffers in rank
+    // order (peer-mapped pointers, this rank's own included), all bf16.  After the dependency wait
+    // the kernel tells every peer that this rank's buffer is complete, waits (bounded) until every
+    // peer has said the same, and only then reads.  comm_rank < 0: no communication.
+    int comm_rank;
+    int comm_window;                       // 0 / 1: which of the layer's two windows (selects the flag row)
+    const uint32_t *comm_flags_local;      // this rank's flag block: uint32 [2][kMaxParts]
+    uint32_t *comm_flags_peer[16];         // every rank's flag block, by rank
+    uint32_t *comm_epoch;                  // this rank's count of completed windows of this kind (device)
+    unsigned *comm_done;                   // CTA ticket of the launch (device)
 };
 cudaError_t launch_window(const WindowArgs &a, cudaStream_t s);
 
@@ -210,6 +220,21 @@ struct PrefetchArgs {
     int *sink;              // scratch word for the load variant (practically never written)
     unsigned long long *plan_out;   // optional: device uint64[kPfMaxNodes], receives the bytes taken per node
 };
+// ---- exchange memory of the real communication window (comm.cu)
+struct CommView {
+    int rank, n_ranks;
+    uint8_t *buf[kMaxParts];      // every rank's exchange buffer of one window, by rank (peer-mapped)
+    uint32_t *flags[kMaxParts];   // every rank's flag block
+    uint32_t *epoch;              // own counters of that window
+    unsigned *done;
+};
+}  // namespace prsv
+struct preserve_comm;
+namespace prsv {
+bool comm_fill(const preserve_comm *c, int window, CommView *v);   // false until every peer is connected
+int comm_hidden(const preserve_comm *c);
+int comm_max_batch(const preserve_comm *c);
+
 // ---- Algorithm 1 over an explicit operator graph (planner.cu; host only).  Successors in CSR form.
 struct PlanHit { int comm, node; uint64_t bytes; };      // prefetch `bytes` of `node` beside communication op `comm`
 int plan_graph(int n_nodes, const int32_t *kind, const uint64_t *mem_bytes, const int32_t *succ_off,

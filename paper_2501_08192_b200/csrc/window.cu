@@ -44,14 +44,54 @@ struct WindowParams {
     int *status;
     int no_hint;         // LEAN: do not even hint the inputs into L2 before the wait (another kernel of the call still writes them)
     int inject;          // test hook: rank 1 of every row withholds its hand-over to rank 0
+    // real communication window (COMM instantiation only)
+    int comm_rank, comm_window;
+    const uint32_t *comm_flags_local;
+    uint32_t *comm_flags_peer[kMaxParts];
+    uint32_t *comm_epoch;
+    unsigned *comm_done;
 };
+
+// Loads and stores of the arrival protocol between GPUs (system scope).
+__device__ __forceinline__ uint32_t ld_acquire_sys(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_sys(uint32_t *p, uint32_t v)
+{
+    asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// 128-bit load that is performed at the memory it names every time (a peer's buffer changes from
+// step to step and must never be served from a stale line of this GPU's caches).
+__device__ __forceinline__ uint4 ld_volatile_v4(const void *p)
+{
+    uint4 r;
+    asm volatile("ld.volatile.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p)
+                 : "memory");
+    return r;
+}
 
 // (One instantiation for all four input forms: the two windows of a layer then run the same
 // instructions, which the second finds in the instruction caches.)
 // LEAN, for big batches (hundreds of CTAs): one chunk per thread and the step's input buffers are only
 // hinted into L2 before the wait and loaded after it, so that a CTA holds few registers while it
 // waits - the grid then fits beside the early-launched GEMM CTAs in one wave instead of several.
-template <bool LEAN>
+// COMM: the real communication window - the partial-sum buffers are the ranks' exchange buffers
+// (one-shot all-reduce: every rank reads every rank's buffer through peer-mapped pointers with plain
+// 128-bit loads and adds them in rank order, so all ranks obtain the same bits).  Arrival protocol,
+// all in this kernel: after the dependency wait (own buffer complete) CTA 0 stores this window's
+// epoch number into every peer's flag block (release, system scope); every CTA then polls its own
+// GPU's flag block until all peers' entries have reached the epoch (acquire, system scope; bounded -
+// a peer that never arrives makes the wait give up with a status code, the kernel still returns).
+// The epoch is a device counter that the last CTA of the launch advances, so a replayed graph
+// needs no new arguments.  Buffers are reused window after window: a rank overwrites its window-A
+// buffer only after it has passed window B of the same layer, by which time every peer has
+// announced its window-B buffer and therefore finished reading window A.
+template <bool LEAN, bool COMM = false>
 __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_constant__ WindowParams p)
 {
     constexpr int kWinMaxChunks = LEAN ? 1 : prsv::kWinMaxChunks;
@@ -102,11 +142,11 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     if (j < p.n_parts && !(PART0_F32 && j == 0))
-                        pre[c][j] = ld_stream(p.parts[j] + row_off + ch);
+                        pre[c][j] = COMM ? ld_volatile_v4(p.parts[j] + row_off + ch) : ld_stream(p.parts[j] + row_off + ch);
             }
         }
     };
-    if constexpr (LEAN) {
+    if constexpr (LEAN && !COMM) {
         // one hint per 128-byte line (8 threads share a line)
         if (!p.no_hint && (threadIdx.x & 7) == 0 && (int)threadIdx.x < chunks) {
             if (!RESID_F32)
@@ -115,7 +155,7 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
                 if (!(PART0_F32 && j == 0))
                     line_prefetch_l2(p.parts[j] + row_off + threadIdx.x);
         }
-    } else {
+    } else if constexpr (!LEAN) {
         load_inputs();
     }
 
@@ -125,6 +165,38 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
     pdl_wait();                // this shard's own partial sum comes from the preceding kernel in the stream
     trace_waited(p.trace);
     const long long t_begin = p.delay_ns ? gtime() : 0;   // the modelled collective starts when its inputs exist
+    if constexpr (COMM) {
+        __shared__ uint32_t epoch_s;
+        if (threadIdx.x == 0)
+            epoch_s = *reinterpret_cast<volatile uint32_t *>(p.comm_epoch) + 1u;
+        __syncthreads();
+        const uint32_t epoch = epoch_s;
+        const int t = threadIdx.x;
+        if (t < p.n_parts && t != p.comm_rank) {
+            if (blockIdx.x == 0) {
+                __threadfence_system();          // own buffer (written by the kernel before) before the flag
+                st_release_sys(p.comm_flags_peer[t] + p.comm_window * kMaxParts + p.comm_rank, epoch);
+            }
+            const uint32_t *flag = p.comm_flags_local + p.comm_window * kMaxParts + t;
+            const long long t0 = clock64();
+            long long limit = kFastWaitCycles;
+            bool arrived = false, asked = false;
+            for (;;) {
+                if ((int32_t)(ld_acquire_sys(flag) - epoch) >= 0) { arrived = true; break; }
+                if (clock64() - t0 >= limit) {
+                    if (asked)
+                        break;
+                    limit = *reinterpret_cast<volatile long long *>(p.status + kStatusLimitWord);
+                    if (limit <= 0 || limit > kMaxWaitCycles)
+                        limit = kMaxWaitCycles;
+                    asked = true;
+                }
+            }
+            if (!arrived)
+                atomicCAS(p.status, ST_OK, ST_TIMEOUT_PEER);
+        }
+        __syncthreads();
+    }
     if constexpr (LEAN)
         load_inputs();
 
@@ -251,6 +323,18 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
             p.x_bf16[p.x_plane + row_off + ch] = lo;
         }
     }
+    if constexpr (COMM) {
+        // the last CTA of the launch to get here advances this window's epoch
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const unsigned ticket = atomicAdd(p.comm_done, 1u);
+            if (ticket == gridDim.x - 1) {
+                *p.comm_done = 0u;
+                __threadfence();
+                atomicAdd(p.comm_epoch, 1u);
+            }
+        }
+    }
     trace_end(p.trace);
 }
 
@@ -280,11 +364,21 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
     const int chunks = a.H / 8 / cl;
     // LEAN (inputs read after the wait) for big batches, and whenever an input buffer may still be
     // written by an earlier kernel of the same call
-    const bool lean = (a.B * cl > 256 || a.inputs_after_wait) && chunks <= 512;
-    if (a.inputs_after_wait && !lean)
+    const bool comm = a.comm_rank >= 0;
+    const bool lean = (a.B * cl > 256 || a.inputs_after_wait || comm) && chunks <= 512;
+    if ((a.inputs_after_wait || comm) && !lean)
+        return cudaErrorInvalidValue;
+    if (comm && (a.n_parts > 8 || a.part0_is_f32 || a.comm_rank >= a.n_parts))
         return cudaErrorInvalidValue;
     p.no_hint = a.inputs_after_wait;
     p.inject = a.inject;
+    p.comm_rank = a.comm_rank;
+    p.comm_window = a.comm_window;
+    p.comm_flags_local = a.comm_flags_local;
+    for (int i = 0; i < kMaxParts; ++i)
+        p.comm_flags_peer[i] = a.comm_flags_peer[i];
+    p.comm_epoch = a.comm_epoch;
+    p.comm_done = a.comm_done;
     int threads = (chunks + kWinMaxChunks - 1) / kWinMaxChunks;
     if (chunks <= 512)
         threads = chunks;
@@ -309,8 +403,10 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
     cfg.numAttrs = n_attr;
     p.resid_f32 = a.resid_is_f32;
     p.part0_f32 = a.part0_is_f32;
-    return lean ? cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<true>, p)
-                : cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<false>, p);
+    if (comm)
+        return cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<true, true>, p);
+    return lean ? cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<true, false>, p)
+                : cudaLaunchKernelEx(&cfg, k_window_reduce_rmsnorm<false, false>, p);
 }
 
 }  // namespace prsv

@@ -78,3 +78,65 @@ def test_bench_byte_accounting_matches_the_library():
     src = open(os.path.join(ROOT, "bench.py")).read()
     ref = src[src.index("def run_reference"):src.index("def main")]
     assert "binding" not in ref and "libpreserve" not in ref
+
+
+# ------------------------------------------------ host protocol of the real communication window
+class _FakeComm:
+    """Stands in for binding.Comm on the CPU: handles are 64 recognisable bytes."""
+
+    def __init__(self, rank, n_ranks):
+        self.rank, self.n_ranks, self.imported = rank, n_ranks, {}
+
+    def export_handle(self):
+        return bytes([self.rank + 1]) * 64
+
+    def import_handle(self, r, h):
+        assert r != self.rank and r not in self.imported
+        self.imported[r] = h
+
+
+def _comm_worker(rank: int, world: int, port: int, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    from datetime import timedelta
+    dist.init_process_group("gloo", rank=rank, world_size=world, timeout=timedelta(seconds=20))
+    from paper_2501_08192_b200 import comm as CM
+    c = _FakeComm(rank, world)
+    CM.connect(c)
+    out[("imported", rank)] = {r: h[0] for r, h in c.imported.items()}
+    guard = CM.StepGuard(CM.control_group(10.0), timeout_s=2.0)
+    # two steps with everybody present; then the last rank leaves BETWEEN steps (nothing in flight)
+    events = []
+    for _ in range(2):
+        events.append(guard.begin_step())
+    if rank == world - 1:
+        out[("events", rank)] = events + ["left"]
+        os._exit(0)                     # gone without a goodbye
+    try:
+        guard.begin_step()
+        events.append("no error")
+    except CM.PeerLost as e:
+        events.append("peer lost")
+        out[("message", rank)] = str(e)
+    out[("events", rank)] = events
+    os._exit(0)                          # (a normal shutdown would wait for the rank that left)
+
+
+def test_exchange_block_handles_travel_and_a_leaving_rank_is_noticed_on_the_host():
+    world, port = 3, 29547
+    mgr = mp.Manager()
+    out = mgr.dict()
+    ctx = mp.get_context("spawn")
+    procs = [ctx.Process(target=_comm_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    for p in procs:
+        p.join(timeout=120)
+        assert p.exitcode == 0
+    for rank in range(world):
+        # every rank mapped every other rank's block, with that rank's handle
+        assert out[("imported", rank)] == {r: r + 1 for r in range(world) if r != rank}
+    assert out[("events", world - 1)] == [1, 2, "left"]
+    # the survivors got a clean error at the next step, not a hang
+    assert out[("events", 0)] == [1, 2, "peer lost"]
+    assert "step 2" in out[("message", 0)]
+    assert out[("events", 1)][:2] == [1, 2] and out[("events", 1)][2] in ("peer lost", "no error")
