@@ -257,6 +257,15 @@ PRESERVE_API int preserve_profile_step(preserve_layer_t *layer, const preserve_s
 PRESERVE_API int preserve_run_kernel(preserve_layer_t *layer, const preserve_step_io_t *io, int32_t which,
                                      void *cuda_stream);
 
+/* Queue only the L2 prefetch that belongs beside window `window` (0: {Wqkv, K/V, Wo}; 1: {Wgate|up,
+ * Wdown}; planned against the budget as in a full step) on the layer's side stream, forked from
+ * `cuda_stream` at this point.  For a caller that runs the communication itself (a library
+ * all-reduce between kernels queued with preserve_run_kernel): call this right before the
+ * collective, the place Algorithm 1 inserts the prefetch operator.  The side stream is joined
+ * again by preserve_run_kernel of the block's last kernel (4 for window 0, 7 for window 1). */
+PRESERVE_API int preserve_prefetch_window(preserve_layer_t *layer, const preserve_step_io_t *io, int32_t window,
+                                          void *cuda_stream);
+
 /* Timeline trace (diagnostics).  While on, every main-stream kernel of a step records, over all
  * its CTAs, PRESERVE_TRACE_SLOTS values in nanoseconds of the GPU's global timer: {earliest
  * start, earliest and latest return from the wait on the previous kernel, latest end, latest

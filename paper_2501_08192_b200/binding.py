@@ -34,6 +34,7 @@ EXPORTS = (
     "preserve_last_status_code", "preserve_comm_create", "preserve_comm_export", "preserve_comm_import",
     "preserve_comm_set_peer", "preserve_comm_write", "preserve_comm_debug_arrive", "preserve_comm_epoch",
     "preserve_comm_destroy", "preserve_layer_set_comm", "preserve_layer_set_external_attention_sum",
+    "preserve_prefetch_window",
 )
 NODE_COMM, NODE_MATMUL, NODE_ATTENTION, NODE_OTHER = 0, 1, 2, 3
 TRACE_SLOTS = 8
@@ -98,6 +99,7 @@ def lib() -> C.CDLL:
         L.preserve_decode_step_host.argtypes = [C.c_void_p, C.POINTER(HostIO), C.c_void_p]
         L.preserve_profile_step.argtypes = [C.c_void_p, C.POINTER(StepIO), C.c_void_p, C.POINTER(C.c_float)]
         L.preserve_run_kernel.argtypes = [C.c_void_p, C.POINTER(StepIO), C.c_int32, C.c_void_p]
+        L.preserve_prefetch_window.argtypes = [C.c_void_p, C.POINTER(StepIO), C.c_int32, C.c_void_p]
         L.preserve_set_trace.argtypes = [C.c_void_p, C.c_int32]
         L.preserve_read_trace.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
         L.preserve_attention_static.argtypes = [C.c_void_p] * 6 + [C.c_int32] * 4 + [C.c_void_p] * 3
@@ -274,6 +276,10 @@ class Layer:
 
     def run_kernel(self, io: StepIO, which: int, stream=None) -> None:
         _check(lib().preserve_run_kernel(self.handle, C.byref(io), which, _stream_ptr(stream)), "preserve_run_kernel")
+
+    def prefetch_window(self, io: StepIO, window: int, stream=None) -> None:
+        _check(lib().preserve_prefetch_window(self.handle, C.byref(io), window, _stream_ptr(stream)),
+               "preserve_prefetch_window")
 
     def set_trace(self, on: bool) -> None:
         _check(lib().preserve_set_trace(self.handle, 1 if on else 0), "preserve_set_trace")

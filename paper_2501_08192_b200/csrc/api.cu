@@ -350,7 +350,7 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
         // down projection start only when it ends and would fetch their first tiles from idle HBM
         // after that; the gate/up CTAs request them into L2 as soon as their own stream is over.
         // (Not when a single kernel is run alone for timing: nothing would consume the bytes.)
-        if (which == 2 && L->only < 0 && L->budget > 0 && !L->no_early && L->wbytes[3] <= L->l2_bytes / 4) {
+        if (which == 2 && L->only == -1 && L->budget > 0 && !L->no_early && L->wbytes[3] <= L->l2_bytes / 4) {
             a.next_w = L->arena + L->off[3];
             a.next_bytes = (size_t)L->wbytes[3];
         }
@@ -393,8 +393,9 @@ void plan_step(preserve_layer *L, const StepPtrs &sp, StepPlan *pl)
     // budget 0 = vanilla execution: every kernel starts after its predecessor has completed and
     // nothing is fetched ahead of the dependency
     pl->pdl = (L->budget > 0 && !L->no_early) ? 1 : 0;
-    pl->pf_a = L->only < 0 && pl->planned[0][0] + pl->planned[0][1] + pl->planned[0][2] > 0;
-    pl->pf_b = L->only < 0 && pl->planned[1][0] + pl->planned[1][1] > 0;
+    // (only == -1: the whole step; -2 / -3: just the prefetch beside window A / B; k >= 0: just kernel k)
+    pl->pf_a = (L->only == -1 || L->only == -2) && pl->planned[0][0] + pl->planned[0][1] + pl->planned[0][2] > 0;
+    pl->pf_b = (L->only == -1 || L->only == -3) && pl->planned[1][0] + pl->planned[1][1] > 0;
     plan_attention(sp.ctx_len_host, B, c.n_kv_heads, L->sm_count, &pl->attn_grid, &pl->attn_tpi);
     pl->attn_items_per_stream = (int)((max_tiles_seq + pl->attn_tpi - 1) / pl->attn_tpi);
     // (the merge kernel sizes its CTAs from this, between 4 and 32 warps: clamp here so that the
@@ -416,7 +417,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
             L->planned[w][j] = pl.planned[w][j];
     const int pdl = pl.pdl;
     const bool pf_a = pl.pf_a, pf_b = pl.pf_b;
-#define WANT(k) (L->only < 0 || L->only == (k))
+#define WANT(k) (L->only == -1 || L->only == (k))
 #define TRACE(k) (L->tracing ? L->trace_buf + PRESERVE_TRACE_SLOTS * (k) : nullptr)
 
     // ---- K/V tensor maps
@@ -1374,6 +1375,28 @@ int preserve_run_kernel(preserve_layer_t *L, const preserve_step_io_t *io, int32
     plan_step(L, sp, &pl);
     // (early launch allowed: the buffers the kernel reads hold an earlier step's results by contract)
     rc = enqueue_step(L, sp, pl, false, static_cast<cudaStream_t>(cuda_stream));
+    L->only = -1;
+    if (rc == PRESERVE_OK && (which == 4 || which == 7) && L->side_pending) {
+        // a prefetch queued by preserve_prefetch_window for this block: joined where the block ends
+        preserve_layer *one[1] = {L};
+        rc = join_side_streams(one, 1, static_cast<cudaStream_t>(cuda_stream));
+    }
+    return rc;
+}
+
+int preserve_prefetch_window(preserve_layer_t *L, const preserve_step_io_t *io, int32_t window, void *cuda_stream)
+{
+    if (window != 0 && window != 1)
+        return PRESERVE_EINVAL;
+    StepPtrs sp = {};
+    int rc = check_step(L, io, &sp);
+    if (rc)
+        return rc;
+    L->only = window == 0 ? -2 : -3;
+    StepPlan pl;
+    sp.first_of_call = 1;
+    plan_step(L, sp, &pl);
+    rc = enqueue_step(L, sp, pl, true, static_cast<cudaStream_t>(cuda_stream));
     L->only = -1;
     return rc;
 }
