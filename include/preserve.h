@@ -191,7 +191,12 @@ PRESERVE_API int preserve_layer_init(const preserve_layer_config_t *cfg, const p
  * while the window runs, in two tiers: (1) the consumer kernels are launched early
  * (programmatic dependent launch) and stage the leading part of their weights / cached
  * K and V in shared memory before they wait for the window's result; (2) a side-stream
- * kernel prefetches the planned byte ranges, up to this limit per window, into L2. */
+ * kernel prefetches the planned byte ranges, up to this limit per window, into L2.
+ * The library's default is PRESERVE_BUDGET_EARLY_LAUNCH_ONLY: tier 1 alone, which is the fastest
+ * setting measured with the single-GPU stand-in windows (they last a few microseconds, too short
+ * for off-chip memory to be idle); give a real budget (a sixteenth to a quarter of the L2 size)
+ * where the communication window lasts 10 us or more. */
+#define PRESERVE_BUDGET_EARLY_LAUNCH_ONLY ((size_t)1)   /* any budget below 128 bytes plans nothing for L2 */
 PRESERVE_API int preserve_set_prefetch_bytes(preserve_layer_t *layer, size_t bytes_per_window);
 
 /* How the side-stream kernel brings the planned bytes into L2: mechanism 0 =

@@ -935,7 +935,10 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     L->pf_chunk = 4096;
     L->prefetch_ctas = 128;
     L->budget_is_default = true;
-    L->budget = (size_t)L->l2_bytes / 16;
+    // Measured on all five benchmark configurations with the bare stand-in windows (a few
+    // microseconds): early launch alone is the fastest setting; the side-stream L2 kernel costs
+    // 1-9 % there and only pays once a window lasts >= ~10 us.  So the default plans nothing for L2.
+    L->budget = PRESERVE_BUDGET_EARLY_LAUNCH_ONLY;
     L->plan_mode = PRESERVE_PLAN_TRUNCATE;
 
 #define CKI(expr)                                   \

@@ -48,6 +48,7 @@ class Op:
     prefetchable: float = 0.0     # read-only operand bytes (weights, or cached K and V): Algorithm 1's memSize
     other_bytes: float = 0.0      # activations read and written (never prefetched)
     comm_bytes: float = 0.0       # payload of a collective
+    overhead: float = 0.0         # seconds of fixed cost of this operator on top of Hardware.kernel_overhead
 
 
 def allreduce_time(hw: Hardware, nbytes: float) -> float:
@@ -60,10 +61,10 @@ def allreduce_time(hw: Hardware, nbytes: float) -> float:
 
 def op_time(hw: Hardware, op: Op, l2_hit_bytes: float = 0.0) -> float:
     if op.kind == "comm":
-        return allreduce_time(hw, op.comm_bytes) + hw.kernel_overhead
+        return allreduce_time(hw, op.comm_bytes) + hw.kernel_overhead + op.overhead
     hit = min(l2_hit_bytes, op.prefetchable)
     mem = (op.prefetchable - hit + op.other_bytes) / hw.hbm_bw + hit / hw.l2_bw
-    return max(op.flops / hw.flops, mem) + hw.kernel_overhead
+    return max(op.flops / hw.flops, mem) + hw.kernel_overhead + op.overhead
 
 
 def layer_ops(hidden: int, n_q_heads: int, n_kv_heads: int, head_dim: int, ffn: int, batch: int, sum_ctx: int,
@@ -138,6 +139,21 @@ def predict(hw: Hardware, ops: Sequence[Op], budget: float = None, truncate: boo
     return {"off": off, "early_launch_only": early, "on": on, "speedup_on_vs_off": off / on,
             "speedup_on_vs_early": early / on,
             "prefetched_bytes": float(sum(hits.values())), "planned_bytes": float(sum(sum(v.values()) for v in plan.values()))}
+
+
+def calibrate_overheads(hw: Hardware, ops: Sequence[Op], measured_seconds: Sequence[float]) -> List[Op]:
+    """Per-operator fixed cost from measured durations of the operators run alone (cold L2):
+    overhead = measured - (the model's compute / memory term), never negative.  The calibrated
+    operators reproduce the measured times without prefetching; what the model then predicts is
+    the effect of moving bytes into L2."""
+    out = []
+    for op, t in zip(ops, measured_seconds):
+        if op.kind == "comm":
+            out.append(replace(op, overhead=0.0))
+            continue
+        base = op_time(replace(hw, kernel_overhead=0.0), replace(op, overhead=0.0))
+        out.append(replace(op, overhead=max(t - base - hw.kernel_overhead, 0.0)))
+    return out
 
 
 def l2_size_sweep(hw: Hardware, ops: Sequence[Op], sizes_mib: Sequence[float]) -> List[Dict[str, float]]:
