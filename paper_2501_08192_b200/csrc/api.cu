@@ -220,7 +220,7 @@ void plan_window(const uint64_t *node_bytes, int n, uint64_t budget, int mode, u
     for (int i = 0; i < n; ++i)
         out[i] = 0;
     for (int i = 0; i < n; ++i) {
-        if (cache_sum + node_bytes[i] < budget) {       // strict, as in the listing
+        if (cache_sum + node_bytes[i] < budget) {       // strict: a node that makes cacheSum reach C is not inserted (Algorithm 1)
             cache_sum += node_bytes[i];
             out[i] = node_bytes[i];
         } else {
