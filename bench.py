@@ -283,10 +283,11 @@ def bench_config(P, I, torch, dist, args, idx, rank, local_rank, world, stream, 
             ms, _ = time_steps(chain_step, n_short, 3)
             sweep.append({"frac_of_l2": round(f, 4), "us_per_layer": round(us(ms), 3)})
         # modelled communication latency added to every window (the single-GPU stand-in has none)
-        for delay_us in (10, 20):
+        for delay_us in (10, 20, 40):
             wl.set_delay(delay_us * 1000)
             row = {"window_delay_us": delay_us}
-            for name, b in (("off", 0), ("early_launch_only", 1), ("on_sixteenth_l2", l2 // 16), ("on_quarter_l2", l2 // 4)):
+            for name, b in (("off", 0), ("early_launch_only", 1), ("on_sixteenth_l2", l2 // 16), ("on_quarter_l2", l2 // 4),
+                            ("on_half_l2", l2 // 2)):
                 wl.set_budget(b)
                 ms, _ = time_steps(chain_step, n_short, 3)
                 row[name + "_us_per_layer"] = round(us(ms), 3)
@@ -402,7 +403,7 @@ def bench_config(P, I, torch, dist, args, idx, rank, local_rank, world, stream, 
                                                                             window_time=win + d_ * 1e-6)["on"]),
                                       "on_quarter_l2_us": us_(M.predict(hw, ops, budget=l2 // 4, truncate=True,
                                                                         window_time=win + d_ * 1e-6)["on"])}
-                                     for d_ in (10, 20)]}
+                                     for d_ in (10, 20, 40)]}
         res["model"] = model
     except Exception as e:      # noqa: BLE001
         res["model"] = {"error": str(e)}

@@ -72,7 +72,7 @@ class HostIO(C.Structure):
 class Info(C.Structure):
     _fields_ = [("sm_count", C.c_int32), ("l2_bytes", C.c_int32), ("max_persisting_l2_bytes", C.c_int32),
                 ("max_access_window_bytes", C.c_int32), ("uses_tensor_path", C.c_int32),
-                ("activation_rows", C.c_int32), ("plan_mode", C.c_int32), ("reserved", C.c_int32),
+                ("activation_rows", C.c_int32), ("plan_mode", C.c_int32), ("normed_activations_fp16", C.c_int32),
                 ("prefetch_budget", C.c_uint64),
                 ("weight_bytes", C.c_uint64 * 4), ("kv_bytes", C.c_uint64),
                 ("planned_bytes", (C.c_uint64 * 3) * 2), ("algorithmic_bytes", C.c_uint64)]

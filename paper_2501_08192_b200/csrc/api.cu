@@ -328,6 +328,12 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
         a.trace = trace;
         a.pdl = pdl;
         a.inject = L->inject == INJECT_TC_RING && which == 0 ? INJECT_TC_RING : INJECT_NONE;
+        // The gate/up projection takes its input as one fp16 plane (an RMSNorm output is bounded, and 11
+        // significant bits keep the SwiGLU output well inside the tolerance): half the activation
+        // traffic and half the MMA work of the largest GEMM.  The QKV projection keeps hi + lo bf16
+        // planes: rounding of q is amplified by the softmax (measured: one fp16 plane put the 70B-shaped
+        // chain's attention partial sums at 1.02 of the bound).
+        a.x_fp16 = which == 2 ? 1 : 0;
         CK(L, launch_gemm_tc(a, L->sm_count, s));
         return PRESERVE_OK;
     }
@@ -501,6 +507,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
         w.h_f32 = L->h_f32;
         w.h_bf16 = nullptr;
         w.x_bf16 = L->x;
+        w.x_fp16 = 0;
         w.x_plane_elems = (size_t)L->rows * H;
         w.B = B; w.H = H;
         w.trace = TRACE(0);
@@ -620,6 +627,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
         w.h_f32 = L->h2_f32;
         w.h_bf16 = sp.residual_out;
         w.x_bf16 = L->x2;
+        w.x_fp16 = L->tensor_path ? 1 : 0;
         w.x_plane_elems = (size_t)L->rows * H;
         w.B = B; w.H = H;
         w.trace = TRACE(5);
@@ -980,10 +988,11 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
         const void *s_dn[1] = {w->w_down};
         const int c_dn[1] = {H};
         auto pack = L->tensor_path ? launch_pack_rows : launch_pack_gemv;
-        CKI(pack(s_qkv, c_qkv, 3, d.k[0], EPI_QKV, L->arena + L->off[0], nullptr));
-        CKI(pack(s_o, c_o, 1, d.k[1], EPI_PLAIN, L->arena + L->off[1], nullptr));
-        CKI(pack(s_gu, c_gu, 2, d.k[2], EPI_SWIGLU, L->arena + L->off[2], nullptr));
-        CKI(pack(s_dn, c_dn, 1, d.k[3], EPI_PLAIN, L->arena + L->off[3], nullptr));
+        // (tensor path: Wgate|up meets the fp16 RMSNorm output x2 and is stored as fp16)
+        CKI(pack(s_qkv, c_qkv, 3, d.k[0], EPI_QKV, L->arena + L->off[0], 0, nullptr));
+        CKI(pack(s_o, c_o, 1, d.k[1], EPI_PLAIN, L->arena + L->off[1], 0, nullptr));
+        CKI(pack(s_gu, c_gu, 2, d.k[2], EPI_SWIGLU, L->arena + L->off[2], 1, nullptr));
+        CKI(pack(s_dn, c_dn, 1, d.k[3], EPI_PLAIN, L->arena + L->off[3], 0, nullptr));
     }
     // rotary frequencies theta^(-2i/d)
     {
@@ -1030,8 +1039,10 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
         // activations as the B operand: [2 * nb_pad, K] = hi rows then lo rows, one box covers both
         const void *xb[4] = {L->x, L->o, L->x2, L->a};
         for (int i = 0; i < 4; ++i) {
+            // x2 (the MLP's RMSNorm output) is one fp16 plane; x, o and a are two bf16 planes (hi rows, lo rows)
+            const uint32_t brows = (uint32_t)(i == 2 ? L->nb_pad : 2 * L->nb_pad);
             if (!make_map_2d(&L->wmap[i], L->arena + L->off[i], d.k[i], d.n[i], 64, 128) ||
-                !make_map_2d(&L->xmap[i], xb[i], d.k[i], 2 * (uint64_t)L->nb_pad, 64, 2 * L->nb_pad)) {
+                !make_map_2d(&L->xmap[i], xb[i], d.k[i], brows, 64, brows)) {
                 preserve_layer_destroy(L);
                 return PRESERVE_EARCH;
             }
@@ -1445,6 +1456,7 @@ int preserve_layer_get_info(const preserve_layer_t *L, preserve_info_t *info)
     info->uses_tensor_path = L->tensor_path ? 1 : 0;
     info->activation_rows = L->rows;
     info->plan_mode = L->plan_mode;
+    info->normed_activations_fp16 = L->tensor_path ? 1 : 0;
     info->prefetch_budget = L->budget;
     for (int i = 0; i < 4; ++i)
         info->weight_bytes[i] = L->wbytes[i];

@@ -29,6 +29,7 @@
 // poisons the rest of the CTA's work, and the CTA still reaches every barrier
 // and frees its TMEM.
 #include <cooperative_groups.h>
+#include <cstdlib>
 #include <type_traits>
 
 #include "epilogue.cuh"
@@ -63,6 +64,7 @@ struct GemmTcParams {
     int *status;
     long long *trace;
     int inject;         // test hook: the producer of CTA (0, 0) never fetches its first weight tile
+    int planes;         // activation planes in the B operand: 2 = bf16 hi + lo, 1 = a single fp16 plane
     int epi_warps;      // 8 or 16
     int producers;      // 1..kTcMaxProducers threads that issue the ring's TMA loads (stage uses dealt round-robin)
 };
@@ -139,7 +141,8 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     const int tile = blockIdx.x;
     const int s = blockIdx.y;
     const int a_bytes = p.mt * kATileBytes;
-    const int stage_bytes = a_bytes + 2 * p.NB * kTcBlockK * 2;
+    const int stage_bytes = a_bytes + p.planes * p.NB * kTcBlockK * 2;
+    const int acc_cols = p.planes * p.NB;      // TMEM columns of one weight tile's accumulator
     const int kb0 = (int)((long long)p.kblocks * s / p.splits);
     const int kb1 = (int)((long long)p.kblocks * (s + 1) / p.splits);
 
@@ -233,7 +236,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                     const uint64_t adesc = make_smem_desc(a_addr + m * kATileBytes);
 #pragma unroll
                     for (int k = 0; k < kTcBlockK / 16; ++k)
-                        tc_mma(tmem_base + m * 2 * p.NB, adesc + 2 * k, bdesc + 2 * k, p.idesc,
+                        tc_mma(tmem_base + m * acc_cols, adesc + 2 * k, bdesc + 2 * k, p.idesc,
                                (kb > kb0 || k > 0) ? 1u : 0u);
                 }
                 tc_commit(&empty[st]);      // slot is free once these MMAs have read it
@@ -314,8 +317,14 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     auto load_chunk = [&](int m, int c, float (&v)[16]) {
         if (have) {
             uint32_t hi[16], lo[16];
-            tc_ld16_issue(t_lane + m * 2 * p.NB + c * 16, hi);
-            tc_ld16_issue(t_lane + m * 2 * p.NB + p.NB + c * 16, lo);
+            tc_ld16_issue(t_lane + m * acc_cols + c * 16, hi);
+            if (p.planes == 2) {
+                tc_ld16_issue(t_lane + m * acc_cols + p.NB + c * 16, lo);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    lo[i] = 0u;
+            }
             tc_ld_wait(hi, lo);
 #pragma unroll
             for (int i = 0; i < 16; ++i)
@@ -349,10 +358,16 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 const int m1 = two ? j1 / nchunks : m0, c1 = two ? j1 % nchunks : c0;
                 uint32_t h0[16], l0[16], h1[16], l1[16];
                 if (have) {
-                    tc_ld16_issue(t_lane + m0 * 2 * p.NB + c0 * 16, h0);
-                    tc_ld16_issue(t_lane + m0 * 2 * p.NB + p.NB + c0 * 16, l0);
-                    tc_ld16_issue(t_lane + m1 * 2 * p.NB + c1 * 16, h1);
-                    tc_ld16_issue(t_lane + m1 * 2 * p.NB + p.NB + c1 * 16, l1);
+                    tc_ld16_issue(t_lane + m0 * acc_cols + c0 * 16, h0);
+                    tc_ld16_issue(t_lane + m1 * acc_cols + c1 * 16, h1);
+                    if (p.planes == 2) {
+                        tc_ld16_issue(t_lane + m0 * acc_cols + p.NB + c0 * 16, l0);
+                        tc_ld16_issue(t_lane + m1 * acc_cols + p.NB + c1 * 16, l1);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            l0[i] = l1[i] = 0u;
+                    }
                     tc_ld_wait4(h0, l0, h1, l1);
                 } else {
 #pragma unroll
@@ -637,6 +652,8 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     p.status = a.status;
     p.trace = a.trace;
     p.inject = a.inject;
+    const int planes = a.x_fp16 ? 1 : 2;
+    p.planes = planes;
     // Two 128-row weight tiles per CTA share one activation tile when the batch is wide enough for
     // the activation tile (2 * NB rows) to weigh as much as a weight tile: halves the L2->SM traffic
     // of the activations, which every CTA re-reads.
@@ -645,7 +662,7 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     if (mt == 2)
         p.w_map = *a.w_map256;
     const int tiles = a.N / (kTcTileM * mt);
-    const int stage_bytes = mt * kATileBytes + 2 * a.NB * kTcBlockK * 2;
+    const int stage_bytes = mt * kATileBytes + planes * a.NB * kTcBlockK * 2;
     // Ring depth, CTAs per SM and cluster splits.  Two CTAs per SM (rings <= 100 KiB) whenever that
     // leaves >= 4 stages: measured better than one CTA with a ring twice as deep, because the second
     // CTA streams while the first is in its epilogue.  The grid (tiles x splits) must fit the
@@ -673,9 +690,13 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     p.stages = stages;
     p.splits = splits;
     int cols = 32;
-    while (cols < mt * 2 * a.NB) cols *= 2;
+    while (cols < mt * planes * a.NB) cols *= 2;
     p.tmem_cols = cols;
-    p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * a.NB) >> 3) << 17) | ((uint32_t)(kTcTileM >> 4) << 24);
+    // instruction descriptor: fp32 accumulate; A (weights) and B (activations) in the same 16-bit format -
+    // both bf16 (B = hi + lo planes) or both fp16 (B = one plane); N = columns of the B tile, M = 128
+    const uint32_t fmt = a.x_fp16 ? 0u : 1u;
+    p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)((planes * a.NB) >> 3) << 17) |
+              ((uint32_t)(kTcTileM >> 4) << 24);
 
     // one-sided split-K reduction when the receive area (one partial tile per CTA) is small - every
     // thread then hands over one or two 16-byte pieces per owner; wide batches keep the pull form,

@@ -81,7 +81,8 @@ struct WindowArgs {
     float eps;
     float *h_f32;                  // optional fp32 [B,H]
     void *h_bf16;                  // optional bf16 [B,H]
-    void *x_bf16;                  // bf16 [2][rows][H]: hi plane then lo plane (x = hi + lo)
+    void *x_bf16;                  // bf16 [2][rows][H]: hi plane then lo plane (x = hi + lo); with x_fp16: fp16 [rows][H]
+    int x_fp16;
     size_t x_plane_elems;          // elements between the planes
     int B, H;
     long long *trace;              // optional timeline slot (kTraceSlots values), see common.cuh
@@ -128,9 +129,9 @@ struct EpilogueArgs {
 // PLAIN has no pairing (identity order).  The packers and the epilogues agree through
 // packed_row_to_feature() in pack.cu / epilogue.cuh.
 cudaError_t launch_pack_gemv(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
-                             void *dst, cudaStream_t s);
+                             void *dst, int to_fp16, cudaStream_t s);
 cudaError_t launch_pack_rows(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
-                             void *dst, cudaStream_t s);
+                             void *dst, int to_fp16, cudaStream_t s);
 
 // ---- split-K GEMV (batch < 16): y[b,n] = sum_k x[b,k] W[n,k]; W in fragment-major tiles
 struct GemvArgs {
@@ -153,7 +154,10 @@ cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s);
 struct GemmTcArgs {
     CUtensorMap w_map;    // dims (K, N), box (64, 128), 128B swizzle
     const CUtensorMap *w_map256;  // optional: same tensor with box (64, 256), for two weight tiles per CTA
-    CUtensorMap x_map;    // dims (K, 2*NB): hi rows then lo rows; box (64, 2*NB), 128B swizzle
+    CUtensorMap x_map;    // dims (K, 2*NB): hi rows then lo rows; box (64, 2*NB), 128B swizzle - or, with x_fp16,
+                          // dims (K, NB): one fp16 plane, box (64, NB)
+    int x_fp16;           // the activations are one fp16 plane (inputs that come out of an RMSNorm: bounded,
+                          // 11 significant bits suffice) instead of bf16 hi + lo planes
     int B, NB, N, K;      // NB = batch rows per plane (multiple of 16)
     EpilogueArgs epi;
     int *status;

@@ -10,6 +10,8 @@
 //
 // Tensor path: plain [N, K] K-major rows (the tcgen05 A operand, fetched by TMA
 // with a 128-byte swizzle).
+#include <cuda_fp16.h>
+
 #include "epilogue.cuh"
 
 namespace prsv {
@@ -19,6 +21,7 @@ struct PackParams {
     int cols[3];
     int n_srcs;
     int N, K, kind;
+    int to_fp16;      // store the weights as fp16 (tensor path, matrices whose activations are one fp16 plane)
     bf16 *dst;
 };
 
@@ -43,11 +46,20 @@ __global__ void k_pack(const __grid_constant__ PackParams p)
         const int kc = k >> 5, t = (k & 31) >> 3, e = k & 7;
         o = ((size_t)rb * (p.K >> 5) + kc) * 512 + (size_t)(g * 4 + t) * 16 + hi * 8 + e;
     }
-    p.dst[o] = v;
+    if (p.to_fp16) {
+        // Both operands of a tcgen05 kind::f16 MMA must have the same 16-bit format, so a matrix that is
+        // multiplied with fp16 activations is stored as fp16: exact for every bf16 weight of magnitude
+        // 2^-17 .. 65504 (fp16 has the longer mantissa); smaller ones round to a multiple of 2^-24 (error
+        // <= 2^-25, far below one bf16 ulp of any output), larger ones saturate
+        const float f = fminf(fmaxf(__bfloat162float(v), -65504.f), 65504.f);
+        reinterpret_cast<__half *>(p.dst)[o] = __float2half_rn(f);
+    } else {
+        p.dst[o] = v;
+    }
 }
 
 static cudaError_t launch_pack(bool tensor, const void *const *srcs, const int *src_cols, int n_srcs, int K,
-                               int kind, void *dst, cudaStream_t s)
+                               int kind, void *dst, int to_fp16, cudaStream_t s)
 {
     PackParams p = {};
     int N = 0;
@@ -60,6 +72,7 @@ static cudaError_t launch_pack(bool tensor, const void *const *srcs, const int *
     p.N = N;
     p.K = K;
     p.kind = kind;
+    p.to_fp16 = to_fp16;
     p.dst = reinterpret_cast<bf16 *>(dst);
     const size_t total = (size_t)N * K;
     const int threads = 256;
@@ -72,14 +85,15 @@ static cudaError_t launch_pack(bool tensor, const void *const *srcs, const int *
 }
 
 cudaError_t launch_pack_gemv(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind, void *dst,
-                             cudaStream_t s)
+                             int to_fp16, cudaStream_t s)
 {
-    return launch_pack(false, srcs, src_cols, n_srcs, K, kind, dst, s);
+    (void)to_fp16;      // the GEMV path keeps bf16 weights and hi + lo bf16 activations
+    return launch_pack(false, srcs, src_cols, n_srcs, K, kind, dst, 0, s);
 }
 cudaError_t launch_pack_rows(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind, void *dst,
-                             cudaStream_t s)
+                             int to_fp16, cudaStream_t s)
 {
-    return launch_pack(true, srcs, src_cols, n_srcs, K, kind, dst, s);
+    return launch_pack(true, srcs, src_cols, n_srcs, K, kind, dst, to_fp16, s);
 }
 
 }  // namespace prsv

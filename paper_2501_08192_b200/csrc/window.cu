@@ -15,6 +15,7 @@
 // The kernel stays narrow (at most 8 B small CTAs): during a real allreduce the
 // SMs idle, which is what leaves HBM bandwidth to the prefetch stream.
 #include <cooperative_groups.h>
+#include <cuda_fp16.h>
 
 #include "common.cuh"
 #include "kernels.h"
@@ -42,6 +43,7 @@ struct WindowParams {
     long long *trace;
     int delay_ns;
     int *status;
+    int x_fp16;          // write x as one fp16 plane (tensor path) instead of bf16 hi + lo planes
     int no_hint;         // LEAN: do not even hint the inputs into L2 before the wait (another kernel of the call still writes them)
     int inject;          // test hook: rank 1 of every row withholds its hand-over to rank 0
     // real communication window (COMM instantiation only)
@@ -314,13 +316,27 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
             xv[2] = v[c][2] * inv * bf_lo(g.y); xv[3] = v[c][3] * inv * bf_hi(g.y);
             xv[4] = v[c][4] * inv * bf_lo(g.z); xv[5] = v[c][5] * inv * bf_hi(g.z);
             xv[6] = v[c][6] * inv * bf_lo(g.w); xv[7] = v[c][7] * inv * bf_hi(g.w);
-            uint4 hi, lo;
-            split_bf16x2(xv[0], xv[1], hi.x, lo.x);
-            split_bf16x2(xv[2], xv[3], hi.y, lo.y);
-            split_bf16x2(xv[4], xv[5], hi.z, lo.z);
-            split_bf16x2(xv[6], xv[7], hi.w, lo.w);
-            p.x_bf16[row_off + ch] = hi;
-            p.x_bf16[p.x_plane + row_off + ch] = lo;
+            if (p.x_fp16) {
+                // normalised activations are bounded (|x| <= sqrt(H) * |gain|): one fp16 plane carries 11
+                // significant bits; clamped to the fp16 range so that an absurd gain cannot make an infinity
+                uint4 o;
+                uint32_t *ow = &o.x;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const __half2 h2 = __floats2half2_rn(fminf(fmaxf(xv[2 * i], -65504.f), 65504.f),
+                                                         fminf(fmaxf(xv[2 * i + 1], -65504.f), 65504.f));
+                    ow[i] = *reinterpret_cast<const uint32_t *>(&h2);
+                }
+                p.x_bf16[row_off + ch] = o;
+            } else {
+                uint4 hi, lo;
+                split_bf16x2(xv[0], xv[1], hi.x, lo.x);
+                split_bf16x2(xv[2], xv[3], hi.y, lo.y);
+                split_bf16x2(xv[4], xv[5], hi.z, lo.z);
+                split_bf16x2(xv[6], xv[7], hi.w, lo.w);
+                p.x_bf16[row_off + ch] = hi;
+                p.x_bf16[p.x_plane + row_off + ch] = lo;
+            }
         }
     }
     if constexpr (COMM) {
@@ -371,6 +387,7 @@ cudaError_t launch_window(const WindowArgs &a, cudaStream_t s)
     if (comm && (a.n_parts > 8 || a.part0_is_f32 || a.comm_rank >= a.n_parts))
         return cudaErrorInvalidValue;
     p.no_hint = a.inputs_after_wait;
+    p.x_fp16 = a.x_fp16;
     p.inject = a.inject;
     p.comm_rank = a.comm_rank;
     p.comm_window = a.comm_window;
