@@ -54,6 +54,7 @@ def lib():
         _lib = C.CDLL(build())
         _lib.oracle_num_threads.restype = C.c_int
         _lib.oracle_layer_step.restype = C.c_int
+        _lib.oracle_layer_step_w8.restype = C.c_int
     return _lib
 
 
@@ -127,8 +128,30 @@ def swiglu(gate, up):
     return a
 
 
+def quantize_weights(w_bits):
+    """Per-output-channel symmetric int8 quantisation of W [K,N] (bf16 bits): (codes int8 [K,N], scale f32 [N])."""
+    w_bits = _u16(w_bits)
+    K, N = w_bits.shape
+    q = np.empty((K, N), np.int8)
+    sc = np.empty(N, np.float32)
+    lib().oracle_quantize_weights(C.c_int(K), C.c_int(N), _p(w_bits), _p(q), _p(sc))
+    return q, sc
+
+
+def matmul_q8(x, q, scale):
+    """x [B,K] f32 times int8 codes q [K,N] with per-column scale [N] -> [B,N] f32."""
+    x = _f32(x)
+    q = np.ascontiguousarray(q, np.int8)
+    scale = _f32(scale)
+    B, K = x.shape
+    N = q.shape[1]
+    y = np.empty((B, N), np.float32)
+    lib().oracle_matmul_q8(C.c_int(B), C.c_int(K), C.c_int(N), _p(x), _p(q), _p(scale), _p(y))
+    return y
+
+
 def layer_step(shape, t: Dict[str, np.ndarray], partials_in=None, residual_in=None,
-               peer_partials=None) -> Dict[str, np.ndarray]:
+               peer_partials=None, int8_weights: bool = False) -> Dict[str, np.ndarray]:
     """One decode step of one shard's layer.
 
     `shape` needs hidden, n_q_heads, n_kv_heads, head_dim, ffn, tp_degree,
@@ -159,8 +182,9 @@ def layer_step(shape, t: Dict[str, np.ndarray], partials_in=None, residual_in=No
     res = {n: np.empty(s, np.float32) for n, s in sizes.items()}
     out = _Out(*[res[n].ctypes.data for n in _OUT_NAMES])
     w = [_u16(t[n]) for n in ("w_q", "w_k", "w_v", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")]
-    rc = lib().oracle_layer_step(C.byref(cfg), *[_p(a) for a in w], _p(ctx_len), _p(parts), _p(peers),
-                                 _p(resid), _p(kc), _p(vc), C.byref(out))
+    fn = lib().oracle_layer_step_w8 if int8_weights else lib().oracle_layer_step
+    rc = fn(C.byref(cfg), *[_p(a) for a in w], _p(ctx_len), _p(parts), _p(peers),
+            _p(resid), _p(kc), _p(vc), C.byref(out))
     if rc != 0:
         raise ValueError("oracle_layer_step rejected the configuration")
     return res

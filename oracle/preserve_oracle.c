@@ -155,6 +155,68 @@ void oracle_matmul(int B, int K, int N, const float *x, const uint16_t *w, float
     }
 }
 
+/* ---- int8 weights (the precision of the paper's measurements: Section 4, "Experimental setup").
+ * The paper does not say how its int8 weights are scaled; reading: symmetric per-output-channel
+ * quantisation.  For output column n of W [K,N]: scale_n = max_k |W[k,n]| / 127 (fp32 division),
+ * code q[k,n] = round-to-nearest-even(W[k,n] / scale_n) in fp32, an integer in [-127, 127]; a column of
+ * zeros has scale 0 and codes 0.  The layer then computes y[b,n] = scale_n * sum_k x[b,k] q[k,n].
+ * The decision of every code is taken in fp32 (one correctly rounded division, one rint), which is
+ * what the CUDA side does too, so the codes agree bit for bit. */
+void oracle_quantize_weights(int K, int N, const uint16_t *w, int8_t *q, float *scale)
+{
+    for (int n = 0; n < N; ++n) {
+        float mx = 0.f;
+        for (int k = 0; k < K; ++k) {
+            float v = fabsf(bf16f(w[(size_t)k * N + n]));
+            if (v > mx)
+                mx = v;
+        }
+        float sc = mx / 127.0f;
+        scale[n] = sc;
+        for (int k = 0; k < K; ++k) {
+            float v = bf16f(w[(size_t)k * N + n]);
+            float r = sc > 0.f ? rintf(v / sc) : 0.f;
+            if (r > 127.f) r = 127.f;
+            if (r < -127.f) r = -127.f;
+            q[(size_t)k * N + n] = (int8_t)r;
+        }
+    }
+}
+
+/* y[b,n] = scale[n] * sum_k x[b,k] q[k,n], sums in double */
+void oracle_matmul_q8(int B, int K, int N, const float *x, const int8_t *q, const float *scale, float *y)
+{
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int b = 0; b < B; ++b) {
+            double acc = 0.0;
+            for (int k = 0; k < K; ++k)
+                acc += (double)x[(size_t)b * K + k] * (double)q[(size_t)k * N + n];
+            y[(size_t)b * N + n] = (float)(acc * (double)scale[n]);
+        }
+}
+
+/* the projection of the layer: bf16 weights as they are, or quantised to int8 first */
+static int layer_matmul(int B, int K, int N, const float *x, const uint16_t *w, float *y, int w8)
+{
+    if (!w8) {
+        oracle_matmul(B, K, N, x, w, y);
+        return 0;
+    }
+    int8_t *q = (int8_t *)malloc((size_t)K * N);
+    float *sc = (float *)malloc(sizeof(float) * (size_t)N);
+    if (!q || !sc) {
+        free(q);
+        free(sc);
+        return -1;
+    }
+    oracle_quantize_weights(K, N, w, q, sc);
+    oracle_matmul_q8(B, K, N, x, q, sc, y);
+    free(q);
+    free(sc);
+    return 0;
+}
+
 /* Rotary embedding in place on u[n_heads][d] at position t (half-split pairs). */
 void oracle_rope(int n_heads, int d, int t, float theta, float *u)
 {
@@ -246,12 +308,12 @@ static float *falloc(size_t n) { return (float *)malloc(sizeof(float) * (n ? n :
  * (the bf16 inputs widened exactly, or a previous layer's unrounded outputs in a chain).
  * Weights bf16 [in,out] row-major; gains bf16 [H]; caches bf16 [B,nkv,cap,d] (read only).
  * Returns 0, or -1 on a bad configuration / allocation failure. */
-int oracle_layer_step(const oracle_cfg_t *c, const uint16_t *w_q, const uint16_t *w_k,
-                      const uint16_t *w_v, const uint16_t *w_o, const uint16_t *w_gate,
-                      const uint16_t *w_up, const uint16_t *w_down, const uint16_t *g_attn,
-                      const uint16_t *g_mlp, const int32_t *ctx_len, const float *partials_in,
-                      const float *peer_partials, const float *residual_in,
-                      const uint16_t *k_cache, const uint16_t *v_cache, oracle_out_t *out)
+static int layer_step_impl(const oracle_cfg_t *c, const uint16_t *w_q, const uint16_t *w_k,
+                           const uint16_t *w_v, const uint16_t *w_o, const uint16_t *w_gate,
+                           const uint16_t *w_up, const uint16_t *w_down, const uint16_t *g_attn,
+                           const uint16_t *g_mlp, const int32_t *ctx_len, const float *partials_in,
+                           const float *peer_partials, const float *residual_in,
+                           const uint16_t *k_cache, const uint16_t *v_cache, oracle_out_t *out, int w8)
 {
     int B = c->batch, H = c->hidden, nq = c->n_q_heads, nkv = c->n_kv_heads, d = c->head_dim;
     int F = c->ffn, P = c->tp_degree, cap = c->kv_capacity;
@@ -274,9 +336,9 @@ int oracle_layer_step(const oracle_cfg_t *c, const uint16_t *w_q, const uint16_t
     /* window A: sum of the P partial buffers + residual, then RMSNorm */
     oracle_window(B, H, P, partials_in, residual_in, g_attn, c->rms_eps, h, x);
     /* input projections */
-    oracle_matmul(B, H, nq * d, x, w_q, q);
-    oracle_matmul(B, H, nkv * d, x, w_k, kn);
-    oracle_matmul(B, H, nkv * d, x, w_v, vn);
+    layer_matmul(B, H, nq * d, x, w_q, q, w8);
+    layer_matmul(B, H, nkv * d, x, w_k, kn, w8);
+    layer_matmul(B, H, nkv * d, x, w_v, vn, w8);
     /* positional embedding at position ctx_len[b] on q and the new k */
     for (int b = 0; b < B; ++b) {
         oracle_rope(nq, d, ctx_len[b], c->rope_theta, q + (size_t)b * nq * d);
@@ -290,17 +352,17 @@ int oracle_layer_step(const oracle_cfg_t *c, const uint16_t *w_q, const uint16_t
     /* self-attention over the cached entries plus the new one */
     oracle_attention(B, nq, nkv, d, cap, ctx_len, q, kn_c, vn_c, k_cache, v_cache, o, NULL);
     /* output projection: this shard's partial sum */
-    oracle_matmul(B, nq * d, H, o, w_o, ap);
+    layer_matmul(B, nq * d, H, o, w_o, ap, w8);
     /* window B: own partial + the P-1 peers' partials + h, then RMSNorm */
     memcpy(parts2, ap, sizeof(float) * BH);
     if (P > 1)
         memcpy(parts2 + BH, peer_partials, sizeof(float) * BH * (size_t)(P - 1));
     oracle_window(B, H, P, parts2, h, g_mlp, c->rms_eps, h2, x2);
     /* MLP */
-    oracle_matmul(B, H, F, x2, w_gate, gate);
-    oracle_matmul(B, H, F, x2, w_up, up);
+    layer_matmul(B, H, F, x2, w_gate, gate, w8);
+    layer_matmul(B, H, F, x2, w_up, up, w8);
     oracle_swiglu((size_t)B * F, gate, up, a);
-    oracle_matmul(B, F, H, a, w_down, mp);
+    layer_matmul(B, F, H, a, w_down, mp, w8);
 
 #define COPY_OUT(dst, src, n) \
     if (out->dst) memcpy(out->dst, src, sizeof(float) * (n))
@@ -321,4 +383,28 @@ done:
     free(h); free(x); free(q); free(kn); free(vn); free(o); free(ap); free(h2); free(x2);
     free(gate); free(up); free(a); free(mp); free(parts2); free(kn_c); free(vn_c);
     return rc;
+}
+
+int oracle_layer_step(const oracle_cfg_t *c, const uint16_t *w_q, const uint16_t *w_k,
+                      const uint16_t *w_v, const uint16_t *w_o, const uint16_t *w_gate,
+                      const uint16_t *w_up, const uint16_t *w_down, const uint16_t *g_attn,
+                      const uint16_t *g_mlp, const int32_t *ctx_len, const float *partials_in,
+                      const float *peer_partials, const float *residual_in,
+                      const uint16_t *k_cache, const uint16_t *v_cache, oracle_out_t *out)
+{
+    return layer_step_impl(c, w_q, w_k, w_v, w_o, w_gate, w_up, w_down, g_attn, g_mlp, ctx_len, partials_in,
+                           peer_partials, residual_in, k_cache, v_cache, out, 0);
+}
+
+/* The same step with every projection's weights quantised to int8 per output channel
+ * (oracle_quantize_weights) before use. */
+int oracle_layer_step_w8(const oracle_cfg_t *c, const uint16_t *w_q, const uint16_t *w_k,
+                         const uint16_t *w_v, const uint16_t *w_o, const uint16_t *w_gate,
+                         const uint16_t *w_up, const uint16_t *w_down, const uint16_t *g_attn,
+                         const uint16_t *g_mlp, const int32_t *ctx_len, const float *partials_in,
+                         const float *peer_partials, const float *residual_in,
+                         const uint16_t *k_cache, const uint16_t *v_cache, oracle_out_t *out)
+{
+    return layer_step_impl(c, w_q, w_k, w_v, w_o, w_gate, w_up, w_down, g_attn, g_mlp, ctx_len, partials_in,
+                           peer_partials, residual_in, k_cache, v_cache, out, 1);
 }

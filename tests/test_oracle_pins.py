@@ -422,3 +422,76 @@ def test_chain_feeds_outputs_forward(oracle):
     assert np.array_equal(redo["mlp_partial"], outs[1]["mlp_partial"])
     ref = torch_layer(shape, layers[1], parts=parts, resid=outs[0]["h2"])
     np.testing.assert_allclose(outs[1]["mlp_partial"], ref["mlp_partial"].numpy(), rtol=1e-4, atol=1e-5)
+
+
+# ---------------------------------------------------------------- int8 weights (per output channel)
+def test_int8_quantiser_closed_forms(oracle):
+    """Pins of oracle_quantize_weights that do not retype its loop: the column maximum maps to +-127
+    and the scale is max / 127; a column that is an exact multiple pattern of its scale is
+    reproduced exactly; codes stay within [-127, 127]; the dequantised weight is within half a step;
+    a zero column gives scale 0 and codes 0; a hand-worked 3 x 2 case."""
+    rng = np.random.default_rng(3)
+    K, N = 64, 9
+    w = rng.standard_normal((K, N)).astype(np.float32) * 0.02
+    w[:, 3] = 0.0
+    # column 4: multiples of 2^-10 from -127 to 127 -> scale 2^-10 exactly, codes = the multiples
+    mult = rng.integers(-127, 128, size=K)
+    mult[0], mult[1] = 127, -127
+    w[:, 4] = mult * 2.0 ** -10
+    bits = I.f32_to_bf16_bits(w)
+    wf = I.bf16_bits_to_f32(bits)
+    q, sc = oracle.quantize_weights(bits)
+    assert q.dtype == np.int8 and q.min() >= -127 and q.max() <= 127
+    mx = np.abs(wf).max(axis=0)
+    assert np.allclose(sc, mx / 127.0, rtol=1e-6)
+    for n in range(N):
+        if n == 3:
+            assert sc[n] == 0 and not q[:, n].any()
+            continue
+        assert np.abs(q[np.abs(wf[:, n]).argmax(), n]) == 127
+        assert np.abs(q[:, n].astype(np.float64) * sc[n] - wf[:, n]).max() <= 0.5000001 * sc[n]
+    assert sc[4] == 2.0 ** -10 and np.array_equal(q[:, 4], mult)
+    # hand-worked: column (0.5, -0.25, 0.125): scale 0.5/127; codes 127, -63.5 -> -64 (ties to even), 31.75 -> 32
+    hand = I.f32_to_bf16_bits(np.array([[0.5, 1.0], [-0.25, -1.0], [0.125, 0.5]], np.float32))
+    qh, sh = oracle.quantize_weights(hand)
+    assert qh[:, 0].tolist() == [127, -64, 32] and qh[:, 1].tolist() == [127, -127, 64]
+    assert abs(sh[0] - 0.5 / 127) < 1e-9 and abs(sh[1] - 1.0 / 127) < 1e-9
+
+
+def test_int8_matmul_and_layer_against_independent_restatements(oracle):
+    """oracle_matmul_q8 against numpy on the dequantised matrix; the int8 layer step against the
+    bf16 layer step run on weights that are already exactly representable in int8 (then both
+    definitions must agree), and against a torch restatement of one projection."""
+    rng = np.random.default_rng(4)
+    x = rng.standard_normal((3, 40)).astype(np.float32)
+    w = I.f32_to_bf16_bits(rng.standard_normal((40, 7)).astype(np.float32) * 0.05)
+    q, sc = oracle.quantize_weights(w)
+    want = x.astype(np.float64) @ (q.astype(np.float64) * sc.astype(np.float64))
+    assert np.allclose(oracle.matmul_q8(x, q, sc), want, rtol=1e-6, atol=1e-7)
+    # weights = small integers times a power of two per column: int8 quantisation is lossless on them,
+    # so the quantised layer equals the plain layer
+    shape = I.small_shape(name="w8_lossless", batch=2, hidden=256, ffn=128, ctx=9, seed=90)
+    t = I.make_layers(shape, 1)[0]
+    for name in ("w_q", "w_k", "w_v", "w_o", "w_gate", "w_up", "w_down"):
+        K, N = t[name].shape
+        codes = rng.integers(-127, 128, size=(K, N))
+        codes[0, :] = 127                                     # every column reaches the extreme code
+        t[name] = I.f32_to_bf16_bits((codes * 2.0 ** -12).astype(np.float32))
+    plain = oracle.layer_step(shape, t)
+    quant = oracle.layer_step(shape, t, int8_weights=True)
+    for k in ("q", "o", "attn_partial", "a", "mlp_partial", "h2"):
+        assert np.allclose(plain[k], quant[k], rtol=2e-6, atol=1e-6), k
+    # generic weights: the quantised layer differs from the plain one, by about the quantisation noise
+    t2 = I.make_layers(shape, 1)[0]
+    p2, q2 = oracle.layer_step(shape, t2), oracle.layer_step(shape, t2, int8_weights=True)
+    rel = np.abs(p2["mlp_partial"] - q2["mlp_partial"]).max() / np.abs(p2["mlp_partial"]).max()
+    assert 1e-5 < rel < 5e-2
+    # one projection restated with torch: q = x W_q with dequantised weights
+    xq = torch.from_numpy(q2["x"].astype(np.float64))
+    qq, ss = oracle.quantize_weights(t2["w_q"])
+    wq = torch.from_numpy(qq.astype(np.float64) * ss.astype(np.float64))
+    if shape.rope_theta <= 0:
+        assert np.allclose((xq @ wq).numpy().reshape(q2["q"].shape), q2["q"], rtol=1e-5, atol=1e-6)
+    v_ref = (torch.from_numpy(q2["x"].astype(np.float64)) @ torch.from_numpy(
+        oracle.quantize_weights(t2["w_v"])[0].astype(np.float64) * oracle.quantize_weights(t2["w_v"])[1].astype(np.float64)))
+    assert np.allclose(v_ref.numpy().reshape(q2["v_new"].shape), q2["v_new"], rtol=1e-5, atol=1e-6)
