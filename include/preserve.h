@@ -87,6 +87,12 @@ extern "C" {
                                        launched early to stage operands in shared memory              */
 #define PRESERVE_FLAG_FORCE_GEMV   8u  /* use the split-K GEMV kernels whatever max_batch is (each launch
                                        covers 16 batch rows)                                          */
+#define PRESERVE_FLAG_INT8_WEIGHTS 32u  /* keep the four weight matrices as int8 codes with one fp32 scale per output
+                                       feature (symmetric: scale = max |w| / 127 over the feature's inputs, code =
+                                       round-to-nearest-even(w / scale), decided in fp32) - the weight precision
+                                       of the paper's measurements (Section 4, "Experimental setup"); activations
+                                       and the KV-cache stay bf16.  Split-K GEMV path only (max_batch < 16 or
+                                       PRESERVE_FLAG_FORCE_GEMV), ffn a multiple of 64; PRESERVE_ESHAPE otherwise */
 #define PRESERVE_FLAG_FORCE_TENSOR 16u /* use the tcgen05 GEMM kernels although max_batch < 16 (needs ffn
                                        to be a multiple of 128)                                       */
 

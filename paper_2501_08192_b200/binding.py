@@ -19,6 +19,7 @@ PRESERVE_ECUDA, PRESERVE_EARCH, PRESERVE_ETIMEOUT, PRESERVE_ETOOBIG = -5, -6, -7
 STATIC_SCRATCH_BYTES = 8 << 20
 PLAN_WHOLE_NODE, PLAN_TRUNCATE = 0, 1
 FLAG_NO_GRAPH, FLAG_PERSIST_L2, FLAG_NO_EARLY_LAUNCH, FLAG_FORCE_GEMV, FLAG_FORCE_TENSOR = 1, 2, 4, 8, 16
+FLAG_INT8_WEIGHTS = 32
 DEBUG_WITHHOLD, DEBUG_WAIT_LIMIT_CYCLES = 0, 1
 WITHHOLD_WINDOW, WITHHOLD_GEMV, WITHHOLD_TENSOR, WITHHOLD_ATTENTION = 1, 2, 3, 4
 

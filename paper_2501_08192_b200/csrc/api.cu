@@ -84,6 +84,9 @@ struct preserve_layer {
     uint64_t wbytes[4];
     void *g_attn, *g_mlp;
     double *inv_freq;
+    bool w8;                     // int8 weights (GEMV path): arena holds codes, `scales` one fp32 per packed row
+    float *scales;
+    size_t soff[4];
 
     float *h_f32;                              // window A sum (residual for window B)
     float *attn_f32, *h2_f32, *mlp_f32;        // unrounded copies: own attention partial (window B input),
@@ -180,6 +183,12 @@ int validate_config(const preserve_layer_config_t *c)
         return PRESERVE_ESHAPE;
     if ((long long)c->max_batch * c->n_kv_heads * ((long long)c->max_ctx + 1) > 0x7fffffffll)
         return PRESERVE_ESHAPE;
+    if (c->flags & PRESERVE_FLAG_INT8_WEIGHTS) {
+        // int8 weights exist for the split-K GEMV kernels only; their 1 KiB tiles cover 64 k
+        const bool gemv = c->max_batch < 16 || (c->flags & PRESERVE_FLAG_FORCE_GEMV);
+        if (!gemv || (c->flags & PRESERVE_FLAG_FORCE_TENSOR) || c->ffn % 64)
+            return PRESERVE_ESHAPE;
+    }
     return PRESERVE_OK;
 }
 
@@ -194,6 +203,13 @@ Dims layer_dims(const preserve_layer_config_t &c)
     d.n[2] = 2 * c.ffn;                                     d.k[2] = c.hidden;
     d.n[3] = c.hidden;                                      d.k[3] = c.ffn;
     return d;
+}
+
+// bytes of weight matrix i as the kernels stream it: bf16, or int8 codes (their fp32 scales, one per
+// output feature, are 4 / K of that and not counted)
+uint64_t weight_bytes(const preserve_layer_config_t &c, const Dims &d, int i)
+{
+    return (uint64_t)d.n[i] * d.k[i] * ((c.flags & PRESERVE_FLAG_INT8_WEIGHTS) ? 1 : 2);
 }
 
 uint64_t activation_bytes(const preserve_layer_config_t &c, int B)
@@ -350,6 +366,8 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
         a.trace = trace;
         a.pdl = pdl;
         a.inject = L->inject == INJECT_GEMV_RING && which == 0 ? INJECT_GEMV_RING : INJECT_NONE;
+        a.w8 = L->w8 ? 1 : 0;
+        a.scales = L->w8 ? L->scales + L->soff[which] : nullptr;
         a.next_w = nullptr;
         a.next_bytes = 0;
         // Prefetching on: the gate/up projection fills both CTA slots of most SMs, so most CTAs of the
@@ -863,7 +881,7 @@ uint64_t preserve_algorithmic_bytes(const preserve_layer_config_t *cfg, int32_t 
     const Dims d = layer_dims(*cfg);
     uint64_t w = 0;
     for (int i = 0; i < 4; ++i)
-        w += (uint64_t)d.n[i] * d.k[i] * 2;
+        w += weight_bytes(*cfg, d, i);
     const uint64_t kv = 2 * sum_ctx * cfg->n_kv_heads * cfg->head_dim * 2;
     return w + kv + activation_bytes(*cfg, batch);
 }
@@ -876,7 +894,7 @@ void preserve_layer_destroy(preserve_layer_t *L)
     if (L->side)
         cudaStreamSynchronize(L->side);
     drop_graphs(L);
-    void *ptrs[] = {L->trace_buf, L->attn_f32, L->h2_f32, L->mlp_f32, L->arena, L->inv_freq, L->h_f32, L->x, L->q, L->o, L->x2, L->a,
+    void *ptrs[] = {L->scales, L->trace_buf, L->attn_f32, L->h2_f32, L->mlp_f32, L->arena, L->inv_freq, L->h_f32, L->x, L->q, L->o, L->x2, L->a,
                     L->part_o, L->part_ml, L->status, L->stage_in, L->stage_out, L->ctx_dev};
     for (void *p : ptrs)
         if (p)
@@ -965,7 +983,7 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     size_t off = 0;
     for (int i = 0; i < 4; ++i) {
         L->off[i] = off;
-        L->wbytes[i] = (uint64_t)d.n[i] * d.k[i] * 2;
+        L->wbytes[i] = weight_bytes(c, d, i);
         off += (size_t)L->wbytes[i];
     }
     const size_t gains_off = off;
@@ -987,12 +1005,26 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
         const int c_gu[2] = {c.ffn, c.ffn};
         const void *s_dn[1] = {w->w_down};
         const int c_dn[1] = {H};
-        auto pack = L->tensor_path ? launch_pack_rows : launch_pack_gemv;
-        // (tensor path: Wgate|up meets the fp16 RMSNorm output x2 and is stored as fp16)
-        CKI(pack(s_qkv, c_qkv, 3, d.k[0], EPI_QKV, L->arena + L->off[0], 0, nullptr));
-        CKI(pack(s_o, c_o, 1, d.k[1], EPI_PLAIN, L->arena + L->off[1], 0, nullptr));
-        CKI(pack(s_gu, c_gu, 2, d.k[2], EPI_SWIGLU, L->arena + L->off[2], 1, nullptr));
-        CKI(pack(s_dn, c_dn, 1, d.k[3], EPI_PLAIN, L->arena + L->off[3], 0, nullptr));
+        L->w8 = (c.flags & PRESERVE_FLAG_INT8_WEIGHTS) != 0;
+        if (L->w8) {
+            size_t so = 0;
+            for (int i = 0; i < 4; ++i) {
+                L->soff[i] = so;
+                so += (size_t)d.n[i];
+            }
+            CKI(cudaMalloc(&L->scales, so * sizeof(float)));
+            CKI(launch_pack_gemv_w8(s_qkv, c_qkv, 3, d.k[0], EPI_QKV, L->arena + L->off[0], L->scales + L->soff[0], nullptr));
+            CKI(launch_pack_gemv_w8(s_o, c_o, 1, d.k[1], EPI_PLAIN, L->arena + L->off[1], L->scales + L->soff[1], nullptr));
+            CKI(launch_pack_gemv_w8(s_gu, c_gu, 2, d.k[2], EPI_SWIGLU, L->arena + L->off[2], L->scales + L->soff[2], nullptr));
+            CKI(launch_pack_gemv_w8(s_dn, c_dn, 1, d.k[3], EPI_PLAIN, L->arena + L->off[3], L->scales + L->soff[3], nullptr));
+        } else {
+            auto pack = L->tensor_path ? launch_pack_rows : launch_pack_gemv;
+            // (tensor path: Wgate|up meets the fp16 RMSNorm output x2 and is stored as fp16)
+            CKI(pack(s_qkv, c_qkv, 3, d.k[0], EPI_QKV, L->arena + L->off[0], 0, nullptr));
+            CKI(pack(s_o, c_o, 1, d.k[1], EPI_PLAIN, L->arena + L->off[1], 0, nullptr));
+            CKI(pack(s_gu, c_gu, 2, d.k[2], EPI_SWIGLU, L->arena + L->off[2], 1, nullptr));
+            CKI(pack(s_dn, c_dn, 1, d.k[3], EPI_PLAIN, L->arena + L->off[3], 0, nullptr));
+        }
     }
     // rotary frequencies theta^(-2i/d)
     {

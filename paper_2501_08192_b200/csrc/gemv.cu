@@ -65,18 +65,31 @@ struct GemvParams {
     uint32_t next_slice;   // bytes of next_w each CTA prefetches
     size_t next_bytes;
     int inject;            // test hook: warp 0 of CTA (0, 0) arms its first ring slot but never fills it
+    const float *scales;   // W8: per packed row
     EpilogueArgs epi;
 };
+
+// two int8 codes (bytes at bit `shift` and `shift + 8` of w) as a bf16 pair: every code is exact in bf16
+__device__ __forceinline__ uint32_t s8x2_to_bf16x2(uint32_t w, int shift)
+{
+    const int a = (int)(w << (24 - shift)) >> 24, b = (int)(w << (16 - shift)) >> 24;
+    return pack_bf16((float)a, (float)b);
+}
+__device__ __forceinline__ float s8_to_f32(uint32_t w, int byte) { return (float)((int)(w << (24 - 8 * byte)) >> 24); }
 
 // RB = 16-row blocks per warp: with two, every activation fragment a warp loads is used for two
 // weight tiles, which halves the activation traffic from L2 (for batch 8 it is otherwise as large
 // as the weight stream itself, and an SM takes in only ~50 GB/s in total).
-template <int NB, bool MMA, int RB>
+// W8: the weights are int8 codes - a 1 KiB tile then covers 16 rows x 64 k (a lane's 16 bytes per row
+// are k = 16 t .. 16 t + 15), the codes are widened to bf16 (exactly) in registers, and every output
+// is multiplied by its row's scale in front of the epilogue.
+template <int NB, bool MMA, int RB, bool W8 = false>
 __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid_constant__ GemvParams p)
 {
     constexpr int NTB = MMA ? NB / 8 : 1;   // n-tiles that cover the batch
     constexpr int NT = 2 * NTB;             // hi planes then lo planes of the activations
-    constexpr int NX = MMA ? NT : 2 * NB;   // activation fragments (uint4) per tile
+    constexpr int XF = W8 ? 2 : 1;          // uint4 of activations per tile, lane and (batch row, plane): 8 k each
+    constexpr int NX = (MMA ? NT : 2 * NB) * XF;   // activation fragments (uint4) per tile
     __shared__ float red[kGemvWarps][RB * 16][NB];       // per-warp partials
     __shared__ float cta_part[kGemvWarps * RB][16][NB];  // per-row-block CTA partials (read across the cluster)
     __shared__ uint64_t bars[kGemvWarps][kRingSlots];
@@ -167,15 +180,20 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
             for (int nt = 0; nt < NT; ++nt) {
                 const int b = (nt % NTB) * 8 + g;
                 const uint4 *plane = p.x + (nt >= NTB ? p.x_plane : 0);
-                xq[nt] = b < p.B ? ld_cached(plane + (size_t)(p.b0 + b) * xrow + c * 4 + t) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int f = 0; f < XF; ++f)
+                    xq[nt * XF + f] = b < p.B ? ld_cached(plane + (size_t)(p.b0 + b) * xrow + c * (4 * XF) + t * XF + f)
+                                              : make_uint4(0, 0, 0, 0);
             }
         } else {
 #pragma unroll
-            for (int b = 0; b < NB; ++b) {
-                xq[b] = b < p.B ? ld_cached(p.x + (size_t)(p.b0 + b) * xrow + c * 4 + t) : make_uint4(0, 0, 0, 0);
-                xq[NB + b] = b < p.B ? ld_cached(p.x + p.x_plane + (size_t)(p.b0 + b) * xrow + c * 4 + t)
-                                     : make_uint4(0, 0, 0, 0);
-            }
+            for (int b = 0; b < NB; ++b)
+#pragma unroll
+                for (int f = 0; f < XF; ++f) {
+                    const size_t o = (size_t)(p.b0 + b) * xrow + c * (4 * XF) + t * XF + f;
+                    xq[b * XF + f] = b < p.B ? ld_cached(p.x + o) : make_uint4(0, 0, 0, 0);
+                    xq[(NB + b) * XF + f] = b < p.B ? ld_cached(p.x + p.x_plane + o) : make_uint4(0, 0, 0, 0);
+                }
         }
     };
 
@@ -194,31 +212,61 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
                 for (int j = 0; j < (MMA ? 4 : 1); ++j)
                     acc[r][i][j] = 0.f;
 
-        auto compute = [&](float (&a_)[MMA ? NT : 2 * NB][MMA ? 4 : 1], const uint4 &wl, const uint4 &wh, const uint4 (&xq)[NX]) {
-            if constexpr (MMA) {
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    mma_bf16_16816(a_[nt], wl.x, wh.x, wl.y, wh.y, xq[nt].x, xq[nt].y);
-                    mma_bf16_16816(a_[nt], wl.z, wh.z, wl.w, wh.w, xq[nt].z, xq[nt].w);
-                }
-            } else {
-                const float l0 = bf_lo(wl.x), l1 = bf_hi(wl.x), l2 = bf_lo(wl.y), l3 = bf_hi(wl.y);
-                const float l4 = bf_lo(wl.z), l5 = bf_hi(wl.z), l6 = bf_lo(wl.w), l7 = bf_hi(wl.w);
-                const float h0 = bf_lo(wh.x), h1 = bf_hi(wh.x), h2 = bf_lo(wh.y), h3 = bf_hi(wh.y);
-                const float h4 = bf_lo(wh.z), h5 = bf_hi(wh.z), h6 = bf_lo(wh.w), h7 = bf_hi(wh.w);
+        // eight weights of row g (wl) and of row g + 8 (wh) against the same eight k of every batch row
+        auto fma8 = [&](float (&a_)[MMA ? NT : 2 * NB][MMA ? 4 : 1], const float (&l)[8], const float (&h)[8],
+                        const uint4 (&xq)[NX], int f) {
+            if constexpr (!MMA) {
 #pragma unroll
                 for (int b = 0; b < NB; ++b) {
-                    const uint4 &xh = xq[b], &xl = xq[NB + b];     // x = hi + lo, exact in fp32
+                    const uint4 &xh = xq[b * XF + f], &xl = xq[(NB + b) * XF + f];     // x = hi + lo, exact in fp32
                     const float x0 = bf_lo(xh.x) + bf_lo(xl.x), x1 = bf_hi(xh.x) + bf_hi(xl.x);
                     const float x2 = bf_lo(xh.y) + bf_lo(xl.y), x3 = bf_hi(xh.y) + bf_hi(xl.y);
                     const float x4 = bf_lo(xh.z) + bf_lo(xl.z), x5 = bf_hi(xh.z) + bf_hi(xl.z);
                     const float x6 = bf_lo(xh.w) + bf_lo(xl.w), x7 = bf_hi(xh.w) + bf_hi(xl.w);
                     float a = a_[2 * b][0], c = a_[2 * b + 1][0];
-                    a = fmaf(l0, x0, a); a = fmaf(l1, x1, a); a = fmaf(l2, x2, a); a = fmaf(l3, x3, a);
-                    a = fmaf(l4, x4, a); a = fmaf(l5, x5, a); a = fmaf(l6, x6, a); a = fmaf(l7, x7, a);
-                    c = fmaf(h0, x0, c); c = fmaf(h1, x1, c); c = fmaf(h2, x2, c); c = fmaf(h3, x3, c);
-                    c = fmaf(h4, x4, c); c = fmaf(h5, x5, c); c = fmaf(h6, x6, c); c = fmaf(h7, x7, c);
+                    a = fmaf(l[0], x0, a); a = fmaf(l[1], x1, a); a = fmaf(l[2], x2, a); a = fmaf(l[3], x3, a);
+                    a = fmaf(l[4], x4, a); a = fmaf(l[5], x5, a); a = fmaf(l[6], x6, a); a = fmaf(l[7], x7, a);
+                    c = fmaf(h[0], x0, c); c = fmaf(h[1], x1, c); c = fmaf(h[2], x2, c); c = fmaf(h[3], x3, c);
+                    c = fmaf(h[4], x4, c); c = fmaf(h[5], x5, c); c = fmaf(h[6], x6, c); c = fmaf(h[7], x7, c);
                     a_[2 * b][0] = a; a_[2 * b + 1][0] = c;
+                }
+            }
+        };
+        auto compute = [&](float (&a_)[MMA ? NT : 2 * NB][MMA ? 4 : 1], const uint4 &wl, const uint4 &wh, const uint4 (&xq)[NX]) {
+            if constexpr (MMA && !W8) {
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    mma_bf16_16816(a_[nt], wl.x, wh.x, wl.y, wh.y, xq[nt].x, xq[nt].y);
+                    mma_bf16_16816(a_[nt], wl.z, wh.z, wl.w, wh.w, xq[nt].z, xq[nt].w);
+                }
+            } else if constexpr (MMA && W8) {
+                // word j of wl / wh = codes of k = 16 t + 4 j .. + 3: one m16n8k16 MMA per word
+                const uint32_t lw[4] = {wl.x, wl.y, wl.z, wl.w}, hw[4] = {wh.x, wh.y, wh.z, wh.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t a0 = s8x2_to_bf16x2(lw[j], 0), a2 = s8x2_to_bf16x2(lw[j], 16);
+                    const uint32_t a1 = s8x2_to_bf16x2(hw[j], 0), a3 = s8x2_to_bf16x2(hw[j], 16);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const uint4 &xv = xq[nt * 2 + (j >> 1)];
+                        mma_bf16_16816(a_[nt], a0, a1, a2, a3, (j & 1) ? xv.z : xv.x, (j & 1) ? xv.w : xv.y);
+                    }
+                }
+            } else if constexpr (!W8) {
+                const float l[8] = {bf_lo(wl.x), bf_hi(wl.x), bf_lo(wl.y), bf_hi(wl.y), bf_lo(wl.z), bf_hi(wl.z), bf_lo(wl.w), bf_hi(wl.w)};
+                const float h[8] = {bf_lo(wh.x), bf_hi(wh.x), bf_lo(wh.y), bf_hi(wh.y), bf_lo(wh.z), bf_hi(wh.z), bf_lo(wh.w), bf_hi(wh.w)};
+                fma8(a_, l, h, xq, 0);
+            } else {
+                const uint32_t lw[4] = {wl.x, wl.y, wl.z, wl.w}, hw[4] = {wh.x, wh.y, wh.z, wh.w};
+#pragma unroll
+                for (int f = 0; f < 2; ++f) {
+                    float l[8], h[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        l[i] = s8_to_f32(lw[2 * f + (i >> 2)], i & 3);
+                        h[i] = s8_to_f32(hw[2 * f + (i >> 2)], i & 3);
+                    }
+                    fma8(a_, l, h, xq, f);
                 }
             }
         };
@@ -327,6 +375,11 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
                         v0 += recv[(size_t)(q - 1) * part_floats + (rl * 16 + r) * NB + b];
                         v1 += recv[(size_t)(q - 1) * part_floats + (rl * 16 + r + 8) * NB + b];
                     }
+                    if constexpr (W8) {
+                        const int prow = (grp * rbs_per_cta + rl) * 16 + r;
+                        v0 *= p.scales[prow];
+                        v1 *= p.scales[prow + 8];
+                    }
                     apply_epilogue(p.epi, tabs, b, false, p.N, p.b0 + b, (grp * rbs_per_cta + rl) * 8 + r, v0, v1);
                 }
             }
@@ -349,6 +402,11 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
                         v0 += remote[q][(rl * 16 + r) * NB + b];
                         v1 += remote[q][(rl * 16 + r + 8) * NB + b];
                     }
+                if constexpr (W8) {
+                    const int prow = (grp * rbs_per_cta + rl) * 16 + r;
+                    v0 *= p.scales[prow];
+                    v1 *= p.scales[prow + 8];
+                }
                 apply_epilogue(p.epi, tabs, b, false, p.N, p.b0 + b, (grp * rbs_per_cta + rl) * 8 + r, v0, v1);
             }
             cluster.sync();   // peers' shared memory must outlive the reads; also fences red/cta_part reuse
@@ -358,8 +416,13 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
                 const int b = i % NB, r = (i / NB) % 8, rl = i / (8 * NB);
                 if (b >= p.B)
                     continue;
-                apply_epilogue(p.epi, tabs, b, false, p.N, p.b0 + b, (grp * rbs_per_cta + rl) * 8 + r,
-                               cta_part[rl][r][b], cta_part[rl][r + 8][b]);
+                float v0 = cta_part[rl][r][b], v1 = cta_part[rl][r + 8][b];
+                if constexpr (W8) {
+                    const int prow = (grp * rbs_per_cta + rl) * 16 + r;
+                    v0 *= p.scales[prow];
+                    v1 *= p.scales[prow + 8];
+                }
+                apply_epilogue(p.epi, tabs, b, false, p.N, p.b0 + b, (grp * rbs_per_cta + rl) * 8 + r, v0, v1);
             }
             __syncthreads();
         }
@@ -367,12 +430,12 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
     trace_end(p.trace);
 }
 
-template <int NB, bool MMA, int RB>
+template <int NB, bool MMA, int RB, bool W8>
 static cudaError_t launch_variant(GemvParams &p, int sm_count, int pdl, cudaStream_t s)
 {
     static PerDeviceSize smem_limit;      // per instantiation and device
     {
-        cudaError_t e = ensure_dynamic_smem(k_gemv_splitk<NB, MMA, RB>, smem_limit, kGemvSmemBytes + 32 * 1024 + 128);
+        cudaError_t e = ensure_dynamic_smem(k_gemv_splitk<NB, MMA, RB, W8>, smem_limit, kGemvSmemBytes + 32 * 1024 + 128);
         if (e != cudaSuccess)
             return e;
     }
@@ -428,12 +491,26 @@ static cudaError_t launch_variant(GemvParams &p, int sm_count, int pdl, cudaStre
     }
     cfg.attrs = at;
     cfg.numAttrs = n;
-    return cudaLaunchKernelEx(&cfg, k_gemv_splitk<NB, MMA, RB>, p);
+    return cudaLaunchKernelEx(&cfg, k_gemv_splitk<NB, MMA, RB, W8>, p);
+}
+
+template <bool W8>
+static cudaError_t launch_by_batch(GemvParams &p, int B, int sm_count, int pdl, cudaStream_t s)
+{
+    // two row blocks per warp whenever the matrix has enough row blocks to still fill the SMs
+    const bool two = p.row_blocks % 2 == 0 && p.row_blocks >= 32;
+    if (B == 1) return two ? launch_variant<1, false, 2, W8>(p, sm_count, pdl, s) : launch_variant<1, false, 1, W8>(p, sm_count, pdl, s);
+    if (B == 2) return two ? launch_variant<2, false, 2, W8>(p, sm_count, pdl, s) : launch_variant<2, false, 1, W8>(p, sm_count, pdl, s);
+    // (int8 weights double the activation fragments a lane holds per tile: batch 3-4 takes the MMA form there)
+    if (B <= 4 && !W8) return two ? launch_variant<4, false, 2, false>(p, sm_count, pdl, s) : launch_variant<4, false, 1, false>(p, sm_count, pdl, s);
+    if (B <= 8) return two ? launch_variant<8, true, 2, W8>(p, sm_count, pdl, s) : launch_variant<8, true, 1, W8>(p, sm_count, pdl, s);
+    return two ? launch_variant<16, true, 2, W8>(p, sm_count, pdl, s) : launch_variant<16, true, 1, W8>(p, sm_count, pdl, s);
 }
 
 cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s)
 {
-    if (a.B < 1 || a.B > 16 || a.N % 16 || a.K % 32)
+    const int tile_k = a.w8 ? 64 : 32;       // k covered by a 1 KiB tile
+    if (a.B < 1 || a.B > 16 || a.N % 16 || a.K % tile_k || (a.w8 && !a.scales))
         return cudaErrorInvalidValue;
     GemvParams p;
     p.w = reinterpret_cast<const uint4 *>(a.w);
@@ -441,22 +518,15 @@ cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s)
     p.x_plane = a.x_plane / 8;
     p.B = a.B; p.N = a.N; p.K = a.K; p.b0 = a.b0;
     p.row_blocks = a.N / 16;
-    p.kchunks = a.K / 32;
+    p.kchunks = a.K / tile_k;
     p.epi = a.epi;
     p.status = a.status;
     p.trace = a.trace;
     p.next_w = reinterpret_cast<const uint8_t *>(a.next_w);
     p.next_bytes = a.next_bytes;
     p.inject = a.inject;
-    const int pdl = a.pdl;
-
-    // two row blocks per warp whenever the matrix has enough row blocks to still fill the SMs
-    const bool two = p.row_blocks % 2 == 0 && p.row_blocks >= 32;
-    if (a.B == 1) return two ? launch_variant<1, false, 2>(p, sm_count, pdl, s) : launch_variant<1, false, 1>(p, sm_count, pdl, s);
-    if (a.B == 2) return two ? launch_variant<2, false, 2>(p, sm_count, pdl, s) : launch_variant<2, false, 1>(p, sm_count, pdl, s);
-    if (a.B <= 4) return two ? launch_variant<4, false, 2>(p, sm_count, pdl, s) : launch_variant<4, false, 1>(p, sm_count, pdl, s);
-    if (a.B <= 8) return two ? launch_variant<8, true, 2>(p, sm_count, pdl, s) : launch_variant<8, true, 1>(p, sm_count, pdl, s);
-    return two ? launch_variant<16, true, 2>(p, sm_count, pdl, s) : launch_variant<16, true, 1>(p, sm_count, pdl, s);
+    p.scales = a.scales;
+    return a.w8 ? launch_by_batch<true>(p, a.B, sm_count, a.pdl, s) : launch_by_batch<false>(p, a.B, sm_count, a.pdl, s);
 }
 
 }  // namespace prsv

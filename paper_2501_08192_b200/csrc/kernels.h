@@ -132,6 +132,11 @@ cudaError_t launch_pack_gemv(const void *const *srcs, const int *src_cols, int n
                              void *dst, int to_fp16, cudaStream_t s);
 cudaError_t launch_pack_rows(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
                              void *dst, int to_fp16, cudaStream_t s);
+// int8 weights for the GEMV path: symmetric per-output-channel quantisation (scale = max |w| / 127 of the
+// output feature's column, code = round-to-nearest-even(w / scale), both in fp32), codes in fragment-major
+// 1 KiB tiles of 16 rows x 64 k, scales [N] in packed row order.
+cudaError_t launch_pack_gemv_w8(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
+                                void *dst_codes, float *dst_scales, cudaStream_t s);
 
 // ---- split-K GEMV (batch < 16): y[b,n] = sum_k x[b,k] W[n,k]; W in fragment-major tiles
 struct GemvArgs {
@@ -147,6 +152,8 @@ struct GemvArgs {
     size_t next_bytes;
     int pdl;
     int inject;
+    int w8;               // the weights are int8 codes (1 KiB tiles of 16 rows x 64 k) with one fp32 scale per packed row
+    const float *scales;  // w8: [N] in packed row order
 };
 cudaError_t launch_gemv(const GemvArgs &a, int sm_count, cudaStream_t s);
 

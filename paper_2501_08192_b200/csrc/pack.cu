@@ -84,6 +84,71 @@ static cudaError_t launch_pack(bool tensor, const void *const *srcs, const int *
     return cudaGetLastError();
 }
 
+// ---- int8 weights (GEMV path)
+struct PackW8Params {
+    const bf16 *src[3];
+    int cols[3];
+    int N, K, kind;
+    int8_t *codes;
+    float *scales;
+};
+
+// scale of every packed row: max |w| over the row's source column, divided by 127 (fp32)
+__global__ void k_w8_scales(const __grid_constant__ PackW8Params p)
+{
+    const int row = blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= p.N)
+        return;
+    int src, col;
+    packed_row_source(p.kind, false, row, p.cols, src, col);
+    float mx = 0.f;
+    for (int k = 0; k < p.K; ++k)
+        mx = fmaxf(mx, fabsf(__bfloat162float(p.src[src][(size_t)k * p.cols[src] + col])));
+    p.scales[row] = __fdiv_rn(mx, 127.0f);
+}
+
+__global__ void k_pack_w8(const __grid_constant__ PackW8Params p)
+{
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t total = (size_t)p.N * p.K;
+    if (idx >= total)
+        return;
+    const int row = (int)(idx % p.N);
+    const int k = (int)(idx / p.N);
+    int src, col;
+    packed_row_source(p.kind, false, row, p.cols, src, col);
+    const float v = __bfloat162float(p.src[src][(size_t)k * p.cols[src] + col]);
+    const float sc = p.scales[row];
+    // the code is decided in fp32: one correctly rounded division, round to nearest even, clamp
+    float r = sc > 0.f ? rintf(__fdiv_rn(v, sc)) : 0.f;
+    r = fminf(fmaxf(r, -127.f), 127.f);
+    const int rb = row >> 4, rr = row & 15, g = rr & 7, hi = rr >> 3;
+    const int kc = k >> 6, t = (k & 63) >> 4, e = k & 15;
+    const size_t o = ((size_t)rb * (p.K >> 6) + kc) * 1024 + (size_t)(g * 4 + t) * 32 + hi * 16 + e;
+    p.codes[o] = (int8_t)(int)r;
+}
+
+cudaError_t launch_pack_gemv_w8(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
+                                void *dst_codes, float *dst_scales, cudaStream_t s)
+{
+    if (K % 64)
+        return cudaErrorInvalidValue;
+    PackW8Params p = {};
+    int N = 0;
+    for (int i = 0; i < n_srcs; ++i) {
+        p.src[i] = reinterpret_cast<const bf16 *>(srcs[i]);
+        p.cols[i] = src_cols[i];
+        N += src_cols[i];
+    }
+    p.N = N; p.K = K; p.kind = kind;
+    p.codes = reinterpret_cast<int8_t *>(dst_codes);
+    p.scales = dst_scales;
+    k_w8_scales<<<(N + 127) / 128, 128, 0, s>>>(p);
+    const size_t total = (size_t)N * K;
+    k_pack_w8<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_pack_gemv(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind, void *dst,
                              int to_fp16, cudaStream_t s)
 {

@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 
 def full_check(oracle, shape, flags=0, budget=None):
     t = I.make_layers(shape, 1)[0]
-    ref = oracle.layer_step(shape, t)
+    ref = oracle.layer_step(shape, t, int8_weights=bool(flags & P.FLAG_INT8_WEIGHTS))
     dl = G.DeviceLayer(shape, t, flags=flags)
     try:
         if budget is not None:
@@ -87,6 +87,49 @@ def test_benchmark_configs_match_oracle(oracle, idx):
     # (with the side-stream L2 prefetch running: a budget of 16 MiB per window; the library's default
     # plans nothing for L2 and is what the small shapes above run with)
     full_check(oracle, I.CONFIGS[idx], budget=16 << 20)
+
+
+W8_SHAPES = [
+    I.small_shape(name="w8_b1", batch=1, tp_degree=1, ctx=37, n_q_heads=2, n_kv_heads=2, seed=112),
+    I.small_shape(name="w8_b2", batch=2, ctx=64, seed=140),
+    I.small_shape(name="w8_b3", batch=3, ctx=200, seed=111),
+    I.small_shape(name="w8_b4_g4", batch=4, ctx=63, n_q_heads=4, n_kv_heads=1, seed=141),
+    I.small_shape(name="w8_b8_ragged", batch=8, ctx=300, ctx_min=10, tp_degree=4, seed=113),
+    I.small_shape(name="w8_b15_g16", batch=15, ctx=65, n_q_heads=16, n_kv_heads=1, tp_degree=16, seed=143),
+    I.small_shape(name="w8_wide_ffn_b8", batch=8, hidden=256, ffn=5120, ctx=70, seed=148),
+    I.small_shape(name="w8_h384_b7", batch=7, hidden=384, ffn=192, ctx=33, seed=149),
+    I.small_shape(name="w8_h2048_b3", batch=3, hidden=2048, ffn=256, ctx=40, tp_degree=5, seed=150),
+]
+
+
+@pytest.mark.parametrize("shape", W8_SHAPES, ids=[s.name for s in W8_SHAPES])
+def test_int8_weights_match_the_quantised_oracle(oracle, shape):
+    """int8 weights (per-output-channel scales) on the split-K GEMV path against the oracle that
+    quantises the same way: every intermediate and output, same tolerance."""
+    full_check(oracle, shape, flags=P.FLAG_INT8_WEIGHTS)
+
+
+@pytest.mark.parametrize("idx", [0, 1])
+def test_int8_weights_on_benchmark_configs(oracle, idx):
+    bits = full_check(oracle, I.CONFIGS[idx], flags=P.FLAG_INT8_WEIGHTS, budget=16 << 20)
+    again = full_check(oracle, I.CONFIGS[idx], flags=P.FLAG_INT8_WEIGHTS, budget=0)
+    for k in bits:
+        assert np.array_equal(bits[k], again[k]), k          # prefetch never changes results, int8 included
+
+
+def test_int8_weights_are_refused_where_no_kernel_has_them():
+    t = I.make_layers(I.small_shape(batch=20), 1)[0]
+    with pytest.raises(P.PreserveError) as e:
+        G.DeviceLayer(I.small_shape(batch=20), t, flags=P.FLAG_INT8_WEIGHTS)         # tensor path
+    assert e.value.code == P.PRESERVE_ESHAPE
+    s = I.small_shape(batch=20, ctx=50, seed=151)
+    dl = G.DeviceLayer(s, I.make_layers(s, 1)[0], flags=P.FLAG_INT8_WEIGHTS | P.FLAG_FORCE_GEMV)
+    try:
+        info = dl.layer.get_info()
+        assert info.uses_tensor_path == 0
+        assert list(info.weight_bytes) == [512 * 1024, 512 * 512, 512 * 768, 384 * 512]   # one byte per weight
+    finally:
+        dl.close()
 
 
 def test_config3_chain_of_four_matches_oracle(oracle):
