@@ -407,6 +407,35 @@ def bench_config(P, I, torch, dist, args, idx, rank, local_rank, world, stream, 
         res["model"] = model
     except Exception as e:      # noqa: BLE001
         res["model"] = {"error": str(e)}
+    # ---- the same configuration with int8 weights (the weight precision of the paper's runs), where the
+    # library has them: the split-K GEMV path
+    if shape.batch < 16 and not args.no_sweep:
+        wl.close()
+        wl8 = Workload(P, I, torch, idx, rank, l2, args.rotation, flags=P.FLAG_INT8_WEIGHTS)
+        alg8 = int(P.preserve_algorithmic_bytes(wl8.cfg, shape.batch, wl8.sum_ctx))
+
+        def chain8():
+            P.preserve_decode_chain(wl8.layers, wl8.ios, link=False, stream=stream)
+        row = {"algorithmic_bytes_per_layer": alg8}
+        for name, b in (("off", 0), ("early_launch_only", 1)):
+            wl8.set_budget(b)
+            with torch.cuda.stream(stream):
+                for _ in range(3):
+                    chain8()
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(stream):
+                e0.record(stream)
+                for _ in range(n_min):
+                    chain8()
+                e1.record(stream)
+            barrier()
+            ms8 = max_over_ranks(e0.elapsed_time(e1) / n_min, world)
+            row[name + "_us_per_layer"] = round(ms8 * 1e3 / wl8.R, 3)
+            row[name + "_gbs"] = round(alg8 * wl8.R / (ms8 * 1e-3) / 1e9, 1)
+        row["speedup_vs_bf16_weights"] = round(us(ms_early) / row["early_launch_only_us_per_layer"], 4)
+        res["int8_weights"] = row
+        wl8.close()
     if headline and rank == 0 and args.cpu_baseline and world == 1:
         res["cpu_baseline"] = cpu_baseline(shape, wl.host_tensors, alg, budget_s=12.0, idx=idx)
     wl.close()
