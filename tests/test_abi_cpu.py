@@ -204,3 +204,23 @@ def test_graph_pass_truncate_mode_and_errors(lib, oracle):
     su = (C.c_int32 * 1)(1)
     assert lib.preserve_plan_graph(2, k, m, so, su, 10, 0, 0, None, None, None, C.byref(n_out)) == P.PRESERVE_ETOOBIG
     assert n_out.value == 1
+
+
+def test_no_process_wide_switches_in_the_kernels_sources():
+    """Distinct handles are independent: the sources keep no mutable process-wide switch (the early-launch
+    flag, the prefetch mechanism and chunk size are per handle and travel as launch arguments), read no
+    environment variable, and the only file-scope state left is per-device bookkeeping."""
+    csrc = os.path.join(ROOT, "paper_2501_08192_b200", "csrc")
+    allowed_static = ("static PerDeviceSize", "static __device__ __align__(256) unsigned char g_static_scratch",
+                      "static const int", "static const int32_t", "static_assert", "static_cast", "static cudaError_t",
+                      "static int reset_trace", "static size_t attn_smem_bytes", "static EncodeTiledFn fn",
+                      "static bool tried", "static constexpr")
+    for name in sorted(os.listdir(csrc)):
+        text = open(os.path.join(csrc, name)).read()
+        assert "getenv" not in text, name
+        for bad in ("g_pdl", "g_pf_mode", "g_pf_chunk", "static bool attr", "static bool np_set"):
+            assert bad not in text, (name, bad)
+        for line in text.splitlines():
+            st = line.strip()
+            if st.startswith("static ") and not st.startswith(allowed_static):
+                raise AssertionError(f"{name}: unexpected file-scope or function-scope static: {st}")
