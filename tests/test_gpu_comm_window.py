@@ -179,3 +179,67 @@ def test_external_attention_sum_and_argument_checks(oracle):
     h = C.c_void_p()
     assert P.lib().preserve_comm_create(0, 9, 4, 512, C.byref(h)) == P.PRESERVE_EINVAL
     assert P.lib().preserve_comm_create(3, 2, 4, 512, C.byref(h)) == P.PRESERVE_EINVAL
+
+
+def _peer_process(conn, shape_kw, a_bits, b_bits):
+    """A second PROCESS on the same GPU that only owns an exchange block: it fills its two buffers,
+    exports the block's handle and keeps the block alive until told to stop.  It launches no kernel
+    that waits for anything."""
+    import torch as _t
+    from paper_2501_08192_b200 import binding as _P
+    import gpu_util as _G
+    _t.cuda.set_device(0)
+    c = _P.Comm(1, 2, shape_kw["batch"], shape_kw["hidden"])
+    c.write(0, _G.bits_to_cuda(a_bits))
+    c.write(1, _G.bits_to_cuda(b_bits))
+    _t.cuda.synchronize()
+    conn.send(c.export_handle())
+    conn.recv()                      # parent is done
+    c.close()
+    conn.send("closed")
+
+
+def test_peer_block_of_another_process_is_read_through_its_ipc_handle(oracle):
+    """The exchange block of rank 1 lives in ANOTHER PROCESS (same GPU): rank 0 maps it from the
+    exported 64-byte handle, as it would map a peer GPU's block, and the fused window reads rank 1's
+    partial sums through that mapping.  Rank 1's arrival is set from the host (it runs no step)."""
+    import multiprocessing as mp
+    import os
+    import sys
+    shape = I.small_shape(name="comm_ipc", batch=4, hidden=512, ffn=256, tp_degree=2, ctx=60, ctx_min=3, seed=84)
+    t = I.make_layers(shape, 1)[0]
+    ref = oracle.layer_step(shape, t)
+    ctx = mp.get_context("spawn")
+    here, there = ctx.Pipe()
+    sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+    child = ctx.Process(target=_peer_process, args=(there, dict(batch=shape.batch, hidden=shape.hidden),
+                                                    t["partials_in"][1], t["attn_peer_partials"][0]))
+    child.start()
+    me = P.Comm(0, 2, shape.batch, shape.hidden)
+    dl = G.DeviceLayer(shape, t)
+    stream = torch.cuda.Stream()
+    try:
+        assert here.poll(120), "the peer process did not export its block"
+        me.import_handle(1, here.recv())
+        me.write(0, G.bits_to_cuda(t["partials_in"][0]))
+        me.debug_arrive(0, 1, FAR)
+        me.debug_arrive(1, 1, FAR)
+        dl.layer.set_comm(me)
+        with torch.cuda.stream(stream):
+            dl.run(stream)
+        stream.synchronize()
+        assert dl.layer.last_status_code() == 0
+        out = dl.outputs()
+        for name in ("attn_partial", "h2", "mlp_partial"):
+            G.assert_close(out[name], ref[name], name)
+        # importing the same rank twice, or the own rank, is refused
+        import ctypes as C
+        buf = (C.c_uint8 * 64)()
+        assert P.lib().preserve_comm_import(me.handle, 1, buf) == P.PRESERVE_EINVAL
+        assert P.lib().preserve_comm_import(me.handle, 0, buf) == P.PRESERVE_EINVAL
+    finally:
+        dl.close()
+        me.close()                    # unmaps the peer's block before the peer frees it
+        here.send("done")
+        child.join(timeout=60)
+        assert child.exitcode == 0
