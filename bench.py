@@ -490,6 +490,18 @@ def measure_streams(P, torch, stream, quick: bool = True):
                 rows.append({"buffer_mib": nbytes >> 20, "source": kind,
                              "path": f"cp.async.bulk {chunk} B x{stages} stages x{producers} lanes of one warp",
                              "ctas_per_sm": 1, "gbs": round(g, 1), "gbs_per_sm": round(g / sms, 2)})
+        # the tcgen05 GEMM's kind of load: 2-D tiled TMA boxes of 64 columns x 128 / 256 rows
+        for nbytes, kind in ((32 << 20, "l2"), (1 << 30, "hbm")):
+            passes = 40 if kind == "l2" else 2
+            for box_rows, stages, producers in ((256, 4, 1), (256, 2, 3), (128, 6, 1), (128, 4, 3)):
+                for per_sm in (1, 2):
+                    if per_sm * stages * box_rows * 128 * producers > 200 * 1024:
+                        continue
+                    g = P.preserve_measure_stream_tma(big, nbytes, passes, sms * per_sm, stages, box_rows, producers,
+                                                      status, stream)
+                    rows.append({"buffer_mib": nbytes >> 20, "source": kind,
+                                 "path": f"TMA 2-D box 64 x {box_rows} ({box_rows * 128} B) x{stages} stages x{producers} threads",
+                                 "ctas_per_sm": per_sm, "gbs": round(g, 1), "gbs_per_sm": round(g / sms, 2)})
     assert int(status[0].item()) == 0
     del big
     return rows

@@ -461,6 +461,14 @@ PRESERVE_API int preserve_measure_stream(const void *device_buffer, size_t bytes
                                          int32_t ctas, int32_t stages, uint32_t chunk_bytes, int32_t producers,
                                          int32_t *status_block, void *cuda_stream, float *gbs_out);
 
+/* The same measurement with the tcgen05 GEMM's kind of weight load: 2-D tiled TMA copies (128-byte
+ * swizzle) of boxes of 64 columns x box_rows rows (8..256, multiple of 8) out of the buffer viewed as
+ * a [bytes / 16384, 8192] bf16 matrix; CTA c walks the 128 column blocks of row tile c mod (number
+ * of tiles) `passes` times, its `producers` issuing threads taking every producers-th block. */
+PRESERVE_API int preserve_measure_stream_tma(const void *device_buffer, size_t bytes, int32_t passes, int32_t ctas,
+                                             int32_t stages, int32_t box_rows, int32_t producers,
+                                             int32_t *status_block, void *cuda_stream, float *gbs_out);
+
 /* Frees everything the library allocated for the handle (NULL is allowed). */
 PRESERVE_API void preserve_layer_destroy(preserve_layer_t *layer);
 

@@ -35,7 +35,7 @@ EXPORTS = (
     "preserve_last_status_code", "preserve_comm_create", "preserve_comm_export", "preserve_comm_import",
     "preserve_comm_set_peer", "preserve_comm_write", "preserve_comm_debug_arrive", "preserve_comm_epoch",
     "preserve_comm_destroy", "preserve_layer_set_comm", "preserve_layer_set_external_attention_sum",
-    "preserve_prefetch_window",
+    "preserve_prefetch_window", "preserve_measure_stream_tma",
 )
 NODE_COMM, NODE_MATMUL, NODE_ATTENTION, NODE_OTHER = 0, 1, 2, 3
 TRACE_SLOTS = 8
@@ -127,6 +127,8 @@ def lib() -> C.CDLL:
         L.preserve_comm_destroy.restype = None
         L.preserve_layer_set_comm.argtypes = [C.c_void_p, C.c_void_p]
         L.preserve_layer_set_external_attention_sum.argtypes = [C.c_void_p, C.c_void_p]
+        L.preserve_measure_stream_tma.argtypes = [C.c_void_p, C.c_size_t, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                                  C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(C.c_float)]
         L.preserve_layer_get_info.argtypes = [C.c_void_p, C.POINTER(Info)]
         L.preserve_last_status.argtypes = [C.c_void_p]
         L.preserve_last_cuda_error.argtypes = [C.c_void_p]
@@ -410,6 +412,16 @@ def preserve_measure_stream(buf, n_bytes: int, passes: int, path: int, ctas: int
     out = C.c_float()
     _check(lib().preserve_measure_stream(_ptr(buf), n_bytes, passes, path, ctas, stages, chunk_bytes, producers,
                                          _ptr(status), _stream_ptr(stream), C.byref(out)), "preserve_measure_stream")
+    return float(out.value)
+
+
+def preserve_measure_stream_tma(buf, n_bytes: int, passes: int, ctas: int, stages: int, box_rows: int,
+                                producers: int, status, stream=None) -> float:
+    """GB/s of 2-D tiled TMA loads (the tcgen05 GEMM's weight loads) over `buf` (see preserve.h)."""
+    out = C.c_float()
+    _check(lib().preserve_measure_stream_tma(_ptr(buf), n_bytes, passes, ctas, stages, box_rows, producers,
+                                             _ptr(status), _stream_ptr(stream), C.byref(out)),
+           "preserve_measure_stream_tma")
     return float(out.value)
 
 

@@ -106,7 +106,103 @@ __global__ void __launch_bounds__(32 * kStreamMaxProducers) k_stream_bulk(const 
     }
 }
 
+// path 3: the tcgen05 GEMM's weight loads - 2-D tiled TMA copies (128-byte swizzle) of boxes of 64 columns x
+// `rows` rows out of a [n_rows, 8192] bf16 matrix (row stride 16 KiB): CTA c walks the 128 column blocks of
+// row tile c mod n_tiles, `passes` times; producer w of the CTA takes the column blocks w, w + producers, ...
+struct StreamTmaParams {
+    CUtensorMap map;
+    int n_tiles, box_rows, passes, stages, producers;
+    uint32_t chunk;
+    int *status;
+};
+constexpr int kStreamK = 8192;
+__global__ void __launch_bounds__(32 * kStreamMaxProducers) k_stream_tma(const __grid_constant__ StreamTmaParams p)
+{
+    extern __shared__ uint8_t stream_smem_raw[];
+    uint8_t *ring0 = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(stream_smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ uint64_t bars[kStreamMaxProducers][kStreamMaxStages];
+    if ((threadIdx.x & 31) != 0)
+        return;
+    const int w = threadIdx.x >> 5;
+    uint8_t *ring = ring0 + (size_t)w * p.stages * p.chunk;
+    for (int i = 0; i < p.stages; ++i)
+        mbar_init(&bars[w][i], 1);
+    mbar_fence_init();
+    const int row0 = (int)(blockIdx.x % p.n_tiles) * p.box_rows;
+    const int kblocks = kStreamK / 64;
+    const int mine = (kblocks - w + p.producers - 1) / p.producers;      // column blocks of this producer per pass
+    const size_t total = (size_t)mine * p.passes;
+    for (size_t i = 0; i < total + p.stages; ++i) {
+        const int st = (int)(i % p.stages);
+        if (i >= (size_t)p.stages) {
+            const uint32_t ph = (uint32_t)((i / p.stages - 1) & 1);
+            if (!mbar_wait(&bars[w][st], ph, p.status, ST_TIMEOUT_FULL))
+                return;
+        }
+        if (i < total) {
+            const int kb = w + (int)(i % mine) * p.producers;
+            mbar_expect_tx(&bars[w][st], p.chunk);
+            tma_load_2d(ring + (size_t)st * p.chunk, &p.map, kb * 64, row0, &bars[w][st]);
+        }
+    }
+}
+
 }  // namespace prsv
+
+extern "C" int preserve_measure_stream_tma(const void *device_buffer, size_t bytes, int32_t passes, int32_t ctas,
+                                           int32_t stages, int32_t box_rows, int32_t producers, int32_t *status_block,
+                                           void *cuda_stream, float *gbs_out)
+{
+    using namespace prsv;
+    if (!device_buffer || !gbs_out || !status_block || passes < 1 || passes > 100000 || ctas < 1 || ctas > 4096 ||
+        (reinterpret_cast<uintptr_t>(device_buffer) & 127) || stages < 1 || stages > kStreamMaxStages ||
+        producers < 1 || producers > kStreamMaxProducers || box_rows < 8 || box_rows > 256 || box_rows % 8 ||
+        (size_t)stages * box_rows * 128 * producers > 200 * 1024)
+        return PRESERVE_EINVAL;
+    const size_t n_rows = bytes / ((size_t)kStreamK * 2);
+    StreamTmaParams p = {};
+    p.n_tiles = (int)(n_rows / box_rows);
+    if (p.n_tiles < 1)
+        return PRESERVE_EINVAL;
+    if (!encode_bf16_map_2d(&p.map, device_buffer, kStreamK, n_rows, 64, (uint32_t)box_rows))
+        return PRESERVE_EARCH;
+    p.box_rows = box_rows;
+    p.stages = stages;
+    p.producers = producers;
+    p.chunk = (uint32_t)box_rows * 128u;
+    p.status = status_block;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const size_t smem = (size_t)stages * p.chunk * producers + 1024;
+    static PerDeviceSize lim;
+    if (ensure_dynamic_smem(k_stream_tma, lim, smem) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return PRESERVE_ECUDA;
+    }
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return PRESERVE_ECUDA;
+    }
+    StreamTmaParams q = p;
+    q.passes = 1;
+    k_stream_tma<<<ctas, 32 * producers, smem, s>>>(q);
+    cudaEventRecord(e0, s);
+    p.passes = passes;
+    k_stream_tma<<<ctas, 32 * producers, smem, s>>>(p);
+    cudaEventRecord(e1, s);
+    cudaError_t err = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    if (err == cudaSuccess)
+        err = cudaEventElapsedTime(&ms, e0, e1);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (err != cudaSuccess || ms <= 0.f) {
+        (void)cudaGetLastError();
+        return PRESERVE_ECUDA;
+    }
+    *gbs_out = (float)((double)box_rows * kStreamK * 2.0 * ctas * passes / (ms * 1e-3) / 1e9);
+    return PRESERVE_OK;
+}
 
 extern "C" int preserve_measure_stream(const void *device_buffer, size_t bytes, int32_t passes, int32_t path,
                                        int32_t ctas, int32_t stages, uint32_t chunk_bytes, int32_t producers,
