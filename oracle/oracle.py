@@ -45,6 +45,13 @@ class _Out(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in _OUT_NAMES]
 
 
+_KV8_NAMES = ("k_codes", "v_codes", "k_scales", "v_scales", "k_codes_new", "v_codes_new", "k_scale_new", "v_scale_new")
+
+
+class _Kv8(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in _KV8_NAMES]
+
+
 _lib = None
 
 
@@ -55,6 +62,7 @@ def lib():
         _lib.oracle_num_threads.restype = C.c_int
         _lib.oracle_layer_step.restype = C.c_int
         _lib.oracle_layer_step_w8.restype = C.c_int
+        _lib.oracle_layer_step_kv8.restype = C.c_int
     return _lib
 
 
@@ -150,9 +158,49 @@ def matmul_q8(x, q, scale):
     return y
 
 
+def quantize_rows(u):
+    """Symmetric int8 quantisation with one scale per vector (last axis): (codes int8, scale f32)."""
+    u = _f32(u)
+    d = u.shape[-1]
+    q = np.empty(u.shape, np.int8)
+    sc = np.empty(u.shape[:-1], np.float32)
+    lib().oracle_quantize_rows(C.c_size_t(u.size // d), C.c_int(d), _p(u), _p(q), _p(sc))
+    return q, sc
+
+
+def _i8(a) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.int8, a.dtype
+    return a
+
+
+def attention_kv8(q, kq_new, ks_new, vq_new, vs_new, k_codes, k_scales, v_codes, v_scales, ctx_len,
+                  want_probs: bool = False):
+    """Decode attention over an int8 cache: codes int8 [B,nkv,cap,d], scales f32 [B,nkv,cap]; the new
+    entry as codes [B,nkv,d] and scales [B,nkv]."""
+    q = _f32(q)
+    kq_new, vq_new, k_codes, v_codes = _i8(kq_new), _i8(vq_new), _i8(k_codes), _i8(v_codes)
+    ks_new, vs_new, k_scales, v_scales = _f32(ks_new), _f32(vs_new), _f32(k_scales), _f32(v_scales)
+    ctx_len = np.ascontiguousarray(ctx_len, dtype=np.int32)
+    B, nq, d = q.shape
+    _, nkv, cap, _ = k_codes.shape
+    assert k_scales.shape == (B, nkv, cap) and v_scales.shape == (B, nkv, cap)
+    o = np.empty((B, nq, d), np.float32)
+    probs = np.zeros((B, nq, cap), np.float32) if want_probs else None
+    lib().oracle_attention_kv8(C.c_int(B), C.c_int(nq), C.c_int(nkv), C.c_int(d), C.c_int(cap), _p(ctx_len),
+                               _p(q), _p(kq_new), _p(ks_new), _p(vq_new), _p(vs_new), _p(k_codes), _p(k_scales),
+                               _p(v_codes), _p(v_scales), _p(o), _p(probs) if want_probs else C.c_void_p(0))
+    return (o, probs) if want_probs else o
+
+
 def layer_step(shape, t: Dict[str, np.ndarray], partials_in=None, residual_in=None,
-               peer_partials=None, int8_weights: bool = False) -> Dict[str, np.ndarray]:
+               peer_partials=None, int8_weights: bool = False, kv8: Optional[Dict[str, np.ndarray]] = None
+               ) -> Dict[str, np.ndarray]:
     """One decode step of one shard's layer.
+
+    kv8 = {"k_codes", "k_scales", "v_codes", "v_scales"} runs the step over that int8 KV-cache
+    instead of t's bf16 cache; the result then also holds the appended entry as stored
+    ("k_codes_new" int8 [B,nkv,d], "k_scale_new" f32 [B,nkv], and the same for v).
 
     `shape` needs hidden, n_q_heads, n_kv_heads, head_dim, ffn, tp_degree,
     rms_eps, rope_theta.  `t` holds the bf16-bit tensors of inputs.make_layer.
@@ -163,8 +211,11 @@ def layer_step(shape, t: Dict[str, np.ndarray], partials_in=None, residual_in=No
         return (np.ascontiguousarray(b, np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
 
     P = shape.tp_degree
-    kc, vc = _u16(t["k_cache"]), _u16(t["v_cache"])
-    B, nkv, cap, d = kc.shape
+    if kv8 is None:
+        kc, vc = _u16(t["k_cache"]), _u16(t["v_cache"])
+        B, nkv, cap, d = kc.shape
+    else:
+        B, nkv, cap, d = kv8["k_codes"].shape
     H = shape.hidden
     parts = _f32(widen(t["partials_in"]) if partials_in is None else partials_in).reshape(P, B, H)
     resid = _f32(widen(t["residual_in"]) if residual_in is None else residual_in).reshape(B, H)
@@ -182,6 +233,20 @@ def layer_step(shape, t: Dict[str, np.ndarray], partials_in=None, residual_in=No
     res = {n: np.empty(s, np.float32) for n, s in sizes.items()}
     out = _Out(*[res[n].ctypes.data for n in _OUT_NAMES])
     w = [_u16(t[n]) for n in ("w_q", "w_k", "w_v", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")]
+    if kv8 is not None:
+        keep = [_i8(kv8["k_codes"]), _i8(kv8["v_codes"]), _f32(kv8["k_scales"]), _f32(kv8["v_scales"])]
+        assert keep[2].shape == (B, nkv, cap) and keep[3].shape == (B, nkv, cap)
+        res["k_codes_new"] = np.empty((B, nkv, d), np.int8)
+        res["v_codes_new"] = np.empty((B, nkv, d), np.int8)
+        res["k_scale_new"] = np.empty((B, nkv), np.float32)
+        res["v_scale_new"] = np.empty((B, nkv), np.float32)
+        kv = _Kv8(*[a.ctypes.data for a in keep],
+                  *[res[n].ctypes.data for n in ("k_codes_new", "v_codes_new", "k_scale_new", "v_scale_new")])
+        rc = lib().oracle_layer_step_kv8(C.byref(cfg), *[_p(a) for a in w], _p(ctx_len), _p(parts), _p(peers),
+                                         _p(resid), C.byref(kv), C.c_int(1 if int8_weights else 0), C.byref(out))
+        if rc != 0:
+            raise ValueError("oracle_layer_step_kv8 rejected the configuration")
+        return res
     fn = lib().oracle_layer_step_w8 if int8_weights else lib().oracle_layer_step
     rc = fn(C.byref(cfg), *[_p(a) for a in w], _p(ctx_len), _p(parts), _p(peers),
             _p(resid), _p(kc), _p(vc), C.byref(out))

@@ -44,7 +44,12 @@
  * repeated KV heads, split-and-merge of the key range, RMSNorm closed forms,
  * identity / one-hot projections, RoPE norm and relative-position invariants,
  * silu constants, sum over both shards == unsharded layer, and an independent
- * torch-CPU restatement of the layer.
+ * torch-CPU restatement of the layer.  The int8 variants (weights per output
+ * channel; KV-cache per cached vector) have their own pins: hand-worked vectors,
+ * the half-step error bound, symmetry and power-of-two covariance of the
+ * quantisers, brute force on the dequantised arrays, agreement with the bf16
+ * routines on data that both represent exactly, and the torch restatement with
+ * its own quantiser.
  */
 #include <math.h>
 #include <stdint.h>
@@ -80,6 +85,13 @@ typedef struct {          /* caller-allocated fp32 outputs; any may be NULL */
     float *a;             /* [B,F]  SwiGLU activation                     */
     float *mlp_partial;   /* [B,H]  a . W_down                            */
 } oracle_out_t;
+
+typedef struct {          /* int8 KV-cache of a step (see oracle_quantize_rows)              */
+    const int8_t *k_codes, *v_codes;    /* [B,nkv,cap,d]                                    */
+    const float *k_scales, *v_scales;   /* [B,nkv,cap]                                      */
+    int8_t *k_codes_new, *v_codes_new;  /* optional outputs [B,nkv,d]: the appended entry   */
+    float *k_scale_new, *v_scale_new;   /* optional outputs [B,nkv]                         */
+} oracle_kv8_t;
 
 static inline float bf16f(uint16_t b)
 {
@@ -292,6 +304,83 @@ void oracle_attention(int B, int nq, int nkv, int d, int cap, const int32_t *ctx
     }
 }
 
+/* ---- int8 KV-cache (the precision of the paper's measurements: Section 4, "Experimental setup").
+ * The paper does not say how its int8 cache is scaled; reading: symmetric quantisation with one
+ * scale per cached vector, i.e. per (sequence, kv head, slot), keys and values alike.  For a vector
+ * u of d values: scale = max_i |u_i| / 127 (fp32 division), code_i = round-to-nearest-even(u_i / scale)
+ * in fp32, an integer in [-127, 127]; a vector of zeros has scale 0 and codes 0.  The cache holds
+ * the codes and the scales, and the value a slot stands for is code * scale.  Every decision is
+ * taken in fp32, so a CUDA side that is given the same fp32 vector produces the same codes. */
+void oracle_quantize_rows(size_t n_rows, int d, const float *u, int8_t *q, float *scale)
+{
+    for (size_t r = 0; r < n_rows; ++r) {
+        const float *v = u + r * (size_t)d;
+        float mx = 0.f;
+        for (int i = 0; i < d; ++i)
+            if (fabsf(v[i]) > mx)
+                mx = fabsf(v[i]);
+        float sc = mx / 127.0f;
+        scale[r] = sc;
+        for (int i = 0; i < d; ++i) {
+            float c = sc > 0.f ? rintf(v[i] / sc) : 0.f;
+            if (c > 127.f) c = 127.f;
+            if (c < -127.f) c = -127.f;
+            q[r * (size_t)d + i] = (int8_t)c;
+        }
+    }
+}
+
+/* Decode attention over an int8 cache.  q [B,nq,d] fp32; the entry of slot ctx_len[b] is given
+ * already quantised: kq_new, vq_new int8 [B,nkv,d] with ks_new, vs_new [B,nkv]; the cache is
+ * k_codes, v_codes int8 [B,nkv,cap,d] with k_scales, v_scales fp32 [B,nkv,cap] (slots < ctx_len[b]
+ * are read).  Every key and value enters as code * scale; o [B,nq,d]; probs optional [B,nq,cap]. */
+void oracle_attention_kv8(int B, int nq, int nkv, int d, int cap, const int32_t *ctx_len, const float *q,
+                          const int8_t *kq_new, const float *ks_new, const int8_t *vq_new, const float *vs_new,
+                          const int8_t *k_codes, const float *k_scales, const int8_t *v_codes,
+                          const float *v_scales, float *o, float *probs)
+{
+    int G = nq / nkv;
+    double scale = 1.0 / sqrt((double)d);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int bh = 0; bh < B * nq; ++bh) {
+        int b = bh / nq, hq = bh % nq, g = hq / G;
+        int t = ctx_len[b];
+        size_t stream = (size_t)b * nkv + g;
+        const float *qv = q + ((size_t)b * nq + hq) * d;
+        double *s = (double *)malloc(sizeof(double) * (size_t)(t + 1));
+        double *acc = (double *)calloc((size_t)d, sizeof(double));
+        double mx = -INFINITY;
+        for (int j = 0; j <= t; ++j) {
+            const int8_t *kc = j < t ? k_codes + (stream * (size_t)cap + j) * d : kq_new + stream * d;
+            double ks = j < t ? (double)k_scales[stream * (size_t)cap + j] : (double)ks_new[stream];
+            double dot = 0.0;
+            for (int i = 0; i < d; ++i)
+                dot += (double)qv[i] * ((double)kc[i] * ks);
+            s[j] = dot * scale;
+            if (s[j] > mx)
+                mx = s[j];
+        }
+        double den = 0.0;
+        for (int j = 0; j <= t; ++j) {
+            s[j] = exp(s[j] - mx);
+            den += s[j];
+        }
+        for (int j = 0; j <= t; ++j) {
+            const int8_t *vc = j < t ? v_codes + (stream * (size_t)cap + j) * d : vq_new + stream * d;
+            double vs = j < t ? (double)v_scales[stream * (size_t)cap + j] : (double)vs_new[stream];
+            double p = s[j] / den;
+            if (probs)
+                probs[((size_t)b * nq + hq) * cap + j] = (float)p;
+            for (int i = 0; i < d; ++i)
+                acc[i] += p * ((double)vc[i] * vs);
+        }
+        for (int i = 0; i < d; ++i)
+            o[((size_t)b * nq + hq) * d + i] = (float)acc[i];
+        free(s);
+        free(acc);
+    }
+}
+
 /* a[i] = silu(gate[i]) * up[i] */
 void oracle_swiglu(size_t n, const float *gate, const float *up, float *a)
 {
@@ -313,7 +402,8 @@ static int layer_step_impl(const oracle_cfg_t *c, const uint16_t *w_q, const uin
                            const uint16_t *w_up, const uint16_t *w_down, const uint16_t *g_attn,
                            const uint16_t *g_mlp, const int32_t *ctx_len, const float *partials_in,
                            const float *peer_partials, const float *residual_in,
-                           const uint16_t *k_cache, const uint16_t *v_cache, oracle_out_t *out, int w8)
+                           const uint16_t *k_cache, const uint16_t *v_cache, oracle_out_t *out, int w8,
+                           const oracle_kv8_t *kv8)
 {
     int B = c->batch, H = c->hidden, nq = c->n_q_heads, nkv = c->n_kv_heads, d = c->head_dim;
     int F = c->ffn, P = c->tp_degree, cap = c->kv_capacity;
@@ -344,13 +434,34 @@ static int layer_step_impl(const oracle_cfg_t *c, const uint16_t *w_q, const uin
         oracle_rope(nq, d, ctx_len[b], c->rope_theta, q + (size_t)b * nq * d);
         oracle_rope(nkv, d, ctx_len[b], c->rope_theta, kn + (size_t)b * nkv * d);
     }
-    /* append: the new entry is stored in the bf16 cache; attention reads it from there */
-    for (size_t i = 0; i < (size_t)B * nkv * d; ++i) {
-        kn_c[i] = round_to_bf16(kn[i]);
-        vn_c[i] = round_to_bf16(vn[i]);
+    if (!kv8) {
+        /* append: the new entry is stored in the bf16 cache; attention reads it from there */
+        for (size_t i = 0; i < (size_t)B * nkv * d; ++i) {
+            kn_c[i] = round_to_bf16(kn[i]);
+            vn_c[i] = round_to_bf16(vn[i]);
+        }
+        /* self-attention over the cached entries plus the new one */
+        oracle_attention(B, nq, nkv, d, cap, ctx_len, q, kn_c, vn_c, k_cache, v_cache, o, NULL);
+    } else {
+        /* append: the new entry is stored in the int8 cache (codes and one scale per vector);
+         * attention reads every entry, the new one included, as code * scale */
+        size_t nv = (size_t)B * nkv;
+        int8_t *kq = (int8_t *)malloc(nv * d), *vq = (int8_t *)malloc(nv * d);
+        float *ks = falloc(nv), *vs = falloc(nv);
+        if (!kq || !vq || !ks || !vs) {
+            free(kq); free(vq); free(ks); free(vs);
+            goto done;
+        }
+        oracle_quantize_rows(nv, d, kn, kq, ks);
+        oracle_quantize_rows(nv, d, vn, vq, vs);
+        oracle_attention_kv8(B, nq, nkv, d, cap, ctx_len, q, kq, ks, vq, vs, kv8->k_codes, kv8->k_scales,
+                             kv8->v_codes, kv8->v_scales, o, NULL);
+        if (kv8->k_codes_new) memcpy(kv8->k_codes_new, kq, nv * d);
+        if (kv8->v_codes_new) memcpy(kv8->v_codes_new, vq, nv * d);
+        if (kv8->k_scale_new) memcpy(kv8->k_scale_new, ks, sizeof(float) * nv);
+        if (kv8->v_scale_new) memcpy(kv8->v_scale_new, vs, sizeof(float) * nv);
+        free(kq); free(vq); free(ks); free(vs);
     }
-    /* self-attention over the cached entries plus the new one */
-    oracle_attention(B, nq, nkv, d, cap, ctx_len, q, kn_c, vn_c, k_cache, v_cache, o, NULL);
     /* output projection: this shard's partial sum */
     layer_matmul(B, nq * d, H, o, w_o, ap, w8);
     /* window B: own partial + the P-1 peers' partials + h, then RMSNorm */
@@ -393,7 +504,7 @@ int oracle_layer_step(const oracle_cfg_t *c, const uint16_t *w_q, const uint16_t
                       const uint16_t *k_cache, const uint16_t *v_cache, oracle_out_t *out)
 {
     return layer_step_impl(c, w_q, w_k, w_v, w_o, w_gate, w_up, w_down, g_attn, g_mlp, ctx_len, partials_in,
-                           peer_partials, residual_in, k_cache, v_cache, out, 0);
+                           peer_partials, residual_in, k_cache, v_cache, out, 0, NULL);
 }
 
 /* The same step with every projection's weights quantised to int8 per output channel
@@ -406,5 +517,20 @@ int oracle_layer_step_w8(const oracle_cfg_t *c, const uint16_t *w_q, const uint1
                          const uint16_t *k_cache, const uint16_t *v_cache, oracle_out_t *out)
 {
     return layer_step_impl(c, w_q, w_k, w_v, w_o, w_gate, w_up, w_down, g_attn, g_mlp, ctx_len, partials_in,
-                           peer_partials, residual_in, k_cache, v_cache, out, 1);
+                           peer_partials, residual_in, k_cache, v_cache, out, 1, NULL);
+}
+
+/* The same step over an int8 KV-cache (oracle_quantize_rows, oracle_attention_kv8); the weights are
+ * bf16 (int8_weights == 0) or quantised per output channel as in oracle_layer_step_w8. */
+int oracle_layer_step_kv8(const oracle_cfg_t *c, const uint16_t *w_q, const uint16_t *w_k,
+                          const uint16_t *w_v, const uint16_t *w_o, const uint16_t *w_gate,
+                          const uint16_t *w_up, const uint16_t *w_down, const uint16_t *g_attn,
+                          const uint16_t *g_mlp, const int32_t *ctx_len, const float *partials_in,
+                          const float *peer_partials, const float *residual_in, const oracle_kv8_t *kv8,
+                          int int8_weights, oracle_out_t *out)
+{
+    if (!kv8 || !kv8->k_codes || !kv8->v_codes || !kv8->k_scales || !kv8->v_scales)
+        return -1;
+    return layer_step_impl(c, w_q, w_k, w_v, w_o, w_gate, w_up, w_down, g_attn, g_mlp, ctx_len, partials_in,
+                           peer_partials, residual_in, NULL, NULL, out, int8_weights ? 1 : 0, kv8);
 }

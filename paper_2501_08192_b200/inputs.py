@@ -174,6 +174,32 @@ def make_layer(shape: ShardShape, rng: np.random.Generator, shard: int = 0,
     return t
 
 
+def make_int8_cache(shape: ShardShape, ctx_len: np.ndarray, seed: int = 0) -> Dict[str, np.ndarray]:
+    """A seeded int8 KV-cache for `shape`: codes int8 [batch, n_kv, ctx+1, head_dim] and one fp32
+    scale per cached vector [batch, n_kv, ctx+1], for keys and for values.  Codes are N(0, 42^2)
+    rounded and clipped to [-127, 127]; scales are 0.02 + 0.01 |N(0, 1)|, so the cached values
+    (code * scale) have about unit variance like the bf16 cache.  Slots at and beyond ctx_len[b]
+    hold code -128 and a NaN scale, so that a read past the length or a missing append shows up.
+    Draw order: K codes, K scales, V codes, V scales."""
+    rng = np.random.Generator(np.random.PCG64([shape.seed, 0x6b76, seed]))
+    B, nkv, cap, d = shape.batch, shape.n_kv_heads, shape.kv_capacity, shape.head_dim
+    out: Dict[str, np.ndarray] = {}
+    for name in ("k", "v"):
+        codes = np.empty((B, nkv, cap, d), np.int8)
+        for b in range(B):                                     # per sequence: bounded temporary
+            v = rng.standard_normal((nkv, cap, d), dtype=np.float32) * np.float32(42.0)
+            codes[b] = np.clip(np.rint(v), -127, 127).astype(np.int8)
+        scales = (np.float32(0.02) + np.float32(0.01) * np.abs(rng.standard_normal((B, nkv, cap), dtype=np.float32))
+                  ).astype(np.float32)
+        for b in range(B):
+            n = int(ctx_len[b])
+            codes[b, :, n:] = -128
+            scales[b, :, n:] = np.nan
+        out[name + "_codes"] = codes
+        out[name + "_scales"] = scales
+    return out
+
+
 def make_layers(shape: ShardShape, n_instances: Optional[int] = None, shard: int = 0,
                 nan_fill_tail: bool = True) -> List[Dict[str, np.ndarray]]:
     """All layer instances of a configuration from one PCG64 stream seeded by shape.seed."""

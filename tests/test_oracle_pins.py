@@ -281,8 +281,16 @@ def test_rope_invariants(oracle):
 
 
 # ---------------------------------------------------------------- whole layer
-def torch_layer(shape, t, parts=None, resid=None, peers=None):
-    """Independent restatement of the layer with torch CPU ops in fp64."""
+def torch_quantize_rows(u):
+    """Per-vector symmetric int8 with torch ops: fp32 division and round-half-even, as the reading says."""
+    u = u.float()
+    sc = u.abs().amax(-1, keepdim=True) / 127.0
+    codes = torch.where(sc > 0, torch.round(u / sc), torch.zeros_like(u)).clamp(-127, 127)
+    return codes.double(), sc.double()
+
+
+def torch_layer(shape, t, parts=None, resid=None, peers=None, kv8=None):
+    """Independent restatement of the layer with torch CPU ops in fp64 (kv8: over that int8 cache)."""
     W = lambda n: torch.from_numpy(widen(t[n])).double()
     P, d, nq, nkv = shape.tp_degree, shape.head_dim, shape.n_q_heads, shape.n_kv_heads
     parts = W("partials_in") if parts is None else torch.from_numpy(parts).double()
@@ -306,8 +314,16 @@ def torch_layer(shape, t, parts=None, resid=None, peers=None):
         return torch.cat([u1 * ang.cos() - u2 * ang.sin(), u2 * ang.cos() + u1 * ang.sin()], -1)
 
     q, k = rot(q), rot(k)
-    k_st, v_st = k.bfloat16().double(), v.bfloat16().double()     # the new entry as the bf16 cache stores it
-    Kc, Vc = W("k_cache").clone(), W("v_cache").clone()
+    if kv8 is None:
+        k_st, v_st = k.bfloat16().double(), v.bfloat16().double()     # the new entry as the bf16 cache stores it
+        Kc, Vc = W("k_cache").clone(), W("v_cache").clone()
+    else:
+        kq, ks = torch_quantize_rows(k)                               # the new entry as the int8 cache stores it
+        vq, vs = torch_quantize_rows(v)
+        k_st, v_st = kq * ks, vq * vs
+        deq = lambda c, s_: torch.from_numpy(kv8[c].astype(np.float64)) * torch.from_numpy(
+            np.nan_to_num(kv8[s_].astype(np.float64)))[..., None]
+        Kc, Vc = deq("k_codes", "k_scales"), deq("v_codes", "v_scales")
     o = torch.zeros(B, nq, d, dtype=torch.float64)
     G = nq // nkv
     for b in range(B):
@@ -495,3 +511,101 @@ def test_int8_matmul_and_layer_against_independent_restatements(oracle):
     v_ref = (torch.from_numpy(q2["x"].astype(np.float64)) @ torch.from_numpy(
         oracle.quantize_weights(t2["w_v"])[0].astype(np.float64) * oracle.quantize_weights(t2["w_v"])[1].astype(np.float64)))
     assert np.allclose(v_ref.numpy().reshape(q2["v_new"].shape), q2["v_new"], rtol=1e-5, atol=1e-6)
+
+
+# ---------------------------------------------------------------- int8 KV-cache (one scale per cached vector)
+def test_int8_row_quantiser_closed_forms(oracle):
+    """Pins of oracle_quantize_rows that do not retype its loop: hand-worked vectors (ties go to the even
+    code), the zero vector, the extreme code at the largest entry, the half-step error bound, odd
+    symmetry, and exact covariance with a power-of-two factor."""
+    hand = np.array([[127.0, -63.5, 0.0, 1.0], [0.5, 0.25, -0.5, 0.125], [0.0, 0.0, 0.0, 0.0]], np.float32)
+    q, sc = oracle.quantize_rows(hand)
+    assert q[0].tolist() == [127, -64, 0, 1] and sc[0] == 1.0
+    assert q[1].tolist() == [127, 64, -127, 32] and abs(sc[1] - 0.5 / 127) < 1e-9
+    assert not q[2].any() and sc[2] == 0.0
+    rng = np.random.default_rng(8)
+    u = (rng.standard_normal((50, 128)) * rng.uniform(0.01, 30.0, (50, 1))).astype(np.float32)
+    q, sc = oracle.quantize_rows(u)
+    assert q.dtype == np.int8 and q.min() >= -127 and q.max() <= 127
+    assert np.allclose(sc, np.abs(u).max(-1) / 127.0, rtol=1e-6)
+    assert (np.abs(q[np.arange(50), np.abs(u).argmax(-1)]) == 127).all()
+    assert (np.abs(q.astype(np.float64) * sc[:, None] - u) <= 0.5000001 * sc[:, None]).all()
+    qn, scn = oracle.quantize_rows(-u)
+    assert np.array_equal(qn, -q) and np.array_equal(scn, sc)
+    q8, sc8 = oracle.quantize_rows(u * np.float32(2.0 ** -7))
+    assert np.array_equal(q8, q) and np.array_equal(sc8, sc * np.float32(2.0 ** -7))
+    # shape handling: leading axes are independent vectors
+    q3, sc3 = oracle.quantize_rows(u.reshape(5, 10, 128))
+    assert np.array_equal(q3.reshape(50, 128), q) and np.array_equal(sc3.reshape(50), sc)
+
+
+def test_int8_attention_against_brute_force_and_the_bf16_routine(oracle):
+    """oracle_attention_kv8 against the brute-force softmax on the dequantised arrays, and against
+    the (separately pinned) bf16 attention on a cache whose entries code * 2^-5 are exact in bf16."""
+    rng = np.random.default_rng(9)
+    B, nq, nkv, d, cap = 2, 4, 2, 8, 11
+    lens = np.array([4, 10], np.int32)
+    q = rng.standard_normal((B, nq, d)).astype(np.float32)
+    codes = lambda *s: rng.integers(-127, 128, size=s).astype(np.int8)
+    kc, vc = codes(B, nkv, cap, d), codes(B, nkv, cap, d)
+    ks = rng.uniform(0.005, 0.02, (B, nkv, cap)).astype(np.float32)
+    vs = rng.uniform(0.005, 0.02, (B, nkv, cap)).astype(np.float32)
+    kqn, vqn = codes(B, nkv, d), codes(B, nkv, d)
+    ksn = rng.uniform(0.005, 0.02, (B, nkv)).astype(np.float32)
+    vsn = rng.uniform(0.005, 0.02, (B, nkv)).astype(np.float32)
+    for b in range(B):                      # dead slots must not be read
+        kc[b, :, lens[b]:], vc[b, :, lens[b]:] = -128, -128
+        ks[b, :, lens[b]:], vs[b, :, lens[b]:] = np.nan, np.nan
+    o, probs = oracle.attention_kv8(q, kqn, ksn, vqn, vsn, kc, ks, vc, vs, lens, want_probs=True)
+    G = nq // nkv
+    for b in range(B):
+        n = int(lens[b])
+        for h in range(nq):
+            g = h // G
+            keys = np.concatenate([kc[b, g, :n].astype(np.float64) * ks[b, g, :n, None].astype(np.float64),
+                                   (kqn[b, g].astype(np.float64) * float(ksn[b, g]))[None]])
+            vals = np.concatenate([vc[b, g, :n].astype(np.float64) * vs[b, g, :n, None].astype(np.float64),
+                                   (vqn[b, g].astype(np.float64) * float(vsn[b, g]))[None]])
+            want, p = brute_attention(q[b, h].astype(np.float64), keys, vals)
+            assert np.allclose(o[b, h], want, rtol=1e-6, atol=1e-7)
+            assert np.allclose(probs[b, h, :n + 1], p, rtol=1e-6, atol=1e-8) and abs(probs[b, h, :n + 1].sum() - 1) < 1e-6
+    # power-of-two scales: every code * scale is a bf16 number, so the bf16 routine sees the same cache
+    ks2 = np.full_like(ks, 2.0 ** -5)
+    vs2 = np.full_like(vs, 2.0 ** -6)
+    kb = I.f32_to_bf16_bits(kc.astype(np.float32) * ks2[..., None])
+    vb = I.f32_to_bf16_bits(vc.astype(np.float32) * vs2[..., None])
+    assert np.array_equal(I.bf16_bits_to_f32(kb), kc.astype(np.float32) * ks2[..., None])
+    ksn2, vsn2 = np.full_like(ksn, 2.0 ** -5), np.full_like(vsn, 2.0 ** -6)
+    o8 = oracle.attention_kv8(q, kqn, ksn2, vqn, vsn2, kc, ks2, vc, vs2, lens)
+    o16 = oracle.attention(q, kqn.astype(np.float32) * ksn2[..., None], vqn.astype(np.float32) * vsn2[..., None], kb, vb, lens)
+    assert np.allclose(o8, o16, rtol=1e-6, atol=1e-7)
+
+
+def test_int8_kv_layer_against_torch_restatement(oracle):
+    """The layer step over an int8 cache against the torch restatement (its own quantiser, its own
+    dequantisation), with bf16 and with int8 weights; the stored new entry is the quantised k_new, v_new."""
+    for shape in (I.small_shape(name="kv8", batch=3, ctx=90, ctx_min=4, seed=95),
+                  I.small_shape(name="kv8_mha", n_q_heads=2, n_kv_heads=2, batch=1, tp_degree=1, ctx=37, seed=96)):
+        t = I.make_layers(shape, 1)[0]
+        kv = I.make_int8_cache(shape, t["ctx_len"])
+        got = oracle.layer_step(shape, t, kv8=kv)
+        ref = torch_layer(shape, t, kv8=kv)
+        for name, r in ref.items():
+            r = r.numpy()
+            np.testing.assert_allclose(got[name].reshape(r.shape), r, rtol=1e-4,
+                                       atol=1e-5 * max(1.0, float(np.abs(r).max())), err_msg=name)
+        kq, ks = torch_quantize_rows(torch.from_numpy(got["k_new"]))
+        vq, vs = torch_quantize_rows(torch.from_numpy(got["v_new"]))
+        assert np.array_equal(got["k_codes_new"], kq.numpy().astype(np.int8))
+        assert np.array_equal(got["v_codes_new"], vq.numpy().astype(np.int8))
+        assert np.allclose(got["k_scale_new"], ks.numpy()[..., 0], rtol=1e-7) and np.allclose(got["v_scale_new"], vs.numpy()[..., 0], rtol=1e-7)
+        # the int8 cache changes the result (it is not the bf16 path in disguise) and composes with int8 weights
+        plain = oracle.layer_step(shape, t)
+        assert not np.allclose(plain["o"], got["o"], rtol=1e-3, atol=1e-4)
+        both = oracle.layer_step(shape, t, kv8=kv, int8_weights=True)
+        w8 = oracle.layer_step(shape, t, int8_weights=True)
+        assert np.array_equal(both["x"], w8["x"]) and np.array_equal(both["q"], w8["q"])
+        o_again = oracle.attention_kv8(both["q"], both["k_codes_new"], both["k_scale_new"], both["v_codes_new"],
+                                       both["v_scale_new"], kv["k_codes"], kv["k_scales"], kv["v_codes"], kv["v_scales"],
+                                       t["ctx_len"])
+        assert np.array_equal(o_again, both["o"])
