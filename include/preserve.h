@@ -93,6 +93,16 @@ extern "C" {
                                        of the paper's measurements (Section 4, "Experimental setup"); activations
                                        and the KV-cache stay bf16.  Split-K GEMV path only (max_batch < 16 or
                                        PRESERVE_FLAG_FORCE_GEMV), ffn a multiple of 64; PRESERVE_ESHAPE otherwise */
+#define PRESERVE_FLAG_INT8_KV 64u      /* the KV-cache is int8 with one fp32 scale per cached vector, i.e. per
+                                       (sequence, kv head, slot): scale = max |u| / 127 over the vector's head_dim
+                                       values, code = round-to-nearest-even(u / scale), decided in fp32; a cached
+                                       value is code * scale (the cache precision of the paper's measurements,
+                                       Section 4 "Experimental setup"; the scaling is this library's reading).
+                                       k_cache and v_cache then each point to ONE buffer laid out as
+                                       preserve_kv8_layout says: the codes, then the scales.  The step quantises its
+                                       new key and value, stores them at slot ctx_len[b] and attends over the
+                                       cache as stored.  At most 8 query heads per KV head; PRESERVE_ESHAPE
+                                       otherwise.  preserve_attention_static does not take this layout.      */
 #define PRESERVE_FLAG_FORCE_TENSOR 16u /* use the tcgen05 GEMM kernels although max_batch < 16 (needs ffn
                                        to be a multiple of 128)                                       */
 
@@ -187,6 +197,15 @@ typedef struct {
  * prefetch_budget; see preserve_set_prefetch_bytes), mode PRESERVE_PLAN_TRUNCATE. */
 PRESERVE_API int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer_weights_t *w,
                         preserve_layer_t **out);
+
+/* Layout of one int8 cache buffer (PRESERVE_FLAG_INT8_KV) for a configuration: bytes [0, S * cap * head_dim)
+ * hold the codes, int8 [max_batch, n_kv_heads, cap, head_dim] with cap = max_ctx + 1 and S = max_batch *
+ * n_kv_heads; the scales follow at *scale_offset_bytes (the code bytes rounded up to 256): fp32 [max_batch,
+ * n_kv_heads, *scale_capacity], *scale_capacity = cap rounded up to 64 (entries at and beyond cap are never
+ * used).  *buffer_bytes = the size to allocate for each of k_cache and v_cache (16-byte aligned base).
+ * Slots at and beyond ctx_len[b] are never read, whatever they hold.  Host only; no device work. */
+PRESERVE_API int preserve_kv8_layout(const preserve_layer_config_t *cfg, uint64_t *scale_offset_bytes,
+                                     int32_t *scale_capacity, uint64_t *buffer_bytes);
 
 /* Upper limit, in bytes, on what one window's prefetch may bring into L2
  * (Algorithm 1's C; Section 3 "L2 capacity requirements").

@@ -20,6 +20,7 @@ STATIC_SCRATCH_BYTES = 8 << 20
 PLAN_WHOLE_NODE, PLAN_TRUNCATE = 0, 1
 FLAG_NO_GRAPH, FLAG_PERSIST_L2, FLAG_NO_EARLY_LAUNCH, FLAG_FORCE_GEMV, FLAG_FORCE_TENSOR = 1, 2, 4, 8, 16
 FLAG_INT8_WEIGHTS = 32
+FLAG_INT8_KV = 64
 DEBUG_WITHHOLD, DEBUG_WAIT_LIMIT_CYCLES = 0, 1
 WITHHOLD_WINDOW, WITHHOLD_GEMV, WITHHOLD_TENSOR, WITHHOLD_ATTENTION = 1, 2, 3, 4
 
@@ -35,7 +36,7 @@ EXPORTS = (
     "preserve_last_status_code", "preserve_comm_create", "preserve_comm_export", "preserve_comm_import",
     "preserve_comm_set_peer", "preserve_comm_write", "preserve_comm_debug_arrive", "preserve_comm_epoch",
     "preserve_comm_destroy", "preserve_layer_set_comm", "preserve_layer_set_external_attention_sum",
-    "preserve_prefetch_window", "preserve_measure_stream_tma",
+    "preserve_prefetch_window", "preserve_measure_stream_tma", "preserve_kv8_layout",
 )
 NODE_COMM, NODE_MATMUL, NODE_ATTENTION, NODE_OTHER = 0, 1, 2, 3
 TRACE_SLOTS = 8
@@ -115,6 +116,8 @@ def lib() -> C.CDLL:
         L.preserve_measure_stream.argtypes = [C.c_void_p, C.c_size_t, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                               C.c_uint32, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(C.c_float)]
         L.preserve_last_status_code.argtypes = [C.c_void_p]
+        L.preserve_kv8_layout.argtypes = [C.POINTER(LayerConfig), C.POINTER(C.c_uint64), C.POINTER(C.c_int32),
+                                          C.POINTER(C.c_uint64)]
         L.preserve_comm_create.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_void_p)]
         L.preserve_comm_export.argtypes = [C.c_void_p, C.c_void_p]
         L.preserve_comm_import.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
@@ -198,6 +201,13 @@ def make_config(shape, max_batch: Optional[int] = None, max_ctx: Optional[int] =
     return LayerConfig(shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn,
                        shape.tp_degree, shape.batch if max_batch is None else max_batch,
                        shape.ctx if max_ctx is None else max_ctx, shape.rms_eps, shape.rope_theta, flags)
+
+
+def preserve_kv8_layout(cfg: LayerConfig):
+    """(scale_offset_bytes, scale_capacity, buffer_bytes) of one int8 cache buffer for `cfg`."""
+    off, cap, tot = C.c_uint64(), C.c_int32(), C.c_uint64()
+    _check(lib().preserve_kv8_layout(C.byref(cfg), C.byref(off), C.byref(cap), C.byref(tot)), "preserve_kv8_layout")
+    return int(off.value), int(cap.value), int(tot.value)
 
 
 def preserve_algorithmic_bytes(cfg: LayerConfig, batch: int, sum_ctx: int) -> int:

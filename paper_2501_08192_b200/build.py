@@ -9,7 +9,7 @@ from concurrent.futures import ThreadPoolExecutor
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libpreserve.so")
-SOURCES = ["api.cu", "window.cu", "gemv.cu", "gemm_tc.cu", "attn.cu", "prefetch.cu", "pack.cu", "stage.cu", "microbench.cu", "planner.cu", "comm.cu"]
+SOURCES = ["api.cu", "window.cu", "gemv.cu", "gemm_tc.cu", "attn.cu", "attn_kv8.cu", "prefetch.cu", "pack.cu", "stage.cu", "microbench.cu", "planner.cu", "comm.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

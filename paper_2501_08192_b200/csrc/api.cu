@@ -53,6 +53,21 @@ bool make_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 2-D uint8 tensor map: `rows` rows of `cols` contiguous bytes, box (box_cols x box_rows), 128-byte swizzle.
+bool make_u8_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_cols, uint32_t box_rows)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn)
+        return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // A replayable graph and everything its kernel nodes were captured with: a cached graph is
 // reused only when the whole signature matches word for word (no bare hash).
 struct GraphEntry {
@@ -69,6 +84,11 @@ bool encode_bf16_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_
                         uint32_t box_rows)
 {
     return make_map_2d(m, base, cols, rows, box_cols, box_rows);
+}
+bool encode_u8_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_cols,
+                      uint32_t box_rows)
+{
+    return make_u8_map_2d(m, base, cols, rows, box_cols, box_rows);
 }
 }  // namespace prsv
 
@@ -87,6 +107,11 @@ struct preserve_layer {
     bool w8;                     // int8 weights (GEMV path): arena holds codes, `scales` one fp32 per packed row
     float *scales;
     size_t soff[4];
+    bool kv8;                    // int8 KV-cache: codes then scales in each cache buffer (preserve_kv8_layout)
+    float *kv_new;               // kv8: the step's new key and value, fp32 [2][max_batch * n_kv][d] (QKV projection ->
+                                 // attention, which quantises them into the cache)
+    uint64_t kv8_scale_off;      // byte offset of the scales inside a cache buffer
+    int kv8_scale_cap;           // scales per (sequence, kv head): capacity rounded up to 64
 
     float *h_f32;                              // window A sum (residual for window B)
     float *attn_f32, *h2_f32, *mlp_f32;        // unrounded copies: own attention partial (window B input),
@@ -189,7 +214,25 @@ int validate_config(const preserve_layer_config_t *c)
         if (!gemv || (c->flags & PRESERVE_FLAG_FORCE_TENSOR) || c->ffn % 64)
             return PRESERVE_ESHAPE;
     }
+    if (c->flags & PRESERVE_FLAG_INT8_KV) {
+        // the int8-cache attention kernel takes groups of at most 8 query heads per KV head
+        if (c->n_q_heads / c->n_kv_heads > 8)
+            return PRESERVE_ESHAPE;
+    }
     return PRESERVE_OK;
+}
+
+// Layout of one int8 cache buffer: codes [max_batch, n_kv, cap, d] int8, then (256-byte aligned) one
+// fp32 scale per cached vector [max_batch, n_kv, scale_cap], scale_cap = cap rounded up to 64.
+void kv8_layout(const preserve_layer_config_t &c, uint64_t *scale_off, int *scale_cap, uint64_t *total)
+{
+    const uint64_t streams = (uint64_t)c.max_batch * c.n_kv_heads, cap = (uint64_t)c.max_ctx + 1;
+    const uint64_t codes = streams * cap * (uint64_t)c.head_dim;
+    const uint64_t off = (codes + 255) & ~uint64_t(255);
+    const uint64_t scap = (cap + 63) & ~uint64_t(63);
+    *scale_off = off;
+    *scale_cap = (int)scap;
+    *total = off + streams * scap * 4;
 }
 
 struct Dims {
@@ -214,12 +257,17 @@ uint64_t weight_bytes(const preserve_layer_config_t &c, const Dims &d, int i)
 
 uint64_t activation_bytes(const preserve_layer_config_t &c, int B)
 {
+    const bool kv8 = (c.flags & PRESERVE_FLAG_INT8_KV) != 0;
     const uint64_t BH = (uint64_t)B * c.hidden * 2, Bq = (uint64_t)B * c.n_q_heads * c.head_dim * 2;
     const uint64_t Bkv = (uint64_t)B * c.n_kv_heads * c.head_dim * 2, BF = (uint64_t)B * c.ffn * 2;
     const uint64_t gain = (uint64_t)c.hidden * 2, P = c.tp_degree;
     uint64_t t = 0;
     t += (P + 1) * BH + gain + 2 * BH;   // window A: reads, gain, writes h and x
-    t += BH + Bq + 2 * Bkv;              // QKV: reads x, writes q, appends k and v
+    t += BH + Bq;                        // QKV: reads x, writes q ...
+    if (!kv8)
+        t += 2 * Bkv;                    // ... and appends k and v
+    else                                 // ... leaves k and v as fp32 (write, read), attention stores codes and scales
+        t += 2 * (2 * Bkv + 2 * Bkv) + Bkv + 2 * (uint64_t)B * c.n_kv_heads * 4;
     t += Bq + Bq;                        // attention: reads q, writes o
     t += Bq + BH;                        // O: reads o, writes the attention partial
     t += (P + 1) * BH + gain + 2 * BH;   // window B
@@ -395,7 +443,9 @@ void plan_step(preserve_layer *L, const StepPtrs &sp, StepPlan *pl)
         const uint64_t nt = (uint64_t)(sp.ctx_len_host[b] + 1 + 63) / 64;
         max_tiles_seq = nt > max_tiles_seq ? nt : max_tiles_seq;
     }
-    pl->kv_bytes = 2 * sum_ctx * c.n_kv_heads * c.head_dim * 2;
+    // K and V bytes of the cached tokens: the SelfAttention node's memSize for Algorithm 1 (an int8
+    // cache: the codes; its scales, 4 bytes per 128, are read too but not prefetched)
+    pl->kv_bytes = 2 * sum_ctx * c.n_kv_heads * c.head_dim * (L->kv8 ? 1 : 2);
     // The layer's operator chain as Algorithm 1 sees it: window A -> Wqkv -> (rotary, append) ->
     // SelfAttention -> Wo -> window B -> Wgate|up -> (activation) -> Wdown -> next window.
     {
@@ -414,13 +464,16 @@ void plan_step(preserve_layer *L, const StepPtrs &sp, StepPlan *pl)
             pl->planned[h.comm == 0 ? 0 : 1][slot_of_node[h.node]] = h.bytes;
     }
     pl->alg_bytes = L->wbytes[0] + L->wbytes[1] + L->wbytes[2] + L->wbytes[3] + pl->kv_bytes + activation_bytes(c, B);
+    if (L->kv8)
+        pl->alg_bytes += 2 * sum_ctx * c.n_kv_heads * 4;
     // budget 0 = vanilla execution: every kernel starts after its predecessor has completed and
     // nothing is fetched ahead of the dependency
     pl->pdl = (L->budget > 0 && !L->no_early) ? 1 : 0;
     // (only == -1: the whole step; -2 / -3: just the prefetch beside window A / B; k >= 0: just kernel k)
     pl->pf_a = (L->only == -1 || L->only == -2) && pl->planned[0][0] + pl->planned[0][1] + pl->planned[0][2] > 0;
     pl->pf_b = (L->only == -1 || L->only == -3) && pl->planned[1][0] + pl->planned[1][1] > 0;
-    plan_attention(sp.ctx_len_host, B, c.n_kv_heads, L->sm_count, &pl->attn_grid, &pl->attn_tpi);
+    plan_attention(sp.ctx_len_host, B, c.n_kv_heads, L->sm_count, &pl->attn_grid, &pl->attn_tpi,
+                   L->kv8 ? attention_kv8_stages() : 3);
     pl->attn_items_per_stream = (int)((max_tiles_seq + pl->attn_tpi - 1) / pl->attn_tpi);
     // (the merge kernel sizes its CTAs from this, between 4 and 32 warps: clamp here so that the
     // number that enters the graph signature changes as rarely as the launch does)
@@ -447,8 +500,11 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
     // ---- K/V tensor maps
     if (sp.k_cache != L->k_ptr || sp.v_cache != L->v_ptr) {
         const uint64_t rows = (uint64_t)c.max_batch * c.n_kv_heads * cap;
-        if (!make_map_2d(&L->k_map, sp.k_cache, kHeadDim, rows, 64, 64) ||
-            !make_map_2d(&L->v_map, sp.v_cache, kHeadDim, rows, 64, 64))
+        const bool ok = L->kv8 ? make_u8_map_2d(&L->k_map, sp.k_cache, kHeadDim, rows, 128, 64) &&
+                                     make_u8_map_2d(&L->v_map, sp.v_cache, kHeadDim, rows, 128, 64)
+                               : make_map_2d(&L->k_map, sp.k_cache, kHeadDim, rows, 64, 64) &&
+                                     make_map_2d(&L->v_map, sp.v_cache, kHeadDim, rows, 64, 64);
+        if (!ok)
             return PRESERVE_EARCH;
         L->k_ptr = sp.k_cache;
         L->v_ptr = sp.v_cache;
@@ -505,8 +561,8 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
         pa.kv_node = 1;
         pa.kv_count = B * c.n_kv_heads;
         pa.kv_ranges_per_seq = c.n_kv_heads;
-        pa.kv_token_bytes = kHeadDim * 2;
-        pa.kv_stride = (uint64_t)cap * kHeadDim * 2;
+        pa.kv_token_bytes = kHeadDim * (L->kv8 ? 1 : 2);
+        pa.kv_stride = (uint64_t)cap * kHeadDim * (L->kv8 ? 1 : 2);
         // Wqkv and Wo are adjacent in the arena
         const int na = persist_window(L->off[0], L->wbytes[0] + L->wbytes[1]);
         CK(L, launch_prefetch(pa, L->prefetch_ctas, L->side, na ? pf_attr : nullptr, na));
@@ -569,6 +625,10 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
         e.ctx_len = sp.ctx_len;
         e.nq = c.n_q_heads; e.nkv = c.n_kv_heads; e.cap = cap;
         e.inv_freq = c.rope_theta > 0.f ? L->inv_freq : nullptr;
+        if (L->kv8) {
+            e.kv_new = L->kv_new;
+            e.kv_new_plane = (size_t)c.max_batch * c.n_kv_heads * kHeadDim;
+        }
         int rc = launch_gemm(L, 0, L->x, B, e, pdl, s, TRACE(1));
         if (rc)
             return rc;
@@ -597,6 +657,16 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
         a.trace = TRACE(2);
         a.pdl = pdl;
         a.inject = L->inject == INJECT_ATTN_RING ? INJECT_ATTN_RING : INJECT_NONE;
+        if (L->kv8) {
+            a.kv8 = 1;
+            a.k_codes = sp.k_cache;
+            a.v_codes = sp.v_cache;
+            a.k_scale = reinterpret_cast<float *>(static_cast<uint8_t *>(sp.k_cache) + L->kv8_scale_off);
+            a.v_scale = reinterpret_cast<float *>(static_cast<uint8_t *>(sp.v_cache) + L->kv8_scale_off);
+            a.scale_cap = L->kv8_scale_cap;
+            a.kv_new = L->kv_new;
+            a.kv_new_plane = (size_t)c.max_batch * c.n_kv_heads * kHeadDim;
+        }
         CK(L, launch_attention(a, s));
     }
     // ---- output projection -> this shard's attention partial sum
@@ -882,8 +952,24 @@ uint64_t preserve_algorithmic_bytes(const preserve_layer_config_t *cfg, int32_t 
     uint64_t w = 0;
     for (int i = 0; i < 4; ++i)
         w += weight_bytes(*cfg, d, i);
-    const uint64_t kv = 2 * sum_ctx * cfg->n_kv_heads * cfg->head_dim * 2;
+    const bool kv8 = (cfg->flags & PRESERVE_FLAG_INT8_KV) != 0;
+    const uint64_t kv = kv8 ? 2 * sum_ctx * cfg->n_kv_heads * ((uint64_t)cfg->head_dim + 4)
+                            : 2 * sum_ctx * cfg->n_kv_heads * cfg->head_dim * 2;
     return w + kv + activation_bytes(*cfg, batch);
+}
+
+int preserve_kv8_layout(const preserve_layer_config_t *cfg, uint64_t *scale_offset_bytes, int32_t *scale_capacity,
+                        uint64_t *buffer_bytes)
+{
+    if (!cfg || !scale_offset_bytes || !scale_capacity || !buffer_bytes)
+        return PRESERVE_EINVAL;
+    int rc = validate_config(cfg);
+    if (rc != PRESERVE_OK)
+        return rc;
+    int scap = 0;
+    kv8_layout(*cfg, scale_offset_bytes, &scap, buffer_bytes);
+    *scale_capacity = scap;
+    return PRESERVE_OK;
 }
 
 void preserve_layer_destroy(preserve_layer_t *L)
@@ -894,7 +980,7 @@ void preserve_layer_destroy(preserve_layer_t *L)
     if (L->side)
         cudaStreamSynchronize(L->side);
     drop_graphs(L);
-    void *ptrs[] = {L->scales, L->trace_buf, L->attn_f32, L->h2_f32, L->mlp_f32, L->arena, L->inv_freq, L->h_f32, L->x, L->q, L->o, L->x2, L->a,
+    void *ptrs[] = {L->kv_new, L->scales, L->trace_buf, L->attn_f32, L->h2_f32, L->mlp_f32, L->arena, L->inv_freq, L->h_f32, L->x, L->q, L->o, L->x2, L->a,
                     L->part_o, L->part_ml, L->status, L->stage_in, L->stage_out, L->ctx_dev};
     for (void *p : ptrs)
         if (p)
@@ -1059,6 +1145,13 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
     L->max_items = L->sm_count * 8 + B * c.n_kv_heads + 8;
     CKI(cudaMalloc(&L->part_o, (size_t)L->max_items * L->group * kHeadDim * 4));
     CKI(cudaMalloc(&L->part_ml, (size_t)L->max_items * L->group * 2 * 4));
+    L->kv8 = (c.flags & PRESERVE_FLAG_INT8_KV) != 0;
+    if (L->kv8) {
+        uint64_t total = 0;
+        kv8_layout(c, &L->kv8_scale_off, &L->kv8_scale_cap, &total);
+        CKI(cudaMalloc(&L->kv_new, (size_t)2 * B * c.n_kv_heads * kHeadDim * sizeof(float)));
+        CKI(cudaMemset(L->kv_new, 0, (size_t)2 * B * c.n_kv_heads * kHeadDim * sizeof(float)));
+    }
     CKI(cudaMalloc(&L->status, 256));
     CKI(cudaMemset(L->status, 0, 256));
     const size_t n_in = (size_t)(2 * c.tp_degree) * BH * 2;

@@ -24,18 +24,15 @@
 #include <cstdlib>
 
 #include "../../include/preserve.h"
+#include "attn_common.cuh"
 #include "common.cuh"
 #include "kernels.h"
 
 namespace prsv {
 
-constexpr int kTileKeys = 64;
 constexpr int kStages = 3;                            // 96 KiB ring: two CTAs per SM
-constexpr int kConsumerWarps = 4;
-constexpr int kAttnThreads = (kConsumerWarps + 1) * 32;
 constexpr int kHalfBytes = kTileKeys * 128;            // one 64x64 bf16 box
 constexpr int kStageBytes = 4 * kHalfBytes;            // K lo, K hi, V lo, V hi
-constexpr int kMaxStreams = 2048;                      // (sequence, kv head) pairs per launch
 
 struct AttnParams {
     CUtensorMap k_map;
@@ -64,11 +61,6 @@ struct AttnSmem {
     int item_base[kMaxStreams + 1];      // last: the launch only asks for the entries it needs
 };
 
-__device__ __forceinline__ void consumer_barrier()
-{
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
-}
-
 // Where consumer warp w keeps row r (a query head of the group) of its O partial inside a ring
 // stage: in the 16 key rows of each 64x64 box that only this warp reads, so no other warp can
 // still be reading the bytes it overwrites.  512 B per row, four rows per box slice.
@@ -79,48 +71,6 @@ __device__ __forceinline__ float *comb_row(uint8_t *stage, int w, int r)
 // float2 slot of head dims (2c, 2c + 1) within a row: XOR swizzle so that the fragment stores
 // (eight rows x four column pairs per instruction) and the row reads are both conflict-free
 __device__ __forceinline__ int comb_col2(int r, int c) { return c ^ ((r & 3) << 2); }
-
-__device__ __forceinline__ int tiles_of(int ctx) { return (ctx + 1 + kTileKeys - 1) / kTileKeys; }
-
-// First item index of every stream, computed identically by every CTA: the lengths are
-// fetched by all threads at once (one memory round trip), then warp 0 scans them.
-__device__ __forceinline__ void build_item_table(const AttnParams &p, int *item_base)
-{
-    const int streams = p.B * p.nkv;
-    for (int i = threadIdx.x; i < streams; i += blockDim.x) {
-        const int nt = tiles_of(p.ctx_len[i / p.nkv]);
-        item_base[i + 1] = (nt + p.tiles_per_item - 1) / p.tiles_per_item;
-    }
-    __syncthreads();
-    if (threadIdx.x < 32) {
-        int carry = 0;
-        for (int base = 0; base < streams; base += 32) {
-            const int i = base + threadIdx.x;
-            int v = i < streams ? item_base[i + 1] : 0;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int n = __shfl_up_sync(0xffffffffu, v, o);
-                if ((int)threadIdx.x >= o)
-                    v += n;
-            }
-            if (i < streams)
-                item_base[i + 1] = carry + v;
-            carry += __shfl_sync(0xffffffffu, v, 31);
-        }
-        if (threadIdx.x == 0)
-            item_base[0] = 0;
-    }
-}
-
-__device__ __forceinline__ int find_stream(const int *item_base, int streams, int item)
-{
-    int lo = 0, hi = streams;     // item_base[lo] <= item < item_base[hi]
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (item_base[mid] <= item) lo = mid; else hi = mid;
-    }
-    return lo;
-}
 
 // NARROW: groups of up to 8 query heads (keys as MMA rows in the QK product), else up to 16.
 template <bool NARROW>
@@ -583,7 +533,8 @@ static size_t attn_smem_bytes(int streams)
     return offsetof(AttnSmem, item_base) + sizeof(int) * (size_t)(streams + 1) + 1024;
 }
 
-void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_count, int *grid, int *tiles_per_item)
+void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_count, int *grid, int *tiles_per_item,
+                    int stages)
 {
     uint64_t total_tiles = 0;
     int longest = 1;
@@ -595,7 +546,7 @@ void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_coun
     // A short cache fits the CTAs' rings whole: items of at most kStages tiles, one per CTA, are then
     // all in shared memory before the queries exist, and what remains after the wait is arithmetic.
     // The shortest such items that leave a (sequence, head) at most one partial per merge warp.
-    for (int tpi = 1; tpi <= kStages; ++tpi) {
+    for (int tpi = 1; tpi <= stages; ++tpi) {
         uint64_t items = 0;
         int per_stream = 0;
         for (int b = 0; b < batch; ++b) {
@@ -614,7 +565,7 @@ void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_coun
     // most of the CTA's share before the queries exist, and half of every SM's shared memory stays
     // free for the kernels before and after.  Longer caches are a steady stream: two CTAs per SM
     // keep twice the bytes in flight.
-    const int g = total_tiles <= (uint64_t)2 * kStages * sm_count ? sm_count : 2 * sm_count;
+    const int g = total_tiles <= (uint64_t)2 * stages * sm_count ? sm_count : 2 * sm_count;
     // Work items = runs of `tpi` 64-key tiles of one sequence, dealt to the CTAs round-robin.  The
     // kernel lasts about rounds x (tpi + the per-item cost of combining and writing a partial,
     // worth ~1.5 tiles), rounds = items / CTAs rounded up: take the tpi that minimises that, between
@@ -664,7 +615,7 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     p.inject = a.inject;
 
     const size_t smem = attn_smem_bytes(a.B * a.nkv);
-    {
+    if (!a.kv8) {
         static PerDeviceSize lim_narrow, lim_wide;      // per device: the attribute belongs to one device
         cudaError_t e = ensure_dynamic_smem(k_attn_decode_splitkv<true>, lim_narrow, attn_smem_bytes(kMaxStreams));
         if (e == cudaSuccess)
@@ -682,7 +633,9 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     cfg.numAttrs = pdl_attr(at, a.pdl);
     const int phases = a.phases ? a.phases : 3;
     cudaError_t e = cudaSuccess;
-    if (phases & 1)
+    if ((phases & 1) && a.kv8)
+        e = launch_attention_kv8_kernel(a, cfg);
+    else if (phases & 1)
         e = p.G <= 8 ? cudaLaunchKernelEx(&cfg, k_attn_decode_splitkv<true>, p)
                      : cudaLaunchKernelEx(&cfg, k_attn_decode_splitkv<false>, p);
     if (e != cudaSuccess)

@@ -118,6 +118,13 @@ __device__ __forceinline__ void epilogue_qkv(const EpilogueArgs &e, int pos, int
     } else {
         const bool is_k = hd < e.nq + e.nkv;
         const int kvh = is_k ? hd - e.nq : hd - e.nq - e.nkv;
+        if (e.kv_new) {
+            // int8 cache: the vector goes to the attention kernel unrounded, which quantises it
+            float *dst = e.kv_new + (is_k ? 0 : e.kv_new_plane) + ((size_t)b * e.nkv + kvh) * kHeadDim + i;
+            dst[0] = v0;
+            dst[kHeadDim / 2] = v1;
+            return;
+        }
         const size_t o = (((size_t)b * e.nkv + kvh) * e.cap + pos) * kHeadDim + i;
         void *dst = is_k ? e.k_cache : e.v_cache;
         store_bf16(dst, o, v0);
@@ -229,6 +236,12 @@ __device__ __forceinline__ void apply_epilogue_quad_t(const EpilogueArgs &e, con
         } else {
             const bool is_k = hd < e.nq + e.nkv;
             const int kvh = is_k ? hd - e.nq : hd - e.nq - e.nkv;
+            if (e.kv_new) {
+                float *dst = e.kv_new + (is_k ? 0 : e.kv_new_plane) + ((size_t)b * e.nkv + kvh) * kHeadDim + i;
+                *reinterpret_cast<float2 *>(dst) = make_float2(a0, c0);
+                *reinterpret_cast<float2 *>(dst + kHeadDim / 2) = make_float2(a1, c1);
+                return;
+            }
             const size_t o = (((size_t)b * e.nkv + kvh) * e.cap + pos) * kHeadDim + i;
             bf16 *dst = reinterpret_cast<bf16 *>(is_k ? e.k_cache : e.v_cache);
             *reinterpret_cast<uint32_t *>(dst + o) = pack_bf16(a0, c0);

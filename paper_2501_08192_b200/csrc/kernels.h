@@ -121,6 +121,8 @@ struct EpilogueArgs {
     const int *ctx_len;   // device [B]
     int nq, nkv, cap;
     const double *inv_freq;  // device [d/2]: theta^(-2i/d); NULL disables the rotary embedding
+    float *kv_new;        // int8 cache: the new k and v go here as fp32 ([2][max_batch*nkv][d], planes kv_new_plane
+    size_t kv_new_plane;  // elements apart) instead of into k_cache / v_cache; NULL: bf16 cache
 };
 
 // Packing kinds: how logical output features map to packed rows.
@@ -196,11 +198,29 @@ struct AttnArgs {
     long long *trace;      // optional: two consecutive timeline slots (split-KV, merge)
     int pdl;
     int inject;
+    // int8 cache (kv8 != 0): k_map / v_map are uint8 maps with dims (d, max_batch*nkv*cap), box (128, 64);
+    // one fp32 scale per cached vector in k_scale / v_scale [max_batch*nkv][scale_cap] (scale_cap a
+    // multiple of 64); the step's new key and value arrive as fp32 vectors in kv_new ([2][max_batch*nkv][d],
+    // written by the QKV projection) and the kernel stores their codes and scales into the cache.
+    int kv8;
+    float *k_scale, *v_scale;
+    void *k_codes, *v_codes;
+    int scale_cap;
+    const float *kv_new;
+    size_t kv_new_plane;
 };
 cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s);
+// the int8-cache split-KV kernel alone (attn_kv8.cu); launch_attention adds the merge kernel
+cudaError_t launch_attention_kv8_kernel(const AttnArgs &a, const cudaLaunchConfig_t &base_cfg);
+int attention_kv8_stages();
 // Grid size (persistent CTAs) and tiles per work item for the given sequence lengths (host array);
 // depends only on the lengths and the SM count.
-void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_count, int *grid, int *tiles_per_item);
+// `stages` = tiles the kernel's ring holds (3 for the bf16 cache, attention_kv8_stages() for int8).
+void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_count, int *grid, int *tiles_per_item,
+                    int stages = 3);
+// 2-D uint8 tensor map (rows x cols bytes, cols contiguous), box (box_cols x box_rows), 128-byte swizzle.
+bool encode_u8_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_cols,
+                      uint32_t box_rows);
 
 // 2-D bf16 tensor map (rows x cols, cols contiguous), box (box_cols x box_rows), 128-byte swizzle.
 bool encode_bf16_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_cols,

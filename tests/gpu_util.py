@@ -45,13 +45,38 @@ class GuardedOut:
         return bool((r[:GUARD] == CANARY).all() and (r[GUARD + self.n:] == CANARY).all())
 
 
+def kv8_buffer(cfg, codes: np.ndarray, scales: np.ndarray) -> torch.Tensor:
+    """One int8 cache buffer on the device in the library's layout: the codes, then the scales."""
+    off, scap, total = P.preserve_kv8_layout(cfg)
+    B, nkv, cap, d = codes.shape
+    buf = torch.zeros(total, dtype=torch.uint8, device="cuda")
+    buf[:codes.size] = torch.from_numpy(np.ascontiguousarray(codes).view(np.uint8).reshape(-1)).cuda()
+    padded = np.full((B, nkv, scap), np.nan, np.float32)
+    padded[:, :, :cap] = scales
+    buf[off:off + padded.size * 4] = torch.from_numpy(padded.view(np.uint8).reshape(-1)).cuda()
+    return buf
+
+
+def kv8_read(cfg, buf: torch.Tensor, B: int, nkv: int, cap: int, d: int):
+    """(codes int8 [B,nkv,cap,d], scales f32 [B,nkv,cap]) back from a device cache buffer."""
+    off, scap, _ = P.preserve_kv8_layout(cfg)
+    raw = buf.cpu().numpy()
+    codes = raw[:B * nkv * cap * d].view(np.int8).reshape(B, nkv, cap, d)
+    scales = raw[off:off + B * nkv * scap * 4].view(np.float32).reshape(B, nkv, scap)[:, :, :cap]
+    return codes.copy(), scales.copy()
+
+
 class DeviceLayer:
-    """One layer instance on the device: library handle, inputs, outputs."""
+    """One layer instance on the device: library handle, inputs, outputs.  kv8 = the int8 cache of
+    inputs.make_int8_cache: the layer is then created with FLAG_INT8_KV and runs over that cache."""
 
     def __init__(self, shape: I.ShardShape, t: Dict[str, np.ndarray], flags: int = 0,
-                 max_batch: Optional[int] = None):
+                 max_batch: Optional[int] = None, kv8: Optional[Dict[str, np.ndarray]] = None):
         self.shape = shape
         self.t = t
+        self.kv8 = kv8
+        if kv8 is not None:
+            flags |= P.FLAG_INT8_KV
         self.cfg = P.make_config(shape, max_batch=max_batch, flags=flags)
         names = ("w_q", "w_k", "w_v", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")
         w = {n: bits_to_cuda(t[n]) for n in names}
@@ -61,8 +86,13 @@ class DeviceLayer:
         self.partials = [bits_to_cuda(t["partials_in"][p]) for p in range(shape.tp_degree)]
         self.peers = [bits_to_cuda(t["attn_peer_partials"][p]) for p in range(shape.tp_degree - 1)]
         self.residual = bits_to_cuda(t["residual_in"])
-        self.k_cache = bits_to_cuda(t["k_cache"])
-        self.v_cache = bits_to_cuda(t["v_cache"])
+        if kv8 is None:
+            self.k_cache = bits_to_cuda(t["k_cache"])
+            self.v_cache = bits_to_cuda(t["v_cache"])
+        else:
+            assert max_batch is None or max_batch == shape.batch
+            self.k_cache = kv8_buffer(self.cfg, kv8["k_codes"], kv8["k_scales"])
+            self.v_cache = kv8_buffer(self.cfg, kv8["v_codes"], kv8["v_scales"])
         self.ctx_host = np.ascontiguousarray(t["ctx_len"], dtype=np.int32)
         self.ctx_dev = torch.from_numpy(self.ctx_host).cuda()
         self.residual_out = GuardedOut((B, H))
@@ -118,6 +148,18 @@ class DeviceLayer:
         k = np.stack([kc[b, :, idx[b]] for b in range(self.shape.batch)])
         v = np.stack([vc[b, :, idx[b]] for b in range(self.shape.batch)])
         return k, v
+
+    def appended_kv8(self):
+        """int8 cache: the slot written by the step, per sequence: (k codes [B,nkv,d], k scales [B,nkv],
+        v codes, v scales)."""
+        torch.cuda.synchronize()
+        s = self.shape
+        out = []
+        for buf in (self.k_cache, self.v_cache):
+            codes, scales = kv8_read(self.cfg, buf, s.batch, s.n_kv_heads, s.kv_capacity, s.head_dim)
+            out.append(np.stack([codes[b, :, self.ctx_host[b]] for b in range(s.batch)]))
+            out.append(np.stack([scales[b, :, self.ctx_host[b]] for b in range(s.batch)]))
+        return tuple(out)
 
     def close(self) -> None:
         self.layer.close()

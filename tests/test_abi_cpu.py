@@ -213,7 +213,7 @@ def test_no_process_wide_switches_in_the_kernels_sources():
     csrc = os.path.join(ROOT, "paper_2501_08192_b200", "csrc")
     allowed_static = ("static PerDeviceSize", "static __device__ __align__(256) unsigned char g_static_scratch",
                       "static const int", "static const int32_t", "static_assert", "static_cast", "static cudaError_t",
-                      "static int reset_trace", "static size_t attn_smem_bytes", "static EncodeTiledFn fn",
+                      "static int reset_trace", "static size_t attn_smem_bytes", "static size_t attn_kv8_smem_bytes", "static EncodeTiledFn fn",
                       "static bool tried", "static constexpr")
     for name in sorted(os.listdir(csrc)):
         text = open(os.path.join(csrc, name)).read()
