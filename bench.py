@@ -177,8 +177,24 @@ class Workload:
         w = {n: to_dev(t[n]) for n in ("w_q", "w_k", "w_v", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")}
         parts0 = [to_dev(t["partials_in"][p]) for p in range(shape.tp_degree)]
         peers0 = [to_dev(t["attn_peer_partials"][p]) for p in range(shape.tp_degree - 1)]
-        resid0, kc0, vc0 = to_dev(t["residual_in"]), to_dev(t["k_cache"]), to_dev(t["v_cache"])
         self.ctx_host = np.ascontiguousarray(t["ctx_len"], np.int32)
+        if flags & P.FLAG_INT8_KV:
+            # int8 cache: one device buffer per tensor in the library's layout (codes, then scales)
+            kv = I.make_int8_cache(shape, self.ctx_host)
+            off, scap, total = P.preserve_kv8_layout(cfg)
+
+            def kv8_buf(codes, scales):
+                buf = torch.zeros(total, dtype=torch.uint8, device="cuda")
+                buf[:codes.size] = torch.from_numpy(codes.view(np.uint8).reshape(-1)).cuda()
+                padded = np.zeros(scales.shape[:2] + (scap,), np.float32)
+                padded[:, :, :scales.shape[2]] = np.nan_to_num(scales)
+                buf[off:off + padded.size * 4] = torch.from_numpy(padded.view(np.uint8).reshape(-1)).cuda()
+                return buf
+            kc0, vc0 = kv8_buf(kv["k_codes"], kv["k_scales"]), kv8_buf(kv["v_codes"], kv["v_scales"])
+            del kv
+        else:
+            kc0, vc0 = to_dev(t["k_cache"]), to_dev(t["v_cache"])
+        resid0 = to_dev(t["residual_in"])
         self.sum_ctx = int(self.ctx_host.sum())
         hp = [pin(t["partials_in"][p]) for p in range(shape.tp_degree)]
         hq = [pin(t["attn_peer_partials"][p]) for p in range(shape.tp_degree - 1)]
@@ -219,9 +235,12 @@ class Workload:
 
 def bench_config(P, I, torch, dist, args, idx, rank, local_rank, world, stream, headline: bool):
     l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size
-    wl = Workload(P, I, torch, idx, rank, l2, args.rotation, keep_host=headline and rank == 0)
+    vflags = (P.FLAG_INT8_KV if args.int8_kv else 0) | (P.FLAG_INT8_WEIGHTS if args.int8_weights else 0)
+    wl = Workload(P, I, torch, idx, rank, l2, args.rotation, keep_host=headline and rank == 0, flags=vflags)
     shape, R, alg = wl.shape, wl.R, wl.alg
     layers, ios, hios = wl.layers, wl.ios, wl.hios
+    if vflags:      # (a profiling aid: the whole run at the int8 precisions; the byte count is the library's)
+        alg = int(P.preserve_algorithmic_bytes(wl.cfg, shape.batch, wl.sum_ctx))
     assert alg == int(P.preserve_algorithmic_bytes(wl.cfg, shape.batch, wl.sum_ctx)) > 0
     info = layers[0].get_info()
     default_budget = int(info.prefetch_budget) if args.budget_bytes < 0 else args.budget_bytes
@@ -407,35 +426,52 @@ def bench_config(P, I, torch, dist, args, idx, rank, local_rank, world, stream, 
         res["model"] = model
     except Exception as e:      # noqa: BLE001
         res["model"] = {"error": str(e)}
-    # ---- the same configuration with int8 weights (the weight precision of the paper's runs), where the
-    # library has them: the split-K GEMV path
-    if shape.batch < 16 and not args.no_sweep:
+    # ---- the same configuration at the precisions of the paper's runs (Section 4: int8 weights and
+    # KV-cache): int8 KV-cache on every configuration; int8 weights where the library has them (the
+    # split-K GEMV path).  Each row: vanilla and early-launch-only times, the attention kernel alone.
+    if not args.no_sweep:
         wl.close()
-        wl8 = Workload(P, I, torch, idx, rank, l2, args.rotation, flags=P.FLAG_INT8_WEIGHTS)
-        alg8 = int(P.preserve_algorithmic_bytes(wl8.cfg, shape.batch, wl8.sum_ctx))
+        variants = [("int8_kv", P.FLAG_INT8_KV)]
+        if shape.batch < 16:
+            variants += [("int8_weights", P.FLAG_INT8_WEIGHTS), ("int8_weights_and_kv", P.FLAG_INT8_WEIGHTS | P.FLAG_INT8_KV)]
+        for vname, vflags in variants:
+            wl8 = Workload(P, I, torch, idx, rank, l2, args.rotation, flags=vflags)
+            alg8 = int(P.preserve_algorithmic_bytes(wl8.cfg, shape.batch, wl8.sum_ctx))
 
-        def chain8():
-            P.preserve_decode_chain(wl8.layers, wl8.ios, link=False, stream=stream)
-        row = {"algorithmic_bytes_per_layer": alg8}
-        for name, b in (("off", 0), ("early_launch_only", 1)):
-            wl8.set_budget(b)
-            with torch.cuda.stream(stream):
-                for _ in range(3):
-                    chain8()
-            barrier()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            with torch.cuda.stream(stream):
-                e0.record(stream)
-                for _ in range(n_min):
-                    chain8()
-                e1.record(stream)
-            barrier()
-            ms8 = max_over_ranks(e0.elapsed_time(e1) / n_min, world)
-            row[name + "_us_per_layer"] = round(ms8 * 1e3 / wl8.R, 3)
-            row[name + "_gbs"] = round(alg8 * wl8.R / (ms8 * 1e-3) / 1e9, 1)
-        row["speedup_vs_bf16_weights"] = round(us(ms_early) / row["early_launch_only_us_per_layer"], 4)
-        res["int8_weights"] = row
-        wl8.close()
+            def chain8():
+                P.preserve_decode_chain(wl8.layers, wl8.ios, link=False, stream=stream)
+
+            def attn8():
+                for L, io in zip(wl8.layers, wl8.ios):
+                    L.run_kernel(io, 2, stream)
+            row = {"algorithmic_bytes_per_layer": alg8}
+            for name, b in (("off", 0), ("early_launch_only", 1)):
+                wl8.set_budget(b)
+                ms8, _ = time_steps(chain8, n_min, 3)
+                row[name + "_us_per_layer"] = round(ms8 * 1e3 / wl8.R, 3)
+                row[name + "_gbs"] = round(alg8 * wl8.R / (ms8 * 1e-3) / 1e9, 1)
+            row["speedup_vs_bf16"] = round(us(ms_early) / row["early_launch_only_us_per_layer"], 4)
+            if vflags & P.FLAG_INT8_KV:
+                with torch.cuda.stream(stream):
+                    attn8()
+                    torch.cuda.synchronize()
+                    g8 = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g8, stream=stream):
+                        for _ in range(4):
+                            attn8()
+                ms_a, _ = time_steps(lambda: g8.replay(), max(5, math.ceil(args.min_layer_steps / (4 * wl8.R))), 3)
+                ms_a /= 4 * wl8.R
+                del g8
+                kv_read = 2 * wl8.sum_ctx * shape.n_kv_heads * (shape.head_dim + 4)
+                qo = 2 * shape.batch * shape.n_q_heads * shape.head_dim * 4
+                row["attn_splitkv_us"] = round(ms_a * 1e3, 3)
+                row["attn_splitkv_gbs"] = round((kv_read + qo) / (ms_a * 1e-3) / 1e9, 1)
+                row["attn_splitkv_frac_of_measured"] = round(row["attn_splitkv_gbs"] / peak, 3)
+            row["device_status"] = max(L.last_status() for L in wl8.layers)
+            res[vname] = row
+            wl8.close()
+            del wl8
+            torch.cuda.empty_cache()
     if headline and rank == 0 and args.cpu_baseline and world == 1:
         res["cpu_baseline"] = cpu_baseline(shape, wl.host_tensors, alg, budget_s=12.0, idx=idx)
     wl.close()
@@ -584,7 +620,8 @@ def run_ours(args):
         "metric": METRIC, "value": round(whole_job_gbs(h["algorithmic_bytes_per_layer"], h["layers_per_step"],
                                                        h["ms_per_step"], world), 2),
         "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": h["ms_per_step"],
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 (fp32 accumulate)",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 (fp32 accumulate)" + (", int8 KV-cache" if args.int8_kv else "") + (", int8 weights" if args.int8_weights else ""),
         "data": "synthetic (seeded N(0,0.02) weights, N(0,1) activations and KV, shapes of the named config; the "
                 "layer instances of a rotation are distinct device buffers holding the same seeded draw)",
         "config": {"workload": h["workload"], "layers_per_step": h["layers_per_step"], "cold_l2": h["cold_l2"],
@@ -955,6 +992,9 @@ def main():
     ap.add_argument("--min-layer-steps", type=int, default=MIN_LAYER_STEPS,
                     help="timed layer-steps per setting (lower it only for profiler captures)")
     ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--int8-kv", action="store_true", help="run the main measurement over an int8 KV-cache (profiling aid)")
+    ap.add_argument("--int8-weights", action="store_true",
+                    help="run the main measurement with int8 weights (batch < 16 configurations; profiling aid)")
     ap.add_argument("--no-kernels", action="store_true", help="skip the isolated per-kernel timing")
     ap.add_argument("--budget-bytes", type=int, default=-1, help="prefetch budget per window (default: the library's)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")

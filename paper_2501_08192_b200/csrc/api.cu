@@ -473,7 +473,7 @@ void plan_step(preserve_layer *L, const StepPtrs &sp, StepPlan *pl)
     pl->pf_a = (L->only == -1 || L->only == -2) && pl->planned[0][0] + pl->planned[0][1] + pl->planned[0][2] > 0;
     pl->pf_b = (L->only == -1 || L->only == -3) && pl->planned[1][0] + pl->planned[1][1] > 0;
     plan_attention(sp.ctx_len_host, B, c.n_kv_heads, L->sm_count, &pl->attn_grid, &pl->attn_tpi,
-                   L->kv8 ? attention_kv8_stages() : 3);
+                   L->kv8 ? attention_kv8_stages() : 3, L->kv8 ? 3.0 : 1.5);
     pl->attn_items_per_stream = (int)((max_tiles_seq + pl->attn_tpi - 1) / pl->attn_tpi);
     // (the merge kernel sizes its CTAs from this, between 4 and 32 warps: clamp here so that the
     // number that enters the graph signature changes as rarely as the launch does)

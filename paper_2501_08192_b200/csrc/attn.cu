@@ -534,7 +534,7 @@ static size_t attn_smem_bytes(int streams)
 }
 
 void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_count, int *grid, int *tiles_per_item,
-                    int stages)
+                    int stages, double item_cost)
 {
     uint64_t total_tiles = 0;
     int longest = 1;
@@ -582,7 +582,7 @@ void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_coun
             items += (uint64_t)nkv * ((nt + tpi - 1) / tpi);
         }
         const uint64_t rounds = (items + g - 1) / g;
-        const double cost = (double)rounds * (tpi + 1.5);
+        const double cost = (double)rounds * (tpi + item_cost);
         if (best_cost < 0 || cost < best_cost) {
             best_cost = cost;
             best = tpi;

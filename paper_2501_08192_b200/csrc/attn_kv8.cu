@@ -7,9 +7,13 @@
 // merge kernel), with these differences:
 //   - a tile of 64 keys is ONE TMA box of 64 x 128 bytes per tensor plus the tile's 64 + 64
 //     scales (two 256-byte bulk copies): 16.5 KiB per stage instead of 32 KiB, four stages;
-//   - the codes are widened to fp16 in registers (exactly: the byte is placed in the mantissa
-//     of 1024.0 and 1152 is subtracted) and the products run on fp16 mma.sync; q is split into
-//     two fp16 planes, the softmax weights are one fp16 plane;
+//   - the codes are widened to fp16 in registers with one byte permute per pair: the byte with its
+//     top bit flipped (code + 128) lands in the mantissa of 1024.0, which is the number
+//     1152 + code exactly.  The products run on fp16 mma.sync with that offset left in: it adds
+//     1152 * (sum of the other operand) to every result, a number the kernel also has (the sum
+//     of q over the head dims, once per item; the sum of the weights over the keys, from one
+//     extra MMA per tile against a row of ones) and subtracts at the end.  q and the softmax
+//     weights are one fp16 plane each (11 significant bits);
 //   - the key scale multiplies the score after the dot product; the value scale multiplies the
 //     softmax weight before the P V product, normalised by a running power of two (the largest
 //     value scale seen so far) so that the fp16 weights never leave [0, 2);
@@ -84,16 +88,21 @@ __device__ __forceinline__ void mma_f16_16816(float (&d)[4], uint32_t a0, uint32
 }
 
 // Two int8 codes of `biased` (= the loaded word with every byte's top bit flipped, i.e. code + 128 as
-// an unsigned byte) widened to an fp16 pair.  SEL picks the bytes: 0x4140 = bytes (0, 1), 0x4342 =
-// (2, 3), 0x4240 = (0, 2), 0x4341 = (1, 3).  The byte lands in the low mantissa bits of 1024.0
-// (0x6400), which makes 1024 + byte exactly; subtracting 1152 leaves the signed code.
+// an unsigned byte) as an fp16 pair holding 1152 + code each.  SEL picks the bytes: 0x4140 = bytes
+// (0, 1), 0x4342 = (2, 3), 0x4240 = (0, 2), 0x4341 = (1, 3).  The byte lands in the low mantissa
+// bits of 1024.0 (0x6400), which is 1024 + byte = 1152 + code exactly.
+constexpr float kCodeOffset = 1152.f;
 template <uint32_t SEL>
-__device__ __forceinline__ uint32_t s8x2_to_f16x2(uint32_t biased)
+__device__ __forceinline__ uint32_t s8x2_to_f16x2_offset(uint32_t biased)
 {
-    uint32_t v = __byte_perm(biased, 0x64646464u, SEL);
-    const uint32_t off = 0x64806480u;      // (1152.0, 1152.0)
-    asm("sub.f16x2 %0, %0, %1;" : "+r"(v) : "r"(off));
-    return v;
+    return __byte_perm(biased, 0x64646464u, SEL);
+}
+
+__device__ __forceinline__ float ex2_fast(float x)      // 2^x; -inf gives 0
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 
 __device__ __forceinline__ uint32_t pack_f16(float lo, float hi)
@@ -211,11 +220,13 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
         const int t0 = chunk * p.tiles_per_item;
         const int t1 = min(nt, t0 + p.tiles_per_item);
 
-        // Q fragments (the B operand of S^T = K Q^T), query head g, as two fp16 planes.  The k index
+        // Q fragments (the B operand of S^T = K Q^T), query head g, as one fp16 plane.  The k index
         // of the MMA runs over the head dims in the order the int8 ldmatrix delivers them: for the
         // 16-dim chunk c, k = 2t, 2t + 1 are dims 16c + 4t, + 1 and k = 2t + 8, 2t + 9 are dims 16c + 4t + 2, + 3.
-        uint32_t qa[2][8][2];
+        uint32_t qa[8][2];
+        float qoff[2];                       // 1152 * (sum over the head dims of q as the MMA sees it), heads 2t, 2t + 1
         {
+            float qs = 0.f;
             const bf16 *qh = p.q + ((size_t)b * p.nq + (size_t)kvh * p.G + g) * kHeadDim;
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
@@ -228,11 +239,14 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
                 const float q2 = bf_lo(hi.y) + bf_lo(lo.y), q3 = bf_hi(hi.y) + bf_hi(lo.y);
                 const __half2 h01 = __floats2half2_rn(q0, q1), h23 = __floats2half2_rn(q2, q3);
                 const float2 f01 = __half22float2(h01), f23 = __half22float2(h23);
-                qa[0][c][0] = *reinterpret_cast<const uint32_t *>(&h01);
-                qa[0][c][1] = *reinterpret_cast<const uint32_t *>(&h23);
-                qa[1][c][0] = pack_f16(q0 - f01.x, q1 - f01.y);
-                qa[1][c][1] = pack_f16(q2 - f23.x, q3 - f23.y);
+                qa[c][0] = *reinterpret_cast<const uint32_t *>(&h01);
+                qa[c][1] = *reinterpret_cast<const uint32_t *>(&h23);
+                qs += (f01.x + f01.y) + (f23.x + f23.y);
             }
+            qs += __shfl_xor_sync(0xffffffffu, qs, 1);       // the four lanes of a head hold 32 dims each
+            qs += __shfl_xor_sync(0xffffffffu, qs, 2);
+            qoff[0] = kCodeOffset * __shfl_sync(0xffffffffu, qs, 8 * t);
+            qoff[1] = kCodeOffset * __shfl_sync(0xffffffffu, qs, 8 * t + 4);
         }
         // O^T accumulators: m-tile i holds head dims 16 i + 2 g (rows 0-7) and 16 i + 2 g + 1 (rows 8-15)
         // for the heads 2t and 2t + 1, in units of 2^(e_run - 127)
@@ -240,6 +254,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
 #pragma unroll
         for (int i = 0; i < 8; ++i)
             o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+        float psum[4] = {0.f, 0.f, 0.f, 0.f};   // [0], [1]: sum over the keys of the scaled weights, heads 2t and 2t + 1
         float m_run[2] = {-INFINITY, -INFINITY};
         float l_run[2] = {0.f, 0.f};
         int e_run = 0;                       // biased exponent of the largest value scale seen so far
@@ -287,10 +302,9 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         const uint32_t w0 = r[2 * h] ^ 0x80808080u, w1 = r[2 * h + 1] ^ 0x80808080u;
-                        const uint32_t a0 = s8x2_to_f16x2<0x4140>(w0), a2 = s8x2_to_f16x2<0x4342>(w0);
-                        const uint32_t a1 = s8x2_to_f16x2<0x4140>(w1), a3 = s8x2_to_f16x2<0x4342>(w1);
-                        mma_f16_16816(sT, a0, a1, a2, a3, qa[0][c + h][0], qa[0][c + h][1]);
-                        mma_f16_16816(sT, a0, a1, a2, a3, qa[1][c + h][0], qa[1][c + h][1]);
+                        const uint32_t a0 = s8x2_to_f16x2_offset<0x4140>(w0), a2 = s8x2_to_f16x2_offset<0x4342>(w0);
+                        const uint32_t a1 = s8x2_to_f16x2_offset<0x4140>(w1), a3 = s8x2_to_f16x2_offset<0x4342>(w1);
+                        mma_f16_16816(sT, a0, a1, a2, a3, qa[c + h][0], qa[c + h][1]);
                     }
                 }
             }
@@ -300,10 +314,11 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
             const float ksA = liveA ? ks_s[warp * 16 + g] : 0.f, ksB = liveB ? ks_s[warp * 16 + g + 8] : 0.f;
             float vsA = liveA ? vs_s[warp * 16 + g] : 0.f, vsB = liveB ? vs_s[warp * 16 + g + 8] : 0.f;
             float v[4], mx[2], corr[2];
-            v[0] = liveA ? sT[0] * ksA * p.scale_log2 : -INFINITY;
-            v[1] = liveA ? sT[1] * ksA * p.scale_log2 : -INFINITY;
-            v[2] = liveB ? sT[2] * ksB * p.scale_log2 : -INFINITY;
-            v[3] = liveB ? sT[3] * ksB * p.scale_log2 : -INFINITY;
+            const float kA = ksA * p.scale_log2, kB = ksB * p.scale_log2;
+            v[0] = liveA ? (sT[0] - qoff[0]) * kA : -INFINITY;
+            v[1] = liveA ? (sT[1] - qoff[1]) * kA : -INFINITY;
+            v[2] = liveB ? (sT[2] - qoff[0]) * kB : -INFINITY;
+            v[3] = liveB ? (sT[3] - qoff[1]) * kB : -INFINITY;
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 mx[j] = fmaxf(v[j], v[2 + j]);
@@ -311,7 +326,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
                 mx[j] = fmaxf(mx[j], __shfl_xor_sync(0xffffffffu, mx[j], 8));
                 mx[j] = fmaxf(mx[j], __shfl_xor_sync(0xffffffffu, mx[j], 16));
                 const float m_new = fmaxf(m_run[j], mx[j]);
-                corr[j] = m_new == -INFINITY ? 1.f : exp2f(m_run[j] - m_new);
+                corr[j] = m_new == -INFINITY ? 1.f : ex2_fast(m_run[j] - m_new);
                 m_run[j] = m_new;
                 l_run[j] *= corr[j];
             }
@@ -324,7 +339,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
                 int e_t = (int)((__float_as_uint(vm) >> 23) & 0xffu);
                 e_t = e_t > 253 ? 253 : e_t;
                 if (e_t > e_run) {
-                    const float down = e_run == 0 ? 0.f : exp2f((float)(e_run - e_t));   // o is still zero while e_run is 0
+                    const float down = e_run == 0 ? 0.f : ex2_fast((float)(e_run - e_t));   // o is still zero while e_run is 0
                     corr[0] *= down;        // (l_run has been updated already: it is not rescaled)
                     corr[1] *= down;
                     e_run = e_t;
@@ -339,7 +354,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float m = m_run[j & 1];
-                    ph4[j] = m == -INFINITY ? 0.f : exp2f(v[j] - m);
+                    ph4[j] = m == -INFINITY ? 0.f : ex2_fast(v[j] - m);
                     l_run[j & 1] += ph4[j];
                 }
                 // P^T (keys x heads) -> (heads x keys), the B fragment of O^T = V^T P^T: two 8 x 8 transposes
@@ -347,11 +362,18 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
                 asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pa0) : "r"(x0));
                 asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pa2) : "r"(x1));
             }
+            // (once the running maximum and the running scale have settled the factors are all one)
+            if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                o[i][0] *= corr[0]; o[i][1] *= corr[1];
-                o[i][2] *= corr[0]; o[i][3] *= corr[1];
+                for (int i = 0; i < 8; ++i) {
+                    o[i][0] *= corr[0]; o[i][1] *= corr[1];
+                    o[i][2] *= corr[0]; o[i][3] *= corr[1];
+                }
+                psum[0] *= corr[0];
+                psum[1] *= corr[1];
             }
+            // the weights against a row of ones: what the code offset adds to every head dim
+            mma_f16_16816(psum, 0x3c003c00u, 0x3c003c00u, 0x3c003c00u, 0x3c003c00u, pa0, pa2);
             // ---- O^T += V^T P^T: a transposed int8 ldmatrix hands lane (g, t) the keys 2t, 2t + 1 of the
             // head dims 2g, 2g + 1 of a chunk, so MMA row g is dim 2g and row g + 8 is dim 2g + 1
             {
@@ -363,8 +385,8 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         const uint32_t w0 = r[2 * h] ^ 0x80808080u, w1 = r[2 * h + 1] ^ 0x80808080u;
-                        const uint32_t a0 = s8x2_to_f16x2<0x4240>(w0), a1 = s8x2_to_f16x2<0x4341>(w0);
-                        const uint32_t a2 = s8x2_to_f16x2<0x4240>(w1), a3 = s8x2_to_f16x2<0x4341>(w1);
+                        const uint32_t a0 = s8x2_to_f16x2_offset<0x4240>(w0), a1 = s8x2_to_f16x2_offset<0x4341>(w0);
+                        const uint32_t a2 = s8x2_to_f16x2_offset<0x4240>(w1), a3 = s8x2_to_f16x2_offset<0x4341>(w1);
                         mma_f16_16816(o[i + h], a0, a1, a2, a3, pa0, pa2);
                     }
                 }
@@ -380,10 +402,11 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
         // ---- back to true units, then combine the four warps' partials
         {
             const float unit = __uint_as_float((uint32_t)e_run << 23);     // 2^(e_run - 127); 0 when every value scale was 0
+            const float off0 = kCodeOffset * psum[0], off1 = kCodeOffset * psum[1];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                o[i][0] *= unit; o[i][1] *= unit;
-                o[i][2] *= unit; o[i][3] *= unit;
+                o[i][0] = (o[i][0] - off0) * unit; o[i][1] = (o[i][1] - off1) * unit;
+                o[i][2] = (o[i][2] - off0) * unit; o[i][3] = (o[i][3] - off1) * unit;
             }
         }
 #pragma unroll

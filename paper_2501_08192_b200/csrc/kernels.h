@@ -215,9 +215,11 @@ cudaError_t launch_attention_kv8_kernel(const AttnArgs &a, const cudaLaunchConfi
 int attention_kv8_stages();
 // Grid size (persistent CTAs) and tiles per work item for the given sequence lengths (host array);
 // depends only on the lengths and the SM count.
-// `stages` = tiles the kernel's ring holds (3 for the bf16 cache, attention_kv8_stages() for int8).
+// `stages` = tiles the kernel's ring holds (3 for the bf16 cache, attention_kv8_stages() for int8);
+// `item_cost` = what starting an item, combining and writing its partial costs, in tile times (an int8
+// tile streams in half the time, so the same fixed work weighs twice as much).
 void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_count, int *grid, int *tiles_per_item,
-                    int stages = 3);
+                    int stages = 3, double item_cost = 1.5);
 // 2-D uint8 tensor map (rows x cols bytes, cols contiguous), box (box_cols x box_rows), 128-byte swizzle.
 bool encode_u8_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_cols,
                       uint32_t box_rows);
