@@ -382,10 +382,10 @@ PRESERVE_API int preserve_debug_copy(preserve_layer_t *layer, int32_t which, voi
  * [batch, n_kv_heads, kv_capacity, 128].  ctx_len is a device array, ctx_len_host the same
  * values on the host; each 0..kv_capacity-1.  At most 16 query heads per KV head.
  *
- * Limits and errors: the partial results of the call (one per run of 64-key tiles that one CTA
- * streams of one sequence and KV head: room is taken for 2 x SM count + batch x n_kv_heads of them,
- * 520 bytes per query head of the group each) must fit in the scratch array, else PRESERVE_ETOOBIG is
- * returned and nothing is queued; other bad arguments return PRESERVE_EINVAL / _EALIGN / _ESHAPE.
+ * Limits and errors: the partials of the call's work items (runs of 64-key tiles of one
+ * sequence and KV head; at most 8 x SM count + batch x n_kv_heads of them, 520 bytes per query
+ * head of the group each) must fit in the scratch array, else PRESERVE_ETOOBIG is returned and nothing is queued; other
+ * bad arguments return PRESERVE_EINVAL / _EALIGN / _ESHAPE.
  *
  * Sharing: all calls on one GPU use the same array, and it keeps whatever the previous
  * call left there (the call clears the one word that must start at zero).  Two calls that
@@ -397,11 +397,9 @@ PRESERVE_API int preserve_debug_copy(preserve_layer_t *layer, int32_t which, voi
  *
  * Status: the bounded waits of the two kernels report into the first word of the array;
  * preserve_attention_static_status() waits for the current device and returns PRESERVE_OK,
- * PRESERVE_ETIMEOUT (a wait gave up: o is undefined) or PRESERVE_ESHAPE (a partial result did
- * not fit the scratch array and was dropped, nothing was written out of bounds, o is wrong;
- * the ids of the partial results do not depend on the sequence lengths, so lengths within
- * kv_capacity cannot cause it).  ctx_len_host only sizes the launch: the kernels split the
- * work from the device values.  It allocates nothing either. */
+ * PRESERVE_ETIMEOUT (a wait gave up: o is undefined) or PRESERVE_ESHAPE (the device ctx_len
+ * described more work than ctx_len_host: the surplus was dropped, nothing was written out
+ * of bounds, o is wrong).  It allocates nothing either. */
 #define PRESERVE_STATIC_SCRATCH_BYTES (8u << 20)
 PRESERVE_API int preserve_attention_static(const void *q_hi, const void *q_lo, const void *k_cache,
                                            const void *v_cache, const int32_t *ctx_len,

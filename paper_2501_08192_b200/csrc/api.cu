@@ -325,7 +325,7 @@ struct StepPlan {
     uint64_t kv_bytes, alg_bytes;
     bool pf_a, pf_b;
     int pdl;
-    int attn_grid, attn_items_per_stream;
+    int attn_grid, attn_tpi, attn_items_per_stream;
 };
 
 int check_step(preserve_layer *L, const preserve_step_io_t *io, StepPtrs *sp)
@@ -437,9 +437,12 @@ void plan_step(preserve_layer *L, const StepPtrs &sp, StepPlan *pl)
 {
     const auto &c = L->cfg;
     const int B = sp.batch;
-    uint64_t sum_ctx = 0;
-    for (int b = 0; b < B; ++b)
+    uint64_t sum_ctx = 0, max_tiles_seq = 0;
+    for (int b = 0; b < B; ++b) {
         sum_ctx += (uint64_t)sp.ctx_len_host[b];
+        const uint64_t nt = (uint64_t)(sp.ctx_len_host[b] + 1 + 63) / 64;
+        max_tiles_seq = nt > max_tiles_seq ? nt : max_tiles_seq;
+    }
     // K and V bytes of the cached tokens: the SelfAttention node's memSize for Algorithm 1 (an int8
     // cache: the codes; its scales, 4 bytes per 128, are read too but not prefetched)
     pl->kv_bytes = 2 * sum_ctx * c.n_kv_heads * c.head_dim * (L->kv8 ? 1 : 2);
@@ -469,8 +472,9 @@ void plan_step(preserve_layer *L, const StepPtrs &sp, StepPlan *pl)
     // (only == -1: the whole step; -2 / -3: just the prefetch beside window A / B; k >= 0: just kernel k)
     pl->pf_a = (L->only == -1 || L->only == -2) && pl->planned[0][0] + pl->planned[0][1] + pl->planned[0][2] > 0;
     pl->pf_b = (L->only == -1 || L->only == -3) && pl->planned[1][0] + pl->planned[1][1] > 0;
-    plan_attention(sp.ctx_len_host, B, c.n_kv_heads, L->sm_count, &pl->attn_grid, &pl->attn_items_per_stream,
-                   L->kv8 ? attention_kv8_stages() : 3);
+    plan_attention(sp.ctx_len_host, B, c.n_kv_heads, L->sm_count, &pl->attn_grid, &pl->attn_tpi,
+                   L->kv8 ? attention_kv8_stages() : 3, L->kv8 ? 3.0 : 1.5);
+    pl->attn_items_per_stream = (int)((max_tiles_seq + pl->attn_tpi - 1) / pl->attn_tpi);
     // (the merge kernel sizes its CTAs from this, between 4 and 32 warps: clamp here so that the
     // number that enters the graph signature changes as rarely as the launch does)
     if (pl->attn_items_per_stream < 4) pl->attn_items_per_stream = 4;
@@ -643,6 +647,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
         a.ctx_len = sp.ctx_len;
         a.B = B; a.nq = c.n_q_heads; a.nkv = c.n_kv_heads; a.cap = cap;
         a.grid = pl.attn_grid;
+        a.tiles_per_item = pl.attn_tpi;
         a.max_items_per_stream = pl.attn_items_per_stream;
         a.max_items = L->max_items;
         a.part_o = L->part_o;
@@ -815,7 +820,7 @@ void step_signature(const preserve_layer *L, const StepPtrs &sp, const StepPlan 
     put((uint64_t)L->budget);
     put((uint64_t)L->window_delay_ns | (uint64_t)L->pf_chunk << 32);
     put((uint64_t)L->prefetch_ctas);
-    put((uint64_t)pl.attn_grid);
+    put((uint64_t)pl.attn_grid | (uint64_t)pl.attn_tpi << 32);
     put((uint64_t)pl.attn_items_per_stream);
     putp(L->comm);
     putp(L->ext_attn_sum);

@@ -8,18 +8,17 @@
 // (sequence, kv head) is one contiguous run and a tile of 64 keys is two TMA
 // boxes of 64 x 64 bf16 (128-byte swizzle) per tensor.
 //
-// Every CTA streams an equal share of the cache: the 64-key tiles of all (sequence, kv head)
-// streams form one line in cache order, CTA c takes the c-th of g equal ranges of it, and a range
-// that crosses from one stream into the next is cut there into segments (attn_common.cuh).  A
-// short cache gives every CTA at most one ring fill, so every tile is in shared memory before the
-// queries exist; otherwise one CTA per SM while the cache is a few ring fills (the kernels before
-// and after can then be co-resident), two per SM for long caches (plan_attention).  Warp 4 is the producer: one lane issues the TMA loads into a
+// Persistent CTAs walk a static list of work items = (sequence, kv head, run of
+// `tiles_per_item` tiles) in address order.  A short cache is cut into items of at most
+// one ring fill, one per CTA, so every tile is in shared memory before the queries exist;
+// otherwise one CTA per SM while the cache is a few ring fills (the kernels before and
+// after can then be co-resident), two per SM for long caches (plan_attention).  Warp 4 is the producer: one lane issues the TMA loads into a
 // 3-stage ring guarded by full/empty mbarriers (all waits bounded).  Warps 0-3 each
 // own 16 of a tile's 64 keys: S = Q K^T with mma.sync (Q rows = query heads padded
 // to 16, from registers; K via ldmatrix), online softmax in fp32 with exp2,
 // O += P V (V via ldmatrix.trans).  At the end of an item the four warps combine
 // their (max, sum, O) through the ring stage they consumed last and the CTA writes
-// ONE fp32 partial per segment (or the final o when the segment is the whole sequence).
+// ONE fp32 partial per item (or the final o when the item is the whole sequence).
 // k_attn_merge then combines the partials of a sequence in fixed order.  Nothing
 // depends on timing, so results are bit-stable.
 #include <cstdlib>
@@ -42,7 +41,7 @@ struct AttnParams {
     size_t q_plane;
     const int *ctx_len;
     int B, nq, nkv, G, cap;
-    int grid;               // CTAs of the split-KV launch (the merge kernel re-derives the split from it)
+    int tiles_per_item;
     int max_items;
     float scale_log2;       // log2(e) / sqrt(d)
     float *part_o;          // [item][G][d] CTA partials (unnormalised, relative to the item's max)
@@ -59,7 +58,7 @@ struct AttnSmem {
     uint64_t full[kStages];
     uint64_t empty[kStages];
     float comb_ml[kConsumerWarps][16][2];
-    int tile_base[kMaxStreams + 1];      // last: the launch only asks for the entries it needs
+    int item_base[kMaxStreams + 1];      // last: the launch only asks for the entries it needs
 };
 
 // Where consumer warp w keeps row r (a query head of the group) of its O partial inside a ring
@@ -93,16 +92,17 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
     }
     trace_start(p.trace);
     pdl_launch_dependents();
-    build_tile_table(p, sm.tile_base);       // sequence lengths are inputs of the step: no dependency
+    build_item_table(p, sm.item_base);       // sequence lengths are inputs of the step: no dependency
     __syncthreads();
-    // This CTA's share of the tile line.  Segment ids stay below grid + streams whatever the lengths
-    // are; the partial buffers hold max_items entries and a segment beyond them is dropped by the
-    // producer and the consumers alike (the result is then wrong, and the status word says why).
-    // (With fewer tiles than CTAs only the first total_tiles CTAs take part, one tile each.)
-    const int total_tiles = sm.tile_base[streams];
-    const int g_eff = min((int)gridDim.x, total_tiles);
-    const int x_lo = (int)blockIdx.x < g_eff ? cta_first_tile(blockIdx.x, g_eff, total_tiles) : 0;
-    const int x_hi = (int)blockIdx.x < g_eff ? cta_first_tile(blockIdx.x + 1, g_eff, total_tiles) : 0;
+    // The partial buffers hold max_items entries, sized from the host copy of the lengths.  Device
+    // lengths that disagree with it must not write past them: the surplus items are dropped (the
+    // result is then wrong, and the status word says why).
+    int total_items = sm.item_base[streams];
+    if (total_items > p.max_items) {
+        total_items = p.max_items;
+        if (threadIdx.x == 0)
+            atomicCAS(p.status, ST_OK, ST_ITEMS_OVERFLOW);
+    }
 
     if (warp == kConsumerWarps) {
         // ------------------------------------------------------------ producer
@@ -113,13 +113,12 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
             const uint64_t pol = policy_evict_first();   // each cached byte is read once per step
             uint32_t it = 0;
             bool ok = true, waited = false;
-            for (int x = x_lo; x < x_hi && ok;) {
-                const Segment sg = next_segment(sm.tile_base, streams, g_eff, blockIdx.x, x_hi, x);
-                if (sg.id >= p.max_items)
-                    continue;
-                const int sidx = sg.sidx;
-                const int nt = sm.tile_base[sidx + 1] - sm.tile_base[sidx];
-                const int t0 = sg.t0, t1 = sg.t1;
+            for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+                const int sidx = find_stream(sm.item_base, streams, item);
+                const int chunk = item - sm.item_base[sidx];
+                const int nt = tiles_of(p.ctx_len[sidx / p.nkv]);
+                const int t0 = chunk * p.tiles_per_item;
+                const int t1 = min(nt, t0 + p.tiles_per_item);
                 for (int tile = t0; tile < t1; ++tile, ++it) {
                     const int st = it % kStages;
                     const uint32_t ph = (it / kStages) & 1;
@@ -150,17 +149,14 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
     bool ok = true;
     pdl_wait();    // q comes from the QKV projection
     trace_waited(p.trace);
-    for (int x = x_lo; x < x_hi;) {
-        const Segment sg = next_segment(sm.tile_base, streams, g_eff, blockIdx.x, x_hi, x);
-        if (sg.id >= p.max_items) {
-            if (threadIdx.x == 0)
-                atomicCAS(p.status, ST_OK, ST_ITEMS_OVERFLOW);
-            continue;
-        }
-        const int sidx = sg.sidx, item = sg.id;
+    for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+        const int sidx = find_stream(sm.item_base, streams, item);
         const int b = sidx / p.nkv, kvh = sidx % p.nkv;
+        const int chunk = item - sm.item_base[sidx];
         const int n_keys = p.ctx_len[b] + 1;
-        const int t0 = sg.t0, t1 = sg.t1;
+        const int nt = tiles_of(p.ctx_len[b]);
+        const int t0 = chunk * p.tiles_per_item;
+        const int t1 = min(nt, t0 + p.tiles_per_item);
 
         constexpr bool narrow = NARROW;
         // Q fragments: rows = query heads of the group (zero beyond G)
@@ -410,7 +406,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
             }
         }
         consumer_barrier();
-        const int n_items_stream = sg.pieces;
+        const int n_items_stream = sm.item_base[sidx + 1] - sm.item_base[sidx];
         // two head dims per consumer thread, the heads of one parity per half of the threads
         const int d2 = threadIdx.x & 63;
         for (int r = threadIdx.x >> 6; r < p.G; r += 2) {
@@ -470,35 +466,22 @@ __global__ void __launch_bounds__(kMergeMaxWarps * 32) k_attn_merge(const __grid
     long long *tr = p.trace ? p.trace + kTraceSlots : nullptr;
     trace_start(tr);
     pdl_launch_dependents();
-    // where this stream lies on the tile line: parallel sums over the streams before it and over all
-    // streams (the lengths are inputs), then the CTAs of the split-KV launch whose ranges touch it
-    __shared__ int tot_s[kMergeMaxWarps];
-    int cnt = 0, tot = 0;
-    for (int s2 = tid; s2 < p.B * p.nkv; s2 += blockDim.x) {
+    // first item of this stream: parallel count over the streams before it (lengths are inputs)
+    int cnt = 0;
+    for (int s2 = tid; s2 < sidx; s2 += blockDim.x) {
         const int nt = tiles_of(p.ctx_len[s2 / p.nkv]);
-        cnt += s2 < sidx ? nt : 0;
-        tot += nt;
+        cnt += (nt + p.tiles_per_item - 1) / p.tiles_per_item;
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
+    for (int o = 16; o > 0; o >>= 1)
         cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-        tot += __shfl_xor_sync(0xffffffffu, tot, o);
-    }
-    if (lane == 0) {
+    if (lane == 0)
         cnt_s[warp] = cnt;
-        tot_s[warp] = tot;
-    }
+    const int n_items = (tiles_of(p.ctx_len[b]) + p.tiles_per_item - 1) / p.tiles_per_item;
     __syncthreads();
-    int first = 0, total_tiles = 0;
-    for (int i = 0; i < n_warps; ++i) {
-        first += cnt_s[i];
-        total_tiles += tot_s[i];
-    }
-    const int g_eff = min(p.grid, total_tiles);
-    const int c_first = cta_of_tile(first, g_eff, total_tiles);
-    const int c_last = cta_of_tile(first + tiles_of(p.ctx_len[b]) - 1, g_eff, total_tiles);
-    const int base = c_first + sidx;
-    const int n_items = c_last - c_first + 1;
+    int base = 0;
+    for (int i = 0; i < n_warps; ++i)
+        base += cnt_s[i];
     pdl_wait();    // the partials come from the split-KV kernel (every CTA waits, also those with nothing to do)
     trace_waited(tr);
     if (n_items > 1) {          // a single item was finished by the split-KV kernel itself
@@ -547,11 +530,11 @@ __global__ void __launch_bounds__(kMergeMaxWarps * 32) k_attn_merge(const __grid
 
 static size_t attn_smem_bytes(int streams)
 {
-    return offsetof(AttnSmem, tile_base) + sizeof(int) * (size_t)(streams + 1) + 1024;
+    return offsetof(AttnSmem, item_base) + sizeof(int) * (size_t)(streams + 1) + 1024;
 }
 
-void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_count, int *grid, int *pieces_per_stream,
-                    int stages)
+void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_count, int *grid, int *tiles_per_item,
+                    int stages, double item_cost)
 {
     uint64_t total_tiles = 0;
     int longest = 1;
@@ -560,17 +543,53 @@ void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_coun
         total_tiles += (uint64_t)nkv * nt;
         longest = nt > longest ? nt : longest;
     }
-    // Every CTA streams an equal share of the tiles (attn_common.cuh).  One CTA per SM while a share
-    // is at most one ring fill: every tile is then in shared memory before the queries exist, what
-    // remains after the wait is arithmetic, and half of every SM's shared memory stays free for the
-    // kernels before and after.  Otherwise two CTAs per SM: up to two ring fills per SM are still all
-    // in flight before the queries exist, and a long cache is a steady stream that wants twice the
-    // bytes in flight.
-    const int g = total_tiles <= (uint64_t)stages * sm_count ? sm_count : 2 * sm_count;
+    // A short cache fits the CTAs' rings whole: items of at most kStages tiles, one per CTA, are then
+    // all in shared memory before the queries exist, and what remains after the wait is arithmetic.
+    // The shortest such items that leave a (sequence, head) at most one partial per merge warp.
+    for (int tpi = 1; tpi <= stages; ++tpi) {
+        uint64_t items = 0;
+        int per_stream = 0;
+        for (int b = 0; b < batch; ++b) {
+            const int nt = (ctx_len_host[b] + 1 + kTileKeys - 1) / kTileKeys;
+            const int n = (nt + tpi - 1) / tpi;
+            items += (uint64_t)nkv * n;
+            per_stream = n > per_stream ? n : per_stream;
+        }
+        if (items <= (uint64_t)2 * sm_count && per_stream <= 32) {
+            *grid = items <= (uint64_t)sm_count ? sm_count : 2 * sm_count;
+            *tiles_per_item = tpi;
+            return;
+        }
+    }
+    // One CTA per SM while the whole cache is at most two ring fills per SM: the ring then holds
+    // most of the CTA's share before the queries exist, and half of every SM's shared memory stays
+    // free for the kernels before and after.  Longer caches are a steady stream: two CTAs per SM
+    // keep twice the bytes in flight.
+    const int g = total_tiles <= (uint64_t)2 * stages * sm_count ? sm_count : 2 * sm_count;
+    // Work items = runs of `tpi` 64-key tiles of one sequence, dealt to the CTAs round-robin.  The
+    // kernel lasts about rounds x (tpi + the per-item cost of combining and writing a partial,
+    // worth ~1.5 tiles), rounds = items / CTAs rounded up: take the tpi that minimises that, between
+    // a quarter of an even share (at most four items per CTA) and a whole share.
+    const int tpi_hi = (int)((total_tiles + g - 1) / g) + 1;
+    int tpi_lo = (int)((total_tiles + 4ull * g - 1) / (4ull * g));
+    tpi_lo = tpi_lo < 1 ? 1 : tpi_lo;
+    int best = tpi_lo;
+    double best_cost = -1.0;
+    for (int tpi = tpi_lo; tpi <= tpi_hi && tpi <= longest + 1; ++tpi) {
+        uint64_t items = 0;
+        for (int b = 0; b < batch; ++b) {
+            const int nt = (ctx_len_host[b] + 1 + kTileKeys - 1) / kTileKeys;
+            items += (uint64_t)nkv * ((nt + tpi - 1) / tpi);
+        }
+        const uint64_t rounds = (items + g - 1) / g;
+        const double cost = (double)rounds * (tpi + item_cost);
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            best = tpi;
+        }
+    }
     *grid = g;
-    // most segments any stream is cut into (sizes the merge CTAs): its tiles over the share, plus one
-    const uint64_t g_eff = total_tiles < (uint64_t)g ? total_tiles : (uint64_t)g;
-    *pieces_per_stream = (int)(((uint64_t)longest * g_eff + total_tiles - 1) / total_tiles) + 1;
+    *tiles_per_item = best;
 }
 
 cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
@@ -585,7 +604,7 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     p.o_plane = a.o_plane;
     p.ctx_len = a.ctx_len;
     p.B = a.B; p.nq = a.nq; p.nkv = a.nkv; p.G = a.nq / a.nkv; p.cap = a.cap;
-    p.grid = a.grid;
+    p.tiles_per_item = a.tiles_per_item;
     p.max_items = a.max_items;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)kHeadDim);
     p.part_o = a.part_o;
@@ -704,11 +723,15 @@ extern "C" int preserve_attention_static(const void *q_hi, const void *q_lo, con
 
     // ---- carve the array: [status word, 256 B][partial O][partial (max, sum)]
     const int G = n_q_heads / n_kv_heads;
-    int grid = 0, pieces = 1;
-    plan_attention(ctx_len_host, batch, n_kv_heads, g_scratch_sms[dev], &grid, &pieces);
-    // segment ids stay below grid + streams (attn_common.cuh)
-    const uint64_t n_items = (uint64_t)grid + (uint64_t)batch * n_kv_heads;
-    const uint64_t max_items_seq = (uint64_t)pieces;
+    int grid = 0, tpi = 1;
+    plan_attention(ctx_len_host, batch, n_kv_heads, g_scratch_sms[dev], &grid, &tpi);
+    uint64_t n_items = 0, max_items_seq = 0;
+    for (int b = 0; b < batch; ++b) {
+        const uint64_t nt = (uint64_t)(ctx_len_host[b] + 1 + kTileKeys - 1) / kTileKeys;
+        const uint64_t ni = (nt + tpi - 1) / tpi;
+        n_items += (uint64_t)n_kv_heads * ni;
+        max_items_seq = ni > max_items_seq ? ni : max_items_seq;
+    }
     const uint64_t o_bytes = n_items * G * kHeadDim * sizeof(float);
     const uint64_t ml_bytes = n_items * G * 2 * sizeof(float);
     if (256 + o_bytes + ml_bytes > PRESERVE_STATIC_SCRATCH_BYTES)
@@ -731,6 +754,7 @@ extern "C" int preserve_attention_static(const void *q_hi, const void *q_lo, con
     a.ctx_len = ctx_len;
     a.B = batch; a.nq = n_q_heads; a.nkv = n_kv_heads; a.cap = kv_capacity;
     a.grid = grid;
+    a.tiles_per_item = tpi;
     a.max_items = (int)n_items;
     a.max_items_per_stream = (int)max_items_seq;
     a.part_o = reinterpret_cast<float *>(base + 256);

@@ -56,6 +56,7 @@ struct AttnKv8Params {
     size_t q_plane;
     const int *ctx_len;
     int B, nq, nkv, G, cap, scale_cap;
+    int tiles_per_item;
     int max_items;
     float scale_log2;
     float *part_o;
@@ -73,7 +74,7 @@ struct AttnKv8Smem {
     float comb_ml[kConsumerWarps][kMaxGroup8][2];
     uint64_t full[kStages8];
     uint64_t empty[kStages8];
-    int tile_base[kMaxStreams + 1];      // last: the launch only asks for the entries it needs
+    int item_base[kMaxStreams + 1];      // last: the launch only asks for the entries it needs
 };
 
 // D(16x8, f32) += A(16x16, f16, row) * B(16x8, f16, col)
@@ -151,14 +152,14 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
     }
     trace_start(p.trace);
     pdl_launch_dependents();
-    build_tile_table(p, sm.tile_base);       // sequence lengths are inputs of the step: no dependency
+    build_item_table(p, sm.item_base);       // sequence lengths are inputs of the step: no dependency
     __syncthreads();
-    // this CTA's share of the tile line (attn_common.cuh); a segment whose id does not fit the partial
-    // buffers is dropped by the producer and the consumers alike, with a status
-    const int total_tiles = sm.tile_base[streams];
-    const int g_eff = min((int)gridDim.x, total_tiles);
-    const int x_lo = (int)blockIdx.x < g_eff ? cta_first_tile(blockIdx.x, g_eff, total_tiles) : 0;
-    const int x_hi = (int)blockIdx.x < g_eff ? cta_first_tile(blockIdx.x + 1, g_eff, total_tiles) : 0;
+    int total_items = sm.item_base[streams];
+    if (total_items > p.max_items) {         // device lengths disagree with the host copy: never write past the partials
+        total_items = p.max_items;
+        if (threadIdx.x == 0)
+            atomicCAS(p.status, ST_OK, ST_ITEMS_OVERFLOW);
+    }
 
     if (warp == kConsumerWarps) {
         // ------------------------------------------------------------ producer
@@ -170,13 +171,12 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
             const uint64_t pol = policy_evict_first();
             uint32_t it = 0;
             bool ok = true, waited = false;
-            for (int x = x_lo; x < x_hi && ok;) {
-                const Segment sg = next_segment(sm.tile_base, streams, g_eff, blockIdx.x, x_hi, x);
-                if (sg.id >= p.max_items)
-                    continue;
-                const int sidx = sg.sidx;
-                const int nt = sm.tile_base[sidx + 1] - sm.tile_base[sidx];
-                const int t0 = sg.t0, t1 = sg.t1;
+            for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+                const int sidx = find_stream(sm.item_base, streams, item);
+                const int chunk = item - sm.item_base[sidx];
+                const int nt = tiles_of(p.ctx_len[sidx / p.nkv]);
+                const int t0 = chunk * p.tiles_per_item;
+                const int t1 = min(nt, t0 + p.tiles_per_item);
                 for (int tile = t0; tile < t1; ++tile, ++it) {
                     const int st = it % kStages8;
                     const uint32_t ph = (it / kStages8) & 1;
@@ -211,17 +211,14 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
     // this lane's ldmatrix row: matrices 0..3 of an x4 load = (keys 0-7 | 8-15) x (chunk c | c + 1)
     const int lkey = warp * 16 + (((lane >> 3) & 1) << 3) + (lane & 7);
     const int lsw = lkey & 7, lch = lane >> 4;
-    for (int x = x_lo; x < x_hi;) {
-        const Segment sg = next_segment(sm.tile_base, streams, g_eff, blockIdx.x, x_hi, x);
-        if (sg.id >= p.max_items) {
-            if (threadIdx.x == 0)
-                atomicCAS(p.status, ST_OK, ST_ITEMS_OVERFLOW);
-            continue;
-        }
-        const int sidx = sg.sidx, item = sg.id;
+    for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+        const int sidx = find_stream(sm.item_base, streams, item);
         const int b = sidx / p.nkv, kvh = sidx % p.nkv;
+        const int chunk = item - sm.item_base[sidx];
         const int n_keys = p.ctx_len[b] + 1;
-        const int t0 = sg.t0, t1 = sg.t1;
+        const int nt = tiles_of(p.ctx_len[b]);
+        const int t0 = chunk * p.tiles_per_item;
+        const int t1 = min(nt, t0 + p.tiles_per_item);
 
         // Q fragments (the B operand of S^T = K Q^T), query head g, as one fp16 plane.  The k index
         // of the MMA runs over the head dims in the order the int8 ldmatrix delivers them: for the
@@ -431,7 +428,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
             }
         }
         consumer_barrier();
-        const int n_items_stream = sg.pieces;
+        const int n_items_stream = sm.item_base[sidx + 1] - sm.item_base[sidx];
         // two head dims per consumer thread, the heads of one parity per half of the threads
         const int d2 = threadIdx.x & 63;
         for (int r = threadIdx.x >> 6; r < p.G; r += 2) {
@@ -471,7 +468,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
 
 static size_t attn_kv8_smem_bytes(int streams)
 {
-    return offsetof(AttnKv8Smem, tile_base) + sizeof(int) * (size_t)(streams + 1) + 1024;
+    return offsetof(AttnKv8Smem, item_base) + sizeof(int) * (size_t)(streams + 1) + 1024;
 }
 
 int attention_kv8_stages() { return kStages8; }
@@ -495,6 +492,7 @@ cudaError_t launch_attention_kv8_kernel(const AttnArgs &a, const cudaLaunchConfi
     p.q_plane = a.q_plane;
     p.ctx_len = a.ctx_len;
     p.B = a.B; p.nq = a.nq; p.nkv = a.nkv; p.G = a.nq / a.nkv; p.cap = a.cap; p.scale_cap = a.scale_cap;
+    p.tiles_per_item = a.tiles_per_item;
     p.max_items = a.max_items;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)kHeadDim);
     p.part_o = a.part_o;

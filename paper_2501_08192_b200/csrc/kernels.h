@@ -184,11 +184,12 @@ struct AttnArgs {
     size_t q_plane;
     const int *ctx_len;   // device [B]; keys attended = ctx_len[b] + 1
     int B, nq, nkv, cap;
-    int grid;             // persistent CTAs: each streams an equal share of the 64-key tiles
-    int max_items;        // capacity of the partial buffers (at least grid + B * nkv)
+    int grid;             // persistent CTAs
+    int tiles_per_item;   // 64-key tiles per work item
+    int max_items;        // capacity of the partial buffers
     float *part_o;        // fp32 [max_items, G, d]: one partial per work item
     float *part_ml;       // fp32 [max_items, G, 2]
-    int max_items_per_stream;   // most partials of one (sequence, kv head) (sizes the merge CTAs)
+    int max_items_per_stream;   // work items of the longest sequence (sizes the merge CTAs)
     void *o_out;          // split bf16 [2][rows][nq,d]
     size_t o_plane;
     int *status;
@@ -212,12 +213,13 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s);
 // the int8-cache split-KV kernel alone (attn_kv8.cu); launch_attention adds the merge kernel
 cudaError_t launch_attention_kv8_kernel(const AttnArgs &a, const cudaLaunchConfig_t &base_cfg);
 int attention_kv8_stages();
-// Grid size (persistent CTAs) for the given sequence lengths (host array); depends only on the lengths
-// and the SM count.
-// `stages` = tiles the kernel's ring holds (3 for the bf16 cache, attention_kv8_stages() for int8).
-// *pieces_per_stream = the most partial results any (sequence, kv head) is cut into.
-void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_count, int *grid, int *pieces_per_stream,
-                    int stages = 3);
+// Grid size (persistent CTAs) and tiles per work item for the given sequence lengths (host array);
+// depends only on the lengths and the SM count.
+// `stages` = tiles the kernel's ring holds (3 for the bf16 cache, attention_kv8_stages() for int8);
+// `item_cost` = what starting an item, combining and writing its partial costs, in tile times (an int8
+// tile streams in half the time, so the same fixed work weighs twice as much).
+void plan_attention(const int32_t *ctx_len_host, int batch, int nkv, int sm_count, int *grid, int *tiles_per_item,
+                    int stages = 3, double item_cost = 1.5);
 // 2-D uint8 tensor map (rows x cols bytes, cols contiguous), box (box_cols x box_rows), 128-byte swizzle.
 bool encode_u8_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_cols,
                       uint32_t box_rows);
