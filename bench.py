@@ -427,13 +427,12 @@ def bench_config(P, I, torch, dist, args, idx, rank, local_rank, world, stream, 
     except Exception as e:      # noqa: BLE001
         res["model"] = {"error": str(e)}
     # ---- the same configuration at the precisions of the paper's runs (Section 4: int8 weights and
-    # KV-cache): int8 KV-cache on every configuration; int8 weights where the library has them (the
-    # split-K GEMV path).  Each row: vanilla and early-launch-only times, the attention kernel alone.
+    # KV-cache): int8 KV-cache, int8 weights, and both.  Each row: vanilla and early-launch-only times,
+    # and (int8 cache) the attention kernel alone.
     if not args.no_sweep:
         wl.close()
-        variants = [("int8_kv", P.FLAG_INT8_KV)]
-        if shape.batch < 16:
-            variants += [("int8_weights", P.FLAG_INT8_WEIGHTS), ("int8_weights_and_kv", P.FLAG_INT8_WEIGHTS | P.FLAG_INT8_KV)]
+        variants = [("int8_kv", P.FLAG_INT8_KV), ("int8_weights", P.FLAG_INT8_WEIGHTS),
+                    ("int8_weights_and_kv", P.FLAG_INT8_WEIGHTS | P.FLAG_INT8_KV)]
         for vname, vflags in variants:
             wl8 = Workload(P, I, torch, idx, rank, l2, args.rotation, flags=vflags)
             alg8 = int(P.preserve_algorithmic_bytes(wl8.cfg, shape.batch, wl8.sum_ctx))
@@ -994,7 +993,7 @@ def main():
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--int8-kv", action="store_true", help="run the main measurement over an int8 KV-cache (profiling aid)")
     ap.add_argument("--int8-weights", action="store_true",
-                    help="run the main measurement with int8 weights (batch < 16 configurations; profiling aid)")
+                    help="run the main measurement with int8 weights (profiling aid)")
     ap.add_argument("--no-kernels", action="store_true", help="skip the isolated per-kernel timing")
     ap.add_argument("--budget-bytes", type=int, default=-1, help="prefetch budget per window (default: the library's)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")

@@ -67,7 +67,31 @@ struct GemmTcParams {
     int planes;         // activation planes in the B operand: 2 = bf16 hi + lo, 1 = a single fp16 plane
     int epi_warps;      // 8 or 16
     int producers;      // 1..kTcMaxProducers threads that issue the ring's TMA loads (stage uses dealt round-robin)
+    int w8;             // the weight tiles arrive as int8 codes ([rows][64] bytes, no swizzle) and are widened in shared memory
+    int a16_off;        // w8: offset of the two widened weight tiles (mt * 16 KiB each) behind the ring
+    const float *wscale;  // w8: one fp32 scale per packed weight row
 };
+
+// int8 -> 16-bit widening of two codes of `biased` (the loaded word with every byte's top bit flipped:
+// code + 128 as an unsigned byte), exact.  SEL places the bytes: 0x4140 = bytes (0, 1), 0x4342 = (2, 3).
+// fp16: the byte lands in the mantissa of 1024.0, i.e. 1152 + code; subtract 1152.
+// bf16 (7 mantissa bits): the low seven bits land in the mantissa of 128.0, i.e. 128 + (byte & 127); subtract
+// 128 when the byte's top bit is set (code >= 0), 256 when it is not.
+template <uint32_t SEL>
+__device__ __forceinline__ uint32_t widen_s8x2(uint32_t biased, bool fp16)
+{
+    uint32_t r;
+    if (fp16) {
+        r = __byte_perm(biased, 0x64646464u, SEL);
+        const uint32_t off = 0x64806480u;      // (1152.0, 1152.0)
+        asm("sub.f16x2 %0, %0, %1;" : "+r"(r) : "r"(off));
+    } else {
+        const uint32_t w = __byte_perm(biased, 0x43434343u, SEL);
+        const uint32_t minuend = w & 0xff7fff7fu, subtrahend = (w & 0x00800080u) ^ 0x43804380u;
+        asm("sub.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(minuend), "r"(subtrahend));
+    }
+    return r;
+}
 
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr)
 {
@@ -133,6 +157,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ uint64_t full[kTcMaxStages], empty[kTcMaxStages], accum_bar, push_bar;
+    __shared__ uint64_t conv[2], a16_free[2];      // int8 weights: a widened tile is complete / has been consumed
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile int poisoned;
     __shared__ EpilogueTables tabs;
@@ -140,7 +165,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile = blockIdx.x;
     const int s = blockIdx.y;
-    const int a_bytes = p.mt * kATileBytes;
+    const int a_bytes = p.mt * (p.w8 ? kATileBytes / 2 : kATileBytes);
     const int stage_bytes = a_bytes + p.planes * p.NB * kTcBlockK * 2;
     const int acc_cols = p.planes * p.NB;      // TMEM columns of one weight tile's accumulator
     const int kb0 = (int)((long long)p.kblocks * s / p.splits);
@@ -155,6 +180,13 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             mbar_init(&empty[i], 1);
         }
         mbar_init(&accum_bar, 1);
+        if (p.w8) {
+            // the epilogue warps that issue no TMA loads widen the tiles: one arrival per warp and tile
+            for (int j = 0; j < 2; ++j) {
+                mbar_init(&conv[j], p.epi_warps - (p.producers - 1));
+                mbar_init(&a16_free[j], 1);
+            }
+        }
         mbar_fence_init();
         poisoned = 0;
         tma_prefetch_desc(&p.w_map);
@@ -227,10 +259,14 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             for (int kb = kb0; kb < kb1; ++kb, ++it) {
                 const int st = it % p.stages;
                 const uint32_t ph = (it / p.stages) & 1;
-                if (!mbar_wait(&full[st], ph, p.status, ST_TIMEOUT_FULL)) { poisoned = 1; ok = false; break; }
+                // (int8 weights: the widened tile of this use, slot it % 2, completes after the stage has landed)
+                const int j = it & 1;
+                if (!(p.w8 ? mbar_wait(&conv[j], (it >> 1) & 1, p.status, ST_TIMEOUT_FULL)
+                           : mbar_wait(&full[st], ph, p.status, ST_TIMEOUT_FULL))) { poisoned = 1; ok = false; break; }
                 tc_fence_after();
-                const uint32_t a_addr = smem_u32(smem + (size_t)st * stage_bytes);
-                const uint64_t bdesc = make_smem_desc(a_addr + a_bytes);
+                const uint32_t st_addr = smem_u32(smem + (size_t)st * stage_bytes);
+                const uint32_t a_addr = p.w8 ? smem_u32(smem + p.a16_off + (size_t)j * p.mt * kATileBytes) : st_addr;
+                const uint64_t bdesc = make_smem_desc(st_addr + a_bytes);
                 for (int m = 0; m < p.mt; ++m) {
                     // each 128-row weight tile has its own accumulator (2 * NB TMEM columns)
                     const uint64_t adesc = make_smem_desc(a_addr + m * kATileBytes);
@@ -240,6 +276,8 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                                (kb > kb0 || k > 0) ? 1u : 0u);
                 }
                 tc_commit(&empty[st]);      // slot is free once these MMAs have read it
+                if (p.w8)
+                    tc_commit(&a16_free[j]);
             }
             if (ok)
                 tc_commit(&accum_bar);      // accumulator complete
@@ -302,6 +340,46 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             run_producer(warp - 1);
         __syncwarp();
     }
+    else if (is_epi && p.w8) {
+        // ---------------------------------------------------- int8 weights: widen every tile
+        // Tile use `itc` is converted from its ring stage into widened slot itc % 2 (the MMA operand
+        // layout: K-major rows, 8-row atoms of 1 KiB, 128-byte swizzle).  A task = 16 codes of one
+        // row (one 16-byte load, two 16-byte stores).  The slot is written again only after the MMAs
+        // of use itc - 2 have read it.
+        const int cw = warp - 1 - p.producers, n_conv = p.epi_warps - (p.producers - 1);
+        const bool f16 = p.planes == 1;
+        uint32_t itc = 0;
+        for (int kb = kb0; kb < kb1; ++kb, ++itc) {
+            const int st = itc % p.stages, j = itc & 1;
+            int ok = 1;
+            if (lane == 0) {
+                ok = mbar_wait(&full[st], (itc / p.stages) & 1, p.status, ST_TIMEOUT_FULL) ? 1 : 0;
+                if (ok && itc >= 2)
+                    ok = mbar_wait(&a16_free[j], ((itc >> 1) & 1) ^ 1, p.status, ST_TIMEOUT_EMPTY) ? 1 : 0;
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) { poisoned = 1; break; }
+            const uint8_t *a8 = smem + (size_t)st * stage_bytes;
+            uint8_t *a16 = smem + p.a16_off + (size_t)j * p.mt * kATileBytes;
+            for (int task = cw * 32 + lane; task < p.mt * 512; task += n_conv * 32) {
+                const int trow = task >> 2, c = task & 3, r = trow & 127;
+                uint4 w = *reinterpret_cast<const uint4 *>(a8 + trow * 64 + c * 16);
+                w.x ^= 0x80808080u; w.y ^= 0x80808080u; w.z ^= 0x80808080u; w.w ^= 0x80808080u;
+                const uint4 lo = make_uint4(widen_s8x2<0x4140>(w.x, f16), widen_s8x2<0x4342>(w.x, f16),
+                                            widen_s8x2<0x4140>(w.y, f16), widen_s8x2<0x4342>(w.y, f16));
+                const uint4 hi = make_uint4(widen_s8x2<0x4140>(w.z, f16), widen_s8x2<0x4342>(w.z, f16),
+                                            widen_s8x2<0x4140>(w.w, f16), widen_s8x2<0x4342>(w.w, f16));
+                uint8_t *base = a16 + (trow >> 7) * kATileBytes + (r >> 3) * 1024 + (r & 7) * 128;
+                *reinterpret_cast<uint4 *>(base + (((2 * c) ^ (r & 7)) << 4)) = lo;
+                *reinterpret_cast<uint4 *>(base + (((2 * c + 1) ^ (r & 7)) << 4)) = hi;
+            }
+            fence_proxy_async_smem();      // the tensor core reads the tile through the async proxy
+            __syncwarp();
+            if (lane == 0)
+                mbar_arrive(&conv[j]);
+        }
+        __syncwarp();
+    }
     bool have = false;
     if (is_epi) {
         have = mbar_wait(&accum_bar, 0, p.status, ST_TIMEOUT_MMA);
@@ -313,6 +391,13 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
     float *red = reinterpret_cast<float *>(smem);      // [mt][NB][128] fp32, reuses the ring
 
+    // int8 weights: every accumulator row (= packed weight row) is multiplied by its scale as it leaves TMEM
+    float wsc[2] = {1.f, 1.f};
+    if (p.w8 && is_epi) {
+        wsc[0] = p.wscale[(size_t)(tile * p.mt) * kTcTileM + row];
+        if (p.mt == 2)
+            wsc[1] = p.wscale[(size_t)(tile * p.mt + 1) * kTcTileM + row];
+    }
     // hi- and lo-plane columns are fetched together, one wait for both
     auto load_chunk = [&](int m, int c, float (&v)[16]) {
         if (have) {
@@ -328,7 +413,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             tc_ld_wait(hi, lo);
 #pragma unroll
             for (int i = 0; i < 16; ++i)
-                v[i] = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
+                v[i] = (__uint_as_float(hi[i]) + __uint_as_float(lo[i])) * (m ? wsc[1] : wsc[0]);
         } else {
 #pragma unroll
             for (int i = 0; i < 16; ++i)
@@ -377,12 +462,12 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 const uint32_t a0 = red_row + (uint32_t)((m0 * p.NB + c0 * 16) * kTcTileM) * 4u;
 #pragma unroll
                 for (int i = 0; i < 16; ++i)
-                    sts_f32(a0 + i * (kTcTileM * 4), __uint_as_float(h0[i]) + __uint_as_float(l0[i]));
+                    sts_f32(a0 + i * (kTcTileM * 4), (__uint_as_float(h0[i]) + __uint_as_float(l0[i])) * (m0 ? wsc[1] : wsc[0]));
                 if (two) {
                     const uint32_t a1 = red_row + (uint32_t)((m1 * p.NB + c1 * 16) * kTcTileM) * 4u;
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
-                        sts_f32(a1 + i * (kTcTileM * 4), __uint_as_float(h1[i]) + __uint_as_float(l1[i]));
+                        sts_f32(a1 + i * (kTcTileM * 4), (__uint_as_float(h1[i]) + __uint_as_float(l1[i])) * (m1 ? wsc[1] : wsc[0]));
                 }
             }
             fence_proxy_async_smem();
@@ -662,15 +747,20 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     if (mt == 2)
         p.w_map = *a.w_map256;
     const int tiles = a.N / (kTcTileM * mt);
-    const int stage_bytes = mt * kATileBytes + planes * a.NB * kTcBlockK * 2;
+    // int8 weights: a stage holds the codes (half a 16-bit tile) and the activations; two widened tiles
+    // (mt * 16 KiB each) sit behind the ring
+    const int stage_bytes = mt * (a.w8 ? kATileBytes / 2 : kATileBytes) + planes * a.NB * kTcBlockK * 2;
+    const int a16_bytes = a.w8 ? 2 * mt * kATileBytes : 0;
+    p.w8 = a.w8;
+    p.wscale = a.scales;
     // Ring depth, CTAs per SM and cluster splits.  Two CTAs per SM (rings <= 100 KiB) whenever that
     // leaves >= 4 stages: measured better than one CTA with a ring twice as deep, because the second
     // CTA streams while the first is in its epilogue.  The grid (tiles x splits) must fit the
     // co-resident slots (a second wave doubles the kernel); splits are a power of two <= 8 that leave
     // every rank >= 2 k-blocks.
-    int stages = (200 * 1024) / stage_bytes, per_sm = 1;
-    if ((100 * 1024) / stage_bytes >= 4) {
-        stages = (100 * 1024) / stage_bytes;
+    int stages = (200 * 1024 - a16_bytes) / stage_bytes, per_sm = 1;
+    if ((100 * 1024 - a16_bytes) / stage_bytes >= 4) {
+        stages = (100 * 1024 - a16_bytes) / stage_bytes;
         per_sm = 2;
     }
     if (stages > kTcMaxStages) stages = kTcMaxStages;
@@ -684,7 +774,7 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     const size_t need16 = (size_t)mt * a.NB * kTcTileM * 4 / 16 * 15;
     const bool sixteen = splits == 8 && tiles * 16 <= slots && tiles * 8 * 5 <= sm_count * 3 && p.kblocks / 16 >= 2 &&
                          a.NB % 16 == 0 &&
-                         (size_t)3 * stage_bytes + need16 + 1024 <= (size_t)(per_sm == 2 ? 108 : 225) * 1024;
+                         (size_t)3 * stage_bytes + a16_bytes + need16 + 1024 <= (size_t)(per_sm == 2 ? 108 : 225) * 1024;
     if (sixteen)
         splits = 16;
     p.stages = stages;
@@ -706,8 +796,8 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     p.push = 0;
     if (splits > 1 && splits <= 8 && recv_bytes <= 16 * 1024) {
         int st = stages;
-        while (st > 3 && (size_t)st * stage_bytes + recv_bytes + 1024 > smem_cap) --st;
-        if ((size_t)st * stage_bytes + recv_bytes + 1024 <= smem_cap) {
+        while (st > 3 && (size_t)st * stage_bytes + a16_bytes + recv_bytes + 1024 > smem_cap) --st;
+        if ((size_t)st * stage_bytes + a16_bytes + recv_bytes + 1024 <= smem_cap) {
             stages = st;
             p.stages = st;
             p.push = 1;
@@ -718,16 +808,17 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     if (splits > 1 && !p.push) {
         const size_t need = recv_bytes / splits * (splits - 1);
         int st = stages;
-        while (st > 3 && (size_t)st * stage_bytes + need + 1024 > smem_cap) --st;
-        if ((size_t)st * stage_bytes + need + 1024 <= smem_cap) {
+        while (st > 3 && (size_t)st * stage_bytes + a16_bytes + need + 1024 > smem_cap) --st;
+        if ((size_t)st * stage_bytes + a16_bytes + need + 1024 <= smem_cap) {
             stages = st;
             p.stages = st;
             p.push = 2;
             recv_alloc = need;
         }
     }
-    p.recv_off = stages * stage_bytes;
-    size_t smem = (size_t)stages * stage_bytes + recv_alloc + 1024;
+    p.a16_off = stages * stage_bytes;
+    p.recv_off = stages * stage_bytes + a16_bytes;
+    size_t smem = (size_t)stages * stage_bytes + a16_bytes + recv_alloc + 1024;
     const size_t red_bytes = (size_t)mt * a.NB * kTcTileM * 4 + 1024;
     if (smem < red_bytes) smem = red_bytes;
     cudaLaunchConfig_t cfg = {};
@@ -737,6 +828,8 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     const int epi_warps = (per_sm == 1 && mt * (a.NB / splits) / 2 >= 8) ? 16 : 8;
     p.epi_warps = epi_warps;
     p.producers = stages < kTcMaxProducers ? stages : kTcMaxProducers;
+    if (a.w8 && (!a.scales || epi_warps - (p.producers - 1) < 1))
+        return cudaErrorInvalidValue;
     cfg.blockDim = dim3((2 + epi_warps) * 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;

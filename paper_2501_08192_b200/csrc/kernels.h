@@ -139,6 +139,9 @@ cudaError_t launch_pack_rows(const void *const *srcs, const int *src_cols, int n
 // 1 KiB tiles of 16 rows x 64 k, scales [N] in packed row order.
 cudaError_t launch_pack_gemv_w8(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
                                 void *dst_codes, float *dst_scales, cudaStream_t s);
+// the same codes and scales for the tensor path: [N, K] K-major rows of int8 in the tensor path's row order
+cudaError_t launch_pack_rows_w8(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
+                                void *dst_codes, float *dst_scales, cudaStream_t s);
 
 // ---- split-K GEMV (batch < 16): y[b,n] = sum_k x[b,k] W[n,k]; W in fragment-major tiles
 struct GemvArgs {
@@ -173,6 +176,11 @@ struct GemmTcArgs {
     long long *trace;
     int pdl;
     int inject;
+    // int8 weights: w_map / w_map256 are uint8 maps over the codes (dims (K, N), box (64, 128 or 256), no
+    // swizzle); the kernel widens every tile to the activations' 16-bit format in shared memory before
+    // the MMA and multiplies every accumulator row by its scale
+    int w8;
+    const float *scales;  // w8: [N] in packed row order
 };
 cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s);
 

@@ -84,11 +84,12 @@ static cudaError_t launch_pack(bool tensor, const void *const *srcs, const int *
     return cudaGetLastError();
 }
 
-// ---- int8 weights (GEMV path)
+// ---- int8 weights (GEMV path: fragment-major tiles; tensor path: [N, K] K-major rows of codes)
 struct PackW8Params {
     const bf16 *src[3];
     int cols[3];
     int N, K, kind;
+    int tensor;       // tensor-path row order and layout
     int8_t *codes;
     float *scales;
 };
@@ -100,7 +101,7 @@ __global__ void k_w8_scales(const __grid_constant__ PackW8Params p)
     if (row >= p.N)
         return;
     int src, col;
-    packed_row_source(p.kind, false, row, p.cols, src, col);
+    packed_row_source(p.kind, p.tensor != 0, row, p.cols, src, col);
     float mx = 0.f;
     for (int k = 0; k < p.K; ++k)
         mx = fmaxf(mx, fabsf(__bfloat162float(p.src[src][(size_t)k * p.cols[src] + col])));
@@ -116,20 +117,25 @@ __global__ void k_pack_w8(const __grid_constant__ PackW8Params p)
     const int row = (int)(idx % p.N);
     const int k = (int)(idx / p.N);
     int src, col;
-    packed_row_source(p.kind, false, row, p.cols, src, col);
+    packed_row_source(p.kind, p.tensor != 0, row, p.cols, src, col);
     const float v = __bfloat162float(p.src[src][(size_t)k * p.cols[src] + col]);
     const float sc = p.scales[row];
     // the code is decided in fp32: one correctly rounded division, round to nearest even, clamp
     float r = sc > 0.f ? rintf(__fdiv_rn(v, sc)) : 0.f;
     r = fminf(fmaxf(r, -127.f), 127.f);
-    const int rb = row >> 4, rr = row & 15, g = rr & 7, hi = rr >> 3;
-    const int kc = k >> 6, t = (k & 63) >> 4, e = k & 15;
-    const size_t o = ((size_t)rb * (p.K >> 6) + kc) * 1024 + (size_t)(g * 4 + t) * 32 + hi * 16 + e;
+    size_t o;
+    if (p.tensor) {
+        o = (size_t)row * p.K + k;
+    } else {
+        const int rb = row >> 4, rr = row & 15, g = rr & 7, hi = rr >> 3;
+        const int kc = k >> 6, t = (k & 63) >> 4, e = k & 15;
+        o = ((size_t)rb * (p.K >> 6) + kc) * 1024 + (size_t)(g * 4 + t) * 32 + hi * 16 + e;
+    }
     p.codes[o] = (int8_t)(int)r;
 }
 
-cudaError_t launch_pack_gemv_w8(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
-                                void *dst_codes, float *dst_scales, cudaStream_t s)
+static cudaError_t launch_pack_w8(bool tensor, const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
+                                  void *dst_codes, float *dst_scales, cudaStream_t s)
 {
     if (K % 64)
         return cudaErrorInvalidValue;
@@ -141,12 +147,24 @@ cudaError_t launch_pack_gemv_w8(const void *const *srcs, const int *src_cols, in
         N += src_cols[i];
     }
     p.N = N; p.K = K; p.kind = kind;
+    p.tensor = tensor ? 1 : 0;
     p.codes = reinterpret_cast<int8_t *>(dst_codes);
     p.scales = dst_scales;
     k_w8_scales<<<(N + 127) / 128, 128, 0, s>>>(p);
     const size_t total = (size_t)N * K;
     k_pack_w8<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(p);
     return cudaGetLastError();
+}
+
+cudaError_t launch_pack_gemv_w8(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
+                                void *dst_codes, float *dst_scales, cudaStream_t s)
+{
+    return launch_pack_w8(false, srcs, src_cols, n_srcs, K, kind, dst_codes, dst_scales, s);
+}
+cudaError_t launch_pack_rows_w8(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
+                                void *dst_codes, float *dst_scales, cudaStream_t s)
+{
+    return launch_pack_w8(true, srcs, src_cols, n_srcs, K, kind, dst_codes, dst_scales, s);
 }
 
 cudaError_t launch_pack_gemv(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind, void *dst,

@@ -102,6 +102,7 @@ def test_int8_cache_on_benchmark_configs(oracle, idx):
 def test_int8_cache_with_int8_weights(oracle):
     kv8_check(oracle, I.small_shape(name="kv8_w8_b5", batch=5, ctx=127, seed=242), flags=P.FLAG_INT8_WEIGHTS)
     kv8_check(oracle, I.CONFIGS[1], flags=P.FLAG_INT8_WEIGHTS)
+    kv8_check(oracle, I.small_shape(name="kv8_w8_b24", batch=24, ctx=127, seed=243), flags=P.FLAG_INT8_WEIGHTS)   # tensor path
 
 
 def test_int8_cache_groups_above_eight_are_refused():

@@ -99,17 +99,24 @@ W8_SHAPES = [
     I.small_shape(name="w8_wide_ffn_b8", batch=8, hidden=256, ffn=5120, ctx=70, seed=148),
     I.small_shape(name="w8_h384_b7", batch=7, hidden=384, ffn=192, ctx=33, seed=149),
     I.small_shape(name="w8_h2048_b3", batch=3, hidden=2048, ffn=256, ctx=40, tp_degree=5, seed=150),
+    # tensor path: the int8 tiles are widened in shared memory in front of the tcgen05 MMA
+    I.small_shape(name="w8_b16", batch=16, ctx=100, seed=115),
+    I.small_shape(name="w8_b33_ragged_g8", batch=33, ctx=300, ctx_min=1, n_q_heads=8, n_kv_heads=1, tp_degree=3, seed=116),
+    I.small_shape(name="w8_b64", batch=64, hidden=1024, ffn=1152, ctx=64, seed=117),
+    I.small_shape(name="w8_b128", batch=128, hidden=256, ffn=128, ctx=20, n_q_heads=2, n_kv_heads=2, seed=144),
+    I.small_shape(name="w8_h8192_b40", batch=40, hidden=8192, ffn=256, ctx=50, ctx_min=3, n_q_heads=2, n_kv_heads=2,
+                  tp_degree=3, seed=157),
 ]
 
 
 @pytest.mark.parametrize("shape", W8_SHAPES, ids=[s.name for s in W8_SHAPES])
 def test_int8_weights_match_the_quantised_oracle(oracle, shape):
-    """int8 weights (per-output-channel scales) on the split-K GEMV path against the oracle that
-    quantises the same way: every intermediate and output, same tolerance."""
+    """int8 weights (per-output-channel scales) on the split-K GEMV path and on the tcgen05 path against
+    the oracle that quantises the same way: every intermediate and output, same tolerance."""
     full_check(oracle, shape, flags=P.FLAG_INT8_WEIGHTS)
 
 
-@pytest.mark.parametrize("idx", [0, 1])
+@pytest.mark.parametrize("idx", [0, 1, 3, 4])
 def test_int8_weights_on_benchmark_configs(oracle, idx):
     bits = full_check(oracle, I.CONFIGS[idx], flags=P.FLAG_INT8_WEIGHTS, budget=16 << 20)
     again = full_check(oracle, I.CONFIGS[idx], flags=P.FLAG_INT8_WEIGHTS, budget=0)
@@ -117,19 +124,21 @@ def test_int8_weights_on_benchmark_configs(oracle, idx):
         assert np.array_equal(bits[k], again[k]), k          # prefetch never changes results, int8 included
 
 
-def test_int8_weights_are_refused_where_no_kernel_has_them():
-    t = I.make_layers(I.small_shape(batch=20), 1)[0]
+def test_int8_weights_on_either_path_report_one_byte_per_weight():
+    for flags, tensor in ((P.FLAG_INT8_WEIGHTS, 1), (P.FLAG_INT8_WEIGHTS | P.FLAG_FORCE_GEMV, 0)):
+        s = I.small_shape(batch=20, ctx=50, seed=151)
+        dl = G.DeviceLayer(s, I.make_layers(s, 1)[0], flags=flags)
+        try:
+            info = dl.layer.get_info()
+            assert info.uses_tensor_path == tensor
+            assert list(info.weight_bytes) == [512 * 1024, 512 * 512, 512 * 768, 384 * 512]   # one byte per weight
+        finally:
+            dl.close()
+    # the GEMV path's int8 tiles cover 64 k: an ffn that is not a multiple of 64 is refused
+    s = I.small_shape(batch=2, ffn=96, ctx=10)
     with pytest.raises(P.PreserveError) as e:
-        G.DeviceLayer(I.small_shape(batch=20), t, flags=P.FLAG_INT8_WEIGHTS)         # tensor path
+        G.DeviceLayer(s, I.make_layers(s, 1)[0], flags=P.FLAG_INT8_WEIGHTS)
     assert e.value.code == P.PRESERVE_ESHAPE
-    s = I.small_shape(batch=20, ctx=50, seed=151)
-    dl = G.DeviceLayer(s, I.make_layers(s, 1)[0], flags=P.FLAG_INT8_WEIGHTS | P.FLAG_FORCE_GEMV)
-    try:
-        info = dl.layer.get_info()
-        assert info.uses_tensor_path == 0
-        assert list(info.weight_bytes) == [512 * 1024, 512 * 512, 512 * 768, 384 * 512]   # one byte per weight
-    finally:
-        dl.close()
 
 
 def test_config3_chain_of_four_matches_oracle(oracle):
