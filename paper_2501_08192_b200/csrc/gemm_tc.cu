@@ -151,7 +151,7 @@ __device__ __forceinline__ void tc_ld_wait(uint32_t (&a)[16], uint32_t (&b)[16])
 
 // KIND: the epilogue; PUSH: the split-K hand-over (0 pull, 1 st.async, 2 bulk copies) - template
 // arguments, so that each instantiation carries a single tail and its instructions stay close together.
-template <int KIND, int PUSH>
+template <int KIND, int PUSH, bool W8 = false>
 __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_constant__ GemmTcParams p)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -165,7 +165,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile = blockIdx.x;
     const int s = blockIdx.y;
-    const int a_bytes = p.mt * (p.w8 ? kATileBytes / 2 : kATileBytes);
+    const int a_bytes = p.mt * (W8 ? kATileBytes / 2 : kATileBytes);
     const int stage_bytes = a_bytes + p.planes * p.NB * kTcBlockK * 2;
     const int acc_cols = p.planes * p.NB;      // TMEM columns of one weight tile's accumulator
     const int kb0 = (int)((long long)p.kblocks * s / p.splits);
@@ -180,7 +180,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             mbar_init(&empty[i], 1);
         }
         mbar_init(&accum_bar, 1);
-        if (p.w8) {
+        if (W8) {
             // the epilogue warps that issue no TMA loads widen the tiles: one arrival per warp and tile
             for (int j = 0; j < 2; ++j) {
                 mbar_init(&conv[j], p.epi_warps - (p.producers - 1));
@@ -261,11 +261,11 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 const uint32_t ph = (it / p.stages) & 1;
                 // (int8 weights: the widened tile of this use, slot it % 2, completes after the stage has landed)
                 const int j = it & 1;
-                if (!(p.w8 ? mbar_wait(&conv[j], (it >> 1) & 1, p.status, ST_TIMEOUT_FULL)
+                if (!(W8 ? mbar_wait(&conv[j], (it >> 1) & 1, p.status, ST_TIMEOUT_FULL)
                            : mbar_wait(&full[st], ph, p.status, ST_TIMEOUT_FULL))) { poisoned = 1; ok = false; break; }
                 tc_fence_after();
                 const uint32_t st_addr = smem_u32(smem + (size_t)st * stage_bytes);
-                const uint32_t a_addr = p.w8 ? smem_u32(smem + p.a16_off + (size_t)j * p.mt * kATileBytes) : st_addr;
+                const uint32_t a_addr = W8 ? smem_u32(smem + p.a16_off + (size_t)j * p.mt * kATileBytes) : st_addr;
                 const uint64_t bdesc = make_smem_desc(st_addr + a_bytes);
                 for (int m = 0; m < p.mt; ++m) {
                     // each 128-row weight tile has its own accumulator (2 * NB TMEM columns)
@@ -276,7 +276,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                                (kb > kb0 || k > 0) ? 1u : 0u);
                 }
                 tc_commit(&empty[st]);      // slot is free once these MMAs have read it
-                if (p.w8)
+                if (W8)
                     tc_commit(&a16_free[j]);
             }
             if (ok)
@@ -340,7 +340,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             run_producer(warp - 1);
         __syncwarp();
     }
-    else if (is_epi && p.w8) {
+    else if (is_epi && W8) {
         // ---------------------------------------------------- int8 weights: widen every tile
         // Tile use `itc` is converted from its ring stage into widened slot itc % 2 (the MMA operand
         // layout: K-major rows, 8-row atoms of 1 KiB, 128-byte swizzle).  A task = 16 codes of one
@@ -393,11 +393,17 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
 
     // int8 weights: every accumulator row (= packed weight row) is multiplied by its scale as it leaves TMEM
     float wsc[2] = {1.f, 1.f};
-    if (p.w8 && is_epi) {
+    if (W8 && is_epi) {
         wsc[0] = p.wscale[(size_t)(tile * p.mt) * kTcTileM + row];
         if (p.mt == 2)
             wsc[1] = p.wscale[(size_t)(tile * p.mt + 1) * kTcTileM + row];
     }
+    auto wscale_of = [&](int m) -> float {
+        if constexpr (W8)
+            return m ? wsc[1] : wsc[0];
+        else
+            return 1.f;
+    };
     // hi- and lo-plane columns are fetched together, one wait for both
     auto load_chunk = [&](int m, int c, float (&v)[16]) {
         if (have) {
@@ -413,7 +419,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             tc_ld_wait(hi, lo);
 #pragma unroll
             for (int i = 0; i < 16; ++i)
-                v[i] = (__uint_as_float(hi[i]) + __uint_as_float(lo[i])) * (m ? wsc[1] : wsc[0]);
+                v[i] = (__uint_as_float(hi[i]) + __uint_as_float(lo[i])) * wscale_of(m);
         } else {
 #pragma unroll
             for (int i = 0; i < 16; ++i)
@@ -462,12 +468,12 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 const uint32_t a0 = red_row + (uint32_t)((m0 * p.NB + c0 * 16) * kTcTileM) * 4u;
 #pragma unroll
                 for (int i = 0; i < 16; ++i)
-                    sts_f32(a0 + i * (kTcTileM * 4), (__uint_as_float(h0[i]) + __uint_as_float(l0[i])) * (m0 ? wsc[1] : wsc[0]));
+                    sts_f32(a0 + i * (kTcTileM * 4), (__uint_as_float(h0[i]) + __uint_as_float(l0[i])) * wscale_of(m0));
                 if (two) {
                     const uint32_t a1 = red_row + (uint32_t)((m1 * p.NB + c1 * 16) * kTcTileM) * 4u;
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
-                        sts_f32(a1 + i * (kTcTileM * 4), (__uint_as_float(h1[i]) + __uint_as_float(l1[i])) * (m1 ? wsc[1] : wsc[0]));
+                        sts_f32(a1 + i * (kTcTileM * 4), (__uint_as_float(h1[i]) + __uint_as_float(l1[i])) * wscale_of(m1));
                 }
             }
             fence_proxy_async_smem();
@@ -703,11 +709,11 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     trace_end(p.trace);
 }
 
-template <int KIND, int PUSH>
+template <int KIND, int PUSH, bool W8 = false>
 static cudaError_t launch_instance(cudaLaunchConfig_t &cfg, const GemmTcParams &p, size_t smem)
 {
     static PerDeviceSize smem_limit, np_set;      // per instantiation and device
-    cudaError_t e = ensure_dynamic_smem(k_gemm_tcgen05<KIND, PUSH>, smem_limit, smem);
+    cudaError_t e = ensure_dynamic_smem(k_gemm_tcgen05<KIND, PUSH, W8>, smem_limit, smem);
     if (e != cudaSuccess)
         return e;
     if (p.splits > 8) {
@@ -715,13 +721,13 @@ static cudaError_t launch_instance(cudaLaunchConfig_t &cfg, const GemmTcParams &
         if (dev < 0)
             return cudaErrorInvalidDevice;
         if (!np_set.v[dev]) {
-            e = cudaFuncSetAttribute(k_gemm_tcgen05<KIND, PUSH>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            e = cudaFuncSetAttribute(k_gemm_tcgen05<KIND, PUSH, W8>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
             if (e != cudaSuccess)
                 return e;
             np_set.v[dev] = 1;
         }
     }
-    return cudaLaunchKernelEx(&cfg, k_gemm_tcgen05<KIND, PUSH>, p);
+    return cudaLaunchKernelEx(&cfg, k_gemm_tcgen05<KIND, PUSH, W8>, p);
 }
 
 cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
@@ -847,7 +853,7 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     const int push = splits > 1 ? p.push : 0;
 #define PRSV_TC_CASE(KIND, PUSH)                                   \
     if (a.epi.kind == (KIND) && push == (PUSH))                    \
-        return launch_instance<KIND, PUSH>(cfg, p, smem);
+        return a.w8 ? launch_instance<KIND, PUSH, true>(cfg, p, smem) : launch_instance<KIND, PUSH, false>(cfg, p, smem);
     PRSV_TC_CASE(EPI_PLAIN, 0) PRSV_TC_CASE(EPI_PLAIN, 1) PRSV_TC_CASE(EPI_PLAIN, 2)
     PRSV_TC_CASE(EPI_QKV, 0) PRSV_TC_CASE(EPI_QKV, 1) PRSV_TC_CASE(EPI_QKV, 2)
     PRSV_TC_CASE(EPI_SWIGLU, 0) PRSV_TC_CASE(EPI_SWIGLU, 1) PRSV_TC_CASE(EPI_SWIGLU, 2)
