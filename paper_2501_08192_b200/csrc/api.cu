@@ -53,10 +53,8 @@ bool make_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// 2-D uint8 tensor map: `rows` rows of `cols` contiguous bytes, box (box_cols x box_rows), 128-byte swizzle
-// (or none: the box then lands as dense rows of box_cols bytes).
-bool make_u8_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_cols, uint32_t box_rows,
-                    bool swizzle = true)
+// 2-D uint8 tensor map: `rows` rows of `cols` contiguous bytes, box (box_cols x box_rows), 128-byte swizzle.
+bool make_u8_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint32_t box_cols, uint32_t box_rows)
 {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn)
@@ -66,8 +64,7 @@ bool make_u8_map_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t ro
     cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -383,7 +380,7 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
 {
     const Dims d = layer_dims(L->cfg);
     if (L->tensor_path) {
-        GemmTcArgs a;
+        GemmTcArgs a = {};
         a.w_map = L->wmap[which];
         a.w_map256 = L->has256[which] ? &L->wmap256[which] : nullptr;
         a.x_map = L->xmap[which];
@@ -402,6 +399,7 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
         a.x_fp16 = which == 2 ? 1 : 0;
         a.w8 = L->w8 ? 1 : 0;
         a.scales = L->w8 ? L->scales + L->soff[which] : nullptr;
+        a.w8_codes = L->w8 ? L->arena + L->off[which] : nullptr;
         CK(L, launch_gemm_tc(a, L->sm_count, s));
         return PRESERVE_OK;
     }
@@ -1103,11 +1101,19 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
                 so += (size_t)d.n[i];
             }
             CKI(cudaMalloc(&L->scales, so * sizeof(float)));
-            auto pack8 = L->tensor_path ? launch_pack_rows_w8 : launch_pack_gemv_w8;
-            CKI(pack8(s_qkv, c_qkv, 3, d.k[0], EPI_QKV, L->arena + L->off[0], L->scales + L->soff[0], nullptr));
-            CKI(pack8(s_o, c_o, 1, d.k[1], EPI_PLAIN, L->arena + L->off[1], L->scales + L->soff[1], nullptr));
-            CKI(pack8(s_gu, c_gu, 2, d.k[2], EPI_SWIGLU, L->arena + L->off[2], L->scales + L->soff[2], nullptr));
-            CKI(pack8(s_dn, c_dn, 1, d.k[3], EPI_PLAIN, L->arena + L->off[3], L->scales + L->soff[3], nullptr));
+            // (tensor path: blocks of one or two 128-row tiles, as the GEMM will take them per CTA)
+            const int nbp = ((c.max_batch + 15) / 16) * 16;
+            auto pack8 = [&](const void *const *srcs, const int *cols, int n, int i, int kind) -> cudaError_t {
+                return L->tensor_path ? launch_pack_rows_w8(srcs, cols, n, d.k[i], kind, L->arena + L->off[i],
+                                                            L->scales + L->soff[i], gemm_tc_w8_tiles(nbp, d.n[i], i == 2),
+                                                            nullptr)
+                                      : launch_pack_gemv_w8(srcs, cols, n, d.k[i], kind, L->arena + L->off[i],
+                                                            L->scales + L->soff[i], nullptr);
+            };
+            CKI(pack8(s_qkv, c_qkv, 3, 0, EPI_QKV));
+            CKI(pack8(s_o, c_o, 1, 1, EPI_PLAIN));
+            CKI(pack8(s_gu, c_gu, 2, 2, EPI_SWIGLU));
+            CKI(pack8(s_dn, c_dn, 1, 3, EPI_PLAIN));
         } else {
             auto pack = L->tensor_path ? launch_pack_rows : launch_pack_gemv;
             // (tensor path: Wgate|up meets the fp16 RMSNorm output x2 and is stored as fp16)
@@ -1171,16 +1177,14 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
         for (int i = 0; i < 4; ++i) {
             // x2 (the MLP's RMSNorm output) is one fp16 plane; x, o and a are two bf16 planes (hi rows, lo rows)
             const uint32_t brows = (uint32_t)(i == 2 ? L->nb_pad : 2 * L->nb_pad);
-            // (int8 weights: rows of codes, fetched as dense [rows][64] byte tiles for the widening stage)
-            const bool wok = L->w8 ? make_u8_map_2d(&L->wmap[i], L->arena + L->off[i], d.k[i], d.n[i], 64, 128, false)
-                                   : make_map_2d(&L->wmap[i], L->arena + L->off[i], d.k[i], d.n[i], 64, 128);
+            // (int8 weights are fetched by plain bulk copies: no map over them)
+            const bool wok = L->w8 || make_map_2d(&L->wmap[i], L->arena + L->off[i], d.k[i], d.n[i], 64, 128);
             if (!wok || !make_map_2d(&L->xmap[i], xb[i], d.k[i], brows, 64, brows)) {
                 preserve_layer_destroy(L);
                 return PRESERVE_EARCH;
             }
-            L->has256[i] = d.n[i] % 256 == 0 &&
-                           (L->w8 ? make_u8_map_2d(&L->wmap256[i], L->arena + L->off[i], d.k[i], d.n[i], 64, 256, false)
-                                  : make_map_2d(&L->wmap256[i], L->arena + L->off[i], d.k[i], d.n[i], 64, 256));
+            L->has256[i] = !L->w8 && d.n[i] % 256 == 0 &&
+                           make_map_2d(&L->wmap256[i], L->arena + L->off[i], d.k[i], d.n[i], 64, 256);
         }
     }
     if ((c.flags & PRESERVE_FLAG_PERSIST_L2) && L->max_persist > 0) {

@@ -39,6 +39,7 @@ namespace cg = cooperative_groups;
 namespace prsv {
 
 constexpr int kTcMaxStages = 12;
+constexpr int kTcMaxW8Slots = 4;          // int8 weights: widened operand tiles behind the ring
 constexpr int kTcMaxEpiWarps = 16;        // 2-4 per TMEM lane group: the epilogue is a chain of short dependent
                                           // operations per output, so its speed is set by how many warps run it
 constexpr int kTcMaxProducers = 3;        // issuing threads of the TMA ring: warp 0, and lane 0 of the first epilogue warps
@@ -68,20 +69,23 @@ struct GemmTcParams {
     int epi_warps;      // 8 or 16
     int producers;      // 1..kTcMaxProducers threads that issue the ring's TMA loads (stage uses dealt round-robin)
     int w8;             // the weight tiles arrive as int8 codes ([rows][64] bytes, no swizzle) and are widened in shared memory
-    int a16_off;        // w8: offset of the two widened weight tiles (mt * 16 KiB each) behind the ring
+    int a16_off;        // w8: offset of the widened weight tiles (w8_slots of mt * 16 KiB each) behind the ring
+    int w8_slots;       // 2..kTcMaxW8Slots
     const float *wscale;  // w8: one fp32 scale per packed weight row
+    const uint8_t *w8_codes;  // w8: the codes, one contiguous block of mt * 128 rows x 64 bytes per (tile, k-block)
 };
 
-// int8 -> 16-bit widening of two codes of `biased` (the loaded word with every byte's top bit flipped:
-// code + 128 as an unsigned byte), exact.  SEL places the bytes: 0x4140 = bytes (0, 1), 0x4342 = (2, 3).
-// fp16: the byte lands in the mantissa of 1024.0, i.e. 1152 + code; subtract 1152.
-// bf16 (7 mantissa bits): the low seven bits land in the mantissa of 128.0, i.e. 128 + (byte & 127); subtract
-// 128 when the byte's top bit is set (code >= 0), 256 when it is not.
-template <uint32_t SEL>
-__device__ __forceinline__ uint32_t widen_s8x2(uint32_t biased, bool fp16)
+// int8 -> 16-bit widening of two weight codes, exact.  The packed matrix holds every code biased by
+// 128 (an unsigned byte), so no sign handling is left for the kernel.  SEL places the bytes: 0x4140 =
+// bytes (0, 1) of the word, 0x4342 = bytes (2, 3).
+// fp16: the byte lands in the mantissa of 1024.0, i.e. the number 1152 + code; subtract 1152.
+// bf16 (7 mantissa bits): the low seven bits land in the mantissa of 128.0, i.e. 128 + (byte & 127);
+// subtract 128 when the byte's top bit is set (code >= 0), 256 when it is not.
+template <uint32_t SEL, bool F16>
+__device__ __forceinline__ uint32_t widen_u8x2(uint32_t biased)
 {
     uint32_t r;
-    if (fp16) {
+    if constexpr (F16) {
         r = __byte_perm(biased, 0x64646464u, SEL);
         const uint32_t off = 0x64806480u;      // (1152.0, 1152.0)
         asm("sub.f16x2 %0, %0, %1;" : "+r"(r) : "r"(off));
@@ -91,6 +95,24 @@ __device__ __forceinline__ uint32_t widen_s8x2(uint32_t biased, bool fp16)
         asm("sub.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(minuend), "r"(subtrahend));
     }
     return r;
+}
+// One widening pass of a converter thread over a tile: `n` tasks of 16 codes (one 16-byte load, two
+// 16-byte stores); consecutive tasks of a thread are `src_step` / `dst_step` bytes apart.
+template <bool F16>
+__device__ __forceinline__ void widen_tile(const uint8_t *src, uint8_t *dst, uint32_t off_lo, uint32_t off_hi, int n,
+                                           uint32_t src_step, uint32_t dst_step)
+{
+    for (int i = 0; i < n; ++i) {
+        const uint4 w = *reinterpret_cast<const uint4 *>(src);
+        const uint4 lo = make_uint4(widen_u8x2<0x4140, F16>(w.x), widen_u8x2<0x4342, F16>(w.x),
+                                    widen_u8x2<0x4140, F16>(w.y), widen_u8x2<0x4342, F16>(w.y));
+        const uint4 hi = make_uint4(widen_u8x2<0x4140, F16>(w.z), widen_u8x2<0x4342, F16>(w.z),
+                                    widen_u8x2<0x4140, F16>(w.w), widen_u8x2<0x4342, F16>(w.w));
+        *reinterpret_cast<uint4 *>(dst + off_lo) = lo;
+        *reinterpret_cast<uint4 *>(dst + off_hi) = hi;
+        src += src_step;
+        dst += dst_step;
+    }
 }
 
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr)
@@ -157,7 +179,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ uint64_t full[kTcMaxStages], empty[kTcMaxStages], accum_bar, push_bar;
-    __shared__ uint64_t conv[2], a16_free[2];      // int8 weights: a widened tile is complete / has been consumed
+    __shared__ uint64_t conv[kTcMaxW8Slots], a16_free[kTcMaxW8Slots];   // int8 weights: a widened tile is complete / has been consumed
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile int poisoned;
     __shared__ EpilogueTables tabs;
@@ -182,14 +204,15 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         mbar_init(&accum_bar, 1);
         if (W8) {
             // the epilogue warps that issue no TMA loads widen the tiles: one arrival per warp and tile
-            for (int j = 0; j < 2; ++j) {
+            for (int j = 0; j < p.w8_slots; ++j) {
                 mbar_init(&conv[j], p.epi_warps - (p.producers - 1));
                 mbar_init(&a16_free[j], 1);
             }
         }
         mbar_fence_init();
         poisoned = 0;
-        tma_prefetch_desc(&p.w_map);
+        if (!W8)
+            tma_prefetch_desc(&p.w_map);
         tma_prefetch_desc(&p.x_map);
     }
     if (warp == 1) {
@@ -226,8 +249,12 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             mbar_expect_tx(&full[i], stage_bytes);
             if (p.inject == INJECT_TC_RING && i == 0 && tile == 0 && s == 0)
                 continue;
-            tma_load_2d_hint(smem + (size_t)i * stage_bytes, &p.w_map, (kb0 + i) * kTcBlockK,
-                             tile * p.mt * kTcTileM, &full[i], pol);
+            if constexpr (W8)
+                bulk_load_hint(smem + (size_t)i * stage_bytes, p.w8_codes + ((size_t)tile * p.kblocks + kb0 + i) * a_bytes,
+                               a_bytes, &full[i], pol);
+            else
+                tma_load_2d_hint(smem + (size_t)i * stage_bytes, &p.w_map, (kb0 + i) * kTcBlockK,
+                                 tile * p.mt * kTcTileM, &full[i], pol);
         }
         pdl_wait();
         if (prod == 0)
@@ -237,15 +264,24 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         int it = prod;
         while (it < pre)
             it += NP;
+        // (stage and phase of use `it` are kept incrementally: no division on this thread's path)
+        int st = it % p.stages;
+        uint32_t ph = (uint32_t)(it / p.stages) & 1;
         for (; it < n_kb; it += NP) {
             const int kb = kb0 + it;
-            const int st = it % p.stages;
-            const uint32_t ph = (uint32_t)(it / p.stages) & 1;
             if (!mbar_wait(&empty[st], ph ^ 1, p.status, ST_TIMEOUT_EMPTY)) { poisoned = 1; break; }
             uint8_t *a_dst = smem + (size_t)st * stage_bytes;
             mbar_expect_tx(&full[st], stage_bytes);
-            tma_load_2d_hint(a_dst, &p.w_map, kb * kTcBlockK, tile * p.mt * kTcTileM, &full[st], pol);
+            if constexpr (W8)
+                bulk_load_hint(a_dst, p.w8_codes + ((size_t)tile * p.kblocks + kb) * a_bytes, a_bytes, &full[st], pol);
+            else
+                tma_load_2d_hint(a_dst, &p.w_map, kb * kTcBlockK, tile * p.mt * kTcTileM, &full[st], pol);
             tma_load_2d(a_dst + a_bytes, &p.x_map, kb * kTcBlockK, 0, &full[st]);
+            st += NP;
+            while (st >= p.stages) {
+                st -= p.stages;
+                ph ^= 1;
+            }
         }
     };
     if (warp == 0) {
@@ -254,14 +290,12 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            uint32_t it = 0;
             bool ok = true;
-            for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                const int st = it % p.stages;
-                const uint32_t ph = (it / p.stages) & 1;
-                // (int8 weights: the widened tile of this use, slot it % 2, completes after the stage has landed)
-                const int j = it & 1;
-                if (!(W8 ? mbar_wait(&conv[j], (it >> 1) & 1, p.status, ST_TIMEOUT_FULL)
+            int st = 0, j = 0;               // ring stage and (int8 weights) widened slot of this use, with their phases
+            uint32_t ph = 0, phj = 0;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                // (int8 weights: the widened tile of this use completes after the stage has landed)
+                if (!(W8 ? mbar_wait(&conv[j], phj, p.status, ST_TIMEOUT_FULL)
                            : mbar_wait(&full[st], ph, p.status, ST_TIMEOUT_FULL))) { poisoned = 1; ok = false; break; }
                 tc_fence_after();
                 const uint32_t st_addr = smem_u32(smem + (size_t)st * stage_bytes);
@@ -276,8 +310,11 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                                (kb > kb0 || k > 0) ? 1u : 0u);
                 }
                 tc_commit(&empty[st]);      // slot is free once these MMAs have read it
-                if (W8)
+                if (W8) {
                     tc_commit(&a16_free[j]);
+                    if (++j == p.w8_slots) { j = 0; phj ^= 1; }
+                }
+                if (++st == p.stages) { st = 0; ph ^= 1; }
             }
             if (ok)
                 tc_commit(&accum_bar);      // accumulator complete
@@ -342,41 +379,44 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     }
     else if (is_epi && W8) {
         // ---------------------------------------------------- int8 weights: widen every tile
-        // Tile use `itc` is converted from its ring stage into widened slot itc % 2 (the MMA operand
+        // Tile use `itc` is converted from its ring stage into widened slot itc % slots (the MMA operand
         // layout: K-major rows, 8-row atoms of 1 KiB, 128-byte swizzle).  A task = 16 codes of one
         // row (one 16-byte load, two 16-byte stores).  The slot is written again only after the MMAs
-        // of use itc - 2 have read it.
+        // of use itc - slots have read it.
+        // A thread's tasks are 8 * n_conv rows apart: the same 16-byte column and the same row within
+        // an 8-row swizzle atom every time, so everything but two base pointers is fixed per thread.
         const int cw = warp - 1 - p.producers, n_conv = p.epi_warps - (p.producers - 1);
         const bool f16 = p.planes == 1;
-        uint32_t itc = 0;
-        for (int kb = kb0; kb < kb1; ++kb, ++itc) {
-            const int st = itc % p.stages, j = itc & 1;
+        const int task0 = cw * 32 + lane, trow0 = task0 >> 2, c = task0 & 3;
+        const int n_tasks = (p.mt * 512 - task0 + n_conv * 32 - 1) / (n_conv * 32);
+        const uint32_t src_off = (uint32_t)trow0 * 64 + c * 16;
+        const uint32_t dst_off = (uint32_t)(trow0 >> 3) * 1024 + (trow0 & 7) * 128;   // (m-tiles are 16 atoms apart: contiguous)
+        const uint32_t off_lo = (uint32_t)((2 * c) ^ (trow0 & 7)) << 4, off_hi = (uint32_t)((2 * c + 1) ^ (trow0 & 7)) << 4;
+        const uint32_t src_step = (uint32_t)n_conv * 8 * 64, dst_step = (uint32_t)n_conv * 1024;
+        int st = 0, j = 0;
+        uint32_t ph = 0, phj = 0;
+        bool reuse = false;          // the slot has been used before: wait until the MMAs of that use are done
+        for (int kb = kb0; kb < kb1; ++kb) {
             int ok = 1;
             if (lane == 0) {
-                ok = mbar_wait(&full[st], (itc / p.stages) & 1, p.status, ST_TIMEOUT_FULL) ? 1 : 0;
-                if (ok && itc >= 2)
-                    ok = mbar_wait(&a16_free[j], ((itc >> 1) & 1) ^ 1, p.status, ST_TIMEOUT_EMPTY) ? 1 : 0;
+                ok = mbar_wait(&full[st], ph, p.status, ST_TIMEOUT_FULL) ? 1 : 0;
+                if (ok && reuse)
+                    ok = mbar_wait(&a16_free[j], phj ^ 1, p.status, ST_TIMEOUT_EMPTY) ? 1 : 0;
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) { poisoned = 1; break; }
-            const uint8_t *a8 = smem + (size_t)st * stage_bytes;
-            uint8_t *a16 = smem + p.a16_off + (size_t)j * p.mt * kATileBytes;
-            for (int task = cw * 32 + lane; task < p.mt * 512; task += n_conv * 32) {
-                const int trow = task >> 2, c = task & 3, r = trow & 127;
-                uint4 w = *reinterpret_cast<const uint4 *>(a8 + trow * 64 + c * 16);
-                w.x ^= 0x80808080u; w.y ^= 0x80808080u; w.z ^= 0x80808080u; w.w ^= 0x80808080u;
-                const uint4 lo = make_uint4(widen_s8x2<0x4140>(w.x, f16), widen_s8x2<0x4342>(w.x, f16),
-                                            widen_s8x2<0x4140>(w.y, f16), widen_s8x2<0x4342>(w.y, f16));
-                const uint4 hi = make_uint4(widen_s8x2<0x4140>(w.z, f16), widen_s8x2<0x4342>(w.z, f16),
-                                            widen_s8x2<0x4140>(w.w, f16), widen_s8x2<0x4342>(w.w, f16));
-                uint8_t *base = a16 + (trow >> 7) * kATileBytes + (r >> 3) * 1024 + (r & 7) * 128;
-                *reinterpret_cast<uint4 *>(base + (((2 * c) ^ (r & 7)) << 4)) = lo;
-                *reinterpret_cast<uint4 *>(base + (((2 * c + 1) ^ (r & 7)) << 4)) = hi;
-            }
+            const uint8_t *a8 = smem + (size_t)st * stage_bytes + src_off;
+            uint8_t *a16 = smem + p.a16_off + (size_t)j * p.mt * kATileBytes + dst_off;
+            if (f16)
+                widen_tile<true>(a8, a16, off_lo, off_hi, n_tasks, src_step, dst_step);
+            else
+                widen_tile<false>(a8, a16, off_lo, off_hi, n_tasks, src_step, dst_step);
             fence_proxy_async_smem();      // the tensor core reads the tile through the async proxy
             __syncwarp();
             if (lane == 0)
                 mbar_arrive(&conv[j]);
+            if (++j == p.w8_slots) { j = 0; phj ^= 1; reuse = true; }
+            if (++st == p.stages) { st = 0; ph ^= 1; }
         }
         __syncwarp();
     }
@@ -730,6 +770,19 @@ static cudaError_t launch_instance(cudaLaunchConfig_t &cfg, const GemmTcParams &
     return cudaLaunchKernelEx(&cfg, k_gemm_tcgen05<KIND, PUSH, W8>, p);
 }
 
+// int8 weights: 128-row weight tiles per CTA (1 or 2).  The two widened tiles behind the ring cost
+// mt * 32 KiB; one weight tile per CTA when that is what lets two CTAs share an SM (the second streams
+// while the first is in its epilogue).  The packed codes are laid out for this number (pack.cu).
+int gemm_tc_w8_tiles(int NB, int N, int x_fp16)
+{
+    if (!(NB >= 48 && N % (2 * kTcTileM) == 0))
+        return 1;
+    const int b_bytes = (x_fp16 ? 1 : 2) * NB * kTcBlockK * 2;
+    const bool two_fit = (100 * 1024 - 4 * kATileBytes) / (kATileBytes + b_bytes) >= 3;
+    const bool one_fits = (100 * 1024 - 2 * kATileBytes) / (kATileBytes / 2 + b_bytes) >= 3;
+    return (!two_fit && one_fits) ? 1 : 2;
+}
+
 cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
 {
     if (a.NB < 16 || a.NB > 128 || a.NB % 16 || a.N % kTcTileM || a.K % kTcBlockK || a.B > a.NB)
@@ -748,15 +801,22 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     // Two 128-row weight tiles per CTA share one activation tile when the batch is wide enough for
     // the activation tile (2 * NB rows) to weigh as much as a weight tile: halves the L2->SM traffic
     // of the activations, which every CTA re-reads.
-    const int mt = (a.NB >= 48 && a.N % (2 * kTcTileM) == 0 && a.w_map256) ? 2 : 1;
+    const int mt = a.w8 ? gemm_tc_w8_tiles(a.NB, a.N, a.x_fp16)
+                        : ((a.NB >= 48 && a.N % (2 * kTcTileM) == 0 && a.w_map256) ? 2 : 1);
+    if (a.w8 && (!a.w8_codes || !a.scales))
+        return cudaErrorInvalidValue;
+    p.w8_codes = static_cast<const uint8_t *>(a.w8_codes);
     p.mt = mt;
-    if (mt == 2)
+    if (mt == 2 && !a.w8)
         p.w_map = *a.w_map256;
     const int tiles = a.N / (kTcTileM * mt);
     // int8 weights: a stage holds the codes (half a 16-bit tile) and the activations; two widened tiles
     // (mt * 16 KiB each) sit behind the ring
     const int stage_bytes = mt * (a.w8 ? kATileBytes / 2 : kATileBytes) + planes * a.NB * kTcBlockK * 2;
-    const int a16_bytes = a.w8 ? 2 * mt * kATileBytes : 0;
+    // (two widened tiles: three or four measured no faster - the stage rate is set by shared-memory traffic)
+    const int w8_slots = a.w8 ? 2 : 0;
+    p.w8_slots = w8_slots;
+    const int a16_bytes = w8_slots * mt * kATileBytes;
     p.w8 = a.w8;
     p.wscale = a.scales;
     // Ring depth, CTAs per SM and cluster splits.  Two CTAs per SM (rings <= 100 KiB) whenever that
@@ -765,7 +825,7 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     // co-resident slots (a second wave doubles the kernel); splits are a power of two <= 8 that leave
     // every rank >= 2 k-blocks.
     int stages = (200 * 1024 - a16_bytes) / stage_bytes, per_sm = 1;
-    if ((100 * 1024 - a16_bytes) / stage_bytes >= 4) {
+    if ((100 * 1024 - a16_bytes) / stage_bytes >= (a.w8 ? 3 : 4)) {
         stages = (100 * 1024 - a16_bytes) / stage_bytes;
         per_sm = 2;
     }

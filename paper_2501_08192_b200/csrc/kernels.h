@@ -139,9 +139,11 @@ cudaError_t launch_pack_rows(const void *const *srcs, const int *src_cols, int n
 // 1 KiB tiles of 16 rows x 64 k, scales [N] in packed row order.
 cudaError_t launch_pack_gemv_w8(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
                                 void *dst_codes, float *dst_scales, cudaStream_t s);
-// the same codes and scales for the tensor path: [N, K] K-major rows of int8 in the tensor path's row order
+// the same codes and scales for the tensor path, rows in the tensor path's order: the codes, biased by 128
+// (unsigned bytes), in contiguous blocks of (tiles * 128 rows) x 64 k, block (row tile, k block) at
+// ((row tile) * K / 64 + k block) * tiles * 8192 - a CTA's stream of k blocks is one contiguous run
 cudaError_t launch_pack_rows_w8(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
-                                void *dst_codes, float *dst_scales, cudaStream_t s);
+                                void *dst_codes, float *dst_scales, int tiles, cudaStream_t s);
 
 // ---- split-K GEMV (batch < 16): y[b,n] = sum_k x[b,k] W[n,k]; W in fragment-major tiles
 struct GemvArgs {
@@ -176,12 +178,16 @@ struct GemmTcArgs {
     long long *trace;
     int pdl;
     int inject;
-    // int8 weights: w_map / w_map256 are uint8 maps over the codes (dims (K, N), box (64, 128 or 256), no
-    // swizzle); the kernel widens every tile to the activations' 16-bit format in shared memory before
-    // the MMA and multiplies every accumulator row by its scale
+    // int8 weights: the codes come from w8_codes by plain bulk copies (w_map / w_map256 are unused); the
+    // kernel widens every tile to the activations' 16-bit format in shared memory before the MMA and
+    // multiplies every accumulator row by its scale
     int w8;
     const float *scales;  // w8: [N] in packed row order
+    const void *w8_codes; // w8: the packed codes (launch_pack_rows_w8 with gemm_tc_w8_tiles() rows per block)
 };
+// int8 weights: 128-row weight tiles per CTA for a matrix of N rows and a padded batch of NB (the packed
+// layout depends on it)
+int gemm_tc_w8_tiles(int NB, int N, int x_fp16);
 cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s);
 
 // ---- split-KV decode attention + merge

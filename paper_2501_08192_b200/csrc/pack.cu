@@ -89,7 +89,7 @@ struct PackW8Params {
     const bf16 *src[3];
     int cols[3];
     int N, K, kind;
-    int tensor;       // tensor-path row order and layout
+    int tensor;       // tensor-path row order and layout: 128-row tiles per block (1 or 2), 0 = GEMV path
     int8_t *codes;
     float *scales;
 };
@@ -125,7 +125,12 @@ __global__ void k_pack_w8(const __grid_constant__ PackW8Params p)
     r = fminf(fmaxf(r, -127.f), 127.f);
     size_t o;
     if (p.tensor) {
-        o = (size_t)row * p.K + k;
+        // the tensor path keeps the codes biased by 128 (unsigned bytes): its widening stage then needs
+        // no sign handling
+        const int block_rows = p.tensor * 128;
+        const size_t block = (size_t)(row / block_rows) * (p.K >> 6) + (k >> 6);
+        p.codes[(block * block_rows + row % block_rows) * 64 + (k & 63)] = (int8_t)(uint8_t)((int)r + 128);
+        return;
     } else {
         const int rb = row >> 4, rr = row & 15, g = rr & 7, hi = rr >> 3;
         const int kc = k >> 6, t = (k & 63) >> 4, e = k & 15;
@@ -134,7 +139,7 @@ __global__ void k_pack_w8(const __grid_constant__ PackW8Params p)
     p.codes[o] = (int8_t)(int)r;
 }
 
-static cudaError_t launch_pack_w8(bool tensor, const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
+static cudaError_t launch_pack_w8(int tensor, const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
                                   void *dst_codes, float *dst_scales, cudaStream_t s)
 {
     if (K % 64)
@@ -147,7 +152,7 @@ static cudaError_t launch_pack_w8(bool tensor, const void *const *srcs, const in
         N += src_cols[i];
     }
     p.N = N; p.K = K; p.kind = kind;
-    p.tensor = tensor ? 1 : 0;
+    p.tensor = tensor;
     p.codes = reinterpret_cast<int8_t *>(dst_codes);
     p.scales = dst_scales;
     k_w8_scales<<<(N + 127) / 128, 128, 0, s>>>(p);
@@ -159,12 +164,14 @@ static cudaError_t launch_pack_w8(bool tensor, const void *const *srcs, const in
 cudaError_t launch_pack_gemv_w8(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
                                 void *dst_codes, float *dst_scales, cudaStream_t s)
 {
-    return launch_pack_w8(false, srcs, src_cols, n_srcs, K, kind, dst_codes, dst_scales, s);
+    return launch_pack_w8(0, srcs, src_cols, n_srcs, K, kind, dst_codes, dst_scales, s);
 }
 cudaError_t launch_pack_rows_w8(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
-                                void *dst_codes, float *dst_scales, cudaStream_t s)
+                                void *dst_codes, float *dst_scales, int tiles, cudaStream_t s)
 {
-    return launch_pack_w8(true, srcs, src_cols, n_srcs, K, kind, dst_codes, dst_scales, s);
+    if (tiles != 1 && tiles != 2)
+        return cudaErrorInvalidValue;
+    return launch_pack_w8(tiles, srcs, src_cols, n_srcs, K, kind, dst_codes, dst_scales, s);
 }
 
 cudaError_t launch_pack_gemv(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind, void *dst,
