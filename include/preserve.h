@@ -91,8 +91,10 @@ extern "C" {
                                        feature (symmetric: scale = max |w| / 127 over the feature's inputs, code =
                                        round-to-nearest-even(w / scale), decided in fp32) - the weight precision
                                        of the paper's measurements (Section 4, "Experimental setup"); activations
-                                       and the KV-cache stay bf16.  Split-K GEMV path only (max_batch < 16 or
-                                       PRESERVE_FLAG_FORCE_GEMV), ffn a multiple of 64; PRESERVE_ESHAPE otherwise */
+                                       stay 16-bit (the KV-cache too unless PRESERVE_FLAG_INT8_KV is given).  Both
+                                       GEMM paths: the split-K GEMV kernels widen the codes in registers, the
+                                       tcgen05 kernels in shared memory in front of the MMA.  ffn a multiple of
+                                       64; PRESERVE_ESHAPE otherwise */
 #define PRESERVE_FLAG_INT8_KV 64u      /* the KV-cache is int8 with one fp32 scale per cached vector, i.e. per
                                        (sequence, kv head, slot): scale = max |u| / 127 over the vector's head_dim
                                        values, code = round-to-nearest-even(u / scale), decided in fp32; a cached
