@@ -99,19 +99,34 @@ __device__ __forceinline__ uint32_t widen_u8x2(uint32_t biased)
 // One widening pass of a converter thread over a tile: `n` tasks of 16 codes (one 16-byte load, two
 // 16-byte stores); consecutive tasks of a thread are `src_step` / `dst_step` bytes apart.
 template <bool F16>
+__device__ __forceinline__ void widen_one(uint4 w, uint8_t *dst, uint32_t off_lo, uint32_t off_hi)
+{
+    const uint4 lo = make_uint4(widen_u8x2<0x4140, F16>(w.x), widen_u8x2<0x4342, F16>(w.x),
+                                widen_u8x2<0x4140, F16>(w.y), widen_u8x2<0x4342, F16>(w.y));
+    const uint4 hi = make_uint4(widen_u8x2<0x4140, F16>(w.z), widen_u8x2<0x4342, F16>(w.z),
+                                widen_u8x2<0x4140, F16>(w.w), widen_u8x2<0x4342, F16>(w.w));
+    *reinterpret_cast<uint4 *>(dst + off_lo) = lo;
+    *reinterpret_cast<uint4 *>(dst + off_hi) = hi;
+}
+template <bool F16>
 __device__ __forceinline__ void widen_tile(const uint8_t *src, uint8_t *dst, uint32_t off_lo, uint32_t off_hi, int n,
                                            uint32_t src_step, uint32_t dst_step)
 {
-    for (int i = 0; i < n; ++i) {
-        const uint4 w = *reinterpret_cast<const uint4 *>(src);
-        const uint4 lo = make_uint4(widen_u8x2<0x4140, F16>(w.x), widen_u8x2<0x4342, F16>(w.x),
-                                    widen_u8x2<0x4140, F16>(w.y), widen_u8x2<0x4342, F16>(w.y));
-        const uint4 hi = make_uint4(widen_u8x2<0x4140, F16>(w.z), widen_u8x2<0x4342, F16>(w.z),
-                                    widen_u8x2<0x4140, F16>(w.w), widen_u8x2<0x4342, F16>(w.w));
-        *reinterpret_cast<uint4 *>(dst + off_lo) = lo;
-        *reinterpret_cast<uint4 *>(dst + off_hi) = hi;
-        src += src_step;
-        dst += dst_step;
+    // four tasks at a time, all loads first: a thread's tasks are independent, and a warp that waits
+    // for every load before it converts leaves most of its issue slots unused
+    while (n > 0) {
+        uint4 w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (i < n)
+                w[i] = *reinterpret_cast<const uint4 *>(src + i * src_step);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (i < n)
+                widen_one<F16>(w[i], dst + i * dst_step, off_lo, off_hi);
+        src += 4 * src_step;
+        dst += 4 * dst_step;
+        n -= 4;
     }
 }
 
