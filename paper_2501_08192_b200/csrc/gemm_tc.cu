@@ -39,7 +39,7 @@ namespace cg = cooperative_groups;
 namespace prsv {
 
 constexpr int kTcMaxStages = 12;
-constexpr int kTcMaxW8Slots = 4;          // int8 weights: widened operand tiles behind the ring
+constexpr int kTcMaxW8Slots = 4;          // int8 weights: widened operand tiles in tensor memory
 constexpr int kTcMaxEpiWarps = 16;        // 2-4 per TMEM lane group: the epilogue is a chain of short dependent
                                           // operations per output, so its speed is set by how many warps run it
 constexpr int kTcMaxProducers = 3;        // issuing threads of the TMA ring: warp 0, and lane 0 of the first epilogue warps
@@ -54,7 +54,7 @@ struct GemmTcParams {
     CUtensorMap x_map;
     int B, NB, N, K;
     int mt;             // 128-row weight tiles per CTA (1 or 2): two tiles share one activation tile
-    int kblocks;        // K / 64
+    int kblocks;        // K / 64 (int8 weights: K / 128 - a stage carries 128 k)
     int splits;         // cluster size along k
     int stages;
     int push;           // split-K reduction by one-sided hand-over: 1 = st.async, 2 = bulk copies (0: every rank reads all ranks)
@@ -68,9 +68,8 @@ struct GemmTcParams {
     int planes;         // activation planes in the B operand: 2 = bf16 hi + lo, 1 = a single fp16 plane
     int epi_warps;      // 8 or 16
     int producers;      // 1..kTcMaxProducers threads that issue the ring's TMA loads (stage uses dealt round-robin)
-    int w8;             // the weight tiles arrive as int8 codes ([rows][64] bytes, no swizzle) and are widened in shared memory
-    int a16_off;        // w8: offset of the widened weight tiles (w8_slots of mt * 16 KiB each) behind the ring
-    int w8_slots;       // 2..kTcMaxW8Slots
+    int w8;             // the weight tiles arrive as int8 codes and are widened into tensor memory (the MMA's A operand)
+    int w8_slots;       // 2..kTcMaxW8Slots widened tiles in tensor memory (mt * 32 columns each) behind the accumulators
     const float *wscale;  // w8: one fp32 scale per packed weight row
     const uint8_t *w8_codes;  // w8: the codes, one contiguous block of mt * 128 rows x 64 bytes per (tile, k-block)
 };
@@ -98,37 +97,24 @@ __device__ __forceinline__ uint32_t widen_u8x2(uint32_t biased)
 }
 // One widening pass of a converter thread over a tile: `n` tasks of 16 codes (one 16-byte load, two
 // 16-byte stores); consecutive tasks of a thread are `src_step` / `dst_step` bytes apart.
+// 16 codes (one 16-byte word group) widened to eight 32-bit registers: k elements 2c (low half) and
+// 2c + 1 (high half) in register c - the packing of a 16-bit A operand in tensor memory.
 template <bool F16>
-__device__ __forceinline__ void widen_one(uint4 w, uint8_t *dst, uint32_t off_lo, uint32_t off_hi)
+__device__ __forceinline__ void widen16(uint4 w, uint32_t (&r)[8])
 {
-    const uint4 lo = make_uint4(widen_u8x2<0x4140, F16>(w.x), widen_u8x2<0x4342, F16>(w.x),
-                                widen_u8x2<0x4140, F16>(w.y), widen_u8x2<0x4342, F16>(w.y));
-    const uint4 hi = make_uint4(widen_u8x2<0x4140, F16>(w.z), widen_u8x2<0x4342, F16>(w.z),
-                                widen_u8x2<0x4140, F16>(w.w), widen_u8x2<0x4342, F16>(w.w));
-    *reinterpret_cast<uint4 *>(dst + off_lo) = lo;
-    *reinterpret_cast<uint4 *>(dst + off_hi) = hi;
+    r[0] = widen_u8x2<0x4140, F16>(w.x); r[1] = widen_u8x2<0x4342, F16>(w.x);
+    r[2] = widen_u8x2<0x4140, F16>(w.y); r[3] = widen_u8x2<0x4342, F16>(w.y);
+    r[4] = widen_u8x2<0x4140, F16>(w.z); r[5] = widen_u8x2<0x4342, F16>(w.z);
+    r[6] = widen_u8x2<0x4140, F16>(w.w); r[7] = widen_u8x2<0x4342, F16>(w.w);
 }
-template <bool F16>
-__device__ __forceinline__ void widen_tile(const uint8_t *src, uint8_t *dst, uint32_t off_lo, uint32_t off_hi, int n,
-                                           uint32_t src_step, uint32_t dst_step)
+// registers -> 8 consecutive TMEM columns of this thread's lane (asynchronous; tc_st_wait completes it)
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&r)[8])
 {
-    // four tasks at a time, all loads first: a thread's tasks are independent, and a warp that waits
-    // for every load before it converts leaves most of its issue slots unused
-    while (n > 0) {
-        uint4 w[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if (i < n)
-                w[i] = *reinterpret_cast<const uint4 *>(src + i * src_step);
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if (i < n)
-                widen_one<F16>(w[i], dst + i * dst_step, off_lo, off_hi);
-        src += 4 * src_step;
-        dst += 4 * dst_step;
-        n -= 4;
-    }
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(r[0]),
+                 "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
 }
+__device__ __forceinline__ void tc_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr)
 {
@@ -142,6 +128,14 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
                  "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+                 : "memory");
+}
+// the same with the A operand in tensor memory (row m of A in lane m, two 16-bit k elements per column)
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+                 "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc)
                  : "memory");
 }
 __device__ __forceinline__ void tc_commit(uint64_t *bar)
@@ -202,26 +196,34 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile = blockIdx.x;
     const int s = blockIdx.y;
-    const int a_bytes = p.mt * (W8 ? kATileBytes / 2 : kATileBytes);
-    const int stage_bytes = a_bytes + p.planes * p.NB * kTcBlockK * 2;
+    // k per stage: 64, or 128 with int8 weights (a weight tile is 16 KiB either way) - what the MMA thread and
+    // the tensor pipe's front end spend per stage does not depend on what the stage carries, and an int8
+    // stage of 64 k carries half the bytes
+    constexpr int kBlk = W8 ? 2 * kTcBlockK : kTcBlockK;
+    const int a_bytes = p.mt * kATileBytes;
+    const int b_bytes = p.planes * p.NB * kBlk * 2;
+    const int stage_bytes = a_bytes + b_bytes;
     const int acc_cols = p.planes * p.NB;      // TMEM columns of one weight tile's accumulator
     const int kb0 = (int)((long long)p.kblocks * s / p.splits);
     const int kb1 = (int)((long long)p.kblocks * (s + 1) / p.splits);
 
+    // MMA-issuing threads (see run_mma): two for the int8 kernels with two weight tiles and sixteen epilogue warps
+    // (the last of them is then not needed as a converter)
+    const int n_issuers = (W8 && p.mt == 2 && p.epi_warps == 16 && p.producers == 3) ? 2 : 1;
     trace_start(p.trace);
     pdl_launch_dependents();
     load_epilogue_tables(p.epi, tabs, 0, p.B);   // inputs of the step: safe before the wait
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.stages; ++i) {
             mbar_init(&full[i], 1);
-            mbar_init(&empty[i], 1);
+            mbar_init(&empty[i], n_issuers);
         }
-        mbar_init(&accum_bar, 1);
+        mbar_init(&accum_bar, n_issuers);
         if (W8) {
             // the epilogue warps that issue no TMA loads widen the tiles: one arrival per warp and tile
             for (int j = 0; j < p.w8_slots; ++j) {
-                mbar_init(&conv[j], p.epi_warps - (p.producers - 1));
-                mbar_init(&a16_free[j], 1);
+                mbar_init(&conv[j], 4);        // one converter warp per TMEM lane quadrant
+                mbar_init(&a16_free[j], n_issuers);
             }
         }
         mbar_fence_init();
@@ -274,8 +276,14 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         pdl_wait();
         if (prod == 0)
             trace_waited(p.trace);
+        auto load_b = [&](int st_, int kb_) {
+            uint8_t *b_dst = smem + (size_t)st_ * stage_bytes + a_bytes;
+            tma_load_2d(b_dst, &p.x_map, kb_ * kBlk, 0, &full[st_]);
+            if constexpr (W8)      // second 64-k box of the stage
+                tma_load_2d(b_dst + b_bytes / 2, &p.x_map, kb_ * kBlk + kTcBlockK, 0, &full[st_]);
+        };
         for (int i = prod; i < pre; i += NP)
-            tma_load_2d(smem + (size_t)i * stage_bytes + a_bytes, &p.x_map, (kb0 + i) * kTcBlockK, 0, &full[i]);
+            load_b(i, kb0 + i);
         int it = prod;
         while (it < pre)
             it += NP;
@@ -291,7 +299,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 bulk_load_hint(a_dst, p.w8_codes + ((size_t)tile * p.kblocks + kb) * a_bytes, a_bytes, &full[st], pol);
             else
                 tma_load_2d_hint(a_dst, &p.w_map, kb * kTcBlockK, tile * p.mt * kTcTileM, &full[st], pol);
-            tma_load_2d(a_dst + a_bytes, &p.x_map, kb * kTcBlockK, 0, &full[st]);
+            load_b(st, kb);
             st += NP;
             while (st >= p.stages) {
                 st -= p.stages;
@@ -299,41 +307,58 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             }
         }
     };
-    if (warp == 0) {
-        if (lane == 0)
-            run_producer(0);
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            bool ok = true;
-            int st = 0, j = 0;               // ring stage and (int8 weights) widened slot of this use, with their phases
-            uint32_t ph = 0, phj = 0;
-            for (int kb = kb0; kb < kb1; ++kb) {
-                // (int8 weights: the widened tile of this use completes after the stage has landed)
-                if (!(W8 ? mbar_wait(&conv[j], phj, p.status, ST_TIMEOUT_FULL)
-                           : mbar_wait(&full[st], ph, p.status, ST_TIMEOUT_FULL))) { poisoned = 1; ok = false; break; }
-                tc_fence_after();
-                const uint32_t st_addr = smem_u32(smem + (size_t)st * stage_bytes);
-                const uint32_t a_addr = W8 ? smem_u32(smem + p.a16_off + (size_t)j * p.mt * kATileBytes) : st_addr;
-                const uint64_t bdesc = make_smem_desc(st_addr + a_bytes);
-                for (int m = 0; m < p.mt; ++m) {
-                    // each 128-row weight tile has its own accumulator (2 * NB TMEM columns)
-                    const uint64_t adesc = make_smem_desc(a_addr + m * kATileBytes);
+    // ------------------------------------------------------------ MMA issuers
+    // One thread issues the MMAs of weight tiles [m_lo, m_hi).  The int8 kernels with two weight tiles
+    // per CTA use two such threads (warp 1 and the last epilogue warp, lane 0 each), one per tile: the
+    // tiles have separate accumulators, so their MMAs are independent, and what one thread spends per
+    // stage (issuing eight MMAs at the pace the tensor pipe takes them, two commits, the next wait) is
+    // longer than an int8 stage may take.  A stage and a widened slot are free once both have committed.
+    auto run_mma = [&](int m_lo, int m_hi) {
+        bool ok = true;
+        int st = 0, j = 0;               // ring stage and (int8 weights) widened slot of this use, with their phases
+        uint32_t ph = 0, phj = 0;
+        for (int kb = kb0; kb < kb1; ++kb) {
+            // (int8 weights: the widened tile of this use completes after the stage has landed)
+            if (!(W8 ? mbar_wait(&conv[j], phj, p.status, ST_TIMEOUT_FULL)
+                       : mbar_wait(&full[st], ph, p.status, ST_TIMEOUT_FULL))) { poisoned = 1; ok = false; break; }
+            tc_fence_after();
+            const uint32_t st_addr = smem_u32(smem + (size_t)st * stage_bytes);
+            const uint64_t bdesc = make_smem_desc(st_addr + a_bytes);
+            for (int m = m_lo; m < m_hi; ++m) {
+                // each 128-row weight tile has its own accumulator (2 * NB TMEM columns)
+                if constexpr (W8) {
+                    // widened tile of this use: 64 columns per weight tile (128 k), 8 per MMA; the activations
+                    // are two 64-k boxes
+                    const uint32_t a_tmem = tmem_base + p.mt * acc_cols + (j * p.mt + m) * 64;
+                    const uint64_t bdesc2 = make_smem_desc(st_addr + a_bytes + b_bytes / 2);
+#pragma unroll
+                    for (int k = 0; k < kBlk / 16; ++k)
+                        tc_mma_ts(tmem_base + m * acc_cols, a_tmem + 8 * k, (k < 4 ? bdesc : bdesc2) + 2 * (k & 3), p.idesc,
+                                  (kb > kb0 || k > 0) ? 1u : 0u);
+                } else {
+                    const uint64_t adesc = make_smem_desc(st_addr + m * kATileBytes);
 #pragma unroll
                     for (int k = 0; k < kTcBlockK / 16; ++k)
                         tc_mma(tmem_base + m * acc_cols, adesc + 2 * k, bdesc + 2 * k, p.idesc,
                                (kb > kb0 || k > 0) ? 1u : 0u);
                 }
-                tc_commit(&empty[st]);      // slot is free once these MMAs have read it
-                if (W8) {
-                    tc_commit(&a16_free[j]);
-                    if (++j == p.w8_slots) { j = 0; phj ^= 1; }
-                }
-                if (++st == p.stages) { st = 0; ph ^= 1; }
             }
-            if (ok)
-                tc_commit(&accum_bar);      // accumulator complete
+            tc_commit(&empty[st]);      // slot is free once these MMAs have read it
+            if (W8) {
+                tc_commit(&a16_free[j]);
+                if (++j == p.w8_slots) { j = 0; phj ^= 1; }
+            }
+            if (++st == p.stages) { st = 0; ph ^= 1; }
         }
+        if (ok)
+            tc_commit(&accum_bar);      // this issuer's accumulators are complete
+    };
+    if (warp == 0) {
+        if (lane == 0)
+            run_producer(0);
+    } else if (warp == 1) {
+        if (lane == 0)
+            run_mma(0, n_issuers == 2 ? 1 : p.mt);
     }
     __syncwarp();
 
@@ -392,44 +417,81 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             run_producer(warp - 1);
         __syncwarp();
     }
+    else if (is_epi && W8 && n_issuers == 2 && warp == 1 + p.epi_warps) {
+        if (lane == 0)
+            run_mma(1, 2);
+        __syncwarp();
+    }
     else if (is_epi && W8) {
         // ---------------------------------------------------- int8 weights: widen every tile
-        // Tile use `itc` is converted from its ring stage into widened slot itc % slots (the MMA operand
-        // layout: K-major rows, 8-row atoms of 1 KiB, 128-byte swizzle).  A task = 16 codes of one
-        // row (one 16-byte load, two 16-byte stores).  The slot is written again only after the MMAs
-        // of use itc - slots have read it.
-        // A thread's tasks are 8 * n_conv rows apart: the same 16-byte column and the same row within
-        // an 8-row swizzle atom every time, so everything but two base pointers is fixed per thread.
-        const int cw = warp - 1 - p.producers, n_conv = p.epi_warps - (p.producers - 1);
+        // Tile use `itc` is widened from its ring stage into tensor-memory slot itc % slots, where the
+        // MMA takes it as its A operand: row r of a weight tile in TMEM lane r, 64 columns per 128 k.
+        // A warp reaches the 32 lanes of its quadrant (warp % 4) only, so the converter warps of a
+        // quadrant share that quadrant's tasks: task (m, q) = rows 32 * quadrant .. + 31 of weight
+        // tile m, k = 16 q .. 16 q + 15 - per lane one 16-byte load (the packed block keeps the four
+        // 16-byte groups of a row in an order that makes these loads conflict-free) and one store of
+        // 8 columns.  The slot is written again only after the MMAs of use itc - slots have read it.
+        // The converter warps form groups of four, one warp per quadrant; group g widens the tile uses
+        // g, g + G, ... on its own, so successive stages are widened concurrently (a single group
+        // needs longer for one stage than the stage may take).
+        const int quad = warp & 3;
+        int iq = 0, n_min = 1 << 30;     // this warp's index among its quadrant's converter warps; the groups
+        for (int q2 = 0; q2 < 4; ++q2) {
+            int n = 0;
+            for (int w2 = p.producers + 1; w2 < 2 + p.epi_warps - (n_issuers == 2 ? 1 : 0); ++w2)
+                if ((w2 & 3) == q2) {
+                    if (q2 == quad && w2 < warp)
+                        ++iq;
+                    ++n;
+                }
+            n_min = n < n_min ? n : n_min;
+        }
+        const int G = n_min;
         const bool f16 = p.planes == 1;
-        const int task0 = cw * 32 + lane, trow0 = task0 >> 2, c = task0 & 3;
-        const int n_tasks = (p.mt * 512 - task0 + n_conv * 32 - 1) / (n_conv * 32);
-        const uint32_t src_off = (uint32_t)trow0 * 64 + c * 16;
-        const uint32_t dst_off = (uint32_t)(trow0 >> 3) * 1024 + (trow0 & 7) * 128;   // (m-tiles are 16 atoms apart: contiguous)
-        const uint32_t off_lo = (uint32_t)((2 * c) ^ (trow0 & 7)) << 4, off_hi = (uint32_t)((2 * c + 1) ^ (trow0 & 7)) << 4;
-        const uint32_t src_step = (uint32_t)n_conv * 8 * 64, dst_step = (uint32_t)n_conv * 1024;
+        const int row = quad * 32 + lane;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(p.mt * acc_cols);
+        const uint32_t src_lane = (uint32_t)row * 128;
+        const uint32_t swz = (uint32_t)(row & 7);
         int st = 0, j = 0;
         uint32_t ph = 0, phj = 0;
         bool reuse = false;          // the slot has been used before: wait until the MMAs of that use are done
-        for (int kb = kb0; kb < kb1; ++kb) {
-            int ok = 1;
-            if (lane == 0) {
-                ok = mbar_wait(&full[st], ph, p.status, ST_TIMEOUT_FULL) ? 1 : 0;
-                if (ok && reuse)
-                    ok = mbar_wait(&a16_free[j], phj ^ 1, p.status, ST_TIMEOUT_EMPTY) ? 1 : 0;
+        int turn = 0;                // use index modulo G
+        for (int kb = kb0; kb < kb1 && iq < G; ++kb) {
+            if (turn == iq) {
+                int ok = 1;
+                if (lane == 0) {
+                    ok = mbar_wait(&full[st], ph, p.status, ST_TIMEOUT_FULL) ? 1 : 0;
+                    if (ok && reuse)
+                        ok = mbar_wait(&a16_free[j], phj ^ 1, p.status, ST_TIMEOUT_EMPTY) ? 1 : 0;
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { poisoned = 1; break; }
+                tc_fence_after();
+                const uint8_t *a8 = smem + (size_t)st * stage_bytes + src_lane;
+                const uint32_t slot_addr = lane_addr + (uint32_t)(j * p.mt * 64);
+                for (int mh = 0; mh < 2 * p.mt; ++mh) {      // (weight tile, half of its 128 k): four 16-byte groups
+                    const int m = mh >> 1, q0 = (mh & 1) * 4;
+                    uint4 w[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        w[q] = *reinterpret_cast<const uint4 *>(a8 + m * (kTcTileM * 128) + (((q0 + q) ^ swz) << 4));
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t r[8];
+                        if (f16)
+                            widen16<true>(w[q], r);
+                        else
+                            widen16<false>(w[q], r);
+                        tc_st8(slot_addr + (uint32_t)(m * 64 + (q0 + q) * 8), r);
+                    }
+                }
+                tc_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0)
+                    mbar_arrive(&conv[j]);
             }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) { poisoned = 1; break; }
-            const uint8_t *a8 = smem + (size_t)st * stage_bytes + src_off;
-            uint8_t *a16 = smem + p.a16_off + (size_t)j * p.mt * kATileBytes + dst_off;
-            if (f16)
-                widen_tile<true>(a8, a16, off_lo, off_hi, n_tasks, src_step, dst_step);
-            else
-                widen_tile<false>(a8, a16, off_lo, off_hi, n_tasks, src_step, dst_step);
-            fence_proxy_async_smem();      // the tensor core reads the tile through the async proxy
-            __syncwarp();
-            if (lane == 0)
-                mbar_arrive(&conv[j]);
+            if (++turn == G) turn = 0;
             if (++j == p.w8_slots) { j = 0; phj ^= 1; reuse = true; }
             if (++st == p.stages) { st = 0; ph ^= 1; }
         }
@@ -790,23 +852,21 @@ static cudaError_t launch_instance(cudaLaunchConfig_t &cfg, const GemmTcParams &
 // while the first is in its epilogue).  The packed codes are laid out for this number (pack.cu).
 int gemm_tc_w8_tiles(int NB, int N, int x_fp16)
 {
-    if (!(NB >= 48 && N % (2 * kTcTileM) == 0))
-        return 1;
-    const int b_bytes = (x_fp16 ? 1 : 2) * NB * kTcBlockK * 2;
-    const bool two_fit = (100 * 1024 - 4 * kATileBytes) / (kATileBytes + b_bytes) >= 3;
-    const bool one_fits = (100 * 1024 - 2 * kATileBytes) / (kATileBytes / 2 + b_bytes) >= 3;
-    return (!two_fit && one_fits) ? 1 : 2;
+    // two tiles whenever the matrix has an even number of them and tensor memory (512 columns) holds two
+    // accumulators plus at least two widened tiles of 2 * 64 columns (128 k)
+    const int acc = (x_fp16 ? 1 : 2) * NB;
+    return (N % (2 * kTcTileM) == 0 && 2 * acc + 2 * 2 * 64 <= 512) ? 2 : 1;
 }
 
 cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
 {
-    if (a.NB < 16 || a.NB > 128 || a.NB % 16 || a.N % kTcTileM || a.K % kTcBlockK || a.B > a.NB)
+    if (a.NB < 16 || a.NB > 128 || a.NB % 16 || a.N % kTcTileM || a.K % (a.w8 ? 2 * kTcBlockK : kTcBlockK) || a.B > a.NB)
         return cudaErrorInvalidValue;
     GemmTcParams p;
     p.w_map = a.w_map;
     p.x_map = a.x_map;
     p.B = a.B; p.NB = a.NB; p.N = a.N; p.K = a.K;
-    p.kblocks = a.K / kTcBlockK;
+    p.kblocks = a.K / (a.w8 ? 2 * kTcBlockK : kTcBlockK);
     p.epi = a.epi;
     p.status = a.status;
     p.trace = a.trace;
@@ -825,13 +885,20 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     if (mt == 2 && !a.w8)
         p.w_map = *a.w_map256;
     const int tiles = a.N / (kTcTileM * mt);
-    // int8 weights: a stage holds the codes (half a 16-bit tile) and the activations; two widened tiles
-    // (mt * 16 KiB each) sit behind the ring
-    const int stage_bytes = mt * (a.w8 ? kATileBytes / 2 : kATileBytes) + planes * a.NB * kTcBlockK * 2;
-    // (two widened tiles: three or four measured no faster - the stage rate is set by shared-memory traffic)
-    const int w8_slots = a.w8 ? 2 : 0;
+    // int8 weights: a stage holds the codes (half a 16-bit tile) and the activations; the widened tiles
+    // live in tensor memory behind the accumulators (as many as fit, at most four), so the whole of
+    // shared memory is ring: a deep ring is what keeps enough int8 bytes in flight.  One CTA per SM
+    // (tensor memory is per SM).
+    const int stage_bytes = mt * kATileBytes + planes * a.NB * (a.w8 ? 2 * kTcBlockK : kTcBlockK) * 2;
+    int w8_slots = 0;
+    if (a.w8) {
+        w8_slots = (512 - mt * planes * a.NB) / (mt * 64);
+        w8_slots = w8_slots > kTcMaxW8Slots ? kTcMaxW8Slots : w8_slots;
+        if (w8_slots < 2)
+            return cudaErrorInvalidValue;
+    }
     p.w8_slots = w8_slots;
-    const int a16_bytes = w8_slots * mt * kATileBytes;
+    const int a16_bytes = 0;
     p.w8 = a.w8;
     p.wscale = a.scales;
     // Ring depth, CTAs per SM and cluster splits.  Two CTAs per SM (rings <= 100 KiB) whenever that
@@ -840,7 +907,7 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     // co-resident slots (a second wave doubles the kernel); splits are a power of two <= 8 that leave
     // every rank >= 2 k-blocks.
     int stages = (200 * 1024 - a16_bytes) / stage_bytes, per_sm = 1;
-    if ((100 * 1024 - a16_bytes) / stage_bytes >= (a.w8 ? 3 : 4)) {
+    if (!a.w8 && (100 * 1024 - a16_bytes) / stage_bytes >= 4) {
         stages = (100 * 1024 - a16_bytes) / stage_bytes;
         per_sm = 2;
     }
@@ -861,7 +928,7 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     p.stages = stages;
     p.splits = splits;
     int cols = 32;
-    while (cols < mt * planes * a.NB) cols *= 2;
+    while (cols < mt * planes * a.NB + w8_slots * mt * 64) cols *= 2;
     p.tmem_cols = cols;
     // instruction descriptor: fp32 accumulate; A (weights) and B (activations) in the same 16-bit format -
     // both bf16 (B = hi + lo planes) or both fp16 (B = one plane); N = columns of the B tile, M = 128
@@ -897,7 +964,6 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
             recv_alloc = need;
         }
     }
-    p.a16_off = stages * stage_bytes;
     p.recv_off = stages * stage_bytes + a16_bytes;
     size_t smem = (size_t)stages * stage_bytes + a16_bytes + recv_alloc + 1024;
     const size_t red_bytes = (size_t)mt * a.NB * kTcTileM * 4 + 1024;

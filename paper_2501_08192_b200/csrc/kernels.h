@@ -140,8 +140,9 @@ cudaError_t launch_pack_rows(const void *const *srcs, const int *src_cols, int n
 cudaError_t launch_pack_gemv_w8(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
                                 void *dst_codes, float *dst_scales, cudaStream_t s);
 // the same codes and scales for the tensor path, rows in the tensor path's order: the codes, biased by 128
-// (unsigned bytes), in contiguous blocks of (tiles * 128 rows) x 64 k, block (row tile, k block) at
-// ((row tile) * K / 64 + k block) * tiles * 8192 - a CTA's stream of k blocks is one contiguous run
+// (unsigned bytes), in contiguous blocks of (tiles * 128 rows) x 128 k, block (row tile, k block) at
+// ((row tile) * K / 128 + k block) * tiles * 16384 - a CTA's stream of k blocks is one contiguous run; inside a
+// row the eight 16-byte groups are permuted by the row index (pack.cu)
 cudaError_t launch_pack_rows_w8(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
                                 void *dst_codes, float *dst_scales, int tiles, cudaStream_t s);
 
@@ -179,8 +180,8 @@ struct GemmTcArgs {
     int pdl;
     int inject;
     // int8 weights: the codes come from w8_codes by plain bulk copies (w_map / w_map256 are unused); the
-    // kernel widens every tile to the activations' 16-bit format in shared memory before the MMA and
-    // multiplies every accumulator row by its scale
+    // kernel widens every tile to the activations' 16-bit format into tensor memory (the MMA's A operand)
+    // and multiplies every accumulator row by its scale
     int w8;
     const float *scales;  // w8: [N] in packed row order
     const void *w8_codes; // w8: the packed codes (launch_pack_rows_w8 with gemm_tc_w8_tiles() rows per block)

@@ -128,8 +128,12 @@ __global__ void k_pack_w8(const __grid_constant__ PackW8Params p)
         // the tensor path keeps the codes biased by 128 (unsigned bytes): its widening stage then needs
         // no sign handling
         const int block_rows = p.tensor * 128;
-        const size_t block = (size_t)(row / block_rows) * (p.K >> 6) + (k >> 6);
-        p.codes[(block * block_rows + row % block_rows) * 64 + (k & 63)] = (int8_t)(uint8_t)((int)r + 128);
+        const size_t block = (size_t)(row / block_rows) * (p.K >> 7) + (k >> 7);
+        // (the eight 16-byte groups of a row's 128 k are stored in the order q ^ (row % 8): the widening
+        // warps read one group per lane, 32 consecutive rows at a time, without bank conflicts)
+        const int rr = row % block_rows, kk = k & 127;
+        const int grp = (kk >> 4) ^ (rr & 7);
+        p.codes[(block * block_rows + rr) * 128 + grp * 16 + (kk & 15)] = (int8_t)(uint8_t)((int)r + 128);
         return;
     } else {
         const int rb = row >> 4, rr = row & 15, g = rr & 7, hi = rr >> 3;
@@ -169,7 +173,7 @@ cudaError_t launch_pack_gemv_w8(const void *const *srcs, const int *src_cols, in
 cudaError_t launch_pack_rows_w8(const void *const *srcs, const int *src_cols, int n_srcs, int K, int kind,
                                 void *dst_codes, float *dst_scales, int tiles, cudaStream_t s)
 {
-    if (tiles != 1 && tiles != 2)
+    if ((tiles != 1 && tiles != 2) || K % 128)
         return cudaErrorInvalidValue;
     return launch_pack_w8(tiles, srcs, src_cols, n_srcs, K, kind, dst_codes, dst_scales, s);
 }
