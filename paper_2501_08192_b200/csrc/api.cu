@@ -396,7 +396,7 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
         // traffic and half the MMA work of the largest GEMM.  The QKV projection keeps hi + lo bf16
         // planes: rounding of q is amplified by the softmax (measured: one fp16 plane put the 70B-shaped
         // chain's attention partial sums at 1.02 of the bound).
-        a.x_fp16 = which == 2 ? 1 : 0;
+        a.x_fp16 = which >= 1 ? 1 : 0;
         a.w8 = L->w8 ? 1 : 0;
         a.scales = L->w8 ? L->scales + L->soff[which] : nullptr;
         a.w8_codes = L->w8 ? L->arena + L->off[which] : nullptr;
@@ -646,6 +646,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
         a.q = L->q;
         a.q_plane = (size_t)L->rows * c.n_q_heads * kHeadDim;
         a.o_plane = a.q_plane;
+        a.o_fp16 = L->tensor_path ? 1 : 0;
         a.ctx_len = sp.ctx_len;
         a.B = B; a.nq = c.n_q_heads; a.nkv = c.n_kv_heads; a.cap = cap;
         a.grid = pl.attn_grid;
@@ -754,6 +755,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
         e.kind = EPI_SWIGLU;
         e.out = L->a;
         e.out_plane = (size_t)L->rows * c.ffn;
+        e.out_fp16 = L->tensor_path ? 1 : 0;
         int rc = launch_gemm(L, 2, L->x2, B, e, pdl, s, TRACE(6));
         if (rc)
             return rc;
@@ -1105,7 +1107,7 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
             const int nbp = ((c.max_batch + 15) / 16) * 16;
             auto pack8 = [&](const void *const *srcs, const int *cols, int n, int i, int kind) -> cudaError_t {
                 return L->tensor_path ? launch_pack_rows_w8(srcs, cols, n, d.k[i], kind, L->arena + L->off[i],
-                                                            L->scales + L->soff[i], gemm_tc_w8_tiles(nbp, d.n[i], i == 2),
+                                                            L->scales + L->soff[i], gemm_tc_w8_tiles(nbp, d.n[i], i >= 1),
                                                             nullptr)
                                       : launch_pack_gemv_w8(srcs, cols, n, d.k[i], kind, L->arena + L->off[i],
                                                             L->scales + L->soff[i], nullptr);
@@ -1118,9 +1120,9 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
             auto pack = L->tensor_path ? launch_pack_rows : launch_pack_gemv;
             // (tensor path: Wgate|up meets the fp16 RMSNorm output x2 and is stored as fp16)
             CKI(pack(s_qkv, c_qkv, 3, d.k[0], EPI_QKV, L->arena + L->off[0], 0, nullptr));
-            CKI(pack(s_o, c_o, 1, d.k[1], EPI_PLAIN, L->arena + L->off[1], 0, nullptr));
+            CKI(pack(s_o, c_o, 1, d.k[1], EPI_PLAIN, L->arena + L->off[1], 1, nullptr));
             CKI(pack(s_gu, c_gu, 2, d.k[2], EPI_SWIGLU, L->arena + L->off[2], 1, nullptr));
-            CKI(pack(s_dn, c_dn, 1, d.k[3], EPI_PLAIN, L->arena + L->off[3], 0, nullptr));
+            CKI(pack(s_dn, c_dn, 1, d.k[3], EPI_PLAIN, L->arena + L->off[3], 1, nullptr));
         }
     }
     // rotary frequencies theta^(-2i/d)
@@ -1176,7 +1178,7 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
         const void *xb[4] = {L->x, L->o, L->x2, L->a};
         for (int i = 0; i < 4; ++i) {
             // x2 (the MLP's RMSNorm output) is one fp16 plane; x, o and a are two bf16 planes (hi rows, lo rows)
-            const uint32_t brows = (uint32_t)(i == 2 ? L->nb_pad : 2 * L->nb_pad);
+            const uint32_t brows = (uint32_t)(i >= 1 ? L->nb_pad : 2 * L->nb_pad);
             // (int8 weights are fetched by plain bulk copies: no map over them)
             const bool wok = L->w8 || make_map_2d(&L->wmap[i], L->arena + L->off[i], d.k[i], d.n[i], 64, 128);
             if (!wok || !make_map_2d(&L->xmap[i], xb[i], d.k[i], brows, 64, brows)) {

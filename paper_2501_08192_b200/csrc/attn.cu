@@ -24,6 +24,8 @@
 #include <cstdlib>
 
 #include "../../include/preserve.h"
+#include <cuda_fp16.h>
+
 #include "attn_common.cuh"
 #include "common.cuh"
 #include "kernels.h"
@@ -48,6 +50,7 @@ struct AttnParams {
     float *part_ml;         // [item][G][2] (max, sum)
     bf16 *o_out;            // hi plane; lo plane at o_out + o_plane
     size_t o_plane;
+    int o_fp16;             // o_out is ONE fp16 plane instead (an attention output is bounded by the largest value)
     int *status;
     long long *trace;
     int inject;             // test hook: the producer of CTA 0 never fetches one box of its first tile
@@ -428,11 +431,15 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv(const _
             if (n_items_stream == 1) {
                 // the item is the whole sequence: finish here
                 const float o0 = acc.x / lsum, o1 = acc.y / lsum;
-                uint32_t hi, lo;
-                split_bf16x2(o0, o1, hi, lo);
                 const size_t oi = ((size_t)b * p.nq + (size_t)kvh * p.G + r) * kHeadDim + 2 * d2;
-                *reinterpret_cast<uint32_t *>(p.o_out + oi) = hi;
-                *reinterpret_cast<uint32_t *>(p.o_out + p.o_plane + oi) = lo;
+                if (p.o_fp16) {
+                    *reinterpret_cast<__half2 *>(reinterpret_cast<__half *>(p.o_out) + oi) = __floats2half2_rn(o0, o1);
+                } else {
+                    uint32_t hi, lo;
+                    split_bf16x2(o0, o1, hi, lo);
+                    *reinterpret_cast<uint32_t *>(p.o_out + oi) = hi;
+                    *reinterpret_cast<uint32_t *>(p.o_out + p.o_plane + oi) = lo;
+                }
             } else {
                 *reinterpret_cast<float2 *>(p.part_o + ((size_t)item * p.G + r) * kHeadDim + 2 * d2) = acc;
                 if (d2 == 0)
@@ -519,10 +526,14 @@ __global__ void __launch_bounds__(kMergeMaxWarps * 32) k_attn_merge(const __grid
                 l += l_s[w];
             }
             const float ov = a / l;
-            const bf16 hi = __float2bfloat16_rn(ov);
             const size_t oi = ((size_t)b * p.nq + hq) * kHeadDim + tid;
-            p.o_out[oi] = hi;
-            p.o_out[p.o_plane + oi] = __float2bfloat16_rn(ov - __bfloat162float(hi));
+            if (p.o_fp16) {
+                reinterpret_cast<__half *>(p.o_out)[oi] = __float2half_rn(ov);
+            } else {
+                const bf16 hi = __float2bfloat16_rn(ov);
+                p.o_out[oi] = hi;
+                p.o_out[p.o_plane + oi] = __float2bfloat16_rn(ov - __bfloat162float(hi));
+            }
         }
     }
     trace_end(tr);
@@ -602,6 +613,7 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     p.q = reinterpret_cast<const bf16 *>(a.q);
     p.q_plane = a.q_plane;
     p.o_plane = a.o_plane;
+    p.o_fp16 = a.o_fp16;
     p.ctx_len = a.ctx_len;
     p.B = a.B; p.nq = a.nq; p.nkv = a.nkv; p.G = a.nq / a.nkv; p.cap = a.cap;
     p.tiles_per_item = a.tiles_per_item;

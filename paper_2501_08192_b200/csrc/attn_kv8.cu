@@ -63,6 +63,7 @@ struct AttnKv8Params {
     float *part_ml;
     bf16 *o_out;
     size_t o_plane;
+    int o_fp16;             // o_out is ONE fp16 plane instead of split bf16
     int *status;
     long long *trace;
     int inject;
@@ -450,11 +451,15 @@ __global__ void __launch_bounds__(kAttnThreads, 2) k_attn_decode_splitkv_kv8(con
             if (n_items_stream == 1) {
                 // the item is the whole sequence: finish here
                 const float o0 = acc.x / lsum, o1 = acc.y / lsum;
-                uint32_t hi, lo;
-                split_bf16x2(o0, o1, hi, lo);
                 const size_t oi = ((size_t)b * p.nq + (size_t)kvh * p.G + r) * kHeadDim + 2 * d2;
-                *reinterpret_cast<uint32_t *>(p.o_out + oi) = hi;
-                *reinterpret_cast<uint32_t *>(p.o_out + p.o_plane + oi) = lo;
+                if (p.o_fp16) {
+                    *reinterpret_cast<__half2 *>(reinterpret_cast<__half *>(p.o_out) + oi) = __floats2half2_rn(o0, o1);
+                } else {
+                    uint32_t hi, lo;
+                    split_bf16x2(o0, o1, hi, lo);
+                    *reinterpret_cast<uint32_t *>(p.o_out + oi) = hi;
+                    *reinterpret_cast<uint32_t *>(p.o_out + p.o_plane + oi) = lo;
+                }
             } else {
                 *reinterpret_cast<float2 *>(p.part_o + ((size_t)item * p.G + r) * kHeadDim + 2 * d2) = acc;
                 if (d2 == 0)
@@ -499,6 +504,7 @@ cudaError_t launch_attention_kv8_kernel(const AttnArgs &a, const cudaLaunchConfi
     p.part_ml = a.part_ml;
     p.o_out = reinterpret_cast<bf16 *>(a.o_out);
     p.o_plane = a.o_plane;
+    p.o_fp16 = a.o_fp16;
     p.status = a.status;
     p.trace = a.trace;
     p.inject = a.inject;

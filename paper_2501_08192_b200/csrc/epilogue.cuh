@@ -9,6 +9,8 @@
 //   GEMV path  : 16-row blocks; rows r and r+8 (r < 8) of block rb are a pair.
 //   tensor path: rows 2m and 2m+1 are a pair.
 #pragma once
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 #include "kernels.h"
 
@@ -169,7 +171,10 @@ __device__ __forceinline__ void apply_epilogue_t(const EpilogueArgs &e, const Ep
         // silu by the fast exponential and division (a few ulp; for v0 < -87 the quotient flushes to 0,
         // its true size being < 1e-36)
         const float a = __fdividef(v0, 1.f + __expf(-v0)) * v1;
-        store_split(e.out, e.out_plane, (size_t)b * (N >> 1) + n0, a);
+        if (e.out_fp16)
+            reinterpret_cast<__half *>(e.out)[(size_t)b * (N >> 1) + n0] = __float2half_rn(fminf(fmaxf(a, -65504.f), 65504.f));
+        else
+            store_split(e.out, e.out_plane, (size_t)b * (N >> 1) + n0, a);
     } else {
         const int pos = tab.pos[b_local];
         epilogue_qkv(e, pos, b, n0, n1, v0, v1, rope_trig(e, tab, pos, n0, n1));
@@ -207,9 +212,14 @@ __device__ __forceinline__ void apply_epilogue_quad_t(const EpilogueArgs &e, con
     } else if constexpr (KIND == EPI_SWIGLU) {
         const float a0 = __fdividef(v.x, 1.f + __expf(-v.x)) * v.y;
         const float a1 = __fdividef(v.z, 1.f + __expf(-v.z)) * v.w;
+        const size_t o = (size_t)b * (N >> 1) + pair0;
+        if (e.out_fp16) {
+            *reinterpret_cast<__half2 *>(reinterpret_cast<__half *>(e.out) + o) =
+                __floats2half2_rn(fminf(fmaxf(a0, -65504.f), 65504.f), fminf(fmaxf(a1, -65504.f), 65504.f));
+            return;
+        }
         uint32_t hi, lo;
         split_bf16x2(a0, a1, hi, lo);
-        const size_t o = (size_t)b * (N >> 1) + pair0;
         *reinterpret_cast<uint32_t *>(reinterpret_cast<bf16 *>(e.out) + o) = hi;
         *reinterpret_cast<uint32_t *>(reinterpret_cast<bf16 *>(e.out) + e.out_plane + o) = lo;
     } else {

@@ -111,6 +111,7 @@ struct EpilogueArgs {
     int kind;
     void *out;            // PLAIN: bf16 [B,N]; SWIGLU: split bf16 [2][rows][N/2]
     size_t out_plane;     // SWIGLU: elements between the hi and lo planes of out
+    int out_fp16;         // SWIGLU: out is ONE fp16 plane [rows][N/2] (clamped to +-65504) instead of split bf16
     void *out2;           // PLAIN: optional second copy of the output (bf16 [B,N])
     float *out_f32;       // PLAIN: optional unrounded copy (fp32 [B,N])
     // QKV: rows are heads [q | k | v] x head_dim; rotary embedding on q and k, k/v appended
@@ -207,6 +208,7 @@ struct AttnArgs {
     int max_items_per_stream;   // work items of the longest sequence (sizes the merge CTAs)
     void *o_out;          // split bf16 [2][rows][nq,d]
     size_t o_plane;
+    int o_fp16;           // o_out is ONE fp16 plane [rows][nq,d] instead
     int *status;
     cudaEvent_t mid_event; // optional: recorded between the split-KV kernel and the merge kernel
     int phases;            // bit 0: split-KV kernel, bit 1: merge kernel (0 = both)

@@ -128,7 +128,7 @@ class DeviceLayer:
         spec = {"x": (1, (H,)), "q": (2, (nq, d)), "o": (3, (nq, d)), "x2": (4, (H,)), "a": (5, (F,))}
         fp16_x = bool(self.layer.get_info().normed_activations_fp16)
         for name, (which, tail) in spec.items():
-            if fp16_x and name == "x2":               # one fp16 plane on the tensor path
+            if fp16_x and name in ("o", "x2", "a"):   # one fp16 plane on the tensor path
                 buf = torch.empty((rows,) + tail, dtype=torch.float16, device="cuda")
                 self.layer.debug_copy(which, buf)
                 torch.cuda.synchronize()
