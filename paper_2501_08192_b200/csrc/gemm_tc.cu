@@ -852,8 +852,12 @@ static cudaError_t launch_instance(cudaLaunchConfig_t &cfg, const GemmTcParams &
 // while the first is in its epilogue).  The packed codes are laid out for this number (pack.cu).
 int gemm_tc_w8_tiles(int NB, int N, int x_fp16)
 {
-    // two tiles whenever the matrix has an even number of them and tensor memory (512 columns) holds two
-    // accumulators plus at least two widened tiles of 2 * 64 columns (128 k)
+    // Narrow batches: one tile, so that two CTAs can share an SM's tensor memory (and the grid has
+    // twice the CTAs to fill the SMs with).  Wide batches: two tiles (one activation tile serves both)
+    // whenever the matrix has an even number of them and tensor memory (512 columns) holds two
+    // accumulators plus at least two widened tiles of 2 * 64 columns (128 k).
+    if (NB <= 32)
+        return 1;
     const int acc = (x_fp16 ? 1 : 2) * NB;
     return (N % (2 * kTcTileM) == 0 && 2 * acc + 2 * 2 * 64 <= 512) ? 2 : 1;
 }
@@ -890,9 +894,14 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     // shared memory is ring: a deep ring is what keeps enough int8 bytes in flight.  One CTA per SM
     // (tensor memory is per SM).
     const int stage_bytes = mt * kATileBytes + planes * a.NB * (a.w8 ? 2 * kTcBlockK : kTcBlockK) * 2;
+    // Two CTAs per SM when each needs at most half of tensor memory (accumulators + at least two widened
+    // tiles in 256 columns) and half of shared memory still holds three stages; else one.
     int w8_slots = 0;
+    bool w8_two = false;
     if (a.w8) {
-        w8_slots = (512 - mt * planes * a.NB) / (mt * 64);
+        const int acc = mt * planes * a.NB;
+        w8_two = acc + 2 * mt * 64 <= 256 && (100 * 1024) / stage_bytes >= 3;
+        w8_slots = ((w8_two ? 256 : 512) - acc) / (mt * 64);
         w8_slots = w8_slots > kTcMaxW8Slots ? kTcMaxW8Slots : w8_slots;
         if (w8_slots < 2)
             return cudaErrorInvalidValue;
@@ -907,7 +916,7 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     // co-resident slots (a second wave doubles the kernel); splits are a power of two <= 8 that leave
     // every rank >= 2 k-blocks.
     int stages = (200 * 1024 - a16_bytes) / stage_bytes, per_sm = 1;
-    if (!a.w8 && (100 * 1024 - a16_bytes) / stage_bytes >= 4) {
+    if (a.w8 ? w8_two : (100 * 1024 - a16_bytes) / stage_bytes >= 4) {
         stages = (100 * 1024 - a16_bytes) / stage_bytes;
         per_sm = 2;
     }
