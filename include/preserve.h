@@ -93,8 +93,8 @@ extern "C" {
                                        of the paper's measurements (Section 4, "Experimental setup"); activations
                                        stay 16-bit (the KV-cache too unless PRESERVE_FLAG_INT8_KV is given).  Both
                                        GEMM paths: the split-K GEMV kernels widen the codes in registers, the
-                                       tcgen05 kernels in shared memory in front of the MMA.  ffn a multiple of
-                                       64; PRESERVE_ESHAPE otherwise */
+                                       tcgen05 kernels into tensor memory (the MMA's A operand).  ffn a
+                                       multiple of 64; PRESERVE_ESHAPE otherwise */
 #define PRESERVE_FLAG_INT8_KV 64u      /* the KV-cache is int8 with one fp32 scale per cached vector, i.e. per
                                        (sequence, kv head, slot): scale = max |u| / 127 over the vector's head_dim
                                        values, code = round-to-nearest-even(u / scale), decided in fp32; a cached
