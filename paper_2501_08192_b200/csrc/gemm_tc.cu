@@ -1,8 +1,8 @@
 // Skinny GEMM on the 5th-generation tensor cores for decode batches >= 16:
 //     y[b, n] = sum_k x[b, k] * W[n, k]
 // computed "swapped": the weight tile is the M = 128 operand, the batch (padded
-// to a multiple of 16, and present twice: the hi and the lo bf16 plane of the
-// activations, x = hi + lo) is the N operand, so one tcgen05.mma per 16 k covers a
+// to a multiple of 16; present twice - the hi and the lo bf16 plane of the
+// activations, x = hi + lo - or once, as one fp16 plane) is the N operand, so one tcgen05.mma per 16 k covers a
 // 128 x 16-k slab of weights for every batch row at once and the CUDA cores stay
 // out of the weight stream entirely.
 //
