@@ -148,6 +148,9 @@ WITHHOLD_CASES = [
     ("gemv", P.WITHHOLD_GEMV, dict(batch=4), 0),
     ("tensor", P.WITHHOLD_TENSOR, dict(batch=20), 0),
     ("attention", P.WITHHOLD_ATTENTION, dict(batch=4), 0),
+    # int8 weights: the GEMV ring of codes, and the tcgen05 ring in front of the widening warps
+    ("gemv_int8", P.WITHHOLD_GEMV, dict(batch=4), P.FLAG_INT8_WEIGHTS),
+    ("tensor_int8", P.WITHHOLD_TENSOR, dict(batch=20), P.FLAG_INT8_WEIGHTS),
 ]
 
 
@@ -158,7 +161,7 @@ def test_a_wait_that_runs_out_is_reported_and_the_handle_survives(oracle, name, 
     clearing it the same handle computes the right result again."""
     shape = I.small_shape(name="timeout_" + name, ctx=150, ctx_min=9, seed=74, **kw)
     t = I.make_layers(shape, 1)[0]
-    ref = oracle.layer_step(shape, t)
+    ref = oracle.layer_step(shape, t, int8_weights=bool(flags & P.FLAG_INT8_WEIGHTS))
     dl = G.DeviceLayer(shape, t, flags=flags)
     stream = torch.cuda.Stream()
     try:
@@ -188,7 +191,7 @@ def test_a_wait_that_runs_out_is_reported_and_the_handle_survives(oracle, name, 
         for n in ("attn_partial", "h2", "mlp_partial"):
             G.assert_close(out[n], ref[n], f"{name} after recovery:{n}")
         # a fresh handle works too
-        d2 = G.DeviceLayer(shape, t)
+        d2 = G.DeviceLayer(shape, t, flags=flags)
         try:
             d2.run()
             assert d2.layer.last_status() == P.PRESERVE_OK
