@@ -25,6 +25,10 @@
 //               epilogue (epilogue.cuh)
 // The kernel is instantiated per (epilogue kind, hand-over form): the tail of one instantiation is
 // a few KB of instructions, which matters for a kernel that runs for microseconds.
+// int8 weights (W8 instantiations): the ring carries the codes of 128 k per stage; the epilogue warps
+// that issue no copies widen them (exactly) to the activations' 16-bit format and store them into
+// tensor memory (tcgen05.st), where the MMA takes them as its A operand - shared memory stays all
+// ring, and nothing widened ever passes through it.  See the converter block below.
 // Every mbarrier wait is bounded; a wait that gives up records a status code,
 // poisons the rest of the CTA's work, and the CTA still reaches every barrier
 // and frees its TMEM.
@@ -188,7 +192,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ uint64_t full[kTcMaxStages], empty[kTcMaxStages], accum_bar, push_bar;
-    __shared__ uint64_t conv[kTcMaxW8Slots], a16_free[kTcMaxW8Slots];   // int8 weights: a widened tile is complete / has been consumed
+    __shared__ uint64_t conv[kTcMaxW8Slots], slot_free[kTcMaxW8Slots];   // int8 weights: a widened tile is complete / has been consumed
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile int poisoned;
     __shared__ EpilogueTables tabs;
@@ -223,7 +227,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             // the epilogue warps that issue no TMA loads widen the tiles: one arrival per warp and tile
             for (int j = 0; j < p.w8_slots; ++j) {
                 mbar_init(&conv[j], 4);        // one converter warp per TMEM lane quadrant
-                mbar_init(&a16_free[j], n_issuers);
+                mbar_init(&slot_free[j], n_issuers);
             }
         }
         mbar_fence_init();
@@ -345,7 +349,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             }
             tc_commit(&empty[st]);      // slot is free once these MMAs have read it
             if (W8) {
-                tc_commit(&a16_free[j]);
+                tc_commit(&slot_free[j]);
                 if (++j == p.w8_slots) { j = 0; phj ^= 1; }
             }
             if (++st == p.stages) { st = 0; ph ^= 1; }
@@ -462,7 +466,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 if (lane == 0) {
                     ok = mbar_wait(&full[st], ph, p.status, ST_TIMEOUT_FULL) ? 1 : 0;
                     if (ok && reuse)
-                        ok = mbar_wait(&a16_free[j], phj ^ 1, p.status, ST_TIMEOUT_EMPTY) ? 1 : 0;
+                        ok = mbar_wait(&slot_free[j], phj ^ 1, p.status, ST_TIMEOUT_EMPTY) ? 1 : 0;
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) { poisoned = 1; break; }
