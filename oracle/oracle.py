@@ -255,18 +255,21 @@ def layer_step(shape, t: Dict[str, np.ndarray], partials_in=None, residual_in=No
     return res
 
 
-def layer_chain(shape, layers: Sequence[Dict[str, np.ndarray]]) -> List[Dict[str, np.ndarray]]:
-    """A chain of layers: layer l+1 takes partials_in[0] = mlp_partial_l and residual_in = h2_l."""
+def layer_chain(shape, layers: Sequence[Dict[str, np.ndarray]], int8_weights: bool = False,
+                kv8: Optional[Sequence[Dict[str, np.ndarray]]] = None) -> List[Dict[str, np.ndarray]]:
+    """A chain of layers: layer l+1 takes partials_in[0] = mlp_partial_l and residual_in = h2_l.
+    kv8: one int8 cache per layer (see layer_step)."""
     outs: List[Dict[str, np.ndarray]] = []
     for i, t in enumerate(layers):
+        kv = None if kv8 is None else kv8[i]
         if i == 0:
-            outs.append(layer_step(shape, t))
+            outs.append(layer_step(shape, t, int8_weights=int8_weights, kv8=kv))
             continue
         prev = outs[-1]
         parts = (np.ascontiguousarray(t["partials_in"], np.uint16).astype(np.uint32)
                  << np.uint32(16)).view(np.float32).copy()
         parts[0] = prev["mlp_partial"]
-        outs.append(layer_step(shape, t, partials_in=parts, residual_in=prev["h2"]))
+        outs.append(layer_step(shape, t, partials_in=parts, residual_in=prev["h2"], int8_weights=int8_weights, kv8=kv))
     return outs
 
 

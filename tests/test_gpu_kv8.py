@@ -194,3 +194,24 @@ def test_int8_cache_layout_and_byte_accounting():
         assert plan.cpu().numpy().reshape(2, 3).tolist() == [list(r) for r in info.planned_bytes]
     finally:
         dl.close()
+
+
+@pytest.mark.parametrize("batch", [6, 24], ids=["gemv", "tensor"])
+def test_int8_linked_chain_matches_the_oracle_chain(oracle, batch):
+    """Three layers linked output to input (fp32 hand-over inside the library), int8 weights and int8
+    cache together, against the oracle stepping the same chain."""
+    shape = I.small_shape(name="kv8_w8_chain", batch=batch, ctx=140, ctx_min=20, layers=3, seed=260)
+    layers = I.make_layers(shape)
+    kvs = [I.make_int8_cache(shape, t["ctx_len"], seed=10 + i) for i, t in enumerate(layers)]
+    refs = oracle.layer_chain(shape, layers, int8_weights=True, kv8=kvs)
+    dls = [G.DeviceLayer(shape, t, flags=P.FLAG_INT8_WEIGHTS, kv8=kv) for t, kv in zip(layers, kvs)]
+    try:
+        P.preserve_decode_chain([d.layer for d in dls], [d.io for d in dls], link=True)
+        for i, (dl, ref) in enumerate(zip(dls, refs)):
+            assert dl.layer.last_status() == P.PRESERVE_OK
+            out = dl.outputs()
+            for name in ("attn_partial", "h2", "mlp_partial"):
+                G.assert_close(out[name], ref[name], f"chain layer {i}:{name}")
+    finally:
+        for d in dls:
+            d.close()
