@@ -872,7 +872,8 @@ def run_decode_loop(P, I, torch, args, stream):
     idx = args.config if args.config >= 0 else 1
     n_layers, n_tokens = args.layers, max(args.steps, 64)
     l2 = torch.cuda.get_device_properties(0).L2_cache_size
-    wl = Workload(P, I, torch, idx, 0, l2, rotation=n_layers)
+    vflags = (P.FLAG_INT8_KV if args.int8_kv else 0) | (P.FLAG_INT8_WEIGHTS if args.int8_weights else 0)
+    wl = Workload(P, I, torch, idx, 0, l2, rotation=n_layers, flags=vflags)
     shape = wl.shape
     # start n_tokens + 8 below the configured context so that the contexts can advance inside the cache
     start = np.maximum(wl.ctx_host - (n_tokens + 8), 1).astype(np.int32)
@@ -915,6 +916,7 @@ def run_decode_loop(P, I, torch, args, stream):
         res[name] = out
     status = max(L.last_status() for L in wl.layers)
     print(json.dumps({"mode": "decode-loop", "layers": n_layers, "tokens": n_tokens,
+                      "precision": "bf16" + (", int8 KV-cache" if args.int8_kv else "") + (", int8 weights" if args.int8_weights else ""),
                       "workload": f"{n_layers} x configs[{idx}] {shape.name} (linked chain), contexts "
                                   f"{int(start.min())}..{int(start.max())} advancing by one per token",
                       "results": res, "device_status": status}), flush=True)
