@@ -881,11 +881,12 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     p.inject = a.inject;
     const int planes = a.x_fp16 ? 1 : 2;
     p.planes = planes;
-    // Two 128-row weight tiles per CTA share one activation tile when the batch is wide enough for
-    // the activation tile (2 * NB rows) to weigh as much as a weight tile: halves the L2->SM traffic
-    // of the activations, which every CTA re-reads.
+    // Two 128-row weight tiles per CTA share one activation tile when the activation tile (planes * NB
+    // rows) weighs about as much as a weight tile: halves the L2->SM traffic of the activations, which
+    // every CTA re-reads.  With a single fp16 plane of 64 rows it does not: one tile per CTA then gives
+    // twice the CTAs (two per SM) and measured 1-1.5 us less on the O and down projections of config 4.
     const int mt = a.w8 ? gemm_tc_w8_tiles(a.NB, a.N, a.x_fp16)
-                        : ((a.NB >= 48 && a.N % (2 * kTcTileM) == 0 && a.w_map256) ? 2 : 1);
+                        : ((planes * a.NB >= 96 && a.N % (2 * kTcTileM) == 0 && a.w_map256) ? 2 : 1);
     if (a.w8 && (!a.w8_codes || !a.scales))
         return cudaErrorInvalidValue;
     p.w8_codes = static_cast<const uint8_t *>(a.w8_codes);
