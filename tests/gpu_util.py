@@ -90,7 +90,6 @@ class DeviceLayer:
             self.k_cache = bits_to_cuda(t["k_cache"])
             self.v_cache = bits_to_cuda(t["v_cache"])
         else:
-            assert max_batch is None or max_batch == shape.batch
             self.k_cache = kv8_buffer(self.cfg, kv8["k_codes"], kv8["k_scales"])
             self.v_cache = kv8_buffer(self.cfg, kv8["v_codes"], kv8["v_scales"])
         self.ctx_host = np.ascontiguousarray(t["ctx_len"], dtype=np.int32)

@@ -215,3 +215,23 @@ def test_int8_linked_chain_matches_the_oracle_chain(oracle, batch):
     finally:
         for d in dls:
             d.close()
+
+
+def test_int8_cache_with_a_smaller_batch_than_max_batch(oracle):
+    """A step of 5 sequences on handles created for 12 (GEMV path) and 40 (tensor path): the cache buffers
+    have the layout of the larger batch (streams of the first sequences first), int8 weights as well."""
+    shape = I.small_shape(name="kv8_b5_of_more", batch=5, ctx=77, ctx_min=3, seed=253)
+    t = I.make_layers(shape, 1)[0]
+    kv = I.make_int8_cache(shape, t["ctx_len"])
+    ref = oracle.layer_step(shape, t, int8_weights=True, kv8=kv)
+    for max_batch in (12, 40):
+        dl = G.DeviceLayer(shape, t, flags=P.FLAG_INT8_WEIGHTS, max_batch=max_batch, kv8=kv)
+        try:
+            dl.run()
+            assert dl.layer.last_status() == P.PRESERVE_OK
+            out = dl.outputs()
+            for name in ("attn_partial", "h2", "mlp_partial"):
+                G.assert_close(out[name], ref[name], f"max_batch {max_batch}:{name}")
+            check_appended(dl, ref, f"max_batch {max_batch}")
+        finally:
+            dl.close()
