@@ -235,3 +235,32 @@ def test_int8_cache_with_a_smaller_batch_than_max_batch(oracle):
             check_appended(dl, ref, f"max_batch {max_batch}")
         finally:
             dl.close()
+
+
+def test_int8_host_buffer_entry_point_matches_the_device_path(oracle):
+    """preserve_decode_step_host over the int8 cache with int8 weights (the cache stays on the device):
+    bit-identical to the device-buffer call on the same inputs."""
+    shape = I.small_shape(name="kv8_host_io", batch=6, ctx=150, ctx_min=3, seed=254)
+    t = I.make_layers(shape, 1)[0]
+    kv = I.make_int8_cache(shape, t["ctx_len"])
+    dl = G.DeviceLayer(shape, t, flags=P.FLAG_INT8_WEIGHTS, kv8=kv)
+    try:
+        k0, v0 = dl.k_cache.clone(), dl.v_cache.clone()
+        dl.run()
+        want = dl.output_bits()
+        dl.k_cache.copy_(k0)
+        dl.v_cache.copy_(v0)
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
+        parts = [pin(t["partials_in"][p]) for p in range(shape.tp_degree)]
+        peers = [pin(t["attn_peer_partials"][p]) for p in range(shape.tp_degree - 1)]
+        resid = pin(t["residual_in"])
+        r_out = torch.zeros((shape.batch, shape.hidden), dtype=torch.int16).pin_memory()
+        m_out = torch.zeros((shape.batch, shape.hidden), dtype=torch.int16).pin_memory()
+        hio = P.make_host_io(dl.cfg, shape.batch, dl.ctx_host, parts, peers, resid, dl.k_cache, dl.v_cache, r_out, m_out)
+        dl.layer.decode_step_host(hio)
+        torch.cuda.synchronize()
+        assert dl.layer.last_status() == P.PRESERVE_OK
+        assert np.array_equal(r_out.numpy().view(np.uint16), want["h2"])
+        assert np.array_equal(m_out.numpy().view(np.uint16), want["mlp_partial"])
+    finally:
+        dl.close()
