@@ -450,6 +450,7 @@ def bench_config(P, I, torch, dist, args, idx, rank, local_rank, world, stream, 
                 row[name + "_us_per_layer"] = round(ms8 * 1e3 / wl8.R, 3)
                 row[name + "_gbs"] = round(alg8 * wl8.R / (ms8 * 1e-3) / 1e9, 1)
             row["speedup_vs_bf16"] = round(us(ms_early) / row["early_launch_only_us_per_layer"], 4)
+            row["speedup_early_vs_off"] = round(row["off_us_per_layer"] / row["early_launch_only_us_per_layer"], 4)
             if vflags & P.FLAG_INT8_KV:
                 with torch.cuda.stream(stream):
                     attn8()
