@@ -826,7 +826,8 @@ def run_timeline(P, I, torch, args, stream):
     predecessor returned, when its operand stream ended, when it ended."""
     idx = args.config if args.config >= 0 else HEADLINE_CONFIG
     l2 = torch.cuda.get_device_properties(0).L2_cache_size
-    wl = Workload(P, I, torch, idx, 0, l2, args.rotation)
+    vflags = (P.FLAG_INT8_KV if args.int8_kv else 0) | (P.FLAG_INT8_WEIGHTS if args.int8_weights else 0)
+    wl = Workload(P, I, torch, idx, 0, l2, args.rotation, flags=vflags)
     if args.budget_bytes >= 0:
         wl.set_budget(args.budget_bytes)
     for L in wl.layers:
@@ -861,6 +862,7 @@ def run_timeline(P, I, torch, args, stream):
     layer_us = float(np.mean(a[:, -1, 3] - a[:, 0, 2])) / 1e3
     print(json.dumps({"mode": "timeline", "config_index": idx, "name": wl.shape.name, "samples": len(rows),
                       "budget_bytes": int(wl.layers[0].get_info().prefetch_budget),
+                      "precision": "bf16" + (", int8 KV-cache" if args.int8_kv else "") + (", int8 weights" if args.int8_weights else ""),
                       "first_wait_return_to_last_end_us": round(layer_us, 2), "kernels": table}), flush=True)
     wl.close()
 

@@ -73,6 +73,7 @@ struct GemmTcParams {
     int epi_warps;      // 8 or 16
     int producers;      // 1..kTcMaxProducers threads that issue the ring's TMA loads (stage uses dealt round-robin)
     int w8;             // the weight tiles arrive as int8 codes and are widened into tensor memory (the MMA's A operand)
+    int w8_early;       // w8: the first ring fill's activation tiles complete their own barrier (codes widened before the wait)
     int w8_slots;       // 2..kTcMaxW8Slots widened tiles in tensor memory (mt * 32 columns each) behind the accumulators
     const float *wscale;  // w8: one fp32 scale per packed weight row
     const uint8_t *w8_codes;  // w8: the codes, one contiguous block of mt * 128 rows x 64 bytes per (tile, k-block)
@@ -186,13 +187,17 @@ __device__ __forceinline__ void tc_ld_wait(uint32_t (&a)[16], uint32_t (&b)[16])
 
 // KIND: the epilogue; PUSH: the split-K hand-over (0 pull, 1 st.async, 2 bulk copies) - template
 // arguments, so that each instantiation carries a single tail and its instructions stay close together.
-template <int KIND, int PUSH, bool W8 = false>
+template <int KIND, int PUSH, bool W8 = false, bool EARLY = false>
 __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_constant__ GemmTcParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ uint64_t full[kTcMaxStages], empty[kTcMaxStages], accum_bar, push_bar;
     __shared__ uint64_t conv[kTcMaxW8Slots], slot_free[kTcMaxW8Slots];   // int8 weights: a widened tile is complete / has been consumed
+    // int8 weights: the activation tiles of the ring's FIRST fill complete a barrier of their own, so that
+    // those codes - which land while the kernel in front is still running - are widened before the
+    // activations exist (later uses of a stage complete one barrier with both, as without int8)
+    __shared__ uint64_t fullb[(W8 && EARLY) ? kTcMaxStages : 1];
     __shared__ uint32_t tmem_base_s;
     __shared__ volatile int poisoned;
     __shared__ EpilogueTables tabs;
@@ -204,6 +209,8 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     // the tensor pipe's front end spend per stage does not depend on what the stage carries, and an int8
     // stage of 64 k carries half the bytes
     constexpr int kBlk = W8 ? 2 * kTcBlockK : kTcBlockK;
+    // int8 weights, narrow batches: the codes of the ring's first fill are widened before the activations exist
+    constexpr bool kEarly = W8 && EARLY;
     const int a_bytes = p.mt * kATileBytes;
     const int b_bytes = p.planes * p.NB * kBlk * 2;
     const int stage_bytes = a_bytes + b_bytes;
@@ -223,6 +230,10 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             mbar_init(&empty[i], n_issuers);
         }
         mbar_init(&accum_bar, n_issuers);
+        if (kEarly) {
+            for (int i = 0; i < p.stages; ++i)
+                mbar_init(&fullb[i], 1);
+        }
         if (W8) {
             // the epilogue warps that issue no TMA loads widen the tiles: one arrival per warp and tile
             for (int j = 0; j < p.w8_slots; ++j) {
@@ -267,7 +278,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         const int n_kb = kb1 - kb0;
         const int pre = n_kb < p.stages ? n_kb : p.stages;
         for (int i = prod; i < pre; i += NP) {
-            mbar_expect_tx(&full[i], stage_bytes);
+            mbar_expect_tx(&full[i], kEarly ? a_bytes : stage_bytes);
             if (p.inject == INJECT_TC_RING && i == 0 && tile == 0 && s == 0)
                 continue;
             if constexpr (W8)
@@ -280,14 +291,20 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         pdl_wait();
         if (prod == 0)
             trace_waited(p.trace);
-        auto load_b = [&](int st_, int kb_) {
+        auto load_b = [&](int st_, int kb_, bool first_fill) {
             uint8_t *b_dst = smem + (size_t)st_ * stage_bytes + a_bytes;
-            tma_load_2d(b_dst, &p.x_map, kb_ * kBlk, 0, &full[st_]);
-            if constexpr (W8)      // second 64-k box of the stage
-                tma_load_2d(b_dst + b_bytes / 2, &p.x_map, kb_ * kBlk + kTcBlockK, 0, &full[st_]);
+            if constexpr (W8) {    // two 64-k boxes
+                uint64_t *bar = (kEarly && first_fill) ? &fullb[st_] : &full[st_];
+                if (kEarly && first_fill)
+                    mbar_expect_tx(bar, b_bytes);
+                tma_load_2d(b_dst, &p.x_map, kb_ * kBlk, 0, bar);
+                tma_load_2d(b_dst + b_bytes / 2, &p.x_map, kb_ * kBlk + kTcBlockK, 0, bar);
+            } else {
+                tma_load_2d(b_dst, &p.x_map, kb_ * kBlk, 0, &full[st_]);
+            }
         };
         for (int i = prod; i < pre; i += NP)
-            load_b(i, kb0 + i);
+            load_b(i, kb0 + i, kEarly);
         int it = prod;
         while (it < pre)
             it += NP;
@@ -303,7 +320,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 bulk_load_hint(a_dst, p.w8_codes + ((size_t)tile * p.kblocks + kb) * a_bytes, a_bytes, &full[st], pol);
             else
                 tma_load_2d_hint(a_dst, &p.w_map, kb * kTcBlockK, tile * p.mt * kTcTileM, &full[st], pol);
-            load_b(st, kb);
+            load_b(st, kb, false);
             st += NP;
             while (st >= p.stages) {
                 st -= p.stages;
@@ -325,6 +342,9 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             // (int8 weights: the widened tile of this use completes after the stage has landed)
             if (!(W8 ? mbar_wait(&conv[j], phj, p.status, ST_TIMEOUT_FULL)
                        : mbar_wait(&full[st], ph, p.status, ST_TIMEOUT_FULL))) { poisoned = 1; ok = false; break; }
+            if constexpr (kEarly) {      // ... and, in the ring's first fill, the stage's activation tiles
+                if (kb - kb0 < p.stages && !mbar_wait(&fullb[st], 0, p.status, ST_TIMEOUT_FULL)) { poisoned = 1; ok = false; break; }
+            }
             tc_fence_after();
             const uint32_t st_addr = smem_u32(smem + (size_t)st * stage_bytes);
             const uint64_t bdesc = make_smem_desc(st_addr + a_bytes);
@@ -373,6 +393,15 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     const int row = lane_grp * 32 + lane;   // row of the tile
     const int nchunks = p.NB / 16;
     const int sub = is_epi ? (warp - 2) >> 2 : 0;        // which of the lane group's warps this is
+    // int8 weights: every accumulator row (= packed weight row) is multiplied by its scale as it leaves
+    // TMEM.  The scales are weights - fetched here, ahead of the stream, not behind the last MMA where
+    // their memory round trip would sit on the kernel's tail.
+    float wsc[2] = {1.f, 1.f};
+    if (W8 && is_epi) {
+        wsc[0] = p.wscale[(size_t)(tile * p.mt) * kTcTileM + row];
+        if (p.mt == 2)
+            wsc[1] = p.wscale[(size_t)(tile * p.mt + 1) * kTcTileM + row];
+    }
     const int kSubs = ((int)blockDim.x / 32 - 2) / 4;    // warps per lane group
     const int par = lane & 1;
     // Rotary factors of this thread's first two finish iterations of a one-sided split-K reduction
@@ -512,13 +541,6 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
     float *red = reinterpret_cast<float *>(smem);      // [mt][NB][128] fp32, reuses the ring
 
-    // int8 weights: every accumulator row (= packed weight row) is multiplied by its scale as it leaves TMEM
-    float wsc[2] = {1.f, 1.f};
-    if (W8 && is_epi) {
-        wsc[0] = p.wscale[(size_t)(tile * p.mt) * kTcTileM + row];
-        if (p.mt == 2)
-            wsc[1] = p.wscale[(size_t)(tile * p.mt + 1) * kTcTileM + row];
-    }
     auto wscale_of = [&](int m) -> float {
         if constexpr (W8)
             return m ? wsc[1] : wsc[0];
@@ -658,6 +680,9 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 finish(std::integral_constant<int, 16>());
         }
         cluster_wait();
+        // (failure path: every peer has issued its copies by now; let those in flight land before the exit)
+        if (poisoned && threadIdx.x == 0)
+            mbar_wait(&push_bar, 0, p.status, ST_TIMEOUT_MMA);
     } else if (PUSH == 1 && p.splits > 1) {
         // Split-K across the cluster, one-sided reduce-scatter: rank q finishes columns [q * cols,
         // (q + 1) * cols).  Every rank stores those columns of its partial tile into rank q's receive
@@ -823,6 +848,19 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     }
     tc_fence_before();
     __syncthreads();
+    if (PUSH == 1 && p.splits > 1 && poisoned) {
+        // A wait of this CTA ran out, so it may be about to leave before every peer has stored its share
+        // into this CTA's receive area - and a store into the shared memory of a CTA that has exited is
+        // a fault.  Stay until every peer has either left (its stores were issued before that) or
+        // reached this point too, then give the stores in flight a bounded time to land.  (A CTA whose
+        // waits all succeeded has received everything and may simply leave: the barrier counts only
+        // threads that have not exited.)
+        cluster_arrive_relaxed();
+        cluster_wait();
+        if (threadIdx.x == 0)
+            mbar_wait(&push_bar, 0, p.status, ST_TIMEOUT_MMA);
+        __syncthreads();
+    }
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols)
                      : "memory");
@@ -830,11 +868,11 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     trace_end(p.trace);
 }
 
-template <int KIND, int PUSH, bool W8 = false>
+template <int KIND, int PUSH, bool W8 = false, bool EARLY = false>
 static cudaError_t launch_instance(cudaLaunchConfig_t &cfg, const GemmTcParams &p, size_t smem)
 {
     static PerDeviceSize smem_limit, np_set;      // per instantiation and device
-    cudaError_t e = ensure_dynamic_smem(k_gemm_tcgen05<KIND, PUSH, W8>, smem_limit, smem);
+    cudaError_t e = ensure_dynamic_smem(k_gemm_tcgen05<KIND, PUSH, W8, EARLY>, smem_limit, smem);
     if (e != cudaSuccess)
         return e;
     if (p.splits > 8) {
@@ -842,13 +880,13 @@ static cudaError_t launch_instance(cudaLaunchConfig_t &cfg, const GemmTcParams &
         if (dev < 0)
             return cudaErrorInvalidDevice;
         if (!np_set.v[dev]) {
-            e = cudaFuncSetAttribute(k_gemm_tcgen05<KIND, PUSH, W8>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            e = cudaFuncSetAttribute(k_gemm_tcgen05<KIND, PUSH, W8, EARLY>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
             if (e != cudaSuccess)
                 return e;
             np_set.v[dev] = 1;
         }
     }
-    return cudaLaunchKernelEx(&cfg, k_gemm_tcgen05<KIND, PUSH, W8>, p);
+    return cudaLaunchKernelEx(&cfg, k_gemm_tcgen05<KIND, PUSH, W8, EARLY>, p);
 }
 
 // int8 weights: 128-row weight tiles per CTA (1 or 2).  The two widened tiles behind the ring cost
@@ -912,6 +950,8 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
             return cudaErrorInvalidValue;
     }
     p.w8_slots = w8_slots;
+    // (measured: pays for narrow batches - two CTAs per SM, few stages per CTA - and costs ~1 % on wide ones)
+    p.w8_early = a.w8 && w8_two;
     const int a16_bytes = 0;
     p.w8 = a.w8;
     p.wscale = a.scales;
@@ -1008,7 +1048,8 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     const int push = splits > 1 ? p.push : 0;
 #define PRSV_TC_CASE(KIND, PUSH)                                   \
     if (a.epi.kind == (KIND) && push == (PUSH))                    \
-        return a.w8 ? launch_instance<KIND, PUSH, true>(cfg, p, smem) : launch_instance<KIND, PUSH, false>(cfg, p, smem);
+        return a.w8 ? (p.w8_early ? launch_instance<KIND, PUSH, true, true>(cfg, p, smem) : launch_instance<KIND, PUSH, true, false>(cfg, p, smem)) \
+                    : launch_instance<KIND, PUSH, false>(cfg, p, smem);
     PRSV_TC_CASE(EPI_PLAIN, 0) PRSV_TC_CASE(EPI_PLAIN, 1) PRSV_TC_CASE(EPI_PLAIN, 2)
     PRSV_TC_CASE(EPI_QKV, 0) PRSV_TC_CASE(EPI_QKV, 1) PRSV_TC_CASE(EPI_QKV, 2)
     PRSV_TC_CASE(EPI_SWIGLU, 0) PRSV_TC_CASE(EPI_SWIGLU, 1) PRSV_TC_CASE(EPI_SWIGLU, 2)

@@ -95,6 +95,7 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
     __shared__ uint64_t bars[kGemvWarps][kRingSlots];
     __shared__ uint64_t push_bar;
     __shared__ EpilogueTables tabs;
+    __shared__ float scale_s[W8 ? kGemvWarps * RB * 16 : 1];   // W8: the scales of the group's rows
     extern __shared__ uint8_t gemv_smem_raw[];
     uint8_t *wsm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(gemv_smem_raw) + 127) & ~uintptr_t(127));
 
@@ -197,11 +198,22 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
         }
     };
 
+    // W8: the scales of a group's rows are weights - fetched ahead of the stream (the first group's even
+    // ahead of the wait), not behind the reduction where their memory round trip would sit on the tail
+    auto load_scales = [&](int grp) {
+        if constexpr (W8) {
+            if (grp < p.groups)
+                for (int i = threadIdx.x; i < rbs_per_cta * 16; i += blockDim.x)
+                    scale_s[i] = p.scales[(size_t)grp * rbs_per_cta * 16 + i];
+        }
+    };
+    load_scales(blockIdx.x);
     pdl_wait();   // x is produced by the previous kernel of the stream
     trace_waited(p.trace);
 
     uint32_t n_consumed = 0;
     bool ok = true;
+    bool push_short = false;      // rank 0: the wait for the other ranks' partial sums ran out
     for (int grp = blockIdx.x; grp < p.groups; grp += gridDim.x) {
         float acc[RB][MMA ? NT : 2 * NB][MMA ? 4 : 1];
 #pragma unroll
@@ -365,7 +377,9 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
                 for (int i = threadIdx.x; i < part_floats / 4; i += blockDim.x)
                     st_async_v4(dst + i * 16, src[i], bar);
             } else {
-                ok = mbar_wait(&push_bar, 0, p.status, ST_TIMEOUT_FULL) && ok;
+                const bool got = mbar_wait(&push_bar, 0, p.status, ST_TIMEOUT_FULL);
+                push_short = !got;
+                ok = got && ok;
                 for (int i = threadIdx.x; i < n_out; i += blockDim.x) {
                     const int b = i % NB, r = (i / NB) % 8, rl = i / (8 * NB);
                     if (b >= p.B)
@@ -376,9 +390,8 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
                         v1 += recv[(size_t)(q - 1) * part_floats + (rl * 16 + r + 8) * NB + b];
                     }
                     if constexpr (W8) {
-                        const int prow = (grp * rbs_per_cta + rl) * 16 + r;
-                        v0 *= p.scales[prow];
-                        v1 *= p.scales[prow + 8];
+                        v0 *= scale_s[rl * 16 + r];
+                        v1 *= scale_s[rl * 16 + r + 8];
                     }
                     apply_epilogue(p.epi, tabs, b, false, p.N, p.b0 + b, (grp * rbs_per_cta + rl) * 8 + r, v0, v1);
                 }
@@ -403,13 +416,13 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
                         v1 += remote[q][(rl * 16 + r + 8) * NB + b];
                     }
                 if constexpr (W8) {
-                    const int prow = (grp * rbs_per_cta + rl) * 16 + r;
-                    v0 *= p.scales[prow];
-                    v1 *= p.scales[prow + 8];
+                    v0 *= scale_s[rl * 16 + r];
+                    v1 *= scale_s[rl * 16 + r + 8];
                 }
                 apply_epilogue(p.epi, tabs, b, false, p.N, p.b0 + b, (grp * rbs_per_cta + rl) * 8 + r, v0, v1);
             }
             cluster.sync();   // peers' shared memory must outlive the reads; also fences red/cta_part reuse
+            load_scales(grp + gridDim.x);
         } else {
             __syncthreads();
             for (int i = threadIdx.x; i < n_out; i += blockDim.x) {
@@ -418,12 +431,26 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
                     continue;
                 float v0 = cta_part[rl][r][b], v1 = cta_part[rl][r + 8][b];
                 if constexpr (W8) {
-                    const int prow = (grp * rbs_per_cta + rl) * 16 + r;
-                    v0 *= p.scales[prow];
-                    v1 *= p.scales[prow + 8];
+                    v0 *= scale_s[rl * 16 + r];
+                    v1 *= scale_s[rl * 16 + r + 8];
                 }
                 apply_epilogue(p.epi, tabs, b, false, p.N, p.b0 + b, (grp * rbs_per_cta + rl) * 8 + r, v0, v1);
             }
+            __syncthreads();
+            load_scales(grp + gridDim.x);
+        }
+    }
+    if (p.push && s == 0) {
+        // Rank 0 gave up waiting for a rank's partial sums: that rank may still store them into this
+        // CTA's shared memory, and a store into a CTA that has exited is a fault.  Stay until every other
+        // rank has left (its stores were issued before that), then give the stores in flight a bounded
+        // time to land.  (The barrier counts only threads that have not exited; the other ranks never
+        // wait on it.)
+        if (__syncthreads_or(push_short ? 1 : 0)) {
+            cluster_arrive_relaxed();
+            cluster_wait();
+            if (threadIdx.x == 0)
+                mbar_wait(&push_bar, 0, p.status, ST_TIMEOUT_FULL);
             __syncthreads();
         }
     }
@@ -444,8 +471,10 @@ static cudaError_t launch_variant(GemvParams &p, int sm_count, int pdl, cudaStre
     // add splits only while the grid stays within the co-resident CTAs; groups beyond the grid
     // become further loop iterations.  Depends only on the shapes and the SM count, never on the
     // prefetch setting.
+    // (an int8 tile covers 64 k, as much as two 16-bit tiles: one per warp is the same slice of k)
+    constexpr int kMinChunks = W8 ? 1 : 2;
     int wk = kGemvWarps;
-    while (wk > 1 && p.kchunks / wk < 2 && p.row_blocks % (2 * RB * kGemvWarps / wk) == 0) wk /= 2;
+    while (wk > 1 && p.kchunks / wk < kMinChunks && p.row_blocks % (2 * RB * kGemvWarps / wk) == 0) wk /= 2;
     p.warps_k = wk;
     p.groups = p.row_blocks / (kGemvWarps / wk * RB);
     // Two CTA slots per SM for every matrix (64 KiB rings, <= 128 registers).  A small projection whose
@@ -454,7 +483,7 @@ static cudaError_t launch_variant(GemvParams &p, int sm_count, int pdl, cudaStre
     // the weights, which are in the rings by then - is what such a kernel's time consists of.
     const int slots_total = 2 * sm_count;
     int splits = 1;
-    while (splits < 8 && p.groups * splits * 2 <= slots_total && p.kchunks / (wk * splits * 2) >= 2) splits *= 2;
+    while (splits < 8 && p.groups * splits * 2 <= slots_total && p.kchunks / (wk * splits * 2) >= kMinChunks) splits *= 2;
     p.splits = splits;
     int clusters = slots_total / p.splits;
     if (clusters > p.groups) clusters = p.groups;

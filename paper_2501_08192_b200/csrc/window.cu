@@ -276,10 +276,12 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
     }
     __syncthreads();
     float row_total = total;
+    bool recv_short = false;     // the wait for the other CTAs' sums ran out
     if (p.cluster > 1) {
         // sum of the slices in rank order (the same order in every CTA of the row)
         row_total = 0.f;
-        if (mbar_wait(&recv_bar, 0, p.status, ST_TIMEOUT_FULL))
+        recv_short = !mbar_wait(&recv_bar, 0, p.status, ST_TIMEOUT_FULL);
+        if (!recv_short)
             for (int q = 0; q < p.cluster; ++q)
                 row_total += recv[q];
     }
@@ -349,6 +351,20 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
                 __threadfence();
                 atomicAdd(p.comm_epoch, 1u);
             }
+        }
+    }
+    if (p.cluster > 1) {
+        // This CTA gave up waiting for a peer's sum: the peer may still store it into this CTA's shared
+        // memory, and a store into a CTA that has exited is a fault.  Stay until every peer has left or
+        // reached this point too (its stores were issued before), then give the stores in flight a
+        // bounded time to land.  (The barrier counts only threads that have not exited; a CTA whose wait
+        // succeeded has received everything and simply leaves.)
+        if (__syncthreads_or(recv_short ? 1 : 0)) {
+            cluster_arrive_relaxed();
+            cluster_wait();
+            if (threadIdx.x == 0)
+                mbar_wait(&recv_bar, 0, p.status, ST_TIMEOUT_FULL);
+            __syncthreads();
         }
     }
     trace_end(p.trace);
