@@ -49,7 +49,7 @@ NCU_TRAFFIC = {
                                     "down projection's weights that this kernel's CTAs prefetch into L2)"),
     ("gate_up_proj", 2): (121910000, "profiles/ncu_full_gemm_tcgen05_config3_small.md"),
     ("attn_splitkv", 4): (542870000, "profiles/ncu_full_attn_splitkv_config5.md"),
-    ("gate_up_proj", 3): (240500736, "profiles/ncu_full_gemm_tcgen05_gate_up_config4.md (read 237.04 MB + write 3.46 MB, "
+    ("gate_up_proj", 3): (240296448, "profiles/ncu_full_gemm_tcgen05_gate_up_config4.md (read 236.03 MB + write 4.27 MB, "
                                      "full-size launch, 2-layer rotation)"),
 }
 
