@@ -680,9 +680,15 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 finish(std::integral_constant<int, 16>());
         }
         cluster_wait();
-        // (failure path: every peer has issued its copies by now; let those in flight land before the exit)
-        if (poisoned && threadIdx.x == 0)
+        // (failure path: every peer has issued its copies by now; let those in flight land before the exit,
+        // and give this CTA's own copies - whose source is its shared memory, and whose receivers may have
+        // arrived at the barrier without them - 20 us to leave it)
+        if (poisoned && threadIdx.x == 0) {
             mbar_wait(&push_bar, 0, p.status, ST_TIMEOUT_MMA);
+            const long long t_lin = gtime();
+            while (gtime() - t_lin < 20000)
+                __nanosleep(1000);
+        }
     } else if (PUSH == 1 && p.splits > 1) {
         // Split-K across the cluster, one-sided reduce-scatter: rank q finishes columns [q * cols,
         // (q + 1) * cols).  Every rank stores those columns of its partial tile into rank q's receive

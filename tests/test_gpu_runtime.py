@@ -147,6 +147,8 @@ WITHHOLD_CASES = [
     ("window", P.WITHHOLD_WINDOW, dict(batch=3, hidden=2048, ffn=256), 0),
     ("gemv", P.WITHHOLD_GEMV, dict(batch=4), 0),
     ("tensor", P.WITHHOLD_TENSOR, dict(batch=20), 0),
+    # batch 64: the split-K hand-over by bulk copies out of the senders' shared memory
+    ("tensor_wide", P.WITHHOLD_TENSOR, dict(batch=64), 0),
     ("attention", P.WITHHOLD_ATTENTION, dict(batch=4), 0),
     # int8 weights: the GEMV ring of codes, and the tcgen05 ring in front of the widening warps
     ("gemv_int8", P.WITHHOLD_GEMV, dict(batch=4), P.FLAG_INT8_WEIGHTS),
