@@ -183,7 +183,7 @@ typedef struct {
     int32_t uses_tensor_path;         /* 1: tcgen05 GEMM (max_batch >= 16); 0: split-K GEMV */
     int32_t activation_rows;          /* rows per plane of the internal split activations (see preserve_debug_copy) */
     int32_t plan_mode;
-    int32_t normed_activations_fp16;  /* 1: o, x2 and a are kept as one fp16 plane each (tensor path), see preserve_debug_copy */
+    int32_t normed_activations_fp16;  /* 1 (tensor path): o, x2 and a are one fp16 plane each, x two fp16 planes; see preserve_debug_copy */
     uint64_t prefetch_budget;         /* bytes per window                               */
     uint64_t weight_bytes[4];         /* Wqkv, Wo, Wgate|up, Wdown                      */
     uint64_t kv_bytes;                /* K+V bytes read by the last planned step        */
@@ -355,7 +355,8 @@ PRESERVE_API int preserve_last_cuda_error(const preserve_layer_t *layer);
  * preserve_layer_get_info); the copy delivers that layout as is.  Exception: where
  * normed_activations_fp16 is set (tensor path), o, x2 and a - an attention output, an RMSNorm output
  * and the SwiGLU output (clamped to +-65504): bounded values - are ONE fp16 plane each,
- * [activation_rows][...] at the start of the buffer.  6: uint64 [2][3], the
+ * [activation_rows][...] at the start of the buffer, and the two planes of x are fp16 (hi = fp16(x),
+ * lo = fp16(x - hi)).  6: uint64 [2][3], the
  * bytes per node that the prefetch kernels of the last step decided to bring in - the same
  * walk as preserve_layer_get_info's planned_bytes, evaluated on the device from the device
  * copy of ctx_len (a window whose host plan is empty launches no kernel and keeps its old

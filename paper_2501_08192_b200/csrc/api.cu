@@ -393,10 +393,11 @@ int launch_gemm(preserve_layer *L, int which, const void *x, int B, const Epilog
         a.inject = L->inject == INJECT_TC_RING && which == 0 ? INJECT_TC_RING : INJECT_NONE;
         // The gate/up projection takes its input as one fp16 plane (an RMSNorm output is bounded, and 11
         // significant bits keep the SwiGLU output well inside the tolerance): half the activation
-        // traffic and half the MMA work of the largest GEMM.  The QKV projection keeps hi + lo bf16
-        // planes: rounding of q is amplified by the softmax (measured: one fp16 plane put the 70B-shaped
-        // chain's attention partial sums at 1.02 of the bound).
-        a.x_fp16 = which >= 1 ? 1 : 0;
+        // traffic and half the MMA work of the largest GEMM.  The QKV projection keeps two planes, hi + lo
+        // (fp16 each, its weights stored as fp16 like the others: with int8 weights the codes then take the
+        // cheap fp16 widening): rounding of q is amplified by the softmax (measured: one fp16 plane put the
+        // 70B-shaped chain's attention partial sums at 1.02 of the bound).
+        a.x_fp16 = which >= 1 ? 1 : 2;
         a.w8 = L->w8 ? 1 : 0;
         a.scales = L->w8 ? L->scales + L->soff[which] : nullptr;
         a.w8_codes = L->w8 ? L->arena + L->off[which] : nullptr;
@@ -583,7 +584,7 @@ int enqueue_step(preserve_layer *L, const StepPtrs &sp, const StepPlan &pl, bool
         w.h_f32 = L->h_f32;
         w.h_bf16 = nullptr;
         w.x_bf16 = L->x;
-        w.x_fp16 = 0;
+        w.x_fp16 = L->tensor_path ? 2 : 0;
         w.x_plane_elems = (size_t)L->rows * H;
         w.B = B; w.H = H;
         w.trace = TRACE(0);
@@ -1119,7 +1120,7 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
         } else {
             auto pack = L->tensor_path ? launch_pack_rows : launch_pack_gemv;
             // (tensor path: Wgate|up meets the fp16 RMSNorm output x2 and is stored as fp16)
-            CKI(pack(s_qkv, c_qkv, 3, d.k[0], EPI_QKV, L->arena + L->off[0], 0, nullptr));
+            CKI(pack(s_qkv, c_qkv, 3, d.k[0], EPI_QKV, L->arena + L->off[0], L->tensor_path ? 1 : 0, nullptr));
             CKI(pack(s_o, c_o, 1, d.k[1], EPI_PLAIN, L->arena + L->off[1], 1, nullptr));
             CKI(pack(s_gu, c_gu, 2, d.k[2], EPI_SWIGLU, L->arena + L->off[2], 1, nullptr));
             CKI(pack(s_dn, c_dn, 1, d.k[3], EPI_PLAIN, L->arena + L->off[3], 1, nullptr));
@@ -1177,7 +1178,7 @@ int preserve_layer_init(const preserve_layer_config_t *cfg, const preserve_layer
         // activations as the B operand: [2 * nb_pad, K] = hi rows then lo rows, one box covers both
         const void *xb[4] = {L->x, L->o, L->x2, L->a};
         for (int i = 0; i < 4; ++i) {
-            // x2 (the MLP's RMSNorm output) is one fp16 plane; x, o and a are two bf16 planes (hi rows, lo rows)
+            // x (two fp16 planes: hi rows, lo rows) feeds the QKV projection; o, x2 and a are one fp16 plane each
             const uint32_t brows = (uint32_t)(i >= 1 ? L->nb_pad : 2 * L->nb_pad);
             // (int8 weights are fetched by plain bulk copies: no map over them)
             const bool wok = L->w8 || make_map_2d(&L->wmap[i], L->arena + L->off[i], d.k[i], d.n[i], 64, 128);

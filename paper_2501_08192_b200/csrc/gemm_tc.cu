@@ -69,7 +69,8 @@ struct GemmTcParams {
     int *status;
     long long *trace;
     int inject;         // test hook: the producer of CTA (0, 0) never fetches its first weight tile
-    int planes;         // activation planes in the B operand: 2 = bf16 hi + lo, 1 = a single fp16 plane
+    int planes;         // activation planes in the B operand: 2 = hi + lo, 1 = a single fp16 plane
+    int f16;            // both operands are fp16 (else bf16)
     int epi_warps;      // 8 or 16
     int producers;      // 1..kTcMaxProducers threads that issue the ring's TMA loads (stage uses dealt round-robin)
     int w8;             // the weight tiles arrive as int8 codes and are widened into tensor memory (the MMA's A operand)
@@ -480,7 +481,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
             n_min = n < n_min ? n : n_min;
         }
         const int G = n_min;
-        const bool f16 = p.planes == 1;
+        const bool f16 = p.f16 != 0;
         const int row = quad * 32 + lane;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(p.mt * acc_cols);
         const uint32_t src_lane = (uint32_t)row * 128;
@@ -923,13 +924,14 @@ cudaError_t launch_gemm_tc(const GemmTcArgs &a, int sm_count, cudaStream_t s)
     p.status = a.status;
     p.trace = a.trace;
     p.inject = a.inject;
-    const int planes = a.x_fp16 ? 1 : 2;
+    const int planes = a.x_fp16 == 1 ? 1 : 2;
     p.planes = planes;
+    p.f16 = a.x_fp16 ? 1 : 0;
     // Two 128-row weight tiles per CTA share one activation tile when the activation tile (planes * NB
     // rows) weighs about as much as a weight tile: halves the L2->SM traffic of the activations, which
     // every CTA re-reads.  With a single fp16 plane of 64 rows it does not: one tile per CTA then gives
     // twice the CTAs (two per SM) and measured 1-1.5 us less on the O and down projections of config 4.
-    const int mt = a.w8 ? gemm_tc_w8_tiles(a.NB, a.N, a.x_fp16)
+    const int mt = a.w8 ? gemm_tc_w8_tiles(a.NB, a.N, a.x_fp16 == 1)
                         : ((planes * a.NB >= 96 && a.N % (2 * kTcTileM) == 0 && a.w_map256) ? 2 : 1);
     if (a.w8 && (!a.w8_codes || !a.scales))
         return cudaErrorInvalidValue;

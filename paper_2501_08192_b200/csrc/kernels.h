@@ -172,7 +172,7 @@ struct GemmTcArgs {
     const CUtensorMap *w_map256;  // optional: same tensor with box (64, 256), for two weight tiles per CTA
     CUtensorMap x_map;    // dims (K, 2*NB): hi rows then lo rows; box (64, 2*NB), 128B swizzle - or, with x_fp16,
                           // dims (K, NB): one fp16 plane, box (64, NB)
-    int x_fp16;           // the activations are one fp16 plane (inputs that come out of an RMSNorm: bounded,
+    int x_fp16;           // 0: two bf16 planes; 2: two fp16 planes (hi rows then lo rows); 1: the activations are one fp16 plane (inputs that come out of an RMSNorm: bounded,
                           // 11 significant bits suffice) instead of bf16 hi + lo planes
     int B, NB, N, K;      // NB = batch rows per plane (multiple of 16)
     EpilogueArgs epi;

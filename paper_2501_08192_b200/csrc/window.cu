@@ -43,7 +43,7 @@ struct WindowParams {
     long long *trace;
     int delay_ns;
     int *status;
-    int x_fp16;          // write x as one fp16 plane (tensor path) instead of bf16 hi + lo planes
+    int x_fp16;          // 0: x as bf16 hi + lo planes; 1: one fp16 plane; 2: fp16 hi + lo planes (x = hi + lo, 22 bits)
     int no_hint;         // LEAN: do not even hint the inputs into L2 before the wait (another kernel of the call still writes them)
     int inject;          // test hook: rank 1 of every row withholds its hand-over to rank 0
     // real communication window (COMM instantiation only)
@@ -318,7 +318,23 @@ __global__ void __launch_bounds__(512) k_window_reduce_rmsnorm(const __grid_cons
             xv[2] = v[c][2] * inv * bf_lo(g.y); xv[3] = v[c][3] * inv * bf_hi(g.y);
             xv[4] = v[c][4] * inv * bf_lo(g.z); xv[5] = v[c][5] * inv * bf_hi(g.z);
             xv[6] = v[c][6] * inv * bf_lo(g.w); xv[7] = v[c][7] * inv * bf_hi(g.w);
-            if (p.x_fp16) {
+            if (p.x_fp16 == 2) {
+                // hi = fp16(x), lo = fp16(x - hi): the operand format of the tensor path's QKV projection
+                uint4 hi, lo;
+                uint32_t *hw = &hi.x, *lw = &lo.x;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float a0 = fminf(fmaxf(xv[2 * i], -65504.f), 65504.f);
+                    const float a1 = fminf(fmaxf(xv[2 * i + 1], -65504.f), 65504.f);
+                    const __half2 h2 = __floats2half2_rn(a0, a1);
+                    const float2 hf = __half22float2(h2);
+                    const __half2 l2 = __floats2half2_rn(a0 - hf.x, a1 - hf.y);
+                    hw[i] = *reinterpret_cast<const uint32_t *>(&h2);
+                    lw[i] = *reinterpret_cast<const uint32_t *>(&l2);
+                }
+                p.x_bf16[row_off + ch] = hi;
+                p.x_bf16[p.x_plane + row_off + ch] = lo;
+            } else if (p.x_fp16) {
                 // normalised activations are bounded (|x| <= sqrt(H) * |gain|): one fp16 plane carries 11
                 // significant bits; clamped to the fp16 range so that an absurd gain cannot make an infinity
                 uint4 o;

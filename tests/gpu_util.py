@@ -133,7 +133,9 @@ class DeviceLayer:
                 torch.cuda.synchronize()
                 out[name] = buf[:B].float().cpu().numpy()
                 continue
-            buf = torch.empty((2, rows) + tail, dtype=torch.bfloat16, device="cuda")
+            # (tensor path: x is hi + lo fp16 planes; everything else hi + lo bf16 planes)
+            dt = torch.float16 if (fp16_x and name == "x") else torch.bfloat16
+            buf = torch.empty((2, rows) + tail, dtype=dt, device="cuda")
             self.layer.debug_copy(which, buf)
             torch.cuda.synchronize()
             out[name] = (buf[0, :B].double() + buf[1, :B].double()).float().cpu().numpy()
