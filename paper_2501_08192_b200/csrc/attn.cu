@@ -662,6 +662,12 @@ cudaError_t launch_attention(const AttnArgs &a, cudaStream_t s)
     // one warp per item partial of the longest sequence (at least the four that write the head dims)
     int warps = a.max_items_per_stream < 4 ? 4 : (a.max_items_per_stream > kMergeMaxWarps ? kMergeMaxWarps
                                                                                           : a.max_items_per_stream);
+    // Many merge CTAs (batch x heads >= 512: seven per SM) with eight warps each fill an SM's thread slots,
+    // and the output projection's CTAs - launched early, to stage their weights during the merge - find no
+    // room: four warps then (a warp takes two partials in turn; config 4: merge +0.9 us, O projection -1.1 us
+    // with its hand-over, layer -0.5 us).
+    if (a.B * a.nq >= 512 && warps > 4)
+        warps = 4;
     cudaLaunchConfig_t cfg2 = {};
     cfg2.gridDim = dim3(a.B * a.nq);
     cfg2.blockDim = dim3(warps * 32);
