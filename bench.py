@@ -854,6 +854,8 @@ def run_timeline(P, I, torch, args, stream):
             "start_to_wait_return_us": round(float(np.mean(w1 - s0)) / 1e3, 2),
             "early_start_before_prev_end_us": round(float(np.mean(prev_end - s0)) / 1e3, 2) if k > 0 else None,
             "wait_return_after_prev_end_us": round(float(np.mean(w1 - prev_end)) / 1e3, 2) if k > 0 else None,
+            "last_cta_start_after_prev_end_us": round(float(np.mean(s1 - prev_end)) / 1e3, 2) if k > 0 else None,
+            "first_wait_return_after_prev_end_us": round(float(np.mean(w0 - prev_end)) / 1e3, 2) if k > 0 else None,
             "wait_return_to_stream_end_us": round(float(np.mean(np.where(st > 0, st - w1, 0.0))) / 1e3, 2),
             "stream_end_to_end_us": round(float(np.mean(np.where(st > 0, e1 - st, e1 - w1))) / 1e3, 2),
             "wait_return_to_end_us": round(float(np.mean(e1 - w1)) / 1e3, 2),

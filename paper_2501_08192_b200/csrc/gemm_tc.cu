@@ -224,7 +224,6 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
     const int n_issuers = (W8 && p.mt == 2 && p.epi_warps == 16 && p.producers == 3) ? 2 : 1;
     trace_start(p.trace);
     pdl_launch_dependents();
-    load_epilogue_tables(p.epi, tabs, 0, p.B);   // inputs of the step: safe before the wait
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.stages; ++i) {
             mbar_init(&full[i], 1);
@@ -242,28 +241,49 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
                 mbar_init(&slot_free[j], n_issuers);
             }
         }
+        if (PUSH && p.splits > 1) {
+            // this rank will receive NB / splits columns of every other rank's partial tile
+            mbar_init(&push_bar, 1);
+        }
         mbar_fence_init();
         poisoned = 0;
-        if (!W8)
-            tma_prefetch_desc(&p.w_map);
+        if (PUSH && p.splits > 1)
+            mbar_expect_tx(&push_bar, (uint32_t)(p.splits - 1) * p.mt * kTcTileM * (p.NB / p.splits) * 4u);
+        // The ring's first fill, weights only, right here: they never depend on earlier kernels, and a CTA
+        // that becomes resident late - after the kernel in front has ended - should have its first bytes
+        // under way before anything else of the prologue (tensor-memory allocation, tables, barriers
+        // across the CTA and the cluster: 1.5-2 us measured from a CTA's start to its dependency wait).
+        {
+            const uint64_t pol = policy_evict_first();   // every weight byte is read once per step
+            const int n_kb = kb1 - kb0;
+            const int pre = n_kb < p.stages ? n_kb : p.stages;
+            for (int i = 0; i < pre; ++i) {
+                mbar_expect_tx(&full[i], kEarly ? a_bytes : stage_bytes);
+                if (p.inject == INJECT_TC_RING && i == 0 && tile == 0 && s == 0)
+                    continue;
+                if constexpr (W8)
+                    bulk_load_hint(smem + (size_t)i * stage_bytes, p.w8_codes + ((size_t)tile * p.kblocks + kb0 + i) * a_bytes,
+                                   a_bytes, &full[i], pol);
+                else
+                    tma_load_2d_hint(smem + (size_t)i * stage_bytes, &p.w_map, (kb0 + i) * kTcBlockK,
+                                     tile * p.mt * kTcTileM, &full[i], pol);
+            }
+        }
         tma_prefetch_desc(&p.x_map);
     }
+    load_epilogue_tables(p.epi, tabs, 0, p.B);   // inputs of the step: safe before the wait
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)),
                      "r"((uint32_t)p.tmem_cols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    if (PUSH && p.splits > 1 && threadIdx.x == 0) {
-        // this rank will receive NB / splits columns of every other rank's partial tile
-        mbar_init(&push_bar, 1);
-        mbar_fence_init();
-        mbar_expect_tx(&push_bar, (uint32_t)(p.splits - 1) * p.mt * kTcTileM * (p.NB / p.splits) * 4u);
-    }
     tc_fence_before();
     __syncthreads();
+    // Every rank's barrier must exist before anybody sends to it: arrive here, wait just before the first
+    // send (the tail), so that the cluster barrier's latency is not part of the prologue.
     if (PUSH && p.splits > 1)
-        cg::this_cluster().sync();      // every rank's barrier exists before anybody sends; overlaps the weight fetch
+        cluster_arrive_relaxed();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
 
@@ -278,17 +298,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         const int NP = p.producers;
         const int n_kb = kb1 - kb0;
         const int pre = n_kb < p.stages ? n_kb : p.stages;
-        for (int i = prod; i < pre; i += NP) {
-            mbar_expect_tx(&full[i], kEarly ? a_bytes : stage_bytes);
-            if (p.inject == INJECT_TC_RING && i == 0 && tile == 0 && s == 0)
-                continue;
-            if constexpr (W8)
-                bulk_load_hint(smem + (size_t)i * stage_bytes, p.w8_codes + ((size_t)tile * p.kblocks + kb0 + i) * a_bytes,
-                               a_bytes, &full[i], pol);
-            else
-                tma_load_2d_hint(smem + (size_t)i * stage_bytes, &p.w_map, (kb0 + i) * kTcBlockK,
-                                 tile * p.mt * kTcTileM, &full[i], pol);
-        }
+        // (the ring's first fill of weight tiles was issued by thread 0 at the top of the kernel)
         pdl_wait();
         if (prod == 0)
             trace_waited(p.trace);
@@ -583,6 +593,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         cg::cluster_group cluster = cg::this_cluster();
         const int cols = p.NB / p.splits;
         float *recv = reinterpret_cast<float *>(smem + p.recv_off);
+        cluster_wait();       // (the arrival at the top of the kernel: every rank's receive barrier exists)
         if (is_epi) {
             // two chunks (four TMEM loads) in flight per wait
             const uint32_t red_row = smem_u32(red) + (uint32_t)row * 4u;
@@ -699,6 +710,7 @@ __global__ void __launch_bounds__(kTcMaxThreads, 1) k_gemm_tcgen05(const __grid_
         const int cols = p.NB / p.splits;
         const uint32_t recv_a = smem_u32(smem + p.recv_off);
         const uint32_t src_stride = (uint32_t)p.mt * kTcTileM * cols * 4u;          // bytes per source rank
+        cluster_wait();       // (the arrival at the top of the kernel: every rank's receive barrier exists)
         if (is_epi) {
             for (int j = sub; j < p.mt * nchunks; j += kSubs) {
                 const int m = j / nchunks, c = j % nchunks;
