@@ -165,13 +165,15 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
     const int part_floats = rbs_per_cta * 16 * NB;   // one rank's partial sums of a group
     if (p.push) {
         // rank 0 will receive the other ranks' partial sums: its barrier must exist (and expect them)
-        // before anybody sends - a cluster barrier here, where it overlaps the weight fetch
+        // before anybody sends - a cluster barrier, split: arrive here, wait just before the sends, so
+        // that a CTA which starts late does not spend the barrier's latency ahead of its dependency wait
         if (s == 0 && threadIdx.x == 0) {
             mbar_init(&push_bar, 1);
             mbar_fence_init();
             mbar_expect_tx(&push_bar, (uint32_t)(p.splits - 1) * part_floats * 4u);
         }
-        cg::this_cluster().sync();
+        __syncwarp();
+        cluster_arrive_relaxed();
     }
     load_epilogue_tables(p.epi, tabs, p.b0, p.B);    // inputs of the step: safe before the wait
     const int xrow = p.K >> 3;                       // uint4 per activation row
@@ -369,6 +371,7 @@ __global__ void __launch_bounds__(kGemvWarps * 32, 2) k_gemv_splitk(const __grid
             // barrier with the bytes, and are done; rank 0 waits for all the bytes and finishes every
             // output.  No cluster barrier on the critical path.  (One group per CTA in this mode.)
             __syncthreads();
+            cluster_wait();       // (the arrival in the prologue: rank 0's barrier exists)
             float *recv = reinterpret_cast<float *>(wsm + p.recv_off);
             if (s != 0) {
                 const uint32_t dst = cluster_map(recv + (size_t)(s - 1) * part_floats, 0);
